@@ -1,0 +1,142 @@
+/* sod2.h — C ABI of the B200-native SoD^2 hot path.
+ *
+ * The library executes the fused operator groups that Rank-and-Dimension Propagation (RDP) makes
+ * possible on dynamic DNNs.  The calls follow the staging the paper describes: static analysis before
+ * deployment (Section 4.1-4.3: operator classification, RDP = Algorithm 1, fusion, partition at
+ * execution-determined operators), then, per input, evaluation of the shape expressions and the
+ * memory allocation plan "at execution time when all tensor sizes are known" (Section 4.4.1), then
+ * inference.
+ *
+ * Conventions
+ *  - Every call returns a sod2_status, never throws, never aborts, never prints.  Out-parameters
+ *    are untouched on error.  sod2_last_error(handle) gives a message for the last failure.
+ *  - Handles are owned by the library and freed by the matching *_destroy.
+ *  - ALL DEVICE MEMORY IS OWNED BY THE CALLER: inputs, outputs, constants, the prepack workspace and
+ *    the arena.  The library never allocates or frees device memory.
+ *  - Batches: a graph is written for ONE request; sod2_bind_dims binds n_requests at once.  Every
+ *    input / output / arena tensor holds the requests' instances back to back in request order
+ *    (instance sizes rounded up to 16 bytes), e.g. x:[1,L,768] for 8 requests is one packed
+ *    [sum L, 768] buffer.  No padding to a maximum length exists anywhere.
+ *  - Pointers named dev_* / inputs / outputs / arena / workspace are DEVICE pointers; all others are
+ *    host pointers.  cuda_stream is a cudaStream_t passed as void*.
+ *  - One thread per handle.  Same inputs => bit-identical outputs (Section 4: deterministic).
+ */
+#ifndef SOD2_H_
+#define SOD2_H_
+#include <stddef.h>
+#include <stdint.h>
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sod2_graph sod2_graph;
+typedef struct sod2_binding sod2_binding;
+typedef struct sod2_plan_s sod2_plan_t;
+
+typedef enum {
+  SOD2_OK = 0, SOD2_E_INVALID_ARG, SOD2_E_PARSE, SOD2_E_UNSUPPORTED_OP, SOD2_E_RANK_MISMATCH,
+  SOD2_E_NOT_CONVERGED, SOD2_E_UNBOUND_SYMBOL, SOD2_E_BAD_DIM, SOD2_E_SHAPE_CONFLICT,
+  SOD2_E_ARENA_TOO_SMALL, SOD2_E_MISALIGNED, SOD2_E_CUDA, SOD2_E_TIMEOUT, SOD2_E_INTERNAL
+} sod2_status;
+
+/* option bits for sod2_graph_create */
+#define SOD2_OPT_NO_FUSION 1u /* every operator is its own group */
+#define SOD2_OPT_NO_REUSE  2u /* every arena tensor keeps its own slot: intermediates stay readable */
+
+/* Parse the graph text (host, ir_len bytes), classify every operator (Table 2), run RDP
+ * (Algorithm 1) to a fixpoint, form fused groups (Section 4.2) and partition at
+ * execution-determined operators (Section 4.3).  Pure host work, no CUDA call. */
+sod2_status sod2_graph_create(const char* ir_text, size_t ir_len, uint32_t opt_flags, sod2_graph** out);
+void sod2_graph_destroy(sod2_graph* g);
+
+/* Attach caller-owned device memory holding a float constant (weights) in the layout the graph
+ * declares (row-major, graph dtype).  The memory must outlive every run. */
+sod2_status sod2_graph_set_const(sod2_graph* g, const char* name, const void* dev_ptr, size_t bytes);
+
+/* GEMM weights are re-laid K-major for the tensor-core kernel.  Query the workspace size, then
+ * prepack once into caller-owned device memory (256-byte aligned); the copies are enqueued on
+ * cuda_stream and must complete before the first run. */
+sod2_status sod2_graph_prepack_bytes(const sod2_graph* g, size_t* bytes);
+sod2_status sod2_graph_prepack(sod2_graph* g, void* dev_workspace, size_t bytes, void* cuda_stream);
+
+/* H0: bind symbol values for n_requests requests.  values is [n_requests][n_syms] row-major (host).
+ * Evaluates every shape expression of every tensor for every request and checks the bind-time
+ * assertions RDP recorded.  Errors: unknown / unbound symbol, value outside the declared range,
+ * shape conflict. */
+sod2_status sod2_bind_dims(sod2_graph* g, int n_requests, int n_syms, const char* const* sym_names,
+                           const int64_t* values, sod2_binding** out);
+void sod2_binding_destroy(sod2_binding* b);
+
+/* H1+H2: arena memory plan (Section 4.4.1, peak-first greedy over one linear arena), kernel-variant
+ * choice by shape class (Section 4.4.2) and launch parameters.  arena_bytes = size the caller must
+ * provide to sod2_run.  The binding must outlive the plan. */
+sod2_status sod2_plan(sod2_graph* g, const sod2_binding* b, sod2_plan_t** out, size_t* arena_bytes);
+void sod2_plan_destroy(sod2_plan_t* p);
+
+typedef struct {
+  int64_t host_enqueue_ns; /* host time spent inside sod2_run */
+  int64_t gpu_launches;    /* kernels enqueued */
+  int64_t reserved[6];
+} sod2_run_info;
+
+/* Enqueue one inference (all requests of the binding) on cuda_stream.  inputs[i] / outputs[j] are
+ * device pointers in graph declaration order, packed per request as described above; outputs whose
+ * shape is execution-determined must be sized for the static upper bound (sod2_binding_shape reports
+ * it) and their true shape is read with sod2_run_output_shape after the stream has been synchronised.
+ * arena: >= arena_bytes, 256-byte aligned (SOD2_E_ARENA_TOO_SMALL / SOD2_E_MISALIGNED).  Asynchronous.
+ * Device-side failures (a bounded wait that ran out) are reported by sod2_plan_device_status. */
+sod2_status sod2_run(sod2_plan_t* p, const void* const* inputs, void* const* outputs, void* arena,
+                     size_t arena_bytes, void* cuda_stream, sod2_run_info* info);
+
+/* Reads the device status word written by the last run (synchronises the stream).
+ * SOD2_OK, or SOD2_E_TIMEOUT if a kernel gave up on a bounded wait. */
+sod2_status sod2_plan_device_status(sod2_plan_t* p, const void* arena, void* cuda_stream);
+
+/* ---- introspection (used by the tests that check the RDP shape expressions) ---- */
+/* rank: -1 undef, -2 nac.  dim_kind[i]: 0 undef, 1 known constant, 2 symbolic constant,
+ * 3 operation-inferred expression, 4 nac (execution determined).  expr_buf receives the shape as
+ * "[e0,e1,...]" in canonical form.  dim_kind may be NULL; it must hold `rank` ints otherwise. */
+sod2_status sod2_graph_tensor_info(const sod2_graph* g, const char* tensor, int* rank, int* dim_kind,
+                                   char* expr_buf, size_t expr_buf_len);
+/* Element type of a tensor: 0 f32, 1 bf16, 2 i64, 3 bool (1 byte). */
+sod2_status sod2_graph_tensor_dtype(const sod2_graph* g, const char* tensor, int* dtype);
+/* Value-map entry of a small integer tensor as "[e0,...]", "undef" or "nac". */
+sod2_status sod2_graph_tensor_value(const sod2_graph* g, const char* tensor, char* buf, size_t buf_len);
+int sod2_graph_num_ops(const sod2_graph* g);
+/* dyn_class / eff_class: 0 ISDO, 1 ISDOS, 2 ISVDOS, 3 EDO (Table 2; eff_class after constant
+ * propagation).  group_id: -1 for operators evaluated by RDP itself or pure views. */
+sod2_status sod2_graph_op_info(const sod2_graph* g, int op, char* op_type, size_t op_type_len, int* dyn_class,
+                               int* eff_class, int* group_id, int* subgraph_id);
+int sod2_graph_num_groups(const sod2_graph* g);
+/* kind_buf: group kernel kind name; versions: fused code versions needed (1 when RDP resolved every
+ * broadcast); n_ops: operators fused into the group. */
+sod2_status sod2_graph_group_info(const sod2_graph* g, int group, char* kind_buf, size_t kind_len, int* n_ops,
+                                  int* versions, int* subgraph_id);
+int sod2_graph_num_subgraphs(const sod2_graph* g);
+int sod2_graph_rdp_sweeps(const sod2_graph* g);
+/* Classification of an operator name alone (Table 2). Returns SOD2_E_UNSUPPORTED_OP if unknown. */
+sod2_status sod2_classify(const char* op_type, int* dyn_class);
+/* Re-run RDP visiting the operators in the given order (a permutation of 0..num_ops-1); used to
+ * check that the fixpoint does not depend on the order. Must be called before any bind. */
+sod2_status sod2_graph_reanalyse(sod2_graph* g, const int* order, int n);
+
+sod2_status sod2_binding_shape(const sod2_binding* b, int request, const char* tensor, int64_t* dims, int* rank);
+/* Arena slot of an inter-group tensor: byte offset, byte size (all requests), defining and last-using step. */
+sod2_status sod2_plan_slot(const sod2_plan_t* p, const char* tensor, size_t* offset, size_t* bytes, int* def_step,
+                           int* last_use_step);
+/* Byte offset of one request's instance inside a packed tensor buffer. */
+sod2_status sod2_plan_instance_offset(const sod2_plan_t* p, const char* tensor, int request, size_t* offset);
+/* arena_bytes, peak live bytes, sum of all inter-group tensor bytes (what no-reuse allocation takes). */
+sod2_status sod2_plan_memory(const sod2_plan_t* p, size_t* arena_bytes, size_t* peak_live_bytes, size_t* sum_bytes);
+/* True shape of an output after a run (execution-determined extents are read back from the device;
+ * synchronises cuda_stream). */
+sod2_status sod2_run_output_shape(sod2_plan_t* p, const void* arena, void* cuda_stream, int request, int output,
+                                  int64_t* dims, int* rank);
+
+/* handle may be a graph, binding or plan; returns "" if there was no error. */
+const char* sod2_last_error(const void* any_handle);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SOD2_H_ */

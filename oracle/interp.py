@@ -226,11 +226,14 @@ def _is_int(a):
 
 # --------------------------------------------------------------------------- interpreter
 def run(text: str, consts: Dict[str, np.ndarray], inputs: Dict[str, np.ndarray],
-        overrides: Optional[Dict[str, np.ndarray]] = None, g: Optional[Graph] = None) -> Dict[str, np.ndarray]:
+        overrides: Optional[Dict[str, np.ndarray]] = None, g: Optional[Graph] = None,
+        computed: Optional[Dict[str, np.ndarray]] = None) -> Dict[str, np.ndarray]:
     """Execute the graph on one request.  Returns every tensor by name.
 
     overrides: tensors whose value is replaced right after they are produced (used to keep
-    the oracle in lock-step with another implementation's data-dependent decisions)."""
+    the oracle in lock-step with another implementation's data-dependent decisions).
+    computed: if given, receives for every overridden tensor the value the oracle itself computed
+    from its (possibly overridden) inputs, i.e. the per-operator lock-step reference."""
     g = g or parse(text)
     env: Dict[str, np.ndarray] = {}
     for name in g.inputs:
@@ -298,7 +301,12 @@ def run(text: str, consts: Dict[str, np.ndarray], inputs: Dict[str, np.ndarray],
             raise NotImplementedError(op)
         outs = out if isinstance(out, tuple) else (out,)
         for name, val in zip(nd.outs, outs):
-            env[name] = np.asarray(overrides[name]).reshape(np.shape(val)) if name in overrides else val
+            if name in overrides:
+                if computed is not None:
+                    computed[name] = val
+                env[name] = np.asarray(overrides[name]).reshape(np.shape(val))
+            else:
+                env[name] = val
     return env
 
 

@@ -1,0 +1,258 @@
+"""ctypes binding of libsod2.so: argument marshalling only, same names as include/sod2.h.
+
+PyTorch is used by callers for device memory and streams; this module never computes.
+The library is built in-tree (paper_2403_00176_b200/build.py); importing fails loudly if it is
+missing, and there is no CPU fallback of any kind.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Sequence, Tuple
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsod2.so")
+
+STATUS = ["SOD2_OK", "SOD2_E_INVALID_ARG", "SOD2_E_PARSE", "SOD2_E_UNSUPPORTED_OP", "SOD2_E_RANK_MISMATCH",
+          "SOD2_E_NOT_CONVERGED", "SOD2_E_UNBOUND_SYMBOL", "SOD2_E_BAD_DIM", "SOD2_E_SHAPE_CONFLICT",
+          "SOD2_E_ARENA_TOO_SMALL", "SOD2_E_MISALIGNED", "SOD2_E_CUDA", "SOD2_E_TIMEOUT", "SOD2_E_INTERNAL"]
+OPT_NO_FUSION = 1
+OPT_NO_REUSE = 2
+DYN_CLASS = ["ISDO", "ISDOS", "ISVDOS", "EDO"]
+
+
+class Sod2Error(RuntimeError):
+    def __init__(self, status: int, msg: str):
+        super().__init__(f"{STATUS[status] if 0 <= status < len(STATUS) else status}: {msg}")
+        self.status = status
+        self.status_name = STATUS[status] if 0 <= status < len(STATUS) else str(status)
+
+
+class RunInfo(C.Structure):
+    _fields_ = [("host_enqueue_ns", C.c_int64), ("gpu_launches", C.c_int64), ("reserved", C.c_int64 * 6)]
+
+
+def _load() -> C.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2403_00176_b200.build` (needs nvcc). "
+                          "There is no fallback path.")
+    lib = C.CDLL(LIB_PATH)
+    vp, cp, sz, i32, i64 = C.c_void_p, C.c_char_p, C.c_size_t, C.c_int, C.c_int64
+    P = C.POINTER
+    sig = {
+        "sod2_graph_create": [cp, sz, C.c_uint32, P(vp)],
+        "sod2_graph_set_const": [vp, cp, vp, sz],
+        "sod2_graph_prepack_bytes": [vp, P(sz)],
+        "sod2_graph_prepack": [vp, vp, sz, vp],
+        "sod2_bind_dims": [vp, i32, i32, P(cp), P(i64), P(vp)],
+        "sod2_plan": [vp, vp, P(vp), P(sz)],
+        "sod2_run": [vp, P(vp), P(vp), vp, sz, vp, P(RunInfo)],
+        "sod2_plan_device_status": [vp, vp, vp],
+        "sod2_graph_tensor_info": [vp, cp, P(i32), P(i32), cp, sz],
+        "sod2_graph_tensor_value": [vp, cp, cp, sz],
+        "sod2_graph_tensor_dtype": [vp, cp, P(i32)],
+        "sod2_graph_op_info": [vp, i32, cp, sz, P(i32), P(i32), P(i32), P(i32)],
+        "sod2_graph_group_info": [vp, i32, cp, sz, P(i32), P(i32), P(i32)],
+        "sod2_classify": [cp, P(i32)],
+        "sod2_graph_reanalyse": [vp, P(i32), i32],
+        "sod2_binding_shape": [vp, i32, cp, P(i64), P(i32)],
+        "sod2_plan_slot": [vp, cp, P(sz), P(sz), P(i32), P(i32)],
+        "sod2_plan_instance_offset": [vp, cp, i32, P(sz)],
+        "sod2_plan_memory": [vp, P(sz), P(sz), P(sz)],
+        "sod2_run_output_shape": [vp, vp, vp, i32, i32, P(i64), P(i32)],
+    }
+    for name, args in sig.items():
+        fn = getattr(lib, name)
+        fn.argtypes = args
+        fn.restype = i32
+    for name in ("sod2_graph_num_ops", "sod2_graph_num_groups", "sod2_graph_num_subgraphs", "sod2_graph_rdp_sweeps"):
+        getattr(lib, name).argtypes = [vp]
+        getattr(lib, name).restype = i32
+    for name in ("sod2_graph_destroy", "sod2_binding_destroy", "sod2_plan_destroy"):
+        getattr(lib, name).argtypes = [vp]
+        getattr(lib, name).restype = None
+    lib.sod2_last_error.argtypes = [vp]
+    lib.sod2_last_error.restype = cp
+    return lib
+
+
+lib = _load()
+EXPORTS = ["sod2_graph_create", "sod2_graph_destroy", "sod2_graph_set_const", "sod2_graph_prepack_bytes",
+           "sod2_graph_prepack", "sod2_bind_dims", "sod2_binding_destroy", "sod2_plan", "sod2_plan_destroy",
+           "sod2_run", "sod2_plan_device_status", "sod2_graph_tensor_info", "sod2_graph_tensor_value", "sod2_graph_tensor_dtype",
+           "sod2_graph_num_ops", "sod2_graph_op_info", "sod2_graph_num_groups", "sod2_graph_group_info",
+           "sod2_graph_num_subgraphs", "sod2_graph_rdp_sweeps", "sod2_classify", "sod2_graph_reanalyse",
+           "sod2_binding_shape", "sod2_plan_slot", "sod2_plan_instance_offset", "sod2_plan_memory",
+           "sod2_run_output_shape", "sod2_last_error"]
+
+
+def _check(status: int, handle=None):
+    if status != 0:
+        msg = lib.sod2_last_error(handle).decode() if handle is not None else lib.sod2_last_error(None).decode()
+        raise Sod2Error(status, msg)
+
+
+def sod2_classify(op: str) -> str:
+    c = C.c_int()
+    _check(lib.sod2_classify(op.encode(), C.byref(c)))
+    return DYN_CLASS[c.value]
+
+
+class Graph:
+    """sod2_graph handle."""
+
+    def __init__(self, ir_text: str, opt_flags: int = 0):
+        raw = ir_text.encode()
+        h = C.c_void_p()
+        _check(lib.sod2_graph_create(raw, len(raw), opt_flags, C.byref(h)))
+        self.h = h
+        self._keep = []
+
+    def __del__(self):
+        if getattr(self, "h", None):
+            lib.sod2_graph_destroy(self.h)
+            self.h = None
+
+    def set_const(self, name: str, dev_ptr: int, nbytes: int, keep=None):
+        _check(lib.sod2_graph_set_const(self.h, name.encode(), C.c_void_p(dev_ptr), nbytes), self.h)
+        if keep is not None:
+            self._keep.append(keep)
+
+    def prepack_bytes(self) -> int:
+        n = C.c_size_t()
+        _check(lib.sod2_graph_prepack_bytes(self.h, C.byref(n)), self.h)
+        return n.value
+
+    def prepack(self, dev_ws: int, nbytes: int, stream: int, keep=None):
+        _check(lib.sod2_graph_prepack(self.h, C.c_void_p(dev_ws), nbytes, C.c_void_p(stream)), self.h)
+        if keep is not None:
+            self._keep.append(keep)
+
+    def bind_dims(self, sym_names: Sequence[str], values: Sequence[Sequence[int]]) -> "Binding":
+        return Binding(self, sym_names, values)
+
+    def tensor_info(self, name: str) -> Tuple[int, List[int], str]:
+        rank = C.c_int()
+        kinds = (C.c_int * 16)()
+        buf = C.create_string_buffer(1024)
+        _check(lib.sod2_graph_tensor_info(self.h, name.encode(), C.byref(rank), kinds, buf, 1024), self.h)
+        return rank.value, list(kinds[: max(rank.value, 0)]), buf.value.decode()
+
+    def tensor_dtype(self, name: str) -> str:
+        d = C.c_int()
+        _check(lib.sod2_graph_tensor_dtype(self.h, name.encode(), C.byref(d)), self.h)
+        return ["f32", "bf16", "i64", "bool"][d.value]
+
+    def tensor_value(self, name: str) -> str:
+        buf = C.create_string_buffer(1024)
+        _check(lib.sod2_graph_tensor_value(self.h, name.encode(), buf, 1024), self.h)
+        return buf.value.decode()
+
+    def num_ops(self) -> int:
+        return lib.sod2_graph_num_ops(self.h)
+
+    def op_info(self, i: int) -> dict:
+        t = C.create_string_buffer(64)
+        a, b, g, s = C.c_int(), C.c_int(), C.c_int(), C.c_int()
+        _check(lib.sod2_graph_op_info(self.h, i, t, 64, C.byref(a), C.byref(b), C.byref(g), C.byref(s)), self.h)
+        return {"op": t.value.decode(), "cls": DYN_CLASS[a.value], "eff_cls": DYN_CLASS[b.value], "group": g.value,
+                "subgraph": s.value}
+
+    def num_groups(self) -> int:
+        return lib.sod2_graph_num_groups(self.h)
+
+    def group_info(self, i: int) -> dict:
+        t = C.create_string_buffer(64)
+        n, v, s = C.c_int(), C.c_int(), C.c_int()
+        _check(lib.sod2_graph_group_info(self.h, i, t, 64, C.byref(n), C.byref(v), C.byref(s)), self.h)
+        return {"kind": t.value.decode(), "n_ops": n.value, "versions": v.value, "subgraph": s.value}
+
+    def num_subgraphs(self) -> int:
+        return lib.sod2_graph_num_subgraphs(self.h)
+
+    def rdp_sweeps(self) -> int:
+        return lib.sod2_graph_rdp_sweeps(self.h)
+
+    def reanalyse(self, order: Sequence[int]):
+        arr = (C.c_int * len(order))(*order)
+        _check(lib.sod2_graph_reanalyse(self.h, arr, len(order)), self.h)
+
+
+class Binding:
+    """sod2_binding handle (per-request symbol values)."""
+
+    def __init__(self, graph: Graph, sym_names: Sequence[str], values: Sequence[Sequence[int]]):
+        self.graph = graph
+        n_req, n_sym = len(values), len(sym_names)
+        names = (C.c_char_p * max(n_sym, 1))(*[s.encode() for s in sym_names])
+        flat = [int(v) for row in values for v in row]
+        vals = (C.c_int64 * max(len(flat), 1))(*flat)
+        h = C.c_void_p()
+        _check(lib.sod2_bind_dims(graph.h, n_req, n_sym, names, vals, C.byref(h)), graph.h)
+        self.h = h
+        self.n_req = n_req
+
+    def __del__(self):
+        if getattr(self, "h", None):
+            lib.sod2_binding_destroy(self.h)
+            self.h = None
+
+    def shape(self, request: int, tensor: str) -> List[int]:
+        dims = (C.c_int64 * 16)()
+        rank = C.c_int()
+        _check(lib.sod2_binding_shape(self.h, request, tensor.encode(), dims, C.byref(rank)), self.graph.h)
+        return list(dims[: rank.value])
+
+    def plan(self) -> "Plan":
+        return Plan(self)
+
+
+class Plan:
+    """sod2_plan_t handle (arena plan + launch plan)."""
+
+    def __init__(self, binding: Binding):
+        self.binding = binding
+        self.graph = binding.graph
+        h = C.c_void_p()
+        ab = C.c_size_t()
+        _check(lib.sod2_plan(self.graph.h, binding.h, C.byref(h), C.byref(ab)), self.graph.h)
+        self.h = h
+        self.arena_bytes = ab.value
+
+    def __del__(self):
+        if getattr(self, "h", None):
+            lib.sod2_plan_destroy(self.h)
+            self.h = None
+
+    def run(self, inputs: Sequence[int], outputs: Sequence[int], arena: int, arena_bytes: int, stream: int) -> RunInfo:
+        ins = (C.c_void_p * max(len(inputs), 1))(*inputs)
+        outs = (C.c_void_p * max(len(outputs), 1))(*outputs)
+        info = RunInfo()
+        _check(lib.sod2_run(self.h, ins, outs, C.c_void_p(arena), arena_bytes, C.c_void_p(stream), C.byref(info)), self.h)
+        return info
+
+    def device_status(self, arena: int, stream: int):
+        _check(lib.sod2_plan_device_status(self.h, C.c_void_p(arena), C.c_void_p(stream)), self.h)
+
+    def slot(self, tensor: str) -> dict:
+        off, nb = C.c_size_t(), C.c_size_t()
+        d, l = C.c_int(), C.c_int()
+        _check(lib.sod2_plan_slot(self.h, tensor.encode(), C.byref(off), C.byref(nb), C.byref(d), C.byref(l)), self.h)
+        return {"offset": off.value, "bytes": nb.value, "def_step": d.value, "last_use_step": l.value}
+
+    def instance_offset(self, tensor: str, request: int) -> int:
+        off = C.c_size_t()
+        _check(lib.sod2_plan_instance_offset(self.h, tensor.encode(), request, C.byref(off)), self.h)
+        return off.value
+
+    def memory(self) -> dict:
+        a, p, s = C.c_size_t(), C.c_size_t(), C.c_size_t()
+        _check(lib.sod2_plan_memory(self.h, C.byref(a), C.byref(p), C.byref(s)), self.h)
+        return {"arena_bytes": a.value, "peak_live_bytes": p.value, "sum_bytes": s.value}
+
+    def output_shape(self, arena: int, stream: int, request: int, output: int) -> List[int]:
+        dims = (C.c_int64 * 16)()
+        rank = C.c_int()
+        _check(lib.sod2_run_output_shape(self.h, C.c_void_p(arena), C.c_void_p(stream), request, output, dims,
+                                         C.byref(rank)), self.h)
+        return list(dims[: rank.value])

@@ -1,0 +1,136 @@
+// Fused groups, per-request binding, arena memory plan and launch plan.
+#pragma once
+#include <memory>
+#include <string>
+#include <vector>
+
+#include "graph.h"
+
+namespace sod2 {
+
+enum OptFlags : uint32_t {
+  OPT_NO_FUSION = 1u,   // every operator is its own group (fused-vs-unfused comparison)
+  OPT_NO_REUSE = 2u,    // every arena tensor gets its own slot (keeps all intermediates readable after a run)
+};
+
+enum class GKind {
+  GEMM,        // MatMul(x, const W) [+bias] [act] [+residual]          (tcgen05, bf16) or the fp32 SIMT kernel [+LayerNorm]
+  ATTENTION,   // MatMul(q,k^T) [*scale] Softmax MatMul(p,v)
+  LAYERNORM,   // LayerNormalization alone on packed rows
+  CHAIN,       // broadcast-elementwise chain [+ trailing Softmax / LayerNormalization]
+  TOPK_KEEP,   // ReduceSumSquare -> TopK(order=index) -> Gather rows
+  NONZERO,
+  CONV,        // Conv [+bias] [act] [+residual] [act]
+  GAP,         // GlobalAveragePool
+  GATE,        // GlobalAveragePool -> Reshape -> MatMul(C x 1) -> Add -> Greater
+  SWITCH,
+  COMBINE,
+  UNSUPPORTED
+};
+const char* gkind_name(GKind k);
+
+struct Group {
+  GKind kind = GKind::UNSUPPORTED;
+  std::vector<int> nodes;
+  std::vector<int> ext_in, ext_out;   // tensors crossing the group boundary
+  int versions = 1;                   // fused code versions needed (2^unresolved broadcast dims, Section 4.2)
+  int subgraph = 0;
+  // roles (tensor ids, -1 = absent)
+  int a = -1, w = -1, bias = -1, res = -1, out = -1, gamma = -1, beta = -1;
+  int q = -1, k = -1, v = -1, out2 = -1, gate = -1;
+  int act = 0;                        // 0 none, 1 gelu, 2 relu
+  int act2 = 0;                       // activation after the residual add
+  int has_ln = 0;
+  int red = 0;                        // chain: 0 none, 1 softmax, 2 layernorm
+  float eps = 1e-5f, scale = 1.0f;
+  int stride = 1, pad = 0, ksize = 1;
+  std::vector<int> chain_ops;         // ChainOp codes
+  std::vector<int> chain_operands;    // tensor id or -1 per op
+  std::string why;                    // for UNSUPPORTED
+};
+
+// How a tensor's storage relates to others (decided once, at graph creation).
+struct Storage {
+  enum Kind { ROOT, VIEW_OF_INPUT, VIEW_OF_OUTPUT, FOLDED } kind = ROOT;
+  int node = -1;    // the view operator
+  int other = -1;   // VIEW_OF_INPUT: the operator's input; VIEW_OF_OUTPUT: the operator's output
+};
+
+struct Compiled {
+  Graph g;
+  uint32_t flags = 0;
+  std::vector<Group> groups;          // in execution order
+  std::vector<Storage> storage;       // per tensor
+  std::vector<int> node_folded;       // per node: 1 = evaluated by RDP (shape arithmetic) or a pure view
+  int n_subgraphs = 1;
+  // prepacked (transposed, K-major) copies of GEMM weights
+  std::vector<int> packed_consts;     // tensor ids
+  std::vector<size_t> packed_off;     // byte offsets in the prepack workspace
+  size_t packed_bytes = 0;
+  void* packed_ws = nullptr;
+  std::string err;
+};
+
+Status form_groups(Compiled* c);
+// Transposed (K-major) copies of the GEMM weights into caller-owned workspace; enqueued on `stream`.
+Status prepack_weights(Compiled* c, void* workspace, size_t bytes, void* stream);
+
+// ---- per-request binding (H0: substitute symbol values into every expression)
+struct Binding {
+  const Compiled* c = nullptr;
+  int n_req = 0;
+  std::vector<std::vector<int64_t>> vals;               // [req][atom]
+  std::vector<std::vector<std::vector<int64_t>>> dims;  // [tensor][req][rank]; empty if not evaluable yet
+  std::string err;
+};
+Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* names, const int64_t* values, Binding* out);
+
+// ---- plan
+struct View {                 // one tensor of one request, resolved to storage
+  int root = -1;              // tensor id owning the bytes
+  int64_t offset = 0;         // elements from the start of the root's instance for this request
+  std::vector<int64_t> dims, strides;  // elements
+  bool contiguous() const {
+    int64_t s = 1;
+    for (int i = static_cast<int>(dims.size()) - 1; i >= 0; --i) { if (dims[i] != 1 && strides[i] != s) return false; s *= dims[i]; }
+    return true;
+  }
+};
+
+struct RootBuf {              // packed storage of a root tensor: the requests' instances back to back
+  enum Where { NONE, INPUT, OUTPUT, CONST, ARENA } where = NONE;
+  int io_index = -1;
+  std::vector<int64_t> inst_off;   // [req] byte offset of the request's instance
+  int64_t bytes = 0;
+  size_t arena_off = 0;
+  int def_step = -1, last_step = -1;
+};
+
+struct Ptr {                  // address resolved at run time
+  int where = 0;              // RootBuf::Where, or 5 = prepack workspace, 6 = scratch in arena
+  int index = -1;
+  int64_t off = 0;
+};
+
+struct Launch;                // defined in exec.cu
+
+struct Plan {
+  const Compiled* c = nullptr;
+  const Binding* b = nullptr;
+  int n_req = 0;
+  std::vector<std::vector<View>> views;   // [tensor][req]
+  std::vector<RootBuf> roots;             // [tensor]
+  size_t arena_bytes = 0, peak_live_bytes = 0, sum_bytes = 0;
+  int peak_step = 0;
+  std::vector<std::shared_ptr<Launch>> launches;
+  std::vector<size_t> scratch_off;        // per group scratch offsets in the arena
+  int gpu_launches = 0;
+  std::string err;
+  // device status word lives at arena offset 0 (first 256 bytes reserved)
+};
+Status make_plan(const Compiled* c, const Binding* b, Plan* p);
+Status build_launches(Plan* p);   // exec.cu
+Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream,
+                int64_t* info);
+
+}  // namespace sod2

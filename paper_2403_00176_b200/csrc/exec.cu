@@ -1,0 +1,542 @@
+// Launch plan (variant choice, tensor maps, kernel parameters) and the executor that enqueues the
+// fused groups on the caller's stream.  All device memory belongs to the caller; this file never
+// allocates device memory.
+#include <chrono>
+#include <cstring>
+#include <functional>
+
+#include "attention.cuh"
+#include "engine.h"
+#include "gemm_tcgen05.cuh"
+#include "kernels_compact.cuh"
+#include "kernels_rows.cuh"
+#include "tmap.h"
+
+namespace sod2 {
+
+struct RunCtx {
+  const void* const* inputs;
+  void* const* outputs;
+  char* arena;
+  char* packed;
+  cudaStream_t stream;
+  const Plan* plan;
+  char* resolve(const Ptr& p) const {
+    switch (p.where) {
+      case RootBuf::INPUT: return const_cast<char*>(static_cast<const char*>(inputs[p.index])) + p.off;
+      case RootBuf::OUTPUT: return static_cast<char*>(outputs[p.index]) + p.off;
+      case RootBuf::CONST: return const_cast<char*>(static_cast<const char*>(plan->c->g.tensors[p.index].dev_ptr)) + p.off;
+      case RootBuf::ARENA: return arena + p.off;
+      case 5: return packed + p.off;
+      default: return nullptr;
+    }
+  }
+};
+
+struct Launch {
+  int group = -1;
+  int n_kernels = 1;
+  std::function<cudaError_t(const RunCtx&)> fn;
+};
+
+namespace {
+
+int64_t numel(const std::vector<int64_t>& d) { int64_t n = 1; for (auto v : d) n *= v; return n; }
+
+struct Builder {
+  Plan& p;
+  const Compiled& c;
+  const Graph& g;
+  size_t scratch_need = 0;
+  explicit Builder(Plan& pp) : p(pp), c(*pp.c), g(pp.c->g) {}
+
+  Status fail(Status s, const std::string& m) { p.err = m; return s; }
+
+  Ptr ptr_of(int t, int r, int64_t extra_elems = 0) const {
+    const View& v = p.views[t][r];
+    const RootBuf& R = p.roots[v.root];
+    Ptr q;
+    q.where = R.where;
+    q.index = (R.where == RootBuf::CONST) ? v.root : R.io_index;
+    q.off = R.inst_off[r] + (v.offset + extra_elems) * dtype_size(g.tensors[t].dtype);
+    if (R.where == RootBuf::ARENA) q.off += static_cast<int64_t>(R.arena_off);
+    return q;
+  }
+  static bool same_base(const Ptr& a, const Ptr& b) { return a.where == b.where && a.index == b.index; }
+
+  // collapse a view to [rows, cols] with unit column stride; returns row pitch in elements
+  bool as_matrix(const View& v, int64_t* rows, int64_t* cols, int64_t* ld) const {
+    if (v.dims.empty()) return false;
+    *cols = v.dims.back();
+    *rows = numel(v.dims) / std::max<int64_t>(*cols, 1);
+    if (v.strides.back() != 1 && *cols != 1) return false;
+    // all leading dims must step uniformly
+    int64_t pitch = -1, run = 1;
+    for (int i = static_cast<int>(v.dims.size()) - 2; i >= 0; --i) {
+      if (v.dims[i] == 1) continue;
+      if (pitch < 0) { pitch = v.strides[i]; run = v.dims[i]; }
+      else { if (v.strides[i] != pitch * run) return false; run *= v.dims[i]; }
+    }
+    *ld = pitch < 0 ? *cols : pitch;
+    return true;
+  }
+
+  // rows of consecutive requests that form one contiguous matrix are merged into one launch
+  struct Seg { int r0, r1; int64_t rows; };
+  Status row_segments(const std::vector<int>& tensors, int64_t* cols_out, std::vector<int64_t>* lds, std::vector<Seg>* segs) {
+    int nt = static_cast<int>(tensors.size());
+    lds->assign(nt, 0);
+    std::vector<std::vector<int64_t>> rows(nt, std::vector<int64_t>(p.n_req));
+    for (int i = 0; i < nt; ++i)
+      for (int r = 0; r < p.n_req; ++r) {
+        int64_t rw, cl, ld;
+        if (!as_matrix(p.views[tensors[i]][r], &rw, &cl, &ld)) return fail(E_UNSUPPORTED_OP, "operand " + g.tensors[tensors[i]].name + " is not a row-major matrix view");
+        if (r == 0) (*lds)[i] = ld;
+        else if (ld != (*lds)[i] && rw > 1) return fail(E_UNSUPPORTED_OP, "row pitch differs between requests");
+        rows[i][r] = rw;
+        if (i == 0) cols_out[0] = cl;
+        if (rw != rows[0][r]) return fail(E_SHAPE_CONFLICT, "row counts differ inside a group");
+      }
+    segs->clear();
+    for (int r = 0; r < p.n_req; ++r) {
+      bool merge = !segs->empty();
+      if (merge) {
+        for (int i = 0; i < nt; ++i) {
+          Ptr a = ptr_of(tensors[i], segs->back().r0), b = ptr_of(tensors[i], r);
+          int esz = dtype_size(g.tensors[tensors[i]].dtype);
+          if (!same_base(a, b) || b.off != a.off + segs->back().rows * (*lds)[i] * esz) merge = false;
+        }
+      }
+      if (merge) { segs->back().r1 = r + 1; segs->back().rows += rows[0][r]; }
+      else segs->push_back({r, r + 1, rows[0][r]});
+    }
+    return OK;
+  }
+
+  void add(int gi, int nk, std::function<cudaError_t(const RunCtx&)> fn) {
+    auto L = std::make_shared<Launch>();
+    L->group = gi;
+    L->n_kernels = nk;
+    L->fn = std::move(fn);
+    p.gpu_launches += nk;
+    p.launches.push_back(L);
+  }
+
+  // ------------------------------------------------------------------------------ GEMM
+  Status build_gemm(int gi, const Group& G) {
+    const Tensor& W = g.tensors[G.w];
+    const int64_t K = W.S.dims[0].e.const_value(), N = W.S.dims[1].e.const_value();
+    std::vector<int> ts = {G.a, G.out};
+    if (G.res >= 0) ts.push_back(G.res);
+    int64_t cols;
+    std::vector<int64_t> lds;
+    std::vector<Seg> segs;
+    Status s = row_segments(ts, &cols, &lds, &segs);
+    if (s != OK) return s;
+    if (cols != K) return fail(E_SHAPE_CONFLICT, "GEMM inner dims differ");
+    const bool f32 = g.tensors[G.a].dtype == DType::F32;
+    if (f32) {
+      if (K > 128 || N > 128 || N % 32) return fail(E_UNSUPPORTED_OP, "fp32 fused group supports K, N <= 128, N % 32 == 0");
+      if (lds[0] != K || lds[1] != N || (G.res >= 0 && lds[2] != N)) return fail(E_UNSUPPORTED_OP, "fp32 fused group needs dense rows");
+      for (auto& sg : segs) {
+        if (sg.rows == 0) continue;
+        Ptr pa = ptr_of(G.a, sg.r0), po = ptr_of(G.out, sg.r0), pr = G.res >= 0 ? ptr_of(G.res, sg.r0) : Ptr();
+        Ptr pw = ptr_of(G.w, 0), pb = G.bias >= 0 ? ptr_of(G.bias, 0) : Ptr(), pg = G.has_ln ? ptr_of(G.gamma, 0) : Ptr(), pbe = G.has_ln ? ptr_of(G.beta, 0) : Ptr();
+        k::MlpLnParams mp{};
+        mp.M = static_cast<int>(sg.rows); mp.K = static_cast<int>(K); mp.N = static_cast<int>(N);
+        mp.act = G.act; mp.has_ln = G.has_ln; mp.eps = G.eps;
+        const bool hb = G.bias >= 0, hr = G.res >= 0, hl = G.has_ln != 0;
+        const int nc = static_cast<int>(N / 32);
+        add(gi, 1, [=](const RunCtx& x) mutable {
+          mp.X = reinterpret_cast<const float*>(x.resolve(pa));
+          mp.W = reinterpret_cast<const float*>(x.resolve(pw));
+          mp.bias = hb ? reinterpret_cast<const float*>(x.resolve(pb)) : nullptr;
+          mp.R = hr ? reinterpret_cast<const float*>(x.resolve(pr)) : nullptr;
+          mp.gamma = hl ? reinterpret_cast<const float*>(x.resolve(pg)) : nullptr;
+          mp.beta = hl ? reinterpret_cast<const float*>(x.resolve(pbe)) : nullptr;
+          mp.Y = reinterpret_cast<float*>(x.resolve(po));
+          const int grid = std::min((mp.M + 7) / 8, 148 * 2);
+          const size_t smem = (static_cast<size_t>(mp.K) * mp.N + 8 * mp.K) * sizeof(float);
+          switch (nc) {
+            case 1: cudaFuncSetAttribute(k::fused_mlp_ln_f32<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024); k::fused_mlp_ln_f32<1><<<grid, 256, smem, x.stream>>>(mp); break;
+            case 2: cudaFuncSetAttribute(k::fused_mlp_ln_f32<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024); k::fused_mlp_ln_f32<2><<<grid, 256, smem, x.stream>>>(mp); break;
+            case 3: cudaFuncSetAttribute(k::fused_mlp_ln_f32<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024); k::fused_mlp_ln_f32<3><<<grid, 256, smem, x.stream>>>(mp); break;
+            default: cudaFuncSetAttribute(k::fused_mlp_ln_f32<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024); k::fused_mlp_ln_f32<4><<<grid, 256, smem, x.stream>>>(mp); break;
+          }
+          return cudaGetLastError();
+        });
+      }
+      return OK;
+    }
+    // bf16 on tcgen05
+    if (G.has_ln || G.act2) return fail(E_UNSUPPORTED_OP, "bf16 GEMM epilogue: unsupported tail");
+    if (K % 8 || lds[0] % 8) return fail(E_UNSUPPORTED_OP, "GEMM operand rows must be 16-byte multiples for TMA");
+    size_t pk = 0;
+    for (size_t i = 0; i < c.packed_consts.size(); ++i) if (c.packed_consts[i] == G.w) pk = c.packed_off[i];
+    for (auto& sg : segs) {
+      if (sg.rows == 0) continue;
+      Ptr pa = ptr_of(G.a, sg.r0), po = ptr_of(G.out, sg.r0), pr = G.res >= 0 ? ptr_of(G.res, sg.r0) : Ptr();
+      Ptr pw; pw.where = 5; pw.off = static_cast<int64_t>(pk);
+      Ptr pb = G.bias >= 0 ? ptr_of(G.bias, 0) : Ptr();
+      const int M = static_cast<int>(sg.rows);
+      const int64_t lda = lds[0], ldo = lds[1], ldr = G.res >= 0 ? lds[2] : 0;
+      // shape-class variant (the paper's multi-version idea, Section 4.4.2): narrow tiles when the
+      // wide ones would leave SMs idle
+      const int tiles_m = (M + 127) / 128;
+      int bn = 128;
+      if (tiles_m * ((N + 127) / 128) < 148 && N > 64) bn = 64;
+      const bool hb = G.bias >= 0, hr = G.res >= 0;
+      const int act = G.act;
+      struct Cache { const void* a = nullptr; const void* w = nullptr; CUtensorMap ta, tb; };
+      auto cache = std::make_shared<Cache>();
+      add(gi, 1, [=](const RunCtx& x) {
+        const void* A = x.resolve(pa);
+        const void* Wt = x.resolve(pw);
+        if (cache->a != A || cache->w != Wt) {
+          if (!encode_bf16_2d(&cache->ta, A, M, K, lda, 128) || !encode_bf16_2d(&cache->tb, Wt, N, K, K, bn)) return cudaErrorInvalidValue;
+          cache->a = A; cache->w = Wt;
+        }
+        k::GemmEpilogue ep{};
+        ep.bias = hb ? reinterpret_cast<const __nv_bfloat16*>(x.resolve(pb)) : nullptr;
+        ep.residual = hr ? reinterpret_cast<const __nv_bfloat16*>(x.resolve(pr)) : nullptr;
+        ep.ldr = ldr;
+        ep.out = reinterpret_cast<__nv_bfloat16*>(x.resolve(po));
+        ep.ldo = ldo;
+        ep.act = act;
+        ep.status = reinterpret_cast<int*>(x.arena);
+        const int grid = tiles_m * static_cast<int>((N + bn - 1) / bn);
+        if (bn == 128) {
+          constexpr int smem = k::GemmSmem<128, 3>::TOTAL;
+          static bool once = (cudaFuncSetAttribute(k::gemm_bf16_tcgen05<128, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);
+          (void)once;
+          k::gemm_bf16_tcgen05<128, 3><<<grid, 128, smem, x.stream>>>(cache->ta, cache->tb, M, static_cast<int>(N), static_cast<int>(K), ep);
+        } else {
+          constexpr int smem = k::GemmSmem<64, 4>::TOTAL;
+          static bool once = (cudaFuncSetAttribute(k::gemm_bf16_tcgen05<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);
+          (void)once;
+          k::gemm_bf16_tcgen05<64, 4><<<grid, 128, smem, x.stream>>>(cache->ta, cache->tb, M, static_cast<int>(N), static_cast<int>(K), ep);
+        }
+        return cudaGetLastError();
+      });
+    }
+    return OK;
+  }
+
+  // ------------------------------------------------------------------------------ attention
+  Status build_attention(int gi, const Group& G) {
+    if (g.tensors[G.q].dtype != DType::BF16) return fail(E_UNSUPPORTED_OP, "attention group is bf16 only");
+    for (int r0 = 0; r0 < p.n_req; r0 += k::ATTN_MAX_REQ) {
+      const int nr = std::min(k::ATTN_MAX_REQ, p.n_req - r0);
+      k::AttnParams ap{};
+      ap.n_req = nr;
+      ap.scale_log2e = G.scale * 1.4426950408889634f;
+      Ptr bq = ptr_of(G.q, r0), bk = ptr_of(G.k, r0), bv = ptr_of(G.v, r0), bo = ptr_of(G.out, r0);
+      int tiles = 0, H = -1;
+      for (int i = 0; i < nr; ++i) {
+        const int r = r0 + i;
+        const View &q = p.views[G.q][r], &kk = p.views[G.k][r], &v = p.views[G.v][r], &o = p.views[G.out][r];
+        const int rk = static_cast<int>(q.dims.size());
+        if (rk < 3 || kk.dims.size() != q.dims.size() || v.dims.size() != q.dims.size()) return fail(E_UNSUPPORTED_OP, "attention operands need rank >= 3");
+        for (int d = 0; d < rk - 3; ++d) if (q.dims[d] != 1) return fail(E_UNSUPPORTED_OP, "attention: leading batch dims must be 1");
+        const int64_t h = q.dims[rk - 3], L = q.dims[rk - 2], dh = q.dims[rk - 1];
+        if (dh != 64) return fail(E_UNSUPPORTED_OP, "attention kernel is specialised for head dim 64");
+        if (kk.dims[rk - 2] != dh || kk.dims[rk - 1] != L || v.dims[rk - 2] != L || v.dims[rk - 1] != dh) return fail(E_SHAPE_CONFLICT, "attention operand shapes");
+        if (q.strides[rk - 1] != 1 || kk.strides[rk - 2] != 1 || v.strides[rk - 1] != 1 || o.strides[rk - 1] != 1) return fail(E_UNSUPPORTED_OP, "attention: head dim must be contiguous");
+        if (H < 0) H = static_cast<int>(h); else if (H != h) return fail(E_UNSUPPORTED_OP, "attention: head count differs");
+        k::AttnReq& R = ap.r[i];
+        Ptr pq = ptr_of(G.q, r), pk2 = ptr_of(G.k, r), pv = ptr_of(G.v, r), po = ptr_of(G.out, r);
+        if (!same_base(pq, bq) || !same_base(pk2, bk) || !same_base(pv, bv) || !same_base(po, bo)) return fail(E_INTERNAL, "attention bases");
+        R.q_off = (pq.off - bq.off) / 2; R.k_off = (pk2.off - bk.off) / 2; R.v_off = (pv.off - bv.off) / 2; R.o_off = (po.off - bo.off) / 2;
+        R.L = static_cast<int>(L);
+        R.q_ts = static_cast<int>(q.strides[rk - 2]); R.k_ts = static_cast<int>(kk.strides[rk - 1]);
+        R.v_ts = static_cast<int>(v.strides[rk - 2]); R.o_ts = static_cast<int>(o.strides[rk - 2]);
+        R.q_hs = static_cast<int>(q.strides[rk - 3]); R.k_hs = static_cast<int>(kk.strides[rk - 3]);
+        R.v_hs = static_cast<int>(v.strides[rk - 3]); R.o_hs = static_cast<int>(o.strides[rk - 3]);
+        if ((R.q_ts | R.k_ts | R.v_ts | R.q_hs | R.k_hs | R.v_hs) % 8 || (pq.off | pk2.off | pv.off) % 16 || (R.o_ts | R.o_hs) % 2 || po.off % 4)
+          return fail(E_MISALIGNED, "attention operands must be 16-byte aligned");
+        ap.tile_start[i] = tiles;
+        tiles += static_cast<int>((L + 63) / 64);
+      }
+      ap.tile_start[nr] = tiles;
+      ap.H = H;
+      if (tiles == 0) continue;
+      add(gi, 1, [=](const RunCtx& x) mutable {
+        ap.q = reinterpret_cast<const __nv_bfloat16*>(x.resolve(bq));
+        ap.k = reinterpret_cast<const __nv_bfloat16*>(x.resolve(bk));
+        ap.v = reinterpret_cast<const __nv_bfloat16*>(x.resolve(bv));
+        ap.o = reinterpret_cast<__nv_bfloat16*>(x.resolve(bo));
+        k::attention_fwd_bf16<<<dim3(tiles, ap.H), 128, 0, x.stream>>>(ap);
+        return cudaGetLastError();
+      });
+    }
+    return OK;
+  }
+
+  // ------------------------------------------------------------------------------ LayerNorm rows
+  Status build_layernorm(int gi, const Group& G) {
+    int64_t D;
+    std::vector<int64_t> lds;
+    std::vector<Seg> segs;
+    Status s = row_segments({G.a, G.out}, &D, &lds, &segs);
+    if (s != OK) return s;
+    if (lds[0] != D || lds[1] != D || D % 8 || D > 1024) return build_chain(gi, G, true);
+    Ptr pg = ptr_of(G.gamma, 0), pb = ptr_of(G.beta, 0);
+    const float eps = G.eps;
+    const int ch = static_cast<int>((D / 8 + 31) / 32);
+    for (auto& sg : segs) {
+      if (!sg.rows) continue;
+      Ptr pa = ptr_of(G.a, sg.r0), po = ptr_of(G.out, sg.r0);
+      const long long rows = sg.rows;
+      add(gi, 1, [=](const RunCtx& x) {
+        auto* X = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pa));
+        auto* Y = reinterpret_cast<__nv_bfloat16*>(x.resolve(po));
+        auto* Gm = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pg));
+        auto* Bt = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pb));
+        const unsigned grid = static_cast<unsigned>((rows + 7) / 8);
+        switch (ch) {
+          case 1: k::layernorm_bf16<1><<<grid, 256, 0, x.stream>>>(X, Gm, Bt, Y, rows, static_cast<int>(D), eps); break;
+          case 2: k::layernorm_bf16<2><<<grid, 256, 0, x.stream>>>(X, Gm, Bt, Y, rows, static_cast<int>(D), eps); break;
+          case 3: k::layernorm_bf16<3><<<grid, 256, 0, x.stream>>>(X, Gm, Bt, Y, rows, static_cast<int>(D), eps); break;
+          default: k::layernorm_bf16<4><<<grid, 256, 0, x.stream>>>(X, Gm, Bt, Y, rows, static_cast<int>(D), eps); break;
+        }
+        return cudaGetLastError();
+      });
+    }
+    return OK;
+  }
+
+  // ------------------------------------------------------------------------------ generic chain
+  void fill_operand(k::ChainOperand* o, int t, int r, const std::vector<int64_t>& odims) {
+    const Tensor& T = g.tensors[t];
+    std::memset(o, 0, sizeof(*o));
+    if (T.kind == TKind::FCONST) { o->ptr = nullptr; o->scalar = static_cast<float>(T.fdata); return; }
+    const View& v = p.views[t][T.kind == TKind::CONST ? 0 : r];
+    o->is_bf16 = T.dtype == DType::BF16;
+    const int rk = static_cast<int>(v.dims.size());
+    for (int i = 0; i < 4; ++i) {
+      int src = i - (4 - rk);
+      o->stride[i] = (src >= 0 && v.dims[src] != 1) ? v.strides[src] : 0;  // broadcast dims read in place
+    }
+    (void)odims;
+  }
+  Status build_chain(int gi, const Group& G, bool ln_only = false) {
+    const Tensor& O = g.tensors[G.out];
+    if (O.S.rank > 4) return fail(E_UNSUPPORTED_OP, "chain kernel supports rank <= 4");
+    for (int r = 0; r < p.n_req; ++r) {
+      const View& ov = p.views[G.out][r];
+      if (!ov.contiguous()) return fail(E_UNSUPPORTED_OP, "chain output must be contiguous");
+      k::ChainParams cp{};
+      std::vector<int64_t> od(4, 1);
+      for (size_t i = 0; i < ov.dims.size(); ++i) od[4 - ov.dims.size() + i] = ov.dims[i];
+      for (int i = 0; i < 4; ++i) cp.dim[i] = od[i];
+      if (numel(ov.dims) == 0) continue;
+      fill_operand(&cp.in0, G.a, r, od);
+      cp.n_ops = ln_only ? 0 : static_cast<int>(G.chain_ops.size());
+      std::vector<Ptr> optr(k::CHAIN_MAX_OPS);
+      std::vector<char> has(k::CHAIN_MAX_OPS, 0);
+      for (int i = 0; i < cp.n_ops; ++i) {
+        cp.op[i] = G.chain_ops[i];
+        int t = G.chain_operands[i];
+        if (t >= 0) {
+          fill_operand(&cp.operand[i], t, r, od);
+          if (g.tensors[t].kind != TKind::FCONST) { optr[i] = ptr_of(t, g.tensors[t].kind == TKind::CONST ? 0 : r); has[i] = 1; }
+        }
+      }
+      cp.out_bf16 = O.dtype == DType::BF16;
+      cp.red = ln_only ? 2 : G.red;
+      cp.eps = G.eps;
+      Ptr pin = ptr_of(G.a, r), pout = ptr_of(G.out, r);
+      Ptr pg = cp.red == 2 ? ptr_of(G.gamma, 0) : Ptr(), pb = cp.red == 2 ? ptr_of(G.beta, 0) : Ptr();
+      cp.gb_bf16 = cp.red == 2 ? g.tensors[G.gamma].dtype == DType::BF16 : 0;
+      const int red = cp.red;
+      if (red && cp.dim[3] * 4 > 200 * 1024) return fail(E_UNSUPPORTED_OP, "row too long for the row-reduction kernel");
+      add(gi, 1, [=](const RunCtx& x) mutable {
+        cp.in0.ptr = x.resolve(pin);
+        for (int i = 0; i < cp.n_ops; ++i) if (has[i]) cp.operand[i].ptr = x.resolve(optr[i]);
+        cp.out = x.resolve(pout);
+        if (red == 2) { cp.gamma = x.resolve(pg); cp.beta = x.resolve(pb); }
+        if (!red) {
+          const long long total = cp.dim[0] * cp.dim[1] * cp.dim[2] * cp.dim[3];
+          const unsigned grid = static_cast<unsigned>(std::min<long long>((total + 255) / 256, 148 * 16));
+          k::chain_elementwise<<<grid, 256, 0, x.stream>>>(cp);
+        } else {
+          const long long rows = cp.dim[0] * cp.dim[1] * cp.dim[2];
+          const size_t smem = static_cast<size_t>(cp.dim[3]) * 4;
+          if (smem > 48 * 1024) cudaFuncSetAttribute(k::chain_rowreduce, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+          k::chain_rowreduce<<<static_cast<unsigned>(std::min<long long>(rows, 148 * 8)), 256, smem, x.stream>>>(cp);
+        }
+        return cudaGetLastError();
+      });
+    }
+    return OK;
+  }
+
+  // ------------------------------------------------------------------------------ top-k keep
+  Status build_topk(int gi, const Group& G) {
+    if (g.tensors[G.a].dtype != DType::BF16) return fail(E_UNSUPPORTED_OP, "top-k keep is bf16 only");
+    for (int r0 = 0; r0 < p.n_req; r0 += k::COMPACT_MAX_REQ) {
+      const int nr = std::min(k::COMPACT_MAX_REQ, p.n_req - r0);
+      k::TopkParams tp{};
+      tp.n_req = nr;
+      Ptr by = ptr_of(G.a, r0), bo = ptr_of(G.out, r0), bi = ptr_of(G.out2, r0);
+      int64_t D = -1, total_rows = 0, first_row = 0;
+      int nmax = 0;
+      for (int i = 0; i < nr; ++i) {
+        const int r = r0 + i;
+        const View &y = p.views[G.a][r], &o = p.views[G.out][r];
+        if (!y.contiguous() || !o.contiguous()) return fail(E_UNSUPPORTED_OP, "top-k keep needs contiguous rows");
+        const int64_t d = y.dims.back(), n = numel(y.dims) / d, kk = numel(o.dims) / d;
+        if (D < 0) D = d; else if (D != d) return fail(E_UNSUPPORTED_OP, "top-k keep: row length differs");
+        if (D % 8) return fail(E_UNSUPPORTED_OP, "top-k keep: rows must be 16-byte multiples");
+        Ptr py = ptr_of(G.a, r), po = ptr_of(G.out, r), pi = ptr_of(G.out2, r);
+        if (!same_base(py, by) || !same_base(po, bo) || !same_base(pi, bi)) return fail(E_INTERNAL, "top-k bases");
+        tp.r[i].row0 = (py.off - by.off) / (D * 2);
+        tp.r[i].out_row0 = (po.off - bo.off) / (D * 2);
+        tp.r[i].idx0 = (pi.off - bi.off) / 8;
+        tp.r[i].n = static_cast<int>(n);
+        tp.r[i].k = static_cast<int>(kk);
+        if (i == 0) first_row = tp.r[i].row0;
+        total_rows = tp.r[i].row0 + n - first_row;
+        nmax = std::max(nmax, static_cast<int>(n));
+      }
+      tp.D = static_cast<int>(D);
+      const size_t sc_bytes = static_cast<size_t>(total_rows) * 8;
+      scratch_need = std::max(scratch_need, sc_bytes);
+      const long long rows = total_rows;
+      const size_t smem = static_cast<size_t>((nmax + 1) & ~1) * 8 + static_cast<size_t>(nmax) * 4;
+      if (smem > 200 * 1024) return fail(E_UNSUPPORTED_OP, "top-k keep: too many tokens for one CTA");
+      add(gi, 2, [=](const RunCtx& x) mutable {
+        double* score = reinterpret_cast<double*>(x.arena + x.plan->scratch_off[0]);
+        tp.y = reinterpret_cast<const __nv_bfloat16*>(x.resolve(by));
+        tp.out = reinterpret_cast<__nv_bfloat16*>(x.resolve(bo));
+        tp.idx = reinterpret_cast<long long*>(x.resolve(bi));
+        tp.score = score;
+        k::ScoreParams sp{tp.y, score, rows, tp.D};
+        if (rows) k::row_sumsq_f64<<<static_cast<unsigned>((rows + 7) / 8), 256, 0, x.stream>>>(sp);
+        if (smem > 48 * 1024) cudaFuncSetAttribute(k::topk_keep, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        k::topk_keep<<<tp.n_req, 1024, smem, x.stream>>>(tp);
+        return cudaGetLastError();
+      });
+    }
+    return OK;
+  }
+
+  // ------------------------------------------------------------------------------ NonZero
+  Status build_nonzero(int gi, const Group& G) {
+    const Tensor& X = g.tensors[G.a];
+    if (X.S.rank > 4 || X.S.rank < 1) return fail(E_UNSUPPORTED_OP, "NonZero supports rank 1..4");
+    // the runtime symbol that names the count
+    const Expr& ce = g.tensors[G.out].S.dims[1].e;
+    const int sym = ce.terms.begin()->first[0].first;
+    for (int r = 0; r < p.n_req; ++r) {
+      const View& v = p.views[G.a][r];
+      if (!v.contiguous()) return fail(E_UNSUPPORTED_OP, "NonZero needs a contiguous input");
+      k::NonZeroParams np{};
+      np.is_bf16 = X.dtype == DType::BF16;
+      np.numel = numel(v.dims);
+      np.rank = static_cast<int>(v.dims.size());
+      for (int i = 0; i < np.rank; ++i) np.dims[i] = v.dims[i];
+      np.nblocks = static_cast<int>((np.numel + k::NZ_BLOCK - 1) / k::NZ_BLOCK);
+      scratch_need = std::max(scratch_need, static_cast<size_t>(np.nblocks + 1) * 4);
+      Ptr px = ptr_of(G.a, r), po = ptr_of(G.out, r);
+      const size_t count_off = 256 + (static_cast<size_t>(sym) * p.n_req + r) * 8;
+      add(gi, 3, [=](const RunCtx& x) mutable {
+        np.x = x.resolve(px);
+        np.out = reinterpret_cast<long long*>(x.resolve(po));
+        np.block_count = reinterpret_cast<int*>(x.arena + x.plan->scratch_off[0]);
+        np.count_out = reinterpret_cast<long long*>(x.arena + count_off);
+        if (np.nblocks == 0) return cudaMemsetAsync(np.count_out, 0, 8, x.stream);
+        k::nonzero_count<<<np.nblocks, k::NZ_BLOCK, 0, x.stream>>>(np);
+        k::nonzero_scan<<<1, 1024, 0, x.stream>>>(np);
+        k::nonzero_write<<<np.nblocks, k::NZ_BLOCK, 0, x.stream>>>(np);
+        return cudaGetLastError();
+      });
+    }
+    return OK;
+  }
+
+  Status run() {
+    p.launches.clear();
+    p.gpu_launches = 0;
+    for (size_t gi = 0; gi < c.groups.size(); ++gi) {
+      const Group& G = c.groups[gi];
+      Status s = OK;
+      switch (G.kind) {
+        case GKind::GEMM: s = build_gemm(static_cast<int>(gi), G); break;
+        case GKind::ATTENTION: s = build_attention(static_cast<int>(gi), G); break;
+        case GKind::LAYERNORM: s = build_layernorm(static_cast<int>(gi), G); break;
+        case GKind::CHAIN: s = build_chain(static_cast<int>(gi), G); break;
+        case GKind::TOPK_KEEP: s = build_topk(static_cast<int>(gi), G); break;
+        case GKind::NONZERO: s = build_nonzero(static_cast<int>(gi), G); break;
+        default: return fail(E_UNSUPPORTED_OP, std::string("no executor yet for group kind ") + gkind_name(G.kind));
+      }
+      if (s != OK) return s;
+    }
+    // one scratch region shared by all groups (they run in stream order), after the tensors
+    p.scratch_off.assign(1, p.arena_bytes);
+    p.arena_bytes += (scratch_need + 255) & ~size_t(255);
+    return OK;
+  }
+};
+
+__global__ void transpose_bf16(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out, int K, int N) {
+  // in [K, N] row-major -> out [N, K] row-major
+  __shared__ __nv_bfloat16 tile[32][33];
+  const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int kk = k0 + i, n = n0 + threadIdx.x;
+    if (kk < K && n < N) tile[i][threadIdx.x] = in[static_cast<long long>(kk) * N + n];
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int n = n0 + i, kk = k0 + threadIdx.x;
+    if (kk < K && n < N) out[static_cast<long long>(n) * K + kk] = tile[threadIdx.x][i];
+  }
+}
+
+}  // namespace
+
+Status build_launches(Plan* p) {
+  Builder b(*p);
+  return b.run();
+}
+
+Status prepack_weights(Compiled* c, void* workspace, size_t bytes, void* stream) {
+  if (c->packed_bytes == 0) { c->packed_ws = workspace; return OK; }
+  if (!workspace || bytes < c->packed_bytes) { c->err = "prepack workspace too small"; return E_ARENA_TOO_SMALL; }
+  if (reinterpret_cast<uintptr_t>(workspace) & 255) { c->err = "prepack workspace must be 256-byte aligned"; return E_MISALIGNED; }
+  for (size_t i = 0; i < c->packed_consts.size(); ++i) {
+    const Tensor& W = c->g.tensors[c->packed_consts[i]];
+    if (!W.dev_ptr) { c->err = "constant " + W.name + " has no device data"; return E_INVALID_ARG; }
+    const int K = static_cast<int>(W.S.dims[0].e.const_value()), N = static_cast<int>(W.S.dims[1].e.const_value());
+    transpose_bf16<<<dim3((N + 31) / 32, (K + 31) / 32), dim3(32, 8), 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const __nv_bfloat16*>(W.dev_ptr), reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + c->packed_off[i]), K, N);
+  }
+  if (cudaGetLastError() != cudaSuccess) { c->err = "prepack launch failed"; return E_CUDA; }
+  c->packed_ws = workspace;
+  return OK;
+}
+
+Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream, int64_t* info) {
+  if (!arena && p->arena_bytes) { p->err = "arena is null"; return E_INVALID_ARG; }
+  if (arena_bytes < p->arena_bytes) { p->err = "arena too small"; return E_ARENA_TOO_SMALL; }
+  if (reinterpret_cast<uintptr_t>(arena) & 255) { p->err = "arena must be 256-byte aligned"; return E_MISALIGNED; }
+  if (p->c->packed_bytes && !p->c->packed_ws) { p->err = "weights are not prepacked"; return E_INVALID_ARG; }
+  auto t0 = std::chrono::steady_clock::now();
+  RunCtx x{inputs, outputs, static_cast<char*>(arena), static_cast<char*>(p->c->packed_ws), static_cast<cudaStream_t>(stream), p};
+  if (cudaMemsetAsync(arena, 0, 256, x.stream) != cudaSuccess) { p->err = "cannot clear the status word"; return E_CUDA; }
+  for (auto& L : p->launches) {
+    cudaError_t e = L->fn(x);
+    if (e != cudaSuccess) {
+      p->err = std::string("launch failed in group ") + std::to_string(L->group) + ": " + cudaGetErrorString(e);
+      return E_CUDA;
+    }
+  }
+  if (info) {
+    info[0] = std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t0).count();
+    info[1] = p->gpu_launches;
+  }
+  return OK;
+}
+
+}  // namespace sod2

@@ -1,0 +1,296 @@
+// Per-request binding (evaluate every RDP expression), view resolution, liveness and the
+// run-time memory allocation plan (Section 4.4.1: one linear arena, planned at execution time once
+// all sizes are known, greedy from the peak-memory step outwards).
+#include <algorithm>
+#include <cstring>
+#include <map>
+
+#include "engine.h"
+
+namespace sod2 {
+
+Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* names, const int64_t* values, Binding* out) {
+  const Graph& g = c->g;
+  if (n_req <= 0 || n_syms < 0) { out->err = "need at least one request"; return E_INVALID_ARG; }
+  out->c = c;
+  out->n_req = n_req;
+  out->vals.assign(n_req, std::vector<int64_t>(g.cx.atoms.size(), INT64_MIN));
+  for (int s = 0; s < n_syms; ++s) {
+    int id = g.cx.find_symbol(names[s]);
+    if (id < 0) { out->err = std::string("unknown symbol ") + names[s]; return E_INVALID_ARG; }
+    const Atom& a = g.cx.atoms[id];
+    for (int r = 0; r < n_req; ++r) {
+      int64_t v = values[static_cast<size_t>(r) * n_syms + s];
+      if (v < a.lo || v > a.hi) { out->err = "symbol " + a.name + " = " + std::to_string(v) + " outside its declared range"; return E_BAD_DIM; }
+      out->vals[r][id] = v;
+    }
+  }
+  for (int id : g.user_syms)
+    if (out->vals[0][id] == INT64_MIN) { out->err = "symbol " + g.cx.atoms[id].name + " is not bound"; return E_UNBOUND_SYMBOL; }
+  // bind-time assertions recorded by RDP (two inferences of one extent must agree)
+  for (int r = 0; r < n_req; ++r)
+    for (auto& as : g.asserts) {
+      bool ok1, ok2;
+      int64_t x = e_eval(g.cx, as.a, out->vals[r], &ok1), y = e_eval(g.cx, as.b, out->vals[r], &ok2);
+      if (ok1 && ok2 && x != y) { out->err = "shape conflict: " + as.what + " (" + std::to_string(x) + " vs " + std::to_string(y) + ")"; return E_SHAPE_CONFLICT; }
+    }
+  out->dims.assign(g.tensors.size(), {});
+  for (size_t t = 0; t < g.tensors.size(); ++t) {
+    const ShapeVal& s = g.tensors[t].S;
+    if (s.rank < 0) continue;
+    bool evaluable = true;
+    std::vector<std::vector<int64_t>> per(n_req, std::vector<int64_t>(s.rank));
+    for (int r = 0; r < n_req && evaluable; ++r)
+      for (int i = 0; i < s.rank; ++i) {
+        if (!s.dims[i].known()) { evaluable = false; break; }
+        bool ok;
+        int64_t v = e_eval(g.cx, s.dims[i].e, out->vals[r], &ok);
+        if (!ok) {  // depends on a runtime symbol: use its static upper bound for planning
+          v = e_upper(g.cx, s.dims[i].e, out->vals[r], &ok);
+          if (!ok) { evaluable = false; break; }
+        }
+        if (v < 0) { out->err = "negative extent for " + g.tensors[t].name; return E_BAD_DIM; }
+        per[r][i] = v;
+      }
+    if (evaluable) out->dims[t] = std::move(per);
+  }
+  return OK;
+}
+
+namespace {
+
+int64_t numel(const std::vector<int64_t>& d) {
+  int64_t n = 1;
+  for (int64_t v : d) n *= v;
+  return n;
+}
+std::vector<int64_t> contiguous_strides(const std::vector<int64_t>& d) {
+  std::vector<int64_t> s(d.size());
+  int64_t acc = 1;
+  for (int i = static_cast<int>(d.size()) - 1; i >= 0; --i) { s[i] = acc; acc *= d[i]; }
+  return s;
+}
+
+// strides of `newd` viewing memory laid out as (oldd, olds); false if a copy would be needed
+bool reshape_view(const std::vector<int64_t>& oldd, const std::vector<int64_t>& olds, const std::vector<int64_t>& newd,
+                  std::vector<int64_t>* news) {
+  news->assign(newd.size(), 0);
+  if (numel(oldd) == 0) { *news = contiguous_strides(newd); return true; }
+  int vd = static_cast<int>(newd.size()) - 1;
+  if (oldd.empty()) { for (auto& s : *news) s = 1; return true; }
+  int64_t chunk_base = olds.back(), tnumel = 1, vnumel = 1;
+  for (int td = static_cast<int>(oldd.size()) - 1; td >= 0; --td) {
+    tnumel *= oldd[td];
+    if (td == 0 || (oldd[td - 1] != 1 && olds[td - 1] != tnumel * chunk_base)) {
+      while (vd >= 0 && (vnumel < tnumel || newd[vd] == 1)) {
+        (*news)[vd] = vnumel * chunk_base;
+        vnumel *= newd[vd];
+        --vd;
+      }
+      if (vnumel != tnumel) return false;
+      if (td > 0) { chunk_base = olds[td - 1]; tnumel = 1; vnumel = 1; }
+    }
+  }
+  return vd == -1;
+}
+
+struct Planner {
+  const Compiled& c;
+  const Graph& g;
+  const Binding& b;
+  Plan& p;
+  std::vector<char> resolved;
+  Planner(const Compiled& cc, const Binding& bb, Plan& pp) : c(cc), g(cc.g), b(bb), p(pp), resolved(cc.g.tensors.size(), 0) {}
+
+  Status fail(Status s, const std::string& m) { p.err = m; return s; }
+
+  Status make_root(int t) {
+    if (b.dims[t].empty()) return fail(E_INTERNAL, "no concrete shape for " + g.tensors[t].name);
+    const Tensor& T = g.tensors[t];
+    RootBuf& R = p.roots[t];
+    R.inst_off.resize(p.n_req);
+    int64_t off = 0;
+    int esz = dtype_size(T.dtype);
+    bool per_request = T.kind != TKind::CONST;
+    for (int r = 0; r < p.n_req; ++r) {
+      View& v = p.views[t][r];
+      v.root = t;
+      v.offset = 0;
+      v.dims = b.dims[t][r];
+      v.strides = contiguous_strides(v.dims);
+      R.inst_off[r] = per_request ? off : 0;
+      int64_t bytes = numel(v.dims) * esz;
+      if (per_request) off += (bytes + 15) & ~int64_t(15);
+      else off = bytes;
+    }
+    R.bytes = off;
+    if (T.kind == TKind::INPUT) { R.where = RootBuf::INPUT; R.io_index = T.io_index; }
+    else if (T.kind == TKind::CONST) { R.where = RootBuf::CONST; }
+    else if (T.is_output) { R.where = RootBuf::OUTPUT; R.io_index = T.io_index; }
+    else R.where = RootBuf::ARENA;
+    resolved[t] = 1;
+    return OK;
+  }
+
+  Status resolve(int t) {
+    if (resolved[t]) return OK;
+    const Storage& st = c.storage[t];
+    if (st.kind == Storage::FOLDED) { resolved[t] = 1; return OK; }
+    if (st.kind == Storage::ROOT) return make_root(t);
+    const Node& n = g.nodes[st.node];
+    if (b.dims[t].empty()) return fail(E_INTERNAL, "no concrete shape for " + g.tensors[t].name);
+    if (st.kind == Storage::VIEW_OF_OUTPUT) {
+      // t is the input of a Transpose whose output `o` owns the bytes
+      int o = st.other;
+      Status s = resolve(o);
+      if (s != OK) return s;
+      std::vector<int64_t> perm = n.attr_list("perm");
+      for (int r = 0; r < p.n_req; ++r) {
+        const View& vo = p.views[o][r];
+        View& v = p.views[t][r];
+        v.root = vo.root;
+        v.offset = vo.offset;
+        v.dims = b.dims[t][r];
+        v.strides.assign(v.dims.size(), 0);
+        for (size_t i = 0; i < perm.size(); ++i) v.strides[perm[i]] = vo.strides[i];
+      }
+      resolved[t] = 1;
+      return OK;
+    }
+    // VIEW_OF_INPUT
+    int in = st.other;
+    Status s = resolve(in);
+    if (s != OK) return s;
+    for (int r = 0; r < p.n_req; ++r) {
+      const View& vi = p.views[in][r];
+      View& v = p.views[t][r];
+      v.root = vi.root;
+      v.offset = vi.offset;
+      v.dims = b.dims[t][r];
+      if (n.op == "Transpose") {
+        std::vector<int64_t> perm = n.attr_list("perm");
+        v.strides.resize(perm.size());
+        for (size_t i = 0; i < perm.size(); ++i) v.strides[i] = vi.strides[perm[i]];
+      } else if (n.op == "Reshape") {
+        if (!reshape_view(vi.dims, vi.strides, v.dims, &v.strides))
+          return fail(E_UNSUPPORTED_OP, "Reshape producing " + g.tensors[t].name + " is not a view of its input layout");
+      } else {  // Slice
+        v.strides = vi.strides;
+        for (size_t ax = 0; ax < vi.dims.size(); ++ax) {
+          int64_t st0 = n.attr_i("_start" + std::to_string(ax), 0), step = n.attr_i("_step" + std::to_string(ax), 1);
+          v.offset += st0 * vi.strides[ax];
+          v.strides[ax] = vi.strides[ax] * step;
+        }
+      }
+    }
+    resolved[t] = 1;
+    return OK;
+  }
+
+  Status run() {
+    size_t T = g.tensors.size();
+    p.views.assign(T, std::vector<View>(p.n_req));
+    p.roots.assign(T, RootBuf());
+    // resolve every tensor a group touches
+    for (auto& G : c.groups) {
+      if (G.kind == GKind::UNSUPPORTED) return fail(E_UNSUPPORTED_OP, "group around " + g.nodes[G.nodes[0]].op + ": " + G.why);
+      for (int t : G.ext_in) { Status s = resolve(t); if (s != OK) return s; }
+      for (int t : G.ext_out) { Status s = resolve(t); if (s != OK) return s; }
+    }
+    for (int t : g.outputs) { Status s = resolve(t); if (s != OK) return s; }
+    // liveness of arena roots over the group sequence
+    int steps = static_cast<int>(c.groups.size());
+    for (int s = 0; s < steps; ++s) {
+      const Group& G = c.groups[s];
+      auto touch = [&](int t, bool def) {
+        if (c.storage[t].kind == Storage::FOLDED || !resolved[t]) return;
+        int root = p.views[t][0].root;
+        if (root < 0) return;
+        RootBuf& R = p.roots[root];
+        if (def && R.def_step < 0) R.def_step = s;
+        R.last_step = std::max(R.last_step, s);
+        if (R.def_step < 0) R.def_step = s;
+      };
+      for (int t : G.ext_out) touch(t, true);
+      for (int t : G.ext_in) touch(t, false);
+    }
+    return plan_arena(steps);
+  }
+
+  // Peak-first greedy: place the tensors live at the peak step contiguously, then walk forward
+  // and backward from the peak, each new tensor taking the smallest free gap that fits (ties: lowest
+  // offset), else extending the arena. Offsets are 256-byte aligned; the first 256 bytes hold the
+  // device status word.
+  Status plan_arena(int steps) {
+    // header: status word (256 B) + one 8-byte count slot per (runtime symbol, request)
+    const size_t HEADER = (256 + 8 * g.cx.atoms.size() * static_cast<size_t>(p.n_req) + 255) & ~size_t(255);
+    std::vector<int> ids;
+    for (size_t t = 0; t < p.roots.size(); ++t)
+      if (p.roots[t].where == RootBuf::ARENA && p.roots[t].def_step >= 0) ids.push_back(static_cast<int>(t));
+    auto sz = [&](int t) { return (static_cast<size_t>(p.roots[t].bytes) + 255) & ~size_t(255); };
+    // scratch of groups is planned like a tensor living for exactly that step
+    std::vector<size_t> live(steps + 1, 0);
+    p.sum_bytes = 0;
+    for (int t : ids) {
+      p.sum_bytes += sz(t);
+      for (int s = p.roots[t].def_step; s <= p.roots[t].last_step; ++s) live[s] += sz(t);
+    }
+    int peak = 0;
+    for (int s = 0; s < steps; ++s) if (live[s] > live[peak]) peak = s;
+    p.peak_step = peak;
+    p.peak_live_bytes = steps ? live[peak] : 0;
+    struct Placed { size_t off, size; int def, last; };
+    std::vector<Placed> placed;
+    size_t top = HEADER;
+    auto place = [&](int t) {
+      RootBuf& R = p.roots[t];
+      size_t need = sz(t);
+      if (c.flags & OPT_NO_REUSE) { R.arena_off = top; top += need; placed.push_back({R.arena_off, need, R.def_step, R.last_step}); return; }
+      // free gaps among tensors whose lifetime overlaps this one
+      std::vector<std::pair<size_t, size_t>> busy;
+      for (auto& q : placed) if (!(q.last < R.def_step || q.def > R.last_step)) busy.push_back({q.off, q.off + q.size});
+      std::sort(busy.begin(), busy.end());
+      size_t best_off = SIZE_MAX, best_gap = SIZE_MAX, cur = HEADER;
+      for (auto& iv : busy) {
+        if (iv.first > cur && iv.first - cur >= need && iv.first - cur < best_gap) { best_gap = iv.first - cur; best_off = cur; }
+        cur = std::max(cur, iv.second);
+      }
+      if (best_off == SIZE_MAX) best_off = cur;  // after the last overlapping tensor (may extend the arena)
+      R.arena_off = best_off;
+      top = std::max(top, best_off + need);
+      placed.push_back({best_off, need, R.def_step, R.last_step});
+    };
+    std::vector<char> done(p.roots.size(), 0);
+    // 1. live set at the peak, in (def step, id) order
+    std::vector<int> at_peak;
+    for (int t : ids) if (p.roots[t].def_step <= peak && p.roots[t].last_step >= peak) at_peak.push_back(t);
+    std::sort(at_peak.begin(), at_peak.end(), [&](int x, int y) { return std::make_pair(p.roots[x].def_step, x) < std::make_pair(p.roots[y].def_step, y); });
+    for (int t : at_peak) { place(t); done[t] = 1; }
+    // 2. forward from the peak
+    std::vector<int> fwd;
+    for (int t : ids) if (!done[t] && p.roots[t].def_step > peak) fwd.push_back(t);
+    std::sort(fwd.begin(), fwd.end(), [&](int x, int y) { return std::make_pair(p.roots[x].def_step, x) < std::make_pair(p.roots[y].def_step, y); });
+    for (int t : fwd) { place(t); done[t] = 1; }
+    // 3. backward from the peak: tensors dead before it, latest last-use first
+    std::vector<int> bwd;
+    for (int t : ids) if (!done[t]) bwd.push_back(t);
+    std::sort(bwd.begin(), bwd.end(), [&](int x, int y) { return std::make_pair(-p.roots[x].last_step, x) < std::make_pair(-p.roots[y].last_step, y); });
+    for (int t : bwd) { place(t); done[t] = 1; }
+    p.arena_bytes = top;
+    return OK;
+  }
+};
+
+}  // namespace
+
+Status make_plan(const Compiled* c, const Binding* b, Plan* p) {
+  p->c = c;
+  p->b = b;
+  p->n_req = b->n_req;
+  Planner pl(*c, *b, *p);
+  Status s = pl.run();
+  if (s != OK) return s;
+  return build_launches(p);
+}
+
+}  // namespace sod2

@@ -1,0 +1,165 @@
+"""GPU parity: the CUDA path through the C ABI against the CPU oracle, element by element."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import interp as O
+from paper_2403_00176_b200 import binding as B
+from paper_2403_00176_b200 import workloads as WL
+from paper_2403_00176_b200.workloads import Request, bf16_round
+from tests.gpu_harness import lockstep, run_batch
+
+pytestmark = pytest.mark.gpu
+
+F32_TOL = 1e-5     # the benchmark spec: 1e-5 relative for fp32
+BF16_TOL = 2e-2    # 2e-2 max relative error for bf16 tensor-core paths
+
+
+def _oracle_out(wl, req, name):
+    return O.run(wl.ir, wl.consts, req.inputs)[name]
+
+
+def test_cfg1_fused_group_fp32_all_requests():
+    wl = WL.cfg1()
+    reqs = wl.batch(0)
+    # add the edge sizes: N = 1 (two rows) and N = 64
+    rng = np.random.default_rng(3)
+    for n in (1, 64, 33):
+        reqs.append(Request({"N": n}, {"X": (rng.standard_normal((2, n, 64)) / 8).astype(np.float32)}))
+    s, p, outs = run_batch(wl, reqs)
+    assert s.graph.num_groups() == 1 and s.graph.group_info(0)["n_ops"] == 5
+    worst = 0.0
+    for r, req in enumerate(reqs):
+        ref = _oracle_out(wl, req, "Y")
+        assert outs[r]["Y"].shape == ref.shape == (2, req.syms["N"], 64)
+        worst = max(worst, O.rel_err(outs[r]["Y"], ref))
+    assert worst <= F32_TOL, worst
+    # determinism: a second run is bit-identical
+    p.run()
+    outs2 = p.outputs()
+    for a, b in zip(outs, outs2):
+        assert np.array_equal(a["Y"], b["Y"])
+
+
+def test_fig4_chain_one_fused_version():
+    for dt, tol in (("f32", F32_TOL), ("bf16", BF16_TOL)):
+        wl = WL.fig4_chain(dt)
+        reqs = wl.batch(0)
+        s, p, outs = run_batch(wl, reqs)
+        assert s.graph.num_groups() == 1 and s.graph.group_info(0)["versions"] == 1
+        for r, req in enumerate(reqs):
+            assert O.rel_err(outs[r]["C"], _oracle_out(wl, req, "C")) <= tol
+
+
+EDGE_L = [1, 15, 16, 17, 63, 64, 65, 127, 128, 129, 200]
+
+
+def _encoder_edge(layers=2):
+    wl = WL.cfg2(layers=layers, D=128, H=2, F=256, n_requests=1, lmin=1, lmax=512)
+    rng = np.random.default_rng(11)
+    reqs = [Request({"L": L}, {"x": bf16_round(rng.standard_normal((1, L, 128)).astype(np.float32))}) for L in EDGE_L]
+    return wl, reqs
+
+
+def test_cfg2_small_encoder_edge_lengths_lockstep():
+    wl, reqs = _encoder_edge()
+    s, p, outs = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE)
+    for r, req in enumerate(reqs):
+        ref = _oracle_out(wl, req, "y")
+        assert outs[r]["y"].shape == ref.shape
+        assert O.rel_err(outs[r]["y"], ref) <= BF16_TOL
+        errs = lockstep(wl, s, p, outs, r, BF16_TOL)
+        assert errs, "no materialised tensor was compared"
+        bad = {k: v for k, v in errs.items() if not (isinstance(v, float) and v <= BF16_TOL)}
+        assert not bad, (req.syms, bad)
+
+
+def test_cfg2_small_encoder_arena_reuse_matches_no_reuse():
+    wl, reqs = _encoder_edge()
+    _, p1, o1 = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE)
+    _, p2, o2 = run_batch(wl, reqs)
+    assert p2.plan.arena_bytes < p1.plan.arena_bytes
+    for a, b in zip(o1, o2):
+        assert np.array_equal(a["y"], b["y"])
+
+
+def test_cfg2_full_config_batch0():
+    wl = WL.cfg2()
+    reqs = wl.batch(0)
+    s, p, outs = run_batch(wl, reqs)
+    order = np.argsort([r.syms["L"] for r in reqs])
+    worst = 0.0
+    for r in (order[0], order[len(order) // 2], order[-1]):    # shortest, median, longest request
+        ref = _oracle_out(wl, reqs[r], "y")
+        worst = max(worst, O.rel_err(outs[r]["y"], ref))
+    assert worst <= BF16_TOL, worst
+    # properties that hold at any size: LayerNorm output rows have mean ~0 and unit mean-square
+    for r in range(len(reqs)):
+        y = outs[r]["y"][0].astype(np.float64)
+        assert np.all(np.isfinite(y))
+        assert np.max(np.abs(y.mean(-1))) < 2e-2
+        assert np.max(np.abs((y * y).mean(-1) - 1.0)) < 5e-2
+
+
+def _check_topk_lockstep(wl, reqs, layers):
+    s, p, outs = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE)
+    banded = 0
+    for r, req in enumerate(reqs):
+        errs = lockstep(wl, s, p, outs, r, BF16_TOL)
+        for name, v in errs.items():
+            if isinstance(v, tuple):     # index mismatch: only acceptable inside the score band
+                _, got, ref = v
+                l = int(name[3:])
+                y = p.read_arena_tensor(f"y{l}", r).astype(np.float64)[0]
+                sc = np.sort((y * y).sum(-1))[::-1]
+                k = ref.shape[-1]
+                assert k < sc.size and abs(sc[k - 1] - sc[k]) <= 2.0 ** -40 * sc[k - 1], (req.syms, name)
+                banded += 1
+            else:
+                assert v <= BF16_TOL, (req.syms, name, v)
+        n = req.syms["N0"]
+        for l in range(layers):
+            n = (7 * n + 9) // 10
+            assert outs[r][f"idx{l}"].shape == (1, n)
+            idx = outs[r][f"idx{l}"][0]
+            assert np.all(np.diff(idx) > 0)          # stable index order, no duplicates
+    assert banded <= max(1, len(reqs) * layers // 1000)
+    return s, p, outs
+
+
+def test_cfg3_small_pruning_lockstep_and_ties():
+    wl = WL.cfg3(layers=3, D=128, H=2, F=256, n_requests=1, nmin=4, nmax=800)
+    rng = np.random.default_rng(5)
+    reqs = []
+    for n0 in (4, 5, 10, 63, 64, 65, 196, 343, 784):
+        x = bf16_round(rng.standard_normal((1, n0, 128)).astype(np.float32))
+        reqs.append(Request({"N0": n0}, {"x": x}))
+    # exact ties: duplicated token rows must keep the lower index
+    x = bf16_round(rng.standard_normal((1, 40, 128)).astype(np.float32))
+    x[0, 20:40] = x[0, 0:20]
+    reqs.append(Request({"N0": 40}, {"x": x}))
+    _check_topk_lockstep(wl, reqs, 3)
+
+
+def test_cfg3_full_config_batch0_lockstep():
+    wl = WL.cfg3()
+    reqs = wl.batch(0)[:4]
+    _check_topk_lockstep(wl, reqs, 12)
+
+
+def test_nonzero_compaction():
+    wl = WL.nonzero_graph()
+    reqs = wl.batch(0)
+    rng = np.random.default_rng(9)
+    reqs.append(Request({"R": 3, "C": 5}, {"x": np.zeros((3, 5), np.float32)}))          # all zero
+    reqs.append(Request({"R": 7, "C": 300}, {"x": np.ones((7, 300), np.float32)}))       # all non-zero
+    big = rng.standard_normal((700, 900)).astype(np.float32)
+    big[rng.uniform(size=big.shape) < 0.7] = 0
+    reqs.append(Request({"R": 700, "C": 900}, {"x": big}))
+    s, p, outs = run_batch(wl, reqs)
+    for r, req in enumerate(reqs):
+        ref = O.run(wl.ir, wl.consts, req.inputs)["nz"] if req.inputs["x"].size < 5000 else np.array(np.nonzero(req.inputs["x"]))
+        assert outs[r]["nz"].shape == ref.shape
+        assert np.array_equal(outs[r]["nz"], ref)
