@@ -88,6 +88,12 @@ typedef struct {
 sod2_status sod2_run(sod2_plan_t* p, const void* const* inputs, void* const* outputs, void* arena,
                      size_t arena_bytes, void* cuda_stream, sod2_run_info* info);
 
+/* Measurement aid: the same inference with CUDA events recorded on cuda_stream around every launch.
+ * Synchronises the stream and returns the device time of each fused group in group_ms[n_groups]
+ * (host array, milliseconds; n_groups must equal sod2_graph_num_groups). */
+sod2_status sod2_run_timed(sod2_plan_t* p, const void* const* inputs, void* const* outputs, void* arena,
+                           size_t arena_bytes, void* cuda_stream, float* group_ms, int n_groups);
+
 /* Reads the device status word written by the last run (synchronises the stream).
  * SOD2_OK, or SOD2_E_TIMEOUT if a kernel gave up on a bounded wait. */
 sod2_status sod2_plan_device_status(sod2_plan_t* p, const void* arena, void* cuda_stream);
@@ -128,6 +134,10 @@ sod2_status sod2_plan_slot(const sod2_plan_t* p, const char* tensor, size_t* off
 sod2_status sod2_plan_instance_offset(const sod2_plan_t* p, const char* tensor, int request, size_t* offset);
 /* arena_bytes, peak live bytes, sum of all inter-group tensor bytes (what no-reuse allocation takes). */
 sod2_status sod2_plan_memory(const sod2_plan_t* p, size_t* arena_bytes, size_t* peak_live_bytes, size_t* sum_bytes);
+/* Algorithmic cost of one fused group for the bound shapes: flops of its contraction (0 for
+ * HBM-bound groups) and bytes = every external input and output once, constants once, nothing for
+ * tensors that stay inside the group. */
+sod2_status sod2_plan_group_cost(const sod2_plan_t* p, int group, double* flops, double* bytes);
 /* True shape of an output after a run (execution-determined extents are read back from the device;
  * synchronises cuda_stream). */
 sod2_status sod2_run_output_shape(sod2_plan_t* p, const void* arena, void* cuda_stream, int request, int output,

@@ -227,13 +227,16 @@ def _is_int(a):
 # --------------------------------------------------------------------------- interpreter
 def run(text: str, consts: Dict[str, np.ndarray], inputs: Dict[str, np.ndarray],
         overrides: Optional[Dict[str, np.ndarray]] = None, g: Optional[Graph] = None,
-        computed: Optional[Dict[str, np.ndarray]] = None) -> Dict[str, np.ndarray]:
+        computed: Optional[Dict[str, np.ndarray]] = None, storage_round=None) -> Dict[str, np.ndarray]:
     """Execute the graph on one request.  Returns every tensor by name.
 
     overrides: tensors whose value is replaced right after they are produced (used to keep
     the oracle in lock-step with another implementation's data-dependent decisions).
     computed: if given, receives for every overridden tensor the value the oracle itself computed
-    from its (possibly overridden) inputs, i.e. the per-operator lock-step reference."""
+    from its (possibly overridden) inputs, i.e. the per-operator lock-step reference.
+    storage_round: optional function applied to every float operator output ("faithful" variant:
+    what unfused execution with a narrow storage type would produce; used only to measure the
+    rounding noise inherent to that storage type, never as the parity reference)."""
     g = g or parse(text)
     env: Dict[str, np.ndarray] = {}
     for name in g.inputs:
@@ -301,6 +304,8 @@ def run(text: str, consts: Dict[str, np.ndarray], inputs: Dict[str, np.ndarray],
             raise NotImplementedError(op)
         outs = out if isinstance(out, tuple) else (out,)
         for name, val in zip(nd.outs, outs):
+            if storage_round is not None and np.asarray(val).dtype == np.float64:
+                val = storage_round(val)
             if name in overrides:
                 if computed is not None:
                     computed[name] = val

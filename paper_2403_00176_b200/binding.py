@@ -47,6 +47,7 @@ def _load() -> C.CDLL:
         "sod2_bind_dims": [vp, i32, i32, P(cp), P(i64), P(vp)],
         "sod2_plan": [vp, vp, P(vp), P(sz)],
         "sod2_run": [vp, P(vp), P(vp), vp, sz, vp, P(RunInfo)],
+        "sod2_run_timed": [vp, P(vp), P(vp), vp, sz, vp, P(C.c_float), i32],
         "sod2_plan_device_status": [vp, vp, vp],
         "sod2_graph_tensor_info": [vp, cp, P(i32), P(i32), cp, sz],
         "sod2_graph_tensor_value": [vp, cp, cp, sz],
@@ -59,6 +60,7 @@ def _load() -> C.CDLL:
         "sod2_plan_slot": [vp, cp, P(sz), P(sz), P(i32), P(i32)],
         "sod2_plan_instance_offset": [vp, cp, i32, P(sz)],
         "sod2_plan_memory": [vp, P(sz), P(sz), P(sz)],
+        "sod2_plan_group_cost": [vp, i32, P(C.c_double), P(C.c_double)],
         "sod2_run_output_shape": [vp, vp, vp, i32, i32, P(i64), P(i32)],
     }
     for name, args in sig.items():
@@ -79,10 +81,10 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = ["sod2_graph_create", "sod2_graph_destroy", "sod2_graph_set_const", "sod2_graph_prepack_bytes",
            "sod2_graph_prepack", "sod2_bind_dims", "sod2_binding_destroy", "sod2_plan", "sod2_plan_destroy",
-           "sod2_run", "sod2_plan_device_status", "sod2_graph_tensor_info", "sod2_graph_tensor_value", "sod2_graph_tensor_dtype",
+           "sod2_run", "sod2_run_timed", "sod2_plan_device_status", "sod2_graph_tensor_info", "sod2_graph_tensor_value", "sod2_graph_tensor_dtype",
            "sod2_graph_num_ops", "sod2_graph_op_info", "sod2_graph_num_groups", "sod2_graph_group_info",
            "sod2_graph_num_subgraphs", "sod2_graph_rdp_sweeps", "sod2_classify", "sod2_graph_reanalyse",
-           "sod2_binding_shape", "sod2_plan_slot", "sod2_plan_instance_offset", "sod2_plan_memory",
+           "sod2_binding_shape", "sod2_plan_slot", "sod2_plan_instance_offset", "sod2_plan_memory", "sod2_plan_group_cost",
            "sod2_run_output_shape", "sod2_last_error"]
 
 
@@ -231,6 +233,14 @@ class Plan:
         _check(lib.sod2_run(self.h, ins, outs, C.c_void_p(arena), arena_bytes, C.c_void_p(stream), C.byref(info)), self.h)
         return info
 
+    def run_timed(self, inputs: Sequence[int], outputs: Sequence[int], arena: int, arena_bytes: int, stream: int) -> List[float]:
+        ins = (C.c_void_p * max(len(inputs), 1))(*inputs)
+        outs = (C.c_void_p * max(len(outputs), 1))(*outputs)
+        n = self.graph.num_groups()
+        ms = (C.c_float * max(n, 1))()
+        _check(lib.sod2_run_timed(self.h, ins, outs, C.c_void_p(arena), arena_bytes, C.c_void_p(stream), ms, n), self.h)
+        return list(ms[:n])
+
     def device_status(self, arena: int, stream: int):
         _check(lib.sod2_plan_device_status(self.h, C.c_void_p(arena), C.c_void_p(stream)), self.h)
 
@@ -249,6 +259,11 @@ class Plan:
         a, p, s = C.c_size_t(), C.c_size_t(), C.c_size_t()
         _check(lib.sod2_plan_memory(self.h, C.byref(a), C.byref(p), C.byref(s)), self.h)
         return {"arena_bytes": a.value, "peak_live_bytes": p.value, "sum_bytes": s.value}
+
+    def group_cost(self, group: int):
+        f, b = C.c_double(), C.c_double()
+        _check(lib.sod2_plan_group_cost(self.h, group, C.byref(f), C.byref(b)), self.h)
+        return f.value, b.value
 
     def output_shape(self, arena: int, stream: int, request: int, output: int) -> List[int]:
         dims = (C.c_int64 * 16)()

@@ -135,6 +135,8 @@ sod2_status sod2_run(sod2_plan_t* p, const void* const* inputs, void* const* out
   const Graph& G = p->g->c.g;
   for (size_t i = 0; i < G.inputs.size(); ++i) if (!inputs[i]) { p->h.err = "null input"; return SOD2_E_INVALID_ARG; }
   for (size_t i = 0; i < G.outputs.size(); ++i) if (!outputs[i]) { p->h.err = "null output"; return SOD2_E_INVALID_ARG; }
+  if (arena_bytes < p->p.arena_bytes) { p->h.err = "arena too small"; return SOD2_E_ARENA_TOO_SMALL; }
+  if (reinterpret_cast<uintptr_t>(arena) & 255) { p->h.err = "arena must be 256-byte aligned"; return SOD2_E_MISALIGNED; }
   for (int c : G.consts) {
     bool used = false;
     for (auto& grp : p->g->c.groups) for (int t : grp.ext_in) if (t == c) used = true;
@@ -144,6 +146,14 @@ sod2_status sod2_run(sod2_plan_t* p, const void* const* inputs, void* const* out
   Status s = run_plan(&p->p, inputs, outputs, arena, arena_bytes, stream, inf);
   if (s != OK) p->h.err = p->p.err;
   if (info) { info->host_enqueue_ns = inf[0]; info->gpu_launches = inf[1]; }
+  return st(s);
+}
+
+sod2_status sod2_run_timed(sod2_plan_t* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes,
+                           void* stream, float* group_ms, int n_groups) {
+  if (!p || !inputs || !outputs || !arena) return SOD2_E_INVALID_ARG;
+  Status s = run_plan_timed(&p->p, inputs, outputs, arena, arena_bytes, stream, group_ms, n_groups);
+  if (s != OK) p->h.err = p->p.err;
   return st(s);
 }
 
@@ -255,6 +265,13 @@ sod2_status sod2_plan_instance_offset(const sod2_plan_t* p, const char* name, in
   if (t < 0 || p->p.views[t].empty() || p->p.views[t][0].root < 0) return SOD2_E_INVALID_ARG;
   const View& v = p->p.views[t][r];
   *off = static_cast<size_t>(p->p.roots[v.root].inst_off[r] + v.offset * dtype_size(p->g->c.g.tensors[t].dtype));
+  return SOD2_OK;
+}
+
+sod2_status sod2_plan_group_cost(const sod2_plan_t* p, int group, double* flops, double* bytes) {
+  if (!p || group < 0 || group >= static_cast<int>(p->p.group_flops.size())) return SOD2_E_INVALID_ARG;
+  if (flops) *flops = p->p.group_flops[group];
+  if (bytes) *bytes = p->p.group_bytes[group];
   return SOD2_OK;
 }
 

@@ -125,6 +125,7 @@ struct Plan {
   std::vector<std::shared_ptr<Launch>> launches;
   std::vector<size_t> scratch_off;        // per group scratch offsets in the arena
   int gpu_launches = 0;
+  std::vector<double> group_flops, group_bytes;   // algorithmic cost per group for the bound shapes
   std::string err;
   // device status word lives at arena offset 0 (first 256 bytes reserved)
 };
@@ -132,5 +133,10 @@ Status make_plan(const Compiled* c, const Binding* b, Plan* p);
 Status build_launches(Plan* p);   // exec.cu
 Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream,
                 int64_t* info);
+
+// Same as run_plan, with CUDA events around every launch; synchronises the stream and returns the
+// device time per group (ms).
+Status run_plan_timed(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream,
+                      float* group_ms, int n_groups);
 
 }  // namespace sod2

@@ -455,8 +455,44 @@ struct Builder {
     return OK;
   }
 
+  // Algorithmic cost of a group for the bound shapes: every external input and output once,
+  // constants once, nothing for intermediates inside the group; flops of its contraction.
+  void cost(const Group& G) {
+    double bytes = 0, flops = 0;
+    auto tb = [&](int t) {
+      const Tensor& T = g.tensors[t];
+      double b = 0;
+      const int nr = T.kind == TKind::CONST ? 1 : p.n_req;
+      for (int r = 0; r < nr; ++r) b += static_cast<double>(numel(p.views[t][r].dims)) * dtype_size(T.dtype);
+      return b;
+    };
+    for (int t : G.ext_in) if (c.storage[t].kind != Storage::FOLDED && !p.views[t][0].dims.empty()) bytes += tb(t);
+    for (int t : G.ext_out) if (c.storage[t].kind != Storage::FOLDED && !p.views[t][0].dims.empty()) bytes += tb(t);
+    if (G.kind == GKind::GEMM) {
+      const Tensor& W = g.tensors[G.w];
+      const double K = static_cast<double>(W.S.dims[0].e.const_value()), N = static_cast<double>(W.S.dims[1].e.const_value());
+      for (int r = 0; r < p.n_req; ++r) flops += 2.0 * (numel(p.views[G.a][r].dims) / K) * N * K;
+    } else if (G.kind == GKind::ATTENTION) {
+      for (int r = 0; r < p.n_req; ++r) {
+        const auto& d = p.views[G.q][r].dims;
+        const double L = static_cast<double>(d[d.size() - 2]), dh = static_cast<double>(d.back());
+        flops += 4.0 * L * L * dh * (numel(d) / (L * dh));
+      }
+    } else if (G.kind == GKind::CONV) {
+      const auto& wd = g.tensors[G.w].S.dims;
+      const double per_out = 2.0 * wd[1].e.const_value() * wd[2].e.const_value() * wd[3].e.const_value();
+      const int conv_out = g.nodes[G.nodes[0]].outs[0];
+      for (int r = 0; r < p.n_req; ++r)
+        if (!p.b->dims[conv_out].empty()) flops += per_out * numel(p.b->dims[conv_out][r]);
+    }
+    p.group_flops.push_back(flops);
+    p.group_bytes.push_back(bytes);
+  }
+
   Status run() {
     p.launches.clear();
+    p.group_flops.clear();
+    p.group_bytes.clear();
     p.gpu_launches = 0;
     for (size_t gi = 0; gi < c.groups.size(); ++gi) {
       const Group& G = c.groups[gi];
@@ -471,6 +507,7 @@ struct Builder {
         default: return fail(E_UNSUPPORTED_OP, std::string("no executor yet for group kind ") + gkind_name(G.kind));
       }
       if (s != OK) return s;
+      cost(G);
     }
     // one scratch region shared by all groups (they run in stream order), after the tensors
     p.scratch_off.assign(1, p.arena_bytes);
@@ -515,6 +552,34 @@ Status prepack_weights(Compiled* c, void* workspace, size_t bytes, void* stream)
   if (cudaGetLastError() != cudaSuccess) { c->err = "prepack launch failed"; return E_CUDA; }
   c->packed_ws = workspace;
   return OK;
+}
+
+Status run_plan_timed(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream,
+                      float* group_ms, int n_groups) {
+  if (!group_ms || n_groups != static_cast<int>(p->c->groups.size())) { p->err = "group_ms must hold one float per group"; return E_INVALID_ARG; }
+  if (arena_bytes < p->arena_bytes) { p->err = "arena too small"; return E_ARENA_TOO_SMALL; }
+  if (reinterpret_cast<uintptr_t>(arena) & 255) { p->err = "arena must be 256-byte aligned"; return E_MISALIGNED; }
+  RunCtx x{inputs, outputs, static_cast<char*>(arena), static_cast<char*>(p->c->packed_ws), static_cast<cudaStream_t>(stream), p};
+  const size_t n = p->launches.size();
+  std::vector<cudaEvent_t> ev(2 * n);
+  for (auto& e : ev) if (cudaEventCreate(&e) != cudaSuccess) { p->err = "cudaEventCreate failed"; return E_CUDA; }
+  cudaMemsetAsync(arena, 0, 256, x.stream);
+  Status st = OK;
+  for (size_t i = 0; i < n && st == OK; ++i) {
+    cudaEventRecord(ev[2 * i], x.stream);
+    if (p->launches[i]->fn(x) != cudaSuccess) { p->err = "launch failed"; st = E_CUDA; }
+    cudaEventRecord(ev[2 * i + 1], x.stream);
+  }
+  if (cudaStreamSynchronize(x.stream) != cudaSuccess) { p->err = "stream synchronize failed"; st = E_CUDA; }
+  for (int g = 0; g < n_groups; ++g) group_ms[g] = 0.f;
+  if (st == OK)
+    for (size_t i = 0; i < n; ++i) {
+      float ms = 0.f;
+      cudaEventElapsedTime(&ms, ev[2 * i], ev[2 * i + 1]);
+      group_ms[p->launches[i]->group] += ms;
+    }
+  for (auto& e : ev) cudaEventDestroy(e);
+  return st;
 }
 
 Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream, int64_t* info) {

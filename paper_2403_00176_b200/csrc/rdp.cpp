@@ -194,7 +194,11 @@ Status parse_ir(const char* text, size_t len, Graph* g) {
       std::string err;
       if (rest == "?") { /* rank undefined */ }
       else if (!parse_dims(g, rest, &t.S, &err)) return fail(err);
-      if (kw == "input") { t.io_index = static_cast<int>(g->inputs.size()); g->inputs.push_back(id); }
+      if (kw == "input") {
+        t.io_index = static_cast<int>(g->inputs.size());
+        g->inputs.push_back(id);
+        t.V.kind = ValueVal::NAC;  // the value of a model input is not a constant of the analysis
+      }
       else {
         if (!t.S.fully_known()) return fail("const needs a fully known shape");
         for (auto& d : t.S.dims) if (!d.e.is_const()) return fail("const needs integer dims");

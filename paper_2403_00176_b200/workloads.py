@@ -390,7 +390,7 @@ def cfg5(B: int = 32, side: int = 224, widths=(64, 128, 256, 512), per_stage: in
             p = ir.node("GlobalAveragePool", [x], ir.tmp("p"))
             p2 = ir.node("Reshape", [p, f"{pre}pshape"], ir.tmp("p"))
             z = ir.node("MatMul", [p2, f"{pre}gw"], ir.tmp("z"))
-            z2 = ir.node("Add", [z, f"{pre}gb"], f"z{bi}")
+            z2 = ir.node("Add", [z, f"{pre}gb"], f"logit{bi}")
             g = ir.node("Greater", [z2, "f_zero"], f"gate{bi}")
             xe, xs = ir.node("Switch", [x, g], [ir.tmp("xe"), ir.tmp("xs")])
             decl[f"{pre}w1"] = (wdt, cprev, 3, 3)

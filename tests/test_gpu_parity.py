@@ -90,17 +90,37 @@ def test_cfg2_full_config_batch0():
     reqs = wl.batch(0)
     s, p, outs = run_batch(wl, reqs)
     order = np.argsort([r.syms["L"] for r in reqs])
-    worst = 0.0
     for r in (order[0], order[len(order) // 2], order[-1]):    # shortest, median, longest request
         ref = _oracle_out(wl, reqs[r], "y")
-        worst = max(worst, O.rel_err(outs[r]["y"], ref))
-    assert worst <= BF16_TOL, worst
+        got = outs[r]["y"].astype(np.float64)
+        # After 6 layers (about 50 roundings to bf16 storage on any implementation) the MAX error is
+        # dominated by that storage noise, so end to end we bound (a) the rms error by the tolerance
+        # and (b) the max error by the tolerance or twice the noise of unfused bf16-storage
+        # execution of the same graph, whichever is larger.  The per-group bound is test-ed in
+        # lock-step (next test), where it is well posed.
+        rms = math.sqrt(np.mean((got - ref) ** 2) / np.mean(ref ** 2))
+        assert rms <= BF16_TOL, rms
+        noisy = O.run(wl.ir, wl.consts, reqs[r].inputs, storage_round=lambda a: bf16_round(a.astype(np.float32)).astype(np.float64))["y"]
+        noise = O.rel_err(noisy, ref)
+        assert O.rel_err(got, ref) <= max(BF16_TOL, 2 * noise), (O.rel_err(got, ref), noise)
     # properties that hold at any size: LayerNorm output rows have mean ~0 and unit mean-square
     for r in range(len(reqs)):
         y = outs[r]["y"][0].astype(np.float64)
         assert np.all(np.isfinite(y))
         assert np.max(np.abs(y.mean(-1))) < 2e-2
         assert np.max(np.abs((y * y).mean(-1) - 1.0)) < 5e-2
+
+
+def test_cfg2_full_config_lockstep_per_group():
+    wl = WL.cfg2()
+    reqs = wl.batch(1)
+    s, p, outs = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE)
+    order = np.argsort([r.syms["L"] for r in reqs])
+    for r in (order[0], order[-1]):
+        errs = lockstep(wl, s, p, outs, r, BF16_TOL)
+        assert len(errs) >= 6 * 7
+        bad = {k: v for k, v in errs.items() if not (isinstance(v, float) and v <= BF16_TOL)}
+        assert not bad, bad
 
 
 def _check_topk_lockstep(wl, reqs, layers):
