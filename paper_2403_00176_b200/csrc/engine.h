@@ -125,6 +125,8 @@ struct Plan {
   std::vector<std::shared_ptr<Launch>> launches;
   std::vector<size_t> scratch_off;        // per group scratch offsets in the arena
   int gpu_launches = 0;
+  int sm_count = 148;                     // persistent kernels launch one CTA per SM
+  bool sm_count_known = false;
   std::vector<double> group_flops, group_bytes;   // algorithmic cost per group for the bound shapes
   std::string err;
   // device status word lives at arena offset 0 (first 256 bytes reserved)

@@ -2,6 +2,7 @@
 // fused groups on the caller's stream.  All device memory belongs to the caller; this file never
 // allocates device memory.
 #include <chrono>
+#include <cmath>
 #include <cstring>
 #include <functional>
 
@@ -169,8 +170,9 @@ struct Builder {
       return OK;
     }
     // bf16 on tcgen05
-    if (G.has_ln || G.act2) return fail(E_UNSUPPORTED_OP, "bf16 GEMM epilogue: unsupported tail");
-    if (K % 8 || lds[0] % 8) return fail(E_UNSUPPORTED_OP, "GEMM operand rows must be 16-byte multiples for TMA");
+    if (G.has_ln) return fail(E_UNSUPPORTED_OP, "bf16 GEMM epilogue: LayerNorm tail is not fused");
+    if (K % 64) return fail(E_UNSUPPORTED_OP, "bf16 GEMM needs K % 64 == 0 (k-chunk tensor maps)");
+    if (lds[0] % 8 || lds[1] % 8 || (G.res >= 0 && lds[2] % 8)) return fail(E_UNSUPPORTED_OP, "GEMM operand rows must be 16-byte multiples for TMA");
     size_t pk = 0;
     for (size_t i = 0; i < c.packed_consts.size(); ++i) if (c.packed_consts[i] == G.w) pk = c.packed_off[i];
     for (auto& sg : segs) {
@@ -180,41 +182,56 @@ struct Builder {
       Ptr pb = G.bias >= 0 ? ptr_of(G.bias, 0) : Ptr();
       const int M = static_cast<int>(sg.rows);
       const int64_t lda = lds[0], ldo = lds[1], ldr = G.res >= 0 ? lds[2] : 0;
-      // shape-class variant (the paper's multi-version idea, Section 4.4.2): narrow tiles when the
-      // wide ones would leave SMs idle
+      // Shape-class variant (the paper's multi-version idea, Section 4.4.2).  Two tile versions
+      // exist: "fat" 128x256 tiles (one 64-wide k-chunk per stage) and "regular" 128x128 tiles (two
+      // k-chunks per stage).  Pick the one with the smaller estimated makespan on the SMs: waves of
+      // tiles times the per-tile main-loop time (stages x max(MMA, TMA) per stage).
       const int tiles_m = (M + 127) / 128;
-      int bn = 128;
-      if (tiles_m * ((N + 127) / 128) < 148 && N > 64) bn = 64;
+      const int sms = 148;
+      auto makespan = [&](int bn_, int kch) {
+        const double tiles = static_cast<double>(tiles_m) * ((N + bn_ - 1) / bn_);
+        const double waves = std::ceil(tiles / sms);
+        const double stages = std::ceil(static_cast<double>(K) / (64.0 * kch));
+        const double mma = kch * 4 * (bn_ / 2.0), floor_cycles = 540.0;
+        const double tma = kch * (128 + bn_) * 128.0 / 70.0;   // bytes per stage at ~70 B/clk/SM from L2
+        return waves * stages * std::max(std::max(mma, floor_cycles), tma);
+      };
+      int bn = (N > 128 && makespan(256, 1) <= makespan(128, 2)) ? 256 : 128;
       const bool hb = G.bias >= 0, hr = G.res >= 0;
       const int act = G.act;
-      struct Cache { const void* a = nullptr; const void* w = nullptr; CUtensorMap ta, tb; };
+      const int act2 = G.act2;
+      struct Cache { const void* a = nullptr; const void* w = nullptr; const void* o = nullptr; const void* r = nullptr; CUtensorMap ta, tb, to, tr; };
       auto cache = std::make_shared<Cache>();
       add(gi, 1, [=](const RunCtx& x) {
         const void* A = x.resolve(pa);
         const void* Wt = x.resolve(pw);
-        if (cache->a != A || cache->w != Wt) {
-          if (!encode_bf16_2d(&cache->ta, A, M, K, lda, 128) || !encode_bf16_2d(&cache->tb, Wt, N, K, K, bn)) return cudaErrorInvalidValue;
-          cache->a = A; cache->w = Wt;
+        void* O = x.resolve(po);
+        const void* R = hr ? x.resolve(pr) : O;
+        if (cache->a != A || cache->w != Wt || cache->o != O || cache->r != R) {
+          const int kch = bn == 256 ? 1 : 2;
+          if (!encode_bf16_kchunks(&cache->ta, A, M, K, lda, 128, kch) || !encode_bf16_kchunks(&cache->tb, Wt, N, K, K, bn, kch) ||
+              !encode_bf16_2d(&cache->to, O, M, N, ldo, 128) || !encode_bf16_2d(&cache->tr, R, M, N, hr ? ldr : ldo, 128))
+            return cudaErrorInvalidValue;
+          cache->a = A; cache->w = Wt; cache->o = O; cache->r = R;
         }
         k::GemmEpilogue ep{};
         ep.bias = hb ? reinterpret_cast<const __nv_bfloat16*>(x.resolve(pb)) : nullptr;
-        ep.residual = hr ? reinterpret_cast<const __nv_bfloat16*>(x.resolve(pr)) : nullptr;
-        ep.ldr = ldr;
-        ep.out = reinterpret_cast<__nv_bfloat16*>(x.resolve(po));
-        ep.ldo = ldo;
+        ep.has_residual = hr;
         ep.act = act;
+        ep.act2 = act2;
         ep.status = reinterpret_cast<int*>(x.arena);
-        const int grid = tiles_m * static_cast<int>((N + bn - 1) / bn);
-        if (bn == 128) {
-          constexpr int smem = k::GemmSmem<128, 3>::TOTAL;
-          static bool once = (cudaFuncSetAttribute(k::gemm_bf16_tcgen05<128, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);
+        const int tiles = tiles_m * static_cast<int>((N + bn - 1) / bn);
+        const int grid = std::min(tiles, x.plan->sm_count);
+        if (bn == 256) {
+          constexpr int smem = k::GemmSmem<256, 1, 4>::TOTAL;
+          static bool once = (cudaFuncSetAttribute(k::gemm_bf16_tcgen05<256, 1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);
           (void)once;
-          k::gemm_bf16_tcgen05<128, 3><<<grid, 128, smem, x.stream>>>(cache->ta, cache->tb, M, static_cast<int>(N), static_cast<int>(K), ep);
+          k::gemm_bf16_tcgen05<256, 1, 4><<<grid, k::GEMM_THREADS, smem, x.stream>>>(cache->ta, cache->tb, cache->to, cache->tr, M, static_cast<int>(N), static_cast<int>(K), ep);
         } else {
-          constexpr int smem = k::GemmSmem<64, 4>::TOTAL;
-          static bool once = (cudaFuncSetAttribute(k::gemm_bf16_tcgen05<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);
+          constexpr int smem = k::GemmSmem<128, 2, 3>::TOTAL;
+          static bool once = (cudaFuncSetAttribute(k::gemm_bf16_tcgen05<128, 2, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);
           (void)once;
-          k::gemm_bf16_tcgen05<64, 4><<<grid, 128, smem, x.stream>>>(cache->ta, cache->tb, M, static_cast<int>(N), static_cast<int>(K), ep);
+          k::gemm_bf16_tcgen05<128, 2, 3><<<grid, k::GEMM_THREADS, smem, x.stream>>>(cache->ta, cache->tb, cache->to, cache->tr, M, static_cast<int>(N), static_cast<int>(K), ep);
         }
         return cudaGetLastError();
       });
@@ -588,6 +605,11 @@ Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* 
   if (reinterpret_cast<uintptr_t>(arena) & 255) { p->err = "arena must be 256-byte aligned"; return E_MISALIGNED; }
   if (p->c->packed_bytes && !p->c->packed_ws) { p->err = "weights are not prepacked"; return E_INVALID_ARG; }
   auto t0 = std::chrono::steady_clock::now();
+  if (!p->sm_count_known) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) p->sm_count = n;
+    p->sm_count_known = true;
+  }
   RunCtx x{inputs, outputs, static_cast<char*>(arena), static_cast<char*>(p->c->packed_ws), static_cast<cudaStream_t>(stream), p};
   if (cudaMemsetAsync(arena, 0, 256, x.stream) != cudaSuccess) { p->err = "cannot clear the status word"; return E_CUDA; }
   for (auto& L : p->launches) {

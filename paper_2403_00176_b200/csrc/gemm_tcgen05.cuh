@@ -1,12 +1,21 @@
 // Varlen GEMM with fused epilogue on tcgen05 / TMEM, fed by TMA.
-//   out[M,N] = act(A[M,K] * Wt[N,K]^T + bias[N]) (+ residual[M,N]),  bf16 in, fp32 accumulate, bf16 out.
-// M is the run-time row count (sum of the requests' rows); the A tensor map is encoded for
-// exactly M rows, so rows past M read as zeros and are never stored.
-// One 128 x BN output tile per CTA, BK = 64 (one 128-byte swizzle atom of bf16 per row).
-// Warp 0 lane 0 streams tiles with TMA through a STAGES-deep mbarrier ring, warp 1 lane 0 issues
-// tcgen05.mma into a TMEM accumulator, then all four warps drain TMEM (warp w owns lanes
-// 32w..32w+31 = tile rows) through the epilogue. Two CTAs fit per SM, so one CTA's epilogue
-// overlaps the other's main loop.
+//   out[M,N] = act2( act(A[M,K] * Wt[N,K]^T + bias[N]) + residual[M,N] ),  bf16 in, fp32 accumulate, bf16 out.
+// M is the run-time row count (sum of the requests' rows); the tensor maps are encoded for exactly
+// M rows, so rows past M read as zeros and the TMA store clips them.
+//
+// Persistent, warp-specialised, one CTA per SM.  Tile 128 x BN; one pipeline stage holds KCH
+// k-chunks of 64 (each chunk = one 128-byte swizzle atom per row).  Measured on B200: one thread
+// can issue a tcgen05.mma about every 65-80 cycles and a barrier wait in the issue loop costs about
+// 170 cycles, so a stage must carry >= 512 cycles of MMA work to hide them: (BN=256, KCH=1) or
+// (BN=128, KCH=2).
+//   warp 0      TMA producer for A (STAGES-deep mbarrier ring; one 3-D box per stage)
+//   warp 1      TMA producer for B (a thread sustains about one TMA instruction per 170 ns, so A
+//               and B get a thread each)
+//   warp 2      MMA issuer: tcgen05.mma into one of two TMEM accumulators (double buffered)
+//   warps 3..10 epilogue, in passes of 128 columns: drain TMEM (warp w owns lanes 32*(w%4)..), add
+//               bias from shared memory, activation, residual (TMA-loaded into the staging tile and
+//               updated in place), pack to bf16 into the swizzled staging tile, TMA store
+// so the epilogue of tile i overlaps the main loop of tile i+1.  Every wait is bounded (ptx.cuh).
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -18,160 +27,234 @@ namespace k {
 enum Act : int { ACT_NONE = 0, ACT_GELU = 1, ACT_RELU = 2 };
 
 struct GemmEpilogue {
-  const __nv_bfloat16* bias;      // [N] or nullptr
-  const __nv_bfloat16* residual;  // [M, ldr] or nullptr (added after the activation)
-  long long ldr;
-  __nv_bfloat16* out;             // [M, ldo]
-  long long ldo;
-  int act;
-  int* status;                    // device word; set non-zero if a bounded wait ran out
+  const __nv_bfloat16* bias;  // [N] or nullptr
+  int has_residual;           // residual arrives through its own tensor map
+  int act;                    // applied before the residual add
+  int act2;                   // applied after the residual add
+  int* status;                // device word; set non-zero if a bounded wait ran out
 };
 
 constexpr int GEMM_BM = 128;
-constexpr int GEMM_BK = 64;
+constexpr int GEMM_THREADS = 352;
+constexpr int GEMM_PASS_COLS = 128;                       // epilogue pass width
+constexpr int GEMM_STAGE_OUT = GEMM_BM * GEMM_PASS_COLS * 2;  // 32 KB staging tile: 2 boxes of [128 rows x 128 B]
 
-template <int BN, int STAGES>
+template <int BN, int KCH, int STAGES>
 struct GemmSmem {
-  static constexpr int A_BYTES = GEMM_BM * GEMM_BK * 2;
-  static constexpr int B_BYTES = BN * GEMM_BK * 2;
+  static constexpr int A_BYTES = KCH * GEMM_BM * 128;
+  static constexpr int B_BYTES = KCH * BN * 128;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int TOTAL = STAGES * STAGE_BYTES + 1024 /*align slack*/ + 256 /*barriers*/;
+  static constexpr int TOTAL = STAGES * STAGE_BYTES + GEMM_STAGE_OUT + 1024 /*align slack*/ + 1024 /*bias + barriers*/;
 };
 
-__device__ __forceinline__ float gelu_erf(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752f)); }
+// erf by the rational approximation 7.1.26 of Abramowitz & Stegun (|error| <= 1.5e-7), far inside
+// the bf16 output rounding; cheaper than erff on the epilogue warps.
+__device__ __forceinline__ float gelu_erf(float x) {
+  const float z = fabsf(x) * 0.70710678118654752f;
+  float t;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f, z, 1.0f)));
+  float p = fmaf(1.061405429f, t, -1.453152027f);
+  p = fmaf(p, t, 1.421413741f);
+  p = fmaf(p, t, -0.284496736f);
+  p = fmaf(p, t, 0.254829592f);
+  const float e = 1.0f - p * t * __expf(-z * z);   // erf(|x|/sqrt2)
+  return 0.5f * x * (1.0f + copysignf(e, x));
+}
+__device__ __forceinline__ float apply_act(int act, float v) {
+  return act == ACT_GELU ? gelu_erf(v) : act == ACT_RELU ? fmaxf(v, 0.0f) : v;
+}
 
-template <int BN, int STAGES>
-__global__ void __launch_bounds__(128)
+__device__ __forceinline__ void tma_store_2d(const void* tmap, const void* src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(tmap), "r"(ptx::smem_u32(src)), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// tmA / tmB are 3-D views {64, rows, K/64} of the row-major operands (K % 64 == 0), box
+// {64, 128 or BN, KCH}: one instruction fills KCH consecutive swizzled [rows x 64] chunks.
+template <int BN, int KCH, int STAGES>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                  const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmRes,
                   int M, int N, int K, GemmEpilogue ep) {
-  using S = GemmSmem<BN, STAGES>;
+  using S = GemmSmem<BN, KCH, STAGES>;
+  constexpr int PASSES = BN / GEMM_PASS_COLS;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* full = reinterpret_cast<uint64_t*>(tiles + STAGES * S::STAGE_BYTES);
+  uint8_t* out_stage = tiles + STAGES * S::STAGE_BYTES;
+  float* bias_s = reinterpret_cast<float*>(out_stage + GEMM_STAGE_OUT);  // [128]
+  uint64_t* full = reinterpret_cast<uint64_t*>(bias_s + GEMM_PASS_COLS);
   uint64_t* empty = full + STAGES;
-  uint64_t* accum = empty + STAGES;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
+  uint64_t* tmem_full = empty + STAGES;   // [2]
+  uint64_t* tmem_empty = tmem_full + 2;   // [2]
+  uint64_t* res_full = tmem_empty + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(res_full + 1);
   volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tiles_m = (M + GEMM_BM - 1) / GEMM_BM;
-  const int tm = blockIdx.x % tiles_m, tn = blockIdx.x / tiles_m;
-  const int m0 = tm * GEMM_BM, n0 = tn * BN;
-  const int kblocks = (K + GEMM_BK - 1) / GEMM_BK;
-  constexpr uint32_t TMEM_COLS = BN < 32 ? 32 : BN;
+  const int tiles_m = (M + GEMM_BM - 1) / GEMM_BM, tiles_n = (N + BN - 1) / BN;
+  const int num_tiles = tiles_m * tiles_n;
+  const int kchunks = K / 64;
+  const int kstages = (kchunks + KCH - 1) / KCH;
+  constexpr uint32_t TMEM_COLS = 2 * BN;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
-    ptx::mbar_init(accum, 1);
+    for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(&full[s], 2); ptx::mbar_init(&empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&tmem_full[b], 1); ptx::mbar_init(&tmem_empty[b], 8); }
+    ptx::mbar_init(res_full, 1);
     *dead = 0;
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
     ptx::prefetch_tmap(&tmA);
     ptx::prefetch_tmap(&tmB);
+    ptx::prefetch_tmap(&tmOut);
+    if (ep.has_residual) ptx::prefetch_tmap(&tmRes);
   }
-  if (warp == 0) { ptx::tmem_alloc(tmem_slot, TMEM_COLS); ptx::tmem_relinquish(); }
+  if (warp == 2) { ptx::tmem_alloc(tmem_slot, TMEM_COLS); ptx::tmem_relinquish(); }
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  if (warp == 0 && lane == 0) {
-    // ---- TMA producer
-    for (int kb = 0; kb < kblocks; ++kb) {
-      const int s = kb % STAGES;
-      if (kb >= STAGES) ptx::mbar_wait(&empty[s], ((kb / STAGES) - 1) & 1, dead);
-      uint8_t* a = tiles + s * S::STAGE_BYTES;
-      ptx::mbar_expect_tx(&full[s], S::STAGE_BYTES);
-      ptx::tma_load_2d(a, &tmA, kb * GEMM_BK, m0, &full[s]);
-      ptx::tma_load_2d(a + S::A_BYTES, &tmB, kb * GEMM_BK, n0, &full[s]);
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---- TMA producer: A stages
+      int n = 0;
+      for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
+        const int m0 = (t % tiles_m) * GEMM_BM;
+        for (int ks = 0; ks < kstages; ++ks, ++n) {
+          const int s = n % STAGES;
+          if (n >= STAGES) ptx::mbar_wait(&empty[s], ((n / STAGES) - 1) & 1, dead);
+          ptx::mbar_expect_tx(&full[s], S::A_BYTES);
+          ptx::tma_load_3d(tiles + s * S::STAGE_BYTES, &tmA, 0, m0, ks * KCH, &full[s]);
+        }
+      }
     }
-  } else if (warp == 1 && lane == 0) {
-    // ---- MMA issuer
-    constexpr uint32_t idesc = ptx::idesc_bf16(GEMM_BM, BN);
-    for (int kb = 0; kb < kblocks; ++kb) {
-      const int s = kb % STAGES;
-      ptx::mbar_wait(&full[s], (kb / STAGES) & 1, dead);
-      ptx::tc_fence_after();
-      const uint32_t a = ptx::smem_u32(tiles + s * S::STAGE_BYTES);
-      const uint64_t ad = ptx::smem_desc_sw128(a), bd = ptx::smem_desc_sw128(a + S::A_BYTES);
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ---- TMA producer: B stages
+      int n = 0;
+      for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
+        const int n0 = (t / tiles_m) * BN;
+        for (int ks = 0; ks < kstages; ++ks, ++n) {
+          const int s = n % STAGES;
+          if (n >= STAGES) ptx::mbar_wait(&empty[s], ((n / STAGES) - 1) & 1, dead);
+          ptx::mbar_expect_tx(&full[s], S::B_BYTES);
+          ptx::tma_load_3d(tiles + s * S::STAGE_BYTES + S::A_BYTES, &tmB, 0, n0, ks * KCH, &full[s]);
+        }
+      }
+    }
+  } else if (warp == 2) {
+    if (lane == 0) {
+      // ---- MMA issuer
+      constexpr uint32_t idesc = ptx::idesc_bf16(GEMM_BM, BN);
+      int n = 0, j = 0;
+      for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++j) {
+        const int acc = j & 1;
+        if (j >= 2) ptx::mbar_wait(&tmem_empty[acc], ((j >> 1) - 1) & 1, dead);
+        ptx::tc_fence_after();
+        const uint32_t d = tmem + acc * BN;
+        for (int ks = 0; ks < kstages; ++ks, ++n) {
+          const int s = n % STAGES;
+          ptx::mbar_wait(&full[s], (n / STAGES) & 1, dead);
+          ptx::tc_fence_after();
+          const uint32_t a = ptx::smem_u32(tiles + s * S::STAGE_BYTES);
 #pragma unroll
-      for (int kk = 0; kk < GEMM_BK / 16; ++kk)
-        ptx::mma_bf16(tmem, ad + 2 * kk, bd + 2 * kk, idesc, (kb | kk) != 0);
-      ptx::mma_commit(&empty[s]);  // frees the stage once these MMAs have read it
+          for (int c = 0; c < KCH; ++c) {
+            if (ks * KCH + c < kchunks) {
+              const uint64_t ad = ptx::smem_desc_sw128(a + c * (GEMM_BM * 128));
+              const uint64_t bd = ptx::smem_desc_sw128(a + S::A_BYTES + c * (BN * 128));
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk) ptx::mma_bf16(d, ad + 2 * kk, bd + 2 * kk, idesc, (ks | c | kk) != 0);
+            }
+          }
+          ptx::mma_commit(&empty[s]);  // frees the stage once these MMAs have read it
+        }
+        ptx::mma_commit(&tmem_full[acc]);
+      }
     }
-    ptx::mma_commit(accum);
-  }
-  __syncwarp();
-
-  // ---- epilogue: all four warps
-  ptx::mbar_wait(accum, 0, dead);
-  __syncwarp();
-  ptx::tc_fence_after();
-  const int row = m0 + warp * 32 + lane;
-  const bool row_ok = row < M;
+  } else {
+    // ---- epilogue warps 3..10
+    const int e = warp - 3;
+    const int q = warp & 3;          // TMEM lane quarter this warp may access
+    const int half = e >> 2;         // which 64-column half of the pass
+    const int et = threadIdx.x - 96; // 0..255
+    const int row = q * 32 + lane;   // row inside the tile
+    int j = 0, rp = 0;               // rp counts residual loads (phase of res_full)
+    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++j) {
+      const int acc = j & 1;
+      const int m0 = (t % tiles_m) * GEMM_BM, n0 = (t / tiles_m) * BN;
 #pragma unroll 1
-  for (int c = 0; c < BN; c += 32) {
-    uint32_t r[32];
-    ptx::tmem_ld32(tmem + (static_cast<uint32_t>(warp * 32) << 16) + c, r);
-    ptx::tmem_ld_wait();
-    const int col0 = n0 + c;
-    if (row_ok && col0 < N) {
-      float v[32];
+      for (int ps = 0; ps < PASSES; ++ps) {
+        const int np = n0 + ps * GEMM_PASS_COLS;   // first global column of this pass
+        // staging tile free again? (the previous TMA store must have finished reading it); then the
+        // residual of this pass is loaded into it
+        if (et == 0) {
+          bulk_wait_read0();
+          if (ep.has_residual && np < N) {
+            ptx::mbar_expect_tx(res_full, GEMM_STAGE_OUT);
+            ptx::tma_load_2d(out_stage, &tmRes, np, m0, res_full);
+            ptx::tma_load_2d(out_stage + 16384, &tmRes, np + 64, m0, res_full);
+          }
+        }
+        if (et < GEMM_PASS_COLS) bias_s[et] = (ep.bias && np + et < N) ? __bfloat162float(ep.bias[np + et]) : 0.0f;
+        epi_bar_sync();
+        if (ps == 0) ptx::mbar_wait(&tmem_full[acc], (j >> 1) & 1, dead);
+        if (ep.has_residual && np < N) ptx::mbar_wait(res_full, rp & 1, dead);
+        __syncwarp();
+        ptx::tc_fence_after();
+        if (np < N) {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-      const bool fullc = (col0 + 32 <= N);
-      if (ep.bias) {
+          for (int c = 0; c < 2; ++c) {
+            const int col = half * 64 + c * 32;  // column inside the pass
+            uint32_t r[32];
+            ptx::tmem_ld32(tmem + (static_cast<uint32_t>(q * 32) << 16) + acc * BN + ps * GEMM_PASS_COLS + col, r);
+            ptx::tmem_ld_wait();
+            uint8_t* obase = out_stage + half * 16384 + row * 128;
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (fullc || col0 + j < N) v[j] += __bfloat162float(ep.bias[col0 + j]);
-      }
-      if (ep.act == ACT_GELU) {
+            for (int g = 0; g < 4; ++g) {
+              float v[8];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
-      } else if (ep.act == ACT_RELU) {
+              for (int i = 0; i < 8; ++i) v[i] = apply_act(ep.act, __uint_as_float(r[g * 8 + i]) + bias_s[col + g * 8 + i]);
+              const int sw = ((c * 4 + g) ^ (row & 7)) << 4;
+              if (ep.has_residual) {
+                const uint4 rv = *reinterpret_cast<const uint4*>(obase + sw);
+                const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&rv);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.0f);
-      }
-      __nv_bfloat16* o = ep.out + static_cast<long long>(row) * ep.ldo + col0;
-      if (fullc && ((reinterpret_cast<uintptr_t>(o) & 15) == 0) &&
-          (!ep.residual || ((reinterpret_cast<uintptr_t>(ep.residual + static_cast<long long>(row) * ep.ldr + col0) & 15) == 0))) {
-        if (ep.residual) {
-          const uint4* rp = reinterpret_cast<const uint4*>(ep.residual + static_cast<long long>(row) * ep.ldr + col0);
+                for (int i = 0; i < 4; ++i) { const float2 f = __bfloat1622float2(h[i]); v[2 * i] += f.x; v[2 * i + 1] += f.y; }
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            uint4 rv = rp[q];
-            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&rv);
+                for (int i = 0; i < 8; ++i) v[i] = apply_act(ep.act2, v[i]);
+              }
+              uint4 ov;
+              __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&ov);
 #pragma unroll
-            for (int t = 0; t < 4; ++t) {
-              float2 f = __bfloat1622float2(h[t]);
-              v[q * 8 + 2 * t] += f.x;
-              v[q * 8 + 2 * t + 1] += f.y;
+              for (int i = 0; i < 4; ++i) oh[i] = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+              *reinterpret_cast<uint4*>(obase + sw) = ov;
             }
           }
         }
-        uint4* op = reinterpret_cast<uint4*>(o);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          uint4 ov;
-          __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&ov);
-#pragma unroll
-          for (int t = 0; t < 4; ++t) h[t] = __floats2bfloat162_rn(v[q * 8 + 2 * t], v[q * 8 + 2 * t + 1]);
-          op[q] = ov;
-        }
-      } else {
-        for (int j = 0; j < 32; ++j) {
-          if (col0 + j < N) {
-            float x = v[j];
-            if (ep.residual) x += __bfloat162float(ep.residual[static_cast<long long>(row) * ep.ldr + col0 + j]);
-            o[j] = __float2bfloat16_rn(x);
-          }
+        if (ep.has_residual && np < N) ++rp;
+        // publish the staging tile to the async proxy; after the last pass the accumulator is free
+        ptx::tc_fence_before();
+        ptx::fence_proxy_async();
+        __syncwarp();
+        if (ps == PASSES - 1 && lane == 0) ptx::mbar_arrive(&tmem_empty[acc]);
+        epi_bar_sync();
+        if (et == 0 && np < N) {
+          tma_store_2d(&tmOut, out_stage, np, m0);
+          if (np + 64 < N) tma_store_2d(&tmOut, out_stage + 16384, np + 64, m0);
+          bulk_commit();
         }
       }
     }
+    if (et == 0) bulk_wait0();
   }
   ptx::tc_fence_before();
   __syncthreads();
-  if (warp == 0) ptx::tmem_dealloc(tmem, TMEM_COLS);
+  if (warp == 2) ptx::tmem_dealloc(tmem, TMEM_COLS);
   if (threadIdx.x == 0 && *dead && ep.status) atomicExch(ep.status, 1);
 }
 
