@@ -12,6 +12,8 @@
 #include <cuda_runtime.h>
 #include <cstdint>
 
+#include "ptx.cuh"
+
 namespace sod2 {
 namespace k {
 
@@ -89,6 +91,8 @@ __global__ void __launch_bounds__(128) attention_fwd_bf16(const __grid_constant_
   const __nv_bfloat16* kg = p.k + R.k_off + static_cast<long long>(head) * R.k_hs;
   const __nv_bfloat16* vg = p.v + R.v_off + static_cast<long long>(head) * R.v_hs;
   const int nkv = (L + 63) >> 6;
+  ptx::pdl_wait();
+  ptx::pdl_launch();
 
   load_tile(sQ, qg, R.q_ts, q0, L, tid);
   load_tile(sK[0], kg, R.k_ts, 0, L, tid);

@@ -42,6 +42,23 @@ struct Launch {
 
 namespace {
 
+// Launch with programmatic dependent launch allowed (see ptx::pdl_wait): only for kernels that call
+// pdl_wait() in every thread.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
 int64_t numel(const std::vector<int64_t>& d) { int64_t n = 1; for (auto v : d) n *= v; return n; }
 
 struct Builder {
@@ -217,22 +234,32 @@ struct Builder {
         k::GemmEpilogue ep{};
         ep.bias = hb ? reinterpret_cast<const __nv_bfloat16*>(x.resolve(pb)) : nullptr;
         ep.has_residual = hr;
-        ep.act = act;
         ep.act2 = act2;
         ep.status = reinterpret_cast<int*>(x.arena);
         const int tiles = tiles_m * static_cast<int>((N + bn - 1) / bn);
         const int grid = std::min(tiles, x.plan->sm_count);
-        if (bn == 256) {
-          constexpr int smem = k::GemmSmem<256, 1, 4>::TOTAL;
-          static bool once = (cudaFuncSetAttribute(k::gemm_bf16_tcgen05<256, 1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);
-          (void)once;
-          k::gemm_bf16_tcgen05<256, 1, 4><<<grid, k::GEMM_THREADS, smem, x.stream>>>(cache->ta, cache->tb, cache->to, cache->tr, M, static_cast<int>(N), static_cast<int>(K), ep);
-        } else {
-          constexpr int smem = k::GemmSmem<128, 2, 3>::TOTAL;
-          static bool once = (cudaFuncSetAttribute(k::gemm_bf16_tcgen05<128, 2, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);
-          (void)once;
-          k::gemm_bf16_tcgen05<128, 2, 3><<<grid, k::GEMM_THREADS, smem, x.stream>>>(cache->ta, cache->tb, cache->to, cache->tr, M, static_cast<int>(N), static_cast<int>(K), ep);
+        const int variant = (bn == 256 ? 0 : 3) + act;
+        const dim3 gd(grid), bd(k::GEMM_THREADS);
+        const int Ni = static_cast<int>(N), Ki = static_cast<int>(K);
+#define SOD2_GEMM_CASE(V, BN_, KCH_, ST_, ACT_)                                                                              \
+        case V: {                                                                                                            \
+          constexpr int smem = k::GemmSmem<BN_, KCH_, ST_>::TOTAL;                                                            \
+          static bool once = (cudaFuncSetAttribute(k::gemm_bf16_tcgen05<BN_, KCH_, ST_, ACT_>,                                \
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);                 \
+          (void)once;                                                                                                        \
+          launch_pdl(k::gemm_bf16_tcgen05<BN_, KCH_, ST_, ACT_>, gd, bd, smem, x.stream, cache->ta, cache->tb, cache->to,     \
+                     cache->tr, M, Ni, Ki, ep);                                                                               \
+        } break;
+        switch (variant) {
+          SOD2_GEMM_CASE(0, 256, 1, 4, 0)
+          SOD2_GEMM_CASE(1, 256, 1, 4, 1)
+          SOD2_GEMM_CASE(2, 256, 1, 4, 2)
+          SOD2_GEMM_CASE(3, 128, 2, 3, 0)
+          SOD2_GEMM_CASE(4, 128, 2, 3, 1)
+          default:
+          SOD2_GEMM_CASE(5, 128, 2, 3, 2)
         }
+#undef SOD2_GEMM_CASE
         return cudaGetLastError();
       });
     }
@@ -282,7 +309,7 @@ struct Builder {
         ap.k = reinterpret_cast<const __nv_bfloat16*>(x.resolve(bk));
         ap.v = reinterpret_cast<const __nv_bfloat16*>(x.resolve(bv));
         ap.o = reinterpret_cast<__nv_bfloat16*>(x.resolve(bo));
-        k::attention_fwd_bf16<<<dim3(tiles, ap.H), 128, 0, x.stream>>>(ap);
+        launch_pdl(k::attention_fwd_bf16, dim3(tiles, ap.H), dim3(128), 0, x.stream, ap);
         return cudaGetLastError();
       });
     }
@@ -311,10 +338,10 @@ struct Builder {
         auto* Bt = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pb));
         const unsigned grid = static_cast<unsigned>((rows + 7) / 8);
         switch (ch) {
-          case 1: k::layernorm_bf16<1><<<grid, 256, 0, x.stream>>>(X, Gm, Bt, Y, rows, static_cast<int>(D), eps); break;
-          case 2: k::layernorm_bf16<2><<<grid, 256, 0, x.stream>>>(X, Gm, Bt, Y, rows, static_cast<int>(D), eps); break;
-          case 3: k::layernorm_bf16<3><<<grid, 256, 0, x.stream>>>(X, Gm, Bt, Y, rows, static_cast<int>(D), eps); break;
-          default: k::layernorm_bf16<4><<<grid, 256, 0, x.stream>>>(X, Gm, Bt, Y, rows, static_cast<int>(D), eps); break;
+          case 1: launch_pdl(k::layernorm_bf16<1>, dim3(grid), dim3(256), 0, x.stream, X, Gm, Bt, Y, rows, static_cast<int>(D), eps); break;
+          case 2: launch_pdl(k::layernorm_bf16<2>, dim3(grid), dim3(256), 0, x.stream, X, Gm, Bt, Y, rows, static_cast<int>(D), eps); break;
+          case 3: launch_pdl(k::layernorm_bf16<3>, dim3(grid), dim3(256), 0, x.stream, X, Gm, Bt, Y, rows, static_cast<int>(D), eps); break;
+          default: launch_pdl(k::layernorm_bf16<4>, dim3(grid), dim3(256), 0, x.stream, X, Gm, Bt, Y, rows, static_cast<int>(D), eps); break;
         }
         return cudaGetLastError();
       });
@@ -429,9 +456,9 @@ struct Builder {
         tp.idx = reinterpret_cast<long long*>(x.resolve(bi));
         tp.score = score;
         k::ScoreParams sp{tp.y, score, rows, tp.D};
-        if (rows) k::row_sumsq_f64<<<static_cast<unsigned>((rows + 7) / 8), 256, 0, x.stream>>>(sp);
+        if (rows) launch_pdl(k::row_sumsq_f64, dim3(static_cast<unsigned>((rows + 7) / 8)), dim3(256), 0, x.stream, sp);
         if (smem > 48 * 1024) cudaFuncSetAttribute(k::topk_keep, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        k::topk_keep<<<tp.n_req, 1024, smem, x.stream>>>(tp);
+        launch_pdl(k::topk_keep, dim3(tp.n_req), dim3(1024), smem, x.stream, tp);
         return cudaGetLastError();
       });
     }

@@ -29,8 +29,7 @@ enum Act : int { ACT_NONE = 0, ACT_GELU = 1, ACT_RELU = 2 };
 struct GemmEpilogue {
   const __nv_bfloat16* bias;  // [N] or nullptr
   int has_residual;           // residual arrives through its own tensor map
-  int act;                    // applied before the residual add
-  int act2;                   // applied after the residual add
+  int act2;                   // applied after the residual add (ACT_NONE or ACT_RELU); the pre-residual one is a template parameter
   int* status;                // device word; set non-zero if a bounded wait ran out
 };
 
@@ -44,7 +43,7 @@ struct GemmSmem {
   static constexpr int A_BYTES = KCH * GEMM_BM * 128;
   static constexpr int B_BYTES = KCH * BN * 128;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int TOTAL = STAGES * STAGE_BYTES + GEMM_STAGE_OUT + 1024 /*align slack*/ + 1024 /*bias + barriers*/;
+  static constexpr int TOTAL = STAGES * STAGE_BYTES + GEMM_STAGE_OUT + 896 /*align slack: the window is at least 128-B aligned*/ + 2048 /*bias*/ + 128 /*barriers*/;
 };
 
 // erf by the rational approximation 7.1.26 of Abramowitz & Stegun (|error| <= 1.5e-7), far inside
@@ -60,8 +59,13 @@ __device__ __forceinline__ float gelu_erf(float x) {
   const float e = 1.0f - p * t * __expf(-z * z);   // erf(|x|/sqrt2)
   return 0.5f * x * (1.0f + copysignf(e, x));
 }
-__device__ __forceinline__ float apply_act(int act, float v) {
-  return act == ACT_GELU ? gelu_erf(v) : act == ACT_RELU ? fmaxf(v, 0.0f) : v;
+// The activation is a template parameter: a run-time switch inside the unrolled element loops
+// turns every element into its own basic block and serialises the dependent FMA / MUFU chains.
+template <int ACT>
+__device__ __forceinline__ float apply_act(float v) {
+  if constexpr (ACT == ACT_GELU) return gelu_erf(v);
+  else if constexpr (ACT == ACT_RELU) return fmaxf(v, 0.0f);
+  else return v;
 }
 
 __device__ __forceinline__ void tma_store_2d(const void* tmap, const void* src, int x, int y) {
@@ -75,7 +79,7 @@ __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 256;"
 
 // tmA / tmB are 3-D views {64, rows, K/64} of the row-major operands (K % 64 == 0), box
 // {64, 128 or BN, KCH}: one instruction fills KCH consecutive swizzled [rows x 64] chunks.
-template <int BN, int KCH, int STAGES>
+template <int BN, int KCH, int STAGES, int ACT>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmRes,
@@ -85,8 +89,8 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* out_stage = tiles + STAGES * S::STAGE_BYTES;
-  float* bias_s = reinterpret_cast<float*>(out_stage + GEMM_STAGE_OUT);  // [128]
-  uint64_t* full = reinterpret_cast<uint64_t*>(bias_s + GEMM_PASS_COLS);
+  float* bias_s = reinterpret_cast<float*>(out_stage + GEMM_STAGE_OUT);  // [2][256]
+  uint64_t* full = reinterpret_cast<uint64_t*>(bias_s + 512);
   uint64_t* empty = full + STAGES;
   uint64_t* tmem_full = empty + STAGES;   // [2]
   uint64_t* tmem_empty = tmem_full + 2;   // [2]
@@ -118,6 +122,9 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  // everything above touched only this CTA's own state; the operands may still be in flight
+  ptx::pdl_wait();
+  ptx::pdl_launch();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -184,66 +191,85 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const int et = threadIdx.x - 96; // 0..255
     const int row = q * 32 + lane;   // row inside the tile
     int j = 0, rp = 0;               // rp counts residual loads (phase of res_full)
+    auto load_bias = [&](int t) -> float {
+      const int idx = (t / tiles_m) * BN + et;
+      return (ep.bias && et < BN && t < num_tiles && idx < N) ? __bfloat162float(ep.bias[idx]) : 0.0f;
+    };
+    float bias_next = load_bias(blockIdx.x);
+    const float relu2_floor = ep.act2 == ACT_RELU ? 0.0f : -INFINITY;  // post-residual activation, branch-free
     for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++j) {
       const int acc = j & 1;
       const int m0 = (t % tiles_m) * GEMM_BM, n0 = (t / tiles_m) * BN;
+      float* bias_t = bias_s + (j & 1) * 256;      // this tile's bias, prefetched during the last tile
+      bias_t[et] = bias_next;
+      bias_next = load_bias(t + gridDim.x);
+      epi_bar_sync();
+      ptx::mbar_wait(&tmem_full[acc], (j >> 1) & 1, dead);
+      __syncwarp();
+      ptx::tc_fence_after();
 #pragma unroll 1
       for (int ps = 0; ps < PASSES; ++ps) {
         const int np = n0 + ps * GEMM_PASS_COLS;   // first global column of this pass
-        // staging tile free again? (the previous TMA store must have finished reading it); then the
-        // residual of this pass is loaded into it
-        if (et == 0) {
-          bulk_wait_read0();
-          if (ep.has_residual && np < N) {
+        const bool live = np < N;
+        const bool res = ep.has_residual && live;
+        if (res) {
+          // the residual tile is TMA-loaded into the staging tile (once the previous store has
+          // finished reading it) and updated in place
+          if (et == 0) {
+            bulk_wait_read0();
             ptx::mbar_expect_tx(res_full, GEMM_STAGE_OUT);
             ptx::tma_load_2d(out_stage, &tmRes, np, m0, res_full);
             ptx::tma_load_2d(out_stage + 16384, &tmRes, np + 64, m0, res_full);
           }
+          ptx::mbar_wait(res_full, rp & 1, dead);
+          __syncwarp();
+          ++rp;
         }
-        if (et < GEMM_PASS_COLS) bias_s[et] = (ep.bias && np + et < N) ? __bfloat162float(ep.bias[np + et]) : 0.0f;
-        epi_bar_sync();
-        if (ps == 0) ptx::mbar_wait(&tmem_full[acc], (j >> 1) & 1, dead);
-        if (ep.has_residual && np < N) ptx::mbar_wait(res_full, rp & 1, dead);
-        __syncwarp();
-        ptx::tc_fence_after();
-        if (np < N) {
+        uint8_t* obase = out_stage + half * 16384 + row * 128;
+        uint4 pk[8];
+        if (live) {
 #pragma unroll
           for (int c = 0; c < 2; ++c) {
             const int col = half * 64 + c * 32;  // column inside the pass
             uint32_t r[32];
             ptx::tmem_ld32(tmem + (static_cast<uint32_t>(q * 32) << 16) + acc * BN + ps * GEMM_PASS_COLS + col, r);
             ptx::tmem_ld_wait();
-            uint8_t* obase = out_stage + half * 16384 + row * 128;
+            const float* bp = bias_t + ps * GEMM_PASS_COLS + col;
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
               float v[8];
 #pragma unroll
-              for (int i = 0; i < 8; ++i) v[i] = apply_act(ep.act, __uint_as_float(r[g * 8 + i]) + bias_s[col + g * 8 + i]);
-              const int sw = ((c * 4 + g) ^ (row & 7)) << 4;
-              if (ep.has_residual) {
-                const uint4 rv = *reinterpret_cast<const uint4*>(obase + sw);
+              for (int i = 0; i < 8; ++i) v[i] = apply_act<ACT>(__uint_as_float(r[g * 8 + i]) + bp[g * 8 + i]);
+              if (res) {
+                const uint4 rv = *reinterpret_cast<const uint4*>(obase + (((c * 4 + g) ^ (row & 7)) << 4));
                 const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&rv);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) { const float2 f = __bfloat1622float2(h[i]); v[2 * i] += f.x; v[2 * i + 1] += f.y; }
 #pragma unroll
-                for (int i = 0; i < 8; ++i) v[i] = apply_act(ep.act2, v[i]);
+                for (int i = 0; i < 8; ++i) v[i] = fmaxf(v[i], relu2_floor);
               }
-              uint4 ov;
-              __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&ov);
+              __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&pk[c * 4 + g]);
 #pragma unroll
               for (int i = 0; i < 4; ++i) oh[i] = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
-              *reinterpret_cast<uint4*>(obase + sw) = ov;
             }
           }
         }
-        if (ep.has_residual && np < N) ++rp;
+        // the math above overlapped the previous pass's TMA store; now the staging tile must be free
+        if (!res) {
+          if (et == 0) bulk_wait_read0();
+          epi_bar_sync();
+        }
+        if (live) {
+#pragma unroll
+          for (int g = 0; g < 8; ++g) *reinterpret_cast<uint4*>(obase + ((g ^ (row & 7)) << 4)) = pk[g];
+        }
         // publish the staging tile to the async proxy; after the last pass the accumulator is free
         ptx::tc_fence_before();
         ptx::fence_proxy_async();
         __syncwarp();
         if (ps == PASSES - 1 && lane == 0) ptx::mbar_arrive(&tmem_empty[acc]);
         epi_bar_sync();
-        if (et == 0 && np < N) {
+        if (et == 0 && live) {
           tma_store_2d(&tmOut, out_stage, np, m0);
           if (np + 64 < N) tma_store_2d(&tmOut, out_stage + 16384, np + 64, m0);
           bulk_commit();

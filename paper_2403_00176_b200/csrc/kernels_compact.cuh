@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <cstdint>
 
+#include "ptx.cuh"
+
 namespace sod2 {
 namespace k {
 
@@ -21,6 +23,8 @@ struct ScoreParams {
   int D;
 };
 __global__ void __launch_bounds__(256) row_sumsq_f64(ScoreParams p) {
+  ptx::pdl_wait();
+  ptx::pdl_launch();
   const int lane = threadIdx.x & 31;
   const long long row = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
   if (row >= p.rows) return;
@@ -73,6 +77,8 @@ __global__ void __launch_bounds__(1024) topk_keep(const __grid_constant__ TopkPa
   int* s_pos = reinterpret_cast<int*>(s_score + ((p.r[blockIdx.x].n + 1) & ~1));  // [n] kept position or -1
   __shared__ int warp_tot[32];
   const TopkReq R = p.r[blockIdx.x];
+  ptx::pdl_wait();
+  ptx::pdl_launch();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int i = tid; i < R.n; i += blockDim.x) s_score[i] = p.score[R.row0 + i];
   __syncthreads();

@@ -7,6 +7,8 @@
 #include <cuda_runtime.h>
 #include <cstdint>
 
+#include "ptx.cuh"
+
 namespace sod2 {
 namespace k {
 
@@ -96,6 +98,8 @@ template <int CH>
 __global__ void __launch_bounds__(256) layernorm_bf16(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ gamma,
                                                        const __nv_bfloat16* __restrict__ beta, __nv_bfloat16* __restrict__ y,
                                                        long long rows, int D, float eps) {
+  ptx::pdl_wait();
+  ptx::pdl_launch();
   const int lane = threadIdx.x & 31;
   const long long row = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
   if (row >= rows) return;

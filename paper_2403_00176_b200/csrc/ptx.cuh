@@ -12,6 +12,14 @@ namespace ptx {
 #define SOD2_SPIN_LIMIT (1u << 22)
 #endif
 
+// Programmatic dependent launch: a kernel launched with the programmatic-stream-serialization
+// attribute may start while its predecessor in the stream is still running; pdl_wait() returns once
+// the predecessor grid has completed and its memory is visible.  Every such kernel calls pdl_wait()
+// in all threads before it touches global memory written or read by earlier kernels, so completion
+// stays transitive along the stream.  pdl_launch() lets the successor's CTAs be scheduled early.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
