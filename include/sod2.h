@@ -143,6 +143,27 @@ sod2_status sod2_plan_group_cost(const sod2_plan_t* p, int group, double* flops,
 sod2_status sod2_run_output_shape(sod2_plan_t* p, const void* arena, void* cuda_stream, int request, int output,
                                   int64_t* dims, int* rank);
 
+/* NonZero without any allocation: for callers that cannot call cudaMalloc (code inside a stream
+ * capture or a serving loop where an allocation would synchronise the device, plug-ins whose host
+ * framework owns all device memory and hands out only input and output buffers, processes under a
+ * fixed memory budget) and therefore cannot provide an arena either.  The paper has no counterpart
+ * of this call; it is a packaging variant of the NonZero compaction above.
+ *   dev_x     device, [dims...] row-major, dtype 0 = f32, 1 = bf16; rank 1..4; dims on the host
+ *   dev_out   device, int64 [rank, nnz] with row pitch nnz; must hold rank * numel entries
+ *   dev_count device, one int64: receives nnz
+ * The scratch (per-block counters) is a fixed array inside the library's device image: inputs of
+ * more than SOD2_NONZERO_STATIC_MAX_ELEMS elements are rejected with SOD2_E_BAD_DIM; every GPU that
+ * loads the library holds the array (about 65 KB) until the process exits; all calls share it, so
+ * calls that overlap on the GPU (two streams, two threads) race; it keeps the previous call's
+ * contents, which is harmless because every call overwrites each counter before reading it.  The
+ * first call on a device looks up the array's address and should be made outside any stream
+ * capture.  Calls no cudaMalloc / cudaFree or allocating routine.  Asynchronous on cuda_stream.
+ * Errors: SOD2_E_INVALID_ARG, SOD2_E_RANK_MISMATCH, SOD2_E_BAD_DIM, SOD2_E_CUDA; message through
+ * sod2_last_error(NULL). */
+#define SOD2_NONZERO_STATIC_MAX_ELEMS 16777216LL
+sod2_status sod2_nonzero_static(const void* dev_x, int dtype, int rank, const int64_t* dims, int64_t* dev_out,
+                                int64_t* dev_count, void* cuda_stream);
+
 /* handle may be a graph, binding or plan; returns "" if there was no error. */
 const char* sod2_last_error(const void* any_handle);
 

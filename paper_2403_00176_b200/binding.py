@@ -62,6 +62,7 @@ def _load() -> C.CDLL:
         "sod2_plan_memory": [vp, P(sz), P(sz), P(sz)],
         "sod2_plan_group_cost": [vp, i32, P(C.c_double), P(C.c_double)],
         "sod2_run_output_shape": [vp, vp, vp, i32, i32, P(i64), P(i32)],
+        "sod2_nonzero_static": [vp, i32, i32, P(i64), vp, vp, vp],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -85,7 +86,7 @@ EXPORTS = ["sod2_graph_create", "sod2_graph_destroy", "sod2_graph_set_const", "s
            "sod2_graph_num_ops", "sod2_graph_op_info", "sod2_graph_num_groups", "sod2_graph_group_info",
            "sod2_graph_num_subgraphs", "sod2_graph_rdp_sweeps", "sod2_classify", "sod2_graph_reanalyse",
            "sod2_binding_shape", "sod2_plan_slot", "sod2_plan_instance_offset", "sod2_plan_memory", "sod2_plan_group_cost",
-           "sod2_run_output_shape", "sod2_last_error"]
+           "sod2_run_output_shape", "sod2_nonzero_static", "sod2_last_error"]
 
 
 def _check(status: int, handle=None):
@@ -98,6 +99,18 @@ def sod2_classify(op: str) -> str:
     c = C.c_int()
     _check(lib.sod2_classify(op.encode(), C.byref(c)))
     return DYN_CLASS[c.value]
+
+
+NONZERO_STATIC_MAX_ELEMS = 16777216
+
+
+def sod2_nonzero_static(dev_x: int, dtype: int, dims: Sequence[int], dev_out: int, dev_count: int, stream: int) -> None:
+    """NonZero for callers that cannot allocate device memory (no arena, no cudaMalloc): the scratch
+    is a fixed array inside the library.  See include/sod2.h for the limits (input size, shared
+    scratch, first call outside stream capture)."""
+    d = (C.c_int64 * max(len(dims), 1))(*[int(v) for v in dims])
+    _check(lib.sod2_nonzero_static(C.c_void_p(dev_x), dtype, len(dims), d, C.c_void_p(dev_out), C.c_void_p(dev_count),
+                                   C.c_void_p(stream)))
 
 
 class Graph:

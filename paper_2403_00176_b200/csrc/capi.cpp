@@ -19,6 +19,10 @@ struct sod2_plan_s { HandleBase h{0x53443250u, ""}; Plan p; sod2_graph* g = null
 
 static thread_local std::string g_create_err;
 
+namespace sod2 {
+void set_thread_error(const std::string& msg) { g_create_err = msg; }
+}  // namespace sod2
+
 static sod2_status st(Status s) { return static_cast<sod2_status>(s); }
 
 static void copy_str(const std::string& s, char* buf, size_t len) {

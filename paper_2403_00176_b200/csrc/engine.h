@@ -71,6 +71,9 @@ struct Compiled {
   std::string err;
 };
 
+// Message returned by sod2_last_error(NULL) on the calling thread (errors of calls without a handle).
+void set_thread_error(const std::string& msg);
+
 Status form_groups(Compiled* c);
 // Transposed (K-major) copies of the GEMM weights into caller-owned workspace; enqueued on `stream`.
 Status prepack_weights(Compiled* c, void* workspace, size_t bytes, void* stream);
