@@ -132,6 +132,9 @@ sod2_status sod2_plan_slot(const sod2_plan_t* p, const char* tensor, size_t* off
                            int* last_use_step);
 /* Byte offset of one request's instance inside a packed tensor buffer. */
 sod2_status sod2_plan_instance_offset(const sod2_plan_t* p, const char* tensor, int request, size_t* offset);
+/* Element strides of one request's instance of a tensor in its buffer (views and channels-last
+ * storage are not contiguous in the logical dim order). strides must hold `rank` entries. */
+sod2_status sod2_plan_tensor_strides(const sod2_plan_t* p, const char* tensor, int request, int64_t* strides, int* rank);
 /* arena_bytes, peak live bytes, sum of all inter-group tensor bytes (what no-reuse allocation takes). */
 sod2_status sod2_plan_memory(const sod2_plan_t* p, size_t* arena_bytes, size_t* peak_live_bytes, size_t* sum_bytes);
 /* Algorithmic cost of one fused group for the bound shapes: flops of its contraction (0 for

@@ -61,6 +61,7 @@ def _load() -> C.CDLL:
         "sod2_plan_instance_offset": [vp, cp, i32, P(sz)],
         "sod2_plan_memory": [vp, P(sz), P(sz), P(sz)],
         "sod2_plan_group_cost": [vp, i32, P(C.c_double), P(C.c_double)],
+        "sod2_plan_tensor_strides": [vp, cp, i32, P(i64), P(i32)],
         "sod2_run_output_shape": [vp, vp, vp, i32, i32, P(i64), P(i32)],
         "sod2_nonzero_static": [vp, i32, i32, P(i64), vp, vp, vp],
     }
@@ -85,7 +86,7 @@ EXPORTS = ["sod2_graph_create", "sod2_graph_destroy", "sod2_graph_set_const", "s
            "sod2_run", "sod2_run_timed", "sod2_plan_device_status", "sod2_graph_tensor_info", "sod2_graph_tensor_value", "sod2_graph_tensor_dtype",
            "sod2_graph_num_ops", "sod2_graph_op_info", "sod2_graph_num_groups", "sod2_graph_group_info",
            "sod2_graph_num_subgraphs", "sod2_graph_rdp_sweeps", "sod2_classify", "sod2_graph_reanalyse",
-           "sod2_binding_shape", "sod2_plan_slot", "sod2_plan_instance_offset", "sod2_plan_memory", "sod2_plan_group_cost",
+           "sod2_binding_shape", "sod2_plan_slot", "sod2_plan_instance_offset", "sod2_plan_memory", "sod2_plan_group_cost", "sod2_plan_tensor_strides",
            "sod2_run_output_shape", "sod2_nonzero_static", "sod2_last_error"]
 
 
@@ -272,6 +273,12 @@ class Plan:
         a, p, s = C.c_size_t(), C.c_size_t(), C.c_size_t()
         _check(lib.sod2_plan_memory(self.h, C.byref(a), C.byref(p), C.byref(s)), self.h)
         return {"arena_bytes": a.value, "peak_live_bytes": p.value, "sum_bytes": s.value}
+
+    def tensor_strides(self, tensor: str, request: int) -> List[int]:
+        st = (C.c_int64 * 16)()
+        rank = C.c_int()
+        _check(lib.sod2_plan_tensor_strides(self.h, tensor.encode(), request, st, C.byref(rank)), self.h)
+        return list(st[: rank.value])
 
     def group_cost(self, group: int):
         f, b = C.c_double(), C.c_double()

@@ -272,6 +272,16 @@ sod2_status sod2_plan_instance_offset(const sod2_plan_t* p, const char* name, in
   return SOD2_OK;
 }
 
+sod2_status sod2_plan_tensor_strides(const sod2_plan_t* p, const char* name, int r, int64_t* strides, int* rank) {
+  if (!p || !name || r < 0 || r >= p->p.n_req) return SOD2_E_INVALID_ARG;
+  int t = p->g->c.g.tensor(name);
+  if (t < 0 || p->p.views[t].empty() || p->p.views[t][0].root < 0) return SOD2_E_INVALID_ARG;
+  const View& v = p->p.views[t][r];
+  if (rank) *rank = static_cast<int>(v.strides.size());
+  if (strides) for (size_t i = 0; i < v.strides.size(); ++i) strides[i] = v.strides[i];
+  return SOD2_OK;
+}
+
 sod2_status sod2_plan_group_cost(const sod2_plan_t* p, int group, double* flops, double* bytes) {
   if (!p || group < 0 || group >= static_cast<int>(p->p.group_flops.size())) return SOD2_E_INVALID_ARG;
   if (flops) *flops = p->p.group_flops[group];

@@ -1,0 +1,379 @@
+// Implicit-GEMM convolution on the tcgen05 main loop of the GEMM kernel, channels-last activations.
+//   y[n,ho,wo,co] = act2( act( sum_{dy,dx,ci} x[n, ho*s+dy-p, wo*s+dx-p, ci] * w[co, (dy,dx), ci] + bias[co] ) + res[n,ho,wo,co] )
+// bf16 in, fp32 accumulate (TMEM), bf16 out.  The "A operand" of output tile (128 pixels = TH x TW
+// patch of one image) for tap (dy,dx) and 64 input channels is ONE 4-D TMA box {64 ch, TW, TH, 1} of
+// the NHWC input at the shifted coordinate: every pixel is one 128-byte swizzled row, out-of-image
+// coordinates are zero-filled by TMA, which is the zero padding; stride-2 convolutions use the
+// tensor map's element stride.  The "B operand" is the prepacked weight matrix [Cout, taps*Cin]
+// (K-major), loaded with the same k-chunk boxes as in the GEMM.  Extents H, W are per request and
+// known only at run time: tensor maps are encoded per bound shape.
+//
+// Warp roles (384 threads, persistent, 1 CTA/SM):
+//   warps 0,1   TMA producers for the A chunks of a stage (even / odd chunk: one thread sustains only
+//               about one TMA instruction per 170 ns)
+//   warp 2      TMA producer for B (one 3-D k-chunk box per stage)
+//   warp 3      MMA issuer, two TMEM accumulators
+//   warps 4..11 epilogue in passes of 64 output channels: TMEM -> +bias -> act -> +residual (TMA-loaded
+//               into the staging tile, updated in place) -> act2 -> bf16 -> swizzled staging -> TMA store
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include "gemm_tcgen05.cuh"
+#include "ptx.cuh"
+
+namespace sod2 {
+namespace k {
+
+struct ConvParams {
+  int n_img, Ho, Wo;         // output extents
+  int Cin, Cout;
+  int ksize, stride, pad;
+  int TW, TH;                // pixel patch of a tile: TW * TH == 128
+  const __nv_bfloat16* bias; // [Cout] or nullptr
+  int has_residual;
+  int act2;                  // ACT_NONE or ACT_RELU after the residual add
+  int* status;
+};
+
+constexpr int CONV_THREADS = 384;
+constexpr int CONV_STAGE_OUT = 128 * 128;   // 16 KB: 128 pixels x 64 channels bf16
+
+template <int BN, int KCH, int STAGES>
+struct ConvSmem {
+  static constexpr int A_BYTES = KCH * 128 * 128;
+  static constexpr int B_BYTES = KCH * BN * 128;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int TOTAL = STAGES * STAGE_BYTES + CONV_STAGE_OUT + 896 + 2048 + 128;
+};
+
+__device__ __forceinline__ void tma_store_4d(const void* tmap, const void* src, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+               ::"l"(tmap), "r"(ptx::smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void conv_epi_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// tmX: {Cin, W, H, N} bf16, box {64, TW, TH, 1}, element strides {1, s, s, 1}
+// tmW: {64, Cout, K/64} k-chunk view of [Cout, K], box {64, BN, KCH}
+// tmOut / tmRes: {Cout, Wo, Ho, N}, box {64, TW, TH, 1}
+template <int BN, int KCH, int STAGES, int ACT>
+__global__ void __launch_bounds__(CONV_THREADS, 1)
+conv_igemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
+                        const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmRes, ConvParams p) {
+  using S = ConvSmem<BN, KCH, STAGES>;
+  constexpr int PASSES = BN / 64;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* out_stage = tiles + STAGES * S::STAGE_BYTES;
+  float* bias_s = reinterpret_cast<float*>(out_stage + CONV_STAGE_OUT);  // [2][256]
+  uint64_t* full = reinterpret_cast<uint64_t*>(bias_s + 512);
+  uint64_t* empty = full + STAGES;
+  uint64_t* tmem_full = empty + STAGES;
+  uint64_t* tmem_empty = tmem_full + 2;
+  uint64_t* res_full = tmem_empty + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(res_full + 1);
+  volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tiles_w = (p.Wo + p.TW - 1) / p.TW, tiles_h = (p.Ho + p.TH - 1) / p.TH;
+  const int tiles_n = (p.Cout + BN - 1) / BN;
+  const int tiles_px = tiles_w * tiles_h * p.n_img;
+  const int num_tiles = tiles_px * tiles_n;
+  const int cchunks = p.Cin / 64;                         // 64-channel chunks per tap
+  const int kchunks = p.ksize * p.ksize * cchunks;        // k-chunks in tap-major order
+  const int kstages = (kchunks + KCH - 1) / KCH;
+  constexpr uint32_t TMEM_COLS = (2 * BN < 32) ? 32 : 2 * BN;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(&full[s], 3); ptx::mbar_init(&empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&tmem_full[b], 1); ptx::mbar_init(&tmem_empty[b], 8); }
+    ptx::mbar_init(res_full, 1);
+    *dead = 0;
+    ptx::fence_barrier_init();
+    ptx::fence_proxy_async();
+    ptx::prefetch_tmap(&tmX);
+    ptx::prefetch_tmap(&tmW);
+    ptx::prefetch_tmap(&tmOut);
+    if (p.has_residual) ptx::prefetch_tmap(&tmRes);
+  }
+  if (warp == 3) { ptx::tmem_alloc(tmem_slot, TMEM_COLS); ptx::tmem_relinquish(); }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  ptx::pdl_wait();
+  ptx::pdl_launch();
+
+  // tile index -> (channel tile, image, patch origin); pixel tiles vary fastest so that CTAs running
+  // together share the weight tile in L2
+  auto decode = [&](int t, int* n0, int* img, int* ho0, int* wo0) {
+    const int tp = t % tiles_px;
+    *n0 = (t / tiles_px) * BN;
+    *img = tp / (tiles_w * tiles_h);
+    const int r = tp % (tiles_w * tiles_h);
+    *ho0 = (r / tiles_w) * p.TH;
+    *wo0 = (r % tiles_w) * p.TW;
+  };
+
+  if (warp < 2) {
+    if (lane == 0) {
+      // ---- A producers: warp 0 loads the even chunks of every stage, warp 1 the odd ones
+      int n = 0;
+      for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
+        int n0, img, ho0, wo0;
+        decode(t, &n0, &img, &ho0, &wo0);
+        for (int ks = 0; ks < kstages; ++ks, ++n) {
+          const int s = n % STAGES;
+          if (n >= STAGES) ptx::mbar_wait(&empty[s], ((n / STAGES) - 1) & 1, dead);
+          int mine = 0;
+          for (int c = warp; c < KCH; c += 2) ++mine;
+          ptx::mbar_expect_tx(&full[s], mine * 128 * 128);
+          for (int c = warp; c < KCH; c += 2) {
+            const int q = ks * KCH + c;          // k-chunk: tap-major, then 64-channel chunk
+            const int tap = q / cchunks, cc = q % cchunks;
+            const int dy = tap / p.ksize, dx = tap % p.ksize;
+            // chunks past the end (K tail of the last stage) are loaded far out of range: zero fill
+            const int hi = q < kchunks ? ho0 * p.stride + dy - p.pad : -100000;
+            ptx::tma_load_4d(tiles + s * S::STAGE_BYTES + c * (128 * 128), &tmX, cc * 64, wo0 * p.stride + dx - p.pad, hi, img, &full[s]);
+          }
+        }
+      }
+    }
+  } else if (warp == 2) {
+    if (lane == 0) {
+      // ---- B producer
+      int n = 0;
+      for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
+        const int n0 = (t / tiles_px) * BN;
+        for (int ks = 0; ks < kstages; ++ks, ++n) {
+          const int s = n % STAGES;
+          if (n >= STAGES) ptx::mbar_wait(&empty[s], ((n / STAGES) - 1) & 1, dead);
+          ptx::mbar_expect_tx(&full[s], S::B_BYTES);
+          ptx::tma_load_3d(tiles + s * S::STAGE_BYTES + S::A_BYTES, &tmW, 0, n0, ks * KCH, &full[s]);
+        }
+      }
+    }
+  } else if (warp == 3) {
+    if (lane == 0) {
+      // ---- MMA issuer
+      constexpr uint32_t idesc = ptx::idesc_bf16(128, BN);
+      int n = 0, j = 0;
+      for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++j) {
+        const int acc = j & 1;
+        if (j >= 2) ptx::mbar_wait(&tmem_empty[acc], ((j >> 1) - 1) & 1, dead);
+        ptx::tc_fence_after();
+        const uint32_t d = tmem + acc * BN;
+        for (int ks = 0; ks < kstages; ++ks, ++n) {
+          const int s = n % STAGES;
+          ptx::mbar_wait(&full[s], (n / STAGES) & 1, dead);
+          ptx::tc_fence_after();
+          const uint32_t a = ptx::smem_u32(tiles + s * S::STAGE_BYTES);
+#pragma unroll
+          for (int c = 0; c < KCH; ++c) {
+            if (ks * KCH + c < kchunks) {
+              const uint64_t ad = ptx::smem_desc_sw128(a + c * (128 * 128));
+              const uint64_t bd = ptx::smem_desc_sw128(a + S::A_BYTES + c * (BN * 128));
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk) ptx::mma_bf16(d, ad + 2 * kk, bd + 2 * kk, idesc, (ks | c | kk) != 0);
+            }
+          }
+          ptx::mma_commit(&empty[s]);
+        }
+        ptx::mma_commit(&tmem_full[acc]);
+      }
+    }
+  } else {
+    // ---- epilogue warps 4..11
+    const int e = warp - 4;
+    const int q = warp & 3;
+    const int half = e >> 2;          // which 32-channel half of the 64-channel pass
+    const int et = threadIdx.x - 128; // 0..255
+    const int row = q * 32 + lane;    // pixel inside the tile
+    const float relu2_floor = p.act2 == ACT_RELU ? 0.0f : -INFINITY;
+    int j = 0, rp = 0;
+    auto load_bias = [&](int t) -> float {
+      const int idx = (t / tiles_px) * BN + et;
+      return (p.bias && et < BN && t < num_tiles && idx < p.Cout) ? __bfloat162float(p.bias[idx]) : 0.0f;
+    };
+    float bias_next = load_bias(blockIdx.x);
+    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++j) {
+      const int acc = j & 1;
+      int n0, img, ho0, wo0;
+      decode(t, &n0, &img, &ho0, &wo0);
+      float* bias_t = bias_s + (j & 1) * 256;
+      bias_t[et] = bias_next;
+      bias_next = load_bias(t + gridDim.x);
+      conv_epi_bar();
+      ptx::mbar_wait(&tmem_full[acc], (j >> 1) & 1, dead);
+      __syncwarp();
+      ptx::tc_fence_after();
+#pragma unroll 1
+      for (int ps = 0; ps < PASSES; ++ps) {
+        const int np = n0 + ps * 64;
+        const bool live = np < p.Cout;
+        const bool res = p.has_residual && live;
+        if (res) {
+          if (et == 0) {
+            bulk_wait_read0();
+            ptx::mbar_expect_tx(res_full, CONV_STAGE_OUT);
+            ptx::tma_load_4d(out_stage, &tmRes, np, wo0, ho0, img, res_full);
+          }
+          ptx::mbar_wait(res_full, rp & 1, dead);
+          __syncwarp();
+          ++rp;
+        }
+        uint8_t* obase = out_stage + row * 128;
+        uint4 pk[4];
+        if (live) {
+          uint32_t r[32];
+          ptx::tmem_ld32(tmem + (static_cast<uint32_t>(q * 32) << 16) + acc * BN + ps * 64 + half * 32, r);
+          ptx::tmem_ld_wait();
+          const float* bp = bias_t + ps * 64 + half * 32;
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            float v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = apply_act<ACT>(__uint_as_float(r[g * 8 + i]) + bp[g * 8 + i]);
+            if (res) {
+              const uint4 rv = *reinterpret_cast<const uint4*>(obase + (((half * 4 + g) ^ (row & 7)) << 4));
+              const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&rv);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) { const float2 f = __bfloat1622float2(h[i]); v[2 * i] += f.x; v[2 * i + 1] += f.y; }
+#pragma unroll
+              for (int i = 0; i < 8; ++i) v[i] = fmaxf(v[i], relu2_floor);
+            }
+            __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&pk[g]);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) oh[i] = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+          }
+        }
+        if (!res) {
+          if (et == 0) bulk_wait_read0();
+          conv_epi_bar();
+        }
+        if (live) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) *reinterpret_cast<uint4*>(obase + (((half * 4 + g) ^ (row & 7)) << 4)) = pk[g];
+        }
+        ptx::tc_fence_before();
+        ptx::fence_proxy_async();
+        __syncwarp();
+        if (ps == PASSES - 1 && lane == 0) ptx::mbar_arrive(&tmem_empty[acc]);
+        conv_epi_bar();
+        if (et == 0 && live) {
+          tma_store_4d(&tmOut, out_stage, np, wo0, ho0, img);
+          bulk_commit();
+        }
+      }
+    }
+    if (et == 0) bulk_wait0();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 3) ptx::tmem_dealloc(tmem, TMEM_COLS);
+  if (threadIdx.x == 0 && *dead && p.status) atomicExch(p.status, 1);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Layout changes between the graph's NCHW tensors and the channels-last layout the convolution
+// groups use internally: [N, C, H*W] <-> [N, H*W, C], 32x32 tiles through shared memory.
+__global__ void __launch_bounds__(256) nchw_to_nhwc_bf16(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out,
+                                                          int C, long long HW) {
+  __shared__ __nv_bfloat16 tile[32][34];
+  const long long img = blockIdx.z;
+  const long long p0 = static_cast<long long>(blockIdx.x) * 32;
+  const int c0 = blockIdx.y * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int i = ty; i < 32; i += 8) {
+    const int c = c0 + i;
+    const long long px = p0 + tx;
+    if (c < C && px < HW) tile[i][tx] = in[(img * C + c) * HW + px];
+  }
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8) {
+    const long long px = p0 + i;
+    const int c = c0 + tx;
+    if (c < C && px < HW) out[(img * HW + px) * C + c] = tile[tx][i];
+  }
+}
+__global__ void __launch_bounds__(256) nhwc_to_nchw_bf16(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out,
+                                                          int C, long long HW) {
+  __shared__ __nv_bfloat16 tile[32][34];
+  const long long img = blockIdx.z;
+  const long long p0 = static_cast<long long>(blockIdx.x) * 32;
+  const int c0 = blockIdx.y * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int i = ty; i < 32; i += 8) {
+    const long long px = p0 + i;
+    const int c = c0 + tx;
+    if (c < C && px < HW) tile[i][tx] = in[(img * HW + px) * C + c];
+  }
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8) {
+    const int c = c0 + i;
+    const long long px = p0 + tx;
+    if (c < C && px < HW) out[(img * C + c) * HW + px] = tile[tx][i];
+  }
+}
+
+// Global average pool of a channels-last tensor with fp64 accumulation (decision scalar / final
+// feature): p[n,c] = mean_{h,w} x[n,h,w,c].  Two kernels with a fixed summation order, so the result
+// is deterministic: pixel slabs -> partial sums in scratch, then a serial sum over the slabs.
+struct GapParams {
+  const __nv_bfloat16* x;   // [N, HW, C]
+  double* partial;          // scratch [N, slabs, C]
+  void* out;                // [N, C] bf16 or f32 (or nullptr when only the fp64 means are wanted)
+  double* out_f64;          // optional [N, C] fp64 means
+  int out_bf16;
+  int C, slabs;
+  long long HW;
+};
+__global__ void __launch_bounds__(256) gap_partial_f64(GapParams p) {
+  __shared__ double part[4][64];
+  ptx::pdl_wait();
+  ptx::pdl_launch();
+  const long long img = blockIdx.z;
+  const int c = blockIdx.x * 64 + (threadIdx.x & 63);
+  const int sub = threadIdx.x >> 6;
+  const long long per = (p.HW + p.slabs - 1) / p.slabs;
+  const long long p0 = blockIdx.y * per, p1 = min(p.HW, p0 + per);
+  double acc = 0.0;
+  if (c < p.C)
+    for (long long px = p0 + sub; px < p1; px += 4) acc += static_cast<double>(__bfloat162float(p.x[(img * p.HW + px) * p.C + c]));
+  part[sub][threadIdx.x & 63] = acc;
+  __syncthreads();
+  if (sub == 0 && c < p.C)
+    p.partial[(img * p.slabs + blockIdx.y) * p.C + c] = (part[0][threadIdx.x] + part[1][threadIdx.x]) + (part[2][threadIdx.x] + part[3][threadIdx.x]);
+}
+__global__ void __launch_bounds__(256) gap_final_f64(GapParams p, int n_img) {
+  ptx::pdl_wait();
+  ptx::pdl_launch();
+  const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= static_cast<long long>(n_img) * p.C) return;
+  const long long img = i / p.C;
+  const int c = static_cast<int>(i % p.C);
+  double acc = 0.0;
+  for (int s = 0; s < p.slabs; ++s) acc += p.partial[(img * p.slabs + s) * p.C + c];
+  const double mean = acc / static_cast<double>(p.HW);
+  if (p.out_f64) p.out_f64[i] = mean;
+  if (p.out) {
+    if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[i] = __double2bfloat16(mean);
+    else reinterpret_cast<float*>(p.out)[i] = static_cast<float>(mean);
+  }
+}
+
+// Conv weights [Cout, Cin, kh, kw] -> K-major [Cout, (dy, dx, ci)] for the implicit-GEMM B operand.
+__global__ void __launch_bounds__(256) reorder_conv_weights(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out,
+                                                             int Cout, int Cin, int kh, int kw) {
+  const long long total = static_cast<long long>(Cout) * Cin * kh * kw;
+  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    long long r = i;
+    const int ci = static_cast<int>(r % Cin); r /= Cin;
+    const int dx = static_cast<int>(r % kw); r /= kw;
+    const int dy = static_cast<int>(r % kh);
+    const int co = static_cast<int>(r / kh);
+    out[i] = in[((static_cast<long long>(co) * Cin + ci) * kh + dy) * kw + dx];
+  }
+}
+
+}  // namespace k
+}  // namespace sod2

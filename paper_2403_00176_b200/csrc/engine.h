@@ -25,6 +25,7 @@ enum class GKind {
   GATE,        // GlobalAveragePool -> Reshape -> MatMul(C x 1) -> Add -> Greater
   SWITCH,
   COMBINE,
+  LAYOUT,      // NCHW <-> channels-last storage change at the ABI boundary of convolution graphs (act: 0 to, 1 from)
   UNSUPPORTED
 };
 const char* gkind_name(GKind k);

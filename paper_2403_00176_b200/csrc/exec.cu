@@ -7,6 +7,7 @@
 #include <functional>
 
 #include "attention.cuh"
+#include "conv_tcgen05.cuh"
 #include "engine.h"
 #include "gemm_tcgen05.cuh"
 #include "kernels_compact.cuh"
@@ -499,6 +500,159 @@ struct Builder {
     return OK;
   }
 
+  // ------------------------------------------------------------------------------ layout change
+  static bool is_channels_last(const View& v) {
+    if (v.dims.size() != 4) return false;
+    const int64_t C = v.dims[1], H = v.dims[2], W = v.dims[3];
+    return (C == 1 || v.strides[1] == 1) && (W == 1 || v.strides[3] == C) && (H == 1 || v.strides[2] == W * C) &&
+           (v.dims[0] == 1 || v.strides[0] == H * W * C);
+  }
+  Status build_layout(int gi, const Group& G) {
+    const Tensor& X = g.tensors[G.a];
+    for (int r = 0; r < p.n_req; ++r) {
+      const View &vi = p.views[G.a][r], &vo = p.views[G.out][r];
+      const int64_t n = numel(vi.dims);
+      if (!n) continue;
+      Ptr pi = ptr_of(G.a, r), po = ptr_of(G.out, r);
+      const bool spatial = vi.dims.size() == 4 && vi.dims[2] * vi.dims[3] > 1 && vi.dims[1] > 1;
+      if (!spatial) {  // both layouts coincide: plain copy
+        const size_t bytes = static_cast<size_t>(n) * dtype_size(X.dtype);
+        add(gi, 1, [=](const RunCtx& x) { return cudaMemcpyAsync(x.resolve(po), x.resolve(pi), bytes, cudaMemcpyDeviceToDevice, x.stream); });
+        continue;
+      }
+      if (X.dtype != DType::BF16) return fail(E_UNSUPPORTED_OP, "layout change is bf16 only");
+      const View& nchw = G.act ? vo : vi;
+      const View& cl = G.act ? vi : vo;
+      if (!nchw.contiguous() || !is_channels_last(cl)) return fail(E_UNSUPPORTED_OP, "layout change between unexpected layouts");
+      const int N = static_cast<int>(vi.dims[0]), C = static_cast<int>(vi.dims[1]);
+      const long long HW = vi.dims[2] * vi.dims[3];
+      const bool from = G.act != 0;
+      add(gi, 1, [=](const RunCtx& x) {
+        const dim3 grid(static_cast<unsigned>((HW + 31) / 32), (C + 31) / 32, N);
+        auto* in = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pi));
+        auto* out = reinterpret_cast<__nv_bfloat16*>(x.resolve(po));
+        if (from) k::nhwc_to_nchw_bf16<<<grid, 256, 0, x.stream>>>(in, out, C, HW);
+        else k::nchw_to_nhwc_bf16<<<grid, 256, 0, x.stream>>>(in, out, C, HW);
+        return cudaGetLastError();
+      });
+    }
+    return OK;
+  }
+
+  // ------------------------------------------------------------------------------ convolution
+  Status build_conv(int gi, const Group& G) {
+    const Tensor& W = g.tensors[G.w];
+    if (W.dtype != DType::BF16) return fail(E_UNSUPPORTED_OP, "convolution is bf16 only");
+    const int Cout = static_cast<int>(W.S.dims[0].e.const_value()), Cin = static_cast<int>(W.S.dims[1].e.const_value());
+    const int ks = static_cast<int>(W.S.dims[2].e.const_value());
+    if (W.S.dims[3].e.const_value() != ks) return fail(E_UNSUPPORTED_OP, "convolution needs a square kernel");
+    if (Cin % 64) return fail(E_UNSUPPORTED_OP, "implicit-GEMM convolution needs Cin % 64 == 0");
+    if (Cout % 64) return fail(E_UNSUPPORTED_OP, "implicit-GEMM convolution needs Cout % 64 == 0");
+    if (G.has_ln || (G.act != 0 && G.act != 2)) return fail(E_UNSUPPORTED_OP, "convolution epilogue: unsupported tail");
+    size_t pk = 0;
+    for (size_t i = 0; i < c.packed_consts.size(); ++i) if (c.packed_consts[i] == G.w) pk = c.packed_off[i];
+    const int bn = (Cout % 128 == 0) ? 128 : 64;
+    const int kch = 2;
+    for (int r = 0; r < p.n_req; ++r) {
+      const View &vx = p.views[G.a][r], &vo = p.views[G.out][r];
+      if (!numel(vo.dims) || !numel(vx.dims)) continue;
+      if (!is_channels_last(vx) || !is_channels_last(vo)) return fail(E_UNSUPPORTED_OP, "convolution operands must be stored channels-last");
+      if (G.res >= 0 && !is_channels_last(p.views[G.res][r])) return fail(E_UNSUPPORTED_OP, "convolution residual must be stored channels-last");
+      if (vx.dims[1] != Cin || vo.dims[1] != Cout) return fail(E_SHAPE_CONFLICT, "convolution channel counts");
+      k::ConvParams cp{};
+      cp.n_img = static_cast<int>(vo.dims[0]);
+      cp.Ho = static_cast<int>(vo.dims[2]); cp.Wo = static_cast<int>(vo.dims[3]);
+      cp.Cin = Cin; cp.Cout = Cout; cp.ksize = ks; cp.stride = G.stride; cp.pad = G.pad;
+      cp.has_residual = G.res >= 0;
+      cp.act2 = G.act2;
+      // pixel patch of a tile: the 128-pixel shape that wastes the fewest padded pixels
+      long long best = -1;
+      for (int tw : {128, 64, 32, 16, 8}) {
+        const int th = 128 / tw;
+        const long long padded = static_cast<long long>((cp.Wo + tw - 1) / tw) * tw * ((cp.Ho + th - 1) / th) * th;
+        if (best < 0 || padded < best) { best = padded; cp.TW = tw; cp.TH = th; }
+      }
+      if (cp.TW * G.stride > 256 || cp.TH * G.stride > 256) return fail(E_UNSUPPORTED_OP, "convolution stride too large for the TMA box");
+      const int H = static_cast<int>(vx.dims[2]), Wd = static_cast<int>(vx.dims[3]);
+      Ptr px = ptr_of(G.a, r), po = ptr_of(G.out, r), pr = G.res >= 0 ? ptr_of(G.res, r) : Ptr();
+      Ptr pw; pw.where = 5; pw.off = static_cast<int64_t>(pk);
+      Ptr pb = G.bias >= 0 ? ptr_of(G.bias, 0) : Ptr();
+      const bool hb = G.bias >= 0, hr = G.res >= 0;
+      const int act = G.act, stride = G.stride;
+      const int K = ks * ks * Cin;
+      const long long tiles = static_cast<long long>((cp.Wo + cp.TW - 1) / cp.TW) * ((cp.Ho + cp.TH - 1) / cp.TH) * cp.n_img * ((Cout + bn - 1) / bn);
+      struct Cache { const void* a = nullptr; const void* w = nullptr; const void* o = nullptr; const void* r = nullptr; CUtensorMap tx, tw, to, tr; };
+      auto cache = std::make_shared<Cache>();
+      add(gi, 1, [=](const RunCtx& x) mutable {
+        const void* X = x.resolve(px);
+        const void* Wp = x.resolve(pw);
+        void* O = x.resolve(po);
+        const void* R = hr ? x.resolve(pr) : O;
+        if (cache->a != X || cache->w != Wp || cache->o != O || cache->r != R) {
+          if (!encode_bf16_nhwc(&cache->tx, X, cp.n_img, H, Wd, Cin, cp.TW, cp.TH, stride) ||
+              !encode_bf16_kchunks(&cache->tw, Wp, Cout, K, K, bn, kch) ||
+              !encode_bf16_nhwc(&cache->to, O, cp.n_img, cp.Ho, cp.Wo, Cout, cp.TW, cp.TH, 1) ||
+              !encode_bf16_nhwc(&cache->tr, R, cp.n_img, cp.Ho, cp.Wo, Cout, cp.TW, cp.TH, 1))
+            return cudaErrorInvalidValue;
+          cache->a = X; cache->w = Wp; cache->o = O; cache->r = R;
+        }
+        cp.bias = hb ? reinterpret_cast<const __nv_bfloat16*>(x.resolve(pb)) : nullptr;
+        cp.status = reinterpret_cast<int*>(x.arena);
+        const dim3 gd(static_cast<unsigned>(std::min<long long>(tiles, x.plan->sm_count))), bd(k::CONV_THREADS);
+        const int variant = (bn == 128 ? 2 : 0) + (act == 2 ? 1 : 0);
+#define SOD2_CONV_CASE(V, BN_, KCH_, ST_, ACT_)                                                                          \
+        case V: {                                                                                                        \
+          constexpr int smem = k::ConvSmem<BN_, KCH_, ST_>::TOTAL;                                                        \
+          static bool once = (cudaFuncSetAttribute(k::conv_igemm_bf16_tcgen05<BN_, KCH_, ST_, ACT_>,                      \
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);             \
+          (void)once;                                                                                                    \
+          launch_pdl(k::conv_igemm_bf16_tcgen05<BN_, KCH_, ST_, ACT_>, gd, bd, smem, x.stream, cache->tx, cache->tw,     \
+                     cache->to, cache->tr, cp);                                                                          \
+        } break;
+        switch (variant) {
+          SOD2_CONV_CASE(0, 64, 2, 4, 0)
+          SOD2_CONV_CASE(1, 64, 2, 4, 2)
+          SOD2_CONV_CASE(2, 128, 2, 3, 0)
+          default:
+          SOD2_CONV_CASE(3, 128, 2, 3, 2)
+        }
+#undef SOD2_CONV_CASE
+        return cudaGetLastError();
+      });
+    }
+    return OK;
+  }
+
+  // ------------------------------------------------------------------------------ global average pool
+  Status build_gap(int gi, const Group& G) {
+    const Tensor& X = g.tensors[G.a];
+    const Tensor& O = g.tensors[G.out];
+    if (X.dtype != DType::BF16) return fail(E_UNSUPPORTED_OP, "global average pool is bf16 only");
+    for (int r = 0; r < p.n_req; ++r) {
+      const View& vx = p.views[G.a][r];
+      if (!numel(vx.dims)) continue;
+      if (!is_channels_last(vx)) return fail(E_UNSUPPORTED_OP, "global average pool reads channels-last storage");
+      k::GapParams gp{};
+      gp.C = static_cast<int>(vx.dims[1]);
+      gp.HW = vx.dims[2] * vx.dims[3];
+      gp.slabs = static_cast<int>(std::max<long long>(1, std::min<long long>(256, gp.HW / 256)));
+      gp.out_bf16 = O.dtype == DType::BF16;
+      const int N = static_cast<int>(vx.dims[0]);
+      scratch_need = std::max(scratch_need, static_cast<size_t>(N) * gp.slabs * gp.C * 8);
+      Ptr px = ptr_of(G.a, r), po = ptr_of(G.out, r);
+      add(gi, 2, [=](const RunCtx& x) mutable {
+        gp.x = reinterpret_cast<const __nv_bfloat16*>(x.resolve(px));
+        gp.partial = reinterpret_cast<double*>(x.arena + x.plan->scratch_off[0]);
+        gp.out = x.resolve(po);
+        gp.out_f64 = nullptr;
+        launch_pdl(k::gap_partial_f64, dim3((gp.C + 63) / 64, gp.slabs, N), dim3(256), 0, x.stream, gp);
+        launch_pdl(k::gap_final_f64, dim3((N * gp.C + 255) / 256), dim3(256), 0, x.stream, gp, N);
+        return cudaGetLastError();
+      });
+    }
+    return OK;
+  }
+
   // Algorithmic cost of a group for the bound shapes: every external input and output once,
   // constants once, nothing for intermediates inside the group; flops of its contraction.
   void cost(const Group& G) {
@@ -548,6 +702,9 @@ struct Builder {
         case GKind::CHAIN: s = build_chain(static_cast<int>(gi), G); break;
         case GKind::TOPK_KEEP: s = build_topk(static_cast<int>(gi), G); break;
         case GKind::NONZERO: s = build_nonzero(static_cast<int>(gi), G); break;
+        case GKind::LAYOUT: s = build_layout(static_cast<int>(gi), G); break;
+        case GKind::CONV: s = build_conv(static_cast<int>(gi), G); break;
+        case GKind::GAP: s = build_gap(static_cast<int>(gi), G); break;
         default: return fail(E_UNSUPPORTED_OP, std::string("no executor yet for group kind ") + gkind_name(G.kind));
       }
       if (s != OK) return s;
@@ -589,6 +746,13 @@ Status prepack_weights(Compiled* c, void* workspace, size_t bytes, void* stream)
   for (size_t i = 0; i < c->packed_consts.size(); ++i) {
     const Tensor& W = c->g.tensors[c->packed_consts[i]];
     if (!W.dev_ptr) { c->err = "constant " + W.name + " has no device data"; return E_INVALID_ARG; }
+    if (W.S.rank == 4) {  // convolution weights [Cout, Cin, kh, kw] -> [Cout, (dy, dx, ci)]
+      const int co = static_cast<int>(W.S.dims[0].e.const_value()), ci = static_cast<int>(W.S.dims[1].e.const_value());
+      const int kh = static_cast<int>(W.S.dims[2].e.const_value()), kw = static_cast<int>(W.S.dims[3].e.const_value());
+      k::reorder_conv_weights<<<148 * 4, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+          static_cast<const __nv_bfloat16*>(W.dev_ptr), reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + c->packed_off[i]), co, ci, kh, kw);
+      continue;
+    }
     const int K = static_cast<int>(W.S.dims[0].e.const_value()), N = static_cast<int>(W.S.dims[1].e.const_value());
     transpose_bf16<<<dim3((N + 31) / 32, (K + 31) / 32), dim3(32, 8), 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const __nv_bfloat16*>(W.dev_ptr), reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + c->packed_off[i]), K, N);

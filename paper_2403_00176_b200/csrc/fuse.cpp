@@ -25,6 +25,7 @@ const char* gkind_name(GKind k) {
     case GKind::GATE: return "gate";
     case GKind::SWITCH: return "switch";
     case GKind::COMBINE: return "combine";
+    case GKind::LAYOUT: return "layout";
     default: return "unsupported";
   }
 }
@@ -405,6 +406,9 @@ struct Fuser {
         Group G; G.kind = GKind::NONZERO; G.nodes = {nid}; G.a = n.ins[0]; G.out = n.outs[0]; finish(G);
       } else if (op == "GlobalAveragePool") {
         if (!try_gate(nid)) { Group G; G.kind = GKind::GAP; G.nodes = {nid}; G.a = n.ins[0]; G.out = n.outs[0]; finish(G); }
+      } else if (op == "ToChannelsLast" || op == "FromChannelsLast") {
+        Group G; G.kind = GKind::LAYOUT; G.nodes = {nid}; G.a = n.ins[0]; G.out = n.outs[0]; G.act = op == "FromChannelsLast";
+        finish(G);
       } else if (op == "Switch") {
         Group G; G.kind = GKind::SWITCH; G.nodes = {nid}; G.a = n.ins[0]; G.gate = n.ins[1]; G.out = n.outs[0]; G.out2 = n.outs.size() > 1 ? n.outs[1] : -1;
         finish(G);
@@ -474,6 +478,17 @@ struct Fuser {
           c.packed_off.push_back(c.packed_bytes);
           const ShapeVal& s = g.tensors[G2.w].S;
           size_t bytes = static_cast<size_t>(s.dims[0].e.const_value() * s.dims[1].e.const_value() * 2);
+          c.packed_bytes += (bytes + 255) & ~size_t(255);
+        }
+      }
+    // ... and convolution weights as [Cout, (dy, dx, ci)] for the implicit GEMM
+    for (auto& G2 : c.groups)
+      if (G2.kind == GKind::CONV && g.tensors[G2.w].dtype == DType::BF16) {
+        if (std::find(c.packed_consts.begin(), c.packed_consts.end(), G2.w) == c.packed_consts.end()) {
+          c.packed_consts.push_back(G2.w);
+          c.packed_off.push_back(c.packed_bytes);
+          size_t bytes = 2;
+          for (auto& d : g.tensors[G2.w].S.dims) bytes *= static_cast<size_t>(d.e.const_value());
           c.packed_bytes += (bytes + 255) & ~size_t(255);
         }
       }

@@ -104,6 +104,7 @@ struct Graph {
   std::vector<Assertion> asserts;
   std::vector<int> order;              // depth-first sorted nodes (Algorithm 1)
   int rdp_sweeps = 0;
+  bool has_conv = false;               // convolution graph: rank-4 float intermediates are stored channels-last
   std::string err;
 
   int tensor(const std::string& n) const { auto it = tindex.find(n); return it == tindex.end() ? -1 : it->second; }

@@ -118,6 +118,12 @@ struct Planner {
       v.offset = 0;
       v.dims = b.dims[t][r];
       v.strides = contiguous_strides(v.dims);
+      // convolution graphs keep rank-4 float intermediates channels-last: [N,C,H,W] with C innermost
+      if (g.has_conv && v.dims.size() == 4 && T.kind == TKind::VALUE && !T.is_output &&
+          (T.dtype == DType::BF16 || T.dtype == DType::F32)) {
+        const int64_t C = v.dims[1], H = v.dims[2], W = v.dims[3];
+        v.strides = {H * W * C, 1, W * C, C};
+      }
       R.inst_off[r] = per_request ? off : 0;
       int64_t bytes = numel(v.dims) * esz;
       if (per_request) off += (bytes + 15) & ~int64_t(15);

@@ -41,6 +41,8 @@ bool classify_op(const std::string& op, DynClass* out) {
       {"Relu", DynClass::ISDOS}, {"Round", DynClass::ISDOS}, {"Sigmoid", DynClass::ISDOS}, {"Softmax", DynClass::ISDOS},
       // same class by the definitions of Section 3 (output shape is a function of input shapes only)
       {"Gelu", DynClass::ISDOS}, {"LayerNormalization", DynClass::ISDOS}, {"Transpose", DynClass::ISDOS},
+      // internal storage-layout operators (inserted by the library, never written in a graph text)
+      {"ToChannelsLast", DynClass::ISDOS}, {"FromChannelsLast", DynClass::ISDOS},
       // Input Shape & Value Determined Output Shape
       {"Expand", DynClass::ISVDOS}, {"GroupNormalization", DynClass::ISVDOS}, {"MaxUnpool", DynClass::ISVDOS},
       {"OneHot", DynClass::ISVDOS}, {"Range", DynClass::ISVDOS}, {"Reshape", DynClass::ISVDOS},
@@ -145,6 +147,8 @@ static bool parse_dims(Graph* g, const std::string& txt, ShapeVal* s, std::strin
   s->rank = static_cast<int>(s->dims.size());
   return true;
 }
+
+void insert_layout_nodes(Graph* g);
 
 Status parse_ir(const char* text, size_t len, Graph* g) {
   std::string all(text, len);
@@ -276,8 +280,73 @@ Status parse_ir(const char* text, size_t len, Graph* g) {
     }
   }
   if (g->outputs.empty()) { g->err = "graph has no output"; return E_PARSE; }
+  insert_layout_nodes(g);
   return OK;
 }
+
+// Layout selection for convolution graphs: the convolution groups work on channels-last storage
+// (one pixel = one 128-byte row of 64 channels, which is what the tensor-core operand layout wants),
+// while the ABI's inputs and outputs are NCHW.  Internal layout operators are inserted at rank-4
+// float graph inputs consumed by a Conv and at rank-4 float graph outputs; they change storage
+// only, every logical shape stays NCHW.
+void insert_layout_nodes(Graph* g) {
+  bool has_conv = false;
+  for (auto& n : g->nodes) if (n.op == "Conv") has_conv = true;
+  g->has_conv = has_conv;
+  if (!has_conv) return;
+  auto add_node = [&](const std::string& op, int in, int out) {
+    Node n;
+    n.op = op;
+    classify_op(op, &n.cls);
+    n.eff_cls = n.cls;
+    n.ins = {in};
+    n.outs = {out};
+    int nid = static_cast<int>(g->nodes.size());
+    g->tensors[in].consumers.push_back(nid);
+    g->tensors[out].producer = nid;
+    g->nodes.push_back(n);
+    return nid;
+  };
+  // inputs: every non-Shape consumer reads the channels-last copy
+  for (int t : std::vector<int>(g->inputs)) {
+    Tensor& T = g->tensors[t];
+    if (T.S.rank != 4 || (T.dtype != DType::BF16 && T.dtype != DType::F32)) continue;
+    bool feeds_conv = false;
+    for (int c : T.consumers) if (g->nodes[c].op == "Conv" && g->nodes[c].ins[0] == t) feeds_conv = true;
+    if (!feeds_conv) continue;
+    int cl = new_tensor(g, T.name + "@cl");
+    g->tensors[cl].dtype = g->tensors[t].dtype;
+    std::vector<int> cons = g->tensors[t].consumers;
+    g->tensors[t].consumers.clear();
+    for (int c : cons) {
+      if (g->nodes[c].op == "Shape") { g->tensors[t].consumers.push_back(c); continue; }
+      for (int& i : g->nodes[c].ins) if (i == t) i = cl;
+      g->tensors[cl].consumers.push_back(c);
+    }
+    add_node("ToChannelsLast", t, cl);
+  }
+  // outputs: the producer writes an internal channels-last tensor, a layout operator fills the output
+  for (int t : std::vector<int>(g->outputs)) {
+    Tensor& T = g->tensors[t];
+    if (T.producer < 0 || T.kind != TKind::VALUE) continue;
+    const std::string& pop = g->nodes[T.producer].op;
+    if (pop != "Conv" && pop != "Add" && pop != "Relu" && pop != "Combine") continue;   // rank known only after RDP: restrict to conv-chain producers
+    int cl = new_tensor(g, g->tensors[t].name + "@cl");
+    Tensor& O = g->tensors[t];
+    Tensor& C = g->tensors[cl];
+    C.dtype = O.dtype;
+    // the internal tensor takes over the producer and the consumers; the output keeps its name
+    C.producer = O.producer;
+    C.out_slot = O.out_slot;
+    for (int& o : g->nodes[C.producer].outs) if (o == t) o = cl;
+    C.consumers = O.consumers;
+    for (int c : C.consumers) for (int& i : g->nodes[c].ins) if (i == t) i = cl;
+    O.consumers.clear();
+    O.producer = -1;
+    add_node("FromChannelsLast", cl, t);
+  }
+}
+
 
 // ------------------------------------------------------------------------------------ transfer helpers
 namespace {
@@ -442,7 +511,7 @@ struct Rdp {
         ch |= refine_value(out(0), vbinary(op, V(in(0)), V(in(1))));
       } else g.tensors[out(0)].dtype = g.tensors[in(0)].kind == TKind::FCONST ? g.tensors[in(1)].dtype : g.tensors[in(0)].dtype;
     } else if (op == "Relu" || op == "Sigmoid" || op == "Gelu" || op == "Softmax" || op == "LayerNormalization" ||
-               op == "Round" || op == "Cast") {
+               op == "Round" || op == "Cast" || op == "ToChannelsLast" || op == "FromChannelsLast") {
       ch |= refine_shape(out(0), S(in(0)));
       g.tensors[out(0)].dtype = g.tensors[in(0)].dtype;
       if (op == "Cast") {
@@ -752,7 +821,8 @@ struct Rdp {
     Node& n = g.nodes[nid];
     const std::string& op = n.op;
     bool ch = false;
-    if ((op == "Relu" || op == "Sigmoid" || op == "Gelu" || op == "Softmax" || op == "LayerNormalization" || op == "Round" || op == "Cast") &&
+    if ((op == "Relu" || op == "Sigmoid" || op == "Gelu" || op == "Softmax" || op == "LayerNormalization" || op == "Round" || op == "Cast" ||
+         op == "ToChannelsLast" || op == "FromChannelsLast") &&
         pred_tensor == n.ins[0]) {
       ch |= refine_shape(pred_tensor, S(n.outs[0]));
     } else if (op == "MatMul") {

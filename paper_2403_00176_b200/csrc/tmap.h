@@ -55,4 +55,21 @@ inline bool encode_bf16_kchunks(CUtensorMap* tm, const void* base, uint64_t rows
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Channels-last activation [N, H, W, C] bf16 viewed as {C, W, H, N}; box = 64 channels x (box_w x box_h)
+// pixels of one image, 128-byte swizzle; `stride` is the traversal stride along W and H (strided
+// convolutions): the box spans box_w*stride x box_h*stride source pixels and loads every stride-th.
+inline bool encode_bf16_nhwc(CUtensorMap* tm, const void* base, uint64_t N, uint64_t H, uint64_t W, uint64_t C,
+                             uint32_t box_w, uint32_t box_h, uint32_t stride) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn || C % 8) return false;
+  cuuint64_t dims[4] = {C, W, H, N};
+  cuuint64_t strides[3] = {C * 2, W * C * 2, H * W * C * 2};
+  cuuint32_t box[4] = {64, box_w * stride, box_h * stride, 1};
+  cuuint32_t estr[4] = {1, stride, stride, 1};
+  if (box[1] > 256 || box[2] > 256) return false;
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace sod2

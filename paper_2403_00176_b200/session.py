@@ -123,4 +123,9 @@ class Prepared:
         off = slot["offset"] + self.plan.instance_offset(name, r)
         cnt = int(np.prod(shp, dtype=np.int64))
         raw = self.arena[off:off + cnt * _ESZ[dt]].cpu().numpy().view(_NP[dt])
-        return _from_storage(raw, dt).reshape(shp)
+        flat = _from_storage(raw, dt)
+        strides = self.plan.tensor_strides(name, r)
+        if cnt == 0:
+            return flat.reshape(shp)
+        # storage order may differ from the logical dim order (channels-last): gather through the strides
+        return np.lib.stride_tricks.as_strided(flat, shape=shp, strides=[s * flat.itemsize for s in strides]).copy()

@@ -183,3 +183,47 @@ def test_nonzero_compaction():
         ref = O.run(wl.ir, wl.consts, req.inputs)["nz"] if req.inputs["x"].size < 5000 else np.array(np.nonzero(req.inputs["x"]))
         assert outs[r]["nz"].shape == ref.shape
         assert np.array_equal(outs[r]["nz"], ref)
+
+
+# ------------------------------------------------------------------------------------------------ cfg 4
+def _conv_requests(wl, shapes, seed=17):
+    rng = np.random.default_rng(seed)
+    return [Request({"H": h, "W": w}, {"x": bf16_round(rng.uniform(-1, 1, (1, 64, h, w)).astype(np.float32))}) for h, w in shapes]
+
+
+def test_cfg4_small_conv_stage_edge_shapes_lockstep():
+    wl = WL.cfg4(blocks=3)
+    shapes = [(1, 1), (3, 5), (8, 16), (16, 8), (17, 33), (4, 130), (33, 40), (64, 64)]
+    reqs = _conv_requests(wl, shapes)
+    s, p, outs = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE)
+    kinds = [s.graph.group_info(i)["kind"] for i in range(s.graph.num_groups())]
+    assert kinds == ["layout", "conv", "conv", "conv", "layout", "gap"]
+    for r, req in enumerate(reqs):
+        env = O.run(wl.ir, wl.consts, req.inputs)
+        for name in ("blk2", "gap"):
+            assert outs[r][name].shape == env[name].shape
+            assert O.rel_err(outs[r][name], env[name]) <= BF16_TOL, (req.syms, name)
+        errs = lockstep(wl, s, p, outs, r, BF16_TOL)
+        bad = {k: v for k, v in errs.items() if not (isinstance(v, float) and v <= BF16_TOL)}
+        assert not bad, (req.syms, bad)
+    # determinism
+    p.run()
+    outs2 = p.outputs()
+    for a, b in zip(outs, outs2):
+        assert np.array_equal(a["blk2"], b["blk2"]) and np.array_equal(a["gap"], b["gap"])
+
+
+def test_cfg4_full_config_smallest_request_and_properties():
+    wl = WL.cfg4()
+    reqs = wl.batch(0)
+    s, p, outs = run_batch(wl, reqs)
+    order = np.argsort([r.syms["H"] * r.syms["W"] for r in reqs])
+    r = int(order[0])
+    env = O.run(wl.ir, wl.consts, reqs[r].inputs)
+    last = [n for n in outs[r] if n.startswith("blk")][0]
+    assert O.rel_err(outs[r][last], env[last]) <= BF16_TOL
+    assert O.rel_err(outs[r]["gap"], env["gap"]) <= BF16_TOL
+    for r in range(len(reqs)):   # properties at any size: shapes, finiteness, gap == mean of the returned map
+        y = outs[r][last].astype(np.float64)
+        assert y.shape == (1, 64, reqs[r].syms["H"], reqs[r].syms["W"]) and np.all(np.isfinite(y))
+        assert np.allclose(outs[r]["gap"].reshape(-1), y.mean(axis=(2, 3)).reshape(-1), rtol=1e-2, atol=1e-2)
