@@ -140,8 +140,8 @@ def op_conv(x, w, b, stride, pad):
     for ky in range(kh):
         for kx in range(kw):
             win = xp[:, :, ky:ky + stride * (ho - 1) + 1:stride, kx:kx + stride * (wo - 1) + 1:stride]
-            # y[n,o,h,w] += sum_c w[o,c,ky,kx] * win[n,c,h,w]
-            y += np.einsum("oc,nchw->nohw", w[:, :, ky, kx], win)
+            # y[n,o,h,w] += sum_c w[o,c,ky,kx] * win[n,c,h,w]   (one matrix product per tap)
+            y += np.moveaxis(np.tensordot(w[:, :, ky, kx], win, axes=(1, 1)), 0, 1)
     if b is not None:
         y += b.reshape(1, o, 1, 1)
     return y

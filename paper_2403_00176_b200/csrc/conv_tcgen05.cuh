@@ -29,6 +29,10 @@ struct ConvParams {
   int Cin, Cout;
   int ksize, stride, pad;
   int TW, TH;                // pixel patch of a tile: TW * TH == 128
+  // execution-determined image count (gated sub-batch): n_img = cnt_a + cnt_b * *n_img_ptr, read on the
+  // device after the producing kernel has finished; n_img above is then only the static upper bound
+  const long long* n_img_ptr;
+  int cnt_a, cnt_b;
   const __nv_bfloat16* bias; // [Cout] or nullptr
   int has_residual;
   int act2;                  // ACT_NONE or ACT_RELU after the residual add
@@ -74,13 +78,6 @@ conv_igemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_co
   volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tiles_w = (p.Wo + p.TW - 1) / p.TW, tiles_h = (p.Ho + p.TH - 1) / p.TH;
-  const int tiles_n = (p.Cout + BN - 1) / BN;
-  const int tiles_px = tiles_w * tiles_h * p.n_img;
-  const int num_tiles = tiles_px * tiles_n;
-  const int cchunks = p.Cin / 64;                         // 64-channel chunks per tap
-  const int kchunks = p.ksize * p.ksize * cchunks;        // k-chunks in tap-major order
-  const int kstages = (kchunks + KCH - 1) / KCH;
   constexpr uint32_t TMEM_COLS = (2 * BN < 32) ? 32 : 2 * BN;
 
   if (threadIdx.x == 0) {
@@ -102,6 +99,14 @@ conv_igemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_co
   const uint32_t tmem = *tmem_slot;
   ptx::pdl_wait();
   ptx::pdl_launch();
+  int n_img = p.n_img;
+  if (p.n_img_ptr) n_img = min(p.n_img, max(0, p.cnt_a + p.cnt_b * static_cast<int>(*p.n_img_ptr)));
+  const int tiles_w = (p.Wo + p.TW - 1) / p.TW, tiles_h = (p.Ho + p.TH - 1) / p.TH;
+  const int tiles_px = tiles_w * tiles_h * n_img;
+  const int num_tiles = tiles_px * ((p.Cout + BN - 1) / BN);
+  const int cchunks = p.Cin / 64;                         // 64-channel chunks per tap
+  const int kchunks = p.ksize * p.ksize * cchunks;        // k-chunks in tap-major order
+  const int kstages = (kchunks + KCH - 1) / KCH;
 
   // tile index -> (channel tile, image, patch origin); pixel tiles vary fastest so that CTAs running
   // together share the weight tile in L2
@@ -359,6 +364,134 @@ __global__ void __launch_bounds__(256) gap_final_f64(GapParams p, int n_img) {
     if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[i] = __double2bfloat16(mean);
     else reinterpret_cast<float*>(p.out)[i] = static_cast<float>(mean);
   }
+}
+
+// [rows, K] -> [rows, Kp] with zero padding (weights of thin-channel convolutions).
+__global__ void __launch_bounds__(256) pad_rows_bf16(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out, int rows, int K, int Kp) {
+  const long long total = static_cast<long long>(rows) * Kp;
+  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const int kk = static_cast<int>(i % Kp);
+    out[i] = kk < K ? in[(i / Kp) * K + kk] : __float2bfloat16(0.0f);
+  }
+}
+
+// Patch gathering for a thin-channel convolution (e.g. the RGB stem): A[pixel, (ci, dy, dx)] from an
+// NCHW image, zero outside the image and in the K padding.  One thread per (pixel, 8-wide k group).
+struct Im2colParams {
+  const __nv_bfloat16* x;   // [N, C, H, W]
+  __nv_bfloat16* a;         // [N*Ho*Wo, Kp]
+  int N, C, H, W, Ho, Wo, ks, stride, pad, K, Kp;
+};
+__global__ void __launch_bounds__(256) im2col_nchw_bf16(Im2colParams p) {
+  const int groups = p.Kp >> 3;
+  const long long total = static_cast<long long>(p.N) * p.Ho * p.Wo * groups;
+  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const int gq = static_cast<int>(i % groups);
+    long long pix = i / groups;
+    const int wo = static_cast<int>(pix % p.Wo);
+    const int ho = static_cast<int>((pix / p.Wo) % p.Ho);
+    const int n = static_cast<int>(pix / (static_cast<long long>(p.Wo) * p.Ho));
+    __align__(16) __nv_bfloat16 v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int kk = gq * 8 + j;
+      float val = 0.0f;
+      if (kk < p.K) {
+        const int dx = kk % p.ks, dy = (kk / p.ks) % p.ks, ci = kk / (p.ks * p.ks);
+        const int h = ho * p.stride + dy - p.pad, w = wo * p.stride + dx - p.pad;
+        if (h >= 0 && h < p.H && w >= 0 && w < p.W) val = __bfloat162float(p.x[((static_cast<long long>(n) * p.C + ci) * p.H + h) * p.W + w]);
+      }
+      v[j] = __float2bfloat16(val);
+    }
+    *reinterpret_cast<uint4*>(p.a + pix * p.Kp + gq * 8) = *reinterpret_cast<const uint4*>(v);
+  }
+}
+
+// Gate of a skip block (decision scalar): z[n] = sum_c w[c] * mean_hw x[n,:,:,c] + b, gate[n] = z[n] > 0,
+// all in fp64 from the bf16 values, so the decision does not depend on the summation order beyond 2^-53.
+// Runs after gap_partial_f64 (slab sums in scratch); one CTA per image.
+struct GateParams {
+  const double* partial;        // [N, slabs, C]
+  const __nv_bfloat16* w;       // [C]
+  const __nv_bfloat16* b;       // [1]
+  unsigned char* gate;          // [N] bytes (0/1)
+  void* z_out;                  // optional logits [N] (bf16 or f32), may be nullptr
+  int z_bf16;
+  int C, slabs;
+  long long HW;
+};
+__global__ void __launch_bounds__(256) gate_logit_f64(GateParams p) {
+  __shared__ double red[256];
+  ptx::pdl_wait();
+  ptx::pdl_launch();
+  const int img = blockIdx.x;
+  double acc = 0.0;
+  for (int c = threadIdx.x; c < p.C; c += 256) {
+    double s = 0.0;
+    for (int k = 0; k < p.slabs; ++k) s += p.partial[(static_cast<long long>(img) * p.slabs + k) * p.C + c];
+    acc += (s / static_cast<double>(p.HW)) * static_cast<double>(__bfloat162float(p.w[c]));
+  }
+  red[threadIdx.x] = acc;
+  __syncthreads();
+  for (int o = 128; o; o >>= 1) { if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o]; __syncthreads(); }
+  if (threadIdx.x == 0) {
+    const double z = red[0] + static_cast<double>(__bfloat162float(p.b[0]));
+    p.gate[img] = z > 0.0 ? 1 : 0;
+    if (p.z_out) {
+      if (p.z_bf16) reinterpret_cast<__nv_bfloat16*>(p.z_out)[img] = __double2bfloat16(z);
+      else reinterpret_cast<float*>(p.z_out)[img] = static_cast<float>(z);
+    }
+  }
+}
+
+// Per-sample regrouping (Switch): stable partition of the sample ids by the gate.  One warp-sized CTA:
+// ballot + prefix popcount per chunk of 32 samples.  *count_exec = executed (the run-time symbol's
+// slot in the arena header), *count_skip = skipped; idx_exec / idx_skip = original sample ids.
+struct PartitionParams {
+  const unsigned char* gate;
+  int n;
+  int* idx_exec; int* idx_skip;    // scratch [n] each
+  long long* count_exec;           // the run-time symbol's slot in the arena header
+  long long* count_skip;
+};
+__global__ void __launch_bounds__(32) gate_partition(PartitionParams p) {
+  ptx::pdl_wait();
+  ptx::pdl_launch();
+  const int lane = threadIdx.x;
+  int ne = 0, ns = 0;
+  for (int base = 0; base < p.n; base += 32) {
+    const int i = base + lane;
+    const bool in = i < p.n;
+    const bool g = in && p.gate[i] != 0;
+    const unsigned be = __ballot_sync(0xffffffffu, g), bs = __ballot_sync(0xffffffffu, in && !g);
+    const unsigned lower = (1u << lane) - 1;
+    if (g) p.idx_exec[ne + __popc(be & lower)] = i;
+    else if (in) p.idx_skip[ns + __popc(bs & lower)] = i;
+    ne += __popc(be);
+    ns += __popc(bs);
+  }
+  if (lane == 0) { *p.count_exec = ne; *p.count_skip = ns; }
+}
+
+// Sample gather / scatter for Switch and Combine: whole per-sample blocks (channels-last, contiguous)
+// copied with 128-bit accesses.  dst[j] = src[idx[j]] (gather) or dst[idx[j]] = src[j] (scatter) for
+// j < *count; grid.y walks the samples, tail blocks exit on the device-side count.
+struct SampleCopyParams {
+  const uint4* src; uint4* dst;
+  const int* idx;
+  const long long* count;
+  long long vec_per_sample;   // 16-byte units per sample
+  int scatter;
+};
+__global__ void __launch_bounds__(256) sample_copy(SampleCopyParams p) {
+  ptx::pdl_wait();
+  ptx::pdl_launch();
+  const int j = blockIdx.y;
+  if (j >= *p.count) return;
+  const long long s = p.idx[j];
+  const uint4* src = p.src + (p.scatter ? static_cast<long long>(j) : s) * p.vec_per_sample;
+  uint4* dst = p.dst + (p.scatter ? s : static_cast<long long>(j)) * p.vec_per_sample;
+  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < p.vec_per_sample; i += static_cast<long long>(gridDim.x) * blockDim.x) dst[i] = src[i];
 }
 
 // Conv weights [Cout, Cin, kh, kw] -> K-major [Cout, (dy, dx, ci)] for the implicit-GEMM B operand.

@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstring>
 #include <functional>
+#include <map>
 
 #include "attention.cuh"
 #include "conv_tcgen05.cuh"
@@ -539,6 +540,66 @@ struct Builder {
     return OK;
   }
 
+  // ------------------------------------------------------------------------------ thin-channel convolution
+  // (e.g. the RGB stem): patches are gathered into an [pixels, Kp] matrix in scratch, then the GEMM
+  // kernel runs with the fused bias / activation epilogue; its [pixels, Cout] output is channels-last.
+  Status build_conv_im2col(int gi, const Group& G) {
+    const Tensor& W = g.tensors[G.w];
+    const int Cout = static_cast<int>(W.S.dims[0].e.const_value()), Cin = static_cast<int>(W.S.dims[1].e.const_value());
+    const int ks = static_cast<int>(W.S.dims[2].e.const_value());
+    if (G.res >= 0 || G.act2 || G.has_ln) return fail(E_UNSUPPORTED_OP, "thin-channel convolution: unsupported epilogue tail");
+    if (Cout % 8) return fail(E_UNSUPPORTED_OP, "thin-channel convolution needs Cout % 8 == 0");
+    size_t pk = 0;
+    for (size_t i = 0; i < c.packed_consts.size(); ++i) if (c.packed_consts[i] == G.w) pk = c.packed_off[i];
+    const int K = Cin * ks * ks, Kp = (K + 63) / 64 * 64;
+    for (int r = 0; r < p.n_req; ++r) {
+      const View &vx = p.views[G.a][r], &vo = p.views[G.out][r];
+      if (!numel(vo.dims)) continue;
+      if (!vx.contiguous()) return fail(E_UNSUPPORTED_OP, "thin-channel convolution reads an NCHW-contiguous input");
+      if (!is_channels_last(vo)) return fail(E_UNSUPPORTED_OP, "convolution output must be stored channels-last");
+      k::Im2colParams ip{};
+      ip.N = static_cast<int>(vx.dims[0]); ip.C = Cin; ip.H = static_cast<int>(vx.dims[2]); ip.W = static_cast<int>(vx.dims[3]);
+      ip.Ho = static_cast<int>(vo.dims[2]); ip.Wo = static_cast<int>(vo.dims[3]);
+      ip.ks = ks; ip.stride = G.stride; ip.pad = G.pad; ip.K = K; ip.Kp = Kp;
+      const long long M = static_cast<long long>(ip.N) * ip.Ho * ip.Wo;
+      scratch_need = std::max(scratch_need, static_cast<size_t>(M) * Kp * 2);
+      Ptr px = ptr_of(G.a, r), po = ptr_of(G.out, r), pb = G.bias >= 0 ? ptr_of(G.bias, 0) : Ptr();
+      Ptr pw; pw.where = 5; pw.off = static_cast<int64_t>(pk);
+      const bool hb = G.bias >= 0;
+      const int act = G.act;
+      struct Cache { const void* a = nullptr; const void* w = nullptr; const void* o = nullptr; CUtensorMap ta, tb, to; };
+      auto cache = std::make_shared<Cache>();
+      add(gi, 2, [=](const RunCtx& x) mutable {
+        ip.x = reinterpret_cast<const __nv_bfloat16*>(x.resolve(px));
+        ip.a = reinterpret_cast<__nv_bfloat16*>(x.arena + x.plan->scratch_off[0]);
+        k::im2col_nchw_bf16<<<148 * 8, 256, 0, x.stream>>>(ip);
+        const void* Wp = x.resolve(pw);
+        void* O = x.resolve(po);
+        if (cache->a != ip.a || cache->w != Wp || cache->o != O) {
+          if (!encode_bf16_kchunks(&cache->ta, ip.a, M, Kp, Kp, 128, 2) || !encode_bf16_kchunks(&cache->tb, Wp, Cout, Kp, Kp, 128, 2) ||
+              !encode_bf16_2d(&cache->to, O, M, Cout, Cout, 128))
+            return cudaErrorInvalidValue;
+          cache->a = ip.a; cache->w = Wp; cache->o = O;
+        }
+        k::GemmEpilogue ep{};
+        ep.bias = hb ? reinterpret_cast<const __nv_bfloat16*>(x.resolve(pb)) : nullptr;
+        ep.status = reinterpret_cast<int*>(x.arena);
+        const long long tiles = ((M + 127) / 128) * ((Cout + 127) / 128);
+        const dim3 gd(static_cast<unsigned>(std::min<long long>(tiles, x.plan->sm_count))), bd(k::GEMM_THREADS);
+        constexpr int smem = k::GemmSmem<128, 2, 3>::TOTAL;
+        if (act == 2) {
+          cudaFuncSetAttribute(k::gemm_bf16_tcgen05<128, 2, 3, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+          launch_pdl(k::gemm_bf16_tcgen05<128, 2, 3, 2>, gd, bd, smem, x.stream, cache->ta, cache->tb, cache->to, cache->to, static_cast<int>(M), Cout, Kp, ep);
+        } else {
+          cudaFuncSetAttribute(k::gemm_bf16_tcgen05<128, 2, 3, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+          launch_pdl(k::gemm_bf16_tcgen05<128, 2, 3, 0>, gd, bd, smem, x.stream, cache->ta, cache->tb, cache->to, cache->to, static_cast<int>(M), Cout, Kp, ep);
+        }
+        return cudaGetLastError();
+      });
+    }
+    return OK;
+  }
+
   // ------------------------------------------------------------------------------ convolution
   Status build_conv(int gi, const Group& G) {
     const Tensor& W = g.tensors[G.w];
@@ -546,7 +607,7 @@ struct Builder {
     const int Cout = static_cast<int>(W.S.dims[0].e.const_value()), Cin = static_cast<int>(W.S.dims[1].e.const_value());
     const int ks = static_cast<int>(W.S.dims[2].e.const_value());
     if (W.S.dims[3].e.const_value() != ks) return fail(E_UNSUPPORTED_OP, "convolution needs a square kernel");
-    if (Cin % 64) return fail(E_UNSUPPORTED_OP, "implicit-GEMM convolution needs Cin % 64 == 0");
+    if (Cin % 64) return build_conv_im2col(gi, G);
     if (Cout % 64) return fail(E_UNSUPPORTED_OP, "implicit-GEMM convolution needs Cout % 64 == 0");
     if (G.has_ln || (G.act != 0 && G.act != 2)) return fail(E_UNSUPPORTED_OP, "convolution epilogue: unsupported tail");
     size_t pk = 0;
@@ -565,6 +626,10 @@ struct Builder {
       cp.Cin = Cin; cp.Cout = Cout; cp.ksize = ks; cp.stride = G.stride; cp.pad = G.pad;
       cp.has_residual = G.res >= 0;
       cp.act2 = G.act2;
+      const RtCount rc = runtime_count(G.out, r);
+      cp.cnt_a = rc.a; cp.cnt_b = rc.b;
+      const bool rt = rc.rt;
+      const size_t rt_slot = rc.slot_off;
       // pixel patch of a tile: the 128-pixel shape that wastes the fewest padded pixels
       long long best = -1;
       for (int tw : {128, 64, 32, 16, 8}) {
@@ -598,6 +663,7 @@ struct Builder {
         }
         cp.bias = hb ? reinterpret_cast<const __nv_bfloat16*>(x.resolve(pb)) : nullptr;
         cp.status = reinterpret_cast<int*>(x.arena);
+        cp.n_img_ptr = rt ? reinterpret_cast<const long long*>(x.arena + rt_slot) : nullptr;
         const dim3 gd(static_cast<unsigned>(std::min<long long>(tiles, x.plan->sm_count))), bd(k::CONV_THREADS);
         const int variant = (bn == 128 ? 2 : 0) + (act == 2 ? 1 : 0);
 #define SOD2_CONV_CASE(V, BN_, KCH_, ST_, ACT_)                                                                          \
@@ -620,6 +686,153 @@ struct Builder {
         return cudaGetLastError();
       });
     }
+    return OK;
+  }
+
+  // ------------------------------------------------------------------------------ run-time sample counts
+  // A tensor whose leading extent is execution determined (gated sub-batch): extent = a + b * count,
+  // where count is the run-time symbol's slot in the arena header, written by the Switch group.
+  struct RtCount { bool rt = false; size_t slot_off = 0; int a = 0, b = 0; };
+  RtCount runtime_count(int t, int r) const {
+    RtCount rc;
+    const ShapeVal& s = g.tensors[t].S;
+    if (s.rank < 1 || !s.dims[0].known() || !e_has_runtime(g.cx, s.dims[0].e)) return rc;
+    int sym = -1;
+    for (auto& term : s.dims[0].e.terms)
+      for (auto& pw : term.first)
+        if (g.cx.atoms[pw.first].kind == AtomKind::SYM && g.cx.atoms[pw.first].runtime) sym = pw.first;
+    if (sym < 0) return rc;
+    std::vector<int64_t> vals = p.b->vals[r];
+    bool ok0, ok1;
+    vals[sym] = 0;
+    const int64_t v0 = e_eval(g.cx, s.dims[0].e, vals, &ok0);
+    vals[sym] = 1;
+    const int64_t v1 = e_eval(g.cx, s.dims[0].e, vals, &ok1);
+    if (!ok0 || !ok1) return rc;
+    rc.rt = true;
+    rc.slot_off = 256 + (static_cast<size_t>(sym) * p.n_req + r) * 8;
+    rc.a = static_cast<int>(v0);
+    rc.b = static_cast<int>(v1 - v0);
+    return rc;
+  }
+  // persistent side storage of a Switch (index lists), found again by the Combine through the gate tensor
+  std::map<int, size_t> switch_aux;   // gate tensor -> offset inside the aux region
+  size_t aux_need = 0;
+
+  // ------------------------------------------------------------------------------ gate (decision scalar)
+  Status build_gate(int gi, const Group& G) {
+    if (g.tensors[G.a].dtype != DType::BF16) return fail(E_UNSUPPORTED_OP, "gate is bf16 only");
+    const bool want_z = std::find(G.ext_out.begin(), G.ext_out.end(), G.out2) != G.ext_out.end();
+    for (int r = 0; r < p.n_req; ++r) {
+      const View& vx = p.views[G.a][r];
+      if (!numel(vx.dims)) continue;
+      if (!is_channels_last(vx)) return fail(E_UNSUPPORTED_OP, "gate reads channels-last storage");
+      k::GapParams gp{};
+      gp.C = static_cast<int>(vx.dims[1]);
+      gp.HW = vx.dims[2] * vx.dims[3];
+      gp.slabs = static_cast<int>(std::max<long long>(1, std::min<long long>(64, gp.HW / 64)));
+      const int N = static_cast<int>(vx.dims[0]);
+      scratch_need = std::max(scratch_need, static_cast<size_t>(N) * gp.slabs * gp.C * 8);
+      Ptr px = ptr_of(G.a, r), pw = ptr_of(G.w, 0), pb = ptr_of(G.bias, 0), pg = ptr_of(G.out, r);
+      Ptr pz = want_z ? ptr_of(G.out2, r) : Ptr();
+      const bool zb = want_z && g.tensors[G.out2].dtype == DType::BF16;
+      add(gi, 2, [=](const RunCtx& x) mutable {
+        gp.x = reinterpret_cast<const __nv_bfloat16*>(x.resolve(px));
+        gp.partial = reinterpret_cast<double*>(x.arena + x.plan->scratch_off[0]);
+        launch_pdl(k::gap_partial_f64, dim3((gp.C + 63) / 64, gp.slabs, N), dim3(256), 0, x.stream, gp);
+        k::GateParams q{};
+        q.partial = gp.partial;
+        q.w = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pw));
+        q.b = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pb));
+        q.gate = reinterpret_cast<unsigned char*>(x.resolve(pg));
+        q.z_out = want_z ? x.resolve(pz) : nullptr;
+        q.z_bf16 = zb;
+        q.C = gp.C; q.slabs = gp.slabs; q.HW = gp.HW;
+        launch_pdl(k::gate_logit_f64, dim3(N), dim3(256), 0, x.stream, q);
+        return cudaGetLastError();
+      });
+    }
+    return OK;
+  }
+
+  // ------------------------------------------------------------------------------ Switch / Combine
+  Status build_switch(int gi, const Group& G) {
+    if (p.n_req != 1) return fail(E_UNSUPPORTED_OP, "Switch/Combine graphs carry the batch inside the graph: bind one request");
+    const View& vx = p.views[G.a][0];
+    if (vx.dims.size() != 4 || !is_channels_last(vx)) return fail(E_UNSUPPORTED_OP, "Switch regroups channels-last samples");
+    const int N = static_cast<int>(vx.dims[0]);
+    const long long bytes = vx.dims[1] * vx.dims[2] * vx.dims[3] * dtype_size(g.tensors[G.a].dtype);
+    if (bytes % 16) return fail(E_UNSUPPORTED_OP, "Switch: sample size must be a multiple of 16 bytes");
+    RtCount rc = runtime_count(G.out, 0);
+    if (!rc.rt || rc.a != 0 || rc.b != 1) return fail(E_INTERNAL, "Switch output has no run-time count");
+    const size_t aux = aux_need;
+    switch_aux[G.gate] = aux;
+    aux_need += (static_cast<size_t>(2 * N) * 4 + 16 + 255) & ~size_t(255);
+    Ptr px = ptr_of(G.a, 0), pg = ptr_of(G.gate, 0), pe = ptr_of(G.out, 0);
+    const bool has_skip = G.out2 >= 0 && !p.views[G.out2][0].dims.empty();
+    Ptr ps = has_skip ? ptr_of(G.out2, 0) : Ptr();
+    const size_t slot = rc.slot_off;
+    add(gi, has_skip ? 3 : 2, [=](const RunCtx& x) {
+      char* auxp = x.arena + x.plan->scratch_off[1] + aux;
+      k::PartitionParams pp{};
+      pp.gate = reinterpret_cast<const unsigned char*>(x.resolve(pg));
+      pp.n = N;
+      pp.idx_exec = reinterpret_cast<int*>(auxp);
+      pp.idx_skip = pp.idx_exec + N;
+      pp.count_exec = reinterpret_cast<long long*>(x.arena + slot);
+      pp.count_skip = reinterpret_cast<long long*>(auxp + 2 * N * 4);
+      launch_pdl(k::gate_partition, dim3(1), dim3(32), 0, x.stream, pp);
+      k::SampleCopyParams sc{};
+      sc.src = reinterpret_cast<const uint4*>(x.resolve(px));
+      sc.vec_per_sample = bytes / 16;
+      sc.scatter = 0;
+      const unsigned gx = static_cast<unsigned>(std::max<long long>(1, std::min<long long>(64, sc.vec_per_sample / 256)));
+      sc.dst = reinterpret_cast<uint4*>(x.resolve(pe));
+      sc.idx = pp.idx_exec;
+      sc.count = pp.count_exec;
+      launch_pdl(k::sample_copy, dim3(gx, N), dim3(256), 0, x.stream, sc);
+      if (has_skip) {
+        sc.dst = reinterpret_cast<uint4*>(x.resolve(ps));
+        sc.idx = pp.idx_skip;
+        sc.count = pp.count_skip;
+        launch_pdl(k::sample_copy, dim3(gx, N), dim3(256), 0, x.stream, sc);
+      }
+      return cudaGetLastError();
+    });
+    return OK;
+  }
+
+  Status build_combine(int gi, const Group& G) {
+    if (p.n_req != 1) return fail(E_UNSUPPORTED_OP, "Switch/Combine graphs carry the batch inside the graph: bind one request");
+    auto it = switch_aux.find(G.gate);
+    if (it == switch_aux.end()) return fail(E_INTERNAL, "Combine without a Switch on the same gate");
+    const size_t aux = it->second;
+    const View& vy = p.views[G.out][0];
+    if (vy.dims.size() != 4 || !is_channels_last(vy)) return fail(E_UNSUPPORTED_OP, "Combine writes channels-last samples");
+    const int N = static_cast<int>(vy.dims[0]);
+    const long long bytes = vy.dims[1] * vy.dims[2] * vy.dims[3] * dtype_size(g.tensors[G.out].dtype);
+    if (bytes % 16) return fail(E_UNSUPPORTED_OP, "Combine: sample size must be a multiple of 16 bytes");
+    RtCount rc = runtime_count(G.a, 0);
+    if (!rc.rt) return fail(E_INTERNAL, "Combine input has no run-time count");
+    Ptr pe = ptr_of(G.a, 0), ps = ptr_of(G.res, 0), py = ptr_of(G.out, 0);
+    const size_t slot = rc.slot_off;
+    add(gi, 2, [=](const RunCtx& x) {
+      char* auxp = x.arena + x.plan->scratch_off[1] + aux;
+      k::SampleCopyParams sc{};
+      sc.dst = reinterpret_cast<uint4*>(x.resolve(py));
+      sc.vec_per_sample = bytes / 16;
+      sc.scatter = 1;
+      const unsigned gx = static_cast<unsigned>(std::max<long long>(1, std::min<long long>(64, sc.vec_per_sample / 256)));
+      sc.src = reinterpret_cast<const uint4*>(x.resolve(pe));
+      sc.idx = reinterpret_cast<const int*>(auxp);
+      sc.count = reinterpret_cast<const long long*>(x.arena + slot);
+      launch_pdl(k::sample_copy, dim3(gx, N), dim3(256), 0, x.stream, sc);
+      sc.src = reinterpret_cast<const uint4*>(x.resolve(ps));
+      sc.idx = reinterpret_cast<const int*>(auxp) + N;
+      sc.count = reinterpret_cast<const long long*>(auxp + 2 * N * 4);
+      launch_pdl(k::sample_copy, dim3(gx, N), dim3(256), 0, x.stream, sc);
+      return cudaGetLastError();
+    });
     return OK;
   }
 
@@ -705,14 +918,19 @@ struct Builder {
         case GKind::LAYOUT: s = build_layout(static_cast<int>(gi), G); break;
         case GKind::CONV: s = build_conv(static_cast<int>(gi), G); break;
         case GKind::GAP: s = build_gap(static_cast<int>(gi), G); break;
+        case GKind::GATE: s = build_gate(static_cast<int>(gi), G); break;
+        case GKind::SWITCH: s = build_switch(static_cast<int>(gi), G); break;
+        case GKind::COMBINE: s = build_combine(static_cast<int>(gi), G); break;
         default: return fail(E_UNSUPPORTED_OP, std::string("no executor yet for group kind ") + gkind_name(G.kind));
       }
       if (s != OK) return s;
       cost(G);
     }
     // one scratch region shared by all groups (they run in stream order), after the tensors
-    p.scratch_off.assign(1, p.arena_bytes);
+    p.scratch_off.assign(2, p.arena_bytes);
     p.arena_bytes += (scratch_need + 255) & ~size_t(255);
+    p.scratch_off[1] = p.arena_bytes;     // index lists of Switch groups: live until their Combine
+    p.arena_bytes += (aux_need + 255) & ~size_t(255);
     return OK;
   }
 };
@@ -749,6 +967,12 @@ Status prepack_weights(Compiled* c, void* workspace, size_t bytes, void* stream)
     if (W.S.rank == 4) {  // convolution weights [Cout, Cin, kh, kw] -> [Cout, (dy, dx, ci)]
       const int co = static_cast<int>(W.S.dims[0].e.const_value()), ci = static_cast<int>(W.S.dims[1].e.const_value());
       const int kh = static_cast<int>(W.S.dims[2].e.const_value()), kw = static_cast<int>(W.S.dims[3].e.const_value());
+      if (ci % 64) {  // thin-channel convolution (im2col path): keep the (ci, dy, dx) order, pad K with zeros
+        const int K = ci * kh * kw, Kp = (K + 63) / 64 * 64;
+        k::pad_rows_bf16<<<148 * 2, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+            static_cast<const __nv_bfloat16*>(W.dev_ptr), reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + c->packed_off[i]), co, K, Kp);
+        continue;
+      }
       k::reorder_conv_weights<<<148 * 4, 256, 0, static_cast<cudaStream_t>(stream)>>>(
           static_cast<const __nv_bfloat16*>(W.dev_ptr), reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + c->packed_off[i]), co, ci, kh, kw);
       continue;

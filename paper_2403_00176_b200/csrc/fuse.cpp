@@ -246,7 +246,7 @@ struct Fuser {
     if (g.tensors[thr].kind != TKind::FCONST || g.tensors[thr].fdata != 0.0) return false;
     Group G;
     G.kind = GKind::GATE;
-    G.nodes = {nid, mm, ad, gr};
+    G.nodes = {nid, r, mm, ad, gr};
     G.a = n.ins[0]; G.w = g.nodes[mm].ins[1]; G.bias = bias; G.out = g.nodes[gr].outs[0]; G.out2 = z;
     c.node_folded[r] = 1;  // the Reshape of the pooled vector lives inside the group
     finish(G);
@@ -487,8 +487,10 @@ struct Fuser {
         if (std::find(c.packed_consts.begin(), c.packed_consts.end(), G2.w) == c.packed_consts.end()) {
           c.packed_consts.push_back(G2.w);
           c.packed_off.push_back(c.packed_bytes);
-          size_t bytes = 2;
-          for (auto& d : g.tensors[G2.w].S.dims) bytes *= static_cast<size_t>(d.e.const_value());
+          const auto& wd = g.tensors[G2.w].S.dims;
+          size_t kk = static_cast<size_t>(wd[1].e.const_value() * wd[2].e.const_value() * wd[3].e.const_value());
+          kk = (kk + 63) / 64 * 64;   // thin-channel convolutions pad K to a whole k-chunk
+          const size_t bytes = static_cast<size_t>(wd[0].e.const_value()) * kk * 2;
           c.packed_bytes += (bytes + 255) & ~size_t(255);
         }
       }

@@ -314,6 +314,8 @@ void insert_layout_nodes(Graph* g) {
     bool feeds_conv = false;
     for (int c : T.consumers) if (g->nodes[c].op == "Conv" && g->nodes[c].ins[0] == t) feeds_conv = true;
     if (!feeds_conv) continue;
+    // a thin-channel image (e.g. RGB) stays NCHW: its convolution gathers patches itself (im2col)
+    if (!T.S.dims[1].known() || !T.S.dims[1].e.is_const() || T.S.dims[1].e.const_value() % 64) continue;
     int cl = new_tensor(g, T.name + "@cl");
     g->tensors[cl].dtype = g->tensors[t].dtype;
     std::vector<int> cons = g->tensors[t].consumers;

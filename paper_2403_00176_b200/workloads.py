@@ -24,6 +24,7 @@ top-k token pruning, per-sample skip gates); values are synthetic.
 from __future__ import annotations
 
 import dataclasses
+import os
 from typing import Dict, List
 
 import numpy as np
@@ -367,7 +368,8 @@ def cfg4(blocks: int = 8, C: int = 64, n_requests: int = 4, side_lo: int = 224, 
 
 
 # --------------------------------------------------------------------------- cfg 5
-def cfg5(B: int = 32, side: int = 224, widths=(64, 128, 256, 512), per_stage: int = 4, cin: int = 3) -> Workload:
+def cfg5(B: int = 32, side: int = 224, widths=(64, 128, 256, 512), per_stage: int = 4, cin: int = 3,
+         calibrated: bool = True) -> Workload:
     """Gated skip network.  Stem conv7x7/2, then residual blocks; each block has a per-sample
     gate (linear on the global average pool, compared with 0).  Samples are regrouped by
     the gate (Switch), only the gated subset runs the block, Combine restores sample order."""
@@ -436,6 +438,14 @@ def cfg5(B: int = 32, side: int = 224, widths=(64, 128, 256, 512), per_stage: in
         else:
             a = rw.standard_normal(shape) * 0.05
         consts[name] = bf16_round(a.astype(np.float32))
+    # gate biases calibrated (by a script that runs only the oracle) so that about 40-70 % of a
+    # calibration batch skips each block; they apply to the default network only
+    cal = os.path.join(os.path.dirname(os.path.abspath(__file__)), "cfg5_gate_bias.txt")
+    if calibrated and os.path.exists(cal) and (side, tuple(widths), per_stage, cin) == (224, (64, 128, 256, 512), 4, 3):
+        vals = [float(ln) for ln in open(cal) if ln.strip() and not ln.startswith("#")]
+        for i, v in enumerate(vals):
+            if f"b{i}.gb" in consts:
+                consts[f"b{i}.gb"] = bf16_round(np.array([v], np.float32))
 
     def batch_fn(j: int) -> List[Request]:
         r = _rng(5, j)

@@ -26,9 +26,11 @@ def materialised(sess, prep, graph):
         for o in nd.outs:
             try:
                 prep.plan.slot(o)
-                names.append(o)
             except B.Sod2Error:
-                pass
+                continue
+            if 4 in sess.graph.tensor_info(o)[1]:
+                continue        # execution-determined extent: the arena slot is sized for the upper bound
+            names.append(o)
     return names
 
 

@@ -227,3 +227,69 @@ def test_cfg4_full_config_smallest_request_and_properties():
         y = outs[r][last].astype(np.float64)
         assert y.shape == (1, 64, reqs[r].syms["H"], reqs[r].syms["W"]) and np.all(np.isfinite(y))
         assert np.allclose(outs[r]["gap"].reshape(-1), y.mean(axis=(2, 3)).reshape(-1), rtol=1e-2, atol=1e-2)
+
+
+# ------------------------------------------------------------------------------------------------ cfg 5
+def _check_gated(wl, reqs, n_blocks):
+    s, p, outs = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE)
+    req = reqs[0]
+    env = O.run(wl.ir, wl.consts, req.inputs)
+    # lock-step: every full-batch tensor (stem, block outputs, gates) from the GPU's own inputs
+    errs = lockstep(wl, s, p, outs, 0, BF16_TOL)
+    assert any(k.startswith("blk") for k in errs)
+    bad = {k: v for k, v in errs.items() if not (isinstance(v, float) and v <= BF16_TOL)}
+    assert not bad, bad
+    gates = np.stack([outs[0][f"gate{i}"].reshape(-1) for i in range(n_blocks)])
+    # gate decisions recomputed by the oracle from the GPU's own block inputs must match bit-exactly
+    g = O.parse(wl.ir)
+    over = {n: p.read_arena_tensor(n, 0).astype(np.float64) for n in ["stem"] + [f"blk{i}" for i in range(n_blocks - 1)]}
+    comp = {}
+    env2 = O.run(wl.ir, wl.consts, req.inputs, overrides=over, g=g, computed=comp)
+    for i in range(n_blocks):
+        assert np.array_equal(outs[0][f"gate{i}"].reshape(-1).astype(bool), env2[f"gate{i}"].reshape(-1)), i
+    assert O.rel_err(outs[0]["gap"], env2["gap"]) <= BF16_TOL
+    # free-running agreement (information + sanity): same decisions unless a logit is within rounding noise
+    free = np.stack([env[f"gate{i}"].reshape(-1) for i in range(n_blocks)])
+    assert (gates.astype(bool) == free).mean() >= 0.9
+    return gates
+
+
+def test_cfg5_small_gated_network_lockstep():
+    wl = WL.cfg5(B=6, side=32, widths=(64, 128), per_stage=2)
+    gates = _check_gated(wl, wl.batch(0), 4)
+    assert gates.shape == (4, 6)
+
+
+def test_cfg5_all_skip_and_all_execute():
+    # degenerate gate batches: nothing executes (Bx = 0 launches no tile) / everything executes
+    for bias_val in (-50.0, 50.0):
+        wl = WL.cfg5(B=4, side=32, widths=(64, 128), per_stage=2)
+        for k in list(wl.consts):
+            if k.endswith(".gb"):
+                wl.consts[k] = np.full_like(wl.consts[k], bias_val)
+        gates = _check_gated(wl, wl.batch(1), 4)
+        assert np.all(gates == (1 if bias_val > 0 else 0))
+
+
+def test_cfg5_full_depth_reduced_batch_lockstep():
+    # all 16 blocks and widths 64..512 at 224x224, 4 images (the oracle needs ~100 GFLOP in fp64)
+    wl = WL.cfg5(B=4)
+    gates = _check_gated(wl, wl.batch(0), 16)
+    assert gates.shape == (16, 4)
+
+
+def test_cfg5_full_config_properties():
+    wl = WL.cfg5()
+    reqs = wl.batch(0)
+    s, p, outs = run_batch(wl, reqs)
+    assert s.graph.num_subgraphs() == 33
+    gates = np.stack([outs[0][f"gate{i}"].reshape(-1) for i in range(16)])
+    assert gates.shape == (16, 32) and set(np.unique(gates)) <= {0, 1}
+    assert np.all(np.isfinite(outs[0]["gap"])) and outs[0]["gap"].shape == (32, 512, 1, 1)
+    assert 0.05 < gates.mean() < 0.95          # both branches are exercised
+    p.run()
+    outs2 = p.outputs()
+    assert np.array_equal(outs[0]["gap"], outs2[0]["gap"])
+    for i in range(16):
+        assert np.array_equal(outs[0][f"gate{i}"], outs2[0][f"gate{i}"])
+    print("skip fraction per block:", 1 - gates.mean(axis=1))
