@@ -283,40 +283,62 @@ conv_igemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_co
 // groups use internally: [N, C, H*W] <-> [N, H*W, C], 32x32 tiles through shared memory.
 __global__ void __launch_bounds__(256) nchw_to_nhwc_bf16(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out,
                                                           int C, long long HW) {
-  __shared__ __nv_bfloat16 tile[32][34];
+  // tile: 64 channels x 64 pixels; reads are 128-byte pixel runs per channel, writes 128-byte channel runs per pixel
+  __shared__ __nv_bfloat16 tile[64][66];
   const long long img = blockIdx.z;
-  const long long p0 = static_cast<long long>(blockIdx.x) * 32;
-  const int c0 = blockIdx.y * 32;
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  for (int i = ty; i < 32; i += 8) {
-    const int c = c0 + i;
-    const long long px = p0 + tx;
-    if (c < C && px < HW) tile[i][tx] = in[(img * C + c) * HW + px];
+  const long long p0 = static_cast<long long>(blockIdx.x) * 64;
+  const int c0 = blockIdx.y * 64;
+  for (int i = threadIdx.x; i < 64 * 32; i += 256) {       // 64 channels x 32 pixel pairs
+    const int c = i >> 5, pp = (i & 31) * 2;
+    const long long px = p0 + pp;
+    if (c0 + c < C) {
+      const __nv_bfloat16* src = in + (img * C + c0 + c) * HW + px;
+      if (px + 1 < HW && ((reinterpret_cast<uintptr_t>(src) & 3) == 0)) {
+        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(src);
+        tile[c][pp] = v.x; tile[c][pp + 1] = v.y;
+      } else {
+        if (px < HW) tile[c][pp] = src[0];
+        if (px + 1 < HW) tile[c][pp + 1] = src[1];
+      }
+    }
   }
   __syncthreads();
-  for (int i = ty; i < 32; i += 8) {
-    const long long px = p0 + i;
-    const int c = c0 + tx;
-    if (c < C && px < HW) out[(img * HW + px) * C + c] = tile[tx][i];
+  for (int i = threadIdx.x; i < 64 * 32; i += 256) {       // 64 pixels x 32 channel pairs
+    const int pxl = i >> 5, cp = (i & 31) * 2;
+    const long long px = p0 + pxl;
+    if (px < HW && c0 + cp < C) {
+      __nv_bfloat16* dst = out + (img * HW + px) * C + c0 + cp;
+      if (c0 + cp + 1 < C && ((reinterpret_cast<uintptr_t>(dst) & 3) == 0)) *reinterpret_cast<__nv_bfloat162*>(dst) = __nv_bfloat162(tile[cp][pxl], tile[cp + 1][pxl]);
+      else { dst[0] = tile[cp][pxl]; if (c0 + cp + 1 < C) dst[1] = tile[cp + 1][pxl]; }
+    }
   }
 }
 __global__ void __launch_bounds__(256) nhwc_to_nchw_bf16(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out,
                                                           int C, long long HW) {
-  __shared__ __nv_bfloat16 tile[32][34];
+  __shared__ __nv_bfloat16 tile[64][66];   // [pixel][channel]
   const long long img = blockIdx.z;
-  const long long p0 = static_cast<long long>(blockIdx.x) * 32;
-  const int c0 = blockIdx.y * 32;
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  for (int i = ty; i < 32; i += 8) {
-    const long long px = p0 + i;
-    const int c = c0 + tx;
-    if (c < C && px < HW) tile[i][tx] = in[(img * HW + px) * C + c];
+  const long long p0 = static_cast<long long>(blockIdx.x) * 64;
+  const int c0 = blockIdx.y * 64;
+  for (int i = threadIdx.x; i < 64 * 32; i += 256) {
+    const int pxl = i >> 5, cp = (i & 31) * 2;
+    const long long px = p0 + pxl;
+    if (px < HW && c0 + cp < C) {
+      const __nv_bfloat16* src = in + (img * HW + px) * C + c0 + cp;
+      if (c0 + cp + 1 < C && ((reinterpret_cast<uintptr_t>(src) & 3) == 0)) {
+        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(src);
+        tile[pxl][cp] = v.x; tile[pxl][cp + 1] = v.y;
+      } else { tile[pxl][cp] = src[0]; if (c0 + cp + 1 < C) tile[pxl][cp + 1] = src[1]; }
+    }
   }
   __syncthreads();
-  for (int i = ty; i < 32; i += 8) {
-    const int c = c0 + i;
-    const long long px = p0 + tx;
-    if (c < C && px < HW) out[(img * C + c) * HW + px] = tile[tx][i];
+  for (int i = threadIdx.x; i < 64 * 32; i += 256) {
+    const int c = i >> 5, pp = (i & 31) * 2;
+    const long long px = p0 + pp;
+    if (c0 + c < C) {
+      __nv_bfloat16* dst = out + (img * C + c0 + c) * HW + px;
+      if (px + 1 < HW && ((reinterpret_cast<uintptr_t>(dst) & 3) == 0)) *reinterpret_cast<__nv_bfloat162*>(dst) = __nv_bfloat162(tile[pp][c], tile[pp + 1][c]);
+      else { if (px < HW) dst[0] = tile[pp][c]; if (px + 1 < HW) dst[1] = tile[pp + 1][c]; }
+    }
   }
 }
 
@@ -333,36 +355,68 @@ struct GapParams {
   long long HW;
 };
 __global__ void __launch_bounds__(256) gap_partial_f64(GapParams p) {
-  __shared__ double part[4][64];
+  // every thread owns 8 channels (one 16-byte load) of a pixel; C/8 threads cover a pixel, the
+  // remaining factor of the CTA walks pixels; fp64 partial sums, fixed-order reduction in shared memory
+  __shared__ double part[256][8];
   ptx::pdl_wait();
   ptx::pdl_launch();
   const long long img = blockIdx.z;
-  const int c = blockIdx.x * 64 + (threadIdx.x & 63);
-  const int sub = threadIdx.x >> 6;
+  const int tpp = (p.C + 7) >> 3;                 // threads per pixel (C <= 2048)
+  const int ppi = 256 / tpp;                      // pixels per CTA iteration
+  const int cg = threadIdx.x % tpp, pg = threadIdx.x / tpp;
   const long long per = (p.HW + p.slabs - 1) / p.slabs;
   const long long p0 = blockIdx.y * per, p1 = min(p.HW, p0 + per);
-  double acc = 0.0;
-  if (c < p.C)
-    for (long long px = p0 + sub; px < p1; px += 4) acc += static_cast<double>(__bfloat162float(p.x[(img * p.HW + px) * p.C + c]));
-  part[sub][threadIdx.x & 63] = acc;
+  double acc[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) acc[i] = 0.0;
+  if (pg < ppi && (p.C & 7) == 0) {
+    for (long long px = p0 + pg; px < p1; px += ppi) {
+      const uint4 u = *reinterpret_cast<const uint4*>(p.x + (img * p.HW + px) * p.C + cg * 8);
+      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { const float2 f = __bfloat1622float2(h[i]); acc[2 * i] += static_cast<double>(f.x); acc[2 * i + 1] += static_cast<double>(f.y); }
+    }
+  } else if (pg < ppi) {
+    for (long long px = p0 + pg; px < p1; px += ppi)
+      for (int i = 0; i < 8 && cg * 8 + i < p.C; ++i) acc[i] += static_cast<double>(__bfloat162float(p.x[(img * p.HW + px) * p.C + cg * 8 + i]));
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) part[threadIdx.x][i] = acc[i];
   __syncthreads();
-  if (sub == 0 && c < p.C)
-    p.partial[(img * p.slabs + blockIdx.y) * p.C + c] = (part[0][threadIdx.x] + part[1][threadIdx.x]) + (part[2][threadIdx.x] + part[3][threadIdx.x]);
+  if (pg == 0) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      double s = 0.0;
+      for (int g2 = 0; g2 < ppi; ++g2) s += part[g2 * tpp + cg][i];
+      if (cg * 8 + i < p.C) p.partial[(img * p.slabs + blockIdx.y) * p.C + cg * 8 + i] = s;
+    }
+  }
 }
 __global__ void __launch_bounds__(256) gap_final_f64(GapParams p, int n_img) {
+  // 32 channels x 8 slab lanes per CTA: lane g sums slabs g, g+8, ... in order, then the 8 lane sums
+  // are added in order: a fixed summation tree, so the result is deterministic
+  __shared__ double part[8][32];
   ptx::pdl_wait();
   ptx::pdl_launch();
-  const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (i >= static_cast<long long>(n_img) * p.C) return;
-  const long long img = i / p.C;
-  const int c = static_cast<int>(i % p.C);
+  const int cl = threadIdx.x & 31, g = threadIdx.x >> 5;
+  const long long i = static_cast<long long>(blockIdx.x) * 32 + cl;     // flat (img, c)
+  const bool ok = i < static_cast<long long>(n_img) * p.C;
+  const long long img = ok ? i / p.C : 0;
+  const int c = ok ? static_cast<int>(i % p.C) : 0;
   double acc = 0.0;
-  for (int s = 0; s < p.slabs; ++s) acc += p.partial[(img * p.slabs + s) * p.C + c];
-  const double mean = acc / static_cast<double>(p.HW);
-  if (p.out_f64) p.out_f64[i] = mean;
-  if (p.out) {
-    if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[i] = __double2bfloat16(mean);
-    else reinterpret_cast<float*>(p.out)[i] = static_cast<float>(mean);
+  if (ok) for (int s = g; s < p.slabs; s += 8) acc += p.partial[(img * p.slabs + s) * p.C + c];
+  part[g][cl] = acc;
+  __syncthreads();
+  if (g == 0 && ok) {
+    double t = 0.0;
+#pragma unroll
+    for (int k2 = 0; k2 < 8; ++k2) t += part[k2][cl];
+    const double mean = t / static_cast<double>(p.HW);
+    if (p.out_f64) p.out_f64[i] = mean;
+    if (p.out) {
+      if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[i] = __double2bfloat16(mean);
+      else reinterpret_cast<float*>(p.out)[i] = static_cast<float>(mean);
+    }
   }
 }
 
@@ -383,26 +437,41 @@ struct Im2colParams {
   int N, C, H, W, Ho, Wo, ks, stride, pad, K, Kp;
 };
 __global__ void __launch_bounds__(256) im2col_nchw_bf16(Im2colParams p) {
+  // CTA = 64 consecutive output pixels of one output row.  The input window (C x ks rows x span
+  // columns) is staged in shared memory with coalesced reads; every thread then writes 16-byte
+  // groups of the K-major patch rows (coalesced: a pixel's row is Kp*2 contiguous bytes).
+  extern __shared__ __nv_bfloat16 win[];          // [C][ks][span]
+  const int segs = (p.Wo + 63) / 64;
+  const int seg = blockIdx.x % segs;
+  const int ho = (blockIdx.x / segs) % p.Ho;
+  const int n = blockIdx.x / (segs * p.Ho);
+  const int wo0 = seg * 64;
+  const int span = 63 * p.stride + p.ks;          // input columns needed by 64 output pixels
+  const int w_in0 = wo0 * p.stride - p.pad, h_in0 = ho * p.stride - p.pad;
+  const int total = p.C * p.ks * span;
+  for (int i = threadIdx.x; i < total; i += 256) {
+    const int col = i % span, row = (i / span) % p.ks, ci = i / (span * p.ks);
+    const int h = h_in0 + row, w = w_in0 + col;
+    float v = 0.0f;
+    if (h >= 0 && h < p.H && w >= 0 && w < p.W) v = __bfloat162float(p.x[((static_cast<long long>(n) * p.C + ci) * p.H + h) * p.W + w]);
+    win[i] = __float2bfloat16(v);
+  }
+  __syncthreads();
   const int groups = p.Kp >> 3;
-  const long long total = static_cast<long long>(p.N) * p.Ho * p.Wo * groups;
-  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += static_cast<long long>(gridDim.x) * blockDim.x) {
-    const int gq = static_cast<int>(i % groups);
-    long long pix = i / groups;
-    const int wo = static_cast<int>(pix % p.Wo);
-    const int ho = static_cast<int>((pix / p.Wo) % p.Ho);
-    const int n = static_cast<int>(pix / (static_cast<long long>(p.Wo) * p.Ho));
+  for (int i = threadIdx.x; i < 64 * groups; i += 256) {
+    const int gq = i % groups, px = i / groups;
+    const int wo = wo0 + px;
+    if (wo >= p.Wo) continue;
     __align__(16) __nv_bfloat16 v[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const int kk = gq * 8 + j;
-      float val = 0.0f;
       if (kk < p.K) {
         const int dx = kk % p.ks, dy = (kk / p.ks) % p.ks, ci = kk / (p.ks * p.ks);
-        const int h = ho * p.stride + dy - p.pad, w = wo * p.stride + dx - p.pad;
-        if (h >= 0 && h < p.H && w >= 0 && w < p.W) val = __bfloat162float(p.x[((static_cast<long long>(n) * p.C + ci) * p.H + h) * p.W + w]);
-      }
-      v[j] = __float2bfloat16(val);
+        v[j] = win[(ci * p.ks + dy) * span + px * p.stride + dx];
+      } else v[j] = __float2bfloat16(0.0f);
     }
+    const long long pix = (static_cast<long long>(n) * p.Ho + ho) * p.Wo + wo;
     *reinterpret_cast<uint4*>(p.a + pix * p.Kp + gq * 8) = *reinterpret_cast<const uint4*>(v);
   }
 }

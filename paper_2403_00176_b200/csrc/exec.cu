@@ -529,7 +529,7 @@ struct Builder {
       const long long HW = vi.dims[2] * vi.dims[3];
       const bool from = G.act != 0;
       add(gi, 1, [=](const RunCtx& x) {
-        const dim3 grid(static_cast<unsigned>((HW + 31) / 32), (C + 31) / 32, N);
+        const dim3 grid(static_cast<unsigned>((HW + 63) / 64), (C + 63) / 64, N);
         auto* in = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pi));
         auto* out = reinterpret_cast<__nv_bfloat16*>(x.resolve(po));
         if (from) k::nhwc_to_nchw_bf16<<<grid, 256, 0, x.stream>>>(in, out, C, HW);
@@ -572,7 +572,11 @@ struct Builder {
       add(gi, 2, [=](const RunCtx& x) mutable {
         ip.x = reinterpret_cast<const __nv_bfloat16*>(x.resolve(px));
         ip.a = reinterpret_cast<__nv_bfloat16*>(x.arena + x.plan->scratch_off[0]);
-        k::im2col_nchw_bf16<<<148 * 8, 256, 0, x.stream>>>(ip);
+        {
+          const int segs = (ip.Wo + 63) / 64;
+          const size_t wsm = static_cast<size_t>(ip.C) * ip.ks * (63 * ip.stride + ip.ks) * 2;
+          k::im2col_nchw_bf16<<<static_cast<unsigned>(segs) * ip.Ho * ip.N, 256, wsm, x.stream>>>(ip);
+        }
         const void* Wp = x.resolve(pw);
         void* O = x.resolve(po);
         if (cache->a != ip.a || cache->w != Wp || cache->o != O) {
@@ -848,7 +852,7 @@ struct Builder {
       k::GapParams gp{};
       gp.C = static_cast<int>(vx.dims[1]);
       gp.HW = vx.dims[2] * vx.dims[3];
-      gp.slabs = static_cast<int>(std::max<long long>(1, std::min<long long>(256, gp.HW / 256)));
+      gp.slabs = static_cast<int>(std::max<long long>(1, std::min<long long>(592, gp.HW / 128)));
       gp.out_bf16 = O.dtype == DType::BF16;
       const int N = static_cast<int>(vx.dims[0]);
       scratch_need = std::max(scratch_need, static_cast<size_t>(N) * gp.slabs * gp.C * 8);
@@ -859,7 +863,7 @@ struct Builder {
         gp.out = x.resolve(po);
         gp.out_f64 = nullptr;
         launch_pdl(k::gap_partial_f64, dim3((gp.C + 63) / 64, gp.slabs, N), dim3(256), 0, x.stream, gp);
-        launch_pdl(k::gap_final_f64, dim3((N * gp.C + 255) / 256), dim3(256), 0, x.stream, gp, N);
+        launch_pdl(k::gap_final_f64, dim3((N * gp.C + 31) / 32), dim3(256), 0, x.stream, gp, N);
         return cudaGetLastError();
       });
     }

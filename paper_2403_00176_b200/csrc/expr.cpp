@@ -232,6 +232,33 @@ int64_t e_upper(const ExprCtx& cx, const Expr& e, const std::vector<int64_t>& va
   return eval_rec(cx, e, vals, ok, 1);
 }
 
+int64_t e_eval_flat(const Expr& e, const std::vector<int64_t>& av, bool* ok) {
+  *ok = true;
+  int64_t sum = 0;
+  for (auto& t : e.terms) {
+    int64_t prod = t.second;
+    for (auto& p : t.first) {
+      const int64_t v = p.first < static_cast<int>(av.size()) ? av[p.first] : INT64_MIN;
+      if (v == INT64_MIN) { *ok = false; return 0; }
+      for (int i = 0; i < p.second; ++i) prod *= v;
+    }
+    sum += prod;
+  }
+  return sum;
+}
+
+void e_eval_atoms(const ExprCtx& cx, std::vector<int64_t>* vals) {
+  vals->resize(cx.atoms.size(), INT64_MIN);
+  for (size_t i = 0; i < cx.atoms.size(); ++i) {
+    const Atom& a = cx.atoms[i];
+    if (a.kind == AtomKind::SYM) continue;
+    bool ok1, ok2;
+    const int64_t x = e_eval_flat(*a.a, *vals, &ok1), y = e_eval_flat(*a.b, *vals, &ok2);
+    if (!ok1 || !ok2 || (a.kind == AtomKind::FLOORDIV && y == 0)) { (*vals)[i] = INT64_MIN; continue; }
+    (*vals)[i] = a.kind == AtomKind::FLOORDIV ? fdiv(x, y) : a.kind == AtomKind::MIN ? std::min(x, y) : std::max(x, y);
+  }
+}
+
 bool e_has_runtime(const ExprCtx& cx, const Expr& e) {
   for (auto& t : e.terms)
     for (auto& p : t.first) {

@@ -69,6 +69,11 @@ std::string e_str(const ExprCtx& cx, const Expr& e);
 // Evaluate with atom values for symbols (vals[id], only read for SYM atoms). ok=false on an unbound
 // symbol (value INT64_MIN) or a division by zero.
 int64_t e_eval(const ExprCtx& cx, const Expr& e, const std::vector<int64_t>& vals, bool* ok);
+// Values of EVERY atom (symbols as given in vals, non-linear atoms evaluated once, children first:
+// atoms are interned after their arguments).  Atoms that cannot be evaluated get INT64_MIN.
+void e_eval_atoms(const ExprCtx& cx, std::vector<int64_t>* vals);
+// Evaluate with a complete atom table from e_eval_atoms (no recursion); ok=false if an atom is unknown.
+int64_t e_eval_flat(const Expr& e, const std::vector<int64_t>& atom_vals, bool* ok);
 bool e_has_runtime(const ExprCtx& cx, const Expr& e);
 // Static upper bound of e using the symbols' declared ranges (all coefficients must be >= 0 and
 // non-linear atoms monotone); ok=false if none can be derived.

@@ -34,6 +34,9 @@ Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* na
       int64_t x = e_eval(g.cx, as.a, out->vals[r], &ok1), y = e_eval(g.cx, as.b, out->vals[r], &ok2);
       if (ok1 && ok2 && x != y) { out->err = "shape conflict: " + as.what + " (" + std::to_string(x) + " vs " + std::to_string(y) + ")"; return E_SHAPE_CONFLICT; }
     }
+  // all non-linear atoms once per request (children first), then every dim is a flat polynomial
+  std::vector<std::vector<int64_t>> atom_vals(n_req);
+  for (int r = 0; r < n_req; ++r) { atom_vals[r] = out->vals[r]; e_eval_atoms(g.cx, &atom_vals[r]); }
   out->dims.assign(g.tensors.size(), {});
   for (size_t t = 0; t < g.tensors.size(); ++t) {
     const ShapeVal& s = g.tensors[t].S;
@@ -44,7 +47,7 @@ Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* na
       for (int i = 0; i < s.rank; ++i) {
         if (!s.dims[i].known()) { evaluable = false; break; }
         bool ok;
-        int64_t v = e_eval(g.cx, s.dims[i].e, out->vals[r], &ok);
+        int64_t v = e_eval_flat(s.dims[i].e, atom_vals[r], &ok);
         if (!ok) {  // depends on a runtime symbol: use its static upper bound for planning
           v = e_upper(g.cx, s.dims[i].e, out->vals[r], &ok);
           if (!ok) { evaluable = false; break; }
