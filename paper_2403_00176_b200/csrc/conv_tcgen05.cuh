@@ -29,6 +29,7 @@ struct ConvParams {
   int Cin, Cout;
   int ksize, stride, pad;
   int TW, TH;                // pixel patch of a tile: TW * TH == 128
+  int korder;                // 0: weight k-chunks in (dy, dx, chunk) order; 1: (dy, chunk, dx) order (3x3 only)
   // execution-determined image count (gated sub-batch): n_img = cnt_a + cnt_b * *n_img_ptr, read on the
   // device after the producing kernel has finished; n_img above is then only the static upper bound
   const long long* n_img_ptr;
@@ -134,8 +135,9 @@ conv_igemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_co
           ptx::mbar_expect_tx(&full[s], mine * 128 * 128);
           for (int c = warp; c < KCH; c += 2) {
             const int q = ks * KCH + c;          // k-chunk: tap-major, then 64-channel chunk
-            const int tap = q / cchunks, cc = q % cchunks;
-            const int dy = tap / p.ksize, dx = tap % p.ksize;
+            int dy, dx, cc;
+            if (p.korder) { dy = q / (3 * cchunks); cc = (q / 3) % cchunks; dx = q % 3; }
+            else { const int tap = q / cchunks; cc = q % cchunks; dy = tap / p.ksize; dx = tap % p.ksize; }
             // chunks past the end (K tail of the last stage) are loaded far out of range: zero fill
             const int hi = q < kchunks ? ho0 * p.stride + dy - p.pad : -100000;
             ptx::tma_load_4d(tiles + s * S::STAGE_BYTES + c * (128 * 128), &tmX, cc * 64, wo0 * p.stride + dx - p.pad, hi, img, &full[s]);

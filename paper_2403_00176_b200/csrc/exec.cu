@@ -9,6 +9,7 @@
 
 #include "attention.cuh"
 #include "conv_tcgen05.cuh"
+#include "conv3x3_tcgen05.cuh"
 #include "engine.h"
 #include "gemm_tcgen05.cuh"
 #include "kernels_compact.cuh"
@@ -628,6 +629,7 @@ struct Builder {
       cp.n_img = static_cast<int>(vo.dims[0]);
       cp.Ho = static_cast<int>(vo.dims[2]); cp.Wo = static_cast<int>(vo.dims[3]);
       cp.Cin = Cin; cp.Cout = Cout; cp.ksize = ks; cp.stride = G.stride; cp.pad = G.pad;
+      cp.korder = ks == 3;
       cp.has_residual = G.res >= 0;
       cp.act2 = G.act2;
       const RtCount rc = runtime_count(G.out, r);
@@ -641,6 +643,10 @@ struct Builder {
         const long long padded = static_cast<long long>((cp.Wo + tw - 1) / tw) * tw * ((cp.Ho + th - 1) / th) * th;
         if (best < 0 || padded < best) { best = padded; cp.TW = tw; cp.TH = th; }
       }
+      // wide images with a 3x3 / stride 1 / pad 1 kernel: row-halo kernel (a tile is 128 pixels of one row)
+      const bool rows = ks == 3 && G.stride == 1 && G.pad == 1 && cp.Wo >= 96 && ((cp.Wo + 127) / 128) * 128 * 4 <= cp.Wo * 5;
+      const bool wres = rows && Cin == 64 && Cout == 64;
+      if (rows) { cp.TW = 128; cp.TH = 1; }
       if (cp.TW * G.stride > 256 || cp.TH * G.stride > 256) return fail(E_UNSUPPORTED_OP, "convolution stride too large for the TMA box");
       const int H = static_cast<int>(vx.dims[2]), Wd = static_cast<int>(vx.dims[3]);
       Ptr px = ptr_of(G.a, r), po = ptr_of(G.out, r), pr = G.res >= 0 ? ptr_of(G.res, r) : Ptr();
@@ -658,8 +664,8 @@ struct Builder {
         void* O = x.resolve(po);
         const void* R = hr ? x.resolve(pr) : O;
         if (cache->a != X || cache->w != Wp || cache->o != O || cache->r != R) {
-          if (!encode_bf16_nhwc(&cache->tx, X, cp.n_img, H, Wd, Cin, cp.TW, cp.TH, stride) ||
-              !encode_bf16_kchunks(&cache->tw, Wp, Cout, K, K, bn, kch) ||
+          if (!encode_bf16_nhwc(&cache->tx, X, cp.n_img, H, Wd, Cin, rows ? 130 : cp.TW, cp.TH, stride) ||
+              !encode_bf16_kchunks(&cache->tw, Wp, Cout, K, K, bn, rows ? 3 : kch) ||
               !encode_bf16_nhwc(&cache->to, O, cp.n_img, cp.Ho, cp.Wo, Cout, cp.TW, cp.TH, 1) ||
               !encode_bf16_nhwc(&cache->tr, R, cp.n_img, cp.Ho, cp.Wo, Cout, cp.TW, cp.TH, 1))
             return cudaErrorInvalidValue;
@@ -669,7 +675,16 @@ struct Builder {
         cp.status = reinterpret_cast<int*>(x.arena);
         cp.n_img_ptr = rt ? reinterpret_cast<const long long*>(x.arena + rt_slot) : nullptr;
         const dim3 gd(static_cast<unsigned>(std::min<long long>(tiles, x.plan->sm_count))), bd(k::CONV_THREADS);
-        const int variant = (bn == 128 ? 2 : 0) + (act == 2 ? 1 : 0);
+        const int variant = (rows ? (wres ? 8 : 4) : 0) + (bn == 128 ? 2 : 0) + (act == 2 ? 1 : 0);
+#define SOD2_CONV3_CASE(V, BN_, RES_, ST_, ACT_)                                                                         \
+        case V: {                                                                                                        \
+          constexpr int smem = k::Conv3Smem<BN_, RES_, ST_>::TOTAL;                                                       \
+          static bool once = (cudaFuncSetAttribute(k::conv3x3_rows_bf16_tcgen05<BN_, RES_, ST_, ACT_>,                    \
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);             \
+          (void)once;                                                                                                    \
+          launch_pdl(k::conv3x3_rows_bf16_tcgen05<BN_, RES_, ST_, ACT_>, gd, dim3(k::CONV3_THREADS), smem, x.stream, cache->tx, cache->tw, \
+                     cache->to, cache->tr, cp);                                                                          \
+        } break;
 #define SOD2_CONV_CASE(V, BN_, KCH_, ST_, ACT_)                                                                          \
         case V: {                                                                                                        \
           constexpr int smem = k::ConvSmem<BN_, KCH_, ST_>::TOTAL;                                                        \
@@ -683,10 +698,17 @@ struct Builder {
           SOD2_CONV_CASE(0, 64, 2, 4, 0)
           SOD2_CONV_CASE(1, 64, 2, 4, 2)
           SOD2_CONV_CASE(2, 128, 2, 3, 0)
-          default:
           SOD2_CONV_CASE(3, 128, 2, 3, 2)
+          SOD2_CONV3_CASE(4, 64, false, 4, 0)
+          SOD2_CONV3_CASE(5, 64, false, 4, 2)
+          SOD2_CONV3_CASE(6, 128, false, 3, 0)
+          SOD2_CONV3_CASE(7, 128, false, 3, 2)
+          SOD2_CONV3_CASE(8, 64, true, 7, 0)
+          default:
+          SOD2_CONV3_CASE(9, 64, true, 7, 2)
         }
 #undef SOD2_CONV_CASE
+#undef SOD2_CONV3_CASE
         return cudaGetLastError();
       });
     }
@@ -975,6 +997,11 @@ Status prepack_weights(Compiled* c, void* workspace, size_t bytes, void* stream)
         const int K = ci * kh * kw, Kp = (K + 63) / 64 * 64;
         k::pad_rows_bf16<<<148 * 2, 256, 0, static_cast<cudaStream_t>(stream)>>>(
             static_cast<const __nv_bfloat16*>(W.dev_ptr), reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + c->packed_off[i]), co, K, Kp);
+        continue;
+      }
+      if (kh == 3 && kw == 3) {  // 3x3: (dy, channel chunk, dx, ci) so that the dx taps of a chunk are adjacent
+        k::reorder_conv3x3_rows<<<148 * 4, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+            static_cast<const __nv_bfloat16*>(W.dev_ptr), reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + c->packed_off[i]), co, ci);
         continue;
       }
       k::reorder_conv_weights<<<148 * 4, 256, 0, static_cast<cudaStream_t>(stream)>>>(
