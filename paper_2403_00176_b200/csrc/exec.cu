@@ -192,7 +192,7 @@ struct Builder {
     // bf16 on tcgen05
     if (G.has_ln) return fail(E_UNSUPPORTED_OP, "bf16 GEMM epilogue: LayerNorm tail is not fused");
     if (K % 64) return fail(E_UNSUPPORTED_OP, "bf16 GEMM needs K % 64 == 0 (k-chunk tensor maps)");
-    if (lds[0] % 8 || lds[1] % 8 || (G.res >= 0 && lds[2] % 8)) return fail(E_UNSUPPORTED_OP, "GEMM operand rows must be 16-byte multiples for TMA");
+    if (lds[0] % 8 || lds[1] % 8 || N % 8 || (G.res >= 0 && lds[2] % 8)) return fail(E_UNSUPPORTED_OP, "GEMM operand rows must be 16-byte multiples");
     size_t pk = 0;
     for (size_t i = 0; i < c.packed_consts.size(); ++i) if (c.packed_consts[i] == G.w) pk = c.packed_off[i];
     for (auto& sg : segs) {

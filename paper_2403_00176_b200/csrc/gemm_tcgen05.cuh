@@ -4,22 +4,31 @@
 // M rows, so rows past M read as zeros and the TMA store clips them.
 //
 // Persistent, warp-specialised, one CTA per SM.  Tile 128 x BN; one pipeline stage holds KCH
-// k-chunks of 64 (each chunk = one 128-byte swizzle atom per row).  Measured on B200: one thread
-// can issue a tcgen05.mma about every 65-80 cycles and a barrier wait in the issue loop costs about
-// 170 cycles, so a stage must carry >= 512 cycles of MMA work to hide them: (BN=256, KCH=1) or
-// (BN=128, KCH=2).
+// k-chunks of 64 (each chunk = one 128-byte swizzle atom per row).  Measured on B200: a
+// tcgen05.mma occupies the tensor pipe for max(~48, BN/2) cycles, and a barrier wait between MMAs
+// leaves the pipe idle for about 320 cycles unless the MMAs queued before it are long enough to
+// cover it, so a stage must carry >= 512 cycles of MMA work: (BN=256, KCH=1) or (BN=128, KCH=2).
+// An SM takes in about 70 bytes per clock from L2, which bounds the main loop of a 128 x 256 tile
+// at about 75 % of the tensor peak.
 //   warp 0      TMA producer for A (STAGES-deep mbarrier ring; one 3-D box per stage)
 //   warp 1      TMA producer for B (a thread sustains about one TMA instruction per 170 ns, so A
-//               and B get a thread each)
+//               and B get a thread each); B is constant, so it does not wait for the previous kernel
 //   warp 2      MMA issuer: tcgen05.mma into one of two TMEM accumulators (double buffered)
-//   warps 3..10 epilogue, in passes of 128 columns: drain TMEM (warp w owns lanes 32*(w%4)..), add
-//               bias from shared memory, activation, residual (TMA-loaded into the staging tile and
-//               updated in place), pack to bf16 into the swizzled staging tile, TMA store
-// so the epilogue of tile i overlaps the main loop of tile i+1.  Every wait is bounded (ptx.cuh).
+//   warps 3..10 epilogue, in passes of 64 columns: drain TMEM (warp w owns lanes 32*(w%4)..), add
+//               bias from shared memory, activation, residual (already in the staging buffer,
+//               updated in place), pack to bf16 into the swizzled staging buffer
+//   warp 11     staging agent: residual TMA loads ahead of the epilogue, TMA stores behind it
+// so the epilogue of tile i overlaps the main loop of tile i+1 and no epilogue thread waits on a
+// TMA round trip.  Every wait is bounded (ptx.cuh).
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include "ptx.cuh"
+
+// Timeline hook for bench probes: expands to nothing in the library build.
+#ifndef SOD2_TRACE
+#define SOD2_TRACE(who, tag)
+#endif
 
 namespace sod2 {
 namespace k {
@@ -34,30 +43,35 @@ struct GemmEpilogue {
 };
 
 constexpr int GEMM_BM = 128;
-constexpr int GEMM_THREADS = 352;
-constexpr int GEMM_PASS_COLS = 128;                       // epilogue pass width
-constexpr int GEMM_STAGE_OUT = GEMM_BM * GEMM_PASS_COLS * 2;  // 32 KB staging tile: 2 boxes of [128 rows x 128 B]
+constexpr int GEMM_THREADS = 384;
+constexpr int GEMM_PASS_COLS = 64;                            // epilogue pass width: one 128-byte swizzled row
+constexpr int GEMM_STAGE_OUT = GEMM_BM * GEMM_PASS_COLS * 2;  // 16 KB staging buffer: [128 rows x 128 B]
+constexpr int GEMM_NSB = 2;                                   // staging buffers
 
 template <int BN, int KCH, int STAGES>
 struct GemmSmem {
   static constexpr int A_BYTES = KCH * GEMM_BM * 128;
   static constexpr int B_BYTES = KCH * BN * 128;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int TOTAL = STAGES * STAGE_BYTES + GEMM_STAGE_OUT + 896 /*align slack: the window is at least 128-B aligned*/ + 2048 /*bias*/ + 128 /*barriers*/;
+  static constexpr int USED = STAGES * STAGE_BYTES + GEMM_NSB * GEMM_STAGE_OUT + 2048 /*bias*/ + 136 /*barriers, TMEM slot, dead flag*/;
+  // plus the pad that brings the tiles to a 1024-byte boundary; the kernel checks the pad it really
+  // needs against the launch's dynamic size and reports an error instead of running past the end
+  static constexpr int TOTAL = USED + 888;
 };
 
-// erf by the rational approximation 7.1.26 of Abramowitz & Stegun (|error| <= 1.5e-7), far inside
-// the bf16 output rounding; cheaper than erff on the epilogue warps.
+// GELU(x) = x * Phi(x) with Phi written as 0.5 * (1 + tanh(u(x))), u(x) = atanh(erf(x / sqrt 2)).
+// u is odd; x * (c0 + c1 x^2 + c2 x^4) fitted by least squares on [-8, 8] reproduces the erf form of
+// GELU to 3e-5 absolute, and the hardware tanh adds a relative 2^-11: both far inside the bf16 output
+// rounding.  x^2 is clamped where the quintic would turn over (|x| > 7; tanh is saturated there).
+// Eight instructions per element instead of seventeen for a polynomial erf: the epilogue of a
+// GELU GEMM is bound by instruction issue.
 __device__ __forceinline__ float gelu_erf(float x) {
-  const float z = fabsf(x) * 0.70710678118654752f;
+  const float x2 = fminf(x * x, 50.0f);
+  const float u = x * fmaf(x2, fmaf(x2, -0.00035873236f, 0.037050345f), 0.79745847f);
   float t;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f, z, 1.0f)));
-  float p = fmaf(1.061405429f, t, -1.453152027f);
-  p = fmaf(p, t, 1.421413741f);
-  p = fmaf(p, t, -0.284496736f);
-  p = fmaf(p, t, 0.254829592f);
-  const float e = 1.0f - p * t * __expf(-z * z);   // erf(|x|/sqrt2)
-  return 0.5f * x * (1.0f + copysignf(e, x));
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
+  const float hx = 0.5f * x;
+  return fmaf(hx, t, hx);
 }
 // The activation is a template parameter: a run-time switch inside the unrolled element loops
 // turns every element into its own basic block and serialises the dependent FMA / MUFU chains.
@@ -79,6 +93,8 @@ __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 256;"
 
 // tmA / tmB are 3-D views {64, rows, K/64} of the row-major operands (K % 64 == 0), box
 // {64, 128 or BN, KCH}: one instruction fills KCH consecutive swizzled [rows x 64] chunks.
+// B must be a constant of the graph (prepacked weights): its producer does not wait for the
+// previous kernel in the stream.
 template <int BN, int KCH, int STAGES, int ACT>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -86,18 +102,28 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   int M, int N, int K, GemmEpilogue ep) {
   using S = GemmSmem<BN, KCH, STAGES>;
   constexpr int PASSES = BN / GEMM_PASS_COLS;
+  constexpr int NSB = GEMM_NSB;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* out_stage = tiles + STAGES * S::STAGE_BYTES;
-  float* bias_s = reinterpret_cast<float*>(out_stage + GEMM_STAGE_OUT);  // [2][256]
+  float* bias_s = reinterpret_cast<float*>(out_stage + NSB * GEMM_STAGE_OUT);  // [2][256]
   uint64_t* full = reinterpret_cast<uint64_t*>(bias_s + 512);
   uint64_t* empty = full + STAGES;
   uint64_t* tmem_full = empty + STAGES;   // [2]
   uint64_t* tmem_empty = tmem_full + 2;   // [2]
-  uint64_t* res_full = tmem_empty + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(res_full + 1);
+  uint64_t* buf_ready = tmem_empty + 2;   // [NSB] staging buffer handed to the epilogue warps (residual loaded, or just free)
+  uint64_t* buf_filled = buf_ready + NSB; // [NSB] epilogue warps have written the buffer
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(buf_filled + NSB);
   volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
+  {
+    uint32_t dyn;
+    asm("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn));
+    if (static_cast<uint32_t>(tiles - smem_raw) + S::USED > dyn) {   // uniform over the CTA
+      if (threadIdx.x == 0 && ep.status) atomicExch(ep.status, 2);
+      return;
+    }
+  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_m = (M + GEMM_BM - 1) / GEMM_BM, tiles_n = (N + BN - 1) / BN;
   const int num_tiles = tiles_m * tiles_n;
@@ -108,7 +134,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(&full[s], 2); ptx::mbar_init(&empty[s], 1); }
     for (int b = 0; b < 2; ++b) { ptx::mbar_init(&tmem_full[b], 1); ptx::mbar_init(&tmem_empty[b], 8); }
-    ptx::mbar_init(res_full, 1);
+    for (int b = 0; b < NSB; ++b) { ptx::mbar_init(&buf_ready[b], 1); ptx::mbar_init(&buf_filled[b], 8); }
     *dead = 0;
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
@@ -122,13 +148,18 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  // everything above touched only this CTA's own state; the operands may still be in flight
-  ptx::pdl_wait();
+  if (threadIdx.x == 0) { SOD2_TRACE(0, 1) }
+  // Everything above touched only this CTA's own state.  Each role waits for the previous kernel
+  // only where it touches that kernel's data: the A producer and the epilogue warps do, the B
+  // producer (constant weights) and the MMA issuer (shared memory and TMEM only) do not, so the
+  // weight stages stream in while the previous kernel drains.
   ptx::pdl_launch();
 
   if (warp == 0) {
     if (lane == 0) {
       // ---- TMA producer: A stages
+      ptx::pdl_wait();
+      SOD2_TRACE(0, 2)
       int n = 0;
       for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
         const int m0 = (t % tiles_m) * GEMM_BM;
@@ -168,6 +199,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           const int s = n % STAGES;
           ptx::mbar_wait(&full[s], (n / STAGES) & 1, dead);
           ptx::tc_fence_after();
+          if (ks == 0) { SOD2_TRACE(1, 10 + j) }
           const uint32_t a = ptx::smem_u32(tiles + s * S::STAGE_BYTES);
 #pragma unroll
           for (int c = 0; c < KCH; ++c) {
@@ -181,16 +213,62 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           ptx::mma_commit(&empty[s]);  // frees the stage once these MMAs have read it
         }
         ptx::mma_commit(&tmem_full[acc]);
+        SOD2_TRACE(1, 20 + j)
       }
     }
+  } else if (warp == 11) {
+    if (lane == 0) {
+      // ---- staging agent: owns the staging buffers' TMA traffic so that no epilogue thread waits on a
+      // TMA round trip.  A unit is one 64-column pass of one tile; unit u uses buffer u % NSB.
+      // prepare(u) hands the buffer to the epilogue warps: with a residual it is TMA-loaded into the
+      // buffer (the epilogue updates it in place), otherwise a plain arrive.  Once the epilogue warps
+      // have filled the buffer the agent stores it and, after the store has read the buffer, prepares
+      // unit u + NSB.  The kernel may end once the last store has read shared memory.
+      ptx::pdl_wait();
+      int my_tiles = 0;
+      for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) ++my_tiles;
+      const int U = my_tiles * PASSES;
+      auto prepare = [&](int u) {
+        const int t = blockIdx.x + (u / PASSES) * gridDim.x;
+        const int m0 = (t % tiles_m) * GEMM_BM, np = (t / tiles_m) * BN + (u % PASSES) * GEMM_PASS_COLS;
+        const int bsel = u % NSB;
+        if (ep.has_residual && np < N) {
+          ptx::mbar_expect_tx(&buf_ready[bsel], GEMM_STAGE_OUT);
+          ptx::tma_load_2d(out_stage + bsel * GEMM_STAGE_OUT, &tmRes, np, m0, &buf_ready[bsel]);
+        } else {
+          ptx::mbar_arrive(&buf_ready[bsel]);
+        }
+      };
+      for (int u = 0; u < NSB && u < U; ++u) prepare(u);
+      for (int u = 0; u < U; ++u) {
+        const int bsel = u % NSB;
+        ptx::mbar_wait(&buf_filled[bsel], (u / NSB) & 1, dead);
+        const int t = blockIdx.x + (u / PASSES) * gridDim.x;
+        const int m0 = (t % tiles_m) * GEMM_BM, np = (t / tiles_m) * BN + (u % PASSES) * GEMM_PASS_COLS;
+        if (np < N) {
+          tma_store_2d(&tmOut, out_stage + bsel * GEMM_STAGE_OUT, np, m0);
+          bulk_commit();
+        }
+        if (u + NSB < U) {
+          bulk_wait_read0();
+          prepare(u + NSB);
+        }
+      }
+      SOD2_TRACE(2, 40)
+      bulk_wait_read0();
+      SOD2_TRACE(2, 41)
+    }
   } else {
-    // ---- epilogue warps 3..10
+    // ---- epilogue warps 3..10: TMEM -> +bias -> act -> (+residual, act2) -> bf16 -> swizzled staging.
+    // Warp (q, half) owns TMEM lanes 32q..32q+31 (a warp may only read its own lane quarter) and the
+    // 32-column half of every 64-column pass; a thread holds one output row.
     const int e = warp - 3;
-    const int q = warp & 3;          // TMEM lane quarter this warp may access
-    const int half = e >> 2;         // which 64-column half of the pass
+    const int q = warp & 3;
+    const int half = e >> 2;
     const int et = threadIdx.x - 96; // 0..255
     const int row = q * 32 + lane;   // row inside the tile
-    int j = 0, rp = 0;               // rp counts residual loads (phase of res_full)
+    ptx::pdl_wait();
+    int j = 0, u = 0;
     auto load_bias = [&](int t) -> float {
       const int idx = (t / tiles_m) * BN + et;
       return (ep.bias && et < BN && t < num_tiles && idx < N) ? __bfloat162float(ep.bias[idx]) : 0.0f;
@@ -199,7 +277,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const float relu2_floor = ep.act2 == ACT_RELU ? 0.0f : -INFINITY;  // post-residual activation, branch-free
     for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++j) {
       const int acc = j & 1;
-      const int m0 = (t % tiles_m) * GEMM_BM, n0 = (t / tiles_m) * BN;
+      const int n0 = (t / tiles_m) * BN;
       float* bias_t = bias_s + (j & 1) * 256;      // this tile's bias, prefetched during the last tile
       bias_t[et] = bias_next;
       bias_next = load_bias(t + gridDim.x);
@@ -207,76 +285,56 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       ptx::mbar_wait(&tmem_full[acc], (j >> 1) & 1, dead);
       __syncwarp();
       ptx::tc_fence_after();
-#pragma unroll 1
-      for (int ps = 0; ps < PASSES; ++ps) {
-        const int np = n0 + ps * GEMM_PASS_COLS;   // first global column of this pass
+      if (et == 0) { SOD2_TRACE(2, 30 + j) }
+      const uint32_t taddr = tmem + (static_cast<uint32_t>(q * 32) << 16) + acc * BN + half * 32;
+      uint32_t r[2][32];
+      ptx::tmem_ld32(taddr, r[0]);
+#pragma unroll
+      for (int ps = 0; ps < PASSES; ++ps, ++u) {
+        const int np = n0 + ps * GEMM_PASS_COLS;
         const bool live = np < N;
         const bool res = ep.has_residual && live;
-        if (res) {
-          // the residual tile is TMA-loaded into the staging tile (once the previous store has
-          // finished reading it) and updated in place
-          if (et == 0) {
-            bulk_wait_read0();
-            ptx::mbar_expect_tx(res_full, GEMM_STAGE_OUT);
-            ptx::tma_load_2d(out_stage, &tmRes, np, m0, res_full);
-            ptx::tma_load_2d(out_stage + 16384, &tmRes, np + 64, m0, res_full);
-          }
-          ptx::mbar_wait(res_full, rp & 1, dead);
+        const int bsel = u % NSB;
+        uint8_t* obase = out_stage + bsel * GEMM_STAGE_OUT + row * 128;
+        ptx::tmem_ld_wait();
+        if (ps + 1 < PASSES) {
+          ptx::tmem_ld32(taddr + (ps + 1) * GEMM_PASS_COLS, r[(ps + 1) & 1]);
+        } else {
+          // every column of this warp's share has left TMEM: the accumulator may be overwritten
+          ptx::tc_fence_before();
           __syncwarp();
-          ++rp;
+          if (lane == 0) ptx::mbar_arrive(&tmem_empty[acc]);
         }
-        uint8_t* obase = out_stage + half * 16384 + row * 128;
-        uint4 pk[8];
+        ptx::mbar_wait(&buf_ready[bsel], (u / NSB) & 1, dead);
+        __syncwarp();
         if (live) {
+          const float* bp = bias_t + ps * GEMM_PASS_COLS + half * 32;
 #pragma unroll
-          for (int c = 0; c < 2; ++c) {
-            const int col = half * 64 + c * 32;  // column inside the pass
-            uint32_t r[32];
-            ptx::tmem_ld32(tmem + (static_cast<uint32_t>(q * 32) << 16) + acc * BN + ps * GEMM_PASS_COLS + col, r);
-            ptx::tmem_ld_wait();
-            const float* bp = bias_t + ps * GEMM_PASS_COLS + col;
+          for (int g = 0; g < 4; ++g) {
+            float v[8];
 #pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              float v[8];
+            for (int i = 0; i < 8; ++i) v[i] = apply_act<ACT>(__uint_as_float(r[ps & 1][g * 8 + i]) + bp[g * 8 + i]);
+            uint4* slot = reinterpret_cast<uint4*>(obase + (((half * 4 + g) ^ (row & 7)) << 4));
+            if (res) {
+              const uint4 rv = *slot;
+              const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&rv);
 #pragma unroll
-              for (int i = 0; i < 8; ++i) v[i] = apply_act<ACT>(__uint_as_float(r[g * 8 + i]) + bp[g * 8 + i]);
-              if (res) {
-                const uint4 rv = *reinterpret_cast<const uint4*>(obase + (((c * 4 + g) ^ (row & 7)) << 4));
-                const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&rv);
+              for (int i = 0; i < 4; ++i) { const float2 f = __bfloat1622float2(h[i]); v[2 * i] += f.x; v[2 * i + 1] += f.y; }
 #pragma unroll
-                for (int i = 0; i < 4; ++i) { const float2 f = __bfloat1622float2(h[i]); v[2 * i] += f.x; v[2 * i + 1] += f.y; }
-#pragma unroll
-                for (int i = 0; i < 8; ++i) v[i] = fmaxf(v[i], relu2_floor);
-              }
-              __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&pk[c * 4 + g]);
-#pragma unroll
-              for (int i = 0; i < 4; ++i) oh[i] = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+              for (int i = 0; i < 8; ++i) v[i] = fmaxf(v[i], relu2_floor);
             }
+            uint4 pk;
+            __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&pk);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) oh[i] = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+            *slot = pk;
           }
         }
-        // the math above overlapped the previous pass's TMA store; now the staging tile must be free
-        if (!res) {
-          if (et == 0) bulk_wait_read0();
-          epi_bar_sync();
-        }
-        if (live) {
-#pragma unroll
-          for (int g = 0; g < 8; ++g) *reinterpret_cast<uint4*>(obase + ((g ^ (row & 7)) << 4)) = pk[g];
-        }
-        // publish the staging tile to the async proxy; after the last pass the accumulator is free
-        ptx::tc_fence_before();
         ptx::fence_proxy_async();
         __syncwarp();
-        if (ps == PASSES - 1 && lane == 0) ptx::mbar_arrive(&tmem_empty[acc]);
-        epi_bar_sync();
-        if (et == 0 && live) {
-          tma_store_2d(&tmOut, out_stage, np, m0);
-          if (np + 64 < N) tma_store_2d(&tmOut, out_stage + 16384, np + 64, m0);
-          bulk_commit();
-        }
+        if (lane == 0) ptx::mbar_arrive(&buf_filled[bsel]);
       }
     }
-    if (et == 0) bulk_wait0();
   }
   ptx::tc_fence_before();
   __syncthreads();
