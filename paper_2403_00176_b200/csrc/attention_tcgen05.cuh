@@ -1,0 +1,295 @@
+// Fused attention group on tcgen05 / TMEM for packed variable-length requests, head dim 64:
+//   O = softmax(Q K^T * scale) V  per (request, head), bf16 in / fp32 accumulate / bf16 out.
+// The score and probability tensors never reach global memory (the fusion argument of Section 4.2).
+// One CTA owns 128 query rows of one (request, head) and walks the request's keys in blocks of 64:
+//   S_j = Q K_j^T          tcgen05.mma, M=128, N=64, K=64; Q and K_j are K-major TMA tiles
+//   P_j = exp2(S_j*c - m)  softmax threads: two threads per query row read the halves of its row of
+//                          S_j from TMEM, write P_j as bf16 into a swizzled tile
+//   O_j = P_j V_j          tcgen05.mma, M=128, N=64, K=64; V_j is the natural [key, d] tile, used
+//                          as an MN-major B operand
+//   o   = o*corr + O_j     running output in registers (the rescale of the online softmax)
+// S and O_j are double buffered in TMEM (4 x 64 columns), P_j, K_j, V_j in shared memory, so the
+// tensor pipe, the softmax warps and TMA overlap inside a CTA; two CTAs share an SM.
+// Q, K, V are 2-D tensor maps over the packed [tokens, row stride] buffers; a tile that runs past a
+// request's rows reads the next request's rows (finite data) or zeros past the end of the buffer, and
+// those keys are masked to -inf before the softmax; query rows past the request are never written.
+// Warps: 0 TMA, 1 issues S = Q K^T, 10 issues O = P V, 2..9 softmax (warp w reads TMEM lane quarter
+// w % 4; two threads per row).
+// Every wait is bounded (ptx.cuh).
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include "ptx.cuh"
+
+namespace sod2 {
+namespace k {
+
+constexpr int ATC_MAX_REQ = 32;
+constexpr int ATC_THREADS = 352;
+struct AtcReq {
+  int L;                       // tokens of this request
+  int q_row, k_row, v_row;     // first row of the request in the Q / K / V tensor maps
+  long long o_off;             // element offset of the request's output view
+};
+struct AtcParams {
+  __nv_bfloat16* o;
+  int n_req, H;
+  int q_col, k_col, v_col;     // column of head 0 in the Q / K / V tensor maps
+  int q_hs, k_hs, v_hs;        // head strides in columns
+  int o_ts, o_hs;              // output token / head strides in elements (multiples of 8)
+  float scale_log2e;
+  int* status;
+  int tile_start[ATC_MAX_REQ + 1];   // prefix sum of ceil(L / 128); requests in descending L
+  AtcReq r[ATC_MAX_REQ];
+};
+
+constexpr int ATC_Q_BYTES = 128 * 128;    // 128 rows x 64 bf16
+constexpr int ATC_KV_BYTES = 64 * 128;    // 64 keys x 64 bf16
+constexpr int ATC_P_BYTES = 128 * 128;    // 128 rows x 64 keys bf16
+constexpr int ATC_SMEM = ATC_Q_BYTES + 4 * ATC_KV_BYTES + 2 * ATC_P_BYTES + 2048 /*row maxima*/ + 1024 /*align*/ + 256 /*barriers*/;
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__global__ void __launch_bounds__(ATC_THREADS, 2)
+attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                       const __grid_constant__ CUtensorMap tmV, const __grid_constant__ AtcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sQ = base;
+  uint8_t* sK = sQ + ATC_Q_BYTES;           // [2]
+  uint8_t* sV = sK + 2 * ATC_KV_BYTES;      // [2]
+  uint8_t* sP = sV + 2 * ATC_KV_BYTES;      // [2]
+  float* xmax = reinterpret_cast<float*>(sP + 2 * ATC_P_BYTES);   // [block parity][column half][row]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(xmax + 512);
+  uint64_t* q_full = bars;            // 1
+  uint64_t* k_full = bars + 1;        // [2] K_j landed
+  uint64_t* v_full = bars + 3;        // [2] V_j landed
+  uint64_t* s_full = bars + 5;        // [2] S_j done (also: K stage free)
+  uint64_t* s_free = bars + 7;        // [2] softmax warps have read S_j
+  uint64_t* p_full = bars + 9;        // [2] softmax warps have written P_j
+  uint64_t* o_full = bars + 11;       // [2] O_j done (also: V stage and P buffer free)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
+  volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // work item: blockIdx.x = tile * H + head, tiles ordered by descending request length
+  const int tile = blockIdx.x / p.H, head = blockIdx.x % p.H;
+  int ri = 0;
+  while (ri + 1 < p.n_req && tile >= p.tile_start[ri + 1]) ++ri;
+  const AtcReq& R = p.r[ri];
+  const int L = R.L;
+  const int q0 = (tile - p.tile_start[ri]) * 128;
+  const int nkv = (L + 63) >> 6;
+
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(q_full, 1);
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(&k_full[b], 1); ptx::mbar_init(&v_full[b], 1);
+      ptx::mbar_init(&s_full[b], 1); ptx::mbar_init(&s_free[b], 8);
+      ptx::mbar_init(&p_full[b], 8); ptx::mbar_init(&o_full[b], 1);
+    }
+    *dead = 0;
+    ptx::fence_barrier_init();
+    ptx::fence_proxy_async();
+    ptx::prefetch_tmap(&tmQ);
+    ptx::prefetch_tmap(&tmK);
+    ptx::prefetch_tmap(&tmV);
+  }
+  if (warp == 1) { ptx::tmem_alloc(tmem_slot, 256); ptx::tmem_relinquish(); }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  ptx::pdl_launch();
+  if (threadIdx.x == 0) { SOD2_TRACE(0, 1) }
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---- TMA producer
+      ptx::pdl_wait();
+      ptx::mbar_expect_tx(q_full, ATC_Q_BYTES);
+      ptx::tma_load_2d(sQ, &tmQ, p.q_col + head * p.q_hs, R.q_row + q0, q_full);
+      for (int j = 0; j < nkv; ++j) {
+        const int b = j & 1;
+        if (j >= 2) ptx::mbar_wait(&s_full[b], ((j >> 1) - 1) & 1, dead);    // S_{j-2} done: K stage free
+        ptx::mbar_expect_tx(&k_full[b], ATC_KV_BYTES);
+        ptx::tma_load_2d(sK + b * ATC_KV_BYTES, &tmK, p.k_col + head * p.k_hs, R.k_row + j * 64, &k_full[b]);
+        if (j >= 2) ptx::mbar_wait(&o_full[b], ((j >> 1) - 1) & 1, dead);    // O_{j-2} done: V stage free
+        ptx::mbar_expect_tx(&v_full[b], ATC_KV_BYTES);
+        ptx::tma_load_2d(sV + b * ATC_KV_BYTES, &tmV, p.v_col + head * p.v_hs, R.v_row + j * 64, &v_full[b]);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ---- S issuer: S_j = Q K_j^T.  A thread that waits on a barrier between MMAs stalls for a few
+      // hundred cycles, so the two products get a thread each and one commit per block: "S_j done"
+      // both publishes S_j and frees the K stage.
+      constexpr uint32_t idesc_qk = ptx::idesc_bf16(128, 64);
+      const uint32_t aQ = ptx::smem_u32(sQ);
+      ptx::mbar_wait(q_full, 0, dead);
+      for (int j = 0; j < nkv; ++j) {
+        const int b = j & 1;
+        ptx::mbar_wait(&k_full[b], (j >> 1) & 1, dead);
+        if (j >= 2) ptx::mbar_wait(&s_free[b], ((j >> 1) - 1) & 1, dead);
+        ptx::tc_fence_after();
+        const uint32_t aK = ptx::smem_u32(sK + b * ATC_KV_BYTES);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          ptx::mma_bf16(tmem + b * 64, ptx::smem_desc_sw128(aQ) + 2 * kk, ptx::smem_desc_sw128(aK) + 2 * kk, idesc_qk, kk != 0);
+        ptx::mma_commit(&s_full[b]);
+        SOD2_TRACE(1, 10 + j)
+      }
+    }
+  } else if (warp == 10) {
+    if (lane == 0) {
+      // ---- O issuer: O_j = P_j V_j.  "O_j done" publishes O_j, frees the V stage and the P buffer.
+      // The softmax warps hand over P_j only after they have read O_{j-2} (program order in their
+      // loop), so the O buffer needs no barrier of its own.
+      constexpr uint32_t idesc_pv = ptx::idesc_bf16(128, 64) | (1u << 16);   // B (= V tile) is MN-major
+      for (int i = 0; i < nkv; ++i) {
+        const int b = i & 1;
+        ptx::mbar_wait(&v_full[b], (i >> 1) & 1, dead);
+        ptx::mbar_wait(&p_full[b], (i >> 1) & 1, dead);
+        ptx::tc_fence_after();
+        const uint32_t aP = ptx::smem_u32(sP + b * ATC_P_BYTES), aV = ptx::smem_u32(sV + b * ATC_KV_BYTES);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)   // 16 keys per step: 32 B along P's rows, 16 rows (2048 B) down V
+          ptx::mma_bf16(tmem + 128 + b * 64, ptx::smem_desc_sw128(aP) + 2 * kk, ptx::smem_desc_sw128(aV + kk * 2048), idesc_pv, kk != 0);
+        ptx::mma_commit(&o_full[b]);
+        SOD2_TRACE(1, 20 + i)
+      }
+    }
+  } else {
+    // ---- softmax warps 2..9: two threads per query row.  Warp w reads TMEM lane quarter w % 4; warps
+    // 2..5 own score columns 0..31 of a block (and output columns 0..31), warps 6..9 the other half.
+    // The two threads of a row exchange their partial row maximum through shared memory once per
+    // block; the row sum stays split until the end.
+    const int q = warp & 3;
+    const int hh = (warp - 2) >> 2;
+    const int row = q * 32 + lane;
+    const bool warp_live = q0 + q * 32 < L;        // a warp whose 32 rows are all past the request only keeps the barriers moving
+    const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
+    const bool tracer = threadIdx.x == 64;
+    ptx::pdl_wait();
+    float o[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) o[i] = 0.f;
+    float m = -INFINITY, l = 0.f, c_prev = 0.f;
+    const float c = p.scale_log2e;
+    auto accumulate = [&](int i, float cf) {
+      // o = o * cf + O_i, this thread's 32 columns of O_i read from TMEM
+      const int b = i & 1;
+      ptx::mbar_wait_warp(&o_full[b], (i >> 1) & 1, dead);
+      ptx::tc_fence_after();
+      uint32_t r[32];
+      ptx::tmem_ld32(tmem + lane_base + 128 + b * 64 + hh * 32, r);
+      ptx::tmem_ld_wait();
+      ptx::tc_fence_before();
+      if (warp_live) {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) o[e] = fmaf(o[e], cf, __uint_as_float(r[e]));
+      }
+    };
+    for (int j = 0; j < nkv; ++j) {
+      const int b = j & 1;
+      ptx::mbar_wait_warp(&s_full[b], (j >> 1) & 1, dead);
+      ptx::tc_fence_after();
+      if (tracer) { SOD2_TRACE(2, 30 + j) }
+      uint32_t s[32];
+      ptx::tmem_ld32(tmem + lane_base + b * 64 + hh * 32, s);
+      ptx::tmem_ld_wait();
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&s_free[b]);
+      // partial row maximum on the raw scores (the scale is positive), exchanged with the row's other thread
+      const int valid = L - j * 64 - hh * 32;      // keys of this thread's half inside the request
+      if (valid < 32) {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) if (e >= valid) s[e] = 0xff800000u;   // -inf
+      }
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+      for (int e = 0; e < 32; e += 4) {
+        mx0 = fmaxf(mx0, __uint_as_float(s[e])); mx1 = fmaxf(mx1, __uint_as_float(s[e + 1]));
+        mx2 = fmaxf(mx2, __uint_as_float(s[e + 2])); mx3 = fmaxf(mx3, __uint_as_float(s[e + 3]));
+      }
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+      xmax[(b * 2 + hh) * 128 + row] = mx;
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      const float m_new = fmaxf(m, fmaxf(mx, xmax[(b * 2 + (hh ^ 1)) * 128 + row]));
+      // p = 2^(s*c - m*c): the scale rides in the FMA that feeds ex2.  The special-function pipe (16
+      // results per clock per SM, shared with the float <-> half conversions) bounds this loop.
+      const float corr = ex2_approx((m - m_new) * c);
+      m = m_new;
+      const float mc = -m_new * c;
+      float sum0 = 0.f, sum1 = 0.f;
+      uint32_t pk[16];
+#pragma unroll
+      for (int e = 0; e < 32; e += 2) {
+        const float p0 = ex2_approx(fmaf(__uint_as_float(s[e]), c, mc)), p1 = ex2_approx(fmaf(__uint_as_float(s[e + 1]), c, mc));
+        sum0 += p0; sum1 += p1;
+        const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+        pk[e >> 1] = warp_live ? *reinterpret_cast<const uint32_t*>(&pb) : 0u;
+      }
+      l = fmaf(l, corr, sum0 + sum1);
+      if (tracer) { SOD2_TRACE(2, 40 + j) }
+      // P_j into the swizzled tile once the MMA that read this buffer two blocks ago has finished
+      if (j >= 2) ptx::mbar_wait_warp(&o_full[b], ((j >> 1) - 1) & 1, dead);    // O_{j-2} done: P buffer free
+      {
+        uint8_t* prow = sP + b * ATC_P_BYTES + row * 128;
+#pragma unroll
+        for (int g = 0; g < 4; ++g)
+          *reinterpret_cast<uint4*>(prow + (((hh * 4 + g) ^ (row & 7)) << 4)) = make_uint4(pk[4 * g], pk[4 * g + 1], pk[4 * g + 2], pk[4 * g + 3]);
+      }
+      ptx::fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&p_full[b]);
+      if (tracer) { SOD2_TRACE(2, 50 + j) }
+      if (j >= 1) accumulate(j - 1, c_prev);
+      if (tracer) { SOD2_TRACE(2, 60 + j) }
+      c_prev = corr;
+    }
+    accumulate(nkv - 1, c_prev);
+    if (tracer) { SOD2_TRACE(2, 70) }
+    // ---- output: the row sums of the two halves are added through shared memory, the scaled rows are
+    // staged (swizzled) in P buffer 0 and written four full 128-byte rows per instruction.  Every MMA
+    // that read the P buffers has completed.
+    {
+      xmax[hh * 128 + row] = l;
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      const float lt = l + xmax[(hh ^ 1) * 128 + row];
+      const float inv = warp_live ? 1.0f / lt : 0.f;
+      uint8_t* prow = sP + row * 128;
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        uint4 v;
+        __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) h2[i] = __floats2bfloat162_rn(o[g * 8 + 2 * i] * inv, o[g * 8 + 2 * i + 1] * inv);
+        *reinterpret_cast<uint4*>(prow + (((hh * 4 + g) ^ (row & 7)) << 4)) = v;
+      }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      __nv_bfloat16* og = p.o + R.o_off + static_cast<long long>(head) * p.o_hs;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int rr = q * 32 + hh * 16 + i * 4 + (lane >> 3), ch = lane & 7;
+        const uint4 v = *reinterpret_cast<const uint4*>(sP + rr * 128 + ((ch ^ (rr & 7)) << 4));
+        if (q0 + rr < L) *reinterpret_cast<uint4*>(og + static_cast<long long>(q0 + rr) * p.o_ts + ch * 8) = v;
+      }
+    }
+  }
+  if (threadIdx.x == 64) { SOD2_TRACE(2, 80) }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) ptx::tmem_dealloc(tmem, 256);
+  if (threadIdx.x == 0 && *dead && p.status) atomicExch(p.status, 1);
+  SOD2_TRACE_DUMP()
+}
+
+}  // namespace k
+}  // namespace sod2

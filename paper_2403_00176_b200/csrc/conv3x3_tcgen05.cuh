@@ -226,8 +226,7 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_
       bias_t[et] = bias_next;
       bias_next = load_bias(t + gridDim.x);
       conv_epi_bar();
-      ptx::mbar_wait(&tmem_full[acc], (j >> 1) & 1, dead);
-      __syncwarp();
+      ptx::mbar_wait_warp(&tmem_full[acc], (j >> 1) & 1, dead);
       ptx::tc_fence_after();
 #pragma unroll 1
       for (int ps = 0; ps < PASSES; ++ps, ++u) {
@@ -246,8 +245,7 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(&tmem_empty[acc]);
         }
-        ptx::mbar_wait(&res_full[bsel], (u / NSB) & 1, dead);
-        __syncwarp();
+        ptx::mbar_wait_warp(&res_full[bsel], (u / NSB) & 1, dead);
         if (live) {
           const float* bp = bias_t + ps * 64 + half * 32;
 #pragma unroll

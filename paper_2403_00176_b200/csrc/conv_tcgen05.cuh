@@ -210,8 +210,7 @@ conv_igemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_co
       bias_t[et] = bias_next;
       bias_next = load_bias(t + gridDim.x);
       conv_epi_bar();
-      ptx::mbar_wait(&tmem_full[acc], (j >> 1) & 1, dead);
-      __syncwarp();
+      ptx::mbar_wait_warp(&tmem_full[acc], (j >> 1) & 1, dead);
       ptx::tc_fence_after();
 #pragma unroll 1
       for (int ps = 0; ps < PASSES; ++ps) {
@@ -224,8 +223,7 @@ conv_igemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_co
             ptx::mbar_expect_tx(res_full, CONV_STAGE_OUT);
             ptx::tma_load_4d(out_stage, &tmRes, np, wo0, ho0, img, res_full);
           }
-          ptx::mbar_wait(res_full, rp & 1, dead);
-          __syncwarp();
+          ptx::mbar_wait_warp(res_full, rp & 1, dead);
           ++rp;
         }
         uint8_t* obase = out_stage + row * 128;

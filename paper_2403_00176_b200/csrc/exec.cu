@@ -8,6 +8,7 @@
 #include <map>
 
 #include "attention.cuh"
+#include "attention_tcgen05.cuh"
 #include "conv_tcgen05.cuh"
 #include "conv3x3_tcgen05.cuh"
 #include "engine.h"
@@ -307,6 +308,65 @@ struct Builder {
       ap.tile_start[nr] = tiles;
       ap.H = H;
       if (tiles == 0) continue;
+      // tcgen05 path: needs Q, K, V as 2-D [token, column] maps over one packed buffer each (the same
+      // token stride, head stride and head-0 column for every request, rows in increasing order)
+      {
+        k::AtcParams tp{};
+        bool ok = true;
+        auto split = [&](long long off, int ts, int* row, int* col) { if (off < 0 || ts <= 0) { ok = false; return; } *row = static_cast<int>(off / ts); *col = static_cast<int>(off % ts); };
+        const k::AttnReq& R0 = ap.r[0];
+        int order[k::ATTN_MAX_REQ];
+        for (int i = 0; i < nr; ++i) order[i] = i;
+        std::stable_sort(order, order + nr, [&](int a, int b) { return ap.r[a].L > ap.r[b].L; });
+        long long rows_q = 0, rows_k = 0, rows_v = 0;
+        int tiles128 = 0;
+        for (int s = 0; s < nr && ok; ++s) {
+          const k::AttnReq& R = ap.r[order[s]];
+          if (R.q_ts != R0.q_ts || R.k_ts != R0.k_ts || R.v_ts != R0.v_ts || R.q_hs != R0.q_hs || R.k_hs != R0.k_hs || R.v_hs != R0.v_hs ||
+              R.o_ts != R0.o_ts || R.o_hs != R0.o_hs || (R.o_ts | R.o_hs) % 8 || R.o_off % 8) { ok = false; break; }
+          k::AtcReq& T = tp.r[s];
+          int cq = 0, ck = 0, cv = 0;
+          split(R.q_off, R.q_ts, &T.q_row, &cq); split(R.k_off, R.k_ts, &T.k_row, &ck); split(R.v_off, R.v_ts, &T.v_row, &cv);
+          if (!ok) break;
+          if (s == 0) { tp.q_col = cq; tp.k_col = ck; tp.v_col = cv; }
+          if (cq != tp.q_col || ck != tp.k_col || cv != tp.v_col) { ok = false; break; }
+          T.L = R.L; T.o_off = R.o_off;
+          rows_q = std::max<long long>(rows_q, T.q_row + R.L); rows_k = std::max<long long>(rows_k, T.k_row + R.L); rows_v = std::max<long long>(rows_v, T.v_row + R.L);
+          tp.tile_start[s] = tiles128;
+          tiles128 += (R.L + 127) / 128;
+        }
+        tp.tile_start[nr] = tiles128;
+        if (ok && (tp.q_col + (H - 1) * R0.q_hs + 64 > R0.q_ts || tp.k_col + (H - 1) * R0.k_hs + 64 > R0.k_ts || tp.v_col + (H - 1) * R0.v_hs + 64 > R0.v_ts ||
+                   (tp.q_col | tp.k_col | tp.v_col) % 8 || bo.off % 16 || !(G.scale > 0.f)))
+          ok = false;
+        if (ok) {
+          tp.n_req = nr; tp.H = H;
+          tp.q_hs = R0.q_hs; tp.k_hs = R0.k_hs; tp.v_hs = R0.v_hs; tp.o_ts = R0.o_ts; tp.o_hs = R0.o_hs;
+          tp.scale_log2e = ap.scale_log2e;
+          const int q_ts = R0.q_ts, k_ts = R0.k_ts, v_ts = R0.v_ts;
+          struct Cache { const void* q = nullptr; const void* k = nullptr; const void* v = nullptr; CUtensorMap tq, tk, tv; };
+          auto cache = std::make_shared<Cache>();
+          add(gi, 1, [=](const RunCtx& x) mutable {
+            const void* Q = x.resolve(bq);
+            const void* Kp = x.resolve(bk);
+            const void* V = x.resolve(bv);
+            if (cache->q != Q || cache->k != Kp || cache->v != V) {
+              if (!encode_bf16_2d(&cache->tq, Q, rows_q, q_ts, q_ts, 128) || !encode_bf16_2d(&cache->tk, Kp, rows_k, k_ts, k_ts, 64) ||
+                  !encode_bf16_2d(&cache->tv, V, rows_v, v_ts, v_ts, 64))
+                return cudaErrorInvalidValue;
+              cache->q = Q; cache->k = Kp; cache->v = V;
+            }
+            tp.o = reinterpret_cast<__nv_bfloat16*>(x.resolve(bo));
+            tp.status = reinterpret_cast<int*>(x.arena);
+            static bool once = (cudaFuncSetAttribute(k::attention_tcgen05_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, k::ATC_SMEM), true);
+            (void)once;
+            launch_pdl(k::attention_tcgen05_bf16, dim3(static_cast<unsigned>(tiles128) * tp.H), dim3(k::ATC_THREADS), k::ATC_SMEM, x.stream,
+                       cache->tq, cache->tk, cache->tv, tp);
+            return cudaGetLastError();
+          });
+          continue;
+        }
+      }
       add(gi, 1, [=](const RunCtx& x) mutable {
         ap.q = reinterpret_cast<const __nv_bfloat16*>(x.resolve(bq));
         ap.k = reinterpret_cast<const __nv_bfloat16*>(x.resolve(bk));

