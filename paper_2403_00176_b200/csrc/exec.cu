@@ -387,6 +387,8 @@ struct Builder {
     Status s = row_segments({G.a, G.out}, &D, &lds, &segs);
     if (s != OK) return s;
     if (lds[0] != D || lds[1] != D || D % 8 || D > 1024) return build_chain(gi, G, true);
+    // the row kernel reads gamma and beta before it waits for the previous kernel: they must be constants
+    if (g.tensors[G.gamma].kind != TKind::CONST || g.tensors[G.beta].kind != TKind::CONST) return build_chain(gi, G, true);
     Ptr pg = ptr_of(G.gamma, 0), pb = ptr_of(G.beta, 0);
     const float eps = G.eps;
     const int ch = static_cast<int>((D / 8 + 31) / 32);

@@ -98,12 +98,19 @@ template <int CH>
 __global__ void __launch_bounds__(256) layernorm_bf16(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ gamma,
                                                        const __nv_bfloat16* __restrict__ beta, __nv_bfloat16* __restrict__ y,
                                                        long long rows, int D, float eps) {
-  ptx::pdl_wait();
-  ptx::pdl_launch();
+  // gamma and beta are constants of the graph: fetch them before waiting for the previous kernel
   const int lane = threadIdx.x & 31;
   const long long row = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
-  if (row >= rows) return;
   const int nvec = D >> 3;
+  uint4 g4[CH], b4[CH];
+#pragma unroll
+  for (int c = 0; c < CH; ++c) {
+    const int i = c * 32 + lane;
+    if (i < nvec) { g4[c] = reinterpret_cast<const uint4*>(gamma)[i]; b4[c] = reinterpret_cast<const uint4*>(beta)[i]; }
+  }
+  ptx::pdl_launch();
+  ptx::pdl_wait();
+  if (row >= rows) return;
   const uint4* xr = reinterpret_cast<const uint4*>(x + row * D);
   float v[CH][8];
   float s = 0.f;
@@ -134,9 +141,9 @@ __global__ void __launch_bounds__(256) layernorm_bf16(const __nv_bfloat16* __res
   for (int c = 0; c < CH; ++c) {
     const int i = c * 32 + lane;
     if (i < nvec) {
-      uint4 g4 = reinterpret_cast<const uint4*>(gamma)[i], b4 = reinterpret_cast<const uint4*>(beta)[i], o;
-      const __nv_bfloat162* gh = reinterpret_cast<const __nv_bfloat162*>(&g4);
-      const __nv_bfloat162* bh = reinterpret_cast<const __nv_bfloat162*>(&b4);
+      uint4 o;
+      const __nv_bfloat162* gh = reinterpret_cast<const __nv_bfloat162*>(&g4[c]);
+      const __nv_bfloat162* bh = reinterpret_cast<const __nv_bfloat162*>(&b4[c]);
       __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&o);
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
