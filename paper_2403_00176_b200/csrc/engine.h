@@ -1,5 +1,6 @@
 // Fused groups, per-request binding, arena memory plan and launch plan.
 #pragma once
+#include <initializer_list>
 #include <memory>
 #include <string>
 #include <vector>
@@ -65,6 +66,9 @@ struct Compiled {
   std::vector<int> node_folded;       // per node: 1 = evaluated by RDP (shape arithmetic) or a pure view
   int n_subgraphs = 1;
   // prepacked (transposed, K-major) copies of GEMM weights
+  // every distinct extent expression once: binding evaluates each per request, tensors index the table
+  std::vector<Expr> dim_exprs;
+  std::vector<std::vector<int>> dim_expr_id;   // [tensor][axis] -> dim_exprs index, -1 if the extent is unknown
   std::vector<int> packed_consts;     // tensor ids
   std::vector<size_t> packed_off;     // byte offsets in the prepack workspace
   size_t packed_bytes = 0;
@@ -80,11 +84,36 @@ Status form_groups(Compiled* c);
 Status prepack_weights(Compiled* c, void* workspace, size_t bytes, void* stream);
 
 // ---- per-request binding (H0: substitute symbol values into every expression)
+// Extents or strides of one tensor instance, stored inline: binding and planning create one per
+// (tensor, request) and a heap vector for each was most of their cost.
+constexpr int MAX_RANK = 8;
+struct DimVec {
+  int64_t v[MAX_RANK];
+  int n = 0;
+  DimVec() {}
+  DimVec(std::initializer_list<int64_t> l) { for (auto x : l) v[n++] = x; }
+  DimVec(size_t count, int64_t val) : n(static_cast<int>(count)) { for (int i = 0; i < n; ++i) v[i] = val; }
+  size_t size() const { return static_cast<size_t>(n); }
+  bool empty() const { return n == 0; }
+  int64_t& operator[](size_t i) { return v[i]; }
+  const int64_t& operator[](size_t i) const { return v[i]; }
+  int64_t* begin() { return v; }
+  int64_t* end() { return v + n; }
+  const int64_t* begin() const { return v; }
+  const int64_t* end() const { return v + n; }
+  int64_t back() const { return v[n - 1]; }
+  void resize(size_t k, int64_t val = 0) { for (int i = n; i < static_cast<int>(k); ++i) v[i] = val; n = static_cast<int>(k); }
+  void assign(size_t k, int64_t val) { n = static_cast<int>(k); for (int i = 0; i < n; ++i) v[i] = val; }
+  void push_back(int64_t x) { v[n++] = x; }
+  bool operator==(const DimVec& o) const { if (n != o.n) return false; for (int i = 0; i < n; ++i) if (v[i] != o.v[i]) return false; return true; }
+  bool operator!=(const DimVec& o) const { return !(*this == o); }
+};
+
 struct Binding {
   const Compiled* c = nullptr;
   int n_req = 0;
-  std::vector<std::vector<int64_t>> vals;               // [req][atom]
-  std::vector<std::vector<std::vector<int64_t>>> dims;  // [tensor][req][rank]; empty if not evaluable yet
+  std::vector<std::vector<int64_t>> vals;   // [req][atom]
+  std::vector<std::vector<DimVec>> dims;    // [tensor][req]; empty if not evaluable yet
   std::string err;
 };
 Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* names, const int64_t* values, Binding* out);
@@ -93,7 +122,7 @@ Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* na
 struct View {                 // one tensor of one request, resolved to storage
   int root = -1;              // tensor id owning the bytes
   int64_t offset = 0;         // elements from the start of the root's instance for this request
-  std::vector<int64_t> dims, strides;  // elements
+  DimVec dims, strides;       // elements
   bool contiguous() const {
     int64_t s = 1;
     for (int i = static_cast<int>(dims.size()) - 1; i >= 0; --i) { if (dims[i] != 1 && strides[i] != s) return false; s *= dims[i]; }

@@ -63,7 +63,7 @@ cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t sme
   return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
 
-int64_t numel(const std::vector<int64_t>& d) { int64_t n = 1; for (auto v : d) n *= v; return n; }
+int64_t numel(const DimVec& d) { int64_t n = 1; for (auto v : d) n *= v; return n; }
 
 struct Builder {
   Plan& p;

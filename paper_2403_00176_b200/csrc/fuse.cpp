@@ -500,9 +500,31 @@ struct Fuser {
 
 }  // namespace
 
+// Table of the distinct extent expressions of the graph (canonical form as the key).
+static void index_dim_exprs(Compiled* c) {
+  const Graph& g = c->g;
+  c->dim_exprs.clear();
+  c->dim_expr_id.assign(g.tensors.size(), {});
+  std::map<std::string, int> seen;
+  for (size_t t = 0; t < g.tensors.size(); ++t) {
+    const ShapeVal& s = g.tensors[t].S;
+    if (s.rank < 0) continue;
+    c->dim_expr_id[t].assign(s.rank, -1);
+    for (int i = 0; i < s.rank; ++i) {
+      if (!s.dims[i].known()) continue;
+      const std::string key = e_str(g.cx, s.dims[i].e);
+      auto it = seen.find(key);
+      if (it == seen.end()) { it = seen.emplace(key, static_cast<int>(c->dim_exprs.size())).first; c->dim_exprs.push_back(s.dims[i].e); }
+      c->dim_expr_id[t][i] = it->second;
+    }
+  }
+}
+
 Status form_groups(Compiled* c) {
   Fuser f(*c);
-  return f.run();
+  Status s = f.run();
+  if (s == OK) index_dim_exprs(c);
+  return s;
 }
 
 }  // namespace sod2

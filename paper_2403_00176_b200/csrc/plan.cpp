@@ -2,6 +2,9 @@
 // run-time memory allocation plan (Section 4.4.1: one linear arena, planned at execution time once
 // all sizes are known, greedy from the peak-memory step outwards).
 #include <algorithm>
+#include <chrono>
+#include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 
@@ -34,49 +37,64 @@ Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* na
       int64_t x = e_eval(g.cx, as.a, out->vals[r], &ok1), y = e_eval(g.cx, as.b, out->vals[r], &ok2);
       if (ok1 && ok2 && x != y) { out->err = "shape conflict: " + as.what + " (" + std::to_string(x) + " vs " + std::to_string(y) + ")"; return E_SHAPE_CONFLICT; }
     }
-  // all non-linear atoms once per request (children first), then every dim is a flat polynomial
-  std::vector<std::vector<int64_t>> atom_vals(n_req);
-  for (int r = 0; r < n_req; ++r) { atom_vals[r] = out->vals[r]; e_eval_atoms(g.cx, &atom_vals[r]); }
+  // all non-linear atoms once per request (children first), then every distinct extent expression once
+  // per request as a flat polynomial; tensors pick their extents from that table
+  const size_t U = c->dim_exprs.size();
+  std::vector<int64_t> uval(static_cast<size_t>(n_req) * U);
+  std::vector<char> uok(static_cast<size_t>(n_req) * U);
+  std::vector<int64_t> atom_vals;
+  for (int r = 0; r < n_req; ++r) {
+    atom_vals = out->vals[r];
+    e_eval_atoms(g.cx, &atom_vals);
+    for (size_t u = 0; u < U; ++u) {
+      bool ok;
+      int64_t v = e_eval_flat(c->dim_exprs[u], atom_vals, &ok);
+      if (!ok) v = e_upper(g.cx, c->dim_exprs[u], out->vals[r], &ok);   // depends on a runtime symbol: static upper bound for planning
+      uval[r * U + u] = v;
+      uok[r * U + u] = ok;
+    }
+  }
   out->dims.assign(g.tensors.size(), {});
   for (size_t t = 0; t < g.tensors.size(); ++t) {
     const ShapeVal& s = g.tensors[t].S;
     if (s.rank < 0) continue;
+    if (s.rank > MAX_RANK) { out->err = "rank above " + std::to_string(MAX_RANK) + " for " + g.tensors[t].name; return E_UNSUPPORTED_OP; }
+    const std::vector<int>& ids = c->dim_expr_id[t];
     bool evaluable = true;
-    std::vector<std::vector<int64_t>> per(n_req, std::vector<int64_t>(s.rank));
+    for (int i = 0; i < s.rank; ++i) if (ids[i] < 0) evaluable = false;
     for (int r = 0; r < n_req && evaluable; ++r)
+      for (int i = 0; i < s.rank; ++i) if (!uok[r * U + ids[i]]) { evaluable = false; break; }
+    if (!evaluable) continue;
+    std::vector<DimVec>& per = out->dims[t];
+    per.resize(n_req);
+    for (int r = 0; r < n_req; ++r) {
+      per[r].n = s.rank;
       for (int i = 0; i < s.rank; ++i) {
-        if (!s.dims[i].known()) { evaluable = false; break; }
-        bool ok;
-        int64_t v = e_eval_flat(s.dims[i].e, atom_vals[r], &ok);
-        if (!ok) {  // depends on a runtime symbol: use its static upper bound for planning
-          v = e_upper(g.cx, s.dims[i].e, out->vals[r], &ok);
-          if (!ok) { evaluable = false; break; }
-        }
+        const int64_t v = uval[r * U + ids[i]];
         if (v < 0) { out->err = "negative extent for " + g.tensors[t].name; return E_BAD_DIM; }
-        per[r][i] = v;
+        per[r].v[i] = v;
       }
-    if (evaluable) out->dims[t] = std::move(per);
+    }
   }
   return OK;
 }
 
 namespace {
 
-int64_t numel(const std::vector<int64_t>& d) {
+int64_t numel(const DimVec& d) {
   int64_t n = 1;
   for (int64_t v : d) n *= v;
   return n;
 }
-std::vector<int64_t> contiguous_strides(const std::vector<int64_t>& d) {
-  std::vector<int64_t> s(d.size());
+DimVec contiguous_strides(const DimVec& d) {
+  DimVec s(d.size(), 0);
   int64_t acc = 1;
   for (int i = static_cast<int>(d.size()) - 1; i >= 0; --i) { s[i] = acc; acc *= d[i]; }
   return s;
 }
 
 // strides of `newd` viewing memory laid out as (oldd, olds); false if a copy would be needed
-bool reshape_view(const std::vector<int64_t>& oldd, const std::vector<int64_t>& olds, const std::vector<int64_t>& newd,
-                  std::vector<int64_t>* news) {
+bool reshape_view(const DimVec& oldd, const DimVec& olds, const DimVec& newd, DimVec* news) {
   news->assign(newd.size(), 0);
   if (numel(oldd) == 0) { *news = contiguous_strides(newd); return true; }
   int vd = static_cast<int>(newd.size()) - 1;
@@ -153,7 +171,7 @@ struct Planner {
       int o = st.other;
       Status s = resolve(o);
       if (s != OK) return s;
-      std::vector<int64_t> perm = n.attr_list("perm");
+      const std::vector<int64_t> perm = n.attr_list("perm");
       for (int r = 0; r < p.n_req; ++r) {
         const View& vo = p.views[o][r];
         View& v = p.views[t][r];
@@ -170,23 +188,30 @@ struct Planner {
     int in = st.other;
     Status s = resolve(in);
     if (s != OK) return s;
+    const int kind = n.op == "Transpose" ? 0 : n.op == "Reshape" ? 1 : 2;
+    std::vector<int64_t> perm, sl_start, sl_step;
+    if (kind == 0) perm = n.attr_list("perm");
+    if (kind == 2)
+      for (size_t ax = 0; ax < p.views[in][0].dims.size(); ++ax) {
+        sl_start.push_back(n.attr_i("_start" + std::to_string(ax), 0));
+        sl_step.push_back(n.attr_i("_step" + std::to_string(ax), 1));
+      }
     for (int r = 0; r < p.n_req; ++r) {
       const View& vi = p.views[in][r];
       View& v = p.views[t][r];
       v.root = vi.root;
       v.offset = vi.offset;
       v.dims = b.dims[t][r];
-      if (n.op == "Transpose") {
-        std::vector<int64_t> perm = n.attr_list("perm");
+      if (kind == 0) {
         v.strides.resize(perm.size());
         for (size_t i = 0; i < perm.size(); ++i) v.strides[i] = vi.strides[perm[i]];
-      } else if (n.op == "Reshape") {
+      } else if (kind == 1) {
         if (!reshape_view(vi.dims, vi.strides, v.dims, &v.strides))
           return fail(E_UNSUPPORTED_OP, "Reshape producing " + g.tensors[t].name + " is not a view of its input layout");
       } else {  // Slice
         v.strides = vi.strides;
         for (size_t ax = 0; ax < vi.dims.size(); ++ax) {
-          int64_t st0 = n.attr_i("_start" + std::to_string(ax), 0), step = n.attr_i("_step" + std::to_string(ax), 1);
+          const int64_t st0 = sl_start[ax], step = sl_step[ax];
           v.offset += st0 * vi.strides[ax];
           v.strides[ax] = vi.strides[ax] * step;
         }
@@ -296,10 +321,19 @@ Status make_plan(const Compiled* c, const Binding* b, Plan* p) {
   p->c = c;
   p->b = b;
   p->n_req = b->n_req;
+  static const bool prof = getenv("SOD2_HOST_PROFILE") != nullptr;
+  auto t0 = std::chrono::steady_clock::now();
   Planner pl(*c, *b, *p);
   Status s = pl.run();
   if (s != OK) return s;
-  return build_launches(p);
+  auto t1 = std::chrono::steady_clock::now();
+  s = build_launches(p);
+  if (prof) {
+    auto t2 = std::chrono::steady_clock::now();
+    fprintf(stderr, "[sod2] plan: views+liveness+arena %.1f us, launches %.1f us\n", std::chrono::duration<double, std::micro>(t1 - t0).count(),
+            std::chrono::duration<double, std::micro>(t2 - t1).count());
+  }
+  return s;
 }
 
 }  // namespace sod2
