@@ -165,6 +165,7 @@ def run_ours(args):
     e2e_times = []
     h2d = d2h = 0
     pinned_in = {}
+    pinned_out = {}
     for i in range(min(args.steps, 10) + 1):
         j = my_batches[i % len(my_batches)]
         reqs = preps[i % len(preps)].reqs
@@ -172,6 +173,7 @@ def run_ours(args):
         key = i % len(preps)
         if key not in pinned_in:
             pinned_in[key] = [torch.from_numpy(h).pin_memory() for h in hin]
+            pinned_out[key] = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in preps[key].out_dev]
         torch.cuda.synchronize(dev)
         t0 = time.perf_counter()
         b = sess.graph.bind_dims(wl.sym_names, [[r.syms[s] for s in wl.sym_names] for r in reqs])
@@ -181,7 +183,9 @@ def run_ours(args):
             dst.copy_(src, non_blocking=True)
         pl.run([t.data_ptr() for t in pr.in_dev], [t.data_ptr() for t in pr.out_dev], pr.arena.data_ptr(), pr.arena.numel(),
                sess.stream)
-        host_out = [t.cpu() for t in pr.out_dev]
+        host_out = pinned_out[key]
+        for dst, src in zip(host_out, pr.out_dev):
+            dst.copy_(src, non_blocking=True)
         torch.cuda.synchronize(dev)
         dt = (time.perf_counter() - t0) * 1e3
         if i > 0:
@@ -230,7 +234,7 @@ def run_ours(args):
             "gpu_launches": int(launches),
             "clocks": clocks,
             "e2e": {"value": e2e_ms, "unit": "ms/inference", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-                    "includes": "bind_dims + plan + H2D (pinned) + run + D2H"},
+                    "includes": "bind_dims + plan + H2D (pinned) + run + D2H (pinned)"},
             "plan_us_per_batch": plan_us,
             "arena": mem,
             "roofline": {"bound": "tensor", "achieved": gemm["tflops"], "peak": peaks["tf_sustained"], "unit": "TFLOP/s",

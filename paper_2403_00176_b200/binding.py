@@ -18,6 +18,7 @@ STATUS = ["SOD2_OK", "SOD2_E_INVALID_ARG", "SOD2_E_PARSE", "SOD2_E_UNSUPPORTED_O
           "SOD2_E_ARENA_TOO_SMALL", "SOD2_E_MISALIGNED", "SOD2_E_CUDA", "SOD2_E_TIMEOUT", "SOD2_E_INTERNAL"]
 OPT_NO_FUSION = 1
 OPT_NO_REUSE = 2
+OPT_SPLITK_LN = 4
 DYN_CLASS = ["ISDO", "ISDOS", "ISVDOS", "EDO"]
 
 

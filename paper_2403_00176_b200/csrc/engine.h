@@ -12,6 +12,7 @@ namespace sod2 {
 enum OptFlags : uint32_t {
   OPT_NO_FUSION = 1u,   // every operator is its own group (fused-vs-unfused comparison)
   OPT_NO_REUSE = 2u,    // every arena tensor gets its own slot (keeps all intermediates readable after a run)
+  OPT_SPLITK_LN = 4u,   // a bf16 GEMM (+bias, +residual) followed by LayerNorm becomes one group: split-K GEMM + finishing kernel
 };
 
 enum class GKind {

@@ -191,11 +191,74 @@ struct Builder {
       return OK;
     }
     // bf16 on tcgen05
-    if (G.has_ln) return fail(E_UNSUPPORTED_OP, "bf16 GEMM epilogue: LayerNorm tail is not fused");
     if (K % 64) return fail(E_UNSUPPORTED_OP, "bf16 GEMM needs K % 64 == 0 (k-chunk tensor maps)");
     if (lds[0] % 8 || lds[1] % 8 || N % 8 || (G.res >= 0 && lds[2] % 8)) return fail(E_UNSUPPORTED_OP, "GEMM operand rows must be 16-byte multiples");
     size_t pk = 0;
     for (size_t i = 0; i < c.packed_consts.size(); ++i) if (c.packed_consts[i] == G.w) pk = c.packed_off[i];
+    if (G.has_ln) {
+      // ---- GEMM (+bias, +residual) -> LayerNorm: K ranges of every 128x256 tile go to different CTAs,
+      // which store their fp32 partial tiles into slabs of a workspace in the scratch region; the finishing
+      // kernel adds a row's slabs in order, adds bias and residual and normalises.
+      if (lds[1] != N || N > 1024) return fail(E_UNSUPPORTED_OP, "GEMM + LayerNorm: output rows must be contiguous and at most 1024 wide");
+      Ptr pg = ptr_of(G.gamma, 0), pbe = ptr_of(G.beta, 0);
+      const float eps = G.eps;
+      const int ch = static_cast<int>((N / 8 + 31) / 32);
+      for (auto& sg : segs) {
+        if (sg.rows == 0) continue;
+        Ptr pa = ptr_of(G.a, sg.r0), po = ptr_of(G.out, sg.r0), pr = G.res >= 0 ? ptr_of(G.res, sg.r0) : Ptr();
+        Ptr pw; pw.where = 5; pw.off = static_cast<int64_t>(pk);
+        Ptr pb = G.bias >= 0 ? ptr_of(G.bias, 0) : Ptr();
+        const int M = static_cast<int>(sg.rows);
+        const int64_t lda = lds[0], ldr = G.res >= 0 ? lds[2] : 0;
+        const int tiles = ((M + 127) / 128) * static_cast<int>((N + 255) / 256);
+        const int kstages = static_cast<int>(K / 64);
+        // as many K ranges as fill the SMs once, at least four stages each
+        int splits = std::max(1, std::min(148 / std::max(tiles, 1), kstages / 4));
+        const int per = (kstages + splits - 1) / splits;
+        splits = (kstages + per - 1) / per;
+        const size_t ws_bytes = static_cast<size_t>(splits) * M * N * 4;
+        scratch_need = std::max(scratch_need, ws_bytes);
+        const bool hb = G.bias >= 0, hr = G.res >= 0;
+        struct Cache { const void* a = nullptr; const void* w = nullptr; const void* o = nullptr; CUtensorMap ta, tb, to; };
+        auto cache = std::make_shared<Cache>();
+        add(gi, 2, [=](const RunCtx& x) {
+          const void* A = x.resolve(pa);
+          const void* Wt = x.resolve(pw);
+          float* ws = reinterpret_cast<float*>(x.arena + x.plan->scratch_off[0]);
+          if (cache->a != A || cache->w != Wt || cache->o != ws) {
+            if (!encode_bf16_kchunks(&cache->ta, A, M, K, lda, 128, 1) || !encode_bf16_kchunks(&cache->tb, Wt, N, K, K, 256, 1) ||
+                !encode_f32_slabs(&cache->to, ws, M, N, splits, 128))
+              return cudaErrorInvalidValue;
+            cache->a = A; cache->w = Wt; cache->o = ws;
+          }
+          k::GemmEpilogue ep{};
+          ep.status = reinterpret_cast<int*>(x.arena);
+          ep.splits = splits;
+          ep.stages_per_split = per;
+          const int grid = std::min(tiles * splits, x.plan->sm_count);
+          constexpr int smem = k::GemmSmem<256, 1, 4>::TOTAL;
+          static bool once = (cudaFuncSetAttribute(k::gemm_bf16_tcgen05<256, 1, 4, 0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);
+          (void)once;
+          launch_pdl(k::gemm_bf16_tcgen05<256, 1, 4, 0, true>, dim3(grid), dim3(k::GEMM_THREADS), smem, x.stream, cache->ta, cache->tb, cache->to,
+                     cache->to, M, static_cast<int>(N), static_cast<int>(K), ep);
+          auto* Bi = hb ? reinterpret_cast<const __nv_bfloat16*>(x.resolve(pb)) : nullptr;
+          auto* R = hr ? reinterpret_cast<const __nv_bfloat16*>(x.resolve(pr)) : nullptr;
+          auto* Gm = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pg));
+          auto* Bt = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pbe));
+          auto* Y = reinterpret_cast<__nv_bfloat16*>(x.resolve(po));
+          const long long rows = M;
+          const unsigned lgrid = static_cast<unsigned>((rows + 7) / 8);
+          switch (ch) {
+            case 1: launch_pdl(k::splitk_ln_finish<1>, dim3(lgrid), dim3(256), 0, x.stream, static_cast<const float*>(ws), splits, Bi, R, static_cast<long long>(ldr), Gm, Bt, Y, rows, static_cast<int>(N), eps); break;
+            case 2: launch_pdl(k::splitk_ln_finish<2>, dim3(lgrid), dim3(256), 0, x.stream, static_cast<const float*>(ws), splits, Bi, R, static_cast<long long>(ldr), Gm, Bt, Y, rows, static_cast<int>(N), eps); break;
+            case 3: launch_pdl(k::splitk_ln_finish<3>, dim3(lgrid), dim3(256), 0, x.stream, static_cast<const float*>(ws), splits, Bi, R, static_cast<long long>(ldr), Gm, Bt, Y, rows, static_cast<int>(N), eps); break;
+            default: launch_pdl(k::splitk_ln_finish<4>, dim3(lgrid), dim3(256), 0, x.stream, static_cast<const float*>(ws), splits, Bi, R, static_cast<long long>(ldr), Gm, Bt, Y, rows, static_cast<int>(N), eps); break;
+          }
+          return cudaGetLastError();
+        });
+      }
+      return OK;
+    }
     for (auto& sg : segs) {
       if (sg.rows == 0) continue;
       Ptr pa = ptr_of(G.a, sg.r0), po = ptr_of(G.out, sg.r0), pr = G.res >= 0 ? ptr_of(G.res, sg.r0) : Ptr();

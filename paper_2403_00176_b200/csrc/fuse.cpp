@@ -142,6 +142,19 @@ struct Fuser {
         G.nodes.push_back(nx); inside.insert(nx);
         cur = n.outs[0];
         break;
+      } else if (n.op == "LayerNormalization" && G.kind == GKind::GEMM && g.tensors[cur].dtype == DType::BF16 && n.attr_i("axis", -1) == -1 &&
+                 G.act2 == 0 && (c.flags & OPT_SPLITK_LN)) {
+        // bf16 GEMM (+bias, +residual) -> LayerNorm: the GEMM runs split along K into an fp32 workspace and
+        // the finishing kernel applies bias, residual and the normalisation (row width must fit a warp)
+        const ShapeVal& cs = g.tensors[cur].S;
+        const Dim& nd = cs.dims[cs.rank - 1];
+        if (!(nd.e.is_const() && nd.e.const_value() <= 1024 && nd.e.const_value() % 8 == 0)) break;
+        if (G.act != 0) break;
+        if (g.tensors[n.ins[1]].kind != TKind::CONST || g.tensors[n.ins[2]].kind != TKind::CONST) break;
+        G.has_ln = 1; G.gamma = n.ins[1]; G.beta = n.ins[2]; G.eps = static_cast<float>(n.attr_f("epsilon", 1e-5));
+        G.nodes.push_back(nx); inside.insert(nx);
+        cur = n.outs[0];
+        break;
       } else break;
       G.nodes.push_back(nx);
       inside.insert(nx);

@@ -35,6 +35,8 @@ struct GemmEpilogue {
   int has_residual;           // residual arrives through its own tensor map
   int act2;                   // applied after the residual add (ACT_NONE or ACT_RELU); the pre-residual one is a template parameter
   int* status;                // device word; set non-zero if a bounded wait ran out
+  int splits;                 // split-K kernels: number of K ranges per tile (work item = tile x range), else unused
+  int stages_per_split;       // split-K kernels: pipeline stages per K range
 };
 
 constexpr int GEMM_BM = 128;
@@ -81,6 +83,10 @@ __device__ __forceinline__ void tma_store_2d(const void* tmap, const void* src, 
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
                ::"l"(tmap), "r"(ptx::smem_u32(src)), "r"(x), "r"(y) : "memory");
 }
+__device__ __forceinline__ void tma_store_3d(const void* tmap, const void* src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(tmap), "r"(ptx::smem_u32(src)), "r"(x), "r"(y), "r"(z) : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
@@ -90,13 +96,17 @@ __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 256;"
 // {64, 128 or BN, KCH}: one instruction fills KCH consecutive swizzled [rows x 64] chunks.
 // B must be a constant of the graph (prepacked weights): its producer does not wait for the
 // previous kernel in the stream.
-template <int BN, int KCH, int STAGES, int ACT>
+// SPLITK: a work item is (tile, K range); the epilogue stores the raw fp32 partial tile into slab
+// `range` of an fp32 [ranges, M, N] workspace (tmOut is then a 3-D fp32 map with boxes of 32 columns)
+// and a finishing kernel adds the slabs in a fixed order and applies bias, residual and LayerNorm.
+// This spreads a GEMM with few output tiles and a long K over all SMs, deterministically.
+template <int BN, int KCH, int STAGES, int ACT, bool SPLITK = false>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmRes,
                   int M, int N, int K, GemmEpilogue ep) {
   using S = GemmSmem<BN, KCH, STAGES>;
-  constexpr int PASSES = BN / GEMM_PASS_COLS;
+  constexpr int PASSES = SPLITK ? BN / 32 : BN / GEMM_PASS_COLS;   // split-K passes are 32 fp32 columns (128-byte rows)
   constexpr int NSB = GEMM_NSB;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -121,15 +131,20 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_m = (M + GEMM_BM - 1) / GEMM_BM, tiles_n = (N + BN - 1) / BN;
-  const int num_tiles = tiles_m * tiles_n;
   const int kchunks = K / 64;
   const int kstages = (kchunks + KCH - 1) / KCH;
+  const int out_tiles = tiles_m * tiles_n;
+  const int num_tiles = SPLITK ? out_tiles * ep.splits : out_tiles;   // work items; item w = (tile w % out_tiles, K range w / out_tiles)
+  auto k_range = [&](int w, int* ks0, int* ks1) {
+    if (SPLITK) { *ks0 = (w / out_tiles) * ep.stages_per_split; *ks1 = min(kstages, *ks0 + ep.stages_per_split); }
+    else { *ks0 = 0; *ks1 = kstages; }
+  };
   constexpr uint32_t TMEM_COLS = 2 * BN;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(&full[s], 2); ptx::mbar_init(&empty[s], 1); }
     for (int b = 0; b < 2; ++b) { ptx::mbar_init(&tmem_full[b], 1); ptx::mbar_init(&tmem_empty[b], 8); }
-    for (int b = 0; b < NSB; ++b) { ptx::mbar_init(&buf_ready[b], 1); ptx::mbar_init(&buf_filled[b], 8); }
+    for (int b = 0; b < NSB; ++b) { ptx::mbar_init(&buf_ready[b], 1); ptx::mbar_init(&buf_filled[b], SPLITK ? 4 : 8); }
     *dead = 0;
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
@@ -156,9 +171,12 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       ptx::pdl_wait();
       SOD2_TRACE(0, 2)
       int n = 0;
-      for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
+      for (int w = blockIdx.x; w < num_tiles; w += gridDim.x) {
+        const int t = SPLITK ? w % out_tiles : w;
         const int m0 = (t % tiles_m) * GEMM_BM;
-        for (int ks = 0; ks < kstages; ++ks, ++n) {
+        int ks0, ks1;
+        k_range(w, &ks0, &ks1);
+        for (int ks = ks0; ks < ks1; ++ks, ++n) {
           const int s = n % STAGES;
           if (n >= STAGES) ptx::mbar_wait(&empty[s], ((n / STAGES) - 1) & 1, dead);
           ptx::mbar_expect_tx(&full[s], S::A_BYTES);
@@ -170,9 +188,12 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     if (lane == 0) {
       // ---- TMA producer: B stages
       int n = 0;
-      for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
+      for (int w = blockIdx.x; w < num_tiles; w += gridDim.x) {
+        const int t = SPLITK ? w % out_tiles : w;
         const int n0 = (t / tiles_m) * BN;
-        for (int ks = 0; ks < kstages; ++ks, ++n) {
+        int ks0, ks1;
+        k_range(w, &ks0, &ks1);
+        for (int ks = ks0; ks < ks1; ++ks, ++n) {
           const int s = n % STAGES;
           if (n >= STAGES) ptx::mbar_wait(&empty[s], ((n / STAGES) - 1) & 1, dead);
           ptx::mbar_expect_tx(&full[s], S::B_BYTES);
@@ -185,12 +206,14 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       // ---- MMA issuer
       constexpr uint32_t idesc = ptx::idesc_bf16(GEMM_BM, BN);
       int n = 0, j = 0;
-      for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++j) {
+      for (int w = blockIdx.x; w < num_tiles; w += gridDim.x, ++j) {
         const int acc = j & 1;
         if (j >= 2) ptx::mbar_wait(&tmem_empty[acc], ((j >> 1) - 1) & 1, dead);
         ptx::tc_fence_after();
         const uint32_t d = tmem + acc * BN;
-        for (int ks = 0; ks < kstages; ++ks, ++n) {
+        int ks0, ks1;
+        k_range(w, &ks0, &ks1);
+        for (int ks = ks0; ks < ks1; ++ks, ++n) {
           const int s = n % STAGES;
           ptx::mbar_wait(&full[s], (n / STAGES) & 1, dead);
           ptx::tc_fence_after();
@@ -202,7 +225,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               const uint64_t ad = ptx::smem_desc_sw128(a + c * (GEMM_BM * 128));
               const uint64_t bd = ptx::smem_desc_sw128(a + S::A_BYTES + c * (BN * 128));
 #pragma unroll
-              for (int kk = 0; kk < 4; ++kk) ptx::mma_bf16(d, ad + 2 * kk, bd + 2 * kk, idesc, (ks | c | kk) != 0);
+              for (int kk = 0; kk < 4; ++kk) ptx::mma_bf16(d, ad + 2 * kk, bd + 2 * kk, idesc, (ks > ks0) || c != 0 || kk != 0);
             }
           }
           ptx::mma_commit(&empty[s]);  // frees the stage once these MMAs have read it
@@ -223,11 +246,13 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       int my_tiles = 0;
       for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) ++my_tiles;
       const int U = my_tiles * PASSES;
+      constexpr int PASS_COLS = SPLITK ? 32 : GEMM_PASS_COLS;
       auto prepare = [&](int u) {
-        const int t = blockIdx.x + (u / PASSES) * gridDim.x;
-        const int m0 = (t % tiles_m) * GEMM_BM, np = (t / tiles_m) * BN + (u % PASSES) * GEMM_PASS_COLS;
+        const int w = blockIdx.x + (u / PASSES) * gridDim.x;
+        const int t = SPLITK ? w % out_tiles : w;
+        const int m0 = (t % tiles_m) * GEMM_BM, np = (t / tiles_m) * BN + (u % PASSES) * PASS_COLS;
         const int bsel = u % NSB;
-        if (ep.has_residual && np < N) {
+        if (!SPLITK && ep.has_residual && np < N) {
           ptx::mbar_expect_tx(&buf_ready[bsel], GEMM_STAGE_OUT);
           ptx::tma_load_2d(out_stage + bsel * GEMM_STAGE_OUT, &tmRes, np, m0, &buf_ready[bsel]);
         } else {
@@ -238,10 +263,12 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       for (int u = 0; u < U; ++u) {
         const int bsel = u % NSB;
         ptx::mbar_wait(&buf_filled[bsel], (u / NSB) & 1, dead);
-        const int t = blockIdx.x + (u / PASSES) * gridDim.x;
-        const int m0 = (t % tiles_m) * GEMM_BM, np = (t / tiles_m) * BN + (u % PASSES) * GEMM_PASS_COLS;
+        const int w = blockIdx.x + (u / PASSES) * gridDim.x;
+        const int t = SPLITK ? w % out_tiles : w;
+        const int m0 = (t % tiles_m) * GEMM_BM, np = (t / tiles_m) * BN + (u % PASSES) * PASS_COLS;
         if (np < N) {
-          tma_store_2d(&tmOut, out_stage + bsel * GEMM_STAGE_OUT, np, m0);
+          if (SPLITK) tma_store_3d(&tmOut, out_stage + bsel * GEMM_STAGE_OUT, np, m0, w / out_tiles);
+          else tma_store_2d(&tmOut, out_stage + bsel * GEMM_STAGE_OUT, np, m0);
           bulk_commit();
         }
         if (u + NSB < U) {
@@ -263,6 +290,44 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const int et = threadIdx.x - 96; // 0..255
     const int row = q * 32 + lane;   // row inside the tile
     ptx::pdl_wait();
+    if constexpr (SPLITK) {
+      // raw fp32 partial sums, 32 columns per pass; the warps of column half h take the passes of
+      // parity h, which are exactly the units of staging buffer h
+      int j = 0;
+      for (int w = blockIdx.x; w < num_tiles; w += gridDim.x, ++j) {
+        const int acc = j & 1;
+        const int n0 = ((w % out_tiles) / tiles_m) * BN;
+        ptx::mbar_wait_warp(&tmem_full[acc], (j >> 1) & 1, dead);
+        ptx::tc_fence_after();
+        const uint32_t taddr = tmem + (static_cast<uint32_t>(q * 32) << 16) + acc * BN;
+        uint32_t r[2][32];
+        ptx::tmem_ld32(taddr + half * 32, r[0]);
+#pragma unroll
+        for (int i = 0; i < PASSES / 2; ++i) {
+          const int ps = 2 * i + half;
+          const int u = j * PASSES + ps;
+          ptx::tmem_ld_wait();
+          if (i + 1 < PASSES / 2) {
+            ptx::tmem_ld32(taddr + (ps + 2) * 32, r[(i + 1) & 1]);
+          } else {
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&tmem_empty[acc]);
+          }
+          ptx::mbar_wait_warp(&buf_ready[half], (u / NSB) & 1, dead);
+          if (n0 + ps * 32 < N) {
+            uint8_t* obase = out_stage + half * GEMM_STAGE_OUT + row * 128;
+#pragma unroll
+            for (int g = 0; g < 8; ++g)
+              *reinterpret_cast<uint4*>(obase + ((g ^ (row & 7)) << 4)) =
+                  make_uint4(r[i & 1][4 * g], r[i & 1][4 * g + 1], r[i & 1][4 * g + 2], r[i & 1][4 * g + 3]);
+          }
+          ptx::fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&buf_filled[half]);
+        }
+      }
+    } else {
     int j = 0, u = 0;
     auto load_bias = [&](int t) -> float {
       const int idx = (t / tiles_m) * BN + et;
@@ -327,6 +392,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&buf_filled[bsel]);
       }
+    }
     }
   }
   ptx::tc_fence_before();

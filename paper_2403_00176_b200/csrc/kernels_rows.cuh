@@ -156,6 +156,90 @@ __global__ void __launch_bounds__(256) layernorm_bf16(const __nv_bfloat16* __res
 }
 
 // ---------------------------------------------------------------------------------------------
+// Finish of a split-K GEMM whose group ends in LayerNorm:
+//   y = LayerNorm(sum_s acc[s] + bias + residual) * gamma + beta,  acc = fp32 [splits, rows, D] workspace
+// holding the K ranges' partial products, added in slab order (deterministic).  The pre-normalisation
+// row never exists in bf16.
+template <int CH>
+__global__ void __launch_bounds__(256) splitk_ln_finish(const float* __restrict__ acc, int splits, const __nv_bfloat16* __restrict__ bias,
+                                                         const __nv_bfloat16* __restrict__ res, long long ldr,
+                                                         const __nv_bfloat16* __restrict__ gamma, const __nv_bfloat16* __restrict__ beta,
+                                                         __nv_bfloat16* __restrict__ y, long long rows, int D, float eps) {
+  const int lane = threadIdx.x & 31;
+  const long long row = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+  const int nvec = D >> 3;
+  uint4 g4[CH], b4[CH], c4[CH];
+#pragma unroll
+  for (int c = 0; c < CH; ++c) {
+    const int i = c * 32 + lane;
+    if (i < nvec) {
+      g4[c] = reinterpret_cast<const uint4*>(gamma)[i]; b4[c] = reinterpret_cast<const uint4*>(beta)[i];
+      c4[c] = bias ? reinterpret_cast<const uint4*>(bias)[i] : make_uint4(0, 0, 0, 0);
+    }
+  }
+  ptx::pdl_launch();
+  ptx::pdl_wait();
+  if (row >= rows) return;
+  const float4* ar = reinterpret_cast<const float4*>(acc + row * D);
+  const long long slab4 = rows * D / 4;      // float4 per slab
+  const uint4* rr = res ? reinterpret_cast<const uint4*>(res + row * ldr) : nullptr;
+  float v[CH][8];
+  float s = 0.f;
+#pragma unroll
+  for (int c = 0; c < CH; ++c) {
+    const int i = c * 32 + lane;
+    if (i < nvec) {
+      float4 a0 = ar[2 * i], a1 = ar[2 * i + 1];
+      for (int sp = 1; sp < splits; ++sp) {
+        const float4 b0 = ar[sp * slab4 + 2 * i], b1 = ar[sp * slab4 + 2 * i + 1];
+        a0.x += b0.x; a0.y += b0.y; a0.z += b0.z; a0.w += b0.w;
+        a1.x += b1.x; a1.y += b1.y; a1.z += b1.z; a1.w += b1.w;
+      }
+      const uint4 ru = rr ? rr[i] : make_uint4(0, 0, 0, 0);
+      const __nv_bfloat162* rh = reinterpret_cast<const __nv_bfloat162*>(&ru);
+      const __nv_bfloat162* ch = reinterpret_cast<const __nv_bfloat162*>(&c4[c]);
+      const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const float2 rf = __bfloat1622float2(rh[t]), cf = __bfloat1622float2(ch[t]);
+        v[c][2 * t] = a[2 * t] + cf.x + rf.x;
+        v[c][2 * t + 1] = a[2 * t + 1] + cf.y + rf.y;
+        s += v[c][2 * t] + v[c][2 * t + 1];
+      }
+    } else {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) v[c][t] = 0.f;
+    }
+  }
+  const float mu = warp_sum(s) / D;
+  float q = 0.f;
+#pragma unroll
+  for (int c = 0; c < CH; ++c)
+    if (c * 32 + lane < nvec) {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) { const float d = v[c][t] - mu; q += d * d; }
+    }
+  const float rstd = rsqrtf(warp_sum(q) / D + eps);
+  uint4* yr = reinterpret_cast<uint4*>(y + row * D);
+#pragma unroll
+  for (int c = 0; c < CH; ++c) {
+    const int i = c * 32 + lane;
+    if (i < nvec) {
+      uint4 o;
+      const __nv_bfloat162* gh = reinterpret_cast<const __nv_bfloat162*>(&g4[c]);
+      const __nv_bfloat162* bh = reinterpret_cast<const __nv_bfloat162*>(&b4[c]);
+      __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        float2 gf = __bfloat1622float2(gh[t]), bf = __bfloat1622float2(bh[t]);
+        oh[t] = __floats2bfloat162_rn((v[c][2 * t] - mu) * rstd * gf.x + bf.x, (v[c][2 * t + 1] - mu) * rstd * gf.y + bf.y);
+      }
+      yr[i] = o;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Generic fused chain: v = load(in0); v = op_i(v [, operand_i]) ...; optional softmax / LayerNorm
 // over the last dim; store. Index space = the group's output [d0..d3] (rank <= 4 after
 // right-alignment); every operand is read through its own strides, 0 on broadcast dims.

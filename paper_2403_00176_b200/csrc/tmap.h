@@ -39,6 +39,20 @@ inline bool encode_bf16_2d(CUtensorMap* tm, const void* base, uint64_t rows, uin
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// `slabs` row-major fp32 matrices [rows, cols] back to back, as {cols, rows, slabs}; box = {32 cols
+// (128-byte rows), box_rows, 1}, 128-B swizzle.  Rows past `rows` are clipped per slab.
+inline bool encode_f32_slabs(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint64_t slabs, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {cols, rows, slabs};
+  cuuint64_t strides[2] = {cols * 4, rows * cols * 4};
+  cuuint32_t box[3] = {32, box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Row-major bf16 matrix [rows, K] (K % 64 == 0) viewed as {64, rows, K/64}: the third coordinate
 // walks the 64-element k-chunks of a row, so one box {64, box_rows, kch} fills kch consecutive
 // swizzled [box_rows x 64] chunk tiles in shared memory.

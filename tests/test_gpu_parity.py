@@ -56,8 +56,8 @@ def test_fig4_chain_one_fused_version():
 EDGE_L = [1, 15, 16, 17, 63, 64, 65, 127, 128, 129, 200]
 
 
-def _encoder_edge(layers=2):
-    wl = WL.cfg2(layers=layers, D=128, H=2, F=256, n_requests=1, lmin=1, lmax=512)
+def _encoder_edge(layers=2, F=256):
+    wl = WL.cfg2(layers=layers, D=128, H=2, F=F, n_requests=1, lmin=1, lmax=512)
     rng = np.random.default_rng(11)
     reqs = [Request({"L": L}, {"x": bf16_round(rng.standard_normal((1, L, 128)).astype(np.float32))}) for L in EDGE_L]
     return wl, reqs
@@ -74,6 +74,25 @@ def test_cfg2_small_encoder_edge_lengths_lockstep():
         assert errs, "no materialised tensor was compared"
         bad = {k: v for k, v in errs.items() if not (isinstance(v, float) and v <= BF16_TOL)}
         assert not bad, (req.syms, bad)
+
+
+def test_cfg2_small_encoder_splitk_layernorm_groups_lockstep():
+    # opt-in form of the residual GEMM + LayerNorm pair: split-K GEMM into fp32 slabs + finishing kernel
+    # (F = 1024 gives the second GEMM 16 pipeline stages, i.e. several K ranges per tile)
+    wl, reqs = _encoder_edge(F=1024)
+    s, p, outs = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE | B.OPT_SPLITK_LN)
+    kinds = [s.graph.group_info(i)["kind"] for i in range(s.graph.num_groups())]
+    assert "layernorm" not in kinds
+    for r, req in enumerate(reqs):
+        ref = _oracle_out(wl, req, "y")
+        assert O.rel_err(outs[r]["y"], ref) <= BF16_TOL
+        errs = lockstep(wl, s, p, outs, r, BF16_TOL)
+        bad = {k: v for k, v in errs.items() if not (isinstance(v, float) and v <= BF16_TOL)}
+        assert errs and not bad, (req.syms, bad)
+    # deterministic: a second run gives the same bits
+    _, _, outs2 = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE | B.OPT_SPLITK_LN)
+    for a, b in zip(outs, outs2):
+        assert np.array_equal(a["y"], b["y"])
 
 
 def test_cfg2_small_encoder_arena_reuse_matches_no_reuse():

@@ -84,6 +84,10 @@ def test_expected_smaps_per_config():
     assert "[1,L,2304]" in shapes.values() and "[1,L,3072]" in shapes.values() and shapes["y"] == "[1,L,768]"
     kinds = [g.group_info(i)["kind"] for i in range(g.num_groups())]
     assert kinds == ["gemm", "attention", "gemm", "layernorm", "gemm", "gemm", "layernorm"]
+    # opt-in: the two residual GEMMs of a post-LN layer absorb their LayerNorm (split-K GEMM + finishing kernel)
+    g2 = B.Graph(wl.ir, B.OPT_SPLITK_LN)
+    kinds2 = [g2.group_info(i)["kind"] for i in range(g2.num_groups())]
+    assert kinds2 == ["gemm", "attention", "gemm", "gemm", "gemm"]
     assert g.num_subgraphs() == 1
     # the Reshape's shape tensor is computed in-graph from Shape(x): its value map is known
     rs = [nd for nd in og.nodes if nd.op == "Reshape"][0]
