@@ -19,6 +19,7 @@ STATUS = ["SOD2_OK", "SOD2_E_INVALID_ARG", "SOD2_E_PARSE", "SOD2_E_UNSUPPORTED_O
 OPT_NO_FUSION = 1
 OPT_NO_REUSE = 2
 OPT_SPLITK_LN = 4
+OPT_LEGACY_ATTENTION = 8
 DYN_CLASS = ["ISDO", "ISDOS", "ISVDOS", "EDO"]
 
 

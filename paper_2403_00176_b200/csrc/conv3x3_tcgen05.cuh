@@ -135,19 +135,26 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_
       // ---- two MMA issuers: warp 3 takes this CTA's even tiles (accumulator 0), warp 12 the odd ones
       // (accumulator 1).  A thread that waits on a barrier between MMAs leaves the tensor pipe idle for a
       // few hundred cycles; with two issuers one thread's wait is covered by the other's MMAs.  Both
-      // consume the same ring: the stages of tile j are n = j * kstages + ks.
+      // consume the same ring, stage n = j * kstages + ks of tile j, and BOTH wait on every stage in
+      // order, also on the other issuer's: a parity wait is only meaningful for a thread that has seen
+      // the barrier's previous phase, and walking all stages keeps each issuer exactly in step (the
+      // in-order producer cannot refill a slot twice while an issuer still owns an earlier stage).
       constexpr uint32_t idesc = ptx::idesc_bf16(128, BN);
-      const int acc = warp == 3 ? 0 : 1;
+      const int me = warp == 3 ? 0 : 1;
       if (RES) ptx::mbar_wait(w_full, 0, dead);
-      int j = acc;
-      for (int t = blockIdx.x + acc * gridDim.x; t < num_tiles; t += 2 * gridDim.x, j += 2) {
-        if (j >= 2) ptx::mbar_wait(&tmem_empty[acc], ((j >> 1) - 1) & 1, dead);
-        ptx::tc_fence_after();
+      int n = 0, j = 0;
+      for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++j) {
+        const int acc = j & 1;
+        const bool mine = acc == me;
+        if (mine) {
+          if (j >= 2) ptx::mbar_wait(&tmem_empty[acc], ((j >> 1) - 1) & 1, dead);
+          ptx::tc_fence_after();
+        }
         const uint32_t d = tmem + acc * BN;
-        int n = j * kstages;
         for (int ks = 0; ks < kstages; ++ks, ++n) {
           const int s = n % STAGES;
           ptx::mbar_wait(&full[s], (n / STAGES) & 1, dead);
+          if (!mine) continue;
           ptx::tc_fence_after();
           const uint32_t a = ptx::smem_u32(tiles + s * S::STAGE_BYTES);
           const uint32_t b = RES ? ptx::smem_u32(wres) + ks * 3 * BN * 128 : a + C3_A_SLOT;
@@ -160,7 +167,7 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_
           }
           ptx::mma_commit(&empty[s]);
         }
-        ptx::mma_commit(&tmem_full[acc]);
+        if (mine) ptx::mma_commit(&tmem_full[acc]);
       }
     }
   } else if (warp == 2) {

@@ -12,6 +12,7 @@ namespace sod2 {
 enum OptFlags : uint32_t {
   OPT_NO_FUSION = 1u,   // every operator is its own group (fused-vs-unfused comparison)
   OPT_NO_REUSE = 2u,    // every arena tensor gets its own slot (keeps all intermediates readable after a run)
+  OPT_LEGACY_ATTENTION = 8u,  // attention groups on the mma.sync kernel even where the tcgen05 kernel applies
   OPT_SPLITK_LN = 4u,   // a bf16 GEMM (+bias, +residual) followed by LayerNorm becomes one group: split-K GEMM + finishing kernel
 };
 

@@ -375,7 +375,7 @@ struct Builder {
       // token stride, head stride and head-0 column for every request, rows in increasing order)
       {
         k::AtcParams tp{};
-        bool ok = true;
+        bool ok = !(c.flags & OPT_LEGACY_ATTENTION);
         auto split = [&](long long off, int ts, int* row, int* col) { if (off < 0 || ts <= 0) { ok = false; return; } *row = static_cast<int>(off / ts); *col = static_cast<int>(off % ts); };
         const k::AttnReq& R0 = ap.r[0];
         int order[k::ATTN_MAX_REQ];

@@ -399,6 +399,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   __syncthreads();
   if (warp == 2) ptx::tmem_dealloc(tmem, TMEM_COLS);
   if (threadIdx.x == 0 && *dead && ep.status) atomicExch(ep.status, 1);
+  SOD2_TRACE_DUMP()
 }
 
 }  // namespace k

@@ -53,7 +53,7 @@ def test_fig4_chain_one_fused_version():
             assert O.rel_err(outs[r]["C"], _oracle_out(wl, req, "C")) <= tol
 
 
-EDGE_L = [1, 15, 16, 17, 63, 64, 65, 127, 128, 129, 200]
+EDGE_L = [1, 15, 16, 17, 63, 64, 65, 127, 128, 129, 200, 257, 512]
 
 
 def _encoder_edge(layers=2, F=256):
@@ -93,6 +93,16 @@ def test_cfg2_small_encoder_splitk_layernorm_groups_lockstep():
     _, _, outs2 = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE | B.OPT_SPLITK_LN)
     for a, b in zip(outs, outs2):
         assert np.array_equal(a["y"], b["y"])
+
+
+def test_cfg2_small_encoder_legacy_attention_kernel_lockstep():
+    # the mma.sync attention kernel is the fallback for operand layouts the tensor maps cannot express
+    wl, reqs = _encoder_edge()
+    s, p, outs = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE | B.OPT_LEGACY_ATTENTION)
+    for r, req in enumerate(reqs):
+        errs = lockstep(wl, s, p, outs, r, BF16_TOL)
+        bad = {k: v for k, v in errs.items() if not (isinstance(v, float) and v <= BF16_TOL)}
+        assert errs and not bad, (req.syms, bad)
 
 
 def test_cfg2_small_encoder_arena_reuse_matches_no_reuse():
