@@ -440,7 +440,7 @@ __global__ void __launch_bounds__(256) im2col_nchw_bf16(Im2colParams p) {
   // CTA = 64 consecutive output pixels of one output row.  The input window (C x ks rows x span
   // columns) is staged in shared memory with coalesced reads; every thread then writes 16-byte
   // groups of the K-major patch rows (coalesced: a pixel's row is Kp*2 contiguous bytes).
-  extern __shared__ __nv_bfloat16 win[];          // [C][ks][span]
+  extern __shared__ __nv_bfloat16 win[];          // [C][ks][span], then int koff[Kp]
   const int segs = (p.Wo + 63) / 64;
   const int seg = blockIdx.x % segs;
   const int ho = (blockIdx.x / segs) % p.Ho;
@@ -449,6 +449,13 @@ __global__ void __launch_bounds__(256) im2col_nchw_bf16(Im2colParams p) {
   const int span = 63 * p.stride + p.ks;          // input columns needed by 64 output pixels
   const int w_in0 = wo0 * p.stride - p.pad, h_in0 = ho * p.stride - p.pad;
   const int total = p.C * p.ks * span;
+  // window offset of every k = (ci, dy, dx), computed once per CTA: the gather loop below would otherwise
+  // spend most of its instructions on the divisions
+  int* koff = reinterpret_cast<int*>(win + ((total + 7) & ~7));
+  for (int kk = threadIdx.x; kk < p.Kp; kk += 256) {
+    const int dx = kk % p.ks, dy = (kk / p.ks) % p.ks, ci = kk / (p.ks * p.ks);
+    koff[kk] = kk < p.K ? (ci * p.ks + dy) * span + dx : -1;
+  }
   for (int i = threadIdx.x; i < total; i += 256) {
     const int col = i % span, row = (i / span) % p.ks, ci = i / (span * p.ks);
     const int h = h_in0 + row, w = w_in0 + col;
@@ -465,11 +472,8 @@ __global__ void __launch_bounds__(256) im2col_nchw_bf16(Im2colParams p) {
     __align__(16) __nv_bfloat16 v[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      const int kk = gq * 8 + j;
-      if (kk < p.K) {
-        const int dx = kk % p.ks, dy = (kk / p.ks) % p.ks, ci = kk / (p.ks * p.ks);
-        v[j] = win[(ci * p.ks + dy) * span + px * p.stride + dx];
-      } else v[j] = __float2bfloat16(0.0f);
+      const int o = koff[gq * 8 + j];
+      v[j] = o >= 0 ? win[o + px * p.stride] : __float2bfloat16(0.0f);
     }
     const long long pix = (static_cast<long long>(n) * p.Ho + ho) * p.Wo + wo;
     *reinterpret_cast<uint4*>(p.a + pix * p.Kp + gq * 8) = *reinterpret_cast<const uint4*>(v);

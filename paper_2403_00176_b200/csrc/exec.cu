@@ -700,7 +700,7 @@ struct Builder {
         ip.a = reinterpret_cast<__nv_bfloat16*>(x.arena + x.plan->scratch_off[0]);
         {
           const int segs = (ip.Wo + 63) / 64;
-          const size_t wsm = static_cast<size_t>(ip.C) * ip.ks * (63 * ip.stride + ip.ks) * 2;
+          const size_t wsm = ((static_cast<size_t>(ip.C) * ip.ks * (63 * ip.stride + ip.ks) + 7) & ~size_t(7)) * 2 + static_cast<size_t>(ip.Kp) * 4;
           k::im2col_nchw_bf16<<<static_cast<unsigned>(segs) * ip.Ho * ip.N, 256, wsm, x.stream>>>(ip);
         }
         const void* Wp = x.resolve(pw);
