@@ -238,7 +238,10 @@ def run_ours(args):
             "plan_us_per_batch": plan_us,
             "arena": mem,
             "roofline": {"bound": "tensor", "achieved": gemm["tflops"], "peak": peaks["tf_sustained"], "unit": "TFLOP/s",
-                         "frac": gemm["tflops"] / peaks["tf_sustained"], "traffic": None,
+                         "frac": gemm["tflops"] / peaks["tf_sustained"],
+                         # mean DRAM bytes per GEMM launch of one layer's four GEMMs at T = 1929 (ncu, cold cache):
+                         # profiles/gemm_bf16_tcgen05_cfg2.md
+                         "traffic": 10.1e6, "traffic_unit": "bytes per launch (ncu dram read+write, T=1929)",
                          "peak_source": peaks["src"] + " cuBLAS bf16, sustained (kernel timed inside a long step)",
                          "kernel": "gemm_bf16_tcgen05", "launches": gemm["launch_groups"],
                          "avg_us": gemm["ms"] / gemm["launch_groups"] * 1e3,
