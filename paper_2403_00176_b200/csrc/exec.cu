@@ -572,21 +572,30 @@ struct Builder {
         nmax = std::max(nmax, static_cast<int>(n));
       }
       tp.D = static_cast<int>(D);
-      const size_t sc_bytes = static_cast<size_t>(total_rows) * 8;
-      scratch_need = std::max(scratch_need, sc_bytes);
+      tp.first_row = first_row;
+      int chunks = 0;
+      for (int i = 0; i < nr; ++i) { tp.chunk_start[i] = chunks; chunks += (tp.r[i].n + k::TOPK_CHUNK - 1) / k::TOPK_CHUNK; }
+      tp.chunk_start[nr] = chunks;
+      const size_t sc_bytes = (static_cast<size_t>(total_rows) * 8 + 15) & ~size_t(15);
+      scratch_need = std::max(scratch_need, sc_bytes + static_cast<size_t>(total_rows));
       const long long rows = total_rows;
-      const size_t smem = static_cast<size_t>((nmax + 1) & ~1) * 8 + static_cast<size_t>(nmax) * 4;
-      if (smem > 200 * 1024) return fail(E_UNSUPPORTED_OP, "top-k keep: too many tokens for one CTA");
-      add(gi, 2, [=](const RunCtx& x) mutable {
+      const size_t smem = static_cast<size_t>(nmax) * 8;
+      if (smem > 200 * 1024) return fail(E_UNSUPPORTED_OP, "top-k keep: too many tokens per request for the shared-memory score table");
+      add(gi, 3, [=](const RunCtx& x) mutable {
         double* score = reinterpret_cast<double*>(x.arena + x.plan->scratch_off[0]);
         tp.y = reinterpret_cast<const __nv_bfloat16*>(x.resolve(by));
         tp.out = reinterpret_cast<__nv_bfloat16*>(x.resolve(bo));
         tp.idx = reinterpret_cast<long long*>(x.resolve(bi));
         tp.score = score;
-        k::ScoreParams sp{tp.y, score, rows, tp.D};
+        tp.keep = reinterpret_cast<unsigned char*>(x.arena + x.plan->scratch_off[0] + sc_bytes);
+        // scores are indexed from the first request's first row
+        k::ScoreParams sp{tp.y + first_row * tp.D, score, rows, tp.D};
         if (rows) launch_pdl(k::row_sumsq_f64, dim3(static_cast<unsigned>((rows + 7) / 8)), dim3(256), 0, x.stream, sp);
-        if (smem > 48 * 1024) cudaFuncSetAttribute(k::topk_keep, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        launch_pdl(k::topk_keep, dim3(tp.n_req), dim3(1024), smem, x.stream, tp);
+        if (chunks) {
+          if (smem > 48 * 1024) cudaFuncSetAttribute(k::topk_flags, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+          launch_pdl(k::topk_flags, dim3(chunks), dim3(256), smem, x.stream, tp);
+          launch_pdl(k::topk_gather, dim3(chunks), dim3(256), 0, x.stream, tp);
+        }
         return cudaGetLastError();
       });
     }

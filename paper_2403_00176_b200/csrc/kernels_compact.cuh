@@ -54,8 +54,13 @@ __global__ void __launch_bounds__(256) row_sumsq_f64(ScoreParams p) {
 // Keep the k highest-scoring tokens of each request in ascending index order.
 //   rank_i = #{j : s_j > s_i} + #{j < i : s_j == s_i};  keep_i = rank_i < k
 //   pos_i  = exclusive scan of keep;  idx[pos_i] = i;  out[pos_i, :] = y[i, :]
-// One CTA per request: ranks by counting against the scores staged in shared memory, block-wide
-// scan of the flags, then warp-per-row gather with 128-bit copies.
+// Two kernels over the same grid, one CTA per chunk of 64 tokens of a request (so a batch of 16
+// requests spreads over about a hundred SMs instead of 16):
+//   topk_flags   the request's fp64 scores staged in shared memory; four threads share a token's
+//                ranking (a quarter of the comparisons each); writes keep_i as a byte
+//   topk_gather  counts the kept tokens before the chunk, scans the chunk's 64 flags with two ballots,
+//                writes the indices and copies the kept rows, one warp per row, 128-bit accesses
+constexpr int TOPK_CHUNK = 64;
 struct TopkReq {
   long long row0;      // first packed input row of the request
   long long out_row0;  // first packed output row
@@ -64,57 +69,96 @@ struct TopkReq {
 };
 struct TopkParams {
   const __nv_bfloat16* y;
-  const double* score;
+  const double* score;       // packed [rows] relative to the first request's row0
+  unsigned char* keep;       // packed [rows], same indexing as score
   __nv_bfloat16* out;
-  long long* idx;      // packed [sum k] int64, per request k entries
+  long long* idx;            // packed [sum k] int64, per request k entries
   int D;
   int n_req;
+  long long first_row;       // row0 of the first request (score / keep are indexed from it)
+  int chunk_start[COMPACT_MAX_REQ + 1];   // prefix sum of ceil(n / 64)
   TopkReq r[COMPACT_MAX_REQ];
 };
 
-__global__ void __launch_bounds__(1024) topk_keep(const __grid_constant__ TopkParams p) {
+__device__ __forceinline__ int topk_locate(const TopkParams& p, int cta, int* chunk) {
+  int ri = 0;
+  while (ri + 1 < p.n_req && cta >= p.chunk_start[ri + 1]) ++ri;
+  *chunk = cta - p.chunk_start[ri];
+  return ri;
+}
+
+__global__ void __launch_bounds__(256) topk_flags(const __grid_constant__ TopkParams p) {
   extern __shared__ double s_score[];                  // [n]
-  int* s_pos = reinterpret_cast<int*>(s_score + ((p.r[blockIdx.x].n + 1) & ~1));  // [n] kept position or -1
-  __shared__ int warp_tot[32];
-  const TopkReq R = p.r[blockIdx.x];
+  int chunk;
+  const TopkReq R = p.r[topk_locate(p, blockIdx.x, &chunk)];
+  ptx::pdl_wait();
+  ptx::pdl_launch();
+  const int tid = threadIdx.x;
+  const double* sc = p.score + (R.row0 - p.first_row);
+  for (int i = tid; i < R.n; i += 256) s_score[i] = sc[i];
+  __syncthreads();
+  const int i = chunk * TOPK_CHUNK + (tid >> 2), part = tid & 3;
+  int rank = 0;
+  if (i < R.n) {
+    const double si = s_score[i];
+    const int per = (R.n + 3) >> 2, j0 = part * per, j1 = min(R.n, j0 + per);
+    for (int j = j0; j < j1; ++j) {
+      const double sj = s_score[j];
+      rank += (sj > si) || (sj == si && j < i);
+    }
+  }
+  rank += __shfl_xor_sync(0xffffffffu, rank, 1);
+  rank += __shfl_xor_sync(0xffffffffu, rank, 2);
+  if (i < R.n && part == 0) p.keep[R.row0 - p.first_row + i] = rank < R.k;
+}
+
+__global__ void __launch_bounds__(256) topk_gather(const __grid_constant__ TopkParams p) {
+  __shared__ int warp_cnt[8];
+  __shared__ int s_pos[TOPK_CHUNK];
+  int chunk;
+  const TopkReq R = p.r[topk_locate(p, blockIdx.x, &chunk)];
   ptx::pdl_wait();
   ptx::pdl_launch();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  for (int i = tid; i < R.n; i += blockDim.x) s_score[i] = p.score[R.row0 + i];
+  const unsigned char* kp = p.keep + (R.row0 - p.first_row);
+  const int base = chunk * TOPK_CHUNK;
+  // kept tokens before this chunk
+  int c = 0;
+  for (int j = tid; j < base; j += 256) c += kp[j];
+#pragma unroll
+  for (int o = 16; o; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+  if (lane == 0) warp_cnt[warp] = c;
   __syncthreads();
-  int carry = 0;  // kept count of earlier chunks (same in every thread)
-  for (int base = 0; base < R.n; base += blockDim.x) {
+  int carry = 0;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) carry += warp_cnt[w];
+  // the chunk's own 64 flags: warps 0 and 1 take 32 each
+  if (warp < 2) {
     const int i = base + tid;
-    int keep = 0;
-    if (i < R.n) {
-      const double si = s_score[i];
-      int rank = 0;
-      for (int j = 0; j < R.n; ++j) {
-        const double sj = s_score[j];
-        rank += (sj > si) || (sj == si && j < i);
-      }
-      keep = rank < R.k;
-    }
-    // block exclusive scan of keep
+    const int keep = i < R.n ? kp[i] : 0;
     const unsigned bal = __ballot_sync(0xffffffffu, keep);
-    const int wpre = __popc(bal & ((1u << lane) - 1));
-    if (lane == 0) warp_tot[warp] = __popc(bal);
-    __syncthreads();
-    int woff = 0, tot = 0;
-    for (int w = 0; w < 32; ++w) { const int c = warp_tot[w]; if (w < warp) woff += c; tot += c; }
-    if (i < R.n) s_pos[i] = keep ? carry + woff + wpre : -1;
-    carry += tot;
-    __syncthreads();
+    const int pre = __popc(bal & ((1u << lane) - 1));
+    if (lane == 0) warp_cnt[warp] = __popc(bal);
+    __syncwarp();
+    s_pos[tid] = keep ? pre : -1;
   }
-  // gather: one warp per source row
-  const int vec = (p.D * 2) >> 4;  // 16-byte chunks per row (D % 8 == 0 checked on the host)
-  for (int i = warp; i < R.n; i += 32) {
-    const int pos = s_pos[i];
-    if (pos < 0) continue;
-    if (lane == 0) p.idx[R.idx0 + pos] = i;
-    const uint4* src = reinterpret_cast<const uint4*>(p.y + (R.row0 + i) * p.D);
-    uint4* dst = reinterpret_cast<uint4*>(p.out + (R.out_row0 + pos) * p.D);
-    for (int c = lane; c < vec; c += 32) dst[c] = src[c];
+  __syncthreads();
+  if (tid < TOPK_CHUNK && s_pos[tid] >= 0) {
+    s_pos[tid] += carry + (tid >= 32 ? warp_cnt[0] : 0);
+    p.idx[R.idx0 + s_pos[tid]] = base + tid;
+  }
+  __syncthreads();
+  // copy the kept rows: (row, 16-byte piece) items spread over the whole CTA, several independent
+  // loads in flight per thread
+  const int vec = (p.D * 2) >> 4;  // 16-byte pieces per row (D % 8 == 0 checked on the host)
+  const uint4* src = reinterpret_cast<const uint4*>(p.y + (R.row0 + base) * p.D);
+  uint4* dst = reinterpret_cast<uint4*>(p.out + R.out_row0 * p.D);
+  const int items = TOPK_CHUNK * vec;
+#pragma unroll 4
+  for (int it = tid; it < items; it += 256) {
+    const int t = it / vec, c4 = it - t * vec;
+    const int pos = s_pos[t];
+    if (pos >= 0) dst[static_cast<long long>(pos) * vec + c4] = src[it];
   }
 }
 
