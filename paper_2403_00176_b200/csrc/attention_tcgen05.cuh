@@ -5,10 +5,10 @@
 //   S_j = Q K_j^T          tcgen05.mma, M=128, N=64, K=64; Q and K_j are K-major TMA tiles
 //   P_j = exp2(S_j*c - m)  softmax threads: two threads per query row read the halves of its row of
 //                          S_j from TMEM, write P_j as bf16 into a swizzled tile
-//   O_j = P_j V_j          tcgen05.mma, M=128, N=64, K=64; V_j is the natural [key, d] tile, used
+//   O  += P_j V_j          tcgen05.mma, M=128, N=64, K=64; V_j is the natural [key, d] tile, used
 //                          as an MN-major B operand
-//   o   = o*corr + O_j     running output in registers (the rescale of the online softmax)
-// S and O_j are double buffered in TMEM (4 x 64 columns), P_j, K_j, V_j in shared memory, so the
+//   (O *= corr)            only when a block's maximum moves the exponent reference by more than 2^8
+// S is double buffered in TMEM, O accumulates there (3 x 64 columns), P_j, K_j, V_j in shared memory, so the
 // tensor pipe, the softmax warps and TMA overlap inside a CTA; two CTAs share an SM.
 // Q, K, V are 2-D tensor maps over the packed [tokens, row stride] buffers; a tile that runs past a
 // request's rows reads the next request's rows (finite data) or zeros past the end of the buffer, and
@@ -147,9 +147,9 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     }
   } else if (warp == 10) {
     if (lane == 0) {
-      // ---- O issuer: O_j = P_j V_j.  "O_j done" publishes O_j, frees the V stage and the P buffer.
-      // The softmax warps hand over P_j only after they have read O_{j-2} (program order in their
-      // loop), so the O buffer needs no barrier of its own.
+      // ---- O issuer: O += P_j V_j, accumulated in TMEM over the request's key blocks.  "O_j done" frees
+      // the V stage and the P buffer.  The softmax warps rescale O (rarely) before they hand over P_j,
+      // so the accumulator needs no barrier of its own.
       constexpr uint32_t idesc_pv = ptx::idesc_bf16(128, 64) | (1u << 16);   // B (= V tile) is MN-major
       for (int i = 0; i < nkv; ++i) {
         const int b = i & 1;
@@ -159,7 +159,7 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const uint32_t aP = ptx::smem_u32(sP + b * ATC_P_BYTES), aV = ptx::smem_u32(sV + b * ATC_KV_BYTES);
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk)   // 16 keys per step: 32 B along P's rows, 16 rows (2048 B) down V
-          ptx::mma_bf16(tmem + 128 + b * 64, ptx::smem_desc_sw128(aP) + 2 * kk, ptx::smem_desc_sw128(aV + kk * 2048), idesc_pv, kk != 0);
+          ptx::mma_bf16(tmem + 128, ptx::smem_desc_sw128(aP) + 2 * kk, ptx::smem_desc_sw128(aV + kk * 2048), idesc_pv, (i | kk) != 0);
         ptx::mma_commit(&o_full[b]);
         SOD2_TRACE(1, 20 + i)
       }
@@ -176,25 +176,13 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
     const bool tracer = threadIdx.x == 64;
     ptx::pdl_wait();
-    float o[32];
-#pragma unroll
-    for (int i = 0; i < 32; ++i) o[i] = 0.f;
-    float m = -INFINITY, l = 0.f, c_prev = 0.f;
+    // Online softmax with a lazily updated reference: the exponent reference m only moves when a block's
+    // row maximum exceeds it by more than 2^8 after scaling, so p stays <= 256 (exact enough in bf16 and
+    // fp32) and the accumulator O in TMEM is rescaled only then -- for almost every block nothing is read
+    // back from TMEM.  l and O always refer to the same m, so O / l at the end is the softmax average.
+    float m = -INFINITY, l = 0.f;
     const float c = p.scale_log2e;
-    auto accumulate = [&](int i, float cf) {
-      // o = o * cf + O_i, this thread's 32 columns of O_i read from TMEM
-      const int b = i & 1;
-      ptx::mbar_wait_warp(&o_full[b], (i >> 1) & 1, dead);
-      ptx::tc_fence_after();
-      uint32_t r[32];
-      ptx::tmem_ld32(tmem + lane_base + 128 + b * 64 + hh * 32, r);
-      ptx::tmem_ld_wait();
-      ptx::tc_fence_before();
-      if (warp_live) {
-#pragma unroll
-        for (int e = 0; e < 32; ++e) o[e] = fmaf(o[e], cf, __uint_as_float(r[e]));
-      }
-    };
+    const uint32_t o_addr = tmem + lane_base + 128 + hh * 32;
     for (int j = 0; j < nkv; ++j) {
       const int b = j & 1;
       ptx::mbar_wait_warp(&s_full[b], (j >> 1) & 1, dead);
@@ -221,12 +209,27 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
       xmax[(b * 2 + hh) * 128 + row] = mx;
       asm volatile("bar.sync 1, 256;" ::: "memory");
-      const float m_new = fmaxf(m, fmaxf(mx, xmax[(b * 2 + (hh ^ 1)) * 128 + row]));
+      const float mrow = fmaxf(mx, xmax[(b * 2 + (hh ^ 1)) * 128 + row]);
+      // move the reference?  (both threads of a row, and both warps of a row group, decide alike)
+      const bool move = warp_live && (mrow - m) * c > 8.0f;
+      float corr = 1.f;
+      if (move) { corr = ex2_approx((m - mrow) * c); m = mrow; l *= corr; }
+      if (j > 0 && __any_sync(0xffffffffu, move)) {
+        // all products issued so far must have landed in O before it is scaled
+        ptx::mbar_wait_warp(&o_full[(j - 1) & 1], ((j - 1) >> 1) & 1, dead);
+        ptx::tc_fence_after();
+        uint32_t r[32];
+        ptx::tmem_ld32(o_addr, r);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * corr);
+        ptx::tmem_st32(o_addr, r);
+        ptx::tmem_st_wait();
+        ptx::tc_fence_before();
+      }
       // p = 2^(s*c - m*c): the scale rides in the FMA that feeds ex2.  The special-function pipe (16
-      // results per clock per SM, shared with the float <-> half conversions) bounds this loop.
-      const float corr = ex2_approx((m - m_new) * c);
-      m = m_new;
-      const float mc = -m_new * c;
+      // results per clock per SM) bounds this loop.
+      const float mc = -m * c;
       float sum0 = 0.f, sum1 = 0.f;
       uint32_t pk[16];
 #pragma unroll
@@ -236,7 +239,7 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
         pk[e >> 1] = warp_live ? *reinterpret_cast<const uint32_t*>(&pb) : 0u;
       }
-      l = fmaf(l, corr, sum0 + sum1);
+      l += sum0 + sum1;
       if (tracer) { SOD2_TRACE(2, 40 + j) }
       // P_j into the swizzled tile once the MMA that read this buffer two blocks ago has finished
       if (j >= 2) ptx::mbar_wait_warp(&o_full[b], ((j >> 1) - 1) & 1, dead);    // O_{j-2} done: P buffer free
@@ -250,16 +253,17 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&p_full[b]);
       if (tracer) { SOD2_TRACE(2, 50 + j) }
-      if (j >= 1) accumulate(j - 1, c_prev);
-      if (tracer) { SOD2_TRACE(2, 60 + j) }
-      c_prev = corr;
     }
-    accumulate(nkv - 1, c_prev);
-    if (tracer) { SOD2_TRACE(2, 70) }
-    // ---- output: the row sums of the two halves are added through shared memory, the scaled rows are
-    // staged (swizzled) in P buffer 0 and written four full 128-byte rows per instruction.  Every MMA
-    // that read the P buffers has completed.
+    // ---- output: O / l.  The row sums of the two halves are added through shared memory, the scaled rows
+    // are staged (swizzled) in P buffer 0 and written four full 128-byte rows per instruction.
     {
+      ptx::mbar_wait_warp(&o_full[(nkv - 1) & 1], ((nkv - 1) >> 1) & 1, dead);   // every product has landed; the P buffers are free
+      ptx::tc_fence_after();
+      uint32_t r[32];
+      ptx::tmem_ld32(o_addr, r);
+      ptx::tmem_ld_wait();
+      ptx::tc_fence_before();
+      if (tracer) { SOD2_TRACE(2, 70) }
       xmax[hh * 128 + row] = l;
       asm volatile("bar.sync 1, 256;" ::: "memory");
       const float lt = l + xmax[(hh ^ 1) * 128 + row];
@@ -270,7 +274,7 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         uint4 v;
         __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&v);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) h2[i] = __floats2bfloat162_rn(o[g * 8 + 2 * i] * inv, o[g * 8 + 2 * i + 1] * inv);
+        for (int i = 0; i < 4; ++i) h2[i] = __floats2bfloat162_rn(__uint_as_float(r[g * 8 + 2 * i]) * inv, __uint_as_float(r[g * 8 + 2 * i + 1]) * inv);
         *reinterpret_cast<uint4*>(prow + (((hh * 4 + g) ^ (row & 7)) << 4)) = v;
       }
       asm volatile("bar.sync 1, 256;" ::: "memory");
