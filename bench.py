@@ -176,11 +176,12 @@ def run_ours(args):
             pinned_out[key] = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in preps[key].out_dev]
         torch.cuda.synchronize(dev)
         t0 = time.perf_counter()
-        b = sess.graph.bind_dims(wl.sym_names, [[r.syms[s] for s in wl.sym_names] for r in reqs])
-        pl = b.plan()
+        # the input copy is enqueued first, so that binding and planning on the host overlap the transfer
         pr = preps[key]
         for dst, src in zip(pr.in_dev, pinned_in[key]):
             dst.copy_(src, non_blocking=True)
+        b = sess.graph.bind_dims(wl.sym_names, [[r.syms[s] for s in wl.sym_names] for r in reqs])
+        pl = b.plan()
         pl.run([t.data_ptr() for t in pr.in_dev], [t.data_ptr() for t in pr.out_dev], pr.arena.data_ptr(), pr.arena.numel(),
                sess.stream)
         host_out = pinned_out[key]
@@ -234,7 +235,7 @@ def run_ours(args):
             "gpu_launches": int(launches),
             "clocks": clocks,
             "e2e": {"value": e2e_ms, "unit": "ms/inference", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-                    "includes": "bind_dims + plan + H2D (pinned) + run + D2H (pinned)"},
+                    "includes": "H2D (pinned, enqueued first) + bind_dims + plan + run + D2H (pinned)"},
             "plan_us_per_batch": plan_us,
             "arena": mem,
             "roofline": {"bound": "tensor", "achieved": gemm["tflops"], "peak": peaks["tf_sustained"], "unit": "TFLOP/s",
