@@ -899,7 +899,7 @@ struct Builder {
       add(gi, 2, [=](const RunCtx& x) mutable {
         gp.x = reinterpret_cast<const __nv_bfloat16*>(x.resolve(px));
         gp.partial = reinterpret_cast<double*>(x.arena + x.plan->scratch_off[0]);
-        launch_pdl(k::gap_partial_f64, dim3((gp.C + 63) / 64, gp.slabs, N), dim3(256), 0, x.stream, gp);
+        launch_pdl(k::gap_partial_f64, dim3(1, gp.slabs, N), dim3(256), 0, x.stream, gp);
         k::GateParams q{};
         q.partial = gp.partial;
         q.w = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pw));
@@ -1018,7 +1018,7 @@ struct Builder {
         gp.partial = reinterpret_cast<double*>(x.arena + x.plan->scratch_off[0]);
         gp.out = x.resolve(po);
         gp.out_f64 = nullptr;
-        launch_pdl(k::gap_partial_f64, dim3((gp.C + 63) / 64, gp.slabs, N), dim3(256), 0, x.stream, gp);
+        launch_pdl(k::gap_partial_f64, dim3(1, gp.slabs, N), dim3(256), 0, x.stream, gp);
         launch_pdl(k::gap_final_f64, dim3((N * gp.C + 31) / 32), dim3(256), 0, x.stream, gp, N);
         return cudaGetLastError();
       });
