@@ -470,12 +470,16 @@ __global__ void __launch_bounds__(256) im2col_nchw_bf16(Im2colParams p) {
     const int dx = kk % p.ks, dy = (kk / p.ks) % p.ks, ci = kk / (p.ks * p.ks);
     koff[kk] = kk < p.K ? (ci * p.ks + dy) * span + dx : -1;
   }
-  for (int i = threadIdx.x; i < total; i += 256) {
-    const int col = i % span, row = (i / span) % p.ks, ci = i / (span * p.ks);
-    const int h = h_in0 + row, w = w_in0 + col;
-    float v = 0.0f;
-    if (h >= 0 && h < p.H && w >= 0 && w < p.W) v = __bfloat162float(p.x[((static_cast<long long>(n) * p.C + ci) * p.H + h) * p.W + w]);
-    win[i] = __float2bfloat16(v);
+  // window rows (one per (channel, kernel row)) by warps, columns by lanes: coalesced, no divisions per element
+  for (int r = threadIdx.x >> 5; r < p.C * p.ks; r += 8) {
+    const int ci = r / p.ks, row = r - ci * p.ks;
+    const int h = h_in0 + row;
+    const bool hok = h >= 0 && h < p.H;
+    const __nv_bfloat16* src = p.x + ((static_cast<long long>(n) * p.C + ci) * p.H + (hok ? h : 0)) * p.W;
+    for (int col = threadIdx.x & 31; col < span; col += 32) {
+      const int w = w_in0 + col;
+      win[r * span + col] = (hok && w >= 0 && w < p.W) ? src[w] : __float2bfloat16(0.0f);
+    }
   }
   __syncthreads();
   const int groups = p.Kp >> 3;
