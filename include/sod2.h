@@ -42,6 +42,7 @@ typedef enum {
 /* option bits for sod2_graph_create */
 #define SOD2_OPT_NO_FUSION 1u /* every operator is its own group */
 #define SOD2_OPT_NO_REUSE  2u /* every arena tensor keeps its own slot: intermediates stay readable */
+#define SOD2_OPT_COPY_REGROUP 16u /* Switch / Combine always copy whole samples (no index-indirect convolutions) */
 #define SOD2_OPT_LEGACY_ATTENTION 8u /* attention groups run the mma.sync kernel even where the tcgen05 kernel applies */
 #define SOD2_OPT_SPLITK_LN 4u /* bf16 GEMM (+bias, +residual) -> LayerNorm as one group: split-K GEMM into fp32 slabs + finishing kernel */
 

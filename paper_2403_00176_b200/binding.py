@@ -20,6 +20,7 @@ OPT_NO_FUSION = 1
 OPT_NO_REUSE = 2
 OPT_SPLITK_LN = 4
 OPT_LEGACY_ATTENTION = 8
+OPT_COPY_REGROUP = 16
 DYN_CLASS = ["ISDO", "ISDOS", "ISVDOS", "EDO"]
 
 

@@ -107,6 +107,7 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_
       for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
         int n0, img, h0, w0;
         decode(t, &n0, &img, &h0, &w0);
+        if (p.in_ids) img = p.in_ids[img];
         for (int ks = 0; ks < kstages; ++ks, ++n) {
           const int s = n % STAGES;
           if (n >= STAGES) ptx::mbar_wait(&empty[s], ((n / STAGES) - 1) & 1, dead);
@@ -188,7 +189,7 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_
         const int bsel = u % NSB;
         if (p.has_residual && np < p.Cout) {
           ptx::mbar_expect_tx(&res_full[bsel], CONV_STAGE_OUT);
-          ptx::tma_load_4d(out_stage + bsel * CONV_STAGE_OUT, &tmRes, np, w0, h0, img, &res_full[bsel]);
+          ptx::tma_load_4d(out_stage + bsel * CONV_STAGE_OUT, &tmRes, np, w0, h0, p.res_ids ? p.res_ids[img] : img, &res_full[bsel]);
         } else {
           ptx::mbar_arrive(&res_full[bsel]);
         }
@@ -202,7 +203,7 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_
         decode(t, &n0, &img, &h0, &w0);
         const int np = n0 + (u % PASSES) * 64;
         if (np < p.Cout) {
-          tma_store_4d(&tmOut, out_stage + bsel * CONV_STAGE_OUT, np, w0, h0, img);
+          tma_store_4d(&tmOut, out_stage + bsel * CONV_STAGE_OUT, np, w0, h0, p.out_ids ? p.out_ids[img] : img);
           bulk_commit();
         }
         if (u + NSB < U) {

@@ -34,6 +34,11 @@ struct ConvParams {
   // device after the producing kernel has finished; n_img above is then only the static upper bound
   const long long* n_img_ptr;
   int cnt_a, cnt_b;
+  // index-indirect operands (gated sub-batch without copies): image n of the operand is image ids[n] of
+  // the tensor the map describes; nullptr = direct
+  const int* in_ids;
+  const int* res_ids;
+  const int* out_ids;
   const __nv_bfloat16* bias; // [Cout] or nullptr
   int has_residual;
   int act2;                  // ACT_NONE or ACT_RELU after the residual add
@@ -127,6 +132,7 @@ conv_igemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_co
       for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
         int n0, img, ho0, wo0;
         decode(t, &n0, &img, &ho0, &wo0);
+        if (p.in_ids) img = p.in_ids[img];
         for (int ks = 0; ks < kstages; ++ks, ++n) {
           const int s = n % STAGES;
           if (n >= STAGES) ptx::mbar_wait(&empty[s], ((n / STAGES) - 1) & 1, dead);
@@ -206,6 +212,7 @@ conv_igemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_co
       const int acc = j & 1;
       int n0, img, ho0, wo0;
       decode(t, &n0, &img, &ho0, &wo0);
+      const int img_r = p.res_ids ? p.res_ids[img] : img, img_o = p.out_ids ? p.out_ids[img] : img;
       float* bias_t = bias_s + (j & 1) * 256;
       bias_t[et] = bias_next;
       bias_next = load_bias(t + gridDim.x);
@@ -221,7 +228,7 @@ conv_igemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_co
           if (et == 0) {
             bulk_wait_read0();
             ptx::mbar_expect_tx(res_full, CONV_STAGE_OUT);
-            ptx::tma_load_4d(out_stage, &tmRes, np, wo0, ho0, img, res_full);
+            ptx::tma_load_4d(out_stage, &tmRes, np, wo0, ho0, img_r, res_full);
           }
           ptx::mbar_wait_warp(res_full, rp & 1, dead);
           ++rp;
@@ -265,7 +272,7 @@ conv_igemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_co
         if (ps == PASSES - 1 && lane == 0) ptx::mbar_arrive(&tmem_empty[acc]);
         conv_epi_bar();
         if (et == 0 && live) {
-          tma_store_4d(&tmOut, out_stage, np, wo0, ho0, img);
+          tma_store_4d(&tmOut, out_stage, np, wo0, ho0, img_o);
           bulk_commit();
         }
       }
@@ -572,7 +579,7 @@ struct SampleCopyParams {
   const int* idx;
   const long long* count;
   long long vec_per_sample;   // 16-byte units per sample
-  int scatter;
+  int scatter;                // 0: dst[j] = src[idx[j]];  1: dst[idx[j]] = src[j];  2: dst[idx[j]] = src[idx[j]]
 };
 __global__ void __launch_bounds__(256) sample_copy(SampleCopyParams p) {
   ptx::pdl_wait();
@@ -580,8 +587,8 @@ __global__ void __launch_bounds__(256) sample_copy(SampleCopyParams p) {
   const int j = blockIdx.y;
   if (j >= *p.count) return;
   const long long s = p.idx[j];
-  const uint4* src = p.src + (p.scatter ? static_cast<long long>(j) : s) * p.vec_per_sample;
-  uint4* dst = p.dst + (p.scatter ? s : static_cast<long long>(j)) * p.vec_per_sample;
+  const uint4* src = p.src + (p.scatter == 1 ? static_cast<long long>(j) : s) * p.vec_per_sample;
+  uint4* dst = p.dst + (p.scatter != 0 ? s : static_cast<long long>(j)) * p.vec_per_sample;
   for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < p.vec_per_sample; i += static_cast<long long>(gridDim.x) * blockDim.x) dst[i] = src[i];
 }
 

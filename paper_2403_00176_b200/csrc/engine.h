@@ -12,6 +12,7 @@ namespace sod2 {
 enum OptFlags : uint32_t {
   OPT_NO_FUSION = 1u,   // every operator is its own group (fused-vs-unfused comparison)
   OPT_NO_REUSE = 2u,    // every arena tensor gets its own slot (keeps all intermediates readable after a run)
+  OPT_COPY_REGROUP = 16u,     // Switch / Combine always move whole samples (no index-indirect convolutions)
   OPT_LEGACY_ATTENTION = 8u,  // attention groups on the mma.sync kernel even where the tcgen05 kernel applies
   OPT_SPLITK_LN = 4u,   // a bf16 GEMM (+bias, +residual) followed by LayerNorm becomes one group: split-K GEMM + finishing kernel
 };
@@ -55,9 +56,14 @@ struct Group {
 
 // How a tensor's storage relates to others (decided once, at graph creation).
 struct Storage {
-  enum Kind { ROOT, VIEW_OF_INPUT, VIEW_OF_OUTPUT, FOLDED } kind = ROOT;
-  int node = -1;    // the view operator
-  int other = -1;   // VIEW_OF_INPUT: the operator's input; VIEW_OF_OUTPUT: the operator's output
+  // INDIRECT_IN: an output of a Switch that is never copied: the samples of the Switch input selected
+  // by the executed / skipped id list.  INDIRECT_OUT: the executed operand of a Combine, written by its
+  // producer straight into the Combine output at the executed ids.
+  enum Kind { ROOT, VIEW_OF_INPUT, VIEW_OF_OUTPUT, FOLDED, INDIRECT_IN, INDIRECT_OUT } kind = ROOT;
+  int node = -1;    // the view operator (Switch / Combine for the indirect kinds)
+  int other = -1;   // VIEW_OF_INPUT / INDIRECT_IN: the operator's input; VIEW_OF_OUTPUT / INDIRECT_OUT: the operator's output
+  int gate = -1;    // indirect kinds: the gate tensor whose partition gives the id lists
+  int list = 0;     // indirect kinds: 0 = executed ids, 1 = skipped ids
 };
 
 struct Compiled {
@@ -125,6 +131,8 @@ struct View {                 // one tensor of one request, resolved to storage
   int root = -1;              // tensor id owning the bytes
   int64_t offset = 0;         // elements from the start of the root's instance for this request
   DimVec dims, strides;       // elements
+  int ind_gate = -1;          // >= 0: sample n of this tensor is sample ids[n] of the root (ids = list `ind_list` of that gate's partition)
+  int ind_list = 0;
   bool contiguous() const {
     int64_t s = 1;
     for (int i = static_cast<int>(dims.size()) - 1; i >= 0; --i) { if (dims[i] != 1 && strides[i] != s) return false; s *= dims[i]; }

@@ -770,6 +770,20 @@ struct Builder {
       cp.cnt_a = rc.a; cp.cnt_b = rc.b;
       const bool rt = rc.rt;
       const size_t rt_slot = rc.slot_off;
+      // index-indirect operands: offsets of their id lists in the Switch groups' index area
+      long long ids_in = -1, ids_res = -1, ids_out = -1;
+      {
+        auto ids_of = [&](const View& v, long long* off) -> bool {
+          if (v.ind_gate < 0) return true;
+          auto it = switch_aux.find(v.ind_gate);
+          if (it == switch_aux.end()) return false;
+          const int Nall = static_cast<int>(p.views[v.root][r].dims[0]);
+          *off = static_cast<long long>(it->second) + (v.ind_list ? static_cast<long long>(Nall) * 4 : 0);
+          return true;
+        };
+        if (!ids_of(vx, &ids_in) || !ids_of(vo, &ids_out) || (G.res >= 0 && !ids_of(p.views[G.res][r], &ids_res)))
+          return fail(E_INTERNAL, "index-indirect convolution operand without a Switch");
+      }
       // pixel patch of a tile: the 128-pixel shape that wastes the fewest padded pixels
       long long best = -1;
       for (int tw : {128, 64, 32, 16, 8}) {
@@ -790,6 +804,10 @@ struct Builder {
       const int act = G.act, stride = G.stride;
       const int K = ks * ks * Cin;
       const long long tiles = static_cast<long long>((cp.Wo + cp.TW - 1) / cp.TW) * ((cp.Ho + cp.TH - 1) / cp.TH) * cp.n_img * ((Cout + bn - 1) / bn);
+      // images covered by each operand's tensor map: all images of the root for an index-indirect operand
+      const int n_in_map = static_cast<int>(vx.ind_gate >= 0 ? p.views[vx.root][r].dims[0] : vx.dims[0]);
+      const int n_out_map = static_cast<int>(vo.ind_gate >= 0 ? p.views[vo.root][r].dims[0] : vo.dims[0]);
+      const int n_res_map = G.res >= 0 ? static_cast<int>(p.views[G.res][r].ind_gate >= 0 ? p.views[p.views[G.res][r].root][r].dims[0] : p.views[G.res][r].dims[0]) : 0;
       struct Cache { const void* a = nullptr; const void* w = nullptr; const void* o = nullptr; const void* r = nullptr; CUtensorMap tx, tw, to, tr; };
       auto cache = std::make_shared<Cache>();
       add(gi, 1, [=](const RunCtx& x) mutable {
@@ -798,16 +816,20 @@ struct Builder {
         void* O = x.resolve(po);
         const void* R = hr ? x.resolve(pr) : O;
         if (cache->a != X || cache->w != Wp || cache->o != O || cache->r != R) {
-          if (!encode_bf16_nhwc(&cache->tx, X, cp.n_img, H, Wd, Cin, rows ? 130 : cp.TW, cp.TH, stride) ||
+          if (!encode_bf16_nhwc(&cache->tx, X, n_in_map, H, Wd, Cin, rows ? 130 : cp.TW, cp.TH, stride) ||
               !encode_bf16_kchunks(&cache->tw, Wp, Cout, K, K, bn, rows ? 3 : kch) ||
-              !encode_bf16_nhwc(&cache->to, O, cp.n_img, cp.Ho, cp.Wo, Cout, cp.TW, cp.TH, 1) ||
-              !encode_bf16_nhwc(&cache->tr, R, cp.n_img, cp.Ho, cp.Wo, Cout, cp.TW, cp.TH, 1))
+              !encode_bf16_nhwc(&cache->to, O, n_out_map, cp.Ho, cp.Wo, Cout, cp.TW, cp.TH, 1) ||
+              !encode_bf16_nhwc(&cache->tr, R, hr ? n_res_map : n_out_map, cp.Ho, cp.Wo, Cout, cp.TW, cp.TH, 1))
             return cudaErrorInvalidValue;
           cache->a = X; cache->w = Wp; cache->o = O; cache->r = R;
         }
         cp.bias = hb ? reinterpret_cast<const __nv_bfloat16*>(x.resolve(pb)) : nullptr;
         cp.status = reinterpret_cast<int*>(x.arena);
         cp.n_img_ptr = rt ? reinterpret_cast<const long long*>(x.arena + rt_slot) : nullptr;
+        const char* auxb = x.arena + x.plan->scratch_off[1];
+        cp.in_ids = ids_in >= 0 ? reinterpret_cast<const int*>(auxb + ids_in) : nullptr;
+        cp.res_ids = ids_res >= 0 ? reinterpret_cast<const int*>(auxb + ids_res) : nullptr;
+        cp.out_ids = ids_out >= 0 ? reinterpret_cast<const int*>(auxb + ids_out) : nullptr;
         const dim3 gd(static_cast<unsigned>(std::min<long long>(tiles, x.plan->sm_count))), bd(k::CONV_THREADS);
         const int variant = (rows ? (wres ? 8 : 4) : 0) + (bn == 128 ? 2 : 0) + (act == 2 ? 1 : 0);
 #define SOD2_CONV3_CASE(V, BN_, RES_, ST_, ACT_)                                                                         \
@@ -928,6 +950,7 @@ struct Builder {
     const size_t aux = aux_need;
     switch_aux[G.gate] = aux;
     aux_need += (static_cast<size_t>(2 * N) * 4 + 16 + 255) & ~size_t(255);
+    const bool indirect = c.storage[G.out].kind == Storage::INDIRECT_IN;
     Ptr px = ptr_of(G.a, 0), pg = ptr_of(G.gate, 0), pe = ptr_of(G.out, 0);
     const bool has_skip = G.out2 >= 0 && !p.views[G.out2][0].dims.empty();
     Ptr ps = has_skip ? ptr_of(G.out2, 0) : Ptr();
@@ -942,6 +965,7 @@ struct Builder {
       pp.count_exec = reinterpret_cast<long long*>(x.arena + slot);
       pp.count_skip = reinterpret_cast<long long*>(auxp + 2 * N * 4);
       launch_pdl(k::gate_partition, dim3(1), dim3(32), 0, x.stream, pp);
+      if (indirect) return cudaGetLastError();   // the consumers read the Switch input through the id lists
       k::SampleCopyParams sc{};
       sc.src = reinterpret_cast<const uint4*>(x.resolve(px));
       sc.vec_per_sample = bytes / 16;
@@ -976,6 +1000,25 @@ struct Builder {
     if (!rc.rt) return fail(E_INTERNAL, "Combine input has no run-time count");
     Ptr pe = ptr_of(G.a, 0), ps = ptr_of(G.res, 0), py = ptr_of(G.out, 0);
     const size_t slot = rc.slot_off;
+    if (c.storage[G.a].kind == Storage::INDIRECT_OUT) {
+      // the executed samples are already in place; the skipped ones move from the Switch input to the
+      // same sample slots of the output
+      if (c.storage[G.res].kind != Storage::INDIRECT_IN) return fail(E_INTERNAL, "Combine: indirect executed operand with a copied skipped operand");
+      add(gi, 1, [=](const RunCtx& x) {
+        char* auxp = x.arena + x.plan->scratch_off[1] + aux;
+        k::SampleCopyParams sc{};
+        sc.dst = reinterpret_cast<uint4*>(x.resolve(py));
+        sc.src = reinterpret_cast<const uint4*>(x.resolve(ps));
+        sc.vec_per_sample = bytes / 16;
+        sc.scatter = 2;
+        sc.idx = reinterpret_cast<const int*>(auxp) + N;
+        sc.count = reinterpret_cast<const long long*>(auxp + 2 * N * 4);
+        const unsigned gx = static_cast<unsigned>(std::max<long long>(1, std::min<long long>(64, sc.vec_per_sample / 256)));
+        launch_pdl(k::sample_copy, dim3(gx, N), dim3(256), 0, x.stream, sc);
+        return cudaGetLastError();
+      });
+      return OK;
+    }
     add(gi, 2, [=](const RunCtx& x) {
       char* auxp = x.arena + x.plan->scratch_off[1] + aux;
       k::SampleCopyParams sc{};

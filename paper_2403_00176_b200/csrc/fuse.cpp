@@ -433,6 +433,50 @@ struct Fuser {
         finish(G);
       }
     }
+    // 3b. index-indirect regrouping: where the executed branch of a Switch is consumed only by
+    // convolutions (as input or residual), the skipped branch only by the matching Combine, and the
+    // Combine's executed operand is a convolution output, nothing is copied at the Switch: the
+    // convolutions read the Switch input through the executed-id list and the last one writes into the
+    // Combine output at those ids; the Combine only moves the skipped samples.
+    if (!(c.flags & (OPT_COPY_REGROUP | OPT_NO_FUSION))) {
+      auto conv_ok = [&](const Group& G) {
+        if (G.kind != GKind::CONV) return false;
+        const Tensor& W = g.tensors[G.w];
+        return W.dtype == DType::BF16 && W.S.rank == 4 && W.S.dims[0].e.is_const() && W.S.dims[1].e.is_const() &&
+               W.S.dims[0].e.const_value() % 64 == 0 && W.S.dims[1].e.const_value() % 64 == 0;
+      };
+      for (size_t si = 0; si < c.groups.size(); ++si) {
+        const Group& S = c.groups[si];
+        if (S.kind != GKind::SWITCH || S.out2 < 0) continue;
+        const int e = S.out, sk = S.out2, x = S.a;
+        if (g.tensors[e].is_output || g.tensors[sk].is_output) continue;
+        int cb = -1;
+        for (size_t ci = 0; ci < c.groups.size(); ++ci)
+          if (c.groups[ci].kind == GKind::COMBINE && c.groups[ci].gate == S.gate && c.groups[ci].res == sk) cb = static_cast<int>(ci);
+        if (cb < 0) continue;
+        const Group& C = c.groups[cb];
+        bool ok = true;
+        for (int cn : data_consumers(e)) {
+          const int gi = assigned[cn];
+          if (gi < 0 || !conv_ok(c.groups[gi])) { ok = false; break; }
+          const Group& G = c.groups[gi];
+          if (!((G.a == e && g.nodes[G.nodes[0]].ins[0] == e) || G.res == e)) { ok = false; break; }
+          if (G.bias == e || G.w == e) { ok = false; break; }
+        }
+        std::vector<int> sc = data_consumers(sk);
+        if (sc.size() != 1 || assigned[sc[0]] != cb) ok = false;
+        const int ye = C.a;
+        const int yp = g.tensors[ye].producer;
+        if (yp < 0 || assigned[yp] < 0 || !conv_ok(c.groups[assigned[yp]]) || c.groups[assigned[yp]].out != ye) ok = false;
+        std::vector<int> yc = data_consumers(ye);
+        if (yc.size() != 1 || assigned[yc[0]] != cb || g.tensors[ye].is_output || g.tensors[C.out].is_output) ok = false;
+        if (c.storage[e].kind != Storage::ROOT || c.storage[sk].kind != Storage::ROOT || c.storage[ye].kind != Storage::ROOT) ok = false;
+        if (!ok) continue;
+        c.storage[e] = Storage{Storage::INDIRECT_IN, S.nodes[0], x, S.gate, 0};
+        c.storage[sk] = Storage{Storage::INDIRECT_IN, S.nodes[0], x, S.gate, 1};
+        c.storage[ye] = Storage{Storage::INDIRECT_OUT, C.nodes[0], C.out, S.gate, 0};
+      }
+    }
     // 4. partition at execution-determined operators (Section 4.3): a node's sub-graph index is
     // one more than that of any execution-determined producer it (transitively) depends on.
     std::vector<int> tsub(g.tensors.size(), 0);

@@ -259,8 +259,8 @@ def test_cfg4_full_config_smallest_request_and_properties():
 
 
 # ------------------------------------------------------------------------------------------------ cfg 5
-def _check_gated(wl, reqs, n_blocks):
-    s, p, outs = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE)
+def _check_gated(wl, reqs, n_blocks, extra_flags=0):
+    s, p, outs = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE | extra_flags)
     req = reqs[0]
     env = O.run(wl.ir, wl.consts, req.inputs)
     # lock-step: every full-batch tensor (stem, block outputs, gates) from the GPU's own inputs
@@ -287,6 +287,18 @@ def test_cfg5_small_gated_network_lockstep():
     wl = WL.cfg5(B=6, side=32, widths=(64, 128), per_stage=2)
     gates = _check_gated(wl, wl.batch(0), 4)
     assert gates.shape == (4, 6)
+
+
+def test_cfg5_small_gated_network_copy_regroup_lockstep():
+    # Switch / Combine as whole-sample copies (the form used where the index-indirect pattern does not apply)
+    wl = WL.cfg5(B=6, side=32, widths=(64, 128), per_stage=2)
+    gates = _check_gated(wl, wl.batch(0), 4, extra_flags=B.OPT_COPY_REGROUP)
+    assert gates.shape == (4, 6)
+    # the default form plans no storage for the regrouped copies
+    g0, g1 = B.Graph(wl.ir), B.Graph(wl.ir, B.OPT_COPY_REGROUP)
+    m0 = g0.bind_dims(wl.sym_names, [[]]).plan().memory()
+    m1 = g1.bind_dims(wl.sym_names, [[]]).plan().memory()
+    assert m0["sum_bytes"] < m1["sum_bytes"]
 
 
 def test_cfg5_all_skip_and_all_execute():
