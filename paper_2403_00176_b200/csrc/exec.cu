@@ -1082,6 +1082,12 @@ struct Builder {
     };
     for (int t : G.ext_in) if (c.storage[t].kind != Storage::FOLDED && !p.views[t][0].dims.empty()) bytes += tb(t);
     for (int t : G.ext_out) if (c.storage[t].kind != Storage::FOLDED && !p.views[t][0].dims.empty()) bytes += tb(t);
+    // index-indirect regrouping moves less: the Switch only partitions the sample ids, the Combine
+    // reads and writes the skipped samples (upper bound: all of them) and never touches the executed operand
+    if (G.kind == GKind::SWITCH && c.storage[G.out].kind == Storage::INDIRECT_IN)
+      bytes = tb(G.gate) + 2.0 * 4.0 * static_cast<double>(p.views[G.a][0].dims[0]);
+    if (G.kind == GKind::COMBINE && c.storage[G.a].kind == Storage::INDIRECT_OUT)
+      bytes = tb(G.res) + tb(G.out) + tb(G.gate);
     if (G.kind == GKind::GEMM) {
       const Tensor& W = g.tensors[G.w];
       const double K = static_cast<double>(W.S.dims[0].e.const_value()), N = static_cast<double>(W.S.dims[1].e.const_value());
