@@ -59,7 +59,9 @@ struct Storage {
   // INDIRECT_IN: an output of a Switch that is never copied: the samples of the Switch input selected
   // by the executed / skipped id list.  INDIRECT_OUT: the executed operand of a Combine, written by its
   // producer straight into the Combine output at the executed ids.
-  enum Kind { ROOT, VIEW_OF_INPUT, VIEW_OF_OUTPUT, FOLDED, INDIRECT_IN, INDIRECT_OUT } kind = ROOT;
+  // ALIAS: the tensor lives in the storage of `other` (same extents): the output of a Combine whose
+  // skipped samples are already where they belong, because the executed ones are written in place.
+  enum Kind { ROOT, VIEW_OF_INPUT, VIEW_OF_OUTPUT, FOLDED, INDIRECT_IN, INDIRECT_OUT, ALIAS } kind = ROOT;
   int node = -1;    // the view operator (Switch / Combine for the indirect kinds)
   int other = -1;   // VIEW_OF_INPUT / INDIRECT_IN: the operator's input; VIEW_OF_OUTPUT / INDIRECT_OUT: the operator's output
   int gate = -1;    // indirect kinds: the gate tensor whose partition gives the id lists

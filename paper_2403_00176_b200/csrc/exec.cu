@@ -1004,6 +1004,7 @@ struct Builder {
       // the executed samples are already in place; the skipped ones move from the Switch input to the
       // same sample slots of the output
       if (c.storage[G.res].kind != Storage::INDIRECT_IN) return fail(E_INTERNAL, "Combine: indirect executed operand with a copied skipped operand");
+      if (c.storage[G.out].kind == Storage::ALIAS) return OK;   // in place: every sample is already where it belongs
       add(gi, 1, [=](const RunCtx& x) {
         char* auxp = x.arena + x.plan->scratch_off[1] + aux;
         k::SampleCopyParams sc{};
@@ -1087,7 +1088,7 @@ struct Builder {
     if (G.kind == GKind::SWITCH && c.storage[G.out].kind == Storage::INDIRECT_IN)
       bytes = tb(G.gate) + 2.0 * 4.0 * static_cast<double>(p.views[G.a][0].dims[0]);
     if (G.kind == GKind::COMBINE && c.storage[G.a].kind == Storage::INDIRECT_OUT)
-      bytes = tb(G.res) + tb(G.out) + tb(G.gate);
+      bytes = c.storage[G.out].kind == Storage::ALIAS ? 0.0 : tb(G.res) + tb(G.out) + tb(G.gate);
     if (G.kind == GKind::GEMM) {
       const Tensor& W = g.tensors[G.w];
       const double K = static_cast<double>(W.S.dims[0].e.const_value()), N = static_cast<double>(W.S.dims[1].e.const_value());

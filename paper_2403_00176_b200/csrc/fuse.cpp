@@ -475,6 +475,27 @@ struct Fuser {
         c.storage[e] = Storage{Storage::INDIRECT_IN, S.nodes[0], x, S.gate, 0};
         c.storage[sk] = Storage{Storage::INDIRECT_IN, S.nodes[0], x, S.gate, 1};
         c.storage[ye] = Storage{Storage::INDIRECT_OUT, C.nodes[0], C.out, S.gate, 0};
+        // In place: if nothing else reads the Switch input (besides the gate that decided the Switch and
+        // the Switch itself), the Combine output takes over its storage; the skipped samples then never
+        // move and the executed ones are overwritten by the block's last convolution, which reads its
+        // residual tile before it stores the same tile.  Not with OPT_NO_REUSE, which promises that every
+        // intermediate stays readable after the run.
+        if (!(c.flags & OPT_NO_REUSE) && !g.tensors[x].is_output && g.tensors[x].kind == TKind::VALUE &&
+            (c.storage[x].kind == Storage::ROOT || c.storage[x].kind == Storage::ALIAS)) {
+          bool only = true;
+          const int gate_prod = g.tensors[S.gate].producer;
+          const int gate_group = gate_prod >= 0 ? assigned[gate_prod] : -1;
+          for (int cn : data_consumers(x)) {
+            const int gi = assigned[cn];
+            if (gi == static_cast<int>(si)) continue;
+            if (gi >= 0 && gi == gate_group && c.groups[gi].kind == GKind::GATE) continue;
+            only = false;
+          }
+          // the block's first convolution must not be the one that writes in place (it reads halos of x)
+          const Group& last = c.groups[assigned[yp]];
+          if (last.a == e) only = false;
+          if (only && c.storage[C.out].kind == Storage::ROOT) c.storage[C.out] = Storage{Storage::ALIAS, C.nodes[0], x, S.gate, 0};
+        }
       }
     }
     // 4. partition at execution-determined operators (Section 4.3): a node's sub-graph index is

@@ -166,6 +166,21 @@ struct Planner {
     if (st.kind == Storage::ROOT) return make_root(t);
     const Node& n = g.nodes[st.node];
     if (b.dims[t].empty()) return fail(E_INTERNAL, "no concrete shape for " + g.tensors[t].name);
+    if (st.kind == Storage::ALIAS) {
+      Status s = resolve(st.other);
+      if (s != OK) return s;
+      for (int r = 0; r < p.n_req; ++r) {
+        const View& vo = p.views[st.other][r];
+        View& v = p.views[t][r];
+        v.root = vo.root;
+        v.offset = vo.offset;
+        v.dims = b.dims[t][r];
+        v.strides = vo.strides;
+        if (v.dims != vo.dims) return fail(E_INTERNAL, "aliased tensors differ in shape: " + g.tensors[t].name);
+      }
+      resolved[t] = 1;
+      return OK;
+    }
     if (st.kind == Storage::INDIRECT_IN || st.kind == Storage::INDIRECT_OUT) {
       // the samples of `other` selected by an id list: same storage, same strides, own (upper-bound) extents
       Status s = resolve(st.other);

@@ -301,6 +301,20 @@ def test_cfg5_small_gated_network_copy_regroup_lockstep():
     assert m0["sum_bytes"] < m1["sum_bytes"]
 
 
+def test_cfg5_small_in_place_blocks_match_the_no_reuse_run():
+    # default flags: identity-shortcut blocks run in place (the Combine output takes over the Switch
+    # input's storage); OPT_NO_REUSE keeps every intermediate in its own buffer.  Same bits either way.
+    wl = WL.cfg5(B=6, side=32, widths=(64, 128), per_stage=3)
+    reqs = wl.batch(0)
+    s0, p0, o0 = run_batch(wl, reqs)
+    s1, p1, o1 = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE)
+    assert p0.plan.memory()["sum_bytes"] < p1.plan.memory()["sum_bytes"]
+    for name in o0[0]:
+        assert np.array_equal(o0[0][name], o1[0][name]), name
+    env = O.run(wl.ir, wl.consts, reqs[0].inputs)
+    assert O.rel_err(o0[0]["gap"], env["gap"]) <= BF16_TOL
+
+
 def test_cfg5_all_skip_and_all_execute():
     # degenerate gate batches: nothing executes (Bx = 0 launches no tile) / everything executes
     for bias_val in (-50.0, 50.0):
