@@ -377,16 +377,16 @@ __global__ void __launch_bounds__(256) gap_partial_f64(GapParams p) {
 #pragma unroll
   for (int i = 0; i < 8; ++i) acc[i] = 0.0;
   if (pg < ppi && (p.C & 7) == 0) {
-    // four loads in flight per thread, added in pixel order (the summation order does not change)
+    // eight loads in flight per thread, added in pixel order (the summation order does not change)
     const __nv_bfloat16* base = p.x + img * p.HW * p.C + cg * 8;
     long long px = p0 + pg;
-    for (; px + 3LL * ppi < p1; px += 4LL * ppi) {
-      uint4 u[4];
+    for (; px + 7LL * ppi < p1; px += 8LL * ppi) {
+      uint4 u[8];
 #pragma unroll
-      for (int k4 = 0; k4 < 4; ++k4) u[k4] = *reinterpret_cast<const uint4*>(base + (px + static_cast<long long>(k4) * ppi) * p.C);
+      for (int k8 = 0; k8 < 8; ++k8) u[k8] = *reinterpret_cast<const uint4*>(base + (px + static_cast<long long>(k8) * ppi) * p.C);
 #pragma unroll
-      for (int k4 = 0; k4 < 4; ++k4) {
-        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u[k4]);
+      for (int k8 = 0; k8 < 8; ++k8) {
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u[k8]);
 #pragma unroll
         for (int i = 0; i < 4; ++i) { const float2 f = __bfloat1622float2(h[i]); acc[2 * i] += static_cast<double>(f.x); acc[2 * i + 1] += static_cast<double>(f.y); }
       }
@@ -404,13 +404,13 @@ __global__ void __launch_bounds__(256) gap_partial_f64(GapParams p) {
 #pragma unroll
   for (int i = 0; i < 8; ++i) part[threadIdx.x][i] = acc[i];
   __syncthreads();
-  if (pg == 0) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      double s = 0.0;
-      for (int g2 = 0; g2 < ppi; ++g2) s += part[g2 * tpp + cg][i];
-      if (cg * 8 + i < p.C) p.partial[(img * p.slabs + blockIdx.y) * p.C + cg * 8 + i] = s;
-    }
+  // fixed-order reduction over the CTA's pixel groups, spread over all threads: thread (cg, i) with
+  // i = channel inside the group of eight adds its column of `part` in group order
+  for (int o = threadIdx.x; o < tpp * 8; o += 256) {
+    const int cg2 = o >> 3, i = o & 7;
+    double s = 0.0;
+    for (int g2 = 0; g2 < ppi; ++g2) s += part[g2 * tpp + cg2][i];
+    if (cg2 * 8 + i < p.C) p.partial[(img * p.slabs + blockIdx.y) * p.C + cg2 * 8 + i] = s;
   }
 }
 __global__ void __launch_bounds__(256) gap_final_f64(GapParams p, int n_img) {
@@ -523,11 +523,18 @@ __global__ void __launch_bounds__(256) gate_logit_f64(GateParams p) {
   ptx::pdl_wait();
   ptx::pdl_launch();
   const int img = blockIdx.x;
+  // eight lanes share a channel: lane part q adds slabs q, q+8, ... in order, then the eight sums are
+  // added in lane order (fixed tree, so the decision does not depend on scheduling)
   double acc = 0.0;
-  for (int c = threadIdx.x; c < p.C; c += 256) {
+  const int q8 = threadIdx.x & 7;
+  for (int c0 = 0; c0 < p.C; c0 += 32) {
+    const int c = c0 + (threadIdx.x >> 3);
     double s = 0.0;
-    for (int k = 0; k < p.slabs; ++k) s += p.partial[(static_cast<long long>(img) * p.slabs + k) * p.C + c];
-    acc += (s / static_cast<double>(p.HW)) * static_cast<double>(__bfloat162float(p.w[c]));
+    if (c < p.C) for (int k = q8; k < p.slabs; k += 8) s += p.partial[(static_cast<long long>(img) * p.slabs + k) * p.C + c];
+    double t = 0.0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) t += __shfl_sync(0xffffffffu, s, (threadIdx.x & 24) + j);
+    if (q8 == 0 && c < p.C) acc += (t / static_cast<double>(p.HW)) * static_cast<double>(__bfloat162float(p.w[c]));
   }
   red[threadIdx.x] = acc;
   __syncthreads();

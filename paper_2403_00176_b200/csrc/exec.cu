@@ -912,7 +912,7 @@ struct Builder {
       k::GapParams gp{};
       gp.C = static_cast<int>(vx.dims[1]);
       gp.HW = vx.dims[2] * vx.dims[3];
-      gp.slabs = static_cast<int>(std::max<long long>(1, std::min<long long>(64, gp.HW / 64)));
+      gp.slabs = static_cast<int>(std::max<long long>(1, std::min<long long>(16, gp.HW / 16)));   // N images x slabs CTAs, each with enough pixels to keep loads in flight
       const int N = static_cast<int>(vx.dims[0]);
       scratch_need = std::max(scratch_need, static_cast<size_t>(N) * gp.slabs * gp.C * 8);
       Ptr px = ptr_of(G.a, r), pw = ptr_of(G.w, 0), pb = ptr_of(G.bias, 0), pg = ptr_of(G.out, r);
@@ -1052,7 +1052,7 @@ struct Builder {
       k::GapParams gp{};
       gp.C = static_cast<int>(vx.dims[1]);
       gp.HW = vx.dims[2] * vx.dims[3];
-      gp.slabs = static_cast<int>(std::max<long long>(1, std::min<long long>(592, gp.HW / 128)));
+      gp.slabs = static_cast<int>(std::max<long long>(1, std::min<long long>(592, gp.HW / (vx.dims[0] >= 16 ? 16 : 128))));
       gp.out_bf16 = O.dtype == DType::BF16;
       const int N = static_cast<int>(vx.dims[0]);
       scratch_need = std::max(scratch_need, static_cast<size_t>(N) * gp.slabs * gp.C * 8);
