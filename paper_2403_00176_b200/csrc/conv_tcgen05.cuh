@@ -349,6 +349,65 @@ __global__ void __launch_bounds__(256) nhwc_to_nchw_bf16(const __nv_bfloat16* __
   }
 }
 
+// The same two layout changes with 16-byte global accesses on both sides (C % 8 == 0, HW % 8 == 0): a
+// 64 x 64 tile goes through shared memory as rows of eight-element vectors whose position inside the row
+// is XOR-ed with the row's group of eight, so that the strided 2-byte gathers of the transposed read hit
+// distinct banks.
+__global__ void __launch_bounds__(256) nchw_to_nhwc_bf16_v8(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out,
+                                                             int C, long long HW) {
+  __shared__ __align__(16) __nv_bfloat16 tile[64][72];   // [channel][pixel vectors, permuted]
+  const long long img = blockIdx.z;
+  const long long p0 = static_cast<long long>(blockIdx.x) * 64;
+  const int c0 = blockIdx.y * 64;
+#pragma unroll
+  for (int it = 0; it < 2; ++it) {
+    const int i = threadIdx.x + it * 256;
+    const int c = i >> 3, v = i & 7;
+    if (c0 + c < C && p0 + v * 8 < HW)
+      *reinterpret_cast<uint4*>(&tile[c][(v ^ ((c >> 3) & 7)) * 8]) = *reinterpret_cast<const uint4*>(in + (img * C + c0 + c) * HW + p0 + v * 8);
+  }
+  __syncthreads();
+#pragma unroll
+  for (int it = 0; it < 2; ++it) {
+    const int i = threadIdx.x + it * 256;
+    const int px = i >> 3, cv = i & 7;
+    if (p0 + px < HW && c0 + cv * 8 < C) {
+      __align__(16) __nv_bfloat16 o[8];
+      const int col = (((px >> 3) ^ cv) * 8) + (px & 7);
+#pragma unroll
+      for (int k8 = 0; k8 < 8; ++k8) o[k8] = tile[cv * 8 + k8][col];
+      *reinterpret_cast<uint4*>(out + (img * HW + p0 + px) * C + c0 + cv * 8) = *reinterpret_cast<const uint4*>(o);
+    }
+  }
+}
+__global__ void __launch_bounds__(256) nhwc_to_nchw_bf16_v8(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out,
+                                                             int C, long long HW) {
+  __shared__ __align__(16) __nv_bfloat16 tile[64][72];   // [pixel][channel vectors, permuted]
+  const long long img = blockIdx.z;
+  const long long p0 = static_cast<long long>(blockIdx.x) * 64;
+  const int c0 = blockIdx.y * 64;
+#pragma unroll
+  for (int it = 0; it < 2; ++it) {
+    const int i = threadIdx.x + it * 256;
+    const int px = i >> 3, cv = i & 7;
+    if (p0 + px < HW && c0 + cv * 8 < C)
+      *reinterpret_cast<uint4*>(&tile[px][(cv ^ ((px >> 3) & 7)) * 8]) = *reinterpret_cast<const uint4*>(in + (img * HW + p0 + px) * C + c0 + cv * 8);
+  }
+  __syncthreads();
+#pragma unroll
+  for (int it = 0; it < 2; ++it) {
+    const int i = threadIdx.x + it * 256;
+    const int c = i >> 3, v = i & 7;
+    if (c0 + c < C && p0 + v * 8 < HW) {
+      __align__(16) __nv_bfloat16 o[8];
+      const int col = (((c >> 3) ^ v) * 8) + (c & 7);
+#pragma unroll
+      for (int k8 = 0; k8 < 8; ++k8) o[k8] = tile[v * 8 + k8][col];
+      *reinterpret_cast<uint4*>(out + (img * C + c0 + c) * HW + p0 + v * 8) = *reinterpret_cast<const uint4*>(o);
+    }
+  }
+}
+
 // Global average pool of a channels-last tensor with fp64 accumulation (decision scalar / final
 // feature): p[n,c] = mean_{h,w} x[n,h,w,c].  Two kernels with a fixed summation order, so the result
 // is deterministic: pixel slabs -> partial sums in scratch, then a serial sum over the slabs.

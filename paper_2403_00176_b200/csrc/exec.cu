@@ -667,8 +667,9 @@ struct Builder {
         const dim3 grid(static_cast<unsigned>((HW + 63) / 64), (C + 63) / 64, N);
         auto* in = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pi));
         auto* out = reinterpret_cast<__nv_bfloat16*>(x.resolve(po));
-        if (from) k::nhwc_to_nchw_bf16<<<grid, 256, 0, x.stream>>>(in, out, C, HW);
-        else k::nchw_to_nhwc_bf16<<<grid, 256, 0, x.stream>>>(in, out, C, HW);
+        const bool v8 = C % 8 == 0 && HW % 8 == 0 && ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15) == 0;
+        if (from) { if (v8) k::nhwc_to_nchw_bf16_v8<<<grid, 256, 0, x.stream>>>(in, out, C, HW); else k::nhwc_to_nchw_bf16<<<grid, 256, 0, x.stream>>>(in, out, C, HW); }
+        else { if (v8) k::nchw_to_nhwc_bf16_v8<<<grid, 256, 0, x.stream>>>(in, out, C, HW); else k::nchw_to_nhwc_bf16<<<grid, 256, 0, x.stream>>>(in, out, C, HW); }
         return cudaGetLastError();
       });
     }
