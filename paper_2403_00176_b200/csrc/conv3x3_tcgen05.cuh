@@ -21,6 +21,17 @@ constexpr int C3_A_SLOT = 17 * 1024;        // 130 rows x 128 B = 16640 B, round
 constexpr int C3_A_BYTES = 130 * 128;
 constexpr int CONV3_THREADS = 416;           // 13 warps, see the kernel's role list
 
+// Up to C3_MAX_REQ requests of one layer in one launch: their tensor maps (extents differ per request)
+// and the prefix of their pixel tiles.  One pool of tiles removes a launch ramp, a weight load and a
+// drain per request and evens out the waves.
+constexpr int C3_MAX_REQ = 8;
+struct Conv3Batch {
+  CUtensorMap tx[C3_MAX_REQ], to[C3_MAX_REQ], tr[C3_MAX_REQ];   // {C, W, H, N} maps: input (box 130 px), output, residual
+  int n_req;
+  int tile_start[C3_MAX_REQ + 1];   // prefix sum of ceil(Wo/128) * Ho * n_img (static image counts)
+  int Ho[C3_MAX_REQ], Wo[C3_MAX_REQ];
+};
+
 template <int BN, bool RES, int STAGES>
 struct Conv3Smem {
   static constexpr int B_STAGE = RES ? 0 : 3 * BN * 128;
@@ -30,12 +41,13 @@ struct Conv3Smem {
   static constexpr int TOTAL = W_RES + STAGES * STAGE_BYTES + NSB * CONV_STAGE_OUT + 896 + 2048 + 128;
 };
 
-// tmX: {Cin, W, H, N}, box {64, 130, 1, 1};  tmW: k-chunk view {64, Cout, K/64} of the weights in
-// (dy, channel chunk, dx, ci) order, box {64, BN, 3};  tmOut / tmRes: {Cout, W, H, N}, box {64, 128, 1, 1}
+// B.tx: {Cin, W, H, N}, box {64, 130, 1, 1};  tmW: k-chunk view {64, Cout, K/64} of the weights in
+// (dy, channel chunk, dx, ci) order, box {64, BN, 3};  B.to / B.tr: {Cout, W, H, N}, box {64, 128, 1, 1}.
+// p.Ho / p.Wo / p.n_img are unused (per request in B); a run-time image count (p.n_img_ptr) is only
+// honoured for single-request launches and then replaces B.tile_start[1].
 template <int BN, bool RES, int STAGES, int ACT>
 __global__ void __launch_bounds__(CONV3_THREADS, 1)
-conv3x3_rows_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
-                          const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmRes, ConvParams p) {
+conv3x3_rows_bf16_tcgen05(const __grid_constant__ Conv3Batch B, const __grid_constant__ CUtensorMap tmW, ConvParams p) {
   using S = Conv3Smem<BN, RES, STAGES>;
   constexpr int PASSES = BN / 64;
   constexpr int NSB = S::NSB;
@@ -66,10 +78,12 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_
     *dead = 0;
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
-    ptx::prefetch_tmap(&tmX);
     ptx::prefetch_tmap(&tmW);
-    ptx::prefetch_tmap(&tmOut);
-    if (p.has_residual) ptx::prefetch_tmap(&tmRes);
+    for (int r = 0; r < B.n_req; ++r) {
+      ptx::prefetch_tmap(&B.tx[r]);
+      ptx::prefetch_tmap(&B.to[r]);
+      if (p.has_residual) ptx::prefetch_tmap(&B.tr[r]);
+    }
   }
   if (warp == 3) { ptx::tmem_alloc(tmem_slot, TMEM_COLS); ptx::tmem_relinquish(); }
   ptx::tc_fence_before();
@@ -83,21 +97,29 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_
   }
   ptx::pdl_wait();
   ptx::pdl_launch();
-  int n_img = p.n_img;
-  if (p.n_img_ptr) n_img = min(p.n_img, max(0, p.cnt_a + p.cnt_b * static_cast<int>(*p.n_img_ptr)));
-  const int tiles_w = (p.Wo + 127) / 128;
-  const int tiles_px = tiles_w * p.Ho * n_img;
+  int tiles_px = B.tile_start[B.n_req];
+  if (p.n_img_ptr) {   // gated sub-batch (single request): the image count is on the device
+    const int n_img = min(p.n_img, max(0, p.cnt_a + p.cnt_b * static_cast<int>(*p.n_img_ptr)));
+    tiles_px = ((B.Wo[0] + 127) / 128) * B.Ho[0] * n_img;
+  }
   const int num_tiles = tiles_px * ((p.Cout + BN - 1) / BN);
   const int cchunks = p.Cin / 64;
   const int kstages = 3 * cchunks;               // stage = (dy, channel chunk), dy outermost
 
-  auto decode = [&](int t, int* n0, int* img, int* h0, int* w0) {
-    const int tp = t % tiles_px;
+  // tile index -> (channel tile, request, image, row, first pixel); pixel tiles vary fastest
+  auto decode = [&](int t, int* n0, int* img, int* h0, int* w0) -> int {
+    int tp = t % tiles_px;
     *n0 = (t / tiles_px) * BN;
-    *img = tp / (tiles_w * p.Ho);
-    const int r = tp % (tiles_w * p.Ho);
-    *h0 = r / tiles_w;
-    *w0 = (r % tiles_w) * 128;
+    int r = 0;
+    while (r + 1 < B.n_req && tp >= B.tile_start[r + 1]) ++r;
+    tp -= B.tile_start[r];
+    const int tiles_w = (B.Wo[r] + 127) / 128;
+    const int per_img = tiles_w * B.Ho[r];
+    *img = tp / per_img;
+    const int rem = tp - *img * per_img;
+    *h0 = rem / tiles_w;
+    *w0 = (rem - *h0 * tiles_w) * 128;
+    return r;
   };
 
   if (warp == 0) {
@@ -106,14 +128,14 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_
       int n = 0;
       for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
         int n0, img, h0, w0;
-        decode(t, &n0, &img, &h0, &w0);
+        const int rq = decode(t, &n0, &img, &h0, &w0);
         if (p.in_ids) img = p.in_ids[img];
         for (int ks = 0; ks < kstages; ++ks, ++n) {
           const int s = n % STAGES;
           if (n >= STAGES) ptx::mbar_wait(&empty[s], ((n / STAGES) - 1) & 1, dead);
           const int dy = ks / cchunks, cc = ks % cchunks;
           ptx::mbar_expect_tx(&full[s], C3_A_BYTES);
-          ptx::tma_load_4d(tiles + s * S::STAGE_BYTES, &tmX, cc * 64, w0 - 1, h0 + dy - 1, img, &full[s]);
+          ptx::tma_load_4d(tiles + s * S::STAGE_BYTES, &B.tx[rq], cc * 64, w0 - 1, h0 + dy - 1, img, &full[s]);
         }
       }
     }
@@ -184,12 +206,12 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_
       auto prepare = [&](int u) {
         const int t = blockIdx.x + (u / PASSES) * gridDim.x;
         int n0, img, h0, w0;
-        decode(t, &n0, &img, &h0, &w0);
+        const int rq = decode(t, &n0, &img, &h0, &w0);
         const int np = n0 + (u % PASSES) * 64;
         const int bsel = u % NSB;
         if (p.has_residual && np < p.Cout) {
           ptx::mbar_expect_tx(&res_full[bsel], CONV_STAGE_OUT);
-          ptx::tma_load_4d(out_stage + bsel * CONV_STAGE_OUT, &tmRes, np, w0, h0, p.res_ids ? p.res_ids[img] : img, &res_full[bsel]);
+          ptx::tma_load_4d(out_stage + bsel * CONV_STAGE_OUT, &B.tr[rq], np, w0, h0, p.res_ids ? p.res_ids[img] : img, &res_full[bsel]);
         } else {
           ptx::mbar_arrive(&res_full[bsel]);
         }
@@ -200,10 +222,10 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_
         ptx::mbar_wait(&stage_ready[bsel], (u / NSB) & 1, dead);
         const int t = blockIdx.x + (u / PASSES) * gridDim.x;
         int n0, img, h0, w0;
-        decode(t, &n0, &img, &h0, &w0);
+        const int rq = decode(t, &n0, &img, &h0, &w0);
         const int np = n0 + (u % PASSES) * 64;
         if (np < p.Cout) {
-          tma_store_4d(&tmOut, out_stage + bsel * CONV_STAGE_OUT, np, w0, h0, p.out_ids ? p.out_ids[img] : img);
+          tma_store_4d(&B.to[rq], out_stage + bsel * CONV_STAGE_OUT, np, w0, h0, p.out_ids ? p.out_ids[img] : img);
           bulk_commit();
         }
         if (u + NSB < U) {

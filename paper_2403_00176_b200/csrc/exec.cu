@@ -754,6 +754,79 @@ struct Builder {
     for (size_t i = 0; i < c.packed_consts.size(); ++i) if (c.packed_consts[i] == G.w) pk = c.packed_off[i];
     const int bn = (Cout % 128 == 0) ? 128 : 64;
     const int kch = 2;
+    // requests that take the row-halo kernel are collected and launched together (up to C3_MAX_REQ per launch)
+    struct RowsReq { Ptr px, po, pr; int H, W, Ho, Wo, n_img, n_in_map, n_out_map, n_res_map; k::ConvParams cp; bool rt; size_t rt_slot; long long ids_in, ids_res, ids_out; };
+    std::vector<RowsReq> rows_reqs;
+    Ptr pw_all; pw_all.where = 5; pw_all.off = static_cast<int64_t>(pk);
+    Ptr pb_all = G.bias >= 0 ? ptr_of(G.bias, 0) : Ptr();
+    auto emit_rows = [&](std::vector<RowsReq> batch) {
+      const bool hb = G.bias >= 0, hr = G.res >= 0;
+      const int act = G.act;
+      const bool wres = Cin == 64 && Cout == 64;
+      const int K = 9 * Cin;
+      const Ptr pw = pw_all, pb = pb_all;
+      struct Cache { std::vector<const void*> key; CUtensorMap tw; k::Conv3Batch B; };
+      auto cache = std::make_shared<Cache>();
+      long long tiles = 0;
+      for (auto& q : batch) tiles += static_cast<long long>((q.Wo + 127) / 128) * q.Ho * q.n_img;
+      tiles *= (Cout + bn - 1) / bn;
+      add(gi, 1, [=](const RunCtx& x) mutable {
+        std::vector<const void*> key;
+        const void* Wp = x.resolve(pw);
+        key.push_back(Wp);
+        for (auto& q : batch) { key.push_back(x.resolve(q.px)); key.push_back(x.resolve(q.po)); key.push_back(hr ? x.resolve(q.pr) : nullptr); }
+        if (cache->key != key) {
+          k::Conv3Batch& B = cache->B;
+          B.n_req = static_cast<int>(batch.size());
+          int ts = 0;
+          for (size_t i = 0; i < batch.size(); ++i) {
+            const RowsReq& q = batch[i];
+            const void* X = key[1 + 3 * i];
+            void* O = const_cast<void*>(key[2 + 3 * i]);
+            const void* R = hr ? key[3 + 3 * i] : O;
+            if (!encode_bf16_nhwc(&B.tx[i], X, q.n_in_map, q.H, q.W, Cin, 130, 1, 1) ||
+                !encode_bf16_nhwc(&B.to[i], O, q.n_out_map, q.Ho, q.Wo, Cout, 128, 1, 1) ||
+                !encode_bf16_nhwc(&B.tr[i], R, hr ? q.n_res_map : q.n_out_map, q.Ho, q.Wo, Cout, 128, 1, 1))
+              return cudaErrorInvalidValue;
+            B.tile_start[i] = ts;
+            ts += ((q.Wo + 127) / 128) * q.Ho * q.n_img;
+            B.Ho[i] = q.Ho; B.Wo[i] = q.Wo;
+          }
+          B.tile_start[batch.size()] = ts;
+          if (!encode_bf16_kchunks(&cache->tw, Wp, Cout, K, K, bn, 3)) return cudaErrorInvalidValue;
+          cache->key = key;
+        }
+        k::ConvParams cp = batch[0].cp;
+        cp.bias = hb ? reinterpret_cast<const __nv_bfloat16*>(x.resolve(pb)) : nullptr;
+        cp.status = reinterpret_cast<int*>(x.arena);
+        cp.n_img_ptr = batch[0].rt ? reinterpret_cast<const long long*>(x.arena + batch[0].rt_slot) : nullptr;
+        const char* auxb = x.arena + x.plan->scratch_off[1];
+        cp.in_ids = batch[0].ids_in >= 0 ? reinterpret_cast<const int*>(auxb + batch[0].ids_in) : nullptr;
+        cp.res_ids = batch[0].ids_res >= 0 ? reinterpret_cast<const int*>(auxb + batch[0].ids_res) : nullptr;
+        cp.out_ids = batch[0].ids_out >= 0 ? reinterpret_cast<const int*>(auxb + batch[0].ids_out) : nullptr;
+        const dim3 gd(static_cast<unsigned>(std::min<long long>(tiles, x.plan->sm_count)));
+        const int variant = (wres ? 4 : 0) + (bn == 128 ? 2 : 0) + (act == 2 ? 1 : 0);
+#define SOD2_CONV3_CASE(V, BN_, RES_, ST_, ACT_)                                                                         \
+        case V: {                                                                                                        \
+          constexpr int smem = k::Conv3Smem<BN_, RES_, ST_>::TOTAL;                                                       \
+          static bool once = (cudaFuncSetAttribute(k::conv3x3_rows_bf16_tcgen05<BN_, RES_, ST_, ACT_>,                    \
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);             \
+          (void)once;                                                                                                    \
+          launch_pdl(k::conv3x3_rows_bf16_tcgen05<BN_, RES_, ST_, ACT_>, gd, dim3(k::CONV3_THREADS), smem, x.stream, cache->B, cache->tw, cp); \
+        } break;
+        switch (variant) {
+          SOD2_CONV3_CASE(0, 64, false, 4, 0)
+          SOD2_CONV3_CASE(1, 64, false, 4, 2)
+          SOD2_CONV3_CASE(2, 128, false, 3, 0)
+          SOD2_CONV3_CASE(3, 128, false, 3, 2)
+          SOD2_CONV3_CASE(4, 64, true, 7, 0)
+          default:
+          SOD2_CONV3_CASE(5, 64, true, 7, 2)
+        }
+#undef SOD2_CONV3_CASE
+        return cudaGetLastError();
+      });
+    };
     for (int r = 0; r < p.n_req; ++r) {
       const View &vx = p.views[G.a][r], &vo = p.views[G.out][r];
       if (!numel(vo.dims) || !numel(vx.dims)) continue;
@@ -809,6 +882,15 @@ struct Builder {
       const int n_in_map = static_cast<int>(vx.ind_gate >= 0 ? p.views[vx.root][r].dims[0] : vx.dims[0]);
       const int n_out_map = static_cast<int>(vo.ind_gate >= 0 ? p.views[vo.root][r].dims[0] : vo.dims[0]);
       const int n_res_map = G.res >= 0 ? static_cast<int>(p.views[G.res][r].ind_gate >= 0 ? p.views[p.views[G.res][r].root][r].dims[0] : p.views[G.res][r].dims[0]) : 0;
+      if (rows) {
+        RowsReq q{px, po, pr, H, Wd, cp.Ho, cp.Wo, cp.n_img, n_in_map, n_out_map, n_res_map, cp, rt, rt_slot, ids_in, ids_res, ids_out};
+        // a run-time image count or id lists belong to one request: such a request is launched alone
+        const bool solo = rt || ids_in >= 0 || ids_res >= 0 || ids_out >= 0;
+        if (solo) { emit_rows({q}); continue; }
+        rows_reqs.push_back(q);
+        if (rows_reqs.size() == static_cast<size_t>(k::C3_MAX_REQ)) { emit_rows(rows_reqs); rows_reqs.clear(); }
+        continue;
+      }
       struct Cache { const void* a = nullptr; const void* w = nullptr; const void* o = nullptr; const void* r = nullptr; CUtensorMap tx, tw, to, tr; };
       auto cache = std::make_shared<Cache>();
       add(gi, 1, [=](const RunCtx& x) mutable {
@@ -817,8 +899,8 @@ struct Builder {
         void* O = x.resolve(po);
         const void* R = hr ? x.resolve(pr) : O;
         if (cache->a != X || cache->w != Wp || cache->o != O || cache->r != R) {
-          if (!encode_bf16_nhwc(&cache->tx, X, n_in_map, H, Wd, Cin, rows ? 130 : cp.TW, cp.TH, stride) ||
-              !encode_bf16_kchunks(&cache->tw, Wp, Cout, K, K, bn, rows ? 3 : kch) ||
+          if (!encode_bf16_nhwc(&cache->tx, X, n_in_map, H, Wd, Cin, cp.TW, cp.TH, stride) ||
+              !encode_bf16_kchunks(&cache->tw, Wp, Cout, K, K, bn, kch) ||
               !encode_bf16_nhwc(&cache->to, O, n_out_map, cp.Ho, cp.Wo, Cout, cp.TW, cp.TH, 1) ||
               !encode_bf16_nhwc(&cache->tr, R, hr ? n_res_map : n_out_map, cp.Ho, cp.Wo, Cout, cp.TW, cp.TH, 1))
             return cudaErrorInvalidValue;
@@ -832,16 +914,7 @@ struct Builder {
         cp.res_ids = ids_res >= 0 ? reinterpret_cast<const int*>(auxb + ids_res) : nullptr;
         cp.out_ids = ids_out >= 0 ? reinterpret_cast<const int*>(auxb + ids_out) : nullptr;
         const dim3 gd(static_cast<unsigned>(std::min<long long>(tiles, x.plan->sm_count))), bd(k::CONV_THREADS);
-        const int variant = (rows ? (wres ? 8 : 4) : 0) + (bn == 128 ? 2 : 0) + (act == 2 ? 1 : 0);
-#define SOD2_CONV3_CASE(V, BN_, RES_, ST_, ACT_)                                                                         \
-        case V: {                                                                                                        \
-          constexpr int smem = k::Conv3Smem<BN_, RES_, ST_>::TOTAL;                                                       \
-          static bool once = (cudaFuncSetAttribute(k::conv3x3_rows_bf16_tcgen05<BN_, RES_, ST_, ACT_>,                    \
-                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);             \
-          (void)once;                                                                                                    \
-          launch_pdl(k::conv3x3_rows_bf16_tcgen05<BN_, RES_, ST_, ACT_>, gd, dim3(k::CONV3_THREADS), smem, x.stream, cache->tx, cache->tw, \
-                     cache->to, cache->tr, cp);                                                                          \
-        } break;
+        const int variant = (bn == 128 ? 2 : 0) + (act == 2 ? 1 : 0);
 #define SOD2_CONV_CASE(V, BN_, KCH_, ST_, ACT_)                                                                          \
         case V: {                                                                                                        \
           constexpr int smem = k::ConvSmem<BN_, KCH_, ST_>::TOTAL;                                                        \
@@ -855,20 +928,14 @@ struct Builder {
           SOD2_CONV_CASE(0, 64, 2, 4, 0)
           SOD2_CONV_CASE(1, 64, 2, 4, 2)
           SOD2_CONV_CASE(2, 128, 2, 3, 0)
-          SOD2_CONV_CASE(3, 128, 2, 3, 2)
-          SOD2_CONV3_CASE(4, 64, false, 4, 0)
-          SOD2_CONV3_CASE(5, 64, false, 4, 2)
-          SOD2_CONV3_CASE(6, 128, false, 3, 0)
-          SOD2_CONV3_CASE(7, 128, false, 3, 2)
-          SOD2_CONV3_CASE(8, 64, true, 7, 0)
           default:
-          SOD2_CONV3_CASE(9, 64, true, 7, 2)
+          SOD2_CONV_CASE(3, 128, 2, 3, 2)
         }
 #undef SOD2_CONV_CASE
-#undef SOD2_CONV3_CASE
         return cudaGetLastError();
       });
     }
+    if (!rows_reqs.empty()) emit_rows(rows_reqs);
     return OK;
   }
 
