@@ -163,6 +163,7 @@ struct Planner {
     if (resolved[t]) return OK;
     const Storage& st = c.storage[t];
     if (st.kind == Storage::FOLDED) { resolved[t] = 1; return OK; }
+    p.views[t].resize(p.n_req);
     if (st.kind == Storage::ROOT) return make_root(t);
     const Node& n = g.nodes[st.node];
     if (b.dims[t].empty()) return fail(E_INTERNAL, "no concrete shape for " + g.tensors[t].name);
@@ -255,7 +256,7 @@ struct Planner {
 
   Status run() {
     size_t T = g.tensors.size();
-    p.views.assign(T, std::vector<View>(p.n_req));
+    p.views.assign(T, {});   // filled per tensor when it is resolved
     p.roots.assign(T, RootBuf());
     // resolve every tensor a group touches
     for (auto& G : c.groups) {
