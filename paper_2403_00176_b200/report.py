@@ -73,7 +73,8 @@ def measure(cfg: int, reps: int, oracle_budget: float):
     kinds = PF.kind_summary(rep)
     sum_ms = sum(r["ms"] for r in rep)
     sum_roof = sum(r["t_roof_ms"] for r in rep)
-    worst = min((r for r in rep if r["t_roof_ms"] > 0), key=lambda r: r["frac"])
+    # worst group among those that matter (at least 1 % of the time of all groups)
+    worst = min((r for r in rep if r["t_roof_ms"] > 0 and r["ms"] >= 0.01 * sum_ms), key=lambda r: r["frac"])
     # planning overhead
     plan_us = []
     for i in range(5):
