@@ -258,6 +258,48 @@ def test_cfg4_full_config_smallest_request_and_properties():
         assert np.allclose(outs[r]["gap"].reshape(-1), y.mean(axis=(2, 3)).reshape(-1), rtol=1e-2, atol=1e-2)
 
 
+def _gemm_graph(K, N, act, residual):
+    lines = ["sym M 1 4096", f"input x bf16 [1,M,{K}]"]
+    if residual:
+        lines.append(f"input r bf16 [1,M,{N}]")
+    lines += [f"const W bf16 [{K},{N}]", f"const b bf16 [{N}]", "node MatMul x W -> t0", "node Add t0 b -> t1"]
+    cur = "t1"
+    if act:
+        lines.append(f"node {act} {cur} -> t2"); cur = "t2"
+    if residual:
+        lines.append(f"node Add {cur} r -> t3"); cur = "t3"
+    lines.append(f"node Relu {cur} -> y" if residual and not act else f"node Add {cur} b -> y")
+    lines.append("output y")
+    return "\n".join(lines) + "\n"
+
+
+def test_gemm_epilogue_forms_ragged_shapes():
+    # the tcgen05 GEMM group over row counts around the 128-row tile, column counts that are not
+    # multiples of the 64-column pass (8-column granularity) and K of one to several 64-chunks, in every
+    # epilogue form: bias, bias+ReLU, bias+GELU, bias+residual(+ReLU)
+    rng = np.random.default_rng(7)
+    cases = [(64, 8, None, False), (64, 72, "Relu", False), (192, 136, "Gelu", False), (128, 264, None, True),
+             (320, 520, "Gelu", False), (64, 768, None, True)]
+    for K, N, act, residual in cases:
+        ir = _gemm_graph(K, N, act, residual)
+        consts = {"W": bf16_round((rng.standard_normal((K, N)) / np.sqrt(K)).astype(np.float32)),
+                  "b": bf16_round(rng.standard_normal(N).astype(np.float32))}
+        reqs = []
+        for M in (1, 127, 128, 129, 300):
+            ins = {"x": bf16_round(rng.standard_normal((1, M, K)).astype(np.float32))}
+            if residual:
+                ins["r"] = bf16_round(rng.standard_normal((1, M, N)).astype(np.float32))
+            reqs.append(Request({"M": M}, ins))
+        wl = WL.Workload("gemm_case", "bf16", ir, consts, ["M"], ["y"], {"batch_fn": lambda j: reqs})
+        s, p, outs = run_batch(wl, reqs)
+        kinds = [s.graph.group_info(i)["kind"] for i in range(s.graph.num_groups())]
+        assert kinds[0] == "gemm", kinds
+        for r, req in enumerate(reqs):
+            ref = O.run(ir, consts, req.inputs)["y"]
+            assert outs[r]["y"].shape == ref.shape
+            assert O.rel_err(outs[r]["y"], ref) <= BF16_TOL, (K, N, act, residual, req.syms)
+
+
 # ------------------------------------------------------------------------------------------------ cfg 5
 def _check_gated(wl, reqs, n_blocks, extra_flags=0):
     s, p, outs = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE | extra_flags)
