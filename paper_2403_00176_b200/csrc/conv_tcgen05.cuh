@@ -484,7 +484,10 @@ __global__ void __launch_bounds__(256) gap_final_f64(GapParams p, int n_img) {
   const long long img = ok ? i / p.C : 0;
   const int c = ok ? static_cast<int>(i % p.C) : 0;
   double acc = 0.0;
-  if (ok) for (int s = g; s < p.slabs; s += 8) acc += p.partial[(img * p.slabs + s) * p.C + c];
+  if (ok) {
+#pragma unroll 8
+    for (int s = g; s < p.slabs; s += 8) acc += p.partial[(img * p.slabs + s) * p.C + c];
+  }
   part[g][cl] = acc;
   __syncthreads();
   if (g == 0 && ok) {
@@ -582,19 +585,19 @@ __global__ void __launch_bounds__(256) gate_logit_f64(GateParams p) {
   ptx::pdl_wait();
   ptx::pdl_launch();
   const int img = blockIdx.x;
-  // eight lanes share a channel: lane part q adds slabs q, q+8, ... in order, then the eight sums are
-  // added in lane order (fixed tree, so the decision does not depend on scheduling)
+  // item (q, c): slabs q, q+8, ... of channel c added in order (independent loads, unrolled), times w[c];
+  // a thread adds its items in index order and the 256 thread sums go through a fixed tree, so the
+  // decision does not depend on scheduling
   double acc = 0.0;
-  const int q8 = threadIdx.x & 7;
-  for (int c0 = 0; c0 < p.C; c0 += 32) {
-    const int c = c0 + (threadIdx.x >> 3);
+  for (int idx = threadIdx.x; idx < 8 * p.C; idx += 256) {
+    const int q8 = idx / p.C, c = idx - q8 * p.C;
+    const double* pp = p.partial + static_cast<long long>(img) * p.slabs * p.C + c;
     double s = 0.0;
-    if (c < p.C) for (int k = q8; k < p.slabs; k += 8) s += p.partial[(static_cast<long long>(img) * p.slabs + k) * p.C + c];
-    double t = 0.0;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) t += __shfl_sync(0xffffffffu, s, (threadIdx.x & 24) + j);
-    if (q8 == 0 && c < p.C) acc += (t / static_cast<double>(p.HW)) * static_cast<double>(__bfloat162float(p.w[c]));
+#pragma unroll 4
+    for (int k = q8; k < p.slabs; k += 8) s += pp[static_cast<long long>(k) * p.C];
+    acc += s * static_cast<double>(__bfloat162float(p.w[c]));
   }
+  acc /= static_cast<double>(p.HW);
   red[threadIdx.x] = acc;
   __syncthreads();
   for (int o = 128; o; o >>= 1) { if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o]; __syncthreads(); }
