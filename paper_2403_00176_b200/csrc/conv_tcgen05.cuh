@@ -216,8 +216,8 @@ conv_igemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_co
       float* bias_t = bias_s + (j & 1) * 256;
       bias_t[et] = bias_next;
       bias_next = load_bias(t + gridDim.x);
+      if (warp == 4) ptx::mbar_wait_warp(&tmem_full[acc], (j >> 1) & 1, dead);   // one polling warp, the others park at the barrier
       conv_epi_bar();
-      ptx::mbar_wait_warp(&tmem_full[acc], (j >> 1) & 1, dead);
       ptx::tc_fence_after();
 #pragma unroll 1
       for (int ps = 0; ps < PASSES; ++ps) {

@@ -341,8 +341,10 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       float* bias_t = bias_s + (j & 1) * 256;      // this tile's bias, prefetched during the last tile
       bias_t[et] = bias_next;
       bias_next = load_bias(t + gridDim.x);
+      // one warp polls for the accumulator, the others park at the hardware barrier: seven more polling
+      // lanes cost the main loop 3-4 % of its issue slots
+      if (warp == 3) ptx::mbar_wait_warp(&tmem_full[acc], (j >> 1) & 1, dead);
       epi_bar_sync();
-      ptx::mbar_wait_warp(&tmem_full[acc], (j >> 1) & 1, dead);
       ptx::tc_fence_after();
       if (et == 0) { SOD2_TRACE(2, 30 + j) }
       const uint32_t taddr = tmem + (static_cast<uint32_t>(q * 32) << 16) + acc * BN + half * 32;
