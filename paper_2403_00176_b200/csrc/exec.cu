@@ -305,26 +305,32 @@ struct Builder {
         ep.status = reinterpret_cast<int*>(x.arena);
         const int tiles = tiles_m * static_cast<int>((N + bn - 1) / bn);
         const int grid = std::min(tiles, x.plan->sm_count);
-        const int variant = (bn == 256 ? 0 : 3) + act;
+        const int variant = (bn == 256 ? 0 : 6) + act * 2 + (hr ? 1 : 0);
         const dim3 gd(grid), bd(k::GEMM_THREADS);
         const int Ni = static_cast<int>(N), Ki = static_cast<int>(K);
-#define SOD2_GEMM_CASE(V, BN_, KCH_, ST_, ACT_)                                                                              \
+#define SOD2_GEMM_CASE(V, BN_, KCH_, ST_, ACT_, RES_)                                                                        \
         case V: {                                                                                                            \
           constexpr int smem = k::GemmSmem<BN_, KCH_, ST_>::TOTAL;                                                            \
-          static bool once = (cudaFuncSetAttribute(k::gemm_bf16_tcgen05<BN_, KCH_, ST_, ACT_>,                                \
+          static bool once = (cudaFuncSetAttribute(k::gemm_bf16_tcgen05<BN_, KCH_, ST_, ACT_, false, RES_>,                   \
                                                    cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);                 \
           (void)once;                                                                                                        \
-          launch_pdl(k::gemm_bf16_tcgen05<BN_, KCH_, ST_, ACT_>, gd, bd, smem, x.stream, cache->ta, cache->tb, cache->to,     \
-                     cache->tr, M, Ni, Ki, ep);                                                                               \
+          launch_pdl(k::gemm_bf16_tcgen05<BN_, KCH_, ST_, ACT_, false, RES_>, gd, bd, smem, x.stream, cache->ta, cache->tb,   \
+                     cache->to, cache->tr, M, Ni, Ki, ep);                                                                    \
         } break;
         switch (variant) {
-          SOD2_GEMM_CASE(0, 256, 1, 4, 0)
-          SOD2_GEMM_CASE(1, 256, 1, 4, 1)
-          SOD2_GEMM_CASE(2, 256, 1, 4, 2)
-          SOD2_GEMM_CASE(3, 128, 2, 3, 0)
-          SOD2_GEMM_CASE(4, 128, 2, 3, 1)
+          SOD2_GEMM_CASE(0, 256, 1, 4, 0, false)
+          SOD2_GEMM_CASE(1, 256, 1, 4, 0, true)
+          SOD2_GEMM_CASE(2, 256, 1, 4, 1, false)
+          SOD2_GEMM_CASE(3, 256, 1, 4, 1, true)
+          SOD2_GEMM_CASE(4, 256, 1, 4, 2, false)
+          SOD2_GEMM_CASE(5, 256, 1, 4, 2, true)
+          SOD2_GEMM_CASE(6, 128, 2, 3, 0, false)
+          SOD2_GEMM_CASE(7, 128, 2, 3, 0, true)
+          SOD2_GEMM_CASE(8, 128, 2, 3, 1, false)
+          SOD2_GEMM_CASE(9, 128, 2, 3, 1, true)
+          SOD2_GEMM_CASE(10, 128, 2, 3, 2, false)
           default:
-          SOD2_GEMM_CASE(5, 128, 2, 3, 2)
+          SOD2_GEMM_CASE(11, 128, 2, 3, 2, true)
         }
 #undef SOD2_GEMM_CASE
         return cudaGetLastError();

@@ -96,11 +96,13 @@ __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 256;"
 // {64, 128 or BN, KCH}: one instruction fills KCH consecutive swizzled [rows x 64] chunks.
 // B must be a constant of the graph (prepacked weights): its producer does not wait for the
 // previous kernel in the stream.
+// RES: the group adds a residual tile (a compile-time switch: a run-time branch inside the unrolled
+// element loops splits them into basic blocks and exposes every shared-memory latency).
 // SPLITK: a work item is (tile, K range); the epilogue stores the raw fp32 partial tile into slab
 // `range` of an fp32 [ranges, M, N] workspace (tmOut is then a 3-D fp32 map with boxes of 32 columns)
 // and a finishing kernel adds the slabs in a fixed order and applies bias, residual and LayerNorm.
 // This spreads a GEMM with few output tiles and a long K over all SMs, deterministically.
-template <int BN, int KCH, int STAGES, int ACT, bool SPLITK = false>
+template <int BN, int KCH, int STAGES, int ACT, bool SPLITK = false, bool RES = false>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmRes,
@@ -151,7 +153,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     ptx::prefetch_tmap(&tmA);
     ptx::prefetch_tmap(&tmB);
     ptx::prefetch_tmap(&tmOut);
-    if (ep.has_residual) ptx::prefetch_tmap(&tmRes);
+    if (RES) ptx::prefetch_tmap(&tmRes);
   }
   if (warp == 2) { ptx::tmem_alloc(tmem_slot, TMEM_COLS); ptx::tmem_relinquish(); }
   ptx::tc_fence_before();
@@ -252,7 +254,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const int t = SPLITK ? w % out_tiles : w;
         const int m0 = (t % tiles_m) * GEMM_BM, np = (t / tiles_m) * BN + (u % PASSES) * PASS_COLS;
         const int bsel = u % NSB;
-        if (!SPLITK && ep.has_residual && np < N) {
+        if (!SPLITK && RES && np < N) {
           ptx::mbar_expect_tx(&buf_ready[bsel], GEMM_STAGE_OUT);
           ptx::tma_load_2d(out_stage + bsel * GEMM_STAGE_OUT, &tmRes, np, m0, &buf_ready[bsel]);
         } else {
@@ -354,7 +356,6 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       for (int ps = 0; ps < PASSES; ++ps, ++u) {
         const int np = n0 + ps * GEMM_PASS_COLS;
         const bool live = np < N;
-        const bool res = ep.has_residual && live;
         const int bsel = u % NSB;
         uint8_t* obase = out_stage + bsel * GEMM_STAGE_OUT + row * 128;
         ptx::tmem_ld_wait();
@@ -375,7 +376,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
             for (int i = 0; i < 8; ++i) v[i] = apply_act<ACT>(__uint_as_float(r[ps & 1][g * 8 + i]) + bp[g * 8 + i]);
             uint4* slot = reinterpret_cast<uint4*>(obase + (((half * 4 + g) ^ (row & 7)) << 4));
-            if (res) {
+            if constexpr (RES) {
               const uint4 rv = *slot;
               const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&rv);
 #pragma unroll
