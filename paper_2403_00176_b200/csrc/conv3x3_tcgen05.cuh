@@ -45,7 +45,7 @@ struct Conv3Smem {
 // (dy, channel chunk, dx, ci) order, box {64, BN, 3};  B.to / B.tr: {Cout, W, H, N}, box {64, 128, 1, 1}.
 // p.Ho / p.Wo / p.n_img are unused (per request in B); a run-time image count (p.n_img_ptr) is only
 // honoured for single-request launches and then replaces B.tile_start[1].
-template <int BN, bool RES, int STAGES, int ACT>
+template <int BN, bool RES, int STAGES, int ACT, bool HASRES>
 __global__ void __launch_bounds__(CONV3_THREADS, 1)
 conv3x3_rows_bf16_tcgen05(const __grid_constant__ Conv3Batch B, const __grid_constant__ CUtensorMap tmW, ConvParams p) {
   using S = Conv3Smem<BN, RES, STAGES>;
@@ -82,7 +82,7 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ Conv3Batch B, const __grid_con
     for (int r = 0; r < B.n_req; ++r) {
       ptx::prefetch_tmap(&B.tx[r]);
       ptx::prefetch_tmap(&B.to[r]);
-      if (p.has_residual) ptx::prefetch_tmap(&B.tr[r]);
+      if (HASRES) ptx::prefetch_tmap(&B.tr[r]);
     }
   }
   if (warp == 3) { ptx::tmem_alloc(tmem_slot, TMEM_COLS); ptx::tmem_relinquish(); }
@@ -209,7 +209,7 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ Conv3Batch B, const __grid_con
         const int rq = decode(t, &n0, &img, &h0, &w0);
         const int np = n0 + (u % PASSES) * 64;
         const int bsel = u % NSB;
-        if (p.has_residual && np < p.Cout) {
+        if (HASRES && np < p.Cout) {
           ptx::mbar_expect_tx(&res_full[bsel], CONV_STAGE_OUT);
           ptx::tma_load_4d(out_stage + bsel * CONV_STAGE_OUT, &B.tr[rq], np, w0, h0, p.res_ids ? p.res_ids[img] : img, &res_full[bsel]);
         } else {
@@ -262,7 +262,6 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ Conv3Batch B, const __grid_con
       for (int ps = 0; ps < PASSES; ++ps, ++u) {
         const int np = n0 + ps * 64;
         const bool live = np < p.Cout;
-        const bool res = p.has_residual && live;
         const int bsel = u % NSB;
         uint8_t* obase = out_stage + bsel * CONV_STAGE_OUT + row * 128;
         uint32_t r[32];
@@ -284,7 +283,7 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ Conv3Batch B, const __grid_con
 #pragma unroll
             for (int i = 0; i < 8; ++i) v[i] = apply_act<ACT>(__uint_as_float(r[g * 8 + i]) + bp[g * 8 + i]);
             uint4* slot = reinterpret_cast<uint4*>(obase + (((half * 4 + g) ^ (row & 7)) << 4));
-            if (res) {
+            if constexpr (HASRES) {
               const uint4 rv = *slot;
               const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&rv);
 #pragma unroll

@@ -65,7 +65,7 @@ __device__ __forceinline__ void conv_epi_bar() { asm volatile("bar.sync 1, 256;"
 // tmX: {Cin, W, H, N} bf16, box {64, TW, TH, 1}, element strides {1, s, s, 1}
 // tmW: {64, Cout, K/64} k-chunk view of [Cout, K], box {64, BN, KCH}
 // tmOut / tmRes: {Cout, Wo, Ho, N}, box {64, TW, TH, 1}
-template <int BN, int KCH, int STAGES, int ACT>
+template <int BN, int KCH, int STAGES, int ACT, bool HASRES>
 __global__ void __launch_bounds__(CONV_THREADS, 1)
 conv_igemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
                         const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmRes, ConvParams p) {
@@ -96,7 +96,7 @@ conv_igemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_co
     ptx::prefetch_tmap(&tmX);
     ptx::prefetch_tmap(&tmW);
     ptx::prefetch_tmap(&tmOut);
-    if (p.has_residual) ptx::prefetch_tmap(&tmRes);
+    if (HASRES) ptx::prefetch_tmap(&tmRes);
   }
   if (warp == 3) { ptx::tmem_alloc(tmem_slot, TMEM_COLS); ptx::tmem_relinquish(); }
   ptx::tc_fence_before();
@@ -223,7 +223,8 @@ conv_igemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_co
       for (int ps = 0; ps < PASSES; ++ps) {
         const int np = n0 + ps * 64;
         const bool live = np < p.Cout;
-        const bool res = p.has_residual && live;
+        constexpr bool res_t = HASRES;
+        const bool res = res_t && live;
         if (res) {
           if (et == 0) {
             bulk_wait_read0();
@@ -245,7 +246,7 @@ conv_igemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_co
             float v[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) v[i] = apply_act<ACT>(__uint_as_float(r[g * 8 + i]) + bp[g * 8 + i]);
-            if (res) {
+            if constexpr (HASRES) {
               const uint4 rv = *reinterpret_cast<const uint4*>(obase + (((half * 4 + g) ^ (row & 7)) << 4));
               const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&rv);
 #pragma unroll

@@ -811,23 +811,29 @@ struct Builder {
         cp.res_ids = batch[0].ids_res >= 0 ? reinterpret_cast<const int*>(auxb + batch[0].ids_res) : nullptr;
         cp.out_ids = batch[0].ids_out >= 0 ? reinterpret_cast<const int*>(auxb + batch[0].ids_out) : nullptr;
         const dim3 gd(static_cast<unsigned>(std::min<long long>(tiles, x.plan->sm_count)));
-        const int variant = (wres ? 4 : 0) + (bn == 128 ? 2 : 0) + (act == 2 ? 1 : 0);
-#define SOD2_CONV3_CASE(V, BN_, RES_, ST_, ACT_)                                                                         \
+        const int variant = ((wres ? 4 : 0) + (bn == 128 ? 2 : 0) + (act == 2 ? 1 : 0)) * 2 + (hr ? 1 : 0);
+#define SOD2_CONV3_CASE(V, BN_, RES_, ST_, ACT_, HR_)                                                                    \
         case V: {                                                                                                        \
           constexpr int smem = k::Conv3Smem<BN_, RES_, ST_>::TOTAL;                                                       \
-          static bool once = (cudaFuncSetAttribute(k::conv3x3_rows_bf16_tcgen05<BN_, RES_, ST_, ACT_>,                    \
+          static bool once = (cudaFuncSetAttribute(k::conv3x3_rows_bf16_tcgen05<BN_, RES_, ST_, ACT_, HR_>,               \
                                                    cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);             \
           (void)once;                                                                                                    \
-          launch_pdl(k::conv3x3_rows_bf16_tcgen05<BN_, RES_, ST_, ACT_>, gd, dim3(k::CONV3_THREADS), smem, x.stream, cache->B, cache->tw, cp); \
+          launch_pdl(k::conv3x3_rows_bf16_tcgen05<BN_, RES_, ST_, ACT_, HR_>, gd, dim3(k::CONV3_THREADS), smem, x.stream, cache->B, cache->tw, cp); \
         } break;
         switch (variant) {
-          SOD2_CONV3_CASE(0, 64, false, 4, 0)
-          SOD2_CONV3_CASE(1, 64, false, 4, 2)
-          SOD2_CONV3_CASE(2, 128, false, 3, 0)
-          SOD2_CONV3_CASE(3, 128, false, 3, 2)
-          SOD2_CONV3_CASE(4, 64, true, 7, 0)
+          SOD2_CONV3_CASE(0, 64, false, 4, 0, false)
+          SOD2_CONV3_CASE(1, 64, false, 4, 0, true)
+          SOD2_CONV3_CASE(2, 64, false, 4, 2, false)
+          SOD2_CONV3_CASE(3, 64, false, 4, 2, true)
+          SOD2_CONV3_CASE(4, 128, false, 3, 0, false)
+          SOD2_CONV3_CASE(5, 128, false, 3, 0, true)
+          SOD2_CONV3_CASE(6, 128, false, 3, 2, false)
+          SOD2_CONV3_CASE(7, 128, false, 3, 2, true)
+          SOD2_CONV3_CASE(8, 64, true, 7, 0, false)
+          SOD2_CONV3_CASE(9, 64, true, 7, 0, true)
+          SOD2_CONV3_CASE(10, 64, true, 7, 2, false)
           default:
-          SOD2_CONV3_CASE(5, 64, true, 7, 2)
+          SOD2_CONV3_CASE(11, 64, true, 7, 2, true)
         }
 #undef SOD2_CONV3_CASE
         return cudaGetLastError();
@@ -920,22 +926,26 @@ struct Builder {
         cp.res_ids = ids_res >= 0 ? reinterpret_cast<const int*>(auxb + ids_res) : nullptr;
         cp.out_ids = ids_out >= 0 ? reinterpret_cast<const int*>(auxb + ids_out) : nullptr;
         const dim3 gd(static_cast<unsigned>(std::min<long long>(tiles, x.plan->sm_count))), bd(k::CONV_THREADS);
-        const int variant = (bn == 128 ? 2 : 0) + (act == 2 ? 1 : 0);
-#define SOD2_CONV_CASE(V, BN_, KCH_, ST_, ACT_)                                                                          \
+        const int variant = ((bn == 128 ? 2 : 0) + (act == 2 ? 1 : 0)) * 2 + (hr ? 1 : 0);
+#define SOD2_CONV_CASE(V, BN_, KCH_, ST_, ACT_, HR_)                                                                     \
         case V: {                                                                                                        \
           constexpr int smem = k::ConvSmem<BN_, KCH_, ST_>::TOTAL;                                                        \
-          static bool once = (cudaFuncSetAttribute(k::conv_igemm_bf16_tcgen05<BN_, KCH_, ST_, ACT_>,                      \
+          static bool once = (cudaFuncSetAttribute(k::conv_igemm_bf16_tcgen05<BN_, KCH_, ST_, ACT_, HR_>,                 \
                                                    cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);             \
           (void)once;                                                                                                    \
-          launch_pdl(k::conv_igemm_bf16_tcgen05<BN_, KCH_, ST_, ACT_>, gd, bd, smem, x.stream, cache->tx, cache->tw,     \
+          launch_pdl(k::conv_igemm_bf16_tcgen05<BN_, KCH_, ST_, ACT_, HR_>, gd, bd, smem, x.stream, cache->tx, cache->tw, \
                      cache->to, cache->tr, cp);                                                                          \
         } break;
         switch (variant) {
-          SOD2_CONV_CASE(0, 64, 2, 4, 0)
-          SOD2_CONV_CASE(1, 64, 2, 4, 2)
-          SOD2_CONV_CASE(2, 128, 2, 3, 0)
+          SOD2_CONV_CASE(0, 64, 2, 4, 0, false)
+          SOD2_CONV_CASE(1, 64, 2, 4, 0, true)
+          SOD2_CONV_CASE(2, 64, 2, 4, 2, false)
+          SOD2_CONV_CASE(3, 64, 2, 4, 2, true)
+          SOD2_CONV_CASE(4, 128, 2, 3, 0, false)
+          SOD2_CONV_CASE(5, 128, 2, 3, 0, true)
+          SOD2_CONV_CASE(6, 128, 2, 3, 2, false)
           default:
-          SOD2_CONV_CASE(3, 128, 2, 3, 2)
+          SOD2_CONV_CASE(7, 128, 2, 3, 2, true)
         }
 #undef SOD2_CONV_CASE
         return cudaGetLastError();
