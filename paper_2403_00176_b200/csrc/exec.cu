@@ -879,7 +879,6 @@ struct Builder {
       }
       // wide images with a 3x3 / stride 1 / pad 1 kernel: row-halo kernel (a tile is 128 pixels of one row)
       const bool rows = ks == 3 && G.stride == 1 && G.pad == 1 && cp.Wo >= 96 && ((cp.Wo + 127) / 128) * 128 * 4 <= cp.Wo * 5;
-      const bool wres = rows && Cin == 64 && Cout == 64;
       if (rows) { cp.TW = 128; cp.TH = 1; }
       if (cp.TW * G.stride > 256 || cp.TH * G.stride > 256) return fail(E_UNSUPPORTED_OP, "convolution stride too large for the TMA box");
       const int H = static_cast<int>(vx.dims[2]), Wd = static_cast<int>(vx.dims[3]);

@@ -339,7 +339,6 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const float relu2_floor = ep.act2 == ACT_RELU ? 0.0f : -INFINITY;  // post-residual activation, branch-free
     for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++j) {
       const int acc = j & 1;
-      const int n0 = (t / tiles_m) * BN;
       float* bias_t = bias_s + (j & 1) * 256;      // this tile's bias, prefetched during the last tile
       bias_t[et] = bias_next;
       bias_next = load_bias(t + gridDim.x);
@@ -354,8 +353,6 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       ptx::tmem_ld32(taddr, r[0]);
 #pragma unroll
       for (int ps = 0; ps < PASSES; ++ps, ++u) {
-        const int np = n0 + ps * GEMM_PASS_COLS;
-        const bool live = np < N;
         const int bsel = u % NSB;
         uint8_t* obase = out_stage + bsel * GEMM_STAGE_OUT + row * 128;
         ptx::tmem_ld_wait();
@@ -367,29 +364,37 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(&tmem_empty[acc]);
         }
-        ptx::mbar_wait_warp(&buf_ready[bsel], (u / NSB) & 1, dead);
-        if (live) {
-          const float* bp = bias_t + ps * GEMM_PASS_COLS + half * 32;
+        // everything that does not need the staging buffer happens before the wait for it: bias and
+        // activation (and, without a residual, the bf16 packing); columns past N compute harmless
+        // values that the agent never stores
+        const float* bp = bias_t + ps * GEMM_PASS_COLS + half * 32;
+        float v[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = apply_act<ACT>(__uint_as_float(r[ps & 1][i]) + bp[i]);
+        uint4 pk[4];
+        if constexpr (!RES) {
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
-            float v[8];
+            __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&pk[g]);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = apply_act<ACT>(__uint_as_float(r[ps & 1][g * 8 + i]) + bp[g * 8 + i]);
-            uint4* slot = reinterpret_cast<uint4*>(obase + (((half * 4 + g) ^ (row & 7)) << 4));
-            if constexpr (RES) {
-              const uint4 rv = *slot;
-              const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&rv);
-#pragma unroll
-              for (int i = 0; i < 4; ++i) { const float2 f = __bfloat1622float2(h[i]); v[2 * i] += f.x; v[2 * i + 1] += f.y; }
-#pragma unroll
-              for (int i = 0; i < 8; ++i) v[i] = fmaxf(v[i], relu2_floor);
-            }
-            uint4 pk;
-            __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&pk);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) oh[i] = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
-            *slot = pk;
+            for (int i = 0; i < 4; ++i) oh[i] = __floats2bfloat162_rn(v[g * 8 + 2 * i], v[g * 8 + 2 * i + 1]);
           }
+        }
+        ptx::mbar_wait_warp(&buf_ready[bsel], (u / NSB) & 1, dead);
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          uint4* slot = reinterpret_cast<uint4*>(obase + (((half * 4 + g) ^ (row & 7)) << 4));
+          if constexpr (RES) {
+            const uint4 rv = *slot;
+            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&rv);
+            __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&pk[g]);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float2 f = __bfloat1622float2(h[i]);
+              oh[i] = __floats2bfloat162_rn(fmaxf(v[g * 8 + 2 * i] + f.x, relu2_floor), fmaxf(v[g * 8 + 2 * i + 1] + f.y, relu2_floor));
+            }
+          }
+          *slot = pk[g];
         }
         ptx::fence_proxy_async();
         __syncwarp();
