@@ -471,12 +471,20 @@ struct Builder {
         auto* Gm = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pg));
         auto* Bt = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pb));
         const unsigned grid = static_cast<unsigned>((rows + 7) / 8);
+        const bool full = D == ch * 256;
+#define SOD2_LN_CASE(CH_)                                                                                                 \
+        case CH_:                                                                                                        \
+          if (full) launch_pdl(k::layernorm_bf16<CH_, true>, dim3(grid), dim3(256), 0, x.stream, X, Gm, Bt, Y, rows, static_cast<int>(D), eps); \
+          else launch_pdl(k::layernorm_bf16<CH_, false>, dim3(grid), dim3(256), 0, x.stream, X, Gm, Bt, Y, rows, static_cast<int>(D), eps);     \
+          break;
         switch (ch) {
-          case 1: launch_pdl(k::layernorm_bf16<1>, dim3(grid), dim3(256), 0, x.stream, X, Gm, Bt, Y, rows, static_cast<int>(D), eps); break;
-          case 2: launch_pdl(k::layernorm_bf16<2>, dim3(grid), dim3(256), 0, x.stream, X, Gm, Bt, Y, rows, static_cast<int>(D), eps); break;
-          case 3: launch_pdl(k::layernorm_bf16<3>, dim3(grid), dim3(256), 0, x.stream, X, Gm, Bt, Y, rows, static_cast<int>(D), eps); break;
-          default: launch_pdl(k::layernorm_bf16<4>, dim3(grid), dim3(256), 0, x.stream, X, Gm, Bt, Y, rows, static_cast<int>(D), eps); break;
+          SOD2_LN_CASE(1)
+          SOD2_LN_CASE(2)
+          SOD2_LN_CASE(3)
+          default:
+          SOD2_LN_CASE(4)
         }
+#undef SOD2_LN_CASE
         return cudaGetLastError();
       });
     }

@@ -94,7 +94,10 @@ __global__ void __launch_bounds__(256) fused_mlp_ln_f32(MlpLnParams p) {
 // ---------------------------------------------------------------------------------------------
 // LayerNorm over the last dim of a packed [rows, D] bf16 matrix, rows known only at run time.
 // One warp per row, 128-bit loads, the row lives in registers (D <= 256 * CH), fp32 math.
-template <int CH>
+// FULL: D == CH * 256, every lane owns CH full vectors: no guards, so the loads of a row are issued
+// back to back (a guard per vector puts every load into a basic block of its own and serialises their
+// latencies).
+template <int CH, bool FULL>
 __global__ void __launch_bounds__(256) layernorm_bf16(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ gamma,
                                                        const __nv_bfloat16* __restrict__ beta, __nv_bfloat16* __restrict__ y,
                                                        long long rows, int D, float eps) {
@@ -106,7 +109,7 @@ __global__ void __launch_bounds__(256) layernorm_bf16(const __nv_bfloat16* __res
 #pragma unroll
   for (int c = 0; c < CH; ++c) {
     const int i = c * 32 + lane;
-    if (i < nvec) { g4[c] = reinterpret_cast<const uint4*>(gamma)[i]; b4[c] = reinterpret_cast<const uint4*>(beta)[i]; }
+    if (FULL || i < nvec) { g4[c] = reinterpret_cast<const uint4*>(gamma)[i]; b4[c] = reinterpret_cast<const uint4*>(beta)[i]; }
   }
   ptx::pdl_launch();
   ptx::pdl_wait();
@@ -117,7 +120,7 @@ __global__ void __launch_bounds__(256) layernorm_bf16(const __nv_bfloat16* __res
 #pragma unroll
   for (int c = 0; c < CH; ++c) {
     const int i = c * 32 + lane;
-    if (i < nvec) {
+    if (FULL || i < nvec) {
       uint4 u = xr[i];
       const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
@@ -131,7 +134,7 @@ __global__ void __launch_bounds__(256) layernorm_bf16(const __nv_bfloat16* __res
   float q = 0.f;
 #pragma unroll
   for (int c = 0; c < CH; ++c)
-    if (c * 32 + lane < nvec) {
+    if (FULL || c * 32 + lane < nvec) {
 #pragma unroll
       for (int t = 0; t < 8; ++t) { const float d = v[c][t] - mu; q += d * d; }
     }
@@ -140,7 +143,7 @@ __global__ void __launch_bounds__(256) layernorm_bf16(const __nv_bfloat16* __res
 #pragma unroll
   for (int c = 0; c < CH; ++c) {
     const int i = c * 32 + lane;
-    if (i < nvec) {
+    if (FULL || i < nvec) {
       uint4 o;
       const __nv_bfloat162* gh = reinterpret_cast<const __nv_bfloat162*>(&g4[c]);
       const __nv_bfloat162* bh = reinterpret_cast<const __nv_bfloat162*>(&b4[c]);
