@@ -44,6 +44,7 @@ typedef enum {
 #define SOD2_OPT_NO_REUSE  2u /* every arena tensor keeps its own slot: intermediates stay readable */
 #define SOD2_OPT_COPY_REGROUP 16u /* Switch / Combine always copy whole samples (no index-indirect convolutions) */
 #define SOD2_OPT_LEGACY_ATTENTION 8u /* attention groups run the mma.sync kernel even where the tcgen05 kernel applies */
+#define SOD2_OPT_NO_SEP 32u /* groups run in their default topological order: no static execution planning (Section 4.3) */
 #define SOD2_OPT_SPLITK_LN 4u /* bf16 GEMM (+bias, +residual) -> LayerNorm as one group: split-K GEMM into fp32 slabs + finishing kernel */
 
 /* Parse the graph text (host, ir_len bytes), classify every operator (Table 2), run RDP
@@ -123,6 +124,15 @@ sod2_status sod2_graph_group_info(const sod2_graph* g, int group, char* kind_buf
                                   int* versions, int* subgraph_id);
 int sod2_graph_num_subgraphs(const sod2_graph* g);
 int sod2_graph_rdp_sweeps(const sod2_graph* g);
+/* Static execution planning (Section 4.3): the order of the fused groups inside each sub-graph of the
+ * nac partition is the one of least peak live intermediate bytes, found by a search over all
+ * topological orders with tensor sizes taken at the upper bounds of the declared symbol ranges
+ * (lower bounds break ties).  out[0], out[1]: peak live bytes of the default order at the upper and
+ * lower corner; out[2], out[3]: the same for the planned order; out[4]: sets of finished groups the
+ * search visited; out[5], out[6], out[7]: sub-graphs searched, reordered, abandoned (state budget
+ * exceeded: default order kept); out[8]: 1 if some tensor size has no static bound (nothing searched).
+ * `out` is host memory for 9 values.  All zero under SOD2_OPT_NO_SEP. */
+sod2_status sod2_graph_order_info(const sod2_graph* g, int64_t* out);
 /* Classification of an operator name alone (Table 2). Returns SOD2_E_UNSUPPORTED_OP if unknown. */
 sod2_status sod2_classify(const char* op_type, int* dyn_class);
 /* Re-run RDP visiting the operators in the given order (a permutation of 0..num_ops-1); used to

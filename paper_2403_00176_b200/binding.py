@@ -21,6 +21,7 @@ OPT_NO_REUSE = 2
 OPT_SPLITK_LN = 4
 OPT_LEGACY_ATTENTION = 8
 OPT_COPY_REGROUP = 16
+OPT_NO_SEP = 32
 DYN_CLASS = ["ISDO", "ISDOS", "ISVDOS", "EDO"]
 
 
@@ -59,6 +60,7 @@ def _load() -> C.CDLL:
         "sod2_graph_group_info": [vp, i32, cp, sz, P(i32), P(i32), P(i32)],
         "sod2_classify": [cp, P(i32)],
         "sod2_graph_reanalyse": [vp, P(i32), i32],
+        "sod2_graph_order_info": [vp, P(i64)],
         "sod2_binding_shape": [vp, i32, cp, P(i64), P(i32)],
         "sod2_plan_slot": [vp, cp, P(sz), P(sz), P(i32), P(i32)],
         "sod2_plan_instance_offset": [vp, cp, i32, P(sz)],
@@ -88,7 +90,7 @@ EXPORTS = ["sod2_graph_create", "sod2_graph_destroy", "sod2_graph_set_const", "s
            "sod2_graph_prepack", "sod2_bind_dims", "sod2_binding_destroy", "sod2_plan", "sod2_plan_destroy",
            "sod2_run", "sod2_run_timed", "sod2_plan_device_status", "sod2_graph_tensor_info", "sod2_graph_tensor_value", "sod2_graph_tensor_dtype",
            "sod2_graph_num_ops", "sod2_graph_op_info", "sod2_graph_num_groups", "sod2_graph_group_info",
-           "sod2_graph_num_subgraphs", "sod2_graph_rdp_sweeps", "sod2_classify", "sod2_graph_reanalyse",
+           "sod2_graph_num_subgraphs", "sod2_graph_rdp_sweeps", "sod2_classify", "sod2_graph_reanalyse", "sod2_graph_order_info",
            "sod2_binding_shape", "sod2_plan_slot", "sod2_plan_instance_offset", "sod2_plan_memory", "sod2_plan_group_cost", "sod2_plan_tensor_strides",
            "sod2_run_output_shape", "sod2_nonzero_static", "sod2_last_error"]
 
@@ -191,6 +193,14 @@ class Graph:
 
     def rdp_sweeps(self) -> int:
         return lib.sod2_graph_rdp_sweeps(self.h)
+
+    def order_info(self) -> dict:
+        """Static execution planning (Section 4.3): peaks of the default and planned group order."""
+        out = (C.c_int64 * 9)()
+        _check(lib.sod2_graph_order_info(self.h, out), self.h)
+        keys = ("default_peak_hi", "default_peak_lo", "planned_peak_hi", "planned_peak_lo", "states",
+                "searched_subgraphs", "reordered_subgraphs", "abandoned_subgraphs", "unbounded")
+        return dict(zip(keys, [int(v) for v in out]))
 
     def reanalyse(self, order: Sequence[int]):
         arr = (C.c_int * len(order))(*order)

@@ -217,6 +217,17 @@ int sod2_graph_num_groups(const sod2_graph* g) { return g ? static_cast<int>(g->
 int sod2_graph_num_subgraphs(const sod2_graph* g) { return g ? g->c.n_subgraphs : -1; }
 int sod2_graph_rdp_sweeps(const sod2_graph* g) { return g ? g->c.g.rdp_sweeps : -1; }
 
+sod2_status sod2_graph_order_info(const sod2_graph* g, int64_t* out) {
+  if (!g || !out) return SOD2_E_INVALID_ARG;
+  const OrderStats& s = g->c.order_stats;
+  out[0] = s.default_peak[0]; out[1] = s.default_peak[1];
+  out[2] = s.planned_peak[0]; out[3] = s.planned_peak[1];
+  out[4] = s.states;
+  out[5] = s.searched_subgraphs; out[6] = s.reordered_subgraphs; out[7] = s.abandoned_subgraphs;
+  out[8] = s.unbounded;
+  return SOD2_OK;
+}
+
 sod2_status sod2_graph_op_info(const sod2_graph* g, int op, char* type, size_t type_len, int* cls, int* eff, int* group, int* sub) {
   if (!g || op < 0 || op >= static_cast<int>(g->c.g.nodes.size())) return SOD2_E_INVALID_ARG;
   const Node& n = g->c.g.nodes[op];

@@ -14,6 +14,7 @@ enum OptFlags : uint32_t {
   OPT_NO_REUSE = 2u,    // every arena tensor gets its own slot (keeps all intermediates readable after a run)
   OPT_COPY_REGROUP = 16u,     // Switch / Combine always move whole samples (no index-indirect convolutions)
   OPT_LEGACY_ATTENTION = 8u,  // attention groups on the mma.sync kernel even where the tcgen05 kernel applies
+  OPT_NO_SEP = 32u,     // groups run in their default topological order (no static execution planning)
   OPT_SPLITK_LN = 4u,   // a bf16 GEMM (+bias, +residual) followed by LayerNorm becomes one group: split-K GEMM + finishing kernel
 };
 
@@ -68,8 +69,18 @@ struct Storage {
   int list = 0;     // indirect kinds: 0 = executed ids, 1 = skipped ids
 };
 
+// Outcome of static execution planning (Section 4.3): peak of live arena bytes of the default and of
+// the planned group order, at the upper [0] and lower [1] corner of the declared symbol ranges.
+struct OrderStats {
+  int64_t default_peak[2] = {0, 0}, planned_peak[2] = {0, 0};
+  int64_t states = 0;                 // sets of finished groups visited by the search
+  int searched_subgraphs = 0, reordered_subgraphs = 0, abandoned_subgraphs = 0;
+  int unbounded = 0;                  // 1: some tensor size has no static bound, nothing was searched
+};
+
 struct Compiled {
   Graph g;
+  OrderStats order_stats;
   uint32_t flags = 0;
   std::vector<Group> groups;          // in execution order
   std::vector<Storage> storage;       // per tensor
@@ -90,6 +101,9 @@ struct Compiled {
 void set_thread_error(const std::string& msg);
 
 Status form_groups(Compiled* c);
+// Static execution planning: `order` (default topological order on entry) becomes the order of least
+// peak live bytes found per sub-graph; deps[g] lists the groups that must precede g.
+void plan_execution_order(Compiled* c, const std::vector<std::vector<int>>& deps, std::vector<int>* order);
 // Transposed (K-major) copies of the GEMM weights into caller-owned workspace; enqueued on `stream`.
 Status prepack_weights(Compiled* c, void* workspace, size_t bytes, void* stream);
 

@@ -543,6 +543,12 @@ struct Fuser {
       done[pick] = 1;
       orderg.push_back(pick);
     }
+    // 5b. static execution planning (Section 4.3): the order of least peak memory inside each sub-graph
+    if (!(c.flags & OPT_NO_SEP)) {
+      std::vector<std::vector<int>> dv(G);
+      for (size_t gi = 0; gi < G; ++gi) dv[gi].assign(deps[gi].begin(), deps[gi].end());
+      plan_execution_order(&c, dv, &orderg);
+    }
     std::vector<Group> sorted;
     std::vector<int> remap(G);
     for (size_t i = 0; i < G; ++i) { remap[orderg[i]] = static_cast<int>(i); sorted.push_back(c.groups[orderg[i]]); }

@@ -7,6 +7,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <map>
+#include <tuple>
 
 #include "engine.h"
 
@@ -309,7 +310,8 @@ struct Planner {
     struct Placed { size_t off, size; int def, last; };
     std::vector<Placed> placed;
     size_t top = HEADER;
-    auto place = [&](int t) {
+    // smallest_gap: the smallest free gap that fits (ties: lowest offset); otherwise the lowest one
+    auto place = [&](int t, bool smallest_gap) {
       RootBuf& R = p.roots[t];
       size_t need = sz(t);
       if (c.flags & OPT_NO_REUSE) { R.arena_off = top; top += need; placed.push_back({R.arena_off, need, R.def_step, R.last_step}); return; }
@@ -319,7 +321,11 @@ struct Planner {
       std::sort(busy.begin(), busy.end());
       size_t best_off = SIZE_MAX, best_gap = SIZE_MAX, cur = HEADER;
       for (auto& iv : busy) {
-        if (iv.first > cur && iv.first - cur >= need && iv.first - cur < best_gap) { best_gap = iv.first - cur; best_off = cur; }
+        if (iv.first > cur && iv.first - cur >= need && iv.first - cur < best_gap) {
+          best_gap = iv.first - cur;
+          best_off = cur;
+          if (!smallest_gap) break;
+        }
         cur = std::max(cur, iv.second);
       }
       if (best_off == SIZE_MAX) best_off = cur;  // after the last overlapping tensor (may extend the arena)
@@ -332,17 +338,37 @@ struct Planner {
     std::vector<int> at_peak;
     for (int t : ids) if (p.roots[t].def_step <= peak && p.roots[t].last_step >= peak) at_peak.push_back(t);
     std::sort(at_peak.begin(), at_peak.end(), [&](int x, int y) { return std::make_pair(p.roots[x].def_step, x) < std::make_pair(p.roots[y].def_step, y); });
-    for (int t : at_peak) { place(t); done[t] = 1; }
+    for (int t : at_peak) { place(t, true); done[t] = 1; }
     // 2. forward from the peak
     std::vector<int> fwd;
     for (int t : ids) if (!done[t] && p.roots[t].def_step > peak) fwd.push_back(t);
     std::sort(fwd.begin(), fwd.end(), [&](int x, int y) { return std::make_pair(p.roots[x].def_step, x) < std::make_pair(p.roots[y].def_step, y); });
-    for (int t : fwd) { place(t); done[t] = 1; }
+    for (int t : fwd) { place(t, true); done[t] = 1; }
     // 3. backward from the peak: tensors dead before it, latest last-use first
     std::vector<int> bwd;
     for (int t : ids) if (!done[t]) bwd.push_back(t);
     std::sort(bwd.begin(), bwd.end(), [&](int x, int y) { return std::make_pair(-p.roots[x].last_step, x) < std::make_pair(-p.roots[y].last_step, y); });
-    for (int t : bwd) { place(t); done[t] = 1; }
+    for (int t : bwd) { place(t, true); done[t] = 1; }
+    // 4. where memory does not fall off monotonically on both sides of the peak (branches whose small
+    // results outlive their large intermediates), the walk above fragments.  If it ended more than 2 %
+    // above the live peak, a second placement is tried, largest tensor first at the lowest offset
+    // that is free over its lifetime, and the smaller arena is kept.
+    if (!(c.flags & OPT_NO_REUSE) && top - HEADER > p.peak_live_bytes + p.peak_live_bytes / 50) {
+      std::vector<size_t> first_off(ids.size());
+      for (size_t i = 0; i < ids.size(); ++i) first_off[i] = p.roots[ids[i]].arena_off;
+      const size_t first_top = top;
+      placed.clear();
+      top = HEADER;
+      std::vector<int> by_size = ids;
+      std::sort(by_size.begin(), by_size.end(), [&](int x, int y) {
+        return std::make_tuple(~sz(x), p.roots[x].def_step, x) < std::make_tuple(~sz(y), p.roots[y].def_step, y);
+      });
+      for (int t : by_size) place(t, false);
+      if (top >= first_top) {
+        for (size_t i = 0; i < ids.size(); ++i) p.roots[ids[i]].arena_off = first_off[i];
+        top = first_top;
+      }
+    }
     p.arena_bytes = top;
     return OK;
   }

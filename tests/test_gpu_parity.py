@@ -300,6 +300,39 @@ def test_gemm_epilogue_forms_ragged_shapes():
             assert O.rel_err(outs[r]["y"], ref) <= BF16_TOL, (K, N, act, residual, req.syms)
 
 
+def test_branched_graph_planned_order_matches_default_order_and_oracle():
+    # static execution planning reorders the groups of a branched graph (smaller live peak); the result
+    # is bit-identical to the default order's and agrees with the oracle
+    from tests.test_execution_order import _branched_graph
+    import random
+    rnd = random.Random(21)
+    ir = _branched_graph(rnd, 4)
+    g = O.parse(ir)
+    rng = np.random.default_rng(3)
+    consts = {}
+    for ln in ir.splitlines():
+        if ln.startswith("const"):
+            _, name, _, shp = ln.split()
+            k, n = [int(v) for v in shp.strip("[]").split(",")]
+            consts[name] = bf16_round((rng.standard_normal((k, n)) / np.sqrt(k)).astype(np.float32))
+    reqs = [Request({"N": n}, {"x": bf16_round(rng.standard_normal((1, n, 64)).astype(np.float32))}) for n in (2, 130, 515)]
+    out_name = [ln.split()[1] for ln in ir.splitlines() if ln.startswith("output")][0]
+    wl = WL.Workload("branched", "bf16", ir, consts, ["N"], [out_name], {"batch_fn": lambda j: reqs})
+    s1, p1, o1 = run_batch(wl, reqs)
+    s2, p2, o2 = run_batch(wl, reqs, opt_flags=B.OPT_NO_SEP)
+    info = s1.graph.order_info()
+    assert info["reordered_subgraphs"] == 1 and info["planned_peak_hi"] < info["default_peak_hi"]
+    assert p1.plan.memory()["peak_live_bytes"] < p2.plan.memory()["peak_live_bytes"]
+    assert p1.plan.memory()["arena_bytes"] < p2.plan.memory()["arena_bytes"]
+    s3, p3, o3 = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE)   # planned order, every intermediate kept
+    for r, req in enumerate(reqs):
+        assert np.array_equal(o1[r][out_name], o2[r][out_name]) and np.array_equal(o1[r][out_name], o3[r][out_name])
+        assert O.rel_err(o1[r][out_name], _oracle_out(wl, req, out_name)) <= BF16_TOL
+        errs = lockstep(wl, s3, p3, o3, r, BF16_TOL)
+        bad = {k: v for k, v in errs.items() if not (isinstance(v, float) and v <= BF16_TOL)}
+        assert errs and not bad, (req.syms, bad)
+
+
 # ------------------------------------------------------------------------------------------------ cfg 5
 def _check_gated(wl, reqs, n_blocks, extra_flags=0):
     s, p, outs = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE | extra_flags)

@@ -126,4 +126,4 @@ def test_plan_vs_exhaustive_optimum_on_small_graphs():
         tensors_top = max(s["offset"] + (s["bytes"] + 255) // 256 * 256 for s in slots.values()) - 256
         assert tensors_top >= opt >= mem["peak_live_bytes"] * 0 and opt >= max(i[0] for i in items)
         ratios.append(tensors_top / opt)
-    assert ratios and max(ratios) <= 1.5 and float(np.mean(ratios)) <= 1.2, ratios
+    assert ratios and max(ratios) <= 1.25 and float(np.mean(ratios)) <= 1.06, ratios
