@@ -130,7 +130,7 @@ class Graph:
         self._keep = []
 
     def __del__(self):
-        if getattr(self, "h", None):
+        if getattr(self, "h", None) and lib is not None:   # lib is None while the interpreter shuts down
             lib.sod2_graph_destroy(self.h)
             self.h = None
 
@@ -222,7 +222,7 @@ class Binding:
         self.n_req = n_req
 
     def __del__(self):
-        if getattr(self, "h", None):
+        if getattr(self, "h", None) and lib is not None:   # lib is None while the interpreter shuts down
             lib.sod2_binding_destroy(self.h)
             self.h = None
 
@@ -249,7 +249,7 @@ class Plan:
         self.arena_bytes = ab.value
 
     def __del__(self):
-        if getattr(self, "h", None):
+        if getattr(self, "h", None) and lib is not None:   # lib is None while the interpreter shuts down
             lib.sod2_plan_destroy(self.h)
             self.h = None
 

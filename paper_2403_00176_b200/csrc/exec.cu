@@ -11,6 +11,7 @@
 #include "attention_tcgen05.cuh"
 #include "conv_tcgen05.cuh"
 #include "conv3x3_tcgen05.cuh"
+#include "conv_stem_tcgen05.cuh"
 #include "engine.h"
 #include "gemm_tcgen05.cuh"
 #include "kernels_compact.cuh"
@@ -64,6 +65,17 @@ cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t sme
 }
 
 int64_t numel(const DimVec& d) { int64_t n = 1; for (auto v : d) n *= v; return n; }
+
+// The RGB stem has a kernel of its own (conv_stem_tcgen05.cuh): 7x7, stride 2, padding 3, 3 -> 64 channels,
+// bias, no or ReLU activation.  Decided per graph, so that the weights are prepacked in its K order.
+bool is_fused_stem(const Compiled& c, const Group& G) {
+  if (G.kind != GKind::CONV || G.w < 0 || G.res >= 0 || G.act2 || G.has_ln || (G.act != 0 && G.act != 2)) return false;
+  const Tensor& W = c.g.tensors[G.w];
+  if (W.dtype != DType::BF16 || W.S.rank != 4) return false;
+  for (int i = 0; i < 4; ++i) if (!W.S.dims[i].known() || !W.S.dims[i].e.is_const()) return false;
+  return W.S.dims[0].e.const_value() == 64 && W.S.dims[1].e.const_value() == 3 && W.S.dims[2].e.const_value() == 7 &&
+         W.S.dims[3].e.const_value() == 7 && G.stride == 2 && G.pad == 3;
+}
 
 struct Builder {
   Plan& p;
@@ -701,6 +713,50 @@ struct Builder {
     if (Cout % 8) return fail(E_UNSUPPORTED_OP, "thin-channel convolution needs Cout % 8 == 0");
     size_t pk = 0;
     for (size_t i = 0; i < c.packed_consts.size(); ++i) if (c.packed_consts[i] == G.w) pk = c.packed_off[i];
+    if (is_fused_stem(c, G)) {
+      for (int r = 0; r < p.n_req; ++r) {
+        const View &vx = p.views[G.a][r], &vo = p.views[G.out][r];
+        if (!numel(vo.dims)) continue;
+        if (!vx.contiguous()) return fail(E_UNSUPPORTED_OP, "thin-channel convolution reads an NCHW-contiguous input");
+        if (!is_channels_last(vo)) return fail(E_UNSUPPORTED_OP, "convolution output must be stored channels-last");
+        k::StemParams sp{};
+        sp.N = static_cast<int>(vx.dims[0]); sp.H = static_cast<int>(vx.dims[2]); sp.W = static_cast<int>(vx.dims[3]);
+        sp.Ho = static_cast<int>(vo.dims[2]); sp.Wo = static_cast<int>(vo.dims[3]);
+        Ptr px = ptr_of(G.a, r), po = ptr_of(G.out, r), pb = G.bias >= 0 ? ptr_of(G.bias, 0) : Ptr();
+        Ptr pw; pw.where = 5; pw.off = static_cast<int64_t>(pk);
+        const bool hb = G.bias >= 0;
+        const int act = G.act;
+        struct Cache { const void* w = nullptr; const void* o = nullptr; CUtensorMap tw, to; };
+        auto cache = std::make_shared<Cache>();
+        add(gi, 1, [=](const RunCtx& x) mutable {
+          sp.x = reinterpret_cast<const __nv_bfloat16*>(x.resolve(px));
+          sp.bias = hb ? reinterpret_cast<const __nv_bfloat16*>(x.resolve(pb)) : nullptr;
+          sp.vec_ok = (reinterpret_cast<uintptr_t>(sp.x) % 16 == 0 && sp.W % 8 == 0) ? 1 : 0;
+          sp.status = reinterpret_cast<int*>(x.arena);
+          const void* Wp = x.resolve(pw);
+          void* O = x.resolve(po);
+          if (cache->w != Wp || cache->o != O) {
+            if (!encode_bf16_kchunks(&cache->tw, Wp, 64, 192, 192, 64, 3) ||
+                !encode_bf16_nhwc(&cache->to, O, static_cast<uint64_t>(sp.N), static_cast<uint64_t>(sp.Ho), static_cast<uint64_t>(sp.Wo), 64, 128, 1, 1))
+              return cudaErrorInvalidValue;
+            cache->w = Wp; cache->o = O;
+          }
+          const long long tiles = static_cast<long long>(sp.N) * sp.Ho * ((sp.Wo + 127) / 128);
+          const dim3 gd(static_cast<unsigned>(std::min<long long>(tiles, x.plan->sm_count))), bd(k::STEM_THREADS);
+          if (act == 2) {
+            static bool once = (cudaFuncSetAttribute(k::conv_stem_bf16_tcgen05<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, k::STEM_SMEM), true);
+            (void)once;
+            launch_pdl(k::conv_stem_bf16_tcgen05<2>, gd, bd, k::STEM_SMEM, x.stream, cache->tw, cache->to, sp);
+          } else {
+            static bool once = (cudaFuncSetAttribute(k::conv_stem_bf16_tcgen05<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, k::STEM_SMEM), true);
+            (void)once;
+            launch_pdl(k::conv_stem_bf16_tcgen05<0>, gd, bd, k::STEM_SMEM, x.stream, cache->tw, cache->to, sp);
+          }
+          return cudaGetLastError();
+        });
+      }
+      return OK;
+    }
     const int K = Cin * ks * ks, Kp = (K + 63) / 64 * 64;
     for (int r = 0; r < p.n_req; ++r) {
       const View &vx = p.views[G.a][r], &vo = p.views[G.out][r];
@@ -1268,6 +1324,13 @@ Status prepack_weights(Compiled* c, void* workspace, size_t bytes, void* stream)
     if (W.S.rank == 4) {  // convolution weights [Cout, Cin, kh, kw] -> [Cout, (dy, dx, ci)]
       const int co = static_cast<int>(W.S.dims[0].e.const_value()), ci = static_cast<int>(W.S.dims[1].e.const_value());
       const int kh = static_cast<int>(W.S.dims[2].e.const_value()), kw = static_cast<int>(W.S.dims[3].e.const_value());
+      bool stem = false;
+      for (const Group& G2 : c->groups) if (G2.kind == GKind::CONV && G2.w == c->packed_consts[i] && is_fused_stem(*c, G2)) stem = true;
+      if (stem) {     // fused RGB stem: (dy, ci, dx + 1) order, 24 units of 8
+        k::reorder_stem_weights<<<48, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+            static_cast<const __nv_bfloat16*>(W.dev_ptr), reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + c->packed_off[i]));
+        continue;
+      }
       if (ci % 64) {  // thin-channel convolution (im2col path): keep the (ci, dy, dx) order, pad K with zeros
         const int K = ci * kh * kw, Kp = (K + 63) / 64 * 64;
         k::pad_rows_bf16<<<148 * 2, 256, 0, static_cast<cudaStream_t>(stream)>>>(

@@ -333,6 +333,33 @@ def test_branched_graph_planned_order_matches_default_order_and_oracle():
         assert errs and not bad, (req.syms, bad)
 
 
+def test_rgb_stem_convolution_fused_kernel_shapes():
+    # the fused 7x7 / stride 2 / 3 -> 64 stem: image widths that are (not) multiples of 8 (16-byte and
+    # element-wise patch copies), odd heights, one to three 128-pixel segments per output row, several
+    # images per request and requests of different sizes in one batch; with and without the ReLU
+    rng = np.random.default_rng(23)
+    for relu in (True, False):
+        lines = ["sym H 8 1024", "sym W 8 1024", "input x bf16 [2,3,H,W]", "const w bf16 [64,3,7,7]", "const b bf16 [64]",
+                 "node Conv x w b -> c {kernel=7 stride=2 pad=3}" if relu else "node Conv x w b -> y {kernel=7 stride=2 pad=3}"]
+        if relu:
+            lines.append("node Relu c -> y")
+        lines.append("output y")
+        ir = "\n".join(lines) + "\n"
+        consts = {"w": bf16_round((rng.standard_normal((64, 3, 7, 7)) / np.sqrt(147)).astype(np.float32)),
+                  "b": bf16_round((rng.standard_normal(64) * 0.1).astype(np.float32))}
+        shapes = [(32, 32), (30, 36), (17, 8), (224, 224), (70, 520)] if relu else [(33, 72), (64, 260)]
+        reqs = [Request({"H": h, "W": w}, {"x": bf16_round(rng.uniform(-1, 1, (2, 3, h, w)).astype(np.float32))}) for h, w in shapes]
+        wl = WL.Workload("stem", "bf16", ir, consts, ["H", "W"], ["y"], {"batch_fn": lambda j: reqs})
+        s, p, outs = run_batch(wl, reqs)
+        kinds = [s.graph.group_info(i)["kind"] for i in range(s.graph.num_groups())]
+        assert "conv" in kinds, kinds
+        assert p.plan.memory()["arena_bytes"] < 8 << 20       # the conv outputs (5.7 MB), no patch matrix (9.6 MB more)
+        for r, req in enumerate(reqs):
+            ref = O.run(ir, consts, req.inputs)["y"]
+            assert outs[r]["y"].shape == ref.shape, (req.syms, outs[r]["y"].shape, ref.shape)
+            assert O.rel_err(outs[r]["y"], ref) <= BF16_TOL, (req.syms, O.rel_err(outs[r]["y"], ref))
+
+
 # ------------------------------------------------------------------------------------------------ cfg 5
 def _check_gated(wl, reqs, n_blocks, extra_flags=0):
     s, p, outs = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE | extra_flags)
