@@ -568,6 +568,32 @@ __global__ void __launch_bounds__(256) im2col_nchw_bf16(Im2colParams p) {
   }
 }
 
+// Per-sample regrouping (Switch): stable partition of the sample ids by the gate.  One warp-sized CTA:
+// ballot + prefix popcount per chunk of 32 samples.  *count_exec = executed (the run-time symbol's
+// slot in the arena header), *count_skip = skipped; idx_exec / idx_skip = original sample ids.
+struct PartitionParams {
+  const unsigned char* gate;
+  int n;
+  int* idx_exec; int* idx_skip;    // scratch [n] each
+  long long* count_exec;           // the run-time symbol's slot in the arena header
+  long long* count_skip;
+};
+__device__ __forceinline__ void partition_by_gate(const PartitionParams& p, int lane) {
+  int ne = 0, ns = 0;
+  for (int base = 0; base < p.n; base += 32) {
+    const int i = base + lane;
+    const bool in = i < p.n;
+    const bool g = in && __ldcg(p.gate + i) != 0;
+    const unsigned be = __ballot_sync(0xffffffffu, g), bs = __ballot_sync(0xffffffffu, in && !g);
+    const unsigned lower = (1u << lane) - 1;
+    if (g) p.idx_exec[ne + __popc(be & lower)] = i;
+    else if (in) p.idx_skip[ns + __popc(bs & lower)] = i;
+    ne += __popc(be);
+    ns += __popc(bs);
+  }
+  if (lane == 0) { *p.count_exec = ne; *p.count_skip = ns; }
+}
+
 // Gate of a skip block (decision scalar): z[n] = sum_c w[c] * mean_hw x[n,:,:,c] + b, gate[n] = z[n] > 0,
 // all in fp64 from the bf16 values, so the decision does not depend on the summation order beyond 2^-53.
 // Runs after gap_partial_f64 (slab sums in scratch); one CTA per image.
@@ -580,9 +606,15 @@ struct GateParams {
   int z_bf16;
   int C, slabs;
   long long HW;
+  // ticket != nullptr: the CTA that finishes last also partitions the sample ids by the gate bits (the
+  // Switch that consumes this gate then launches nothing for it).  *ticket is zero on entry (the run
+  // clears the arena header) and is left at zero.
+  int* ticket;
+  PartitionParams part;
 };
 __global__ void __launch_bounds__(256) gate_logit_f64(GateParams p) {
   __shared__ double red[256];
+  __shared__ int last_cta;
   ptx::pdl_wait();
   ptx::pdl_launch();
   const int img = blockIdx.x;
@@ -609,36 +641,25 @@ __global__ void __launch_bounds__(256) gate_logit_f64(GateParams p) {
       if (p.z_bf16) reinterpret_cast<__nv_bfloat16*>(p.z_out)[img] = __double2bfloat16(z);
       else reinterpret_cast<float*>(p.z_out)[img] = static_cast<float>(z);
     }
+    if (p.ticket) {
+      __threadfence();
+      last_cta = atomicAdd(p.ticket, 1) == static_cast<int>(gridDim.x) - 1;
+    }
+  }
+  if (p.ticket) {
+    __syncthreads();
+    if (last_cta && threadIdx.x < 32) {
+      __threadfence();
+      partition_by_gate(p.part, threadIdx.x);
+      if (threadIdx.x == 0) *p.ticket = 0;
+    }
   }
 }
 
-// Per-sample regrouping (Switch): stable partition of the sample ids by the gate.  One warp-sized CTA:
-// ballot + prefix popcount per chunk of 32 samples.  *count_exec = executed (the run-time symbol's
-// slot in the arena header), *count_skip = skipped; idx_exec / idx_skip = original sample ids.
-struct PartitionParams {
-  const unsigned char* gate;
-  int n;
-  int* idx_exec; int* idx_skip;    // scratch [n] each
-  long long* count_exec;           // the run-time symbol's slot in the arena header
-  long long* count_skip;
-};
 __global__ void __launch_bounds__(32) gate_partition(PartitionParams p) {
   ptx::pdl_wait();
   ptx::pdl_launch();
-  const int lane = threadIdx.x;
-  int ne = 0, ns = 0;
-  for (int base = 0; base < p.n; base += 32) {
-    const int i = base + lane;
-    const bool in = i < p.n;
-    const bool g = in && p.gate[i] != 0;
-    const unsigned be = __ballot_sync(0xffffffffu, g), bs = __ballot_sync(0xffffffffu, in && !g);
-    const unsigned lower = (1u << lane) - 1;
-    if (g) p.idx_exec[ne + __popc(be & lower)] = i;
-    else if (in) p.idx_skip[ns + __popc(bs & lower)] = i;
-    ne += __popc(be);
-    ns += __popc(bs);
-  }
-  if (lane == 0) { *p.count_exec = ne; *p.count_skip = ns; }
+  partition_by_gate(p, threadIdx.x);
 }
 
 // Sample gather / scatter for Switch and Combine: whole per-sample blocks (channels-last, contiguous)

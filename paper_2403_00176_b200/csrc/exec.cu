@@ -6,6 +6,7 @@
 #include <cstring>
 #include <functional>
 #include <map>
+#include <set>
 
 #include "attention.cuh"
 #include "attention_tcgen05.cuh"
@@ -1047,6 +1048,8 @@ struct Builder {
   // persistent side storage of a Switch (index lists), found again by the Combine through the gate tensor
   std::map<int, size_t> switch_aux;   // gate tensor -> offset inside the aux region
   size_t aux_need = 0;
+  std::set<int> partition_fused;      // gate tensors whose id partition is computed by the gate kernel
+  int n_tickets = 0;
 
   // ------------------------------------------------------------------------------ gate (decision scalar)
   Status build_gate(int gi, const Group& G) {
@@ -1065,6 +1068,27 @@ struct Builder {
       Ptr px = ptr_of(G.a, r), pw = ptr_of(G.w, 0), pb = ptr_of(G.bias, 0), pg = ptr_of(G.out, r);
       Ptr pz = want_z ? ptr_of(G.out2, r) : Ptr();
       const bool zb = want_z && g.tensors[G.out2].dtype == DType::BF16;
+      // The Switch that regroups the samples by this gate needs the stable partition of the sample ids.
+      // The last CTA of the logit kernel computes it (ticket counters live in bytes 128.. of the arena
+      // header, which every run clears), so the Switch launches nothing of its own for it.
+      bool fuse_part = false;
+      size_t part_aux = 0, part_slot = 0;
+      const int ticket = n_tickets;
+      if (p.n_req == 1 && ticket < 32) {
+        for (const Group& S : c.groups) {
+          if (S.kind != GKind::SWITCH || S.gate != G.out || switch_aux.count(S.gate)) continue;
+          RtCount rc = runtime_count(S.out, 0);
+          if (!rc.rt || rc.a != 0 || rc.b != 1) break;
+          part_aux = aux_need;
+          switch_aux[S.gate] = part_aux;
+          aux_need += (static_cast<size_t>(2 * N) * 4 + 16 + 255) & ~size_t(255);
+          part_slot = rc.slot_off;
+          partition_fused.insert(S.gate);
+          fuse_part = true;
+          ++n_tickets;
+          break;
+        }
+      }
       add(gi, 2, [=](const RunCtx& x) mutable {
         gp.x = reinterpret_cast<const __nv_bfloat16*>(x.resolve(px));
         gp.partial = reinterpret_cast<double*>(x.arena + x.plan->scratch_off[0]);
@@ -1077,6 +1101,16 @@ struct Builder {
         q.z_out = want_z ? x.resolve(pz) : nullptr;
         q.z_bf16 = zb;
         q.C = gp.C; q.slabs = gp.slabs; q.HW = gp.HW;
+        if (fuse_part) {
+          char* auxp = x.arena + x.plan->scratch_off[1] + part_aux;
+          q.ticket = reinterpret_cast<int*>(x.arena + 128) + ticket;
+          q.part.gate = q.gate;
+          q.part.n = N;
+          q.part.idx_exec = reinterpret_cast<int*>(auxp);
+          q.part.idx_skip = q.part.idx_exec + N;
+          q.part.count_exec = reinterpret_cast<long long*>(x.arena + part_slot);
+          q.part.count_skip = reinterpret_cast<long long*>(auxp + 2 * N * 4);
+        }
         launch_pdl(k::gate_logit_f64, dim3(N), dim3(256), 0, x.stream, q);
         return cudaGetLastError();
       });
@@ -1094,15 +1128,19 @@ struct Builder {
     if (bytes % 16) return fail(E_UNSUPPORTED_OP, "Switch: sample size must be a multiple of 16 bytes");
     RtCount rc = runtime_count(G.out, 0);
     if (!rc.rt || rc.a != 0 || rc.b != 1) return fail(E_INTERNAL, "Switch output has no run-time count");
-    const size_t aux = aux_need;
-    switch_aux[G.gate] = aux;
-    aux_need += (static_cast<size_t>(2 * N) * 4 + 16 + 255) & ~size_t(255);
+    const bool fused = partition_fused.count(G.gate) != 0;   // the gate kernel has already partitioned the ids
+    const size_t aux = fused ? switch_aux[G.gate] : aux_need;
+    if (!fused) {
+      switch_aux[G.gate] = aux;
+      aux_need += (static_cast<size_t>(2 * N) * 4 + 16 + 255) & ~size_t(255);
+    }
     const bool indirect = c.storage[G.out].kind == Storage::INDIRECT_IN;
+    if (fused && indirect) return OK;
     Ptr px = ptr_of(G.a, 0), pg = ptr_of(G.gate, 0), pe = ptr_of(G.out, 0);
     const bool has_skip = G.out2 >= 0 && !p.views[G.out2][0].dims.empty();
     Ptr ps = has_skip ? ptr_of(G.out2, 0) : Ptr();
     const size_t slot = rc.slot_off;
-    add(gi, has_skip ? 3 : 2, [=](const RunCtx& x) {
+    add(gi, (has_skip ? 3 : 2) - (fused ? 1 : 0), [=](const RunCtx& x) {
       char* auxp = x.arena + x.plan->scratch_off[1] + aux;
       k::PartitionParams pp{};
       pp.gate = reinterpret_cast<const unsigned char*>(x.resolve(pg));
@@ -1111,7 +1149,7 @@ struct Builder {
       pp.idx_skip = pp.idx_exec + N;
       pp.count_exec = reinterpret_cast<long long*>(x.arena + slot);
       pp.count_skip = reinterpret_cast<long long*>(auxp + 2 * N * 4);
-      launch_pdl(k::gate_partition, dim3(1), dim3(32), 0, x.stream, pp);
+      if (!fused) launch_pdl(k::gate_partition, dim3(1), dim3(32), 0, x.stream, pp);
       if (indirect) return cudaGetLastError();   // the consumers read the Switch input through the id lists
       k::SampleCopyParams sc{};
       sc.src = reinterpret_cast<const uint4*>(x.resolve(px));
