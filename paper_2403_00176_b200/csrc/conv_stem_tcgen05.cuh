@@ -111,29 +111,35 @@ conv_stem_bf16_tcgen05(const __grid_constant__ CUtensorMap tmW, const __grid_con
       const int oy = static_cast<int>(rowi % p.Ho), n = static_cast<int>(rowi / p.Ho);
       const int c_first = 2 * (seg * 128) - 8;
       uint8_t* dst = sPatch + s * STEM_PATCH_BYTES;
-      for (int i = tb; i < STEM_ROWS * (STEM_PITCH / 8); i += 256) {
-        const int r = i / (STEM_PITCH / 8), ch = i % (STEM_PITCH / 8);
-        const int dy = r / 3, ci = r % 3;
-        const int iy = 2 * oy + dy - 3, c0 = c_first + ch * 8;
-        const uint32_t d = ptx::smem_u32(dst + (r * STEM_PITCH + ch * 8) * 2);
+      // warp wb takes rows wb, wb + 8, wb + 16; a lane takes 16-byte chunks lane and lane + 32 of a row
+      for (int r = tb >> 5; r < STEM_ROWS; r += 8) {
+        const int dy = r / 3, ci = r - dy * 3;
+        const int iy = 2 * oy + dy - 3;
         const bool row_in = iy >= 0 && iy < p.H;
         const __nv_bfloat16* src = p.x + ((static_cast<long long>(n) * 3 + ci) * p.H + (row_in ? iy : 0)) * p.W;
-        if (p.vec_ok) {
-          if (row_in && c0 >= 0 && c0 + 8 <= p.W) {
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src + c0) : "memory");
-          } else {
-            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(d), "r"(0u) : "memory");
-          }
-        } else {
-          uint32_t wv[4];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int ca = c0 + 2 * j, cb = ca + 1;
-            const uint32_t lo = (row_in && ca >= 0 && ca < p.W) ? static_cast<uint32_t>(__bfloat16_as_ushort(src[ca])) : 0u;
-            const uint32_t hi = (row_in && cb >= 0 && cb < p.W) ? static_cast<uint32_t>(__bfloat16_as_ushort(src[cb])) : 0u;
-            wv[j] = lo | (hi << 16);
+        for (int h = 0; h < 2; ++h) {
+          const int ch = (tb & 31) + 32 * h;
+          if (ch >= STEM_PITCH / 8) break;
+          const int c0 = c_first + ch * 8;
+          const uint32_t d = ptx::smem_u32(dst + (r * STEM_PITCH + ch * 8) * 2);
+          if (p.vec_ok) {
+            if (row_in && c0 >= 0 && c0 + 8 <= p.W) {
+              asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src + c0) : "memory");
+            } else {
+              asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(d), "r"(0u) : "memory");
+            }
+          } else {
+            uint32_t wv[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int ca = c0 + 2 * j, cb = ca + 1;
+              const uint32_t lo = (row_in && ca >= 0 && ca < p.W) ? static_cast<uint32_t>(__bfloat16_as_ushort(src[ca])) : 0u;
+              const uint32_t hi = (row_in && cb >= 0 && cb < p.W) ? static_cast<uint32_t>(__bfloat16_as_ushort(src[cb])) : 0u;
+              wv[j] = lo | (hi << 16);
+            }
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d), "r"(wv[0]), "r"(wv[1]), "r"(wv[2]), "r"(wv[3]) : "memory");
           }
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d), "r"(wv[0]), "r"(wv[1]), "r"(wv[2]), "r"(wv[3]) : "memory");
         }
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
@@ -216,11 +222,13 @@ conv_stem_bf16_tcgen05(const __grid_constant__ CUtensorMap tmW, const __grid_con
 #pragma unroll
       for (int g = 0; g < 8; ++g) {
         __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&pk[g]);
+        const float4 b0 = *reinterpret_cast<const float4*>(bias_s + g * 8), b1 = *reinterpret_cast<const float4*>(bias_s + g * 8 + 4);
+        const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int cch = g * 8 + 2 * i;
-          const float v0 = apply_act<ACT>(__uint_as_float(r[cch >> 5][cch & 31]) + bias_s[cch]);
-          const float v1 = apply_act<ACT>(__uint_as_float(r[(cch + 1) >> 5][(cch + 1) & 31]) + bias_s[cch + 1]);
+          const float v0 = apply_act<ACT>(__uint_as_float(r[cch >> 5][cch & 31]) + bb[2 * i]);
+          const float v1 = apply_act<ACT>(__uint_as_float(r[(cch + 1) >> 5][(cch + 1) & 31]) + bb[2 * i + 1]);
           oh[i] = __floats2bfloat162_rn(v0, v1);
         }
       }
