@@ -72,7 +72,7 @@ conv_stem_bf16_tcgen05(const __grid_constant__ CUtensorMap tmW, const __grid_con
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nseg = (p.Wo + 127) >> 7;
-  const long long n_tiles = static_cast<long long>(p.N) * p.Ho * nseg;
+  const int n_tiles = p.N * p.Ho * nseg;   // the host keeps it below 2^31 (64-bit divisions in the tile loop cost more than the tile)
 
   if (threadIdx.x == 0) {
     ptx::mbar_init(w_full, 1);
@@ -105,72 +105,96 @@ conv_stem_bf16_tcgen05(const __grid_constant__ CUtensorMap tmW, const __grid_con
     const int m = tb & 127, ug = tb >> 7;
     ptx::pdl_wait();
     // copy of the patch of tile t into ring slot s: rows (dy, ci), columns 2*ox0 - 8 .. 2*ox0 + 263
-    auto load_patch = [&](long long t, int s) {
-      const int seg = static_cast<int>(t % nseg);
-      const long long rowi = t / nseg;
-      const int oy = static_cast<int>(rowi % p.Ho), n = static_cast<int>(rowi / p.Ho);
-      const int c_first = 2 * (seg * 128) - 8;
-      uint8_t* dst = sPatch + s * STEM_PATCH_BYTES;
-      // warp wb takes rows wb, wb + 8, wb + 16; a lane takes 16-byte chunks lane and lane + 32 of a row
-      for (int r = tb >> 5; r < STEM_ROWS; r += 8) {
-        const int dy = r / 3, ci = r - dy * 3;
-        const int iy = 2 * oy + dy - 3;
+    // warp wb copies patch rows wb, wb + 8, wb + 16; a lane copies the 16-byte chunks lane and lane + 32
+    // of a row (34 chunks).  What does not depend on the tile is computed once.
+    const int wb = tb >> 5;
+    int row_dy[3], row_ci[3];
+    uint32_t row_dst[3];
+#pragma unroll
+    for (int j = 0; j < 3; ++j) {
+      const int r = wb + 8 * j;
+      row_dy[j] = r / 3;
+      row_ci[j] = r - row_dy[j] * 3;
+      row_dst[j] = static_cast<uint32_t>((r * STEM_PITCH + lane * 8) * 2);
+    }
+    const long long plane = static_cast<long long>(p.H) * p.W;
+    auto load_patch = [&](int t, int s) {
+      const int rowi = t / nseg, seg = t - rowi * nseg;
+      const int n = rowi / p.Ho, oy = rowi - n * p.Ho;
+      const int c0a = 2 * (seg * 128) - 8 + lane * 8, c0b = c0a + 256;
+      const uint32_t dst = ptx::smem_u32(sPatch + s * STEM_PATCH_BYTES);
+      const __nv_bfloat16* img = p.x + static_cast<long long>(n) * 3 * plane;
+#pragma unroll
+      for (int j = 0; j < 3; ++j) {
+        if (wb + 8 * j >= STEM_ROWS) break;
+        const int iy = 2 * oy + row_dy[j] - 3;
         const bool row_in = iy >= 0 && iy < p.H;
-        const __nv_bfloat16* src = p.x + ((static_cast<long long>(n) * 3 + ci) * p.H + (row_in ? iy : 0)) * p.W;
+        const __nv_bfloat16* src = img + row_ci[j] * plane + static_cast<long long>(row_in ? iy : 0) * p.W;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-          const int ch = (tb & 31) + 32 * h;
-          if (ch >= STEM_PITCH / 8) break;
-          const int c0 = c_first + ch * 8;
-          const uint32_t d = ptx::smem_u32(dst + (r * STEM_PITCH + ch * 8) * 2);
+          if (h == 1 && lane >= STEM_PITCH / 8 - 32) break;
+          const int c0 = h ? c0b : c0a;
+          const uint32_t d = dst + row_dst[j] + h * 512;
           if (p.vec_ok) {
             if (row_in && c0 >= 0 && c0 + 8 <= p.W) {
-              asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src + c0) : "memory");
+              asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src + c0));
             } else {
-              asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(d), "r"(0u) : "memory");
+              asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(d), "r"(0u));
             }
           } else {
             uint32_t wv[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const int ca = c0 + 2 * j, cb = ca + 1;
+            for (int q2 = 0; q2 < 4; ++q2) {
+              const int ca = c0 + 2 * q2, cb = ca + 1;
               const uint32_t lo = (row_in && ca >= 0 && ca < p.W) ? static_cast<uint32_t>(__bfloat16_as_ushort(src[ca])) : 0u;
               const uint32_t hi = (row_in && cb >= 0 && cb < p.W) ? static_cast<uint32_t>(__bfloat16_as_ushort(src[cb])) : 0u;
-              wv[j] = lo | (hi << 16);
+              wv[q2] = lo | (hi << 16);
             }
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d), "r"(wv[0]), "r"(wv[1]), "r"(wv[2]), "r"(wv[3]) : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d), "r"(wv[0]), "r"(wv[1]), "r"(wv[2]), "r"(wv[3]));
           }
         }
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    const long long t0 = blockIdx.x, step = gridDim.x;
+    const int t0 = blockIdx.x, step = gridDim.x;
     if (t0 < n_tiles) load_patch(t0, 0); else asm volatile("cp.async.commit_group;" ::: "memory");
     if (t0 + step < n_tiles) load_patch(t0 + step, 1); else asm volatile("cp.async.commit_group;" ::: "memory");
     int it = 0;
-    for (long long t = t0; t < n_tiles; t += step, ++it) {
+    for (int t = t0; t < n_tiles; t += step, ++it) {
       // this thread's copies for tile `it` have landed (one newer group may be in flight); after the
       // barrier so have everyone's, and every builder has finished reading the slot of tile it - 1
       asm volatile("cp.async.wait_group 1;" ::: "memory");
       asm volatile("bar.sync 2, 256;" ::: "memory");
+      if (tb == 0) { SOD2_TRACE(0, 10) }
       if (t + 2 * step < n_tiles) load_patch(t + 2 * step, (it + 2) % 3); else asm volatile("cp.async.commit_group;" ::: "memory");
       const int buf = it & 1;
       if (it >= 2) ptx::mbar_wait_warp(&a_free[buf], ((it >> 1) - 1) & 1, dead);
+      if (tb == 0) { SOD2_TRACE(0, 20) }
       const uint8_t* patch = sPatch + (it % 3) * STEM_PATCH_BYTES;
       uint8_t* arow = sA + buf * STEM_A_BYTES + m * 128;
+      // all loads first, then the stores: patch and A live in the same array, so the compiler would keep
+      // every store ahead of the next unit's loads
+      uint4 v[12];
 #pragma unroll
       for (int i = 0; i < 12; ++i) {
         const int u = ug + 2 * i;                       // unit = patch row (dy, ci); 21..23 are padding
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        v[i] = make_uint4(0u, 0u, 0u, 0u);
         if (u < STEM_ROWS) {
-          const uint32_t* src = reinterpret_cast<const uint32_t*>(patch + (u * STEM_PITCH + 2 * m + 4) * 2);
-          v = make_uint4(src[0] & 0xffff0000u, src[1], src[2], src[3]);   // dx' = 0 has no tap
+          const uint32_t sa = ptx::smem_u32(patch + (u * STEM_PITCH + 2 * m + 4) * 2);
+          asm volatile("ld.shared.b32 %0, [%4];\n\tld.shared.b32 %1, [%4+4];\n\tld.shared.b32 %2, [%4+8];\n\tld.shared.b32 %3, [%4+12];"
+                       : "=r"(v[i].x), "=r"(v[i].y), "=r"(v[i].z), "=r"(v[i].w) : "r"(sa));
+          v[i].x &= 0xffff0000u;                        // dx' = 0 has no tap
         }
-        *reinterpret_cast<uint4*>(arow + (u >> 3) * (128 * 128) + (((u & 7) ^ (m & 7)) << 4)) = v;
+      }
+#pragma unroll
+      for (int i = 0; i < 12; ++i) {
+        const int u = ug + 2 * i;
+        *reinterpret_cast<uint4*>(arow + (u >> 3) * (128 * 128) + (((u & 7) ^ (m & 7)) << 4)) = v[i];
       }
       ptx::fence_proxy_async();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&a_full[buf]);
+      if (tb == 0) { SOD2_TRACE(0, 30) }
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
   } else if (warp == 13) {
@@ -180,10 +204,12 @@ conv_stem_bf16_tcgen05(const __grid_constant__ CUtensorMap tmW, const __grid_con
       ptx::mbar_wait(w_full, 0, dead);
       const uint32_t aW = ptx::smem_u32(sW);
       int it = 0;
-      for (long long t = blockIdx.x; t < n_tiles; t += gridDim.x, ++it) {
+      for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++it) {
         const int b = it & 1;
         ptx::mbar_wait(&a_full[b], (it >> 1) & 1, dead);
+        SOD2_TRACE(1, 40)
         if (it >= 2) ptx::mbar_wait(&acc_free[b], ((it >> 1) - 1) & 1, dead);
+        SOD2_TRACE(1, 41)
         ptx::tc_fence_after();
         const uint32_t aA = ptx::smem_u32(sA + b * STEM_A_BYTES);
 #pragma unroll
@@ -194,6 +220,7 @@ conv_stem_bf16_tcgen05(const __grid_constant__ CUtensorMap tmW, const __grid_con
         }
         ptx::mma_commit(&a_free[b]);
         ptx::mma_commit(&acc_full[b]);
+        SOD2_TRACE(1, 42)
       }
     }
   } else {
@@ -203,13 +230,13 @@ conv_stem_bf16_tcgen05(const __grid_constant__ CUtensorMap tmW, const __grid_con
     const bool leader = threadIdx.x == 9 * 32;
     ptx::pdl_wait();
     int it = 0;
-    for (long long t = blockIdx.x; t < n_tiles; t += gridDim.x, ++it) {
+    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++it) {
       const int b = it & 1;
-      const int seg = static_cast<int>(t % nseg);
-      const long long rowi = t / nseg;
-      const int oy = static_cast<int>(rowi % p.Ho), n = static_cast<int>(rowi / p.Ho);
+      const int rowi = t / nseg, seg = t - rowi * nseg;
+      const int n = rowi / p.Ho, oy = rowi - n * p.Ho;
       ptx::mbar_wait_warp(&acc_full[b], (it >> 1) & 1, dead);
       ptx::tc_fence_after();
+      if (leader) { SOD2_TRACE(2, 50) }
       uint32_t r[2][32];
       const uint32_t taddr = tmem + (static_cast<uint32_t>(q * 32) << 16) + b * 64;
       ptx::tmem_ld32(taddr, r[0]);
@@ -218,6 +245,7 @@ conv_stem_bf16_tcgen05(const __grid_constant__ CUtensorMap tmW, const __grid_con
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&acc_free[b]);
+      if (leader) { SOD2_TRACE(2, 51) }
       uint4 pk[8];
 #pragma unroll
       for (int g = 0; g < 8; ++g) {
@@ -243,6 +271,7 @@ conv_stem_bf16_tcgen05(const __grid_constant__ CUtensorMap tmW, const __grid_con
       if (leader) {
         tma_store_4d(&tmOut, sOut + b * STEM_OUT_BYTES, 0, seg * 128, oy, n);
         bulk_commit();
+        SOD2_TRACE(2, 52)
       }
     }
     if (leader) bulk_wait_read0();

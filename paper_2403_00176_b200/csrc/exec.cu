@@ -743,6 +743,7 @@ struct Builder {
             cache->w = Wp; cache->o = O;
           }
           const long long tiles = static_cast<long long>(sp.N) * sp.Ho * ((sp.Wo + 127) / 128);
+          if (tiles >= (1ll << 31)) return cudaErrorInvalidValue;
           const dim3 gd(static_cast<unsigned>(std::min<long long>(tiles, x.plan->sm_count))), bd(k::STEM_THREADS);
           if (act == 2) {
             static bool once = (cudaFuncSetAttribute(k::conv_stem_bf16_tcgen05<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, k::STEM_SMEM), true);
