@@ -274,29 +274,41 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ Conv3Batch B, const __grid_con
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(&tmem_empty[acc]);
         }
+        // bias and activation before the wait for the staging buffer; then the residual loads together, the
+        // arithmetic, and the stores together (loads and stores of one buffer are not reordered by the compiler)
+        const float* bp = bias_t + ps * 64 + half * 32;
+        float v[32];
+        if (live) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = apply_act<ACT>(__uint_as_float(r[i]) + bp[i]);
+        }
         ptx::mbar_wait_warp(&res_full[bsel], (u / NSB) & 1, dead);
         if (live) {
-          const float* bp = bias_t + ps * 64 + half * 32;
+          uint4 pk[4];
+          if constexpr (HASRES) {
+            uint4 rv[4];
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            float v[8];
+            for (int g = 0; g < 4; ++g) rv[g] = *reinterpret_cast<const uint4*>(obase + (((half * 4 + g) ^ (row & 7)) << 4));
 #pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = apply_act<ACT>(__uint_as_float(r[g * 8 + i]) + bp[g * 8 + i]);
-            uint4* slot = reinterpret_cast<uint4*>(obase + (((half * 4 + g) ^ (row & 7)) << 4));
-            if constexpr (HASRES) {
-              const uint4 rv = *slot;
-              const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&rv);
+            for (int g = 0; g < 4; ++g) {
+              const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&rv[g]);
+              __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&pk[g]);
 #pragma unroll
-              for (int i = 0; i < 4; ++i) { const float2 f = __bfloat1622float2(h[i]); v[2 * i] += f.x; v[2 * i + 1] += f.y; }
-#pragma unroll
-              for (int i = 0; i < 8; ++i) v[i] = fmaxf(v[i], relu2_floor);
+              for (int i = 0; i < 4; ++i) {
+                const float2 f = __bfloat1622float2(h[i]);
+                oh[i] = __floats2bfloat162_rn(fmaxf(v[g * 8 + 2 * i] + f.x, relu2_floor), fmaxf(v[g * 8 + 2 * i + 1] + f.y, relu2_floor));
+              }
             }
-            uint4 pk;
-            __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&pk);
+          } else {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) oh[i] = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
-            *slot = pk;
+            for (int g = 0; g < 4; ++g) {
+              __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&pk[g]);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) oh[i] = __floats2bfloat162_rn(v[g * 8 + 2 * i], v[g * 8 + 2 * i + 1]);
+            }
           }
+#pragma unroll
+          for (int g = 0; g < 4; ++g) *reinterpret_cast<uint4*>(obase + (((half * 4 + g) ^ (row & 7)) << 4)) = pk[g];
         }
         ptx::fence_proxy_async();
         __syncwarp();

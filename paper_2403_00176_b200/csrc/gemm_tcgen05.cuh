@@ -381,12 +381,15 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
         }
         ptx::mbar_wait_warp(&buf_ready[bsel], (u / NSB) & 1, dead);
+        if constexpr (RES) {
+          // the four residual loads first, then the arithmetic, then the four stores: loads and stores go
+          // to the same buffer, so interleaved the compiler keeps each load behind the previous store
+          uint4 rv[4];
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          uint4* slot = reinterpret_cast<uint4*>(obase + (((half * 4 + g) ^ (row & 7)) << 4));
-          if constexpr (RES) {
-            const uint4 rv = *slot;
-            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&rv);
+          for (int g = 0; g < 4; ++g) rv[g] = *reinterpret_cast<const uint4*>(obase + (((half * 4 + g) ^ (row & 7)) << 4));
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&rv[g]);
             __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&pk[g]);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -394,8 +397,9 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               oh[i] = __floats2bfloat162_rn(fmaxf(v[g * 8 + 2 * i] + f.x, relu2_floor), fmaxf(v[g * 8 + 2 * i + 1] + f.y, relu2_floor));
             }
           }
-          *slot = pk[g];
         }
+#pragma unroll
+        for (int g = 0; g < 4; ++g) *reinterpret_cast<uint4*>(obase + (((half * 4 + g) ^ (row & 7)) << 4)) = pk[g];
         ptx::fence_proxy_async();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&buf_filled[bsel]);
