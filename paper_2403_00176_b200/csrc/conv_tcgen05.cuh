@@ -421,13 +421,25 @@ struct GapParams {
   int C, slabs;
   long long HW;
 };
-__global__ void __launch_bounds__(256) gap_partial_f64(GapParams p) {
+// Up to GAP_MAX_SEG tensors (the requests of a batch) pooled by one launch: blockIdx.z walks the images of
+// all segments, blockIdx.y the pixel slabs (CTAs past a segment's slab count exit).
+constexpr int GAP_MAX_SEG = 8;
+struct GapBatch {
+  int n_seg;
+  int img_start[GAP_MAX_SEG + 1];
+  GapParams seg[GAP_MAX_SEG];
+};
+__global__ void __launch_bounds__(256) gap_partial_f64(const __grid_constant__ GapBatch B) {
   // every thread owns 8 channels (one 16-byte load) of a pixel; C/8 threads cover a pixel, the
   // remaining factor of the CTA walks pixels; fp64 partial sums, fixed-order reduction in shared memory
   __shared__ double part[256][8];
   ptx::pdl_wait();
   ptx::pdl_launch();
-  const long long img = blockIdx.z;
+  int si = 0;
+  while (si + 1 < B.n_seg && static_cast<int>(blockIdx.z) >= B.img_start[si + 1]) ++si;
+  const GapParams& p = B.seg[si];
+  if (static_cast<int>(blockIdx.y) >= p.slabs) return;
+  const long long img = static_cast<int>(blockIdx.z) - B.img_start[si];
   const int tpp = (p.C + 7) >> 3;                 // threads per pixel (C <= 2048)
   const int ppi = 256 / tpp;                      // pixels per CTA iteration
   const int cg = threadIdx.x % tpp, pg = threadIdx.x / tpp;
@@ -473,28 +485,31 @@ __global__ void __launch_bounds__(256) gap_partial_f64(GapParams p) {
     if (cg2 * 8 + i < p.C) p.partial[(img * p.slabs + blockIdx.y) * p.C + cg2 * 8 + i] = s;
   }
 }
-__global__ void __launch_bounds__(256) gap_final_f64(GapParams p, int n_img) {
-  // 32 channels x 8 slab lanes per CTA: lane g sums slabs g, g+8, ... in order, then the 8 lane sums
-  // are added in order: a fixed summation tree, so the result is deterministic
-  __shared__ double part[8][32];
+__global__ void __launch_bounds__(256) gap_final_f64(const __grid_constant__ GapBatch B) {
+  // 8 channels x 32 slab lanes per CTA (blockIdx.y = segment): lane g sums slabs g, g+32, ... in order,
+  // then the 32 lane sums are added in order: a fixed summation tree, so the result is deterministic
+  __shared__ double part[32][8];
   ptx::pdl_wait();
   ptx::pdl_launch();
-  const int cl = threadIdx.x & 31, g = threadIdx.x >> 5;
-  const long long i = static_cast<long long>(blockIdx.x) * 32 + cl;     // flat (img, c)
+  const GapParams& p = B.seg[blockIdx.y];
+  const int n_img = B.img_start[blockIdx.y + 1] - B.img_start[blockIdx.y];
+  const int cl = threadIdx.x & 7, g = threadIdx.x >> 3;
+  const long long i = static_cast<long long>(blockIdx.x) * 8 + cl;     // flat (img, c)
+  if (static_cast<long long>(blockIdx.x) * 8 >= static_cast<long long>(n_img) * p.C) return;
   const bool ok = i < static_cast<long long>(n_img) * p.C;
   const long long img = ok ? i / p.C : 0;
   const int c = ok ? static_cast<int>(i % p.C) : 0;
   double acc = 0.0;
   if (ok) {
-#pragma unroll 8
-    for (int s = g; s < p.slabs; s += 8) acc += p.partial[(img * p.slabs + s) * p.C + c];
+#pragma unroll 4
+    for (int s = g; s < p.slabs; s += 32) acc += p.partial[(img * p.slabs + s) * p.C + c];
   }
   part[g][cl] = acc;
   __syncthreads();
   if (g == 0 && ok) {
     double t = 0.0;
 #pragma unroll
-    for (int k2 = 0; k2 < 8; ++k2) t += part[k2][cl];
+    for (int k2 = 0; k2 < 32; ++k2) t += part[k2][cl];
     const double mean = t / static_cast<double>(p.HW);
     if (p.out_f64) p.out_f64[i] = mean;
     if (p.out) {

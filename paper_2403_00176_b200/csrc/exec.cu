@@ -1093,7 +1093,9 @@ struct Builder {
       add(gi, 2, [=](const RunCtx& x) mutable {
         gp.x = reinterpret_cast<const __nv_bfloat16*>(x.resolve(px));
         gp.partial = reinterpret_cast<double*>(x.arena + x.plan->scratch_off[0]);
-        launch_pdl(k::gap_partial_f64, dim3(1, gp.slabs, N), dim3(256), 0, x.stream, gp);
+        k::GapBatch gb{};
+        gb.n_seg = 1; gb.img_start[0] = 0; gb.img_start[1] = N; gb.seg[0] = gp;
+        launch_pdl(k::gap_partial_f64, dim3(1, gp.slabs, N), dim3(256), 0, x.stream, gb);
         k::GateParams q{};
         q.partial = gp.partial;
         q.w = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pw));
@@ -1231,25 +1233,43 @@ struct Builder {
     const Tensor& X = g.tensors[G.a];
     const Tensor& O = g.tensors[G.out];
     if (X.dtype != DType::BF16) return fail(E_UNSUPPORTED_OP, "global average pool is bf16 only");
-    for (int r = 0; r < p.n_req; ++r) {
-      const View& vx = p.views[G.a][r];
-      if (!numel(vx.dims)) continue;
-      if (!is_channels_last(vx)) return fail(E_UNSUPPORTED_OP, "global average pool reads channels-last storage");
-      k::GapParams gp{};
-      gp.C = static_cast<int>(vx.dims[1]);
-      gp.HW = vx.dims[2] * vx.dims[3];
-      gp.slabs = static_cast<int>(std::max<long long>(1, std::min<long long>(592, gp.HW / (vx.dims[0] >= 16 ? 16 : 128))));
-      gp.out_bf16 = O.dtype == DType::BF16;
-      const int N = static_cast<int>(vx.dims[0]);
-      scratch_need = std::max(scratch_need, static_cast<size_t>(N) * gp.slabs * gp.C * 8);
-      Ptr px = ptr_of(G.a, r), po = ptr_of(G.out, r);
+    // the requests of a batch are pooled together, up to GAP_MAX_SEG per launch pair
+    for (int r0 = 0; r0 < p.n_req; r0 += k::GAP_MAX_SEG) {
+      k::GapBatch gb{};
+      std::vector<Ptr> px, po;
+      std::vector<size_t> poff;
+      size_t part_bytes = 0;
+      int max_slabs = 1, max_nc = 0;
+      for (int r = r0; r < std::min(p.n_req, r0 + k::GAP_MAX_SEG); ++r) {
+        const View& vx = p.views[G.a][r];
+        if (!numel(vx.dims)) continue;
+        if (!is_channels_last(vx)) return fail(E_UNSUPPORTED_OP, "global average pool reads channels-last storage");
+        k::GapParams gp{};
+        gp.C = static_cast<int>(vx.dims[1]);
+        gp.HW = vx.dims[2] * vx.dims[3];
+        gp.slabs = static_cast<int>(std::max<long long>(1, std::min<long long>(592, gp.HW / (vx.dims[0] >= 16 ? 16 : 128))));
+        gp.out_bf16 = O.dtype == DType::BF16;
+        const int N = static_cast<int>(vx.dims[0]);
+        const int si = gb.n_seg++;
+        gb.img_start[si + 1] = gb.img_start[si] + N;
+        gb.seg[si] = gp;
+        px.push_back(ptr_of(G.a, r)); po.push_back(ptr_of(G.out, r)); poff.push_back(part_bytes);
+        part_bytes += static_cast<size_t>(N) * gp.slabs * gp.C * 8;
+        max_slabs = std::max(max_slabs, gp.slabs);
+        max_nc = std::max(max_nc, N * gp.C);
+      }
+      if (!gb.n_seg) continue;
+      scratch_need = std::max(scratch_need, part_bytes);
+      const int n_img = gb.img_start[gb.n_seg];
       add(gi, 2, [=](const RunCtx& x) mutable {
-        gp.x = reinterpret_cast<const __nv_bfloat16*>(x.resolve(px));
-        gp.partial = reinterpret_cast<double*>(x.arena + x.plan->scratch_off[0]);
-        gp.out = x.resolve(po);
-        gp.out_f64 = nullptr;
-        launch_pdl(k::gap_partial_f64, dim3(1, gp.slabs, N), dim3(256), 0, x.stream, gp);
-        launch_pdl(k::gap_final_f64, dim3((N * gp.C + 31) / 32), dim3(256), 0, x.stream, gp, N);
+        for (int si = 0; si < gb.n_seg; ++si) {
+          gb.seg[si].x = reinterpret_cast<const __nv_bfloat16*>(x.resolve(px[si]));
+          gb.seg[si].partial = reinterpret_cast<double*>(x.arena + x.plan->scratch_off[0] + poff[si]);
+          gb.seg[si].out = x.resolve(po[si]);
+          gb.seg[si].out_f64 = nullptr;
+        }
+        launch_pdl(k::gap_partial_f64, dim3(1, max_slabs, n_img), dim3(256), 0, x.stream, gb);
+        launch_pdl(k::gap_final_f64, dim3((max_nc + 7) / 8, gb.n_seg), dim3(256), 0, x.stream, gb);
         return cudaGetLastError();
       });
     }
