@@ -1,15 +1,21 @@
 // Fused attention group on tcgen05 / TMEM for packed variable-length requests, head dim 64:
 //   O = softmax(Q K^T * scale) V  per (request, head), bf16 in / fp32 accumulate / bf16 out.
 // The score and probability tensors never reach global memory (the fusion argument of Section 4.2).
-// One CTA owns 128 query rows of one (request, head) and walks the request's keys in blocks of 64:
-//   S_j = Q K_j^T          tcgen05.mma, M=128, N=64, K=64; Q and K_j are K-major TMA tiles
-//   P_j = exp2(S_j*c - m)  softmax threads: two threads per query row read the halves of its row of
-//                          S_j from TMEM, write P_j as bf16 into a swizzled tile
-//   O  += P_j V_j          tcgen05.mma, M=128, N=64, K=64; V_j is the natural [key, d] tile, used
+// One CTA owns 128 query rows of one (request, head) and walks the request's keys in blocks of 128:
+//   S_j = Q K_j^T          tcgen05.mma, M=128, N=128, K=64; Q and K_j are K-major TMA tiles
+//   P_j = exp2(S_j*c - m)  softmax threads: two threads per query row, each owns 64 of the block's 128
+//                          score columns and reads them from TMEM in two 32-column halves, twice: once for
+//                          the row maximum, once for the exponentials (a TMEM read is cheaper than holding
+//                          64 scores in registers at two CTAs per SM); P_j goes as bf16 into two swizzled
+//                          [128 x 64] tiles
+//   O  += P_j V_j          tcgen05.mma, M=128, N=64, K=128; V_j is the natural [key, d] tile, used
 //                          as an MN-major B operand
 //   (O *= corr)            only when a block's maximum moves the exponent reference by more than 2^8
-// S is double buffered in TMEM, O accumulates there (3 x 64 columns), P_j, K_j, V_j in shared memory, so the
-// tensor pipe, the softmax warps and TMA overlap inside a CTA; two CTAs share an SM.
+// A block of 128 keys halves the number of hand-overs per key (barrier round trips, the row-maximum
+// exchange, the P hand-over cost about as much as the exponentials of 64 keys).  S (128 columns) and O
+// (64 columns) live in TMEM; S is single buffered: the softmax threads release it after their last read,
+// about half way through the block, and the next S = Q K^T runs under the second half of the
+// exponentials.  K and P are single buffered, V double buffered; two CTAs share an SM.
 // Q, K, V are 2-D tensor maps over the packed [tokens, row stride] buffers; a tile that runs past a
 // request's rows reads the next request's rows (finite data) or zeros past the end of the buffer, and
 // those keys are masked to -inf before the softmax; query rows past the request are never written.
@@ -44,10 +50,11 @@ struct AtcParams {
   AtcReq r[ATC_MAX_REQ];
 };
 
+constexpr int ATC_KB = 128;               // keys per block
 constexpr int ATC_Q_BYTES = 128 * 128;    // 128 rows x 64 bf16
-constexpr int ATC_KV_BYTES = 64 * 128;    // 64 keys x 64 bf16
-constexpr int ATC_P_BYTES = 128 * 128;    // 128 rows x 64 keys bf16
-constexpr int ATC_SMEM = ATC_Q_BYTES + 4 * ATC_KV_BYTES + 2 * ATC_P_BYTES + 2048 /*row maxima*/ + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int ATC_KV_BYTES = ATC_KB * 128;   // 128 keys x 64 bf16
+constexpr int ATC_P_BYTES = 2 * 128 * 128;   // 128 rows x 128 keys bf16: two [128 x 64] chunks
+constexpr int ATC_SMEM = ATC_Q_BYTES + 3 * ATC_KV_BYTES + ATC_P_BYTES + 2048 /*row maxima*/ + 1024 /*align*/ + 256 /*barriers*/;
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
@@ -61,19 +68,19 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sQ = base;
-  uint8_t* sK = sQ + ATC_Q_BYTES;           // [2]
-  uint8_t* sV = sK + 2 * ATC_KV_BYTES;      // [2]
-  uint8_t* sP = sV + 2 * ATC_KV_BYTES;      // [2]
-  float* xmax = reinterpret_cast<float*>(sP + 2 * ATC_P_BYTES);   // [block parity][column half][row]
+  uint8_t* sK = sQ + ATC_Q_BYTES;
+  uint8_t* sV = sK + ATC_KV_BYTES;          // [2]
+  uint8_t* sP = sV + 2 * ATC_KV_BYTES;
+  float* xmax = reinterpret_cast<float*>(sP + ATC_P_BYTES);   // [block parity][column half][row]
   uint64_t* bars = reinterpret_cast<uint64_t*>(xmax + 512);
   uint64_t* q_full = bars;            // 1
-  uint64_t* k_full = bars + 1;        // [2] K_j landed
-  uint64_t* v_full = bars + 3;        // [2] V_j landed
-  uint64_t* s_full = bars + 5;        // [2] S_j done (also: K stage free)
-  uint64_t* s_free = bars + 7;        // [2] softmax warps have read S_j
-  uint64_t* p_full = bars + 9;        // [2] softmax warps have written P_j
-  uint64_t* o_full = bars + 11;       // [2] O_j done (also: V stage and P buffer free)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
+  uint64_t* k_full = bars + 1;        // K_j landed (one phase per block)
+  uint64_t* v_full = bars + 2;        // [2] V_j landed
+  uint64_t* s_full = bars + 4;        // S_j done (also: the K buffer is free)
+  uint64_t* s_free = bars + 5;        // softmax warps have read S_j for the last time
+  uint64_t* p_full = bars + 6;        // softmax warps have written P_j
+  uint64_t* o_full = bars + 7;        // [2] O_j done (also: V stage j & 1 and the P buffer are free)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 9);
   volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -84,15 +91,12 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   const AtcReq& R = p.r[ri];
   const int L = R.L;
   const int q0 = (tile - p.tile_start[ri]) * 128;
-  const int nkv = (L + 63) >> 6;
+  const int nkv = (L + ATC_KB - 1) / ATC_KB;
 
   if (threadIdx.x == 0) {
     ptx::mbar_init(q_full, 1);
-    for (int b = 0; b < 2; ++b) {
-      ptx::mbar_init(&k_full[b], 1); ptx::mbar_init(&v_full[b], 1);
-      ptx::mbar_init(&s_full[b], 1); ptx::mbar_init(&s_free[b], 8);
-      ptx::mbar_init(&p_full[b], 8); ptx::mbar_init(&o_full[b], 1);
-    }
+    ptx::mbar_init(k_full, 1); ptx::mbar_init(s_full, 1); ptx::mbar_init(s_free, 8); ptx::mbar_init(p_full, 8);
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&v_full[b], 1); ptx::mbar_init(&o_full[b], 1); }
     *dead = 0;
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
@@ -116,32 +120,29 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       ptx::tma_load_2d(sQ, &tmQ, p.q_col + head * p.q_hs, R.q_row + q0, q_full);
       for (int j = 0; j < nkv; ++j) {
         const int b = j & 1;
-        if (j >= 2) ptx::mbar_wait(&s_full[b], ((j >> 1) - 1) & 1, dead);    // S_{j-2} done: K stage free
-        ptx::mbar_expect_tx(&k_full[b], ATC_KV_BYTES);
-        ptx::tma_load_2d(sK + b * ATC_KV_BYTES, &tmK, p.k_col + head * p.k_hs, R.k_row + j * 64, &k_full[b]);
+        if (j >= 1) ptx::mbar_wait(s_full, (j - 1) & 1, dead);               // S_{j-1} done: the K buffer is free
+        ptx::mbar_expect_tx(k_full, ATC_KV_BYTES);
+        ptx::tma_load_2d(sK, &tmK, p.k_col + head * p.k_hs, R.k_row + j * ATC_KB, k_full);
         if (j >= 2) ptx::mbar_wait(&o_full[b], ((j >> 1) - 1) & 1, dead);    // O_{j-2} done: V stage free
         ptx::mbar_expect_tx(&v_full[b], ATC_KV_BYTES);
-        ptx::tma_load_2d(sV + b * ATC_KV_BYTES, &tmV, p.v_col + head * p.v_hs, R.v_row + j * 64, &v_full[b]);
+        ptx::tma_load_2d(sV + b * ATC_KV_BYTES, &tmV, p.v_col + head * p.v_hs, R.v_row + j * ATC_KB, &v_full[b]);
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
       // ---- S issuer: S_j = Q K_j^T.  A thread that waits on a barrier between MMAs stalls for a few
       // hundred cycles, so the two products get a thread each and one commit per block: "S_j done"
-      // both publishes S_j and frees the K stage.
-      constexpr uint32_t idesc_qk = ptx::idesc_bf16(128, 64);
-      const uint32_t aQ = ptx::smem_u32(sQ);
+      // both publishes S_j and frees the K buffer.
+      constexpr uint32_t idesc_qk = ptx::idesc_bf16(128, ATC_KB);
+      const uint64_t dQ = ptx::smem_desc_sw128(ptx::smem_u32(sQ)), dK = ptx::smem_desc_sw128(ptx::smem_u32(sK));
       ptx::mbar_wait(q_full, 0, dead);
       for (int j = 0; j < nkv; ++j) {
-        const int b = j & 1;
-        ptx::mbar_wait(&k_full[b], (j >> 1) & 1, dead);
-        if (j >= 2) ptx::mbar_wait(&s_free[b], ((j >> 1) - 1) & 1, dead);
+        ptx::mbar_wait(k_full, j & 1, dead);
+        if (j >= 1) ptx::mbar_wait(s_free, (j - 1) & 1, dead);
         ptx::tc_fence_after();
-        const uint32_t aK = ptx::smem_u32(sK + b * ATC_KV_BYTES);
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk)
-          ptx::mma_bf16(tmem + b * 64, ptx::smem_desc_sw128(aQ) + 2 * kk, ptx::smem_desc_sw128(aK) + 2 * kk, idesc_qk, kk != 0);
-        ptx::mma_commit(&s_full[b]);
+        for (int kk = 0; kk < 4; ++kk) ptx::mma_bf16(tmem, dQ + 2 * kk, dK + 2 * kk, idesc_qk, kk != 0);
+        ptx::mma_commit(s_full);
         SOD2_TRACE(1, 10 + j)
       }
     }
@@ -151,15 +152,16 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       // the V stage and the P buffer.  The softmax warps rescale O (rarely) before they hand over P_j,
       // so the accumulator needs no barrier of its own.
       constexpr uint32_t idesc_pv = ptx::idesc_bf16(128, 64) | (1u << 16);   // B (= V tile) is MN-major
+      const uint32_t aP = ptx::smem_u32(sP);
       for (int i = 0; i < nkv; ++i) {
         const int b = i & 1;
         ptx::mbar_wait(&v_full[b], (i >> 1) & 1, dead);
-        ptx::mbar_wait(&p_full[b], (i >> 1) & 1, dead);
+        ptx::mbar_wait(p_full, i & 1, dead);
         ptx::tc_fence_after();
-        const uint32_t aP = ptx::smem_u32(sP + b * ATC_P_BYTES), aV = ptx::smem_u32(sV + b * ATC_KV_BYTES);
+        const uint32_t aV = ptx::smem_u32(sV + b * ATC_KV_BYTES);
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk)   // 16 keys per step: 32 B along P's rows, 16 rows (2048 B) down V
-          ptx::mma_bf16(tmem + 128, ptx::smem_desc_sw128(aP) + 2 * kk, ptx::smem_desc_sw128(aV + kk * 2048), idesc_pv, (i | kk) != 0);
+        for (int kk = 0; kk < 8; ++kk)   // 16 keys per step: 32 B along P's rows (chunk kk / 4), 16 rows (2048 B) down V
+          ptx::mma_bf16(tmem + 128, ptx::smem_desc_sw128(aP + (kk >> 2) * (128 * 128)) + 2 * (kk & 3), ptx::smem_desc_sw128(aV + kk * 2048), idesc_pv, (i | kk) != 0);
         ptx::mma_commit(&o_full[b]);
         SOD2_TRACE(1, 20 + i)
       }
@@ -183,33 +185,41 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     float m = -INFINITY, l = 0.f;
     const float c = p.scale_log2e;
     const uint32_t o_addr = tmem + lane_base + 128 + hh * 32;
+    const uint32_t s_addr = tmem + lane_base + hh * 64;      // this thread's 64 score columns of the block
     for (int j = 0; j < nkv; ++j) {
       const int b = j & 1;
-      ptx::mbar_wait_warp(&s_full[b], (j >> 1) & 1, dead);
+      ptx::mbar_wait_warp(s_full, j & 1, dead);
       ptx::tc_fence_after();
       if (tracer) { SOD2_TRACE(2, 30 + j) }
-      uint32_t s[32];
-      ptx::tmem_ld32(tmem + lane_base + b * 64 + hh * 32, s);
-      ptx::tmem_ld_wait();
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&s_free[b]);
-      // partial row maximum on the raw scores (the scale is positive), exchanged with the row's other thread
-      const int valid = L - j * 64 - hh * 32;      // keys of this thread's half inside the request
-      if (valid < 32) {
+      const int valid = L - j * ATC_KB - hh * 64;     // keys of this thread's 64 columns inside the request
+      // ---- pass 1: partial row maximum on the raw scores (the scale is positive), both 32-column halves
+      // (a 32-column half that lies entirely past the request is skipped in both passes: `valid` is uniform
+      // over the warp)
+      float mx = -INFINITY;
 #pragma unroll
-        for (int e = 0; e < 32; ++e) if (e >= valid) s[e] = 0xff800000u;   // -inf
-      }
-      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+      for (int h2 = 0; h2 < 2; ++h2) {
+        const int v2 = valid - h2 * 32;
+        if (v2 > 0) {
+          uint32_t s[32];
+          ptx::tmem_ld32(s_addr + h2 * 32, s);
+          ptx::tmem_ld_wait();
+          if (v2 < 32) {
 #pragma unroll
-      for (int e = 0; e < 32; e += 4) {
-        mx0 = fmaxf(mx0, __uint_as_float(s[e])); mx1 = fmaxf(mx1, __uint_as_float(s[e + 1]));
-        mx2 = fmaxf(mx2, __uint_as_float(s[e + 2])); mx3 = fmaxf(mx3, __uint_as_float(s[e + 3]));
+            for (int e = 0; e < 32; ++e) if (e >= v2) s[e] = 0xff800000u;
+          }
+          float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+          for (int e = 0; e < 32; e += 4) {
+            mx0 = fmaxf(mx0, __uint_as_float(s[e])); mx1 = fmaxf(mx1, __uint_as_float(s[e + 1]));
+            mx2 = fmaxf(mx2, __uint_as_float(s[e + 2])); mx3 = fmaxf(mx3, __uint_as_float(s[e + 3]));
+          }
+          mx = fmaxf(mx, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)));
+        }
       }
-      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
       xmax[(b * 2 + hh) * 128 + row] = mx;
       asm volatile("bar.sync 1, 256;" ::: "memory");
       const float mrow = fmaxf(mx, xmax[(b * 2 + (hh ^ 1)) * 128 + row]);
+      if (tracer) { SOD2_TRACE(2, 60 + j) }
       // move the reference?  (both threads of a row, and both warps of a row group, decide alike)
       const bool move = warp_live && (mrow - m) * c > 8.0f;
       float corr = 1.f;
@@ -227,31 +237,56 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         ptx::tmem_st_wait();
         ptx::tc_fence_before();
       }
-      // p = 2^(s*c - m*c): the scale rides in the FMA that feeds ex2.  The special-function pipe (16
-      // results per clock per SM) bounds this loop.
+      // ---- pass 2: p = 2^(s*c - m*c), 32 columns at a time: the scale rides in the FMA that feeds ex2.  The
+      // special-function pipe (16 results per clock per SM) bounds this loop.
       const float mc = -m * c;
       float sum0 = 0.f, sum1 = 0.f;
-      uint32_t pk[16];
+      uint32_t pk[2][16];
 #pragma unroll
-      for (int e = 0; e < 32; e += 2) {
-        const float p0 = ex2_approx(fmaf(__uint_as_float(s[e]), c, mc)), p1 = ex2_approx(fmaf(__uint_as_float(s[e + 1]), c, mc));
-        sum0 += p0; sum1 += p1;
-        const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-        pk[e >> 1] = warp_live ? *reinterpret_cast<const uint32_t*>(&pb) : 0u;
+      for (int h2 = 0; h2 < 2; ++h2) {
+        const int v2 = valid - h2 * 32;
+        uint32_t s[32];
+        if (v2 > 0) {
+          ptx::tmem_ld32(s_addr + h2 * 32, s);
+          ptx::tmem_ld_wait();
+        }
+        if (h2 == 1) {
+          // last read of S_j: the next S = Q K^T may overwrite it
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(s_free);
+        }
+        if (v2 > 0) {
+          if (v2 < 32) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) if (e >= v2) s[e] = 0xff800000u;   // -inf
+          }
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const float p0 = ex2_approx(fmaf(__uint_as_float(s[e]), c, mc)), p1 = ex2_approx(fmaf(__uint_as_float(s[e + 1]), c, mc));
+            sum0 += p0; sum1 += p1;
+            const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+            pk[h2][e >> 1] = warp_live ? *reinterpret_cast<const uint32_t*>(&pb) : 0u;
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) pk[h2][e] = 0u;
+        }
       }
       l += sum0 + sum1;
       if (tracer) { SOD2_TRACE(2, 40 + j) }
-      // P_j into the swizzled tile once the MMA that read this buffer two blocks ago has finished
-      if (j >= 2) ptx::mbar_wait_warp(&o_full[b], ((j >> 1) - 1) & 1, dead);    // O_{j-2} done: P buffer free
+      // P_j into the two swizzled chunks once the MMA that read the buffer for the last block has finished
+      if (j >= 1) ptx::mbar_wait_warp(&o_full[(j - 1) & 1], ((j - 1) >> 1) & 1, dead);    // O_{j-1} done: the P buffer is free
       {
-        uint8_t* prow = sP + b * ATC_P_BYTES + row * 128;
+        uint8_t* prow = sP + hh * (128 * 128) + row * 128;     // chunk hh holds this thread's 64 keys
 #pragma unroll
-        for (int g = 0; g < 4; ++g)
-          *reinterpret_cast<uint4*>(prow + (((hh * 4 + g) ^ (row & 7)) << 4)) = make_uint4(pk[4 * g], pk[4 * g + 1], pk[4 * g + 2], pk[4 * g + 3]);
+        for (int g = 0; g < 8; ++g)
+          *reinterpret_cast<uint4*>(prow + ((g ^ (row & 7)) << 4)) =
+              make_uint4(pk[g >> 2][4 * (g & 3)], pk[g >> 2][4 * (g & 3) + 1], pk[g >> 2][4 * (g & 3) + 2], pk[g >> 2][4 * (g & 3) + 3]);
       }
       ptx::fence_proxy_async();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&p_full[b]);
+      if (lane == 0) ptx::mbar_arrive(p_full);
       if (tracer) { SOD2_TRACE(2, 50 + j) }
     }
     // ---- output: O / l.  The row sums of the two halves are added through shared memory, the scaled rows

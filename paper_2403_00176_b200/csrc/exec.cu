@@ -433,8 +433,8 @@ struct Builder {
             const void* Kp = x.resolve(bk);
             const void* V = x.resolve(bv);
             if (cache->q != Q || cache->k != Kp || cache->v != V) {
-              if (!encode_bf16_2d(&cache->tq, Q, rows_q, q_ts, q_ts, 128) || !encode_bf16_2d(&cache->tk, Kp, rows_k, k_ts, k_ts, 64) ||
-                  !encode_bf16_2d(&cache->tv, V, rows_v, v_ts, v_ts, 64))
+              if (!encode_bf16_2d(&cache->tq, Q, rows_q, q_ts, q_ts, 128) || !encode_bf16_2d(&cache->tk, Kp, rows_k, k_ts, k_ts, k::ATC_KB) ||
+                  !encode_bf16_2d(&cache->tv, V, rows_v, v_ts, v_ts, k::ATC_KB))
                 return cudaErrorInvalidValue;
               cache->q = Q; cache->k = Kp; cache->v = V;
             }
