@@ -196,6 +196,39 @@ def run_ours(args):
         del pl, b
     e2e_ms = sum(e2e_times) / len(e2e_times)
 
+    # ---- the same loop through the plan cache, every batch seen before (a serving process meets the same
+    # bound symbol tuples again; reported beside the uncached number, which stays the e2e value)
+    sess.graph.set_plan_cache(len(preps) + 1)
+    e2e_hit = []
+    n_e2e = min(args.steps, 10) + 1
+    for i in range(2 * n_e2e):
+        key = i % len(preps)
+        if key not in pinned_in:
+            continue
+        pr = preps[key]
+        torch.cuda.synchronize(dev)
+        t0 = time.perf_counter()
+        for dst, src in zip(pr.in_dev, pinned_in[key]):
+            dst.copy_(src, non_blocking=True)
+        _, pl, hit = sess.graph.plan_cached(wl.sym_names, [[r.syms[s] for s in wl.sym_names] for r in pr.reqs])
+        pl.run([t.data_ptr() for t in pr.in_dev], [t.data_ptr() for t in pr.out_dev], pr.arena.data_ptr(), pr.arena.numel(),
+               sess.stream)
+        for dst, src in zip(pinned_out[key], pr.out_dev):
+            dst.copy_(src, non_blocking=True)
+        torch.cuda.synchronize(dev)
+        if hit:
+            e2e_hit.append((time.perf_counter() - t0) * 1e3)
+    e2e_hit_ms = sum(e2e_hit) / len(e2e_hit) if e2e_hit else None
+    th = []
+    for i in range(5):
+        pr = preps[i % len(preps)]
+        t0 = time.perf_counter()
+        _, pl, hit = sess.graph.plan_cached(wl.sym_names, [[r.syms[s] for s in wl.sym_names] for r in pr.reqs])
+        if hit:
+            th.append((time.perf_counter() - t0) * 1e6)
+    plan_hit_us = sorted(th)[len(th) // 2] if th else None
+    sess.graph.set_plan_cache(0)
+
     # ---- planning overhead (host): bind + plan per batch
     tb = []
     for i in range(5):
@@ -235,8 +268,10 @@ def run_ours(args):
             "gpu_launches": int(launches),
             "clocks": clocks,
             "e2e": {"value": e2e_ms, "unit": "ms/inference", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-                    "includes": "H2D (pinned, enqueued first) + bind_dims + plan + run + D2H (pinned)"},
+                    "includes": "H2D (pinned, enqueued first) + bind_dims + plan + run + D2H (pinned)",
+                    "value_plan_cache_hit": e2e_hit_ms},
             "plan_us_per_batch": plan_us,
+            "plan_us_per_batch_cache_hit": plan_hit_us,
             "arena": mem,
             "roofline": {"bound": "tensor", "achieved": gemm["tflops"], "peak": peaks["tf_sustained"], "unit": "TFLOP/s",
                          "frac": gemm["tflops"] / peaks["tf_sustained"],

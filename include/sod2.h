@@ -77,6 +77,19 @@ void sod2_binding_destroy(sod2_binding* b);
 sod2_status sod2_plan(sod2_graph* g, const sod2_binding* b, sod2_plan_t** out, size_t* arena_bytes);
 void sod2_plan_destroy(sod2_plan_t* p);
 
+/* Plan cache.  Planning happens at execution time, when the sizes are known (Section 4.4.1); a request
+ * mix whose bound symbol tuple has been seen before needs no new plan.  sod2_graph_set_plan_cache sets
+ * the number of (binding, plan) pairs the graph keeps, least recently used first out (0, the default,
+ * disables and empties the cache).  sod2_plan_cached = sod2_bind_dims + sod2_plan through the cache:
+ * *hit = 1 if the pair was found.  The handles it returns are BORROWED: they belong to the graph and
+ * stay valid until the entry is evicted by later misses, the capacity is lowered or the graph is
+ * destroyed; sod2_binding_destroy / sod2_plan_destroy ignore them.  A plan does not depend on the
+ * addresses it ran with, so a cached plan may be run with any inputs, outputs and arena. */
+sod2_status sod2_graph_set_plan_cache(sod2_graph* g, int capacity);
+sod2_status sod2_plan_cached(sod2_graph* g, int n_requests, int n_syms, const char* const* sym_names,
+                             const int64_t* values, sod2_binding** binding_out, sod2_plan_t** plan_out,
+                             size_t* arena_bytes, int* hit);
+
 typedef struct {
   int64_t host_enqueue_ns; /* host time spent inside sod2_run */
   int64_t gpu_launches;    /* kernels enqueued */

@@ -50,6 +50,8 @@ def _load() -> C.CDLL:
         "sod2_graph_prepack": [vp, vp, sz, vp],
         "sod2_bind_dims": [vp, i32, i32, P(cp), P(i64), P(vp)],
         "sod2_plan": [vp, vp, P(vp), P(sz)],
+        "sod2_graph_set_plan_cache": [vp, i32],
+        "sod2_plan_cached": [vp, i32, i32, P(cp), P(i64), P(vp), P(vp), P(sz), P(i32)],
         "sod2_run": [vp, P(vp), P(vp), vp, sz, vp, P(RunInfo)],
         "sod2_run_timed": [vp, P(vp), P(vp), vp, sz, vp, P(C.c_float), i32],
         "sod2_plan_device_status": [vp, vp, vp],
@@ -87,7 +89,7 @@ def _load() -> C.CDLL:
 
 lib = _load()
 EXPORTS = ["sod2_graph_create", "sod2_graph_destroy", "sod2_graph_set_const", "sod2_graph_prepack_bytes",
-           "sod2_graph_prepack", "sod2_bind_dims", "sod2_binding_destroy", "sod2_plan", "sod2_plan_destroy",
+           "sod2_graph_prepack", "sod2_bind_dims", "sod2_binding_destroy", "sod2_plan", "sod2_plan_destroy", "sod2_graph_set_plan_cache", "sod2_plan_cached",
            "sod2_run", "sod2_run_timed", "sod2_plan_device_status", "sod2_graph_tensor_info", "sod2_graph_tensor_value", "sod2_graph_tensor_dtype",
            "sod2_graph_num_ops", "sod2_graph_op_info", "sod2_graph_num_groups", "sod2_graph_group_info",
            "sod2_graph_num_subgraphs", "sod2_graph_rdp_sweeps", "sod2_classify", "sod2_graph_reanalyse", "sod2_graph_order_info",
@@ -148,6 +150,24 @@ class Graph:
         _check(lib.sod2_graph_prepack(self.h, C.c_void_p(dev_ws), nbytes, C.c_void_p(stream)), self.h)
         if keep is not None:
             self._keep.append(keep)
+
+    def set_plan_cache(self, capacity: int):
+        _check(lib.sod2_graph_set_plan_cache(self.h, capacity), self.h)
+
+    def plan_cached(self, sym_names: Sequence[str], values: Sequence[Sequence[int]]):
+        """bind_dims + plan through the graph's plan cache: (Binding, Plan, hit).  The handles are borrowed
+        from the graph (valid until evicted); the wrappers keep the graph alive and never destroy them."""
+        n_req, n_sym = len(values), len(sym_names)
+        names = (C.c_char_p * max(n_sym, 1))(*[s.encode() for s in sym_names])
+        flat = [int(v) for row in values for v in row]
+        vals = (C.c_int64 * max(len(flat), 1))(*flat)
+        hb, hp, ab, hit = C.c_void_p(), C.c_void_p(), C.c_size_t(), C.c_int()
+        _check(lib.sod2_plan_cached(self.h, n_req, n_sym, names, vals, C.byref(hb), C.byref(hp), C.byref(ab), C.byref(hit)), self.h)
+        b = Binding.__new__(Binding)
+        b.graph, b.h, b.n_req, b.borrowed = self, hb, n_req, True
+        p = Plan.__new__(Plan)
+        p.binding, p.graph, p.h, p.arena_bytes, p.borrowed = b, self, hp, ab.value, True
+        return b, p, bool(hit.value)
 
     def bind_dims(self, sym_names: Sequence[str], values: Sequence[Sequence[int]]) -> "Binding":
         return Binding(self, sym_names, values)
@@ -222,7 +242,7 @@ class Binding:
         self.n_req = n_req
 
     def __del__(self):
-        if getattr(self, "h", None) and lib is not None:   # lib is None while the interpreter shuts down
+        if getattr(self, "h", None) and lib is not None and not getattr(self, "borrowed", False):   # lib is None at shutdown
             lib.sod2_binding_destroy(self.h)
             self.h = None
 
@@ -249,7 +269,7 @@ class Plan:
         self.arena_bytes = ab.value
 
     def __del__(self):
-        if getattr(self, "h", None) and lib is not None:   # lib is None while the interpreter shuts down
+        if getattr(self, "h", None) and lib is not None and not getattr(self, "borrowed", False):   # lib is None at shutdown
             lib.sod2_plan_destroy(self.h)
             self.h = None
 

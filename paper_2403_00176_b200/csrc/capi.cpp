@@ -2,7 +2,9 @@
 #include <cuda_runtime.h>
 
 #include <cstring>
+#include <list>
 #include <new>
+#include <unordered_map>
 
 #include "../../include/sod2.h"
 #include "engine.h"
@@ -13,9 +15,24 @@ struct HandleBase {
   uint32_t magic;
   std::string err;
 };
-struct sod2_graph { HandleBase h{0x53443247u, ""}; Compiled c; };
-struct sod2_binding { HandleBase h{0x53443242u, ""}; Binding b; sod2_graph* g = nullptr; };
-struct sod2_plan_s { HandleBase h{0x53443250u, ""}; Plan p; sod2_graph* g = nullptr; };
+struct sod2_binding { HandleBase h{0x53443242u, ""}; Binding b; sod2_graph* g = nullptr; bool cached = false; };
+struct sod2_plan_s { HandleBase h{0x53443250u, ""}; Plan p; sod2_graph* g = nullptr; bool cached = false; };
+// Plan cache: binding + plan per bound symbol tuple, least recently used first out.  The entries belong
+// to the graph; handles given out by sod2_plan_cached are borrowed.
+struct PlanCacheEntry { std::string key; sod2_binding* b; sod2_plan_s* p; };
+struct sod2_graph {
+  HandleBase h{0x53443247u, ""};
+  Compiled c;
+  int cache_cap = 0;
+  std::list<PlanCacheEntry> lru;                                             // front = most recently used
+  std::unordered_map<std::string, std::list<PlanCacheEntry>::iterator> cache;
+  void clear_cache() {
+    for (auto& e : lru) { delete e.p; delete e.b; }
+    lru.clear();
+    cache.clear();
+  }
+  ~sod2_graph() { clear_cache(); }
+};
 
 static thread_local std::string g_create_err;
 
@@ -118,7 +135,7 @@ sod2_status sod2_bind_dims(sod2_graph* g, int n_req, int n_syms, const char* con
   *out = b;
   return SOD2_OK;
 }
-void sod2_binding_destroy(sod2_binding* b) { delete b; }
+void sod2_binding_destroy(sod2_binding* b) { if (b && !b->cached) delete b; }
 
 sod2_status sod2_plan(sod2_graph* g, const sod2_binding* b, sod2_plan_t** out, size_t* arena_bytes) {
   if (!g || !b || !out || b->g != g) return SOD2_E_INVALID_ARG;
@@ -131,7 +148,59 @@ sod2_status sod2_plan(sod2_graph* g, const sod2_binding* b, sod2_plan_t** out, s
   *out = p;
   return SOD2_OK;
 }
-void sod2_plan_destroy(sod2_plan_t* p) { delete p; }
+void sod2_plan_destroy(sod2_plan_t* p) { if (p && !p->cached) delete p; }
+
+sod2_status sod2_graph_set_plan_cache(sod2_graph* g, int capacity) {
+  if (!g || capacity < 0) return SOD2_E_INVALID_ARG;
+  g->cache_cap = capacity;
+  while (static_cast<int>(g->lru.size()) > capacity) {
+    PlanCacheEntry& e = g->lru.back();
+    g->cache.erase(e.key);
+    delete e.p;
+    delete e.b;
+    g->lru.pop_back();
+  }
+  return SOD2_OK;
+}
+
+sod2_status sod2_plan_cached(sod2_graph* g, int n_req, int n_syms, const char* const* names, const int64_t* values,
+                             sod2_binding** binding_out, sod2_plan_t** plan_out, size_t* arena_bytes, int* hit) {
+  if (!g || !plan_out || n_req < 0 || n_syms < 0 || (n_syms > 0 && (!names || !values))) return SOD2_E_INVALID_ARG;
+  if (g->cache_cap <= 0) { g->h.err = "the plan cache is disabled: call sod2_graph_set_plan_cache first"; return SOD2_E_INVALID_ARG; }
+  std::string key(reinterpret_cast<const char*>(&n_req), sizeof n_req);
+  for (int i = 0; i < n_syms; ++i) { key += names[i]; key.push_back('\0'); }
+  key.append(reinterpret_cast<const char*>(values), static_cast<size_t>(n_req) * n_syms * sizeof(int64_t));
+  auto it = g->cache.find(key);
+  if (it != g->cache.end()) {
+    g->lru.splice(g->lru.begin(), g->lru, it->second);   // most recently used
+    if (hit) *hit = 1;
+  } else {
+    sod2_binding* b = new (std::nothrow) sod2_binding();
+    sod2_plan_s* p = new (std::nothrow) sod2_plan_s();
+    if (!b || !p) { delete b; delete p; return SOD2_E_INTERNAL; }
+    b->g = g; b->cached = true;
+    p->g = g; p->cached = true;
+    Status s = bind_dims(&g->c, n_req, n_syms, names, values, &b->b);
+    if (s != OK) { g->h.err = b->b.err; delete b; delete p; return st(s); }
+    s = make_plan(&g->c, &b->b, &p->p);
+    if (s != OK) { g->h.err = p->p.err; delete p; delete b; return st(s); }
+    if (static_cast<int>(g->lru.size()) >= g->cache_cap) {
+      PlanCacheEntry& e = g->lru.back();
+      g->cache.erase(e.key);
+      delete e.p;
+      delete e.b;
+      g->lru.pop_back();
+    }
+    g->lru.push_front(PlanCacheEntry{key, b, p});
+    g->cache[key] = g->lru.begin();
+    if (hit) *hit = 0;
+  }
+  PlanCacheEntry& e = g->lru.front();
+  if (binding_out) *binding_out = e.b;
+  *plan_out = e.p;
+  if (arena_bytes) *arena_bytes = e.p->p.arena_bytes;
+  return SOD2_OK;
+}
 
 sod2_status sod2_run(sod2_plan_t* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes,
                      void* stream, sod2_run_info* info) {

@@ -10,6 +10,7 @@ from paper_2403_00176_b200 import binding as B
 from paper_2403_00176_b200 import workloads as WL
 from paper_2403_00176_b200.workloads import Request, bf16_round
 from tests.gpu_harness import lockstep, run_batch
+from paper_2403_00176_b200.session import Session
 
 pytestmark = pytest.mark.gpu
 
@@ -112,6 +113,26 @@ def test_cfg2_small_encoder_arena_reuse_matches_no_reuse():
     assert p2.plan.arena_bytes < p1.plan.arena_bytes
     for a, b in zip(o1, o2):
         assert np.array_equal(a["y"], b["y"])
+
+
+def test_cfg2_plan_cache_reuses_a_plan_with_other_buffers():
+    # a cached plan run with fresh inputs, outputs and arena gives the bits of a freshly made plan
+    wl, reqs = _encoder_edge()
+    s1, p1, o1 = run_batch(wl, reqs)
+    s = Session(wl)
+    s.graph.set_plan_cache(2)
+    names = wl.sym_names
+    vals = [[r.syms[n] for n in names] for r in reqs]
+    for rep in range(2):
+        b, pl, hit = s.graph.plan_cached(names, vals)
+        assert hit == (rep == 1)
+        pr = s.prepare(reqs)                      # its own buffers and arena
+        assert pr.arena.numel() >= pl.arena_bytes
+        pl.run([t.data_ptr() for t in pr.in_dev], [t.data_ptr() for t in pr.out_dev], pr.arena.data_ptr(), pr.arena.numel(), s.stream)
+        pl.device_status(pr.arena.data_ptr(), s.stream)
+        outs = pr.outputs()
+        for r in range(len(reqs)):
+            assert np.array_equal(outs[r]["y"], o1[r]["y"])
 
 
 def test_cfg2_full_config_batch0():
