@@ -84,6 +84,16 @@ def measure(cfg: int, reps: int, oracle_budget: float):
         pl = b.plan()
         plan_us.append((time.perf_counter() - t0) * 1e6)
         del pl, b
+    # the same through the plan cache, every bound symbol tuple seen before
+    sess.graph.set_plan_cache(len(preps) + 1)
+    hit_us = []
+    for i in range(2 * len(preps) + 3):
+        reqs = preps[i % len(preps)].reqs
+        t0 = time.perf_counter()
+        _, _, hit = sess.graph.plan_cached(wl.sym_names, [[r.syms[s] for s in wl.sym_names] for r in reqs])
+        if hit:
+            hit_us.append((time.perf_counter() - t0) * 1e6)
+    sess.graph.set_plan_cache(0)
     mem = preps[0].plan.memory()
     # oracle on a bounded sample
     t0 = time.perf_counter()
@@ -114,7 +124,7 @@ def measure(cfg: int, reps: int, oracle_budget: float):
         "sum_t_roof_over_sum_t_groups": sum_roof / sum_ms, "sum_t_roof_over_t_step": sum_roof / float(np.median(times)),
         "worst_group": {"kind": worst["kind"], "frac": worst["frac"], "bound": worst["bound"], "ms": worst["ms"]},
         "kinds": {k: {"ms": round(v["ms"], 4), "frac": round(v["frac"], 3), "tflops": round(v["tflops"], 1), "gbs": round(v["gbs"], 1)} for k, v in kinds.items()},
-        "plan_us_median": float(np.median(plan_us)), "arena_bytes": mem["arena_bytes"], "peak_live_bytes": mem["peak_live_bytes"],
+        "plan_us_median": float(np.median(plan_us)), "plan_us_cache_hit": float(np.median(hit_us)) if hit_us else None, "arena_bytes": mem["arena_bytes"], "peak_live_bytes": mem["peak_live_bytes"],
         "sum_tensor_bytes": mem["sum_bytes"], "n_groups": sess.graph.num_groups(), "n_ops": sess.graph.num_ops(),
         "gpu_launches": preps[0].plan.run_timed and None,
         "oracle_ms": oracle_ms, "oracle_cores": os.cpu_count(), "oracle_sample": sample, "peaks": src,
@@ -133,11 +143,11 @@ def main():
         r.pop("gpu_launches", None)
         print(json.dumps(r), flush=True)
         rows.append(r)
-    print("\n| cfg | ms per inference (median, min) | ms per request | sum t_roof / t_step | worst group: fraction, bound | bind+plan us | arena / peak-live MB | oracle ms (cores) |")
+    print("\n| cfg | ms per inference (median, min) | ms per request | sum t_roof / t_step | worst group: fraction, bound | bind+plan us (cache hit) | arena / peak-live MB | oracle ms (cores) |")
     print("|---|---|---|---|---|---|---|---|")
     for r in rows:
         print(f"| {r['cfg']} | {r['ms_median']:.3f}, {r['ms_min']:.3f} | {r['ms_per_request']:.4f} | {r['sum_t_roof_over_t_step']:.3f} | "
-              f"{r['worst_group']['kind']}: {r['worst_group']['frac']:.3f}, {r['worst_group']['bound']} | {r['plan_us_median']:.0f} | "
+              f"{r['worst_group']['kind']}: {r['worst_group']['frac']:.3f}, {r['worst_group']['bound']} | {r['plan_us_median']:.0f} ({r['plan_us_cache_hit'] or 0:.0f}) | "
               f"{r['arena_bytes'] / 1e6:.1f} / {r['peak_live_bytes'] / 1e6:.1f} | {r['oracle_ms']:.0f} ({r['oracle_cores']}) |")
 
 
