@@ -44,6 +44,7 @@ typedef enum {
 #define SOD2_OPT_NO_REUSE  2u /* every arena tensor keeps its own slot: intermediates stay readable */
 #define SOD2_OPT_COPY_REGROUP 16u /* Switch / Combine always copy whole samples (no index-indirect convolutions) */
 #define SOD2_OPT_LEGACY_ATTENTION 8u /* attention groups run the mma.sync kernel even where the tcgen05 kernel applies */
+#define SOD2_OPT_MULTI_VERSION 64u /* fuse elementwise chains across broadcasts RDP cannot resolve: 2^d fused versions (Section 4.2), the version (a stride table) chosen at bind time */
 #define SOD2_OPT_NO_SEP 32u /* groups run in their default topological order: no static execution planning (Section 4.3) */
 #define SOD2_OPT_SPLITK_LN 4u /* bf16 GEMM (+bias, +residual) -> LayerNorm as one group: split-K GEMM into fp32 slabs + finishing kernel */
 

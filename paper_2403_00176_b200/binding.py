@@ -22,6 +22,7 @@ OPT_SPLITK_LN = 4
 OPT_LEGACY_ATTENTION = 8
 OPT_COPY_REGROUP = 16
 OPT_NO_SEP = 32
+OPT_MULTI_VERSION = 64
 DYN_CLASS = ["ISDO", "ISDOS", "ISVDOS", "EDO"]
 
 

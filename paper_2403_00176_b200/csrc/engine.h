@@ -14,6 +14,7 @@ enum OptFlags : uint32_t {
   OPT_NO_REUSE = 2u,    // every arena tensor gets its own slot (keeps all intermediates readable after a run)
   OPT_COPY_REGROUP = 16u,     // Switch / Combine always move whole samples (no index-indirect convolutions)
   OPT_LEGACY_ATTENTION = 8u,  // attention groups on the mma.sync kernel even where the tcgen05 kernel applies
+  OPT_MULTI_VERSION = 64u,    // fuse elementwise chains across unresolved broadcasts: 2^d versions, chosen at bind time
   OPT_NO_SEP = 32u,     // groups run in their default topological order (no static execution planning)
   OPT_SPLITK_LN = 4u,   // a bf16 GEMM (+bias, +residual) followed by LayerNorm becomes one group: split-K GEMM + finishing kernel
 };

@@ -307,6 +307,7 @@ struct Fuser {
     G.chain_operands.push_back(operand);
     G.nodes = {nid};
     int unres = static_cast<int>(n0.attr_i("unresolved_bcast", 0));
+    int vbits = 0;                      // unresolved extent pairs fused across (multi-version fusion)
     cur = out0;
     while (fuse && G.chain_ops.size() < 8) {
       int nx = sole_consumer(cur);
@@ -322,8 +323,17 @@ struct Fuser {
           // share the output's index space or broadcast into it dim by dim ("1" or "same")
           if (!(resolved_bcast(n.outs[0], opd) && resolved_bcast(n.outs[0], cur))) {
             int u = static_cast<int>(n.attr_i("unresolved_bcast", 0));
-            if (u) { G.versions = std::max(G.versions, 1 << u); }
-            break;
+            // Multi-version fusion (Section 4.2): d unresolved extent pairs need 2^d fused versions.  The
+            // chain kernel is parametric in its strides, so a "version" is a stride table and is chosen at
+            // bind time, when the extents are known (a broadcast extent reads with stride 0); the bind-time
+            // assertions reject pairs that are neither equal nor 1.  Off by default: without the flag the
+            // operators stay unfused, which is what RDP's resolution of the extents saves.
+            const bool all_known = g.tensors[n.outs[0]].S.fully_known() && g.tensors[opd].S.fully_known() && g.tensors[cur].S.fully_known();
+            if (u && (c.flags & OPT_MULTI_VERSION) && all_known && vbits + u <= 16) { vbits += u; }
+            else {
+              if (u) { G.versions = std::max(G.versions, 1 << u); }
+              break;
+            }
           }
           std::set<int> inside(G.nodes.begin(), G.nodes.end());
           if (depends_on(opd, inside)) break;
@@ -340,7 +350,7 @@ struct Fuser {
         break;
       } else break;
     }
-    if (unres) G.versions = 1 << unres;
+    if (unres + vbits) G.versions = std::max(G.versions, 1 << (unres + vbits));
     G.out = cur;
     finish(G);
   }

@@ -92,6 +92,7 @@ struct Node {
 struct Assertion {           // bind-time check produced when two inferences must agree
   Expr a, b;
   std::string what;
+  int kind = 0;              // 0: a == b; 1: broadcast-compatible (a == b, or one of them is 1)
 };
 
 struct Graph {

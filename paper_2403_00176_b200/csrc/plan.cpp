@@ -36,7 +36,10 @@ Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* na
     for (auto& as : g.asserts) {
       bool ok1, ok2;
       int64_t x = e_eval(g.cx, as.a, out->vals[r], &ok1), y = e_eval(g.cx, as.b, out->vals[r], &ok2);
-      if (ok1 && ok2 && x != y) { out->err = "shape conflict: " + as.what + " (" + std::to_string(x) + " vs " + std::to_string(y) + ")"; return E_SHAPE_CONFLICT; }
+      if (ok1 && ok2 && x != y && !(as.kind == 1 && (x == 1 || y == 1))) {
+        out->err = "shape conflict: " + as.what + " (" + std::to_string(x) + " vs " + std::to_string(y) + ")";
+        return E_SHAPE_CONFLICT;
+      }
     }
   // all non-linear atoms once per request (children first), then every distinct extent expression once
   // per request as a flat polynomial; tensors pick their extents from that table

@@ -360,8 +360,14 @@ struct Rdp {
 
   void add_assert(const Expr& a, const Expr& b, const std::string& what) {
     if (a == b) return;
-    for (auto& x : g.asserts) if ((x.a == a && x.b == b) || (x.a == b && x.b == a)) return;
-    g.asserts.push_back({a, b, what});
+    for (auto& x : g.asserts) if (x.kind == 0 && ((x.a == a && x.b == b) || (x.a == b && x.b == a))) return;
+    g.asserts.push_back({a, b, what, 0});
+  }
+  // An extent pair that RDP can resolve neither to "same" nor to "1" is legal only if the bound values do
+  // (Section 4.2: the fused version is chosen once the extents are known).
+  void add_bcast_assert(const Expr& a, const Expr& b, const std::string& what) {
+    for (auto& x : g.asserts) if (x.kind == 1 && ((x.a == a && x.b == b) || (x.a == b && x.b == a))) return;
+    g.asserts.push_back({a, b, what, 1});
   }
 
   // Move one component down the lattice. Two different constants from two inference sources must
@@ -433,6 +439,7 @@ struct Rdp {
       } else {
         // neither provably 1 nor provably equal: both fused versions would be needed
         if (unresolved) ++*unresolved;
+        add_bcast_assert(da.e, db.e, who + ": broadcast of " + e_str(g.cx, da.e) + " with " + e_str(g.cx, db.e));
         o.dims[i] = Dim::val(e_max(g.cx, da.e, db.e));
       }
     }

@@ -57,6 +57,43 @@ def test_fig4_chain_one_fused_version():
 EDGE_L = [1, 15, 16, 17, 63, 64, 65, 127, 128, 129, 200, 257, 512]
 
 
+def test_multi_version_chain_version_chosen_at_bind_time():
+    # extent pairs that RDP cannot resolve (three at the Add; three more at the Mul, whose left extents are
+    # max(I, Ip) etc.): with multi-version fusion the three operators are one group with 2^6 versions;
+    # every request of the batch binds another version (which operand broadcasts where)
+    ir = """
+sym I 1 64
+sym J 1 64
+sym K 1 640
+sym Ip 1 64
+sym Jp 1 64
+sym Kp 1 640
+input A f32 [Ip,Jp,Kp]
+input B f32 [I,J,K]
+node Sigmoid A -> s
+node Add s B -> t
+node Mul t B -> C
+output C
+"""
+    rng = np.random.default_rng(5)
+    combos = [(4, 5, 6, 4, 1, 1), (4, 5, 6, 1, 5, 1), (4, 5, 6, 1, 1, 6), (4, 5, 6, 4, 5, 6), (1, 5, 6, 4, 5, 6), (7, 1, 300, 7, 9, 1),
+              (1, 1, 1, 3, 2, 5), (5, 1, 1, 1, 4, 1)]
+    reqs = []
+    for i_, j_, k_, ip, jp, kp in combos:
+        reqs.append(Request({"I": i_, "J": j_, "K": k_, "Ip": ip, "Jp": jp, "Kp": kp},
+                            {"A": rng.standard_normal((ip, jp, kp)).astype(np.float32), "B": rng.standard_normal((i_, j_, k_)).astype(np.float32)}))
+    wl = WL.Workload("multi_version", "f32", ir, {}, ["I", "J", "K", "Ip", "Jp", "Kp"], ["C"], {"batch_fn": lambda j: reqs})
+    s, p, outs = run_batch(wl, reqs, opt_flags=B.OPT_MULTI_VERSION)
+    assert s.graph.num_groups() == 1 and s.graph.group_info(0)["versions"] == 64
+    s0, p0, outs0 = run_batch(wl, reqs)                       # unfused: the default
+    assert s0.graph.num_groups() >= 2
+    for r, req in enumerate(reqs):
+        ref = O.run(ir, {}, req.inputs)["C"]
+        assert outs[r]["C"].shape == ref.shape, (req.syms, outs[r]["C"].shape)
+        assert O.rel_err(outs[r]["C"], ref) <= F32_TOL, req.syms
+        assert np.array_equal(outs[r]["C"], outs0[r]["C"])
+
+
 def _encoder_edge(layers=2, F=256):
     wl = WL.cfg2(layers=layers, D=128, H=2, F=F, n_requests=1, lmin=1, lmax=512)
     rng = np.random.default_rng(11)

@@ -188,6 +188,20 @@ output C
     # binding that violates "1 or same" is caught by the recorded assertion-free max() rule:
     b = g.bind_dims(["I", "J", "K", "Ip", "Jp", "Kp"], [[4, 5, 6, 4, 1, 1]])
     assert b.shape(0, "C") == [4, 5, 6]
+    # an extent pair that is neither equal nor 1 is rejected when the symbols are bound
+    with pytest.raises(B.Sod2Error) as e:
+        g.bind_dims(["I", "J", "K", "Ip", "Jp", "Kp"], [[4, 5, 6, 3, 1, 1]])
+    assert "SHAPE_CONFLICT" in str(e.value) and "broadcast" in str(e.value)
+    # multi-version fusion: the chain is fused across the three unresolved pairs, 2^3 versions, the version
+    # (which extents broadcast) being chosen when the symbols are bound
+    g2 = B.Graph(ir, B.OPT_MULTI_VERSION)
+    assert g2.num_groups() == 1 and g2.group_info(0)["versions"] == 8 and g2.group_info(0)["n_ops"] == 2
+    for vals, shape in [([4, 5, 6, 4, 1, 1], [4, 5, 6]), ([4, 5, 6, 1, 5, 1], [4, 5, 6]), ([4, 1, 6, 4, 5, 6], [4, 5, 6]), ([1, 1, 1, 2, 3, 4], [2, 3, 4])]:
+        b2 = g2.bind_dims(["I", "J", "K", "Ip", "Jp", "Kp"], [vals])
+        assert b2.shape(0, "C") == shape
+        b2.plan()
+    with pytest.raises(B.Sod2Error):
+        g2.bind_dims(["I", "J", "K", "Ip", "Jp", "Kp"], [[4, 5, 6, 4, 2, 1]])
 
 
 def test_backward_transfer():
