@@ -773,6 +773,86 @@ struct Rdp {
         ValueVal v; v.kind = ValueVal::NAC;
         ch |= refine_value(out(0), v);
       }
+    } else if (op == "EyeLike" || op == "GroupNormalization") {    // output shape = shape of the first input
+      g.tensors[out(0)].dtype = g.tensors[in(0)].dtype;
+      if (S(in(0)).rank != RANK_UNDEF) ch |= refine_shape(out(0), S(in(0)));
+    } else if (op == "AveragePool" || op == "MaxPool") {           // F^fs_ISDOS: windows over H, W
+      const ShapeVal& x = S(in(0));
+      g.tensors[out(0)].dtype = g.tensors[in(0)].dtype;
+      if (x.rank == 4) {
+        const int64_t k = n.attr_i("kernel", 2), s_ = n.attr_i("stride", k), p = n.attr_i("pad", 0);
+        ShapeVal s; s.rank = 4; s.dims = {x.dims[0], x.dims[1], x.dims[2], x.dims[3]};
+        for (int d = 2; d < 4; ++d)
+          if (x.dims[d].known()) s.dims[d] = Dim::val(e_floordiv(g.cx, x.dims[d].e + Expr(2 * p - k), Expr(s_)) + Expr(1));
+        ch |= refine_shape(out(0), s);
+      } else if (x.rank >= 0) fail(E_RANK_MISMATCH, op + " needs NCHW input");
+    } else if (op == "Expand") {                                   // F^fs_ISVDOS: broadcast against the VALUE of the shape input
+      const ValueVal& v = V(in(1));
+      g.tensors[out(0)].dtype = g.tensors[in(0)].dtype;
+      if (v.kind == ValueVal::KNOWN) {
+        ShapeVal t; t.rank = static_cast<int>(v.elems.size()); t.dims = v.elems;
+        int unres = 0;
+        ShapeVal s = bcast(S(in(0)), t, "Expand -> " + g.tensors[out(0)].name, &unres);
+        n.attrs["unresolved_bcast"] = std::to_string(unres);
+        ch |= refine_shape(out(0), s);
+      } else if (v.kind == ValueVal::NAC) { ShapeVal s; s.rank = RANK_NAC; ch |= refine_shape(out(0), s); }
+    } else if (op == "Resize" || op == "Upsample") {                // F^fs_ISVDOS: sizes input (values) or integer scales attribute
+      const ShapeVal& x = S(in(0));
+      g.tensors[out(0)].dtype = g.tensors[in(0)].dtype;
+      const std::vector<int64_t> sc = n.attr_list("scales");
+      if (n.ins.size() > 1) {
+        const ValueVal& v = V(in(1));
+        if (v.kind == ValueVal::KNOWN) {
+          ShapeVal s; s.rank = static_cast<int>(v.elems.size()); s.dims = v.elems;
+          if (x.rank >= 0 && x.rank != s.rank) fail(E_RANK_MISMATCH, op + ": sizes must have the input's rank");
+          else ch |= refine_shape(out(0), s);
+        } else if (v.kind == ValueVal::NAC && x.rank >= 0) {
+          ShapeVal s; s.rank = x.rank; s.dims.assign(x.rank, Dim::nac());
+          ch |= refine_shape(out(0), s);
+        }
+      } else if (x.rank >= 0) {
+        if (static_cast<int>(sc.size()) != x.rank) fail(E_BAD_DIM, op + ": scales must list one integer per axis");
+        else {
+          ShapeVal s; s.rank = x.rank; s.dims.resize(x.rank);
+          for (int d = 0; d < x.rank; ++d) s.dims[d] = x.dims[d].known() ? Dim::val(x.dims[d].e * Expr(sc[d])) : x.dims[d];
+          ch |= refine_shape(out(0), s);
+        }
+      }
+    } else if (op == "OneHot") {                                    // F^fs_ISVDOS: indices shape + [depth value]
+      const ShapeVal& x = S(in(0));
+      const ValueVal& v = V(in(1));
+      if (x.rank >= 0 && v.kind == ValueVal::KNOWN && v.elems.size() == 1) {
+        ShapeVal s = x; s.rank = x.rank + 1; s.dims.push_back(v.elems[0]);
+        ch |= refine_shape(out(0), s);
+      } else if (x.rank >= 0 && v.kind == ValueVal::NAC) {
+        ShapeVal s = x; s.rank = x.rank + 1; s.dims.push_back(Dim::nac());
+        ch |= refine_shape(out(0), s);
+      }
+    } else if (op == "MaxUnpool") {                                 // F^fs_ISVDOS: output_shape input (values), else from the window
+      const ShapeVal& x = S(in(0));
+      g.tensors[out(0)].dtype = g.tensors[in(0)].dtype;
+      if (n.ins.size() > 2) {
+        const ValueVal& v = V(in(2));
+        if (v.kind == ValueVal::KNOWN) { ShapeVal s; s.rank = static_cast<int>(v.elems.size()); s.dims = v.elems; ch |= refine_shape(out(0), s); }
+        else if (v.kind == ValueVal::NAC && x.rank >= 0) { ShapeVal s; s.rank = x.rank; s.dims.assign(x.rank, Dim::nac()); ch |= refine_shape(out(0), s); }
+      } else if (x.rank == 4) {
+        const int64_t k = n.attr_i("kernel", 2), s_ = n.attr_i("stride", k), p = n.attr_i("pad", 0);
+        ShapeVal s; s.rank = 4; s.dims = {x.dims[0], x.dims[1], x.dims[2], x.dims[3]};
+        for (int d = 2; d < 4; ++d)
+          if (x.dims[d].known()) s.dims[d] = Dim::val((x.dims[d].e - Expr(1)) * Expr(s_) + Expr(k - 2 * p));
+        ch |= refine_shape(out(0), s);
+      }
+    } else if (op == "NonMaxSuppression") {                         // F^fs_EDO: [selected, 3], the count known only after execution
+      const ShapeVal& sc = S(in(1));                                // scores [batch, classes, boxes]
+      g.tensors[out(0)].dtype = DType::I64;
+      if (sc.rank >= 0) {
+        int sym = g.cx.symbol("nms(" + g.tensors[in(1)].name + ")", 0, INT64_MAX, true);
+        if (sc.fully_known()) g.cx.atoms[sym].hi_expr = std::make_shared<Expr>(numel(sc));
+        ShapeVal s; s.rank = 2; s.dims = {Dim::val(Expr::atom(sym)), Dim::c(3)};
+        ch |= refine_shape(out(0), s);
+        ValueVal v; v.kind = ValueVal::NAC;
+        ch |= refine_value(out(0), v);
+      }
     } else {
       fail(E_UNSUPPORTED_OP, "no transfer function for " + op);
     }
