@@ -54,6 +54,7 @@ def _load() -> C.CDLL:
         "sod2_graph_set_plan_cache": [vp, i32],
         "sod2_plan_cached": [vp, i32, i32, P(cp), P(i64), P(vp), P(vp), P(sz), P(i32)],
         "sod2_run": [vp, P(vp), P(vp), vp, sz, vp, P(RunInfo)],
+        "sod2_run_graph": [vp, P(vp), P(vp), vp, sz, vp, P(RunInfo)],
         "sod2_run_timed": [vp, P(vp), P(vp), vp, sz, vp, P(C.c_float), i32],
         "sod2_plan_device_status": [vp, vp, vp],
         "sod2_graph_tensor_info": [vp, cp, P(i32), P(i32), cp, sz],
@@ -91,7 +92,7 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = ["sod2_graph_create", "sod2_graph_destroy", "sod2_graph_set_const", "sod2_graph_prepack_bytes",
            "sod2_graph_prepack", "sod2_bind_dims", "sod2_binding_destroy", "sod2_plan", "sod2_plan_destroy", "sod2_graph_set_plan_cache", "sod2_plan_cached",
-           "sod2_run", "sod2_run_timed", "sod2_plan_device_status", "sod2_graph_tensor_info", "sod2_graph_tensor_value", "sod2_graph_tensor_dtype",
+           "sod2_run", "sod2_run_graph", "sod2_run_timed", "sod2_plan_device_status", "sod2_graph_tensor_info", "sod2_graph_tensor_value", "sod2_graph_tensor_dtype",
            "sod2_graph_num_ops", "sod2_graph_op_info", "sod2_graph_num_groups", "sod2_graph_group_info",
            "sod2_graph_num_subgraphs", "sod2_graph_rdp_sweeps", "sod2_classify", "sod2_graph_reanalyse", "sod2_graph_order_info",
            "sod2_binding_shape", "sod2_plan_slot", "sod2_plan_instance_offset", "sod2_plan_memory", "sod2_plan_group_cost", "sod2_plan_tensor_strides",
@@ -279,6 +280,14 @@ class Plan:
         outs = (C.c_void_p * max(len(outputs), 1))(*outputs)
         info = RunInfo()
         _check(lib.sod2_run(self.h, ins, outs, C.c_void_p(arena), arena_bytes, C.c_void_p(stream), C.byref(info)), self.h)
+        return info
+
+    def run_graph(self, inputs: Sequence[int], outputs: Sequence[int], arena: int, arena_bytes: int, stream: int) -> RunInfo:
+        """The same inference as one CUDA graph (captured on first use and when a buffer pointer changes)."""
+        ins = (C.c_void_p * max(len(inputs), 1))(*inputs)
+        outs = (C.c_void_p * max(len(outputs), 1))(*outputs)
+        info = RunInfo()
+        _check(lib.sod2_run_graph(self.h, ins, outs, C.c_void_p(arena), arena_bytes, C.c_void_p(stream), C.byref(info)), self.h)
         return info
 
     def run_timed(self, inputs: Sequence[int], outputs: Sequence[int], arena: int, arena_bytes: int, stream: int) -> List[float]:

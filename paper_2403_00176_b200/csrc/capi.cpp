@@ -222,6 +222,24 @@ sod2_status sod2_run(sod2_plan_t* p, const void* const* inputs, void* const* out
   return st(s);
 }
 
+sod2_status sod2_run_graph(sod2_plan_t* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes,
+                           void* stream, sod2_run_info* info) {
+  if (!p || !inputs || !outputs) return SOD2_E_INVALID_ARG;
+  const Graph& G = p->g->c.g;
+  for (size_t i = 0; i < G.inputs.size(); ++i) if (!inputs[i]) { p->h.err = "null input"; return SOD2_E_INVALID_ARG; }
+  for (size_t i = 0; i < G.outputs.size(); ++i) if (!outputs[i]) { p->h.err = "null output"; return SOD2_E_INVALID_ARG; }
+  for (int c : G.consts) {
+    bool used = false;
+    for (auto& grp : p->g->c.groups) for (int t : grp.ext_in) if (t == c) used = true;
+    if (used && !G.tensors[c].dev_ptr) { p->h.err = "constant " + G.tensors[c].name + " has no device data"; return SOD2_E_INVALID_ARG; }
+  }
+  int64_t inf[8] = {0};
+  Status s = run_plan_graph(&p->p, inputs, outputs, arena, arena_bytes, stream, inf);
+  if (s != OK) p->h.err = p->p.err;
+  if (info) { info->host_enqueue_ns = inf[0]; info->gpu_launches = inf[1]; info->reserved[1] = inf[3]; }
+  return st(s);
+}
+
 sod2_status sod2_run_timed(sod2_plan_t* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes,
                            void* stream, float* group_ms, int n_groups) {
   if (!p || !inputs || !outputs || !arena) return SOD2_E_INVALID_ARG;

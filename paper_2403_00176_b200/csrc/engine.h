@@ -190,8 +190,21 @@ struct Plan {
   std::vector<double> group_flops, group_bytes;   // algorithmic cost per group for the bound shapes
   std::string err;
   // device status word lives at arena offset 0 (first 256 bytes reserved)
+  // CUDA graph of the whole launch sequence for one set of buffers (run_plan_graph)
+  void* graph_exec = nullptr;             // cudaGraphExec_t
+  void* capture_stream = nullptr;         // cudaStream_t the sequence is captured on
+  std::vector<const void*> graph_key;     // inputs, outputs, arena the graph was captured with
+  Plan() = default;
+  Plan(const Plan&) = delete;
+  Plan& operator=(const Plan&) = delete;
+  ~Plan();                                // exec.cu: releases the graph and the capture stream
 };
 Status make_plan(const Compiled* c, const Binding* b, Plan* p);
+// The launch sequence of run_plan as one CUDA graph: captured (on a stream of the plan's own, so that
+// the caller may pass the legacy default stream) the first time and whenever an input, output or arena
+// pointer differs from the captured ones, then replayed on `stream`.  info[3] = 1 if this call captured.
+Status run_plan_graph(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream,
+                      int64_t* info);
 Status build_launches(Plan* p);   // exec.cu
 Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream,
                 int64_t* info);

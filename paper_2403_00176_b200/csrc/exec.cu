@@ -1442,6 +1442,55 @@ Status run_plan_timed(Plan* p, const void* const* inputs, void* const* outputs, 
   return st;
 }
 
+Plan::~Plan() {
+  if (graph_exec) cudaGraphExecDestroy(static_cast<cudaGraphExec_t>(graph_exec));
+  if (capture_stream) cudaStreamDestroy(static_cast<cudaStream_t>(capture_stream));
+}
+
+Status run_plan_graph(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream,
+                      int64_t* info) {
+  const Graph& G = p->c->g;
+  std::vector<const void*> key;
+  key.reserve(G.inputs.size() + G.outputs.size() + 1);
+  for (size_t i = 0; i < G.inputs.size(); ++i) key.push_back(inputs[i]);
+  for (size_t i = 0; i < G.outputs.size(); ++i) key.push_back(outputs[i]);
+  key.push_back(arena);
+  auto t0 = std::chrono::steady_clock::now();
+  int64_t captured = 0;
+  if (!p->graph_exec || key != p->graph_key) {
+    if (p->graph_exec) { cudaGraphExecDestroy(static_cast<cudaGraphExec_t>(p->graph_exec)); p->graph_exec = nullptr; }
+    if (!p->capture_stream) {
+      cudaStream_t cs;
+      if (cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking) != cudaSuccess) { p->err = "cannot create the capture stream"; return E_CUDA; }
+      p->capture_stream = cs;
+    }
+    cudaStream_t cs = static_cast<cudaStream_t>(p->capture_stream);
+    if (cudaStreamBeginCapture(cs, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { p->err = "cannot begin the stream capture"; return E_CUDA; }
+    Status s = run_plan(p, inputs, outputs, arena, arena_bytes, cs, nullptr);
+    cudaGraph_t graph = nullptr;
+    const cudaError_t e = cudaStreamEndCapture(cs, &graph);     // always ended, also after a failed launch
+    if (s != OK) { if (graph) cudaGraphDestroy(graph); cudaGetLastError(); return s; }
+    if (e != cudaSuccess || !graph) { p->err = std::string("stream capture failed: ") + cudaGetErrorString(e); cudaGetLastError(); return E_CUDA; }
+    cudaGraphExec_t exec = nullptr;
+    const cudaError_t ei = cudaGraphInstantiate(&exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (ei != cudaSuccess) { p->err = std::string("graph instantiation failed: ") + cudaGetErrorString(ei); cudaGetLastError(); return E_CUDA; }
+    p->graph_exec = exec;
+    p->graph_key = key;
+    captured = 1;
+  } else {
+    if (arena_bytes < p->arena_bytes) { p->err = "arena too small"; return E_ARENA_TOO_SMALL; }
+  }
+  const cudaError_t el = cudaGraphLaunch(static_cast<cudaGraphExec_t>(p->graph_exec), static_cast<cudaStream_t>(stream));
+  if (el != cudaSuccess) { p->err = std::string("graph launch failed: ") + cudaGetErrorString(el); return E_CUDA; }
+  if (info) {
+    info[0] = std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t0).count();
+    info[1] = p->gpu_launches;
+    info[3] = captured;
+  }
+  return OK;
+}
+
 Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream, int64_t* info) {
   if (!arena && p->arena_bytes) { p->err = "arena is null"; return E_INVALID_ARG; }
   if (arena_bytes < p->arena_bytes) { p->err = "arena too small"; return E_ARENA_TOO_SMALL; }

@@ -68,6 +68,20 @@ def measure(cfg: int, reps: int, oracle_budget: float):
         e1.record(stream)
         torch.cuda.synchronize(dev)
         times.append(e0.elapsed_time(e1))
+    # the same batches, each replayed as one CUDA graph (captured beforehand)
+    for p in preps:
+        p.run_graph()
+    torch.cuda.synchronize(dev)
+    gtimes = []
+    for i in range(reps):
+        flush.fill_(i & 0xFF)
+        p = preps[i % len(preps)]
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        p.run_graph()
+        e1.record(stream)
+        torch.cuda.synchronize(dev)
+        gtimes.append(e0.elapsed_time(e1))
     # per-group roofline on the first batch
     rep = PF.group_report(preps[0], hbm, tf, reps=5)
     kinds = PF.kind_summary(rep)
@@ -120,6 +134,7 @@ def measure(cfg: int, reps: int, oracle_budget: float):
     n_req = len(reqs0) if cfg != 5 else reqs0[0].inputs["x"].shape[0]
     return {
         "cfg": cfg, "workload": wl.name, "ms_median": float(np.median(times)), "ms_min": float(np.min(times)),
+        "ms_graph_median": float(np.median(gtimes)), "ms_graph_min": float(np.min(gtimes)),
         "ms_per_request": float(np.median(times)) / n_req, "units_batch0": units, "unit": uname,
         "sum_t_roof_over_sum_t_groups": sum_roof / sum_ms, "sum_t_roof_over_t_step": sum_roof / float(np.median(times)),
         "worst_group": {"kind": worst["kind"], "frac": worst["frac"], "bound": worst["bound"], "ms": worst["ms"]},
@@ -143,10 +158,10 @@ def main():
         r.pop("gpu_launches", None)
         print(json.dumps(r), flush=True)
         rows.append(r)
-    print("\n| cfg | ms per inference (median, min) | ms per request | sum t_roof / t_step | worst group: fraction, bound | bind+plan us (cache hit) | arena / peak-live MB | oracle ms (cores) |")
-    print("|---|---|---|---|---|---|---|---|")
+    print("\n| cfg | ms per inference (median, min) | as one CUDA graph (median, min) | ms per request | sum t_roof / t_step | worst group: fraction, bound | bind+plan us (cache hit) | arena / peak-live MB | oracle ms (cores) |")
+    print("|---|---|---|---|---|---|---|---|---|")
     for r in rows:
-        print(f"| {r['cfg']} | {r['ms_median']:.3f}, {r['ms_min']:.3f} | {r['ms_per_request']:.4f} | {r['sum_t_roof_over_t_step']:.3f} | "
+        print(f"| {r['cfg']} | {r['ms_median']:.3f}, {r['ms_min']:.3f} | {r['ms_graph_median']:.3f}, {r['ms_graph_min']:.3f} | {r['ms_per_request']:.4f} | {r['sum_t_roof_over_t_step']:.3f} | "
               f"{r['worst_group']['kind']}: {r['worst_group']['frac']:.3f}, {r['worst_group']['bound']} | {r['plan_us_median']:.0f} ({r['plan_us_cache_hit'] or 0:.0f}) | "
               f"{r['arena_bytes'] / 1e6:.1f} / {r['peak_live_bytes'] / 1e6:.1f} | {r['oracle_ms']:.0f} ({r['oracle_cores']}) |")
 

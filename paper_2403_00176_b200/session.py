@@ -95,6 +95,11 @@ class Prepared:
         return self.plan.run([t.data_ptr() for t in self.in_dev], [t.data_ptr() for t in self.out_dev],
                              self.arena.data_ptr(), self.arena.numel(), self.s.stream)
 
+    def run_graph(self) -> B.RunInfo:
+        """The inference as one CUDA graph over this batch's own buffers (captured by the first call)."""
+        return self.plan.run_graph([t.data_ptr() for t in self.in_dev], [t.data_ptr() for t in self.out_dev],
+                                   self.arena.data_ptr(), self.arena.numel(), self.s.stream)
+
     def check_device_status(self):
         self.plan.device_status(self.arena.data_ptr(), self.s.stream)
 

@@ -172,6 +172,32 @@ def test_cfg2_plan_cache_reuses_a_plan_with_other_buffers():
             assert np.array_equal(outs[r]["y"], o1[r]["y"])
 
 
+def test_cuda_graph_replay_matches_stream_launches():
+    # the whole launch sequence as one CUDA graph: captured by the first call, replayed by the next,
+    # captured again for other buffers; bit-identical to the stream launches.  All kernel kinds: encoder
+    # (GEMM, attention, LayerNorm), token pruning (scores, top-k), gated convolutions (device-side counts).
+    cases = [(WL.cfg2(layers=2, D=128, H=2, F=256), "y"), (WL.cfg3(layers=2, D=128, H=2, F=256), None),
+             (WL.cfg5(B=6, side=32, widths=(64, 128), per_stage=2), None)]
+    for wl, _ in cases:
+        reqs = wl.batch(0)
+        s = Session(wl)
+        a, b = s.prepare(reqs), s.prepare(reqs)          # two sets of buffers, one plan each
+        a.run()
+        a.check_device_status()
+        ref = a.outputs()
+        i1 = a.run_graph(); a.check_device_status(); o1 = a.outputs()
+        i2 = a.run_graph(); a.check_device_status(); o2 = a.outputs()
+        assert i1.reserved[1] == 1 and i2.reserved[1] == 0 and i1.gpu_launches == i2.gpu_launches > 0
+        # the same plan with the other buffers: a new capture
+        i3 = a.plan.run_graph([t.data_ptr() for t in b.in_dev], [t.data_ptr() for t in b.out_dev], b.arena.data_ptr(), b.arena.numel(), s.stream)
+        assert i3.reserved[1] == 1
+        o3 = b.outputs()
+        for r in range(len(reqs)):
+            for name in ref[r]:
+                assert np.array_equal(ref[r][name], o1[r][name]) and np.array_equal(ref[r][name], o2[r][name]), (wl.name, name)
+                assert np.array_equal(ref[r][name], o3[r][name]), (wl.name, name)
+
+
 def test_cfg2_full_config_batch0():
     wl = WL.cfg2()
     reqs = wl.batch(0)
