@@ -310,6 +310,17 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ Conv3Batch B, const __grid_con
 #pragma unroll
           for (int g = 0; g < 4; ++g) *reinterpret_cast<uint4*>(obase + (((half * 4 + g) ^ (row & 7)) << 4)) = pk[g];
         }
+        if (p.gap_sum) {
+          conv_epi_bar();                               // every row of the tile is in the staging buffer
+          if (live) {
+            int n0g, img, h0, w0;
+            const int rq = decode(t, &n0g, &img, &h0, &w0);
+            const int img_o = p.out_ids ? p.out_ids[img] : img;
+            const int wo = B.Wo[rq];
+            gap_accumulate_tile(out_stage + bsel * CONV_STAGE_OUT, et, p.gap_sum + static_cast<long long>(img_o) * p.Cout + np,
+                                [&](int px) { return w0 + px < wo; });
+          }
+        }
         ptx::fence_proxy_async();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&stage_ready[bsel]);

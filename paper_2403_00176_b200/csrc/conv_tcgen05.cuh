@@ -40,6 +40,11 @@ struct ConvParams {
   const int* res_ids;
   const int* out_ids;
   const __nv_bfloat16* bias; // [Cout] or nullptr
+  // optional: per-(image, channel) sums of the stored (bf16) outputs, added with fp64 atomics to
+  // gap_sum[image id][Cout] -- the global-average-pool numerators of the next gate, accumulated where the
+  // tensor is produced instead of re-reading it (a decision scalar: the order of the fp64 additions moves
+  // it by less than n * 2^-53, far inside the band in which decisions are compared)
+  double* gap_sum;
   int has_residual;
   int act2;                  // ACT_NONE or ACT_RELU after the residual add
   int* status;
@@ -61,6 +66,27 @@ __device__ __forceinline__ void tma_store_4d(const void* tmap, const void* src, 
                ::"l"(tmap), "r"(ptx::smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
 __device__ __forceinline__ void conv_epi_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// Sum over the valid pixels of one staged [128 pixels x 64 channels] bf16 tile (128-byte rows, 16-byte
+// granules XOR-ed with the row), by the 256 epilogue threads, in fp64 (a bf16 value is exact in fp64; masked
+// pixels add +0.0).  valid(px) tells whether tile pixel px lies in the image.
+template <typename Valid>
+__device__ __forceinline__ void gap_accumulate_tile(const uint8_t* stage, int et, double* dst_row, Valid valid) {
+  // thread (channel pair et & 31, pixel group et >> 5): 16 pixels x 2 channels, one 32-bit shared load per
+  // pixel, four independent fp64 chains (even / odd pixels x two channels), then two atomics
+  const int chp = et & 31, pg = et >> 5;
+  double a0 = 0.0, a1 = 0.0, b0 = 0.0, b1 = 0.0;
+#pragma unroll
+  for (int i = 0; i < 16; i += 2) {
+    const int px0 = pg * 16 + i, px1 = px0 + 1;
+    const uint32_t w0 = valid(px0) ? *reinterpret_cast<const uint32_t*>(stage + px0 * 128 + ((((chp >> 2) ^ (px0 & 7)) << 4) + (chp & 3) * 4)) : 0u;
+    const uint32_t w1 = valid(px1) ? *reinterpret_cast<const uint32_t*>(stage + px1 * 128 + ((((chp >> 2) ^ (px1 & 7)) << 4) + (chp & 3) * 4)) : 0u;
+    a0 += static_cast<double>(__uint_as_float(w0 << 16)); a1 += static_cast<double>(__uint_as_float(w0 & 0xffff0000u));
+    b0 += static_cast<double>(__uint_as_float(w1 << 16)); b1 += static_cast<double>(__uint_as_float(w1 & 0xffff0000u));
+  }
+  atomicAdd(dst_row + 2 * chp, a0 + b0);
+  atomicAdd(dst_row + 2 * chp + 1, a1 + b1);
+}
 
 // tmX: {Cin, W, H, N} bf16, box {64, TW, TH, 1}, element strides {1, s, s, 1}
 // tmW: {64, Cout, K/64} k-chunk view of [Cout, K], box {64, BN, KCH}
@@ -275,6 +301,12 @@ conv_igemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmX, const __grid_co
         if (et == 0 && live) {
           tma_store_4d(&tmOut, out_stage, np, wo0, ho0, img_o);
           bulk_commit();
+        }
+        if (p.gap_sum && live) {
+          const int tw_shift = __ffs(p.TW) - 1;      // TW * TH == 128: a power of two
+          gap_accumulate_tile(out_stage, et, p.gap_sum + static_cast<long long>(img_o) * p.Cout + np, [&](int px) {
+            return ho0 + (px >> tw_shift) < p.Ho && wo0 + (px & (p.TW - 1)) < p.Wo;
+          });
         }
       }
     }
@@ -593,7 +625,7 @@ struct PartitionParams {
   long long* count_exec;           // the run-time symbol's slot in the arena header
   long long* count_skip;
 };
-__device__ __forceinline__ void partition_by_gate(const PartitionParams& p, int lane) {
+__device__ __forceinline__ int partition_by_gate(const PartitionParams& p, int lane) {
   int ne = 0, ns = 0;
   for (int base = 0; base < p.n; base += 32) {
     const int i = base + lane;
@@ -607,6 +639,7 @@ __device__ __forceinline__ void partition_by_gate(const PartitionParams& p, int 
     ns += __popc(bs);
   }
   if (lane == 0) { *p.count_exec = ne; *p.count_skip = ns; }
+  return ne;
 }
 
 // Gate of a skip block (decision scalar): z[n] = sum_c w[c] * mean_hw x[n,:,:,c] + b, gate[n] = z[n] > 0,
@@ -626,10 +659,13 @@ struct GateParams {
   // clears the arena header) and is left at zero.
   int* ticket;
   PartitionParams part;
+  // zero_rows != nullptr: the last CTA also clears the rows of the executed samples in the [N, C] table of
+  // per-sample channel sums, which the block's last convolution then accumulates anew (ConvParams::gap_sum)
+  double* zero_rows;
 };
 __global__ void __launch_bounds__(256) gate_logit_f64(GateParams p) {
   __shared__ double red[256];
-  __shared__ int last_cta;
+  __shared__ int last_cta, n_exec;
   ptx::pdl_wait();
   ptx::pdl_launch();
   const int img = blockIdx.x;
@@ -663,10 +699,20 @@ __global__ void __launch_bounds__(256) gate_logit_f64(GateParams p) {
   }
   if (p.ticket) {
     __syncthreads();
-    if (last_cta && threadIdx.x < 32) {
-      __threadfence();
-      partition_by_gate(p.part, threadIdx.x);
-      if (threadIdx.x == 0) *p.ticket = 0;
+    if (last_cta) {
+      if (threadIdx.x < 32) {
+        __threadfence();
+        const int ne = partition_by_gate(p.part, threadIdx.x);
+        if (threadIdx.x == 0) { *p.ticket = 0; n_exec = ne; }
+      }
+      if (p.zero_rows) {
+        __syncthreads();                                  // uniform over the CTA: last_cta is shared
+        // a warp per executed sample: the id is read once, the lanes clear the row
+        for (int k2 = threadIdx.x >> 5; k2 < n_exec; k2 += 8) {
+          double* rowp = p.zero_rows + static_cast<long long>(p.part.idx_exec[k2]) * p.C;
+          for (int cc = threadIdx.x & 31; cc < p.C; cc += 32) rowp[cc] = 0.0;
+        }
+      }
     }
   }
 }

@@ -826,6 +826,9 @@ struct Builder {
     for (size_t i = 0; i < c.packed_consts.size(); ++i) if (c.packed_consts[i] == G.w) pk = c.packed_off[i];
     const int bn = (Cout % 128 == 0) ? 128 : 64;
     const int kch = 2;
+    // the table of per-sample channel sums this convolution adds its outputs to (the last convolution of an
+    // in-place gated block), or SIZE_MAX
+    const size_t gap_table = gap_accum.count(gi) ? gap_accum[gi] : SIZE_MAX;
     // requests that take the row-halo kernel are collected and launched together (up to C3_MAX_REQ per launch)
     struct RowsReq { Ptr px, po, pr; int H, W, Ho, Wo, n_img, n_in_map, n_out_map, n_res_map; k::ConvParams cp; bool rt; size_t rt_slot; long long ids_in, ids_res, ids_out; };
     std::vector<RowsReq> rows_reqs;
@@ -876,6 +879,7 @@ struct Builder {
         cp.in_ids = batch[0].ids_in >= 0 ? reinterpret_cast<const int*>(auxb + batch[0].ids_in) : nullptr;
         cp.res_ids = batch[0].ids_res >= 0 ? reinterpret_cast<const int*>(auxb + batch[0].ids_res) : nullptr;
         cp.out_ids = batch[0].ids_out >= 0 ? reinterpret_cast<const int*>(auxb + batch[0].ids_out) : nullptr;
+        cp.gap_sum = (gap_table != SIZE_MAX && batch.size() == 1) ? reinterpret_cast<double*>(const_cast<char*>(auxb) + gap_table) : nullptr;
         const dim3 gd(static_cast<unsigned>(std::min<long long>(tiles, x.plan->sm_count)));
         const int variant = ((wres ? 4 : 0) + (bn == 128 ? 2 : 0) + (act == 2 ? 1 : 0)) * 2 + (hr ? 1 : 0);
 #define SOD2_CONV3_CASE(V, BN_, RES_, ST_, ACT_, HR_)                                                                    \
@@ -990,6 +994,7 @@ struct Builder {
         cp.in_ids = ids_in >= 0 ? reinterpret_cast<const int*>(auxb + ids_in) : nullptr;
         cp.res_ids = ids_res >= 0 ? reinterpret_cast<const int*>(auxb + ids_res) : nullptr;
         cp.out_ids = ids_out >= 0 ? reinterpret_cast<const int*>(auxb + ids_out) : nullptr;
+        cp.gap_sum = gap_table != SIZE_MAX ? reinterpret_cast<double*>(const_cast<char*>(auxb) + gap_table) : nullptr;
         const dim3 gd(static_cast<unsigned>(std::min<long long>(tiles, x.plan->sm_count))), bd(k::CONV_THREADS);
         const int variant = ((bn == 128 ? 2 : 0) + (act == 2 ? 1 : 0)) * 2 + (hr ? 1 : 0);
 #define SOD2_CONV_CASE(V, BN_, KCH_, ST_, ACT_, HR_)                                                                     \
@@ -1051,6 +1056,12 @@ struct Builder {
   size_t aux_need = 0;
   std::set<int> partition_fused;      // gate tensors whose id partition is computed by the gate kernel
   int n_tickets = 0;
+  // Per-sample channel sums carried from gate to gate (aux region): `gapsum_root` is the storage root whose
+  // current contents the table at `gapsum_aux` describes.  A gate on that storage skips the pooling pass; the
+  // last convolution of an in-place block (group index in gap_accum) adds the executed samples' new sums.
+  int gapsum_root = -1;
+  size_t gapsum_aux = 0;
+  std::map<int, size_t> gap_accum;    // convolution group -> offset of the table it accumulates into
 
   // ------------------------------------------------------------------------------ gate (decision scalar)
   Status build_gate(int gi, const Group& G) {
@@ -1090,22 +1101,64 @@ struct Builder {
           break;
         }
       }
-      add(gi, 2, [=](const RunCtx& x) mutable {
+      // Per-sample channel sums: reuse the table if it describes this tensor's storage, else pool (two
+      // launches) into a new table.  If the block is an in-place, index-indirect one, its last convolution
+      // accumulates the executed samples' sums into the table and the next gate finds it up to date.
+      const int xroot = vx.root;
+      const bool whole = vx.offset == 0 && vx.ind_gate < 0;
+      const bool have_sums = fuse_part && whole && gapsum_root >= 0 && gapsum_root == xroot;
+      size_t table = gapsum_aux;
+      bool keep_table = false;
+      if (fuse_part && whole) {
+        if (!have_sums) { table = aux_need; aux_need += (static_cast<size_t>(N) * gp.C * 8 + 255) & ~size_t(255); }
+        // look ahead: Switch on this gate -> index-indirect -> Combine whose output lives in this storage -> its writer
+        int writer = -1;
+        bool in_place = false;          // the block overwrites this storage
+        for (size_t ci = 0; ci < c.groups.size() && writer < 0; ++ci) {
+          const Group& Cb = c.groups[ci];
+          if (Cb.kind != GKind::COMBINE || Cb.gate != G.out || c.storage[Cb.out].kind != Storage::ALIAS) continue;
+          if (p.views[Cb.out].empty() || p.views[Cb.out][0].root != xroot) continue;
+          in_place = true;
+          for (size_t wi = 0; wi < c.groups.size(); ++wi) {
+            const Group& Wg = c.groups[wi];
+            if (Wg.kind == GKind::CONV && Wg.out >= 0 && c.storage[Wg.out].kind == Storage::INDIRECT_OUT && c.storage[Wg.out].other == Cb.out &&
+                g.tensors[Wg.w].S.dims[1].e.const_value() % 64 == 0) { writer = static_cast<int>(wi); break; }
+          }
+        }
+        // accumulating in the convolution's epilogue costs about as much per byte as the pooling pass it
+        // replaces; what it saves is the pass's two launches, which only outweighs it on the smaller tensors
+        if (writer >= 0 && static_cast<double>(N) * gp.C * static_cast<double>(gp.HW) * 2.0 > 32e6) writer = -1;
+        if (writer >= 0) { gap_accum[writer] = table; keep_table = true; }
+        gapsum_root = (in_place && writer < 0) ? -1 : xroot;   // overwritten without the sums being kept: the table goes stale
+        gapsum_aux = table;
+      }
+      const bool zero_exec = keep_table;
+      const bool pool = !have_sums;
+      const bool to_table = fuse_part && whole;     // sums go to the aux table (else: slab partials in scratch, as before)
+      add(gi, pool ? (to_table ? 3 : 2) : 1, [=](const RunCtx& x) mutable {
+        char* auxb = x.arena + x.plan->scratch_off[1];
+        double* sums = reinterpret_cast<double*>(auxb + table);
         gp.x = reinterpret_cast<const __nv_bfloat16*>(x.resolve(px));
         gp.partial = reinterpret_cast<double*>(x.arena + x.plan->scratch_off[0]);
         k::GapBatch gb{};
         gb.n_seg = 1; gb.img_start[0] = 0; gb.img_start[1] = N; gb.seg[0] = gp;
-        launch_pdl(k::gap_partial_f64, dim3(1, gp.slabs, N), dim3(256), 0, x.stream, gb);
+        if (pool) {
+          launch_pdl(k::gap_partial_f64, dim3(1, gp.slabs, N), dim3(256), 0, x.stream, gb);
+          if (to_table) {          // slab partials -> sums (HW = 1: no division) in the table
+            gb.seg[0].out = nullptr; gb.seg[0].out_f64 = sums; gb.seg[0].HW = 1;
+            launch_pdl(k::gap_final_f64, dim3((N * gp.C + 7) / 8, 1), dim3(256), 0, x.stream, gb);
+          }
+        }
         k::GateParams q{};
-        q.partial = gp.partial;
+        q.partial = to_table ? sums : gp.partial;
         q.w = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pw));
         q.b = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pb));
         q.gate = reinterpret_cast<unsigned char*>(x.resolve(pg));
         q.z_out = want_z ? x.resolve(pz) : nullptr;
         q.z_bf16 = zb;
-        q.C = gp.C; q.slabs = gp.slabs; q.HW = gp.HW;
+        q.C = gp.C; q.slabs = to_table ? 1 : gp.slabs; q.HW = gp.HW;
         if (fuse_part) {
-          char* auxp = x.arena + x.plan->scratch_off[1] + part_aux;
+          char* auxp = auxb + part_aux;
           q.ticket = reinterpret_cast<int*>(x.arena + 128) + ticket;
           q.part.gate = q.gate;
           q.part.n = N;
@@ -1113,6 +1166,7 @@ struct Builder {
           q.part.idx_skip = q.part.idx_exec + N;
           q.part.count_exec = reinterpret_cast<long long*>(x.arena + part_slot);
           q.part.count_skip = reinterpret_cast<long long*>(auxp + 2 * N * 4);
+          q.zero_rows = zero_exec ? sums : nullptr;
         }
         launch_pdl(k::gate_logit_f64, dim3(N), dim3(256), 0, x.stream, q);
         return cudaGetLastError();
