@@ -5,13 +5,15 @@
 // With three input channels neither TMA im2col nor a channels-last box applies (a pixel is 6 bytes), and
 // materialising the [pixels, 147 -> 192] patch matrix costs 16 x the input in traffic.  Here a CTA
 // owns a segment of up to 128 pixels of one output row.  The 7 input rows x 3 channels the segment
-// needs are copied into shared memory (16-byte cp.async, zero filled outside the image), and the
+// needs are copied into shared memory (six TMA boxes of 7 rows x 144 columns per tile: three channels x
+// two overlapping column halves, zero filled outside the image; for images whose width is not a multiple
+// of 8 the builder warps copy them instead), and the
 // A tile [128 pixels x 192] is built from them in the 128-byte-swizzled K-major layout: K is ordered
 // (dy, ci, dx') with dx' = dx + 1 in 0..7, so that one 16-byte unit of a pixel's row of A is eight
 // consecutive input columns starting at the even column 2*ox - 4 -- four aligned 32-bit shared loads.
 // dx' = 0 carries a zero weight (and is zeroed in A), units 21..23 are zero padding: K = 24 x 8.
-//   warp 0       weights (24 KB, resident) by TMA
-//   warps 1..8   builders: patch copy (three-deep ring), A tile (double buffered)
+//   warp 0       weights (24 KB, resident) and the input patches (three-deep ring) by TMA
+//   warps 1..8   builders: A tile (double buffered) from the patch
 //   warps 9..12  epilogue: TMEM -> +bias -> activation -> bf16 -> swizzled staging -> TMA store
 //   warp 13      MMA issuer: 12 x tcgen05.mma (M=128, N=64, K=16) per tile into one of two accumulators
 // Persistent, one CTA per SM.  Every wait is bounded (ptx.cuh).
@@ -32,10 +34,13 @@ struct StemParams {
 constexpr int STEM_THREADS = 448;
 constexpr int STEM_PITCH = 272;                       // patch columns: 2 * 128 + 16
 constexpr int STEM_ROWS = 21;                         // (dy, ci)
-constexpr int STEM_PATCH_BYTES = 11520;               // 21 * 272 * 2 = 11424, rounded up to a multiple of 128
+constexpr int STEM_PATCH_BYTES = 12288;               // 21 rows x 272 columns (11424 B), or six TMA boxes 2048 B apart
 constexpr int STEM_A_BYTES = 3 * 128 * 128;           // three k-chunks of [128 x 64]
 constexpr int STEM_W_BYTES = 3 * 64 * 128;
 constexpr int STEM_OUT_BYTES = 128 * 128;
+constexpr int STEM_BOX_W = 144;                       // columns of a TMA box: two of them, 128 apart, cover the 272 patch columns
+constexpr int STEM_BOX_BYTES = 7 * STEM_BOX_W * 2;    // one TMA box: 7 input rows (2016 B)
+constexpr int STEM_BOX_STRIDE = 2048;                 // boxes 2048 B apart: a TMA destination is 128-byte aligned
 constexpr int STEM_SMEM = STEM_W_BYTES + 2 * STEM_A_BYTES + 2 * STEM_OUT_BYTES + 3 * STEM_PATCH_BYTES + 256 /*bias*/ + 128 /*barriers*/ + 1024 /*align*/;
 
 // Weights [64, 3, 7, 7] -> [64, 192] in the (dy, ci, dx') order of the kernel, zero where dx' = 0 or unit >= 21.
@@ -51,9 +56,11 @@ __global__ void reorder_stem_weights(const __nv_bfloat16* __restrict__ w, __nv_b
   }
 }
 
-template <int ACT>
+// TMA_PATCH: tmX is a map {W, H, N * 3} of the input with boxes {144, 7, 1} (W % 8 == 0); otherwise tmX is unused.
+template <int ACT, bool TMA_PATCH>
 __global__ void __launch_bounds__(STEM_THREADS, 1)
-conv_stem_bf16_tcgen05(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmOut, const StemParams p) {
+conv_stem_bf16_tcgen05(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmOut,
+                       const __grid_constant__ CUtensorMap tmX, const StemParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sW = base;
@@ -67,7 +74,9 @@ conv_stem_bf16_tcgen05(const __grid_constant__ CUtensorMap tmW, const __grid_con
   uint64_t* a_free = bars + 3;        // [2] the MMAs that read A[b] have completed
   uint64_t* acc_full = bars + 5;      // [2]
   uint64_t* acc_free = bars + 7;      // [2] the epilogue warps have drained accumulator b
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 9);
+  uint64_t* patch_full = bars + 9;    // [3] the tile's six boxes have landed
+  uint64_t* patch_free = bars + 12;   // [3] the builder warps have read the patch
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 15);
   volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -80,11 +89,13 @@ conv_stem_bf16_tcgen05(const __grid_constant__ CUtensorMap tmW, const __grid_con
       ptx::mbar_init(&a_full[b], 8); ptx::mbar_init(&a_free[b], 1);
       ptx::mbar_init(&acc_full[b], 1); ptx::mbar_init(&acc_free[b], 4);
     }
+    for (int b = 0; b < 3; ++b) { ptx::mbar_init(&patch_full[b], 1); ptx::mbar_init(&patch_free[b], 8); }
     *dead = 0;
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
     ptx::prefetch_tmap(&tmW);
     ptx::prefetch_tmap(&tmOut);
+    if (TMA_PATCH) ptx::prefetch_tmap(&tmX);
   }
   if (threadIdx.x < 64) bias_s[threadIdx.x] = p.bias ? __bfloat162float(p.bias[threadIdx.x]) : 0.0f;   // a constant of the graph
   if (warp == 13) { ptx::tmem_alloc(tmem_slot, 128); ptx::tmem_relinquish(); }
@@ -98,6 +109,23 @@ conv_stem_bf16_tcgen05(const __grid_constant__ CUtensorMap tmW, const __grid_con
     if (lane == 0) {
       ptx::mbar_expect_tx(w_full, STEM_W_BYTES);
       ptx::tma_load_3d(sW, &tmW, 0, 0, 0, w_full);
+      if constexpr (TMA_PATCH) {
+        // ---- patch producer: box (ci, half) of tile t = input rows 2*oy-3 .. 2*oy+3 of channel ci, columns
+        // 2*ox0 - 8 + 128*half .. +143 (the halves overlap by 16, so a pixel's 8 columns always lie inside one box)
+        ptx::pdl_wait();
+        int it = 0;
+        for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++it) {
+          const int s = it % 3;
+          if (it >= 3) ptx::mbar_wait(&patch_free[s], ((it / 3) - 1) & 1, dead);
+          const int rowi = t / nseg, seg = t - rowi * nseg;
+          const int n = rowi / p.Ho, oy = rowi - n * p.Ho;
+          ptx::mbar_expect_tx(&patch_full[s], 6 * STEM_BOX_BYTES);
+#pragma unroll
+          for (int bx = 0; bx < 6; ++bx)
+            ptx::tma_load_3d(sPatch + s * STEM_PATCH_BYTES + bx * STEM_BOX_STRIDE, &tmX, 256 * seg - 8 + 128 * (bx & 1), 2 * oy - 3,
+                             n * 3 + (bx >> 1), &patch_full[s]);
+        }
+      }
     }
   } else if (warp <= 8) {
     // ---- builders
@@ -157,20 +185,39 @@ conv_stem_bf16_tcgen05(const __grid_constant__ CUtensorMap tmW, const __grid_con
       asm volatile("cp.async.commit_group;" ::: "memory");
     };
     const int t0 = blockIdx.x, step = gridDim.x;
-    if (t0 < n_tiles) load_patch(t0, 0); else asm volatile("cp.async.commit_group;" ::: "memory");
-    if (t0 + step < n_tiles) load_patch(t0 + step, 1); else asm volatile("cp.async.commit_group;" ::: "memory");
+    // source offset of unit i of this thread inside a patch, per layout
+    uint32_t uoff[12];
+#pragma unroll
+    for (int i = 0; i < 12; ++i) {
+      const int u = ug + 2 * i;
+      const int dy = u / 3, ci = u - dy * 3;
+      if constexpr (TMA_PATCH) {
+        const int half = m >= 64 ? 1 : 0;   // columns 2m+4 .. 2m+11: inside box 0 (0..143) for m <= 66, box 1 (128..271) for m >= 62
+        uoff[i] = static_cast<uint32_t>((ci * 2 + half) * STEM_BOX_STRIDE + dy * (STEM_BOX_W * 2) + (2 * m + 4 - 128 * half) * 2);
+      } else {
+        uoff[i] = static_cast<uint32_t>((u * STEM_PITCH + 2 * m + 4) * 2);
+      }
+    }
+    if constexpr (!TMA_PATCH) {
+      if (t0 < n_tiles) load_patch(t0, 0); else asm volatile("cp.async.commit_group;" ::: "memory");
+      if (t0 + step < n_tiles) load_patch(t0 + step, 1); else asm volatile("cp.async.commit_group;" ::: "memory");
+    }
     int it = 0;
     for (int t = t0; t < n_tiles; t += step, ++it) {
-      // this thread's copies for tile `it` have landed (one newer group may be in flight); after the
-      // barrier so have everyone's, and every builder has finished reading the slot of tile it - 1
-      asm volatile("cp.async.wait_group 1;" ::: "memory");
-      asm volatile("bar.sync 2, 256;" ::: "memory");
+      if constexpr (TMA_PATCH) {
+        ptx::mbar_wait_warp(&patch_full[it % 3], (it / 3) & 1, dead);
+      } else {
+        // this thread's copies for tile `it` have landed (one newer group may be in flight); after the
+        // barrier so have everyone's, and every builder has finished reading the slot of tile it - 1
+        asm volatile("cp.async.wait_group 1;" ::: "memory");
+        asm volatile("bar.sync 2, 256;" ::: "memory");
+        if (t + 2 * step < n_tiles) load_patch(t + 2 * step, (it + 2) % 3); else asm volatile("cp.async.commit_group;" ::: "memory");
+      }
       if (tb == 0) { SOD2_TRACE(0, 10) }
-      if (t + 2 * step < n_tiles) load_patch(t + 2 * step, (it + 2) % 3); else asm volatile("cp.async.commit_group;" ::: "memory");
       const int buf = it & 1;
       if (it >= 2) ptx::mbar_wait_warp(&a_free[buf], ((it >> 1) - 1) & 1, dead);
       if (tb == 0) { SOD2_TRACE(0, 20) }
-      const uint8_t* patch = sPatch + (it % 3) * STEM_PATCH_BYTES;
+      const uint32_t patch = ptx::smem_u32(sPatch + (it % 3) * STEM_PATCH_BYTES);
       uint8_t* arow = sA + buf * STEM_A_BYTES + m * 128;
       // all loads first, then the stores: patch and A live in the same array, so the compiler would keep
       // every store ahead of the next unit's loads
@@ -180,7 +227,7 @@ conv_stem_bf16_tcgen05(const __grid_constant__ CUtensorMap tmW, const __grid_con
         const int u = ug + 2 * i;                       // unit = patch row (dy, ci); 21..23 are padding
         v[i] = make_uint4(0u, 0u, 0u, 0u);
         if (u < STEM_ROWS) {
-          const uint32_t sa = ptx::smem_u32(patch + (u * STEM_PITCH + 2 * m + 4) * 2);
+          const uint32_t sa = patch + uoff[i];
           asm volatile("ld.shared.b32 %0, [%4];\n\tld.shared.b32 %1, [%4+4];\n\tld.shared.b32 %2, [%4+8];\n\tld.shared.b32 %3, [%4+12];"
                        : "=r"(v[i].x), "=r"(v[i].y), "=r"(v[i].z), "=r"(v[i].w) : "r"(sa));
           v[i].x &= 0xffff0000u;                        // dx' = 0 has no tap
@@ -193,10 +240,13 @@ conv_stem_bf16_tcgen05(const __grid_constant__ CUtensorMap tmW, const __grid_con
       }
       ptx::fence_proxy_async();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&a_full[buf]);
+      if (lane == 0) {
+        ptx::mbar_arrive(&a_full[buf]);
+        if (TMA_PATCH) ptx::mbar_arrive(&patch_free[it % 3]);   // the stores above depend on every value read from the patch
+      }
       if (tb == 0) { SOD2_TRACE(0, 30) }
     }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if constexpr (!TMA_PATCH) asm volatile("cp.async.wait_group 0;" ::: "memory");
   } else if (warp == 13) {
     if (lane == 0) {
       // ---- MMA issuer

@@ -727,7 +727,7 @@ struct Builder {
         Ptr pw; pw.where = 5; pw.off = static_cast<int64_t>(pk);
         const bool hb = G.bias >= 0;
         const int act = G.act;
-        struct Cache { const void* w = nullptr; const void* o = nullptr; CUtensorMap tw, to; };
+        struct Cache { const void* w = nullptr; const void* o = nullptr; const void* xin = nullptr; CUtensorMap tw, to, tx; };
         auto cache = std::make_shared<Cache>();
         add(gi, 1, [=](const RunCtx& x) mutable {
           sp.x = reinterpret_cast<const __nv_bfloat16*>(x.resolve(px));
@@ -736,24 +736,28 @@ struct Builder {
           sp.status = reinterpret_cast<int*>(x.arena);
           const void* Wp = x.resolve(pw);
           void* O = x.resolve(po);
-          if (cache->w != Wp || cache->o != O) {
+          if (cache->w != Wp || cache->o != O || cache->xin != sp.x) {
             if (!encode_bf16_kchunks(&cache->tw, Wp, 64, 192, 192, 64, 3) ||
                 !encode_bf16_nhwc(&cache->to, O, static_cast<uint64_t>(sp.N), static_cast<uint64_t>(sp.Ho), static_cast<uint64_t>(sp.Wo), 64, 128, 1, 1))
               return cudaErrorInvalidValue;
-            cache->w = Wp; cache->o = O;
+            // input patches by TMA where the rows are 16-byte multiples; otherwise the builder warps copy them
+            if (sp.vec_ok && !encode_bf16_planes(&cache->tx, sp.x, static_cast<uint64_t>(sp.N) * 3, static_cast<uint64_t>(sp.H), static_cast<uint64_t>(sp.W), k::STEM_BOX_W, 7))
+              return cudaErrorInvalidValue;
+            if (!sp.vec_ok) cache->tx = cache->tw;      // unused by that variant
+            cache->w = Wp; cache->o = O; cache->xin = sp.x;
           }
           const long long tiles = static_cast<long long>(sp.N) * sp.Ho * ((sp.Wo + 127) / 128);
           if (tiles >= (1ll << 31)) return cudaErrorInvalidValue;
           const dim3 gd(static_cast<unsigned>(std::min<long long>(tiles, x.plan->sm_count))), bd(k::STEM_THREADS);
-          if (act == 2) {
-            static bool once = (cudaFuncSetAttribute(k::conv_stem_bf16_tcgen05<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, k::STEM_SMEM), true);
-            (void)once;
-            launch_pdl(k::conv_stem_bf16_tcgen05<2>, gd, bd, k::STEM_SMEM, x.stream, cache->tw, cache->to, sp);
-          } else {
-            static bool once = (cudaFuncSetAttribute(k::conv_stem_bf16_tcgen05<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, k::STEM_SMEM), true);
-            (void)once;
-            launch_pdl(k::conv_stem_bf16_tcgen05<0>, gd, bd, k::STEM_SMEM, x.stream, cache->tw, cache->to, sp);
+#define SOD2_STEM_CASE(ACT_, TMA_)                                                                                            \
+          {                                                                                                                  \
+            static bool once = (cudaFuncSetAttribute(k::conv_stem_bf16_tcgen05<ACT_, TMA_>, cudaFuncAttributeMaxDynamicSharedMemorySize, k::STEM_SMEM), true); \
+            (void)once;                                                                                                      \
+            launch_pdl(k::conv_stem_bf16_tcgen05<ACT_, TMA_>, gd, bd, k::STEM_SMEM, x.stream, cache->tw, cache->to, cache->tx, sp);  \
           }
+          if (act == 2) { if (sp.vec_ok) SOD2_STEM_CASE(2, true) else SOD2_STEM_CASE(2, false) }
+          else { if (sp.vec_ok) SOD2_STEM_CASE(0, true) else SOD2_STEM_CASE(0, false) }
+#undef SOD2_STEM_CASE
           return cudaGetLastError();
         });
       }

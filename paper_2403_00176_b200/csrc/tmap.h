@@ -86,4 +86,18 @@ inline bool encode_bf16_nhwc(CUtensorMap* tm, const void* base, uint64_t N, uint
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Planes of rows: bf16 [planes, H, W] (e.g. an NCHW tensor with planes = N * C) viewed as {W, H, planes};
+// box = {box_w columns, box_h rows, 1 plane}, no swizzle.  Requirements: W % 8 == 0, box_w % 8 == 0.
+inline bool encode_bf16_planes(CUtensorMap* tm, const void* base, uint64_t planes, uint64_t H, uint64_t W, uint32_t box_w, uint32_t box_h) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn || W % 8 || box_w % 8 || box_w > 256 || box_h > 256) return false;
+  cuuint64_t dims[3] = {W, H, planes};
+  cuuint64_t strides[2] = {W * 2, H * W * 2};
+  cuuint32_t box[3] = {box_w, box_h, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace sod2
