@@ -386,11 +386,33 @@ __global__ void __launch_bounds__(256) nhwc_to_nchw_bf16(const __nv_bfloat16* __
 // 64 x 64 tile goes through shared memory as rows of eight-element vectors whose position inside the row
 // is XOR-ed with the row's group of eight, so that the strided 2-byte gathers of the transposed read hit
 // distinct banks.
-__global__ void __launch_bounds__(256) nchw_to_nhwc_bf16_v8(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out,
-                                                             int C, long long HW) {
+// Up to LAYOUT_MAX_SEG tensors (the requests of a batch, each with its own image size) per launch: blockIdx.x
+// walks the 64-pixel tiles of all images of all segments.
+constexpr int LAYOUT_MAX_SEG = 8;
+struct LayoutBatch {
+  int n_seg, C;
+  int tile_start[LAYOUT_MAX_SEG + 1];        // prefix sum of images * ceil(HW / 64)
+  const __nv_bfloat16* in[LAYOUT_MAX_SEG];
+  __nv_bfloat16* out[LAYOUT_MAX_SEG];
+  long long HW[LAYOUT_MAX_SEG];
+};
+__device__ __forceinline__ int layout_locate(const LayoutBatch& B, long long* img, long long* p0) {
+  int si = 0;
+  while (si + 1 < B.n_seg && static_cast<int>(blockIdx.x) >= B.tile_start[si + 1]) ++si;
+  const int tl = static_cast<int>(blockIdx.x) - B.tile_start[si];
+  const int per_img = static_cast<int>((B.HW[si] + 63) / 64);
+  *img = tl / per_img;
+  *p0 = static_cast<long long>(tl - static_cast<int>(*img) * per_img) * 64;
+  return si;
+}
+__global__ void __launch_bounds__(256) nchw_to_nhwc_bf16_v8(const __grid_constant__ LayoutBatch B) {
   __shared__ __align__(16) __nv_bfloat16 tile[64][72];   // [channel][pixel vectors, permuted]
-  const long long img = blockIdx.z;
-  const long long p0 = static_cast<long long>(blockIdx.x) * 64;
+  long long img, p0;
+  const int si = layout_locate(B, &img, &p0);
+  const __nv_bfloat16* __restrict__ in = B.in[si];
+  __nv_bfloat16* __restrict__ out = B.out[si];
+  const int C = B.C;
+  const long long HW = B.HW[si];
   const int c0 = blockIdx.y * 64;
 #pragma unroll
   for (int it = 0; it < 2; ++it) {
@@ -413,11 +435,14 @@ __global__ void __launch_bounds__(256) nchw_to_nhwc_bf16_v8(const __nv_bfloat16*
     }
   }
 }
-__global__ void __launch_bounds__(256) nhwc_to_nchw_bf16_v8(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out,
-                                                             int C, long long HW) {
+__global__ void __launch_bounds__(256) nhwc_to_nchw_bf16_v8(const __grid_constant__ LayoutBatch B) {
   __shared__ __align__(16) __nv_bfloat16 tile[64][72];   // [pixel][channel vectors, permuted]
-  const long long img = blockIdx.z;
-  const long long p0 = static_cast<long long>(blockIdx.x) * 64;
+  long long img, p0;
+  const int si = layout_locate(B, &img, &p0);
+  const __nv_bfloat16* __restrict__ in = B.in[si];
+  __nv_bfloat16* __restrict__ out = B.out[si];
+  const int C = B.C;
+  const long long HW = B.HW[si];
   const int c0 = blockIdx.y * 64;
 #pragma unroll
   for (int it = 0; it < 2; ++it) {

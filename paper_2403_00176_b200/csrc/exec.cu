@@ -672,6 +672,45 @@ struct Builder {
   }
   Status build_layout(int gi, const Group& G) {
     const Tensor& X = g.tensors[G.a];
+    const bool from = G.act != 0;
+    // requests whose tensors qualify for the vectorised kernels are collected and converted by one launch
+    struct Seg { Ptr pi, po; long long HW; int N; };
+    std::vector<Seg> segs;
+    int segC = -1;
+    auto flush = [&]() {
+      if (segs.empty()) return;
+      std::vector<Seg> batch = segs;
+      const int C = segC;
+      segs.clear();
+      add(gi, 1, [=](const RunCtx& x) {
+        k::LayoutBatch B{};
+        B.n_seg = static_cast<int>(batch.size());
+        B.C = C;
+        int tiles = 0;
+        bool aligned = true;
+        for (int i = 0; i < B.n_seg; ++i) {
+          B.in[i] = reinterpret_cast<const __nv_bfloat16*>(x.resolve(batch[i].pi));
+          B.out[i] = reinterpret_cast<__nv_bfloat16*>(x.resolve(batch[i].po));
+          B.HW[i] = batch[i].HW;
+          B.tile_start[i] = tiles;
+          tiles += batch[i].N * static_cast<int>((batch[i].HW + 63) / 64);
+          aligned = aligned && ((reinterpret_cast<uintptr_t>(B.in[i]) | reinterpret_cast<uintptr_t>(B.out[i])) & 15) == 0;
+        }
+        B.tile_start[B.n_seg] = tiles;
+        if (aligned) {
+          const dim3 grid(static_cast<unsigned>(tiles), (C + 63) / 64, 1);
+          if (from) k::nhwc_to_nchw_bf16_v8<<<grid, 256, 0, x.stream>>>(B);
+          else k::nchw_to_nhwc_bf16_v8<<<grid, 256, 0, x.stream>>>(B);
+        } else {   // a caller buffer that is not 16-byte aligned: the element-wise kernels, one tensor at a time
+          for (int i = 0; i < B.n_seg; ++i) {
+            const dim3 grid(static_cast<unsigned>((B.HW[i] + 63) / 64), (C + 63) / 64, batch[i].N);
+            if (from) k::nhwc_to_nchw_bf16<<<grid, 256, 0, x.stream>>>(B.in[i], B.out[i], C, B.HW[i]);
+            else k::nchw_to_nhwc_bf16<<<grid, 256, 0, x.stream>>>(B.in[i], B.out[i], C, B.HW[i]);
+          }
+        }
+        return cudaGetLastError();
+      });
+    };
     for (int r = 0; r < p.n_req; ++r) {
       const View &vi = p.views[G.a][r], &vo = p.views[G.out][r];
       const int64_t n = numel(vi.dims);
@@ -689,17 +728,23 @@ struct Builder {
       if (!nchw.contiguous() || !is_channels_last(cl)) return fail(E_UNSUPPORTED_OP, "layout change between unexpected layouts");
       const int N = static_cast<int>(vi.dims[0]), C = static_cast<int>(vi.dims[1]);
       const long long HW = vi.dims[2] * vi.dims[3];
-      const bool from = G.act != 0;
+      if (C % 8 == 0 && HW % 8 == 0 && N * ((HW + 63) / 64) < (1ll << 28)) {
+        if (segC >= 0 && segC != C) flush();
+        segC = C;
+        segs.push_back(Seg{pi, po, HW, N});
+        if (segs.size() == static_cast<size_t>(k::LAYOUT_MAX_SEG)) flush();
+        continue;
+      }
       add(gi, 1, [=](const RunCtx& x) {
         const dim3 grid(static_cast<unsigned>((HW + 63) / 64), (C + 63) / 64, N);
         auto* in = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pi));
         auto* out = reinterpret_cast<__nv_bfloat16*>(x.resolve(po));
-        const bool v8 = C % 8 == 0 && HW % 8 == 0 && ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15) == 0;
-        if (from) { if (v8) k::nhwc_to_nchw_bf16_v8<<<grid, 256, 0, x.stream>>>(in, out, C, HW); else k::nhwc_to_nchw_bf16<<<grid, 256, 0, x.stream>>>(in, out, C, HW); }
-        else { if (v8) k::nchw_to_nhwc_bf16_v8<<<grid, 256, 0, x.stream>>>(in, out, C, HW); else k::nchw_to_nhwc_bf16<<<grid, 256, 0, x.stream>>>(in, out, C, HW); }
+        if (from) k::nhwc_to_nchw_bf16<<<grid, 256, 0, x.stream>>>(in, out, C, HW);
+        else k::nchw_to_nhwc_bf16<<<grid, 256, 0, x.stream>>>(in, out, C, HW);
         return cudaGetLastError();
       });
     }
+    flush();
     return OK;
   }
 
