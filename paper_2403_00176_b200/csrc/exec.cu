@@ -1123,8 +1123,9 @@ struct Builder {
       k::GapParams gp{};
       gp.C = static_cast<int>(vx.dims[1]);
       gp.HW = vx.dims[2] * vx.dims[3];
-      gp.slabs = static_cast<int>(std::max<long long>(1, std::min<long long>(16, gp.HW / 16)));   // N images x slabs CTAs, each with enough pixels to keep loads in flight
       const int N = static_cast<int>(vx.dims[0]);
+      // N images x slabs CTAs: about four per SM, each with enough pixels to keep loads in flight
+      gp.slabs = static_cast<int>(std::max<long long>(1, std::min<long long>(std::max(1, 592 / N), gp.HW / 16)));
       scratch_need = std::max(scratch_need, static_cast<size_t>(N) * gp.slabs * gp.C * 8);
       Ptr px = ptr_of(G.a, r), pw = ptr_of(G.w, 0), pb = ptr_of(G.bias, 0), pg = ptr_of(G.out, r);
       Ptr pz = want_z ? ptr_of(G.out2, r) : Ptr();
@@ -1343,6 +1344,13 @@ struct Builder {
       std::vector<size_t> poff;
       size_t part_bytes = 0;
       int max_slabs = 1, max_nc = 0;
+      // about four CTAs per SM over the whole launch, shared among the images in proportion to their pixels: the
+      // kernel streams at the HBM rate once it runs, and more, shorter CTAs only add to its fixed cost
+      double total_px = 0.0;
+      for (int r = r0; r < std::min(p.n_req, r0 + k::GAP_MAX_SEG); ++r) {
+        const View& vx = p.views[G.a][r];
+        if (numel(vx.dims)) total_px += static_cast<double>(vx.dims[0]) * static_cast<double>(vx.dims[2] * vx.dims[3]);
+      }
       for (int r = r0; r < std::min(p.n_req, r0 + k::GAP_MAX_SEG); ++r) {
         const View& vx = p.views[G.a][r];
         if (!numel(vx.dims)) continue;
@@ -1350,7 +1358,8 @@ struct Builder {
         k::GapParams gp{};
         gp.C = static_cast<int>(vx.dims[1]);
         gp.HW = vx.dims[2] * vx.dims[3];
-        gp.slabs = static_cast<int>(std::max<long long>(1, std::min<long long>(592, gp.HW / (vx.dims[0] >= 16 ? 16 : 128))));
+        const long long share = static_cast<long long>(std::ceil(592.0 * static_cast<double>(gp.HW) / total_px));
+        gp.slabs = static_cast<int>(std::max<long long>(1, std::min<long long>(share, gp.HW / (vx.dims[0] >= 16 ? 16 : 128))));
         gp.out_bf16 = O.dtype == DType::BF16;
         const int N = static_cast<int>(vx.dims[0]);
         const int si = gb.n_seg++;

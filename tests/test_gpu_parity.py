@@ -342,6 +342,35 @@ def test_cfg4_full_config_smallest_request_and_properties():
         assert np.allclose(outs[r]["gap"].reshape(-1), y.mean(axis=(2, 3)).reshape(-1), rtol=1e-2, atol=1e-2)
 
 
+@pytest.mark.parametrize("C", [64, 1088])
+def test_global_average_pool_sums_are_exact_over_a_wide_range(C):
+    """The pooling kernel adds groups of eight inputs in fp32 where that is provably exact and in fp64
+    where it is not.  Inputs 26 binades apart that cancel across the image: any fp32 shortcut taken
+    where it is not exact loses the small terms, and the mean with them."""
+    H, W = 48, 40
+    ir = (f"input x bf16 [1,{C},{H},{W}]\nconst w bf16 [{C},{C},1,1]\nconst b bf16 [{C}]\n"
+          "node Conv x w b -> c1 {kernel=1 stride=1 pad=0}\nnode Relu c1 -> r2\nnode Add x r2 -> y\n"
+          "node GlobalAveragePool y -> gap\noutput gap\noutput y\n")
+    consts = {"w": np.zeros((C, C, 1, 1), np.float32), "b": np.zeros((C,), np.float32)}   # y == x
+    rng = np.random.default_rng(C)
+    x = np.full((1, C, H, W), 2.0 ** -6, np.float32)
+    x[0, 1::4] = bf16_round(rng.uniform(-2, 2, (len(range(1, C, 4)), H, W)).astype(np.float32))   # ordinary channels
+    x[0, 2::4] = 0.0
+    x[0, 2::4, ::3, ::5] = -0.0
+    big = 2.0 ** 20
+    x[0, 0::4, 0, 0] = big
+    x[0, 0::4, H - 1, W - 1] = -big
+    x[0, 3::4, H // 2, 3] = big
+    x[0, 3::4, 1, W - 2] = -big
+    wl = WL.Workload("gap_exact", "bf16", ir, consts, [], ["gap", "y"], {})
+    s, p, outs = run_batch(wl, [Request({}, {"x": x})])
+    assert np.array_equal(outs[0]["y"].astype(np.float32), x)
+    exact = bf16_round(x.astype(np.float64).mean(axis=(2, 3)).astype(np.float32)).reshape(-1)
+    got = outs[0]["gap"].astype(np.float32).reshape(-1)
+    assert exact[0] == bf16_round(np.float32((H * W - 2) * 2.0 ** -6 / (H * W)))   # the small terms ARE the mean
+    assert np.array_equal(got, exact), np.flatnonzero(got != exact)[:8]
+
+
 def _gemm_graph(K, N, act, residual):
     lines = ["sym M 1 4096", f"input x bf16 [1,M,{K}]"]
     if residual:
