@@ -366,7 +366,7 @@ sod2_status sod2_plan_instance_offset(const sod2_plan_t* p, const char* name, in
   int t = p->g->c.g.tensor(name);
   if (t < 0 || p->p.views[t].empty() || p->p.views[t][0].root < 0) return SOD2_E_INVALID_ARG;
   const View& v = p->p.views[t][r];
-  *off = static_cast<size_t>(p->p.roots[v.root].inst_off[r] + v.offset * dtype_size(p->g->c.g.tensors[t].dtype));
+  *off = static_cast<size_t>(p->p.inst_off[v.root][r] + v.offset * dtype_size(p->g->c.g.tensors[t].dtype));
   return SOD2_OK;
 }
 

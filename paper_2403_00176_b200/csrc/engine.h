@@ -2,7 +2,9 @@
 #pragma once
 #include <initializer_list>
 #include <memory>
+#include <new>
 #include <string>
+#include <type_traits>
 #include <vector>
 
 #include "graph.h"
@@ -91,6 +93,10 @@ struct Compiled {
   // every distinct extent expression once: binding evaluates each per request, tensors index the table
   std::vector<Expr> dim_exprs;
   std::vector<std::vector<int>> dim_expr_id;   // [tensor][axis] -> dim_exprs index, -1 if the extent is unknown
+  // per tensor stored as a view: the operator's parameters read out of its attributes once (Transpose:
+  // a = perm; Slice: a = start, b = step per axis of the input), so that planning touches no strings
+  struct ViewParam { int op = -1; std::vector<int64_t> a, b; };   // op: 0 Transpose, 1 Reshape, 2 Slice
+  std::vector<ViewParam> view_param;
   std::vector<int> packed_consts;     // tensor ids
   std::vector<size_t> packed_off;     // byte offsets in the prepack workspace
   size_t packed_bytes = 0;
@@ -134,11 +140,54 @@ struct DimVec {
   bool operator!=(const DimVec& o) const { return !(*this == o); }
 };
 
+// [tensor][request] table in one block of memory: binding and planning fill a few thousand small entries per
+// batch, and one vector per tensor made the allocator the largest cost of both.  A row exists once make(t) was
+// called; the others read as empty.  T must be trivially destructible (nothing is destroyed).
+template <class T>
+class ReqTable {
+ public:
+  template <class U>
+  class RowT {
+   public:
+    RowT(U* p, int n) : p_(p), n_(n) {}
+    bool empty() const { return n_ == 0; }
+    size_t size() const { return static_cast<size_t>(n_); }
+    U& operator[](size_t r) const { return p_[r]; }
+    U* begin() const { return p_; }
+    U* end() const { return p_ + n_; }
+   private:
+    U* p_;
+    int n_;
+  };
+  using Row = RowT<T>;
+  using ConstRow = RowT<const T>;
+  void reset(size_t n_tensors, int n_req) {
+    static_assert(std::is_trivially_destructible<T>::value, "rows are never destroyed");
+    n_req_ = n_req;
+    has_.assign(n_tensors, 0);
+    const size_t need = n_tensors * static_cast<size_t>(n_req) * sizeof(T);
+    if (need > cap_) { raw_.reset(new unsigned char[need]); cap_ = need; }
+  }
+  Row make(size_t t) {
+    T* p = reinterpret_cast<T*>(raw_.get()) + t * n_req_;
+    if (!has_[t]) { for (int r = 0; r < n_req_; ++r) new (p + r) T(); has_[t] = 1; }
+    return Row(p, n_req_);
+  }
+  Row operator[](size_t t) { return has_[t] ? Row(reinterpret_cast<T*>(raw_.get()) + t * n_req_, n_req_) : Row(nullptr, 0); }
+  ConstRow operator[](size_t t) const { return has_[t] ? ConstRow(reinterpret_cast<const T*>(raw_.get()) + t * n_req_, n_req_) : ConstRow(nullptr, 0); }
+  size_t size() const { return has_.size(); }
+ private:
+  std::unique_ptr<unsigned char[]> raw_;
+  size_t cap_ = 0;
+  std::vector<char> has_;
+  int n_req_ = 0;
+};
+
 struct Binding {
   const Compiled* c = nullptr;
   int n_req = 0;
   std::vector<std::vector<int64_t>> vals;   // [req][atom]
-  std::vector<std::vector<DimVec>> dims;    // [tensor][req]; empty if not evaluable yet
+  ReqTable<DimVec> dims;                    // [tensor][req]; empty if not evaluable yet
   std::string err;
 };
 Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* names, const int64_t* values, Binding* out);
@@ -160,7 +209,6 @@ struct View {                 // one tensor of one request, resolved to storage
 struct RootBuf {              // packed storage of a root tensor: the requests' instances back to back
   enum Where { NONE, INPUT, OUTPUT, CONST, ARENA } where = NONE;
   int io_index = -1;
-  std::vector<int64_t> inst_off;   // [req] byte offset of the request's instance
   int64_t bytes = 0;
   size_t arena_off = 0;
   int def_step = -1, last_step = -1;
@@ -178,7 +226,8 @@ struct Plan {
   const Compiled* c = nullptr;
   const Binding* b = nullptr;
   int n_req = 0;
-  std::vector<std::vector<View>> views;   // [tensor][req]
+  ReqTable<View> views;                   // [tensor][req]
+  ReqTable<int64_t> inst_off;             // [root tensor][req] byte offset of the request's instance in the root's packed storage
   std::vector<RootBuf> roots;             // [tensor]
   size_t arena_bytes = 0, peak_live_bytes = 0, sum_bytes = 0;
   int peak_step = 0;

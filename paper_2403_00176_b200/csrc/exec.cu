@@ -93,7 +93,7 @@ struct Builder {
     Ptr q;
     q.where = R.where;
     q.index = (R.where == RootBuf::CONST) ? v.root : R.io_index;
-    q.off = R.inst_off[r] + (v.offset + extra_elems) * dtype_size(g.tensors[t].dtype);
+    q.off = p.inst_off[v.root][r] + (v.offset + extra_elems) * dtype_size(g.tensors[t].dtype);
     if (R.where == RootBuf::ARENA) q.off += static_cast<int64_t>(R.arena_off);
     return q;
   }

@@ -614,10 +614,31 @@ static void index_dim_exprs(Compiled* c) {
   }
 }
 
+// Parameters of the view operators, per tensor stored as a view.
+static void index_view_params(Compiled* c) {
+  const Graph& g = c->g;
+  c->view_param.assign(g.tensors.size(), {});
+  for (size_t t = 0; t < g.tensors.size() && t < c->storage.size(); ++t) {
+    const Storage& st = c->storage[t];
+    if ((st.kind != Storage::VIEW_OF_INPUT && st.kind != Storage::VIEW_OF_OUTPUT) || st.node < 0) continue;
+    const Node& n = g.nodes[st.node];
+    Compiled::ViewParam& vp = c->view_param[t];
+    vp.op = n.op == "Transpose" ? 0 : n.op == "Reshape" ? 1 : 2;
+    if (vp.op == 0) vp.a = n.attr_list("perm");
+    if (vp.op == 2 && st.kind == Storage::VIEW_OF_INPUT && st.other >= 0) {
+      const int rank = g.tensors[st.other].S.rank;
+      for (int ax = 0; ax < rank; ++ax) {
+        vp.a.push_back(n.attr_i("_start" + std::to_string(ax), 0));
+        vp.b.push_back(n.attr_i("_step" + std::to_string(ax), 1));
+      }
+    }
+  }
+}
+
 Status form_groups(Compiled* c) {
   Fuser f(*c);
   Status s = f.run();
-  if (s == OK) index_dim_exprs(c);
+  if (s == OK) { index_dim_exprs(c); index_view_params(c); }
   return s;
 }
 

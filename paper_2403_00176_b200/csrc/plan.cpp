@@ -31,6 +31,8 @@ Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* na
   }
   for (int id : g.user_syms)
     if (out->vals[0][id] == INT64_MIN) { out->err = "symbol " + g.cx.atoms[id].name + " is not bound"; return E_UNBOUND_SYMBOL; }
+  static const bool prof = getenv("SOD2_HOST_PROFILE") != nullptr;
+  auto t0 = std::chrono::steady_clock::now();
   // bind-time assertions recorded by RDP (two inferences of one extent must agree)
   for (int r = 0; r < n_req; ++r)
     for (auto& as : g.asserts) {
@@ -43,6 +45,7 @@ Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* na
     }
   // all non-linear atoms once per request (children first), then every distinct extent expression once
   // per request as a flat polynomial; tensors pick their extents from that table
+  auto t1 = std::chrono::steady_clock::now();
   const size_t U = c->dim_exprs.size();
   std::vector<int64_t> uval(static_cast<size_t>(n_req) * U);
   std::vector<char> uok(static_cast<size_t>(n_req) * U);
@@ -58,7 +61,8 @@ Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* na
       uok[r * U + u] = ok;
     }
   }
-  out->dims.assign(g.tensors.size(), {});
+  auto t2 = std::chrono::steady_clock::now();
+  out->dims.reset(g.tensors.size(), n_req);
   for (size_t t = 0; t < g.tensors.size(); ++t) {
     const ShapeVal& s = g.tensors[t].S;
     if (s.rank < 0) continue;
@@ -69,8 +73,7 @@ Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* na
     for (int r = 0; r < n_req && evaluable; ++r)
       for (int i = 0; i < s.rank; ++i) if (!uok[r * U + ids[i]]) { evaluable = false; break; }
     if (!evaluable) continue;
-    std::vector<DimVec>& per = out->dims[t];
-    per.resize(n_req);
+    auto per = out->dims.make(t);
     for (int r = 0; r < n_req; ++r) {
       per[r].n = s.rank;
       for (int i = 0; i < s.rank; ++i) {
@@ -79,6 +82,12 @@ Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* na
         per[r].v[i] = v;
       }
     }
+  }
+  if (prof) {
+    auto t3 = std::chrono::steady_clock::now();
+    auto us = [](auto a, auto b) { return std::chrono::duration<double, std::micro>(b - a).count(); };
+    fprintf(stderr, "[sod2] bind: %zu assertions %.1f us, %zu extent expressions %.1f us, %zu tensors %.1f us\n", g.asserts.size(), us(t0, t1), U,
+            us(t1, t2), g.tensors.size(), us(t2, t3));
   }
   return OK;
 }
@@ -133,7 +142,7 @@ struct Planner {
     if (b.dims[t].empty()) return fail(E_INTERNAL, "no concrete shape for " + g.tensors[t].name);
     const Tensor& T = g.tensors[t];
     RootBuf& R = p.roots[t];
-    R.inst_off.resize(p.n_req);
+    auto inst_off = p.inst_off.make(t);
     int64_t off = 0;
     int esz = dtype_size(T.dtype);
     bool per_request = T.kind != TKind::CONST;
@@ -149,7 +158,7 @@ struct Planner {
         const int64_t C = v.dims[1], H = v.dims[2], W = v.dims[3];
         v.strides = {H * W * C, 1, W * C, C};
       }
-      R.inst_off[r] = per_request ? off : 0;
+      inst_off[r] = per_request ? off : 0;
       int64_t bytes = numel(v.dims) * esz;
       if (per_request) off += (bytes + 15) & ~int64_t(15);
       else off = bytes;
@@ -167,9 +176,8 @@ struct Planner {
     if (resolved[t]) return OK;
     const Storage& st = c.storage[t];
     if (st.kind == Storage::FOLDED) { resolved[t] = 1; return OK; }
-    p.views[t].resize(p.n_req);
+    p.views.make(t);
     if (st.kind == Storage::ROOT) return make_root(t);
-    const Node& n = g.nodes[st.node];
     if (b.dims[t].empty()) return fail(E_INTERNAL, "no concrete shape for " + g.tensors[t].name);
     if (st.kind == Storage::ALIAS) {
       Status s = resolve(st.other);
@@ -208,7 +216,7 @@ struct Planner {
       int o = st.other;
       Status s = resolve(o);
       if (s != OK) return s;
-      const std::vector<int64_t> perm = n.attr_list("perm");
+      const std::vector<int64_t>& perm = c.view_param[t].a;
       for (int r = 0; r < p.n_req; ++r) {
         const View& vo = p.views[o][r];
         View& v = p.views[t][r];
@@ -225,14 +233,12 @@ struct Planner {
     int in = st.other;
     Status s = resolve(in);
     if (s != OK) return s;
-    const int kind = n.op == "Transpose" ? 0 : n.op == "Reshape" ? 1 : 2;
-    std::vector<int64_t> perm, sl_start, sl_step;
-    if (kind == 0) perm = n.attr_list("perm");
-    if (kind == 2)
-      for (size_t ax = 0; ax < p.views[in][0].dims.size(); ++ax) {
-        sl_start.push_back(n.attr_i("_start" + std::to_string(ax), 0));
-        sl_step.push_back(n.attr_i("_step" + std::to_string(ax), 1));
-      }
+    const Compiled::ViewParam& vp = c.view_param[t];
+    const int kind = vp.op;
+    const std::vector<int64_t>& perm = vp.a;
+    const std::vector<int64_t>& sl_start = vp.a;
+    const std::vector<int64_t>& sl_step = vp.b;
+    if (kind == 2 && sl_start.size() != p.views[in][0].dims.size()) return fail(E_INTERNAL, "slice parameters of " + g.tensors[t].name);
     for (int r = 0; r < p.n_req; ++r) {
       const View& vi = p.views[in][r];
       View& v = p.views[t][r];
@@ -259,8 +265,10 @@ struct Planner {
   }
 
   Status run() {
+    auto t0 = std::chrono::steady_clock::now();
     size_t T = g.tensors.size();
-    p.views.assign(T, {});   // filled per tensor when it is resolved
+    p.inst_off.reset(T, p.n_req);
+    p.views.reset(T, p.n_req);   // rows are made per tensor when it is resolved
     p.roots.assign(T, RootBuf());
     // resolve every tensor a group touches
     for (auto& G : c.groups) {
@@ -269,6 +277,8 @@ struct Planner {
       for (int t : G.ext_out) { Status s = resolve(t); if (s != OK) return s; }
     }
     for (int t : g.outputs) { Status s = resolve(t); if (s != OK) return s; }
+    static const bool prof = getenv("SOD2_HOST_PROFILE") != nullptr;
+    auto t1 = std::chrono::steady_clock::now();
     // liveness of arena roots over the group sequence
     int steps = static_cast<int>(c.groups.size());
     for (int s = 0; s < steps; ++s) {
@@ -285,7 +295,14 @@ struct Planner {
       for (int t : G.ext_out) touch(t, true);
       for (int t : G.ext_in) touch(t, false);
     }
-    return plan_arena(steps);
+    auto t2 = std::chrono::steady_clock::now();
+    Status s = plan_arena(steps);
+    if (prof) {
+      auto t3 = std::chrono::steady_clock::now();
+      auto us = [](auto a, auto b) { return std::chrono::duration<double, std::micro>(b - a).count(); };
+      fprintf(stderr, "[sod2] plan: views %.1f us, liveness %.1f us, arena %.1f us\n", us(t0, t1), us(t1, t2), us(t2, t3));
+    }
+    return s;
   }
 
   // Peak-first greedy: place the tensors live at the peak step contiguously, then walk forward
