@@ -222,6 +222,13 @@ def test_cfg2_full_config_batch0():
         assert np.all(np.isfinite(y))
         assert np.max(np.abs(y.mean(-1))) < 2e-2
         assert np.max(np.abs((y * y).mean(-1) - 1.0)) < 5e-2
+    # the launch configuration the benchmark times: the same plan replayed as one CUDA graph, same bits
+    p.run_graph()
+    p.run_graph()
+    p.check_device_status()
+    outs_graph = p.outputs()
+    for r in range(len(reqs)):
+        assert np.array_equal(outs[r]["y"], outs_graph[r]["y"])
 
 
 def test_cfg2_full_config_lockstep_per_group():
