@@ -117,11 +117,24 @@ __global__ void __launch_bounds__(256) topk_gather(const __grid_constant__ TopkP
   __shared__ int s_pos[TOPK_CHUNK];
   int chunk;
   const TopkReq R = p.r[topk_locate(p, blockIdx.x, &chunk)];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int base = chunk * TOPK_CHUNK;
+  // The rows of the chunk are fetched before the dependency wait: they were written by the kernel before the
+  // score kernel, which had completed before the flag kernel (the one waited for here) let this one start, so
+  // only the flags are still in flight.  Whether a row is kept is not known yet: all rows of the chunk are read.
+  const int vec = (p.D * 2) >> 4;  // 16-byte pieces per row (D % 8 == 0 checked on the host)
+  const uint4* src = reinterpret_cast<const uint4*>(p.y + (R.row0 + base) * p.D);
+  const int items = min(TOPK_CHUNK, R.n - base) * vec;
+  constexpr int PRE = 12;
+  uint4 pre[PRE];
+#pragma unroll
+  for (int u = 0; u < PRE; ++u) {
+    const int it = tid + u * 256;
+    if (it < items) pre[u] = src[it];
+  }
   ptx::pdl_wait();
   ptx::pdl_launch();
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned char* kp = p.keep + (R.row0 - p.first_row);
-  const int base = chunk * TOPK_CHUNK;
   // kept tokens before this chunk
   int c = 0;
   for (int j = tid; j < base; j += 256) c += kp[j];
@@ -148,14 +161,20 @@ __global__ void __launch_bounds__(256) topk_gather(const __grid_constant__ TopkP
     p.idx[R.idx0 + s_pos[tid]] = base + tid;
   }
   __syncthreads();
-  // copy the kept rows: (row, 16-byte piece) items spread over the whole CTA, several independent
-  // loads in flight per thread
-  const int vec = (p.D * 2) >> 4;  // 16-byte pieces per row (D % 8 == 0 checked on the host)
-  const uint4* src = reinterpret_cast<const uint4*>(p.y + (R.row0 + base) * p.D);
+  // write the kept rows: (row, 16-byte piece) items spread over the whole CTA; the first PRE per thread are
+  // already in registers, wider rows load the rest now
   uint4* dst = reinterpret_cast<uint4*>(p.out + R.out_row0 * p.D);
-  const int items = TOPK_CHUNK * vec;
+#pragma unroll
+  for (int u = 0; u < PRE; ++u) {
+    const int it = tid + u * 256;
+    if (it < items) {
+      const int t = it / vec, c4 = it - t * vec;
+      const int pos = s_pos[t];
+      if (pos >= 0) dst[static_cast<long long>(pos) * vec + c4] = pre[u];
+    }
+  }
 #pragma unroll 4
-  for (int it = tid; it < items; it += 256) {
+  for (int it = tid + PRE * 256; it < items; it += 256) {
     const int t = it / vec, c4 = it - t * vec;
     const int pos = s_pos[t];
     if (pos >= 0) dst[static_cast<long long>(pos) * vec + c4] = src[it];
