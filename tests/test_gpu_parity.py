@@ -280,6 +280,11 @@ def test_cfg3_small_pruning_lockstep_and_ties():
     x = bf16_round(rng.standard_normal((1, 40, 128)).astype(np.float32))
     x[0, 20:40] = x[0, 0:20]
     reqs.append(Request({"N0": 40}, {"x": x}))
+    # a request of several 64-token chunks with ties across the chunk boundaries
+    x = bf16_round(rng.standard_normal((1, 300, 128)).astype(np.float32))
+    x[0, 120:140] = x[0, 100:120]
+    x[0, 250:270] = x[0, 100:120]
+    reqs.append(Request({"N0": 300}, {"x": x}))
     _check_topk_lockstep(wl, reqs, 3)
 
 
