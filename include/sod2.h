@@ -204,6 +204,12 @@ sod2_status sod2_run_output_shape(sod2_plan_t* p, const void* arena, void* cuda_
 sod2_status sod2_nonzero_static(const void* dev_x, int dtype, int rank, const int64_t* dims, int64_t* dev_out,
                                 int64_t* dev_count, void* cuda_stream);
 
+/* Launches one kernel that does nothing (one thread, no arguments) on cuda_stream.  A measuring aid:
+ * the smallest fused groups (a few thousand elements per request) take about as long as this launch,
+ * so their time is reported as a multiple of it rather than as a fraction of a roofline.
+ * Asynchronous.  Errors: SOD2_E_CUDA; message through sod2_last_error(NULL). */
+sod2_status sod2_launch_empty(void* cuda_stream);
+
 /* handle may be a graph, binding or plan; returns "" if there was no error. */
 const char* sod2_last_error(const void* any_handle);
 

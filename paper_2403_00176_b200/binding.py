@@ -73,6 +73,7 @@ def _load() -> C.CDLL:
         "sod2_plan_tensor_strides": [vp, cp, i32, P(i64), P(i32)],
         "sod2_run_output_shape": [vp, vp, vp, i32, i32, P(i64), P(i32)],
         "sod2_nonzero_static": [vp, i32, i32, P(i64), vp, vp, vp],
+        "sod2_launch_empty": [vp],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -96,7 +97,7 @@ EXPORTS = ["sod2_graph_create", "sod2_graph_destroy", "sod2_graph_set_const", "s
            "sod2_graph_num_ops", "sod2_graph_op_info", "sod2_graph_num_groups", "sod2_graph_group_info",
            "sod2_graph_num_subgraphs", "sod2_graph_rdp_sweeps", "sod2_classify", "sod2_graph_reanalyse", "sod2_graph_order_info",
            "sod2_binding_shape", "sod2_plan_slot", "sod2_plan_instance_offset", "sod2_plan_memory", "sod2_plan_group_cost", "sod2_plan_tensor_strides",
-           "sod2_run_output_shape", "sod2_nonzero_static", "sod2_last_error"]
+           "sod2_run_output_shape", "sod2_nonzero_static", "sod2_launch_empty", "sod2_last_error"]
 
 
 def _check(status: int, handle=None):
@@ -112,6 +113,11 @@ def sod2_classify(op: str) -> str:
 
 
 NONZERO_STATIC_MAX_ELEMS = 16777216
+
+
+def sod2_launch_empty(stream: int) -> None:
+    """One kernel that does nothing, on `stream`: the yardstick for launch-bound groups."""
+    _check(lib.sod2_launch_empty(C.c_void_p(stream)))
 
 
 def sod2_nonzero_static(dev_x: int, dtype: int, dims: Sequence[int], dev_out: int, dev_count: int, stream: int) -> None:

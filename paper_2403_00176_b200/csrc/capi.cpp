@@ -251,6 +251,10 @@ sod2_status sod2_run_timed(sod2_plan_t* p, const void* const* inputs, void* cons
 sod2_status sod2_plan_device_status(sod2_plan_t* p, const void* arena, void* stream) {
   if (!p || !arena) return SOD2_E_INVALID_ARG;
   int word = 0;
+  if (!p->p.uses_header) {   // no kernel of this plan has a bounded wait: the word is never written (nor cleared)
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) { p->h.err = "cannot synchronise the stream"; return SOD2_E_CUDA; }
+    return SOD2_OK;
+  }
   if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess ||
       cudaMemcpy(&word, arena, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) {
     p->h.err = "cannot read the device status word";

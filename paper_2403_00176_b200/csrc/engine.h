@@ -236,6 +236,7 @@ struct Plan {
   int gpu_launches = 0;
   int sm_count = 148;                     // persistent kernels launch one CTA per SM
   bool sm_count_known = false;
+  bool uses_header = true;                // false: no kernel of the plan writes the status word, a ticket or a count: nothing to clear or read
   std::vector<double> group_flops, group_bytes;   // algorithmic cost per group for the bound shapes
   std::string err;
   // device status word lives at arena offset 0 (first 256 bytes reserved)

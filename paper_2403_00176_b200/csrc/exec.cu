@@ -193,10 +193,10 @@ struct Builder {
           const int grid = std::min((mp.M + 7) / 8, 148 * 2);
           const size_t smem = (static_cast<size_t>(mp.K) * mp.N + 8 * mp.K) * sizeof(float);
           switch (nc) {
-            case 1: cudaFuncSetAttribute(k::fused_mlp_ln_f32<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024); k::fused_mlp_ln_f32<1><<<grid, 256, smem, x.stream>>>(mp); break;
-            case 2: cudaFuncSetAttribute(k::fused_mlp_ln_f32<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024); k::fused_mlp_ln_f32<2><<<grid, 256, smem, x.stream>>>(mp); break;
-            case 3: cudaFuncSetAttribute(k::fused_mlp_ln_f32<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024); k::fused_mlp_ln_f32<3><<<grid, 256, smem, x.stream>>>(mp); break;
-            default: cudaFuncSetAttribute(k::fused_mlp_ln_f32<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024); k::fused_mlp_ln_f32<4><<<grid, 256, smem, x.stream>>>(mp); break;
+            case 1: { static bool once = (cudaFuncSetAttribute(k::fused_mlp_ln_f32<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024), true); (void)once; k::fused_mlp_ln_f32<1><<<grid, 256, smem, x.stream>>>(mp); break; }
+            case 2: { static bool once = (cudaFuncSetAttribute(k::fused_mlp_ln_f32<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024), true); (void)once; k::fused_mlp_ln_f32<2><<<grid, 256, smem, x.stream>>>(mp); break; }
+            case 3: { static bool once = (cudaFuncSetAttribute(k::fused_mlp_ln_f32<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024), true); (void)once; k::fused_mlp_ln_f32<3><<<grid, 256, smem, x.stream>>>(mp); break; }
+            default: { static bool once = (cudaFuncSetAttribute(k::fused_mlp_ln_f32<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024), true); (void)once; k::fused_mlp_ln_f32<4><<<grid, 256, smem, x.stream>>>(mp); break; }
           }
           return cudaGetLastError();
         });
@@ -1433,6 +1433,10 @@ struct Builder {
     p.group_flops.clear();
     p.group_bytes.clear();
     p.gpu_launches = 0;
+    // the fp32 row kernel and the elementwise chains have no bounded waits, tickets or device-side counts
+    p.uses_header = false;
+    for (const Group& G : c.groups)
+      if (!((G.kind == GKind::GEMM && g.tensors[G.a].dtype == DType::F32) || G.kind == GKind::CHAIN)) p.uses_header = true;
     for (size_t gi = 0; gi < c.groups.size(); ++gi) {
       const Group& G = c.groups[gi];
       Status s = OK;
@@ -1535,7 +1539,7 @@ Status run_plan_timed(Plan* p, const void* const* inputs, void* const* outputs, 
   const size_t n = p->launches.size();
   std::vector<cudaEvent_t> ev(2 * n);
   for (auto& e : ev) if (cudaEventCreate(&e) != cudaSuccess) { p->err = "cudaEventCreate failed"; return E_CUDA; }
-  cudaMemsetAsync(arena, 0, 256, x.stream);
+  if (p->uses_header) cudaMemsetAsync(arena, 0, 256, x.stream);
   Status st = OK;
   for (size_t i = 0; i < n && st == OK; ++i) {
     cudaEventRecord(ev[2 * i], x.stream);
@@ -1615,7 +1619,7 @@ Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* 
     p->sm_count_known = true;
   }
   RunCtx x{inputs, outputs, static_cast<char*>(arena), static_cast<char*>(p->c->packed_ws), static_cast<cudaStream_t>(stream), p};
-  if (cudaMemsetAsync(arena, 0, 256, x.stream) != cudaSuccess) { p->err = "cannot clear the status word"; return E_CUDA; }
+  if (p->uses_header && cudaMemsetAsync(arena, 0, 256, x.stream) != cudaSuccess) { p->err = "cannot clear the status word"; return E_CUDA; }
   for (auto& L : p->launches) {
     cudaError_t e = L->fn(x);
     if (e != cudaSuccess) {

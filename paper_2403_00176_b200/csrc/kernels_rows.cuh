@@ -48,11 +48,46 @@ __global__ void __launch_bounds__(256) fused_mlp_ln_f32(MlpLnParams p) {
   float* Ws = smem_f;                 // [K][N]
   float* Xs = smem_f + p.K * p.N;     // [8 warps][K]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int i = threadIdx.x; i < p.K * p.N; i += blockDim.x) Ws[i] = p.W[i];
+  // The group is a few thousand elements per request, so its time is its chain of round trips to memory:
+  // everything the warp's first row needs (the row, the per-column constants, its residual) is requested
+  // together with W, before the first wait.
+  const int row0 = blockIdx.x * 8 + warp;
+  float xpre[4];                      // K <= 128
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int kk = lane + 32 * q;
+    xpre[q] = (row0 < p.M && kk < p.K) ? p.X[static_cast<long long>(row0) * p.K + kk] : 0.f;
+  }
+  float bias_r[NC], gam[NC], bet[NC], res[NC];
+#pragma unroll
+  for (int c = 0; c < NC; ++c) {
+    const int col = c * 32 + lane;
+    bias_r[c] = p.bias ? p.bias[col] : 0.f;
+    gam[c] = p.has_ln ? p.gamma[col] : 1.f;
+    bet[c] = p.has_ln ? p.beta[col] : 0.f;
+    res[c] = (p.R && row0 < p.M) ? p.R[static_cast<long long>(row0) * p.N + col] : 0.f;
+  }
+  if ((reinterpret_cast<uintptr_t>(p.W) & 15) == 0) {      // K * N is a multiple of 32
+    const float4* W4 = reinterpret_cast<const float4*>(p.W);
+    float4* Ws4 = reinterpret_cast<float4*>(Ws);
+#pragma unroll 4
+    for (int i = threadIdx.x; i < (p.K * p.N) >> 2; i += 256) Ws4[i] = W4[i];
+  } else {
+    for (int i = threadIdx.x; i < p.K * p.N; i += 256) Ws[i] = p.W[i];
+  }
   __syncthreads();
   float* xs = Xs + warp * p.K;
-  for (int row = blockIdx.x * 8 + warp; row < p.M; row += gridDim.x * 8) {
-    for (int kk = lane; kk < p.K; kk += 32) xs[kk] = p.X[static_cast<long long>(row) * p.K + kk];
+  for (int row = row0; row < p.M; row += gridDim.x * 8) {
+    if (row == row0) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) { const int kk = lane + 32 * q; if (kk < p.K) xs[kk] = xpre[q]; }
+    } else {
+      for (int kk = lane; kk < p.K; kk += 32) xs[kk] = p.X[static_cast<long long>(row) * p.K + kk];
+      if (p.R) {
+#pragma unroll
+        for (int c = 0; c < NC; ++c) res[c] = p.R[static_cast<long long>(row) * p.N + c * 32 + lane];
+      }
+    }
     __syncwarp();
     float acc[NC];
 #pragma unroll
@@ -65,11 +100,10 @@ __global__ void __launch_bounds__(256) fused_mlp_ln_f32(MlpLnParams p) {
     float s = 0.f;
 #pragma unroll
     for (int c = 0; c < NC; ++c) {
-      const int col = c * 32 + lane;
       float v = acc[c];
-      if (p.bias) v += p.bias[col];
+      if (p.bias) v += bias_r[c];
       v = act_apply(p.act, v);
-      if (p.R) v += p.R[static_cast<long long>(row) * p.N + col];
+      if (p.R) v += res[c];
       acc[c] = v;
       s += v;
     }
@@ -80,10 +114,7 @@ __global__ void __launch_bounds__(256) fused_mlp_ln_f32(MlpLnParams p) {
       for (int c = 0; c < NC; ++c) { const float d = acc[c] - mu; q += d * d; }
       const float rstd = rsqrtf(warp_sum(q) / p.N + p.eps);
 #pragma unroll
-      for (int c = 0; c < NC; ++c) {
-        const int col = c * 32 + lane;
-        acc[c] = (acc[c] - mu) * rstd * p.gamma[col] + p.beta[col];
-      }
+      for (int c = 0; c < NC; ++c) acc[c] = (acc[c] - mu) * rstd * gam[c] + bet[c];
     }
 #pragma unroll
     for (int c = 0; c < NC; ++c) p.Y[static_cast<long long>(row) * p.N + c * 32 + lane] = acc[c];

@@ -159,3 +159,14 @@ extern "C" sod2_status sod2_nonzero_static(const void* dev_x, int dtype, int ran
   if (e != cudaSuccess) return nzs_fail(SOD2_E_CUDA, std::string("sod2_nonzero_static: launch failed: ") + cudaGetErrorString(e));
   return SOD2_OK;
 }
+
+namespace {
+__global__ void empty_kernel() {}
+}  // namespace
+
+extern "C" sod2_status sod2_launch_empty(void* cuda_stream) {
+  empty_kernel<<<1, 1, 0, static_cast<cudaStream_t>(cuda_stream)>>>();
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return nzs_fail(SOD2_E_CUDA, std::string("sod2_launch_empty: launch failed: ") + cudaGetErrorString(e));
+  return SOD2_OK;
+}

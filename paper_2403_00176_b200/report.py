@@ -82,6 +82,31 @@ def measure(cfg: int, reps: int, oracle_budget: float):
         e1.record(stream)
         torch.cuda.synchronize(dev)
         gtimes.append(e0.elapsed_time(e1))
+    extra = {}
+    if cfg == 1:
+        # launch-bound: one request per inference (its own plan, one launch), against a kernel that does nothing
+        from paper_2403_00176_b200 import binding as B
+
+        def timed(fn, n):
+            ts = []
+            for i in range(n):
+                flush.fill_(i & 0xFF)      # also keeps the GPU busy while the host enqueues: device time, not enqueue time
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                fn()
+                e1.record(stream)
+                torch.cuda.synchronize(dev)
+                ts.append(e0.elapsed_time(e1))
+            return float(np.median(ts))
+
+        singles = [sess.prepare([r]) for r in wl.batch(0)]
+        for p1 in singles:
+            p1.run()
+        B.sod2_launch_empty(sess.stream)
+        torch.cuda.synchronize(dev)
+        single_ms = float(np.median([timed(p1.run, 10) for p1 in singles]))
+        empty_ms = timed(lambda: B.sod2_launch_empty(sess.stream), 50)
+        extra = {"ms_one_request_per_inference": single_ms, "ms_empty_kernel": empty_ms, "ratio_to_empty_kernel": single_ms / empty_ms}
     # per-group roofline on the first batch
     rep = PF.group_report(preps[0], hbm, tf, reps=5)
     kinds = PF.kind_summary(rep)
@@ -143,6 +168,7 @@ def measure(cfg: int, reps: int, oracle_budget: float):
         "sum_tensor_bytes": mem["sum_bytes"], "n_groups": sess.graph.num_groups(), "n_ops": sess.graph.num_ops(),
         "gpu_launches": preps[0].plan.run_timed and None,
         "oracle_ms": oracle_ms, "oracle_cores": os.cpu_count(), "oracle_sample": sample, "peaks": src,
+        **extra,
     }
 
 
@@ -164,6 +190,12 @@ def main():
         print(f"| {r['cfg']} | {r['ms_median']:.3f}, {r['ms_min']:.3f} | {r['ms_graph_median']:.3f}, {r['ms_graph_min']:.3f} | {r['ms_per_request']:.4f} | {r['sum_t_roof_over_t_step']:.3f} | "
               f"{r['worst_group']['kind']}: {r['worst_group']['frac']:.3f}, {r['worst_group']['bound']} | {r['plan_us_median']:.0f} ({r['plan_us_cache_hit'] or 0:.0f}) | "
               f"{r['arena_bytes'] / 1e6:.1f} / {r['peak_live_bytes'] / 1e6:.1f} | {r['oracle_ms']:.0f} ({r['oracle_cores']}) |")
+    for r in rows:
+        if "ratio_to_empty_kernel" in r:
+            print(f"\ncfg {r['cfg']} is launch-bound: one request per inference {r['ms_one_request_per_inference'] * 1e3:.2f} us, "
+                  f"a kernel that does nothing {r['ms_empty_kernel'] * 1e3:.2f} us (ratio {r['ratio_to_empty_kernel']:.2f}); "
+                  f"the {r['units_batch0']} rows of all requests as one packed launch {r['ms_median'] * 1e3:.2f} us. "
+                  "A roofline fraction says nothing at this size.")
 
 
 if __name__ == "__main__":
