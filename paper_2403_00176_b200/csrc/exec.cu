@@ -294,6 +294,9 @@ struct Builder {
         return waves * stages * std::max(std::max(mma, floor_cycles), tma);
       };
       int bn = (N > 128 && makespan(256, 1) <= makespan(128, 2)) ? 256 : 128;
+      // Small problems: while 128x64 tiles still fit one wave, a CTA's time is pipeline fill + main loop +
+      // epilogue of ONE tile, and both of the latter shrink with the tile (the epilogue is 0.6 us per 64 columns).
+      if (bn == 128 && N > 64 && static_cast<int64_t>(tiles_m) * ((N + 63) / 64) <= sms) bn = 64;
       const bool hb = G.bias >= 0, hr = G.res >= 0;
       const int act = G.act;
       const int act2 = G.act2;
@@ -318,7 +321,7 @@ struct Builder {
         ep.status = reinterpret_cast<int*>(x.arena);
         const int tiles = tiles_m * static_cast<int>((N + bn - 1) / bn);
         const int grid = std::min(tiles, x.plan->sm_count);
-        const int variant = (bn == 256 ? 0 : 6) + act * 2 + (hr ? 1 : 0);
+        const int variant = (bn == 256 ? 0 : bn == 128 ? 6 : 12) + act * 2 + (hr ? 1 : 0);
         const dim3 gd(grid), bd(k::GEMM_THREADS);
         const int Ni = static_cast<int>(N), Ki = static_cast<int>(K);
 #define SOD2_GEMM_CASE(V, BN_, KCH_, ST_, ACT_, RES_)                                                                        \
@@ -342,8 +345,14 @@ struct Builder {
           SOD2_GEMM_CASE(8, 128, 2, 3, 1, false)
           SOD2_GEMM_CASE(9, 128, 2, 3, 1, true)
           SOD2_GEMM_CASE(10, 128, 2, 3, 2, false)
-          default:
           SOD2_GEMM_CASE(11, 128, 2, 3, 2, true)
+          SOD2_GEMM_CASE(12, 64, 2, 3, 0, false)
+          SOD2_GEMM_CASE(13, 64, 2, 3, 0, true)
+          SOD2_GEMM_CASE(14, 64, 2, 3, 1, false)
+          SOD2_GEMM_CASE(15, 64, 2, 3, 1, true)
+          SOD2_GEMM_CASE(16, 64, 2, 3, 2, false)
+          default:
+          SOD2_GEMM_CASE(17, 64, 2, 3, 2, true)
         }
 #undef SOD2_GEMM_CASE
         return cudaGetLastError();
