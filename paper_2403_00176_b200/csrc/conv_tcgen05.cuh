@@ -742,6 +742,67 @@ __global__ void __launch_bounds__(256) gate_logit_f64(GateParams p) {
   }
 }
 
+// The same gate as ONE CTA: a warp per image (lane-strided channels in order, fixed shuffle tree), then warp 0
+// partitions the ids and all warps clear the executed rows.  No ticket, no second trip through global memory
+// for the gate bits and the id list: what the grid form above spends on its chain of dependent round trips
+// (ticket atomic, gate bytes, id list) this form does behind one CTA barrier.  For the table form of the sums
+// (a few slabs per image at most), where one SM can read all of them in about a microsecond.
+__global__ void __launch_bounds__(1024) gate_logit_block_f64(GateParams p, int N) {
+  __shared__ int n_exec;
+  ptx::pdl_wait();
+  ptx::pdl_launch();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const double bias = static_cast<double>(__bfloat162float(p.b[0]));
+  for (int img = warp; img < N; img += 32) {
+    const double* pp = p.partial + static_cast<long long>(img) * p.slabs * p.C;
+    double acc = 0.0;
+    if (p.slabs == 1) {
+      for (int c0 = lane; c0 < p.C; c0 += 128) {       // four loads in flight per lane, added in channel order
+        double v[4], w[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int c = c0 + 32 * q;
+          v[q] = c < p.C ? pp[c] : 0.0;
+          w[q] = c < p.C ? static_cast<double>(__bfloat162float(p.w[c])) : 0.0;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc += v[q] * w[q];
+      }
+    } else {
+      for (int c = lane; c < p.C; c += 32) {
+        double sl = 0.0;
+        for (int k = 0; k < p.slabs; ++k) sl += pp[static_cast<long long>(k) * p.C + c];
+        acc += sl * static_cast<double>(__bfloat162float(p.w[c]));
+      }
+    }
+    acc /= static_cast<double>(p.HW);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) {
+      const double z = acc + bias;
+      p.gate[img] = z > 0.0 ? 1 : 0;
+      if (p.z_out) {
+        if (p.z_bf16) reinterpret_cast<__nv_bfloat16*>(p.z_out)[img] = __double2bfloat16(z);
+        else reinterpret_cast<float*>(p.z_out)[img] = static_cast<float>(z);
+      }
+    }
+  }
+  if (p.ticket) {          // here only a flag: partition the ids too
+    __syncthreads();       // the gate bytes written above are visible to warp 0
+    if (warp == 0) {
+      const int ne = partition_by_gate(p.part, lane);
+      if (lane == 0) n_exec = ne;
+    }
+    if (p.zero_rows) {
+      __syncthreads();     // the id list written by warp 0 is visible to the CTA
+      for (int k2 = warp; k2 < n_exec; k2 += 32) {
+        double* rowp = p.zero_rows + static_cast<long long>(p.part.idx_exec[k2]) * p.C;
+        for (int cc = lane; cc < p.C; cc += 32) rowp[cc] = 0.0;
+      }
+    }
+  }
+}
+
 __global__ void __launch_bounds__(32) gate_partition(PartitionParams p) {
   ptx::pdl_wait();
   ptx::pdl_launch();

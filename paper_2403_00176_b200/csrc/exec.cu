@@ -1227,7 +1227,9 @@ struct Builder {
           q.part.count_skip = reinterpret_cast<long long*>(auxp + 2 * N * 4);
           q.zero_rows = zero_exec ? sums : nullptr;
         }
-        launch_pdl(k::gate_logit_f64, dim3(N), dim3(256), 0, x.stream, q);
+        // the sums table (or a few slabs per image): one CTA, a warp per image; many slabs: a CTA per image and a ticket
+        if (q.slabs <= 4) launch_pdl(k::gate_logit_block_f64, dim3(1), dim3(1024), 0, x.stream, q, N);
+        else launch_pdl(k::gate_logit_f64, dim3(N), dim3(256), 0, x.stream, q);
         return cudaGetLastError();
       });
     }
