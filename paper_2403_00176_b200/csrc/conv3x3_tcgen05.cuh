@@ -134,6 +134,7 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ Conv3Batch B, const __grid_con
           const int s = n % STAGES;
           if (n >= STAGES) ptx::mbar_wait(&empty[s], ((n / STAGES) - 1) & 1, dead);
           const int dy = ks / cchunks, cc = ks % cchunks;
+          SOD2_TRACE(0, 100 + ks)
           ptx::mbar_expect_tx(&full[s], C3_A_BYTES);
           ptx::tma_load_4d(tiles + s * S::STAGE_BYTES, &B.tx[rq], cc * 64, w0 - 1, h0 + dy - 1, img, &full[s]);
         }
@@ -179,6 +180,7 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ Conv3Batch B, const __grid_con
           ptx::mbar_wait(&full[s], (n / STAGES) & 1, dead);
           if (!mine) continue;
           ptx::tc_fence_after();
+          if (me == 0) { SOD2_TRACE(1, 200 + ks) }
           const uint32_t a = ptx::smem_u32(tiles + s * S::STAGE_BYTES);
           const uint32_t b = RES ? ptx::smem_u32(wres) + ks * 3 * BN * 128 : a + C3_A_SLOT;
 #pragma unroll
@@ -191,6 +193,7 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ Conv3Batch B, const __grid_con
           ptx::mma_commit(&empty[s]);
         }
         if (mine) ptx::mma_commit(&tmem_full[acc]);
+        if (mine && me == 0) { SOD2_TRACE(1, 210) }
       }
     }
   } else if (warp == 2) {
@@ -220,6 +223,7 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ Conv3Batch B, const __grid_con
       for (int u = 0; u < U; ++u) {
         const int bsel = u % NSB;
         ptx::mbar_wait(&stage_ready[bsel], (u / NSB) & 1, dead);
+        SOD2_TRACE(2, 300)
         const int t = blockIdx.x + (u / PASSES) * gridDim.x;
         int n0, img, h0, w0;
         const int rq = decode(t, &n0, &img, &h0, &w0);
@@ -230,6 +234,7 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ Conv3Batch B, const __grid_con
         }
         if (u + NSB < U) {
           bulk_wait_read0();
+          SOD2_TRACE(2, 310)
           prepare(u + NSB);
         }
       }
@@ -258,6 +263,7 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ Conv3Batch B, const __grid_con
       if (warp == 4) ptx::mbar_wait_warp(&tmem_full[acc], (j >> 1) & 1, dead);   // one polling warp, the others park at the barrier
       conv_epi_bar();
       ptx::tc_fence_after();
+      if (et == 0) { SOD2_TRACE(3, 400) }
 #pragma unroll 1
       for (int ps = 0; ps < PASSES; ++ps, ++u) {
         const int np = n0 + ps * 64;
@@ -283,6 +289,7 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ Conv3Batch B, const __grid_con
           for (int i = 0; i < 32; ++i) v[i] = apply_act<ACT>(__uint_as_float(r[i]) + bp[i]);
         }
         ptx::mbar_wait_warp(&res_full[bsel], (u / NSB) & 1, dead);
+        if (et == 0) { SOD2_TRACE(3, 410) }
         if (live) {
           uint4 pk[4];
           if constexpr (HASRES) {
@@ -324,6 +331,7 @@ conv3x3_rows_bf16_tcgen05(const __grid_constant__ Conv3Batch B, const __grid_con
         ptx::fence_proxy_async();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&stage_ready[bsel]);
+        if (et == 0) { SOD2_TRACE(3, 420) }
       }
     }
   }
