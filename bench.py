@@ -236,6 +236,52 @@ def run_ours(args):
         if hit:
             th.append((time.perf_counter() - t0) * 1e6)
     plan_hit_us = sorted(th)[len(th) // 2] if th else None
+
+    # ---- the same work as a serving loop would issue it: the copies of neighbouring inferences overlap the
+    # kernels (input copies on one stream, kernels on a second, result copies on a third, ordered by events; every
+    # batch has its own device buffers).  Still host buffers in, host buffers out, every inference; what is
+    # reported is the time per inference of the whole loop (a throughput figure, not the latency of one call).
+    e2e_pipe_ms = None
+    keys = [k for k in range(len(preps)) if k in pinned_in]
+    if use_graph and len(keys) >= 3:
+        s_in, s_run, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+        for k in keys:      # plans cached and graphs captured for the stream they will run on
+            pr = preps[k]
+            _, pl, _ = sess.graph.plan_cached(wl.sym_names, [[r.syms[s] for s in wl.sym_names] for r in pr.reqs])
+            pl.run_graph([t.data_ptr() for t in pr.in_dev], [t.data_ptr() for t in pr.out_dev], pr.arena.data_ptr(), pr.arena.numel(),
+                         s_run.cuda_stream)
+        torch.cuda.synchronize(dev)
+        n_pipe = 4 * len(keys)
+        last_run, last_out = {}, {}     # a batch's buffers are reused every len(keys) inferences: order the reuse
+        t0 = time.perf_counter()
+        for i in range(n_pipe):
+            k = keys[i % len(keys)]
+            pr = preps[k]
+            with torch.cuda.stream(s_in):
+                if k in last_run:
+                    s_in.wait_event(last_run[k])       # the kernels that read these input buffers last time
+                for dst, src in zip(pr.in_dev, pinned_in[k]):
+                    dst.copy_(src, non_blocking=True)
+                ev_in = torch.cuda.Event()
+                ev_in.record(s_in)
+            _, pl, _ = sess.graph.plan_cached(wl.sym_names, [[r.syms[s] for s in wl.sym_names] for r in pr.reqs])
+            s_run.wait_event(ev_in)
+            if k in last_out:
+                s_run.wait_event(last_out[k])          # the copy that read these output buffers last time
+            pl.run_graph([t.data_ptr() for t in pr.in_dev], [t.data_ptr() for t in pr.out_dev], pr.arena.data_ptr(), pr.arena.numel(),
+                         s_run.cuda_stream)
+            ev_run = torch.cuda.Event()
+            ev_run.record(s_run)
+            last_run[k] = ev_run
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_run)
+                for dst, src in zip(pinned_out[k], pr.out_dev):
+                    dst.copy_(src, non_blocking=True)
+                ev_out = torch.cuda.Event()
+                ev_out.record(s_out)
+                last_out[k] = ev_out
+        torch.cuda.synchronize(dev)
+        e2e_pipe_ms = (time.perf_counter() - t0) * 1e3 / n_pipe
     sess.graph.set_plan_cache(0)
 
     # ---- planning overhead (host): bind + plan per batch
@@ -279,7 +325,9 @@ def run_ours(args):
             "clocks": clocks,
             "e2e": {"value": e2e_ms, "unit": "ms/inference", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                     "includes": "H2D (pinned, enqueued first) + bind_dims + plan + run + D2H (pinned)",
-                    "value_plan_cache_hit": e2e_hit_ms},
+                    "value_plan_cache_hit": e2e_hit_ms,
+                    "value_pipelined": e2e_pipe_ms,
+                    "pipelined": "plan cache + graph replay, copies of neighbouring inferences overlapped on their own streams: loop time per inference"},
             "plan_us_per_batch": plan_us,
             "plan_us_per_batch_cache_hit": plan_hit_us,
             "arena": mem,
