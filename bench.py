@@ -202,7 +202,10 @@ def run_ours(args):
             h2d = sum(t.numel() for t in pinned_in[key])
             d2h = sum(t.numel() for t in host_out)
         del pl, b
-    e2e_ms = sum(e2e_times) / len(e2e_times)
+    # per-call wall-clock times on a shared host carry outliers (another tenant's interrupt costs a call 0.3-0.7 ms):
+    # the median is the figure, the mean is printed beside it
+    e2e_mean_ms = sum(e2e_times) / len(e2e_times)
+    e2e_ms = sorted(e2e_times)[len(e2e_times) // 2]
 
     # ---- the same loop through the plan cache, every batch seen before (a serving process meets the same
     # bound symbol tuples again; reported beside the uncached number, which stays the e2e value)
@@ -227,7 +230,7 @@ def run_ours(args):
         torch.cuda.synchronize(dev)
         if hit and not info.reserved[1]:      # a cached plan whose graph exists already
             e2e_hit.append((time.perf_counter() - t0) * 1e3)
-    e2e_hit_ms = sum(e2e_hit) / len(e2e_hit) if e2e_hit else None
+    e2e_hit_ms = sorted(e2e_hit)[len(e2e_hit) // 2] if e2e_hit else None
     th = []
     for i in range(5):
         pr = preps[i % len(preps)]
@@ -324,7 +327,8 @@ def run_ours(args):
             "gpu_launches": int(launches),
             "clocks": clocks,
             "e2e": {"value": e2e_ms, "unit": "ms/inference", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-                    "includes": "H2D (pinned, enqueued first) + bind_dims + plan + run + D2H (pinned)",
+                    "includes": "H2D (pinned, enqueued first) + bind_dims + plan + run + D2H (pinned); median over the timed calls",
+                    "value_mean": e2e_mean_ms,
                     "value_plan_cache_hit": e2e_hit_ms,
                     "value_pipelined": e2e_pipe_ms,
                     "pipelined": "plan cache + graph replay, copies of neighbouring inferences overlapped on their own streams: loop time per inference"},
