@@ -288,6 +288,19 @@ def test_cfg3_small_pruning_lockstep_and_ties():
     _check_topk_lockstep(wl, reqs, 3)
 
 
+def test_more_requests_than_one_attention_or_pruning_launch_holds():
+    # attention and the pruning step take up to 32 requests per launch: 40 requests make them launch twice
+    rng = np.random.default_rng(31)
+    wl2 = WL.cfg2(layers=1, D=128, H=2, F=256, n_requests=1, lmin=1, lmax=512)
+    reqs2 = [Request({"L": int(L)}, {"x": bf16_round(rng.standard_normal((1, int(L), 128)).astype(np.float32))}) for L in rng.integers(1, 90, 40)]
+    s, p, outs = run_batch(wl2, reqs2)
+    for r in (0, 17, 31, 32, 39):
+        assert O.rel_err(outs[r]["y"], _oracle_out(wl2, reqs2[r], "y")) <= BF16_TOL, reqs2[r].syms
+    wl3 = WL.cfg3(layers=2, D=128, H=2, F=256, n_requests=1, nmin=4, nmax=800)
+    reqs3 = [Request({"N0": int(n)}, {"x": bf16_round(rng.standard_normal((1, int(n), 128)).astype(np.float32))}) for n in rng.integers(4, 150, 40)]
+    _check_topk_lockstep(wl3, reqs3, 2)
+
+
 def test_cfg3_full_config_batch0_lockstep():
     wl = WL.cfg3()
     reqs = wl.batch(0)[:4]
@@ -336,6 +349,21 @@ def test_cfg4_small_conv_stage_edge_shapes_lockstep():
     outs2 = p.outputs()
     for a, b in zip(outs, outs2):
         assert np.array_equal(a["blk2"], b["blk2"]) and np.array_equal(a["gap"], b["gap"])
+
+
+def test_cfg4_more_requests_than_one_launch_holds():
+    # layout changes, row-halo convolutions and pooling take up to eight requests per launch: nineteen requests
+    # (wide rows for the row-halo kernel, narrow ones for the general kernel, mixed) make every group flush twice
+    wl = WL.cfg4(blocks=2)
+    rng = np.random.default_rng(23)
+    shapes = [(int(rng.integers(1, 12)), int(rng.choice([5, 40, 96, 128, 130, 200]))) for _ in range(19)]
+    reqs = _conv_requests(wl, shapes, seed=29)
+    s, p, outs = run_batch(wl, reqs)
+    for r, req in enumerate(reqs):
+        env = O.run(wl.ir, wl.consts, req.inputs)
+        for name in ("blk1", "gap"):
+            assert outs[r][name].shape == env[name].shape
+            assert O.rel_err(outs[r][name], env[name]) <= BF16_TOL, (req.syms, name)
 
 
 def test_cfg4_full_config_smallest_request_and_properties():
