@@ -544,6 +544,13 @@ def test_cfg5_small_gated_network_lockstep():
     assert gates.shape == (4, 6)
 
 
+def test_cfg5_more_samples_than_a_warp_of_gate_lanes():
+    # 45 samples: the one-CTA gate kernel walks its 32 warps over the images twice and partitions two chunks of ids
+    wl = WL.cfg5(B=45, side=32, widths=(64,), per_stage=2, calibrated=False)
+    gates = _check_gated(wl, wl.batch(0), 2)
+    assert gates.shape == (2, 45) and 0 < gates.sum() < gates.size
+
+
 def test_cfg5_small_gated_network_copy_regroup_lockstep():
     # Switch / Combine as whole-sample copies (the form used where the index-indirect pattern does not apply)
     wl = WL.cfg5(B=6, side=32, widths=(64, 128), per_stage=2)
