@@ -139,8 +139,9 @@ __global__ void __launch_bounds__(256) layernorm_bf16(const __nv_bfloat16* __res
   uint4 g4[CH], b4[CH];
 #pragma unroll
   for (int c = 0; c < CH; ++c) {
-    const int i = c * 32 + lane;
-    if (FULL || i < nvec) { g4[c] = reinterpret_cast<const uint4*>(gamma)[i]; b4[c] = reinterpret_cast<const uint4*>(beta)[i]; }
+    const int i = FULL ? c * 32 + lane : min(c * 32 + lane, nvec - 1);
+    g4[c] = reinterpret_cast<const uint4*>(gamma)[i];
+    b4[c] = reinterpret_cast<const uint4*>(beta)[i];
   }
   ptx::pdl_launch();
   ptx::pdl_wait();
@@ -149,16 +150,21 @@ __global__ void __launch_bounds__(256) layernorm_bf16(const __nv_bfloat16* __res
   float v[CH][8];
   float s = 0.f;
 #pragma unroll
+  // all loads of the row first, unconditionally (a lane past the row's end re-reads the last vector and
+  // discards it): guarded loads would sit in basic blocks of their own and wait for one another
+  uint4 u4[CH];
+#pragma unroll
+  for (int c = 0; c < CH; ++c) u4[c] = xr[FULL ? c * 32 + lane : min(c * 32 + lane, nvec - 1)];
+#pragma unroll
   for (int c = 0; c < CH; ++c) {
-    const int i = c * 32 + lane;
-    if (FULL || i < nvec) {
-      uint4 u = xr[i];
-      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+    const bool in = FULL || c * 32 + lane < nvec;
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u4[c]);
 #pragma unroll
-      for (int t = 0; t < 4; ++t) { float2 f = __bfloat1622float2(h[t]); v[c][2 * t] = f.x; v[c][2 * t + 1] = f.y; s += f.x + f.y; }
-    } else {
-#pragma unroll
-      for (int t = 0; t < 8; ++t) v[c][t] = 0.f;
+    for (int t = 0; t < 4; ++t) {
+      const float2 f = __bfloat1622float2(h[t]);
+      v[c][2 * t] = in ? f.x : 0.f;
+      v[c][2 * t + 1] = in ? f.y : 0.f;
+      s += in ? f.x + f.y : 0.f;
     }
   }
   const float mu = warp_sum(s) / D;
