@@ -823,8 +823,9 @@ __global__ void __launch_bounds__(256) sample_copy(SampleCopyParams p) {
   ptx::pdl_wait();
   ptx::pdl_launch();
   const int j = blockIdx.y;
-  if (j >= *p.count) return;
-  const long long s = p.idx[j];
+  const long long cnt = *p.count;
+  const long long s = p.idx[j];      // requested together with the count (the list has an entry for every j of the grid)
+  if (j >= cnt) return;
   const uint4* src = p.src + (p.scatter == 1 ? static_cast<long long>(j) : s) * p.vec_per_sample;
   uint4* dst = p.dst + (p.scatter != 0 ? s : static_cast<long long>(j)) * p.vec_per_sample;
   for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < p.vec_per_sample; i += static_cast<long long>(gridDim.x) * blockDim.x) dst[i] = src[i];
