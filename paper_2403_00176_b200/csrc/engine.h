@@ -243,6 +243,12 @@ struct Plan {
   // CUDA graph of the whole launch sequence for one set of buffers (run_plan_graph)
   void* graph_exec = nullptr;             // cudaGraphExec_t
   void* capture_stream = nullptr;         // cudaStream_t the sequence is captured on
+  // groups that run beside their predecessor on a second stream (forked before the predecessor's first launch,
+  // joined after their own last one): both only read what came before and write their own outputs
+  std::vector<char> side_group;           // [group]
+  void* side_stream = nullptr;            // cudaStream_t
+  void* ev_fork = nullptr;                // cudaEvent_t
+  void* ev_join = nullptr;                // cudaEvent_t
   std::vector<const void*> graph_key;     // inputs, outputs, arena the graph was captured with
   Plan() = default;
   Plan(const Plan&) = delete;

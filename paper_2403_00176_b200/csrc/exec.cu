@@ -1445,6 +1445,13 @@ struct Builder {
     p.group_bytes.clear();
     p.gpu_launches = 0;
     // the fp32 row kernel and the elementwise chains have no bounded waits, tickets or device-side counts
+    // a pooling group right after a layout change of the same tensor: neither reads what the other writes
+    p.side_group.assign(c.groups.size(), 0);
+    for (size_t gi = 1; gi < c.groups.size(); ++gi) {
+      const Group &A = c.groups[gi - 1], &Bg = c.groups[gi];
+      if (Bg.kind == GKind::GAP && A.kind == GKind::LAYOUT && Bg.a != A.out && A.a != Bg.out && !p.side_group[gi - 1])
+        p.side_group[gi] = 1;
+    }
     p.uses_header = false;
     for (const Group& G : c.groups)
       if (!((G.kind == GKind::GEMM && g.tensors[G.a].dtype == DType::F32) || G.kind == GKind::CHAIN)) p.uses_header = true;
@@ -1572,6 +1579,25 @@ Status run_plan_timed(Plan* p, const void* const* inputs, void* const* outputs, 
 Plan::~Plan() {
   if (graph_exec) cudaGraphExecDestroy(static_cast<cudaGraphExec_t>(graph_exec));
   if (capture_stream) cudaStreamDestroy(static_cast<cudaStream_t>(capture_stream));
+  if (side_stream) cudaStreamDestroy(static_cast<cudaStream_t>(side_stream));
+  if (ev_fork) cudaEventDestroy(static_cast<cudaEvent_t>(ev_fork));
+  if (ev_join) cudaEventDestroy(static_cast<cudaEvent_t>(ev_join));
+}
+
+// The second stream and the two events of a plan with side groups (made outside any stream capture).
+static bool ensure_side_stream(Plan* p) {
+  bool any = false;
+  for (char c : p->side_group) any = any || c;
+  if (!any || p->side_stream) return true;
+  cudaStream_t s;
+  cudaEvent_t a, b;
+  if (cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess) return false;
+  if (cudaEventCreateWithFlags(&a, cudaEventDisableTiming) != cudaSuccess || cudaEventCreateWithFlags(&b, cudaEventDisableTiming) != cudaSuccess) {
+    cudaStreamDestroy(s);
+    return false;
+  }
+  p->side_stream = s; p->ev_fork = a; p->ev_join = b;
+  return true;
 }
 
 Status run_plan_graph(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream,
@@ -1592,6 +1618,7 @@ Status run_plan_graph(Plan* p, const void* const* inputs, void* const* outputs, 
       p->capture_stream = cs;
     }
     cudaStream_t cs = static_cast<cudaStream_t>(p->capture_stream);
+    if (!ensure_side_stream(p)) { p->err = "cannot create the second stream"; return E_CUDA; }
     if (cudaStreamBeginCapture(cs, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { p->err = "cannot begin the stream capture"; return E_CUDA; }
     Status s = run_plan(p, inputs, outputs, arena, arena_bytes, cs, nullptr);
     cudaGraph_t graph = nullptr;
@@ -1631,12 +1658,42 @@ Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* 
   }
   RunCtx x{inputs, outputs, static_cast<char*>(arena), static_cast<char*>(p->c->packed_ws), static_cast<cudaStream_t>(stream), p};
   if (p->uses_header && cudaMemsetAsync(arena, 0, 256, x.stream) != cudaSuccess) { p->err = "cannot clear the status word"; return E_CUDA; }
-  for (auto& L : p->launches) {
-    cudaError_t e = L->fn(x);
+  if (!ensure_side_stream(p)) { p->err = "cannot create the second stream"; return E_CUDA; }
+  const int n_groups = static_cast<int>(p->side_group.size());
+  cudaStream_t side = static_cast<cudaStream_t>(p->side_stream);
+  bool open_fork = false;
+  for (size_t i = 0; i < p->launches.size(); ++i) {
+    auto& L = p->launches[i];
+    const int g = L->group;
+    const bool first_of_group = i == 0 || p->launches[i - 1]->group != g;
+    const bool last_of_group = i + 1 == p->launches.size() || p->launches[i + 1]->group != g;
+    const bool on_side = side && g >= 0 && g < n_groups && p->side_group[g] && open_fork;
+    if (side && first_of_group && !open_fork && g + 1 < n_groups && p->side_group[g + 1]) {
+      // the next group runs beside this one: it may start as soon as everything before this group is done
+      if (cudaEventRecord(static_cast<cudaEvent_t>(p->ev_fork), x.stream) != cudaSuccess ||
+          cudaStreamWaitEvent(side, static_cast<cudaEvent_t>(p->ev_fork), 0) != cudaSuccess) { p->err = "fork failed"; return E_CUDA; }
+      open_fork = true;
+    }
+    RunCtx xs = x;
+    if (on_side) xs.stream = side;
+    cudaError_t e = L->fn(xs);
+    if (e == cudaSuccess && on_side && last_of_group) {
+      if (cudaEventRecord(static_cast<cudaEvent_t>(p->ev_join), side) != cudaSuccess ||
+          cudaStreamWaitEvent(x.stream, static_cast<cudaEvent_t>(p->ev_join), 0) != cudaSuccess) { p->err = "join failed"; return E_CUDA; }
+      open_fork = false;
+    }
     if (e != cudaSuccess) {
+      if (open_fork) {   // never leave the second stream forked (a capture could not end)
+        cudaEventRecord(static_cast<cudaEvent_t>(p->ev_join), side);
+        cudaStreamWaitEvent(x.stream, static_cast<cudaEvent_t>(p->ev_join), 0);
+      }
       p->err = std::string("launch failed in group ") + std::to_string(L->group) + ": " + cudaGetErrorString(e);
       return E_CUDA;
     }
+  }
+  if (open_fork) {       // a side group without launches: join all the same
+    cudaEventRecord(static_cast<cudaEvent_t>(p->ev_join), side);
+    cudaStreamWaitEvent(x.stream, static_cast<cudaEvent_t>(p->ev_join), 0);
   }
   if (info) {
     info[0] = std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t0).count();
