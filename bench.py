@@ -7,7 +7,12 @@ padding-free).  One "step" = one inference = one sod2_run over one batch.
 
 Prints ONE JSON line.  `value` is ms per inference with inputs resident in HBM; `e2e` is the same
 through the public API with host buffers (bind + plan + H2D + run + D2H per step).  `roofline`
-describes the dominant kernel (the tcgen05 GEMM), `cpu_baseline` the oracle on the host cores.
+describes the dominant kernel (the tcgen05 GEMM), `cpu_baseline` the oracle on the host cores, and
+`configs` carries one record per workload (cfg 1..5: latency stream-launched and graph-replayed, end to
+end, roofline sums, worst group, planning overhead, arena), measured in the same process.
+
+A plain `python bench.py --gpus N` (N > 1, no WORLD_SIZE in the environment) re-executes itself under
+torch.distributed.run with N ranks on 127.0.0.1: N independent replicas, no collective on the data path.
 """
 from __future__ import annotations
 
@@ -87,8 +92,18 @@ class ClockSampler:
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(s)}
 
 
-def gemm_algorithmic_flops(T, D=768, F=3072, layers=6):
-    return 2.0 * T * (D * 3 * D + D * D + D * F + F * D) * layers
+def _stored_traffic():
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary (the line
+    `traffic_bytes_per_launch: <bytes> (commit <hash>, T = <tokens>)`); None if the summary has no such line."""
+    import re
+    path = os.path.join(ROOT, "profiles", "gemm_bf16_tcgen05_cfg2.md")
+    try:
+        m = re.search(r"traffic_bytes_per_launch:\s*([0-9.eE+]+)\s*\(commit\s+(\w+),\s*T\s*=\s*(\d+)\)", open(path).read())
+    except OSError:
+        return None
+    if not m:
+        return None
+    return {"bytes": float(m.group(1)), "commit": m.group(2), "tokens": int(m.group(3)), "file": "profiles/gemm_bf16_tcgen05_cfg2.md"}
 
 
 def run_ours(args):
@@ -162,7 +177,7 @@ def run_ours(args):
 
     # ---- per-group device times (CUDA events recorded by the library on this stream around every
     # launch) against each group's algorithmic roofline; the dominant kernel is the tcgen05 GEMM.
-    from paper_2403_00176_b200 import profile as PF
+    import report as PF
     mid = sorted(range(len(preps)), key=lambda i: tokens[i])[len(preps) // 2]
     report = PF.group_report(preps[mid], peaks["hbm_gbs"], peaks["tf_sustained"], reps=7)
     kinds = PF.kind_summary(report)
@@ -313,6 +328,7 @@ def run_ours(args):
         ms_per_step = my_ms / args.steps
         cpu = None if args.skip_cpu_baseline else cpu_baseline(wl)
         mem = preps[0].plan.memory()
+        traffic = _stored_traffic()
         line = {
             "metric": METRIC, "value": ms_per_step, "unit": "ms/inference", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
@@ -337,13 +353,16 @@ def run_ours(args):
             "arena": mem,
             "roofline": {"bound": "tensor", "achieved": gemm["tflops"], "peak": peaks["tf_sustained"], "unit": "TFLOP/s",
                          "frac": gemm["tflops"] / peaks["tf_sustained"],
-                         # mean DRAM bytes per GEMM launch of one layer's four GEMMs at T = 1929 (ncu, cold cache):
-                         # profiles/gemm_bf16_tcgen05_cfg2.md
-                         "traffic": 10.1e6, "traffic_unit": "bytes per launch (ncu dram read+write, T=1929)",
+                         "traffic": traffic["bytes"] if traffic else None,
+                         "traffic_unit": (f"bytes per launch (ncu dram read+write, cold cache, T={traffic['tokens']}, commit {traffic['commit']}, "
+                                          f"{traffic['file']})") if traffic else None,
+                         "timing": "CUDA events around every launch of the group's kernels on the run's stream (sod2_run_timed): no overlap "
+                                   "between dependent kernels and no graph, so the groups sum to more than ms_per_step and frac understates "
+                                   "what the kernel reaches inside the replayed graph",
                          "peak_source": peaks["src"] + " cuBLAS bf16, sustained (kernel timed inside a long step)",
                          "kernel": "gemm_bf16_tcgen05", "launches": gemm["launch_groups"],
                          "avg_us": gemm["ms"] / gemm["launch_groups"] * 1e3,
-                         "share_of_step": gemm["ms"] / step_sum_ms,
+                         "share_of_group_sum": gemm["ms"] / step_sum_ms,
                          "batch_tokens": tokens[mid]},
             "groups": {k: {"ms": round(v["ms"], 4), "frac": round(v["frac"], 3), "share": round(v["ms"] / step_sum_ms, 3),
                            "tflops": round(v["tflops"], 1), "gbs": round(v["gbs"], 1)} for k, v in kinds.items()},
@@ -351,6 +370,22 @@ def run_ours(args):
             "cpu_baseline": cpu,
             "wall_s": t_wall,
         }
+        if not args.no_configs:
+            # one record per workload, same process and GPU; cfg 2's record repeats the headline protocol on 5 batches
+            del preps, flush
+            torch.cuda.empty_cache()
+            line["configs"] = {}
+            for cfg in (1, 2, 3, 4, 5):
+                r = PF.measure(cfg, args.config_reps, device=f"cuda:{local}")
+                line["configs"][f"cfg{cfg}"] = {
+                    "workload": r["workload"], "ms": r["ms_median"], "ms_graph": r["ms_graph_median"], "e2e_ms": r["e2e_ms"],
+                    "sum_t_roof_over_t": r["sum_t_roof_over_t_step"], "sum_t_roof_over_group_sum": r["sum_t_roof_over_sum_t_groups"],
+                    "worst_group": r["worst_group"], "kinds": r["kinds"], "plan_us": r["plan_us_median"],
+                    "plan_us_cache_hit": r["plan_us_cache_hit"], "arena_bytes": r["arena_bytes"], "peak_live_bytes": r["peak_live_bytes"],
+                    "gpu_launches": r["gpu_launches"], "units": r["units_batch0"], "unit": r["unit"],
+                    **{k: r[k] for k in ("ms_one_request_per_inference", "ms_empty_kernel", "ratio_to_empty_kernel") if k in r}}
+            line["configs_note"] = ("ms / ms_graph: device time per inference (median, L2 flushed), stream-launched / replayed as one CUDA graph; "
+                                    "e2e_ms: pinned H2D + bind + plan + run + D2H; group figures: CUDA events around every launch")
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -416,8 +451,18 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--skip-cpu-baseline", action="store_true", help="omit the oracle timing (profiling runs)")
     ap.add_argument("--no-graph", action="store_true", help="one launch per kernel in the timed steps instead of one CUDA graph per batch")
+    ap.add_argument("--no-configs", action="store_true", help="omit the per-config records (profiling runs)")
+    ap.add_argument("--config-reps", type=int, default=20, help="timed inferences per config for the per-config records")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # plain `python bench.py --gpus N`: become N ranks (one replica per GPU) under torch.distributed.run
+        import socket
+        with socket.socket() as s:
+            s.bind(("127.0.0.1", 0))
+            port = s.getsockname()[1]
+        os.execv(sys.executable, [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+                                  "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *sys.argv[1:]])
     if args.impl == "reference":
         run_reference(args)
     else:

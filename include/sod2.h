@@ -4,7 +4,7 @@
  * possible on dynamic DNNs.  The calls follow the staging the paper describes: static analysis before
  * deployment (Section 4.1-4.3: operator classification, RDP = Algorithm 1, fusion, partition at
  * execution-determined operators), then, per input, evaluation of the shape expressions and the
- * memory allocation plan "at execution time when all tensor sizes are known" (Section 4.4.1), then
+ * memory allocation plan, made once the input has fixed every tensor size (Section 4.4.1), then
  * inference.
  *
  * Conventions
@@ -54,7 +54,8 @@ typedef enum {
 sod2_status sod2_graph_create(const char* ir_text, size_t ir_len, uint32_t opt_flags, sod2_graph** out);
 void sod2_graph_destroy(sod2_graph* g);
 
-/* Attach caller-owned device memory holding a float constant (weights) in the layout the graph
+/* Attach caller-owned device memory holding a float constant (weights: the constant inputs of the
+ * computational graph, Section 3) in the layout the graph
  * declares (row-major, graph dtype).  The memory must outlive every run. */
 sod2_status sod2_graph_set_const(sod2_graph* g, const char* name, const void* dev_ptr, size_t bytes);
 
@@ -64,7 +65,8 @@ sod2_status sod2_graph_set_const(sod2_graph* g, const char* name, const void* de
 sod2_status sod2_graph_prepack_bytes(const sod2_graph* g, size_t* bytes);
 sod2_status sod2_graph_prepack(sod2_graph* g, void* dev_workspace, size_t bytes, void* cuda_stream);
 
-/* H0: bind symbol values for n_requests requests.  values is [n_requests][n_syms] row-major (host).
+/* H0: bind symbol values for n_requests requests (Section 4.1: the symbolic constants of the RDP
+ * lattice get their values once an input arrives; Section 4.4.1: all sizes are then known).  values is [n_requests][n_syms] row-major (host).
  * Evaluates every shape expression of every tensor for every request and checks the bind-time
  * assertions RDP recorded.  Errors: unknown / unbound symbol, value outside the declared range,
  * shape conflict. */
@@ -97,7 +99,10 @@ typedef struct {
   int64_t reserved[6];
 } sod2_run_info;
 
-/* Enqueue one inference (all requests of the binding) on cuda_stream.  inputs[i] / outputs[j] are
+/* Enqueue one inference (all requests of the binding) on cuda_stream: the fused groups (Section 4.2) of
+ * each sub-graph of the partition at execution-determined operators (Section 4.3), in planned order, in
+ * the arena laid out by sod2_plan (Section 4.4.1), each group by the kernel version chosen for its bound
+ * shapes (Section 4.4.2).  inputs[i] / outputs[j] are
  * device pointers in graph declaration order, packed per request as described above; outputs whose
  * shape is execution-determined must be sized for the static upper bound (sod2_binding_shape reports
  * it) and their true shape is read with sod2_run_output_shape after the stream has been synchronised.
@@ -197,7 +202,8 @@ sod2_status sod2_run_output_shape(sod2_plan_t* p, const void* arena, void* cuda_
  * calls that overlap on the GPU (two streams, two threads) race; it keeps the previous call's
  * contents, which is harmless because every call overwrites each counter before reading it.  The
  * first call on a device looks up the array's address and should be made outside any stream
- * capture.  Calls no cudaMalloc / cudaFree or allocating routine.  Asynchronous on cuda_stream.
+ * capture.  The device that holds dev_x must be the current device and own cuda_stream.  Calls no
+ * cudaMalloc / cudaFree or allocating routine.  Asynchronous on cuda_stream.
  * Errors: SOD2_E_INVALID_ARG, SOD2_E_RANK_MISMATCH, SOD2_E_BAD_DIM, SOD2_E_CUDA; message through
  * sod2_last_error(NULL). */
 #define SOD2_NONZERO_STATIC_MAX_ELEMS 16777216LL

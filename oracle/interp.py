@@ -17,8 +17,12 @@ Pins (tests/test_oracle_pins.py): MatMul and Conv against hand loops and scipy's
 correlate2d, 1x1 conv == MatMul, delta-kernel conv == shift; Gelu against math.erf and
 the identity Gelu(x)-Gelu(-x)=x; LayerNorm and Softmax invariants; top-k keep against a
 stable argsort; NonZero against numpy.nonzero; Switch/Combine against masked
-execute-all; the Fig. 4 chain against explicit loops.  Nothing here is "parity unpinned"
-except the reading of tolerances and decision bands, which is a convention, not a value.
+execute-all; the Fig. 4 chain against explicit loops; GlobalAveragePool, the gate chain
+(pool -> linear -> Greater, with a logit of exactly zero), LayerNorm and Softmax values against
+loops; Greater, Range, ConstantOfShape, Cast, Div, Sub, Reshape's 0 / -1 rules, ReduceSumSquare,
+Relu, Shape, Transpose, Concat, Gather and Slice against literal arrays.  Nothing here is
+"parity unpinned" except the reading of tolerances and decision bands, which is a convention,
+not a value.
 """
 from __future__ import annotations
 

@@ -128,13 +128,28 @@ extern "C" sod2_status sod2_nonzero_static(const void* dev_x, int dtype, int ran
   long long numel = 1;
   for (int i = 0; i < rank; ++i) {
     if (dims[i] < 0) return nzs_fail(SOD2_E_BAD_DIM, "sod2_nonzero_static: negative extent");
-    numel *= dims[i];
-    if (numel > NZS_MAX_ELEMS)
+    // compared before multiplying: the product of two large extents would wrap around the 64-bit range and
+    // pass as a small (or empty) input.  An extent of 0 anywhere makes the input empty, whatever the others are.
+    if (numel > 0 && dims[i] > NZS_MAX_ELEMS / numel)
       return nzs_fail(SOD2_E_BAD_DIM, "sod2_nonzero_static: input has more than " + std::to_string(NZS_MAX_ELEMS) +
                                           " elements, the limit of the built-in scratch; use the arena-based path");
+    numel *= dims[i];
   }
+  // every extent is checked even when an earlier one is 0 (an empty input must still have sane extents)
+  for (int i = 0; i < rank; ++i)
+    if (dims[i] > NZS_MAX_ELEMS)
+      return nzs_fail(SOD2_E_BAD_DIM, "sod2_nonzero_static: an extent exceeds " + std::to_string(NZS_MAX_ELEMS));
+  // the scratch array of the device that owns the input (the stream must belong to the same device)
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nzs_fail(SOD2_E_CUDA, "sod2_nonzero_static: no current device");
+  {
+    cudaPointerAttributes at{};
+    if (cudaPointerGetAttributes(&at, dev_x) == cudaSuccess && at.type == cudaMemoryTypeDevice) dev = at.device;
+    else { cudaGetLastError(); if (cudaGetDevice(&dev) != cudaSuccess) return nzs_fail(SOD2_E_CUDA, "sod2_nonzero_static: no current device"); }
+  }
+  if (dev < 0 || dev >= 64) return nzs_fail(SOD2_E_CUDA, "sod2_nonzero_static: device index out of range");
+  int cur = 0;
+  if (cudaGetDevice(&cur) != cudaSuccess) return nzs_fail(SOD2_E_CUDA, "sod2_nonzero_static: no current device");
+  if (cur != dev) return nzs_fail(SOD2_E_INVALID_ARG, "sod2_nonzero_static: the device that holds dev_x must be the current device");
   if (!g_nzs_addr[dev]) {
     int* ptr = nullptr;
     const cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_nzs_counters);

@@ -1,8 +1,9 @@
-"""Per-config measurement report (all five workloads): latency, per-group roofline fractions, planning
-overhead, arena size, and the oracle timed on the host cores.  Prints one JSON object per config and a
-markdown table.  Measurement only: every device number comes from CUDA events.
+"""Per-config measurement (all five workloads): latency, per-group roofline fractions, planning
+overhead and arena size.  Prints one JSON object per config and a markdown table.  Measurement only:
+every device number comes from CUDA events, and nothing here touches the CPU oracle (bench.py times
+that, in its cpu_baseline leg).  bench.py calls measure() for the per-config records of its line.
 
-    python -m paper_2403_00176_b200.report [--configs 1,2,3,4,5] [--reps 30] [--oracle-budget 10]
+    python report.py [--configs 1,2,3,4,5] [--reps 30]
 """
 from __future__ import annotations
 
@@ -11,12 +12,51 @@ import json
 import os
 import sys
 import time
+from typing import Dict, List
 
 import numpy as np
 
-ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
+
+
+def group_times(prep, reps: int = 5) -> List[float]:
+    """Median device time (ms) of every fused group over `reps` timed inferences."""
+    ins = [t.data_ptr() for t in prep.in_dev]
+    outs = [t.data_ptr() for t in prep.out_dev]
+    runs = [prep.plan.run_timed(ins, outs, prep.arena.data_ptr(), prep.arena.numel(), prep.s.stream) for _ in range(reps)]
+    return [float(np.median([r[g] for r in runs])) for g in range(len(runs[0]))]
+
+
+def group_report(prep, hbm_gbs: float, tensor_tflops: float, reps: int = 5) -> List[Dict]:
+    """Per group: kind, ms, algorithmic flops / bytes, roofline time and fraction."""
+    g = prep.s.graph
+    ms = group_times(prep, reps)
+    out = []
+    for gi in range(g.num_groups()):
+        info = g.group_info(gi)
+        flops, nbytes = prep.plan.group_cost(gi)
+        t_hbm = nbytes / (hbm_gbs * 1e9) * 1e3
+        t_tc = flops / (tensor_tflops * 1e12) * 1e3
+        t_roof = max(t_hbm, t_tc)
+        out.append({"group": gi, "kind": info["kind"], "n_ops": info["n_ops"], "ms": ms[gi], "flops": flops, "bytes": nbytes,
+                    "bound": "tensor" if t_tc >= t_hbm else "hbm", "t_roof_ms": t_roof, "frac": t_roof / ms[gi] if ms[gi] > 0 else 0.0})
+    return out
+
+
+def kind_summary(report: List[Dict]) -> Dict[str, Dict]:
+    agg: Dict[str, Dict] = {}
+    for r in report:
+        a = agg.setdefault(r["kind"], {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "t_roof_ms": 0.0, "launch_groups": 0})
+        for k in ("ms", "flops", "bytes", "t_roof_ms"):
+            a[k] += r[k]
+        a["launch_groups"] += 1
+    for a in agg.values():
+        a["tflops"] = a["flops"] / (a["ms"] * 1e-3) / 1e12 if a["ms"] > 0 else 0.0
+        a["gbs"] = a["bytes"] / (a["ms"] * 1e-3) / 1e9 if a["ms"] > 0 else 0.0
+        a["frac"] = a["t_roof_ms"] / a["ms"] if a["ms"] > 0 else 0.0
+    return agg
 
 
 def _peaks():
@@ -39,16 +79,14 @@ def _units(cfg, reqs):
     return reqs[0].inputs["x"].shape[0], "images"
 
 
-def measure(cfg: int, reps: int, oracle_budget: float):
+def measure(cfg: int, reps: int, device: str = "cuda:0"):
     import torch
-    from oracle import interp as O
-    from paper_2403_00176_b200 import profile as PF
     from paper_2403_00176_b200 import workloads as WL
     from paper_2403_00176_b200.session import Session
 
     hbm, tf, src = _peaks()
     wl = {1: WL.cfg1, 2: WL.cfg2, 3: WL.cfg3, 4: WL.cfg4, 5: WL.cfg5}[cfg]()
-    sess = Session(wl)
+    sess = Session(wl, device=device)
     n_batches = 3 if cfg in (4, 5) else 5
     preps = [sess.prepare(wl.batch(j)) for j in range(n_batches)]
     dev = sess.dev
@@ -108,8 +146,8 @@ def measure(cfg: int, reps: int, oracle_budget: float):
         empty_ms = timed(lambda: B.sod2_launch_empty(sess.stream), 50)
         extra = {"ms_one_request_per_inference": single_ms, "ms_empty_kernel": empty_ms, "ratio_to_empty_kernel": single_ms / empty_ms}
     # per-group roofline on the first batch
-    rep = PF.group_report(preps[0], hbm, tf, reps=5)
-    kinds = PF.kind_summary(rep)
+    rep = group_report(preps[0], hbm, tf, reps=5)
+    kinds = kind_summary(rep)
     sum_ms = sum(r["ms"] for r in rep)
     sum_roof = sum(r["t_roof_ms"] for r in rep)
     # worst group among those that matter (at least 1 % of the time of all groups)
@@ -133,41 +171,42 @@ def measure(cfg: int, reps: int, oracle_budget: float):
         if hit:
             hit_us.append((time.perf_counter() - t0) * 1e6)
     sess.graph.set_plan_cache(0)
+    # end to end through the public API with host buffers: H2D (pinned) + bind + plan + run + D2H (pinned)
+    pin_in = [[torch.from_numpy(h).pin_memory() for h in p.in_host] for p in preps]
+    pin_out = [[torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in p.out_dev] for p in preps]
+    e2e = []
+    for i in range(2 * len(preps) + 1):
+        k = i % len(preps)
+        pr = preps[k]
+        torch.cuda.synchronize(dev)
+        t0 = time.perf_counter()
+        for dst, src_ in zip(pr.in_dev, pin_in[k]):
+            dst.copy_(src_, non_blocking=True)
+        b = sess.graph.bind_dims(wl.sym_names, [[r.syms[s] for s in wl.sym_names] for r in pr.reqs])
+        pl = b.plan()
+        pl.run([t.data_ptr() for t in pr.in_dev], [t.data_ptr() for t in pr.out_dev], pr.arena.data_ptr(), pr.arena.numel(), sess.stream)
+        for dst, src_ in zip(pin_out[k], pr.out_dev):
+            dst.copy_(src_, non_blocking=True)
+        torch.cuda.synchronize(dev)
+        if i > 0:
+            e2e.append((time.perf_counter() - t0) * 1e3)
+        del pl, b
     mem = preps[0].plan.memory()
-    # oracle on a bounded sample
-    t0 = time.perf_counter()
-    done = 0
     reqs0 = preps[0].reqs
-    if cfg == 5:
-        small = WL.cfg5(B=2)
-        O.run(small.ir, small.consts, small.batch(0)[0].inputs)
-        dt = time.perf_counter() - t0
-        oracle_ms = dt * 1e3 * (32 / 2)
-        sample = "2 of 32 images, scaled by images"
-    else:
-        order = sorted(range(len(reqs0)), key=lambda i: _units(cfg, [reqs0[i]])[0])
-        for i in order:
-            O.run(wl.ir, wl.consts, reqs0[i].inputs)
-            done += _units(cfg, [reqs0[i]])[0]
-            if time.perf_counter() - t0 > oracle_budget:
-                break
-        dt = time.perf_counter() - t0
-        total = _units(cfg, reqs0)[0]
-        oracle_ms = dt * 1e3 * total / done
-        sample = f"{done} of {total} {_units(cfg, reqs0)[1]} of batch 0, scaled"
     units, uname = _units(cfg, reqs0)
     n_req = len(reqs0) if cfg != 5 else reqs0[0].inputs["x"].shape[0]
     return {
         "cfg": cfg, "workload": wl.name, "ms_median": float(np.median(times)), "ms_min": float(np.min(times)),
         "ms_graph_median": float(np.median(gtimes)), "ms_graph_min": float(np.min(gtimes)),
+        "e2e_ms": float(np.median(e2e)), "h2d_bytes": int(sum(t.numel() for t in pin_in[0])), "d2h_bytes": int(sum(t.numel() for t in pin_out[0])),
         "ms_per_request": float(np.median(times)) / n_req, "units_batch0": units, "unit": uname,
         "sum_t_roof_over_sum_t_groups": sum_roof / sum_ms, "sum_t_roof_over_t_step": sum_roof / float(np.median(times)),
         "worst_group": {"kind": worst["kind"], "frac": worst["frac"], "bound": worst["bound"], "ms": worst["ms"]},
         "kinds": {k: {"ms": round(v["ms"], 4), "frac": round(v["frac"], 3), "tflops": round(v["tflops"], 1), "gbs": round(v["gbs"], 1)} for k, v in kinds.items()},
         "plan_us_median": float(np.median(plan_us)), "plan_us_cache_hit": float(np.median(hit_us)) if hit_us else None, "arena_bytes": mem["arena_bytes"], "peak_live_bytes": mem["peak_live_bytes"],
         "sum_tensor_bytes": mem["sum_bytes"], "n_groups": sess.graph.num_groups(), "n_ops": sess.graph.num_ops(),
-        "gpu_launches": preps[0].plan.run_timed and None,
-        "oracle_ms": oracle_ms, "oracle_cores": os.cpu_count(), "oracle_sample": sample, "peaks": src,
+        "gpu_launches": int(preps[0].run().gpu_launches), "peaks": src,
+        "group_times": "CUDA events around every launch (no overlap between dependent kernels, no graph): the groups sum to more than ms_median",
         **extra,
     }
 
@@ -176,20 +215,18 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="1,2,3,4,5")
     ap.add_argument("--reps", type=int, default=30)
-    ap.add_argument("--oracle-budget", type=float, default=10.0)
     a = ap.parse_args()
     rows = []
     for c in [int(x) for x in a.configs.split(",")]:
-        r = measure(c, a.reps, a.oracle_budget)
-        r.pop("gpu_launches", None)
+        r = measure(c, a.reps)
         print(json.dumps(r), flush=True)
         rows.append(r)
-    print("\n| cfg | ms per inference (median, min) | as one CUDA graph (median, min) | ms per request | sum t_roof / t_step | worst group: fraction, bound | bind+plan us (cache hit) | arena / peak-live MB | oracle ms (cores) |")
-    print("|---|---|---|---|---|---|---|---|---|")
+    print("\n| cfg | ms per inference (median, min) | as one CUDA graph (median, min) | ms per request | sum t_roof / t_step | worst group: fraction, bound | bind+plan us (cache hit) | arena / peak-live MB |")
+    print("|---|---|---|---|---|---|---|---|")
     for r in rows:
         print(f"| {r['cfg']} | {r['ms_median']:.3f}, {r['ms_min']:.3f} | {r['ms_graph_median']:.3f}, {r['ms_graph_min']:.3f} | {r['ms_per_request']:.4f} | {r['sum_t_roof_over_t_step']:.3f} | "
               f"{r['worst_group']['kind']}: {r['worst_group']['frac']:.3f}, {r['worst_group']['bound']} | {r['plan_us_median']:.0f} ({r['plan_us_cache_hit'] or 0:.0f}) | "
-              f"{r['arena_bytes'] / 1e6:.1f} / {r['peak_live_bytes'] / 1e6:.1f} | {r['oracle_ms']:.0f} ({r['oracle_cores']}) |")
+              f"{r['arena_bytes'] / 1e6:.1f} / {r['peak_live_bytes'] / 1e6:.1f} |")
     for r in rows:
         if "ratio_to_empty_kernel" in r:
             print(f"\ncfg {r['cfg']} is launch-bound: one request per inference {r['ms_one_request_per_inference'] * 1e3:.2f} us, "

@@ -5,14 +5,14 @@ Calls only the oracle and the workload generator.  For block i the target skip f
 q_i ~ U(0.4, 0.7) (seeded); with the logits z sorted ascending and m = round(q_i * B), the bias is
 b_i = -(z_(m) + z_(m+1)) / 2 so that exactly m samples have z + b_i <= 0.  Decisions of earlier
 blocks change the features of later ones, so the pass is repeated a few times from the previous
-biases until the skip counts settle.  Usage:  python -m oracle.calibrate_cfg5_gates [passes]
+biases until the skip counts settle.  Usage:  python tests/golden/calibrate_cfg5_gates.py [passes]
 """
 import os
 import sys
 
 import numpy as np
 
-ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+ROOT = os.path.dirname(os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
 sys.path.insert(0, ROOT)
 
 from oracle import interp as O  # noqa: E402
@@ -54,7 +54,7 @@ def main(passes: int = 3):
         if all(ok):
             break
     with open(OUT, "w") as f:
-        f.write("# gate bias per block of the default gated skip network (written by oracle/calibrate_cfg5_gates.py)\n")
+        f.write("# gate bias per block of the default gated skip network (written by tests/golden/calibrate_cfg5_gates.py)\n")
         for b in bias:
             f.write(f"{float(bf16_round(np.array([b], np.float32))[0])!r}\n")
     print("wrote", OUT)

@@ -232,3 +232,151 @@ def test_rel_err_metric():
     a = np.array([1.0, -2.0, 0.0])
     assert O.rel_err(a, a) == 0
     assert O.rel_err(np.array([]), np.array([])) == 0
+
+
+# --------------------------------------------------------------------------- pins through tiny graphs
+# Each test below writes a few lines of graph text, runs the interpreter and compares with literal
+# arrays or explicit loops, so that every operator branch of the interpreter meets something that is
+# not the interpreter (a wrong axis, sign, comparison direction or off-by-one fails here).
+def _run(ir, inputs=None, consts=None):
+    return O.run(ir, consts or {}, inputs or {})
+
+
+def test_global_average_pool_vs_loops_non_square():
+    x = rng.standard_normal((2, 3, 4, 7))          # H != W, N != C: a wrong axis pair changes shape or values
+    env = _run("input x f32 [2,3,4,7]\nnode GlobalAveragePool x -> p\noutput p\n", {"x": x})
+    assert env["p"].shape == (2, 3, 1, 1)
+    for n in range(2):
+        for c in range(3):
+            s = 0.0
+            for h in range(4):
+                for w in range(7):
+                    s += x[n, c, h, w]
+            assert abs(env["p"][n, c, 0, 0] - s / 28.0) < 1e-14
+
+
+def test_greater_is_strict_and_directed():
+    a = np.array([[-1.0], [0.0], [0.5], [2.0]])
+    env = _run("input a f32 [4,1]\nfconst z f32 [] = 0.0\nfconst one f32 [] = 1.0\n"
+               "node Greater a z -> g0\nnode Greater z a -> g1\nnode Greater a one -> g2\n", {"a": a})
+    assert env["g0"].reshape(-1).tolist() == [False, False, True, True]      # 0 > 0 is false
+    assert env["g1"].reshape(-1).tolist() == [True, False, False, False]     # operands are not swapped
+    assert env["g2"].reshape(-1).tolist() == [False, False, False, True]
+
+
+def test_gate_chain_of_gated_block_vs_loops_with_exact_zero_logit():
+    # the gate of a block: z_b = sum_c w_c * mean_hw x[b,c] + b0, gate_b = z_b > 0 (true = execute);
+    # sample 1 is built so that z is exactly 0 and must be skipped
+    wl = WL.cfg5(B=4, side=16, widths=(4, 8), per_stage=2, calibrated=False)
+    g = O.parse(wl.ir)
+    x = np.zeros((4, 4, 8, 8))
+    x[0] = rng.integers(-4, 5, size=(4, 8, 8)) / 4.0
+    x[1] = 0.0                                     # pooled features 0 -> z = bias
+    x[2] = rng.integers(-4, 5, size=(4, 8, 8)) / 4.0 + 1.0
+    x[3] = -x[2]
+    gw = np.array([[0.5], [-1.0], [2.0], [0.25]])
+    consts = dict(wl.consts)
+    consts["b0.gw"] = gw
+    consts["b0.gb"] = np.array([0.0])              # exact zero logit for sample 1
+    env = O.run(wl.ir, consts, wl.batch(0)[0].inputs, overrides={"stem": x}, g=g)
+    z = []
+    for b in range(4):
+        acc = 0.0
+        for c in range(4):
+            m = 0.0
+            for h in range(8):
+                for w in range(8):
+                    m += x[b, c, h, w]
+            acc += gw[c, 0] * (m / 64.0)
+        z.append(acc + 0.0)
+    assert z[1] == 0.0
+    want = [bool(v > 0) for v in z]
+    assert want[1] is False and any(want) and not all(want)
+    assert env["gate0"].reshape(-1).astype(bool).tolist() == want
+    assert np.allclose(env["logit0"].reshape(-1), z, atol=1e-14)
+    # and the block output follows the decision sample by sample: skipped samples pass through unchanged
+    for b in range(4):
+        if not want[b]:
+            assert np.array_equal(env["blk0"][b], x[b])
+        else:
+            assert not np.array_equal(env["blk0"][b], x[b])
+
+
+def test_range_constant_of_shape_cast_literals():
+    env = _run("iconst s i64 [] = 2\niconst e i64 [] = 11\niconst d i64 [] = 3\niconst dn i64 [] = -4\niconst shp i64 [2] = 2 3\n"
+               "input f f32 [4]\n"
+               "node Range s e d -> r\nnode Range e s dn -> rn\nnode ConstantOfShape shp -> c {value=1.5}\n"
+               "node Cast f -> fi {to=i64}\nnode Cast r -> rf {to=f32}\n",
+               {"f": np.array([1.9, -1.9, 0.0, 7.2])})
+    assert env["r"].tolist() == [2, 5, 8] and env["r"].dtype == np.int64           # end is exclusive
+    assert env["rn"].tolist() == [11, 7, 3]                                        # negative step counts down
+    assert env["c"].shape == (2, 3) and np.all(env["c"] == 1.5)
+    assert env["fi"].tolist() == [1, -1, 0, 7] and env["fi"].dtype == np.int64     # truncation toward zero
+    assert env["rf"].dtype == np.float64 and env["rf"].tolist() == [2.0, 5.0, 8.0]
+
+
+def test_float_div_sub_and_integer_div_literals():
+    a = np.array([[6.0, -3.0], [1.0, 0.5]])
+    b = np.array([4.0, 2.0])                      # broadcast over rows
+    env = _run("input a f32 [2,2]\ninput b f32 [2]\niconst i i64 [3] = 7 -7 9\niconst j i64 [] = 2\n"
+               "node Div a b -> q\nnode Sub a b -> d\nnode Sub b a -> e\nnode Div i j -> iq\nnode Mul a b -> m\nnode Add a b -> s\n",
+               {"a": a, "b": b})
+    assert env["q"].tolist() == [[1.5, -1.5], [0.25, 0.25]]
+    assert env["d"].tolist() == [[2.0, -5.0], [-3.0, -1.5]]
+    assert env["e"].tolist() == [[-2.0, 5.0], [3.0, 1.5]]                          # Sub is not commutative: operand order
+    assert env["iq"].tolist() == [3, -4, 4] and env["iq"].dtype == np.int64        # integer Div floors
+    assert env["m"].tolist() == [[24.0, -6.0], [4.0, 1.0]]
+    assert env["s"].tolist() == [[10.0, -1.0], [5.0, 2.5]]
+
+
+def test_reshape_zero_and_minus_one_rules():
+    x = np.arange(24.0).reshape(2, 3, 4)
+    env = _run("input x f32 [2,3,4]\niconst a i64 [3] = 0 -1 2\niconst b i64 [2] = -1 0\niconst c i64 [3] = 0 0 4\n"
+               "node Reshape x a -> ra\nnode Reshape x b -> rb\nnode Reshape x c -> rc\n", {"x": x})
+    assert env["ra"].shape == (2, 6, 2)            # 0 copies input dim 0, -1 takes the rest
+    assert env["rb"].shape == (8, 3)               # 0 at position 1 copies input dim 1 (= 3)
+    assert env["rc"].shape == (2, 3, 4)
+    assert env["ra"].reshape(-1).tolist() == list(range(24))     # row-major order is kept
+    assert env["ra"][1, 2, 1] == 17.0 and env["rb"][5, 1] == 16.0
+
+
+def test_reduce_sum_square_relu_shape_transpose_concat_gather_slice_literals():
+    x = np.array([[1.0, -2.0, 3.0], [0.5, 0.0, -1.0]])
+    env = _run("input x f32 [2,3]\niconst ix i64 [2] = 2 0\niconst i0 i64 [1] = 1\n"
+               "iconst st i64 [1] = 1\niconst en i64 [1] = 3\niconst ax i64 [1] = 1\n"
+               "node ReduceSumSquare x -> q {axis=-1 keepdims=0}\nnode ReduceSumSquare x -> qk {axis=-1 keepdims=1}\n"
+               "node Relu x -> r\nnode Shape x -> s\nnode Transpose x -> t {perm=1,0}\nnode Concat x x -> c {axis=0}\n"
+               "node Concat x x -> c1 {axis=1}\nnode Gather x ix -> g {axis=1}\nnode Gather x i0 -> g0 {axis=0}\n"
+               "node Slice x st en ax -> sl\n",
+               {"x": x})
+    assert env["q"].tolist() == [14.0, 1.25] and env["qk"].shape == (2, 1)         # squares, no square root
+    assert env["r"].tolist() == [[1.0, 0.0, 3.0], [0.5, 0.0, 0.0]]
+    assert env["s"].tolist() == [2, 3]
+    assert env["t"].tolist() == [[1.0, 0.5], [-2.0, 0.0], [3.0, -1.0]]
+    assert env["c"].shape == (4, 3) and env["c1"].shape == (2, 6) and env["c1"][1].tolist() == [0.5, 0.0, -1.0, 0.5, 0.0, -1.0]
+    assert env["g"].tolist() == [[3.0, 1.0], [-1.0, 0.5]]                          # columns 2 and 0, in that order
+    assert env["g0"].tolist() == [[0.5, 0.0, -1.0]]
+    assert env["sl"].tolist() == [[-2.0, 3.0], [0.0, -1.0]]                        # columns 1..2
+
+
+def test_sigmoid_values_and_softmax_axis():
+    v = O.op_sigmoid(np.array([1.0, -2.0]))
+    assert abs(v[0] - 1.0 / (1.0 + math.exp(-1.0))) < 1e-16 and abs(v[1] - 1.0 / (1.0 + math.exp(2.0))) < 1e-16
+    x = rng.standard_normal((3, 4))
+    env = _run("input x f32 [3,4]\nnode Softmax x -> p {axis=-1}\nnode Softmax x -> p0 {axis=0}\n", {"x": x})
+    for i in range(3):
+        den = sum(math.exp(x[i, j]) for j in range(4))
+        for j in range(4):
+            assert abs(env["p"][i, j] - math.exp(x[i, j]) / den) < 1e-14
+    assert np.allclose(env["p0"].sum(0), 1.0, atol=1e-14) and not np.allclose(env["p0"].sum(1), 1.0)
+
+
+def test_layernorm_values_vs_loops():
+    x = rng.standard_normal((2, 5)) * 2 + 0.7
+    g, b = rng.standard_normal(5), rng.standard_normal(5)
+    y = O.op_layernorm(x, g, b, -1, 1e-3)
+    for i in range(2):
+        mu = sum(x[i]) / 5
+        var = sum((v - mu) ** 2 for v in x[i]) / 5
+        for j in range(5):
+            assert abs(y[i, j] - ((x[i, j] - mu) / math.sqrt(var + 1e-3) * g[j] + b[j])) < 1e-13

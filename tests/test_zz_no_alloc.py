@@ -54,3 +54,8 @@ def test_static_scratch_nonzero_edges_and_limit():
     with pytest.raises(B.Sod2Error) as e:     # rejected on the host, before any launch
         B.sod2_nonzero_static(buf.data_ptr(), 0, [B.NONZERO_STATIC_MAX_ELEMS + 1], buf.data_ptr(), buf.data_ptr(), 0)
     assert e.value.status_name == "SOD2_E_BAD_DIM" and "limit" in str(e.value)
+    # extents whose product wraps around the 64-bit range must be rejected, not taken for a small or empty input
+    for dims in ([1 << 24, 1 << 40], [2, 1 << 62, 4], [1 << 32, 1 << 32], [0, 1 << 40]):
+        with pytest.raises(B.Sod2Error) as e:
+            B.sod2_nonzero_static(buf.data_ptr(), 0, dims, buf.data_ptr(), buf.data_ptr(), 0)
+        assert e.value.status_name == "SOD2_E_BAD_DIM", dims
