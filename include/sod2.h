@@ -46,6 +46,8 @@ typedef enum {
 #define SOD2_OPT_LEGACY_ATTENTION 8u /* attention groups run the mma.sync kernel even where the tcgen05 kernel applies */
 #define SOD2_OPT_MULTI_VERSION 64u /* fuse elementwise chains across broadcasts RDP cannot resolve: 2^d fused versions (Section 4.2), the version (a stride table) chosen at bind time */
 #define SOD2_OPT_NO_SEP 32u /* groups run in their default topological order: no static execution planning (Section 4.3) */
+#define SOD2_OPT_LN_FOLD 128u /* a LayerNorm between bf16 GEMMs is folded into its neighbours (Section 4.2: fusion removes the materialised intermediate): the producing GEMM writes per-row statistics, the consuming GEMMs read the raw rows and normalise in their epilogues, the normalised tensor is never stored.  Opt-in: measured slower on the encoder workloads, where the LayerNorm kernel runs beside the next GEMM's pipeline fill */
+#define SOD2_OPT_GEMM_CHAIN 256u /* consecutive GEMM groups that depend on each other row block by row block run as one persistent kernel with per-row-block dependency counters in the arena header (their operands stay live over the whole chain).  Opt-in: measured slower than one launch per GEMM at a few thousand rows */
 #define SOD2_OPT_SPLITK_LN 4u /* bf16 GEMM (+bias, +residual) -> LayerNorm as one group: split-K GEMM into fp32 slabs + finishing kernel */
 
 /* Parse the graph text (host, ir_len bytes), classify every operator (Table 2), run RDP
@@ -123,7 +125,8 @@ sod2_status sod2_run_graph(sod2_plan_t* p, const void* const* inputs, void* cons
 
 /* Measurement aid: the same inference with CUDA events recorded on cuda_stream around every launch.
  * Synchronises the stream and returns the device time of each fused group in group_ms[n_groups]
- * (host array, milliseconds; n_groups must equal sod2_graph_num_groups). */
+ * (host array, milliseconds; n_groups must equal sod2_graph_num_groups).  A launch that runs several
+ * groups (a chain of GEMMs) is divided among them in proportion to their algorithmic flops. */
 sod2_status sod2_run_timed(sod2_plan_t* p, const void* const* inputs, void* const* outputs, void* arena,
                            size_t arena_bytes, void* cuda_stream, float* group_ms, int n_groups);
 

@@ -23,6 +23,8 @@ OPT_LEGACY_ATTENTION = 8
 OPT_COPY_REGROUP = 16
 OPT_NO_SEP = 32
 OPT_MULTI_VERSION = 64
+OPT_LN_FOLD = 128
+OPT_GEMM_CHAIN = 256
 DYN_CLASS = ["ISDO", "ISDOS", "ISVDOS", "EDO"]
 
 

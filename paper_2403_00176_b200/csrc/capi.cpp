@@ -92,7 +92,7 @@ sod2_status sod2_graph_reanalyse(sod2_graph* g, const int* order, int n) {
   Status s = rdp_analysis(&G, &ord);
   if (s != OK) { g->h.err = G.err; return st(s); }
   g->c.groups.clear();
-  g->c.packed_consts.clear(); g->c.packed_off.clear(); g->c.packed_bytes = 0;
+  g->c.packed_consts.clear(); g->c.packed_off.clear(); g->c.packed_ln.clear(); g->c.packed_bytes = 0;
   for (auto& nd : G.nodes) nd.group = -1;
   s = form_groups(&g->c);
   if (s != OK) g->h.err = g->c.err;

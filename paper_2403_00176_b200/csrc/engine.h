@@ -19,6 +19,8 @@ enum OptFlags : uint32_t {
   OPT_MULTI_VERSION = 64u,    // fuse elementwise chains across unresolved broadcasts: 2^d versions, chosen at bind time
   OPT_NO_SEP = 32u,     // groups run in their default topological order (no static execution planning)
   OPT_SPLITK_LN = 4u,   // a bf16 GEMM (+bias, +residual) followed by LayerNorm becomes one group: split-K GEMM + finishing kernel
+  OPT_LN_FOLD = 128u,     // a LayerNorm between bf16 GEMMs is folded into their epilogues (the normalised tensor is never stored)
+  OPT_GEMM_CHAIN = 256u,  // consecutive dependent GEMM groups run as one persistent kernel with row-block dependency counters
 };
 
 enum class GKind {
@@ -53,6 +55,13 @@ struct Group {
   int red = 0;                        // chain: 0 none, 1 softmax, 2 layernorm
   float eps = 1e-5f, scale = 1.0f;
   int stride = 1, pad = 0, ksize = 1;
+  // LayerNorm folded into the neighbouring GEMMs (fuse.cpp, step 3c): the normalised tensor is never stored.
+  //   ln_a >= 0:   the A operand is LayerNorm(ln_a): the kernel multiplies the raw rows by gamma-scaled weights and
+  //                its epilogue applies the rows' mean / rstd and two precomputed vectors
+  //   ln_res >= 0: the residual operand is LayerNorm(ln_res): the epilogue normalises the staged raw tile
+  //   emit_stats:  the epilogue also writes per-row partial statistics of the output (beside the output's storage)
+  int ln_a = -1, ln_res = -1, ln_gamma = -1, ln_beta = -1, emit_stats = 0;
+  float ln_eps = 1e-5f;
   std::vector<int> chain_ops;         // ChainOp codes
   std::vector<int> chain_operands;    // tensor id or -1 per op
   std::string why;                    // for UNSUPPORTED
@@ -99,6 +108,13 @@ struct Compiled {
   std::vector<ViewParam> view_param;
   std::vector<int> packed_consts;     // tensor ids
   std::vector<size_t> packed_off;     // byte offsets in the prepack workspace
+  // entry i with packed_ln[i].gamma >= 0 is the weight of a GEMM whose A operand is a folded LayerNorm:
+  // [N,K] bf16 copy of gamma[k] * W[k,n], then fp32 c1[N] = column sums of that copy, then fp32
+  // c2[N] = sum_k beta[k] * W[k,n] + bias[n]
+  struct PackedLn { int gamma = -1, beta = -1, bias = -1; };
+  std::vector<PackedLn> packed_ln;
+  // per tensor: > 0 = row width of a tensor whose producer writes LayerNorm row statistics beside it
+  std::vector<int> stats_width;
   size_t packed_bytes = 0;
   void* packed_ws = nullptr;
   std::string err;
@@ -212,6 +228,10 @@ struct RootBuf {              // packed storage of a root tensor: the requests' 
   int64_t bytes = 0;
   size_t arena_off = 0;
   int def_step = -1, last_step = -1;
+  // LayerNorm row statistics written by the producing GEMM (folded LayerNorm): `stats_slots` planes of
+  // `stats_rows` (mean, M2) float pairs at byte `stats_off` of this root's storage, one pair per packed row
+  int64_t stats_off = -1, stats_rows = 0;
+  int stats_slots = 0;
 };
 
 struct Ptr {                  // address resolved at run time
@@ -238,6 +258,18 @@ struct Plan {
   bool sm_count_known = false;
   bool uses_header = true;                // false: no kernel of the plan writes the status word, a ticket or a count: nothing to clear or read
   std::vector<double> group_flops, group_bytes;   // algorithmic cost per group for the bound shapes
+  // per tensor with row statistics: slots the producer's tile version really writes and columns per slot
+  struct StatsLayout { int slots = 0, cols = 0; };
+  std::vector<StatsLayout> stats_layout;
+  // Runs of consecutive GEMM groups that execute as one persistent kernel (gemm_chain_tcgen05.cuh): decided after
+  // view resolution and before liveness, because the members run concurrently: everything a member reads stays
+  // live, and everything a member writes is live, over the whole run.
+  struct Chain { std::vector<int> groups; int rows = 0; size_t counter_word = 0; };
+  std::vector<Chain> chains;
+  std::vector<int> chain_of;              // [group] index into chains, -1 = a launch of its own
+  size_t chain_counter_off = 0;           // byte offset in the arena header of the chains' row-block counters
+  size_t chain_counter_words = 0;
+  size_t header_clear_bytes = 256;        // what a run zeroes at the start of the arena (status word, tickets, chain counters)
   std::string err;
   // device status word lives at arena offset 0 (first 256 bytes reserved)
   // CUDA graph of the whole launch sequence for one set of buffers (run_plan_graph)
@@ -262,6 +294,7 @@ Status make_plan(const Compiled* c, const Binding* b, Plan* p);
 Status run_plan_graph(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream,
                       int64_t* info);
 Status build_launches(Plan* p);   // exec.cu
+Status detect_chains(Plan* p);    // exec.cu: fills Plan::chains / chain_of from the resolved views
 Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream,
                 int64_t* info);
 

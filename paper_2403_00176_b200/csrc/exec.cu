@@ -15,6 +15,7 @@
 #include "conv_stem_tcgen05.cuh"
 #include "engine.h"
 #include "gemm_tcgen05.cuh"
+#include "gemm_chain_tcgen05.cuh"
 #include "kernels_compact.cuh"
 #include "kernels_rows.cuh"
 #include "tmap.h"
@@ -44,6 +45,8 @@ struct Launch {
   int group = -1;
   int n_kernels = 1;
   std::function<cudaError_t(const RunCtx&)> fn;
+  // a launch that runs several groups (a GEMM chain): (group, share of the launch's time by algorithmic flops)
+  std::vector<std::pair<int, double>> share;
 };
 
 namespace {
@@ -76,6 +79,56 @@ bool is_fused_stem(const Compiled& c, const Group& G) {
   for (int i = 0; i < 4; ++i) if (!W.S.dims[i].known() || !W.S.dims[i].e.is_const()) return false;
   return W.S.dims[0].e.const_value() == 64 && W.S.dims[1].e.const_value() == 3 && W.S.dims[2].e.const_value() == 7 &&
          W.S.dims[3].e.const_value() == 7 && G.stride == 2 && G.pad == 3;
+}
+
+// One instantiation of the tcgen05 GEMM: sets its shared-memory limit once and launches it with programmatic
+// dependent launch.
+template <int BN, int KCH, int ST, int ACT, bool RES, int LN, bool EMIT>
+cudaError_t launch_gemm_variant(dim3 grid, cudaStream_t st, const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to,
+                                const CUtensorMap& tr, int M, int N, int K, const k::GemmEpilogue& ep) {
+  constexpr int smem = k::GemmSmem<BN, KCH, ST>::TOTAL;
+  static bool once = (cudaFuncSetAttribute(k::gemm_bf16_tcgen05<BN, KCH, ST, ACT, false, RES, LN, EMIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);
+  (void)once;
+  return launch_pdl(k::gemm_bf16_tcgen05<BN, KCH, ST, ACT, false, RES, LN, EMIT>, grid, dim3(k::GEMM_THREADS), smem, st, ta, tb, to, tr, M, N, K, ep);
+}
+// Epilogue versions of one tile version: plain (activation x residual), normalised A operand (LN = 1, any
+// activation), normalised residual (LN = 2, tiles up to 128 wide), each of the residual forms with or without
+// row statistics of the output (EMIT).
+template <int BN, int KCH, int ST>
+cudaError_t gemm_dispatch(int act, bool res, int ln, bool emit, dim3 grid, cudaStream_t st, const CUtensorMap& ta, const CUtensorMap& tb,
+                          const CUtensorMap& to, const CUtensorMap& tr, int M, int N, int K, const k::GemmEpilogue& ep) {
+#define SOD2_GV(ACT_, RES_, LN_, EMIT_) return launch_gemm_variant<BN, KCH, ST, ACT_, RES_, LN_, EMIT_>(grid, st, ta, tb, to, tr, M, N, K, ep)
+  if (ln == 0 && !emit) {
+    switch (act * 2 + (res ? 1 : 0)) {
+      case 0: SOD2_GV(0, false, 0, false);
+      case 1: SOD2_GV(0, true, 0, false);
+      case 2: SOD2_GV(1, false, 0, false);
+      case 3: SOD2_GV(1, true, 0, false);
+      case 4: SOD2_GV(2, false, 0, false);
+      default: SOD2_GV(2, true, 0, false);
+    }
+  }
+  if (ln == 1 && !res && !emit) {
+    switch (act) {
+      case 0: SOD2_GV(0, false, 1, false);
+      case 1: SOD2_GV(1, false, 1, false);
+      default: SOD2_GV(2, false, 1, false);
+    }
+  }
+  if (act != 0) return cudaErrorInvalidValue;
+  if (ln == 2 && res) {
+    if constexpr (BN <= 128) {
+      if (emit) SOD2_GV(0, true, 2, true);
+      SOD2_GV(0, true, 2, false);
+    }
+    return cudaErrorInvalidValue;
+  }
+  if (ln == 0 && emit) {
+    if (res) SOD2_GV(0, true, 0, true);
+    SOD2_GV(0, false, 0, true);
+  }
+#undef SOD2_GV
+  return cudaErrorInvalidValue;
 }
 
 struct Builder {
@@ -206,8 +259,15 @@ struct Builder {
     // bf16 on tcgen05
     if (K % 64) return fail(E_UNSUPPORTED_OP, "bf16 GEMM needs K % 64 == 0 (k-chunk tensor maps)");
     if (lds[0] % 8 || lds[1] % 8 || N % 8 || (G.res >= 0 && lds[2] % 8)) return fail(E_UNSUPPORTED_OP, "GEMM operand rows must be 16-byte multiples");
+    const bool lna = G.ln_a >= 0, lnr = G.ln_res >= 0, emit = G.emit_stats != 0;
     size_t pk = 0;
-    for (size_t i = 0; i < c.packed_consts.size(); ++i) if (c.packed_consts[i] == G.w) pk = c.packed_off[i];
+    bool pk_found = false;
+    for (size_t i = 0; i < c.packed_consts.size(); ++i)
+      if (c.packed_consts[i] == G.w) {
+        const Compiled::PackedLn& e = c.packed_ln[i];
+        if (lna ? (e.gamma == G.ln_gamma && e.beta == G.ln_beta && e.bias == G.bias) : e.gamma < 0) { pk = c.packed_off[i]; pk_found = true; }
+      }
+    if (!pk_found) return fail(E_INTERNAL, "no prepacked copy of " + W.name);
     if (G.has_ln) {
       // ---- GEMM (+bias, +residual) -> LayerNorm: K ranges of every 128x256 tile go to different CTAs,
       // which store their fp32 partial tiles into slabs of a workspace in the scratch region; the finishing
@@ -272,6 +332,22 @@ struct Builder {
       }
       return OK;
     }
+    // folded LayerNorm: where the statistics of the normalised rows live, and where this group's own go
+    if ((lna || lnr) && (lds[lna ? 0 : 2] != (lna ? K : N))) return fail(E_UNSUPPORTED_OP, "folded LayerNorm needs densely packed rows");
+    if (emit && lds[1] != N) return fail(E_UNSUPPORTED_OP, "row statistics need densely packed output rows");
+    if (p.stats_layout.size() != g.tensors.size()) p.stats_layout.assign(g.tensors.size(), Plan::StatsLayout());
+    auto stats_ptr = [&](int t, int r0, int64_t width, Ptr* out, int64_t* pitch) -> bool {
+      const int root = p.views[t][r0].root;
+      const RootBuf& RR = p.roots[root];
+      if (RR.where != RootBuf::ARENA || RR.stats_off < 0 || p.views[t][r0].offset != 0) return false;
+      const int64_t row0 = p.inst_off[root][r0] / (width * 2);
+      out->where = RootBuf::ARENA;
+      out->index = -1;
+      out->off = static_cast<int64_t>(RR.arena_off) + RR.stats_off + row0 * 8;
+      *pitch = RR.stats_rows;
+      return true;
+    };
+    int bn_group = 0;   // a group that writes row statistics uses one tile width for all its launches
     for (auto& sg : segs) {
       if (sg.rows == 0) continue;
       Ptr pa = ptr_of(G.a, sg.r0), po = ptr_of(G.out, sg.r0), pr = G.res >= 0 ? ptr_of(G.res, sg.r0) : Ptr();
@@ -297,9 +373,33 @@ struct Builder {
       // Small problems: while 128x64 tiles still fit one wave, a CTA's time is pipeline fill + main loop +
       // epilogue of ONE tile, and both of the latter shrink with the tile (the epilogue is 0.6 us per 64 columns).
       if (bn == 128 && N > 64 && static_cast<int64_t>(tiles_m) * ((N + 63) / 64) <= sms) bn = 64;
+      // the normalised-residual epilogue keeps three column vectors in shared memory (tiles up to 128 wide); row
+      // statistics are written per whole tile width
+      if (lnr && bn > 128) bn = 128;
+      if (emit) {
+        if (bn_group) bn = bn_group;
+        while (bn > 64 && N % bn) bn /= 2;
+        if (N % bn) return fail(E_UNSUPPORTED_OP, "row statistics need an output width that is a multiple of 64");
+        bn_group = bn;
+        p.stats_layout[G.out] = {static_cast<int>(N / bn) * 2, bn / 2};
+      }
       const bool hb = G.bias >= 0, hr = G.res >= 0;
       const int act = G.act;
       const int act2 = G.act2;
+      const int ln = lna ? 1 : lnr ? 2 : 0;
+      Ptr ps_in, ps_out, pc1, pg, pbt;
+      int64_t pitch_in = 0, pitch_out = 0;
+      Plan::StatsLayout lay;
+      if (ln) {
+        const int raw = lna ? G.ln_a : G.ln_res;
+        lay = p.stats_layout[raw];
+        if (!lay.slots || !stats_ptr(raw, sg.r0, lna ? K : N, &ps_in, &pitch_in)) return fail(E_INTERNAL, "row statistics of " + g.tensors[raw].name + " are not planned");
+        if (static_cast<int64_t>(lay.slots) * lay.cols != (lna ? K : N)) return fail(E_INTERNAL, "row statistics layout of " + g.tensors[raw].name);
+        if (lna) { pc1.where = 5; pc1.off = static_cast<int64_t>(pk + ((static_cast<size_t>(N) * K * 2 + 255) & ~size_t(255))); }
+        else { pg = ptr_of(G.ln_gamma, 0); pbt = ptr_of(G.ln_beta, 0); }
+      }
+      if (emit && !stats_ptr(G.out, sg.r0, N, &ps_out, &pitch_out)) return fail(E_INTERNAL, "row statistics of " + g.tensors[G.out].name + " are not planned");
+      const float ln_eps = G.ln_eps;
       struct Cache { const void* a = nullptr; const void* w = nullptr; const void* o = nullptr; const void* r = nullptr; CUtensorMap ta, tb, to, tr; };
       auto cache = std::make_shared<Cache>();
       add(gi, 1, [=](const RunCtx& x) {
@@ -319,45 +419,265 @@ struct Builder {
         ep.has_residual = hr;
         ep.act2 = act2;
         ep.status = reinterpret_cast<int*>(x.arena);
+        if (ln) {
+          ep.ln_stats = reinterpret_cast<const float2*>(x.resolve(ps_in));
+          ep.ln_pitch = pitch_in;
+          ep.ln_slots = lay.slots;
+          ep.ln_cols = lay.cols;
+          ep.ln_eps = ln_eps;
+          if (ln == 1) {
+            ep.ln_c1 = reinterpret_cast<const float*>(x.resolve(pc1));
+            ep.ln_c2 = ep.ln_c1 + N;
+          } else {
+            ep.ln_gamma = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pg));
+            ep.ln_beta = reinterpret_cast<const __nv_bfloat16*>(x.resolve(pbt));
+          }
+        }
+        if (emit) {
+          ep.emit_stats = reinterpret_cast<float2*>(x.resolve(ps_out));
+          ep.emit_pitch = pitch_out;
+        }
         const int tiles = tiles_m * static_cast<int>((N + bn - 1) / bn);
         const int grid = std::min(tiles, x.plan->sm_count);
-        const int variant = (bn == 256 ? 0 : bn == 128 ? 6 : 12) + act * 2 + (hr ? 1 : 0);
-        const dim3 gd(grid), bd(k::GEMM_THREADS);
+        const dim3 gd(grid);
         const int Ni = static_cast<int>(N), Ki = static_cast<int>(K);
-#define SOD2_GEMM_CASE(V, BN_, KCH_, ST_, ACT_, RES_)                                                                        \
-        case V: {                                                                                                            \
-          constexpr int smem = k::GemmSmem<BN_, KCH_, ST_>::TOTAL;                                                            \
-          static bool once = (cudaFuncSetAttribute(k::gemm_bf16_tcgen05<BN_, KCH_, ST_, ACT_, false, RES_>,                   \
-                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);                 \
-          (void)once;                                                                                                        \
-          launch_pdl(k::gemm_bf16_tcgen05<BN_, KCH_, ST_, ACT_, false, RES_>, gd, bd, smem, x.stream, cache->ta, cache->tb,   \
-                     cache->to, cache->tr, M, Ni, Ki, ep);                                                                    \
-        } break;
-        switch (variant) {
-          SOD2_GEMM_CASE(0, 256, 1, 4, 0, false)
-          SOD2_GEMM_CASE(1, 256, 1, 4, 0, true)
-          SOD2_GEMM_CASE(2, 256, 1, 4, 1, false)
-          SOD2_GEMM_CASE(3, 256, 1, 4, 1, true)
-          SOD2_GEMM_CASE(4, 256, 1, 4, 2, false)
-          SOD2_GEMM_CASE(5, 256, 1, 4, 2, true)
-          SOD2_GEMM_CASE(6, 128, 2, 3, 0, false)
-          SOD2_GEMM_CASE(7, 128, 2, 3, 0, true)
-          SOD2_GEMM_CASE(8, 128, 2, 3, 1, false)
-          SOD2_GEMM_CASE(9, 128, 2, 3, 1, true)
-          SOD2_GEMM_CASE(10, 128, 2, 3, 2, false)
-          SOD2_GEMM_CASE(11, 128, 2, 3, 2, true)
-          SOD2_GEMM_CASE(12, 64, 2, 3, 0, false)
-          SOD2_GEMM_CASE(13, 64, 2, 3, 0, true)
-          SOD2_GEMM_CASE(14, 64, 2, 3, 1, false)
-          SOD2_GEMM_CASE(15, 64, 2, 3, 1, true)
-          SOD2_GEMM_CASE(16, 64, 2, 3, 2, false)
-          default:
-          SOD2_GEMM_CASE(17, 64, 2, 3, 2, true)
-        }
-#undef SOD2_GEMM_CASE
-        return cudaGetLastError();
+        cudaError_t e;
+        if (bn == 256) e = gemm_dispatch<256, 1, 4>(act, hr, ln, emit, gd, x.stream, cache->ta, cache->tb, cache->to, cache->tr, M, Ni, Ki, ep);
+        else if (bn == 128) e = gemm_dispatch<128, 2, 3>(act, hr, ln, emit, gd, x.stream, cache->ta, cache->tb, cache->to, cache->tr, M, Ni, Ki, ep);
+        else e = gemm_dispatch<64, 2, 3>(act, hr, ln, emit, gd, x.stream, cache->ta, cache->tb, cache->to, cache->tr, M, Ni, Ki, ep);
+        return e != cudaSuccess ? e : cudaGetLastError();
       });
     }
+    return OK;
+  }
+
+  // ------------------------------------------------------------------------------ GEMM chains
+  // Epilogue version of the chain kernel for a group, or -1 if the group cannot be a chain member.
+  int chain_epi(const Group& G) const {
+    if (G.kind != GKind::GEMM || G.has_ln || G.act2 || g.tensors[G.a].dtype != DType::BF16) return -1;
+    const bool res = G.res >= 0, emit = G.emit_stats != 0;
+    const int ln = G.ln_a >= 0 ? 1 : G.ln_res >= 0 ? 2 : 0;
+    if (G.act == 0 && !res && ln == 0 && !emit) return k::CE_PLAIN;
+    if (G.act == 0 && res && ln == 0 && !emit) return k::CE_RES;
+    if (G.act == 1 && !res && ln == 0 && !emit) return k::CE_GELU;
+    if (G.act == 0 && res && ln == 0 && emit) return k::CE_RES_EMIT;
+    if (G.act == 0 && res && ln == 2 && !emit) return k::CE_RES_LN2;
+    if (G.act == 0 && res && ln == 2 && emit) return k::CE_RES_LN2_EMIT;
+    if (G.act == 0 && !res && ln == 1 && !emit) return k::CE_LN1;
+    if (G.act == 1 && !res && ln == 1 && !emit) return k::CE_LN1_GELU;
+    return -1;
+  }
+  struct ChainMember { int64_t M = 0, N = 0, K = 0, lda = 0, ldo = 0, ldr = 0; int epi = -1; };
+  // A group as a chain member: one launch segment over all requests, shapes the 128 x 128 tile version takes.
+  bool chain_member(const Group& G, ChainMember* cm) {
+    cm->epi = chain_epi(G);
+    if (cm->epi < 0) return false;
+    const Tensor& W = g.tensors[G.w];
+    cm->K = W.S.dims[0].e.const_value();
+    cm->N = W.S.dims[1].e.const_value();
+    std::vector<int> ts = {G.a, G.out};
+    if (G.res >= 0) ts.push_back(G.res);
+    int64_t cols;
+    std::vector<int64_t> lds;
+    std::vector<Seg> segs;
+    const std::string keep = p.err;
+    if (row_segments(ts, &cols, &lds, &segs) != OK) { p.err = keep; return false; }
+    if (segs.size() != 1 || segs[0].rows <= 0 || cols != cm->K) return false;
+    if (cm->K % 64 || lds[0] % 8 || lds[1] % 8 || cm->N % 8 || (G.res >= 0 && lds[2] % 8)) return false;
+    if (G.emit_stats && (cm->N % 128 || lds[1] != cm->N)) return false;
+    if (G.ln_a >= 0 && lds[0] != cm->K) return false;
+    if (G.ln_res >= 0 && lds[2] != cm->N) return false;
+    cm->M = segs[0].rows;
+    cm->lda = lds[0]; cm->ldo = lds[1]; cm->ldr = G.res >= 0 ? lds[2] : 0;
+    return true;
+  }
+  // the same bytes in the same order: root, offset, extents and strides of request 0 (the members are one segment)
+  bool same_view(int t1, int t2) const {
+    const View &a = p.views[t1][0], &b = p.views[t2][0];
+    return a.root == b.root && a.offset == b.offset && a.dims == b.dims && a.strides == b.strides;
+  }
+  // Maximal runs of consecutive chainable GEMM groups with equal row counts.  A member may read rows written by an
+  // earlier member only as its A operand or its residual and only as the very view the earlier member wrote
+  // (row block i then depends on row block i alone); any other overlap ends the run.
+  Status find_chains() {
+    p.chains.clear();
+    p.chain_of.assign(c.groups.size(), -1);
+    p.chain_counter_words = 0;
+    if (!(c.flags & OPT_GEMM_CHAIN) || (c.flags & OPT_NO_FUSION)) return OK;
+    size_t gi = 0;
+    while (gi < c.groups.size()) {
+      ChainMember first;
+      if (!chain_member(c.groups[gi], &first)) { ++gi; continue; }
+      std::vector<int> run = {static_cast<int>(gi)};
+      size_t gj = gi + 1;
+      static const int chain_max = [] { const char* e = getenv("SOD2_CHAIN_MAX"); const int v = e ? atoi(e) : k::CHAIN_MAX; return std::max(1, std::min(v, k::CHAIN_MAX)); }();
+      while (gj < c.groups.size() && run.size() < static_cast<size_t>(chain_max)) {
+        ChainMember cm;
+        const Group& G = c.groups[gj];
+        if (!chain_member(G, &cm) || cm.M != first.M) break;
+        bool ok = true;
+        for (int t : G.ext_in) {
+          if (g.tensors[t].kind == TKind::CONST || c.storage[t].kind == Storage::FOLDED || p.views[t].empty()) continue;
+          for (int m : run) {
+            const int o = c.groups[m].out;
+            if (p.views[t][0].root != p.views[o][0].root) continue;
+            if (!((t == G.a || t == G.res) && same_view(t, o))) ok = false;
+          }
+        }
+        // nothing a member writes may be storage an earlier member reads or writes
+        for (int m : run) {
+          const Group& E = c.groups[m];
+          for (int t : E.ext_in) if (!p.views[t].empty() && p.views[t][0].root == p.views[G.out][0].root) ok = false;
+          if (p.views[E.out][0].root == p.views[G.out][0].root) ok = false;
+        }
+        if (!ok) break;
+        run.push_back(static_cast<int>(gj));
+        ++gj;
+      }
+      if (run.size() >= 2) {
+        Plan::Chain ch;
+        ch.groups = run;
+        ch.rows = static_cast<int>(first.M);
+        ch.counter_word = p.chain_counter_words;
+        p.chain_counter_words += run.size() * static_cast<size_t>((first.M + 127) / 128);
+        for (int m : run) p.chain_of[m] = static_cast<int>(p.chains.size());
+        p.chains.push_back(ch);
+        gi = gj;
+      } else {
+        ++gi;
+      }
+    }
+    return OK;
+  }
+
+  // One launch for all members of chain `ci`.
+  Status build_gemm_chain(int ci) {
+    const Plan::Chain& ch = p.chains[ci];
+    const int n = static_cast<int>(ch.groups.size());
+    if (p.stats_layout.size() != g.tensors.size()) p.stats_layout.assign(g.tensors.size(), Plan::StatsLayout());
+    struct Mem {
+      ChainMember cm;
+      Ptr pa, po, pr, pw, pb, pc1, pg, pbt, ps_in, ps_out;
+      int64_t pitch_in = 0, pitch_out = 0;
+      Plan::StatsLayout lay;
+      bool hb = false, hr = false, emit = false;
+      int ln = 0, dep_a = -1, dep_r = -1;
+      float eps = 1e-5f;
+    };
+    std::vector<Mem> ms(n);
+    auto stats_ptr = [&](int t, int64_t width, Ptr* out, int64_t* pitch) -> bool {
+      const int root = p.views[t][0].root;
+      const RootBuf& RR = p.roots[root];
+      if (RR.where != RootBuf::ARENA || RR.stats_off < 0 || p.views[t][0].offset != 0) return false;
+      const int64_t row0 = p.inst_off[root][0] / (width * 2);
+      out->where = RootBuf::ARENA;
+      out->index = -1;
+      out->off = static_cast<int64_t>(RR.arena_off) + RR.stats_off + row0 * 8;
+      *pitch = RR.stats_rows;
+      return true;
+    };
+    double flops_total = 0.0;
+    std::vector<double> fl(n);
+    for (int i = 0; i < n; ++i) {
+      const Group& G = c.groups[ch.groups[i]];
+      Mem& m = ms[i];
+      if (!chain_member(G, &m.cm)) return fail(E_INTERNAL, "chain member changed its mind");
+      const int64_t N = m.cm.N, K = m.cm.K;
+      m.hb = G.bias >= 0; m.hr = G.res >= 0; m.emit = G.emit_stats != 0;
+      m.ln = G.ln_a >= 0 ? 1 : G.ln_res >= 0 ? 2 : 0;
+      m.eps = G.ln_eps;
+      m.pa = ptr_of(G.a, 0); m.po = ptr_of(G.out, 0);
+      if (m.hr) m.pr = ptr_of(G.res, 0);
+      if (m.hb) m.pb = ptr_of(G.bias, 0);
+      size_t pk = 0;
+      bool found = false;
+      for (size_t q = 0; q < c.packed_consts.size(); ++q)
+        if (c.packed_consts[q] == G.w) {
+          const Compiled::PackedLn& e = c.packed_ln[q];
+          if (m.ln == 1 ? (e.gamma == G.ln_gamma && e.beta == G.ln_beta && e.bias == G.bias) : e.gamma < 0) { pk = c.packed_off[q]; found = true; }
+        }
+      if (!found) return fail(E_INTERNAL, "no prepacked copy of " + g.tensors[G.w].name);
+      m.pw.where = 5; m.pw.off = static_cast<int64_t>(pk);
+      if (m.emit) {
+        p.stats_layout[G.out] = {static_cast<int>(N / k::CHAIN_BN) * 2, k::CHAIN_BN / 2};
+        if (!stats_ptr(G.out, N, &m.ps_out, &m.pitch_out)) return fail(E_INTERNAL, "row statistics of " + g.tensors[G.out].name + " are not planned");
+      }
+      if (m.ln) {
+        const int raw = m.ln == 1 ? G.ln_a : G.ln_res;
+        m.lay = p.stats_layout[raw];
+        if (!m.lay.slots || !stats_ptr(raw, m.ln == 1 ? K : N, &m.ps_in, &m.pitch_in)) return fail(E_INTERNAL, "row statistics of " + g.tensors[raw].name + " are not planned");
+        if (static_cast<int64_t>(m.lay.slots) * m.lay.cols != (m.ln == 1 ? K : N)) return fail(E_INTERNAL, "row statistics layout of " + g.tensors[raw].name);
+        if (m.ln == 1) { m.pc1.where = 5; m.pc1.off = static_cast<int64_t>(pk + ((static_cast<size_t>(N) * K * 2 + 255) & ~size_t(255))); }
+        else { m.pg = ptr_of(G.ln_gamma, 0); m.pbt = ptr_of(G.ln_beta, 0); }
+      }
+      for (int j = 0; j < i; ++j) {
+        const int o = c.groups[ch.groups[j]].out;
+        if (p.views[G.a][0].root == p.views[o][0].root) m.dep_a = j;
+        if (m.hr && p.views[G.res][0].root == p.views[o][0].root) m.dep_r = j;
+      }
+      fl[i] = 2.0 * static_cast<double>(m.cm.M) * N * K;
+      flops_total += fl[i];
+    }
+    const int M = ch.rows;
+    const int tiles_m = (M + 127) / 128;
+    const size_t counter_off = p.chain_counter_off + 4 * ch.counter_word;   // chain_counter_off is final: the arena is planned
+    struct Cache { std::vector<const void*> key; k::GemmChainMaps maps; };
+    auto cache = std::make_shared<Cache>();
+    auto L = std::make_shared<Launch>();
+    L->group = ch.groups[0];
+    L->n_kernels = 1;
+    for (int i = 0; i < n; ++i) L->share.push_back({ch.groups[i], flops_total > 0 ? fl[i] / flops_total : 1.0 / n});
+    L->fn = [=](const RunCtx& x) {
+      std::vector<const void*> key;
+      k::GemmChainParams cp{};
+      cp.n = n; cp.M = M; cp.tiles_m = tiles_m;
+      cp.done = reinterpret_cast<unsigned*>(x.arena + counter_off);
+      int tile0 = 0;
+      const void* A[k::CHAIN_MAX]; const void* Wt[k::CHAIN_MAX]; void* O[k::CHAIN_MAX]; const void* R[k::CHAIN_MAX];
+      for (int i = 0; i < n; ++i) {
+        const Mem& m = ms[i];
+        A[i] = x.resolve(m.pa); Wt[i] = x.resolve(m.pw); O[i] = x.resolve(m.po); R[i] = m.hr ? x.resolve(m.pr) : O[i];
+        key.push_back(A[i]); key.push_back(Wt[i]); key.push_back(O[i]); key.push_back(R[i]);
+        k::GemmChainProblem& P = cp.p[i];
+        P.N = static_cast<int>(m.cm.N); P.K = static_cast<int>(m.cm.K);
+        P.tiles_n = static_cast<int>((m.cm.N + k::CHAIN_BN - 1) / k::CHAIN_BN);
+        P.tile0 = tile0;
+        tile0 += tiles_m * P.tiles_n;
+        P.epi = m.cm.epi; P.dep_a = m.dep_a; P.dep_r = m.dep_r;
+        P.ep.bias = m.hb ? reinterpret_cast<const __nv_bfloat16*>(x.resolve(m.pb)) : nullptr;
+        P.ep.has_residual = m.hr;
+        P.ep.status = reinterpret_cast<int*>(x.arena);
+        if (m.ln) {
+          P.ep.ln_stats = reinterpret_cast<const float2*>(x.resolve(m.ps_in));
+          P.ep.ln_pitch = m.pitch_in; P.ep.ln_slots = m.lay.slots; P.ep.ln_cols = m.lay.cols; P.ep.ln_eps = m.eps;
+          if (m.ln == 1) { P.ep.ln_c1 = reinterpret_cast<const float*>(x.resolve(m.pc1)); P.ep.ln_c2 = P.ep.ln_c1 + m.cm.N; }
+          else { P.ep.ln_gamma = reinterpret_cast<const __nv_bfloat16*>(x.resolve(m.pg)); P.ep.ln_beta = reinterpret_cast<const __nv_bfloat16*>(x.resolve(m.pbt)); }
+        }
+        if (m.emit) { P.ep.emit_stats = reinterpret_cast<float2*>(x.resolve(m.ps_out)); P.ep.emit_pitch = m.pitch_out; }
+      }
+      cp.total_tiles = tile0;
+      if (cache->key != key) {
+        for (int i = 0; i < n; ++i) {
+          const Mem& m = ms[i];
+          if (!encode_bf16_kchunks(&cache->maps.a[i], A[i], M, m.cm.K, m.cm.lda, 128, k::CHAIN_KCH) ||
+              !encode_bf16_kchunks(&cache->maps.b[i], Wt[i], m.cm.N, m.cm.K, m.cm.K, k::CHAIN_BN, k::CHAIN_KCH) ||
+              !encode_bf16_2d(&cache->maps.o[i], O[i], M, m.cm.N, m.cm.ldo, 128) ||
+              !encode_bf16_2d(&cache->maps.r[i], R[i], M, m.cm.N, m.hr ? m.cm.ldr : m.cm.ldo, 128))
+            return cudaErrorInvalidValue;
+        }
+        for (int i = n; i < k::CHAIN_MAX; ++i) { cache->maps.a[i] = cache->maps.a[0]; cache->maps.b[i] = cache->maps.b[0]; cache->maps.o[i] = cache->maps.o[0]; cache->maps.r[i] = cache->maps.r[0]; }
+        cache->key = key;
+      }
+      constexpr int smem = k::GemmSmem<k::CHAIN_BN, k::CHAIN_KCH, k::CHAIN_STAGES>::TOTAL;
+      static bool once = (cudaFuncSetAttribute(k::gemm_chain_bf16_tcgen05, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);
+      (void)once;
+      const int grid = std::min(cp.total_tiles, x.plan->sm_count);
+      const cudaError_t e = launch_pdl(k::gemm_chain_bf16_tcgen05, dim3(grid), dim3(k::GEMM_THREADS), smem, x.stream, cache->maps, cp,
+                                       reinterpret_cast<int*>(x.arena));
+      return e != cudaSuccess ? e : cudaGetLastError();
+    };
+    p.gpu_launches += 1;
+    p.launches.push_back(L);
     return OK;
   }
 
@@ -1445,11 +1765,13 @@ struct Builder {
     p.group_bytes.clear();
     p.gpu_launches = 0;
     // the fp32 row kernel and the elementwise chains have no bounded waits, tickets or device-side counts
-    // a pooling group right after a layout change of the same tensor: neither reads what the other writes
+    // a pooling group right after a layout change of the SAME tensor: neither reads what the other writes, and the
+    // shared input stays live over both steps, so the arena plan (liveness by step) cannot hand the pooled output a
+    // slot that the layout kernel still reads
     p.side_group.assign(c.groups.size(), 0);
     for (size_t gi = 1; gi < c.groups.size(); ++gi) {
       const Group &A = c.groups[gi - 1], &Bg = c.groups[gi];
-      if (Bg.kind == GKind::GAP && A.kind == GKind::LAYOUT && Bg.a != A.out && A.a != Bg.out && !p.side_group[gi - 1])
+      if (Bg.kind == GKind::GAP && A.kind == GKind::LAYOUT && Bg.a == A.a && Bg.a != A.out && A.a != Bg.out && !p.side_group[gi - 1])
         p.side_group[gi] = 1;
     }
     p.uses_header = false;
@@ -1458,6 +1780,13 @@ struct Builder {
     for (size_t gi = 0; gi < c.groups.size(); ++gi) {
       const Group& G = c.groups[gi];
       Status s = OK;
+      if (gi < p.chain_of.size() && p.chain_of[gi] >= 0) {
+        // the first member builds the launch for the whole chain
+        if (p.chains[p.chain_of[gi]].groups.front() == static_cast<int>(gi)) s = build_gemm_chain(p.chain_of[gi]);
+        if (s != OK) return s;
+        cost(G);
+        continue;
+      }
       switch (G.kind) {
         case GKind::GEMM: s = build_gemm(static_cast<int>(gi), G); break;
         case GKind::ATTENTION: s = build_attention(static_cast<int>(gi), G); break;
@@ -1500,11 +1829,51 @@ __global__ void transpose_bf16(const __nv_bfloat16* __restrict__ in, __nv_bfloat
   }
 }
 
+// Weights of a GEMM whose A operand is a folded LayerNorm: out[n, k] = bf16(gamma[k] * in[k, n]).
+__global__ void transpose_scale_bf16(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16* __restrict__ gamma,
+                                     __nv_bfloat16* __restrict__ out, int K, int N) {
+  __shared__ __nv_bfloat16 tile[32][33];
+  const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int kk = k0 + i, n = n0 + threadIdx.x;
+    if (kk < K && n < N) tile[i][threadIdx.x] = __float2bfloat16_rn(__bfloat162float(in[static_cast<long long>(kk) * N + n]) * __bfloat162float(gamma[kk]));
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int n = n0 + i, kk = k0 + threadIdx.x;
+    if (kk < K && n < N) out[static_cast<long long>(n) * K + kk] = tile[threadIdx.x][i];
+  }
+}
+// The two epilogue vectors of that GEMM, one warp per output column, fp64 sums in a fixed order:
+//   c1[n] = sum_k Wp[n, k]  (of the scaled copy as rounded to bf16, so that it cancels what the MMA adds up)
+//   c2[n] = sum_k beta[k] * W[k, n] + bias[n]
+__global__ void ln_fold_vectors(const __nv_bfloat16* __restrict__ Wp, const __nv_bfloat16* __restrict__ W, const __nv_bfloat16* __restrict__ beta,
+                                const __nv_bfloat16* __restrict__ bias, float* __restrict__ c1, float* __restrict__ c2, int K, int N) {
+  const int n = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (n >= N) return;
+  double a = 0.0, b = 0.0;
+  for (int kk = lane; kk < K; kk += 32) {
+    a += static_cast<double>(__bfloat162float(Wp[static_cast<long long>(n) * K + kk]));
+    b += static_cast<double>(__bfloat162float(beta[kk])) * static_cast<double>(__bfloat162float(W[static_cast<long long>(kk) * N + n]));
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) { a += __shfl_xor_sync(0xffffffffu, a, o); b += __shfl_xor_sync(0xffffffffu, b, o); }
+  if (lane == 0) {
+    c1[n] = static_cast<float>(a);
+    c2[n] = static_cast<float>(b + (bias ? static_cast<double>(__bfloat162float(bias[n])) : 0.0));
+  }
+}
+
 }  // namespace
 
 Status build_launches(Plan* p) {
   Builder b(*p);
   return b.run();
+}
+
+Status detect_chains(Plan* p) {
+  Builder b(*p);
+  return b.find_chains();
 }
 
 Status prepack_weights(Compiled* c, void* workspace, size_t bytes, void* stream) {
@@ -1540,6 +1909,20 @@ Status prepack_weights(Compiled* c, void* workspace, size_t bytes, void* stream)
       continue;
     }
     const int K = static_cast<int>(W.S.dims[0].e.const_value()), N = static_cast<int>(W.S.dims[1].e.const_value());
+    if (c->packed_ln[i].gamma >= 0) {   // folded LayerNorm: gamma-scaled copy + the two epilogue vectors
+      const Compiled::PackedLn& e = c->packed_ln[i];
+      const Tensor &Gm = c->g.tensors[e.gamma], &Bt = c->g.tensors[e.beta];
+      const Tensor* Bi = e.bias >= 0 ? &c->g.tensors[e.bias] : nullptr;
+      if (!Gm.dev_ptr || !Bt.dev_ptr || (Bi && !Bi->dev_ptr)) { c->err = "LayerNorm constants of " + W.name + " have no device data"; return E_INVALID_ARG; }
+      __nv_bfloat16* Wp = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + c->packed_off[i]);
+      float* c1 = reinterpret_cast<float*>(static_cast<char*>(workspace) + c->packed_off[i] + ((static_cast<size_t>(N) * K * 2 + 255) & ~size_t(255)));
+      transpose_scale_bf16<<<dim3((N + 31) / 32, (K + 31) / 32), dim3(32, 8), 0, static_cast<cudaStream_t>(stream)>>>(
+          static_cast<const __nv_bfloat16*>(W.dev_ptr), static_cast<const __nv_bfloat16*>(Gm.dev_ptr), Wp, K, N);
+      ln_fold_vectors<<<(N + 7) / 8, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+          Wp, static_cast<const __nv_bfloat16*>(W.dev_ptr), static_cast<const __nv_bfloat16*>(Bt.dev_ptr),
+          Bi ? static_cast<const __nv_bfloat16*>(Bi->dev_ptr) : nullptr, c1, c1 + N, K, N);
+      continue;
+    }
     transpose_bf16<<<dim3((N + 31) / 32, (K + 31) / 32), dim3(32, 8), 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const __nv_bfloat16*>(W.dev_ptr), reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + c->packed_off[i]), K, N);
   }
@@ -1557,7 +1940,7 @@ Status run_plan_timed(Plan* p, const void* const* inputs, void* const* outputs, 
   const size_t n = p->launches.size();
   std::vector<cudaEvent_t> ev(2 * n);
   for (auto& e : ev) if (cudaEventCreate(&e) != cudaSuccess) { p->err = "cudaEventCreate failed"; return E_CUDA; }
-  if (p->uses_header) cudaMemsetAsync(arena, 0, 256, x.stream);
+  if (p->uses_header) cudaMemsetAsync(arena, 0, p->header_clear_bytes, x.stream);
   Status st = OK;
   for (size_t i = 0; i < n && st == OK; ++i) {
     cudaEventRecord(ev[2 * i], x.stream);
@@ -1570,7 +1953,8 @@ Status run_plan_timed(Plan* p, const void* const* inputs, void* const* outputs, 
     for (size_t i = 0; i < n; ++i) {
       float ms = 0.f;
       cudaEventElapsedTime(&ms, ev[2 * i], ev[2 * i + 1]);
-      group_ms[p->launches[i]->group] += ms;
+      if (p->launches[i]->share.empty()) group_ms[p->launches[i]->group] += ms;
+      else for (auto& sh : p->launches[i]->share) group_ms[sh.first] += ms * static_cast<float>(sh.second);   // a chain: by algorithmic flops
     }
   for (auto& e : ev) cudaEventDestroy(e);
   return st;
@@ -1657,7 +2041,7 @@ Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* 
     p->sm_count_known = true;
   }
   RunCtx x{inputs, outputs, static_cast<char*>(arena), static_cast<char*>(p->c->packed_ws), static_cast<cudaStream_t>(stream), p};
-  if (p->uses_header && cudaMemsetAsync(arena, 0, 256, x.stream) != cudaSuccess) { p->err = "cannot clear the status word"; return E_CUDA; }
+  if (p->uses_header && cudaMemsetAsync(arena, 0, p->header_clear_bytes, x.stream) != cudaSuccess) { p->err = "cannot clear the status word"; return E_CUDA; }
   if (!ensure_side_stream(p)) { p->err = "cannot create the second stream"; return E_CUDA; }
   const int n_groups = static_cast<int>(p->side_group.size());
   cudaStream_t side = static_cast<cudaStream_t>(p->side_stream);

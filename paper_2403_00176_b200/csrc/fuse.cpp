@@ -355,6 +355,81 @@ struct Fuser {
     finish(G);
   }
 
+  // 3c. LayerNorm folded into the neighbouring GEMMs (RDP-enabled fusion, Section 4.2: the row width is a known
+  // constant and the operands' index spaces are proven equal, so the normalisation distributes over the product):
+  //   LayerNorm(x) W + b = rstd_i (x_i . (gamma o W)) - rstd_i mean_i (gamma^T W) + (beta^T W + b).
+  // A bf16 LayerNorm whose input is the output of a GEMM group and whose every consumer is a GEMM group (as the A
+  // operand or as the residual) is removed: the producing GEMM also writes per-row statistics, the consumers read
+  // the raw rows and normalise in their epilogues; the normalised tensor becomes an alias of the raw one and is
+  // never stored.  One kernel and one round trip of the tensor through memory less per LayerNorm.
+  void fold_layernorms() {
+    c.stats_width.assign(g.tensors.size(), 0);
+    if (!(c.flags & OPT_LN_FOLD) || (c.flags & (OPT_NO_FUSION | OPT_SPLITK_LN))) return;
+    std::vector<char> drop(c.groups.size(), 0);
+    for (size_t li = 0; li < c.groups.size(); ++li) {
+      const Group L = c.groups[li];
+      if (L.kind != GKind::LAYERNORM) continue;
+      const int raw = L.a, ln = L.out;
+      const Tensor& R = g.tensors[raw];
+      if (R.dtype != DType::BF16 || R.kind != TKind::VALUE || R.is_output || g.tensors[ln].is_output) continue;
+      if (c.storage[raw].kind != Storage::ROOT || c.storage[ln].kind != Storage::ROOT) continue;
+      if (R.S.rank < 1 || !R.S.dims[R.S.rank - 1].known() || !R.S.dims[R.S.rank - 1].e.is_const()) continue;
+      const int64_t D = R.S.dims[R.S.rank - 1].e.const_value();
+      if (D % 64 || D < 64 || D > 4096) continue;
+      if (!is_const_vec(L.gamma, R.S.dims[R.S.rank - 1]) || !is_const_vec(L.beta, R.S.dims[R.S.rank - 1])) continue;
+      if (g.tensors[L.gamma].dtype != DType::BF16 || g.tensors[L.beta].dtype != DType::BF16) continue;
+      // the producer: a plain bf16 GEMM group (no activation: the statistics are taken of the stored rows)
+      const int pn = R.producer;
+      if (pn < 0 || assigned[pn] < 0) continue;
+      const int pi = assigned[pn];
+      const Group& P = c.groups[pi];
+      if (P.kind != GKind::GEMM || P.out != raw || P.has_ln || P.act || P.act2 || P.ln_a >= 0 || g.tensors[P.a].dtype != DType::BF16) continue;
+      // the consumers
+      std::vector<std::pair<int, int>> uses;   // (group, 1 = A operand, 2 = residual)
+      bool ok = true;
+      for (int cn : data_consumers(ln)) {
+        const int gi = assigned[cn];
+        if (gi < 0) { ok = false; break; }
+        const Group& G = c.groups[gi];
+        if (G.kind != GKind::GEMM || G.has_ln || G.ln_a >= 0 || G.ln_res >= 0 || g.tensors[G.w].dtype != DType::BF16) { ok = false; break; }
+        for (auto& u : uses) if (u.first == gi) ok = false;                       // one role per group
+        if (!ok) break;
+        if (cn == G.nodes[0] && G.a == ln && g.nodes[cn].ins[0] == ln && G.res != ln) {
+          if (G.res >= 0 || G.emit_stats || G.act2) { ok = false; break; }
+          uses.push_back({gi, 1});
+        } else if (G.res == ln && G.a != ln && G.act == 0 && G.act2 == 0) {
+          const ShapeVal& ws = g.tensors[G.w].S;
+          if (!(ws.dims[1].e.is_const() && ws.dims[1].e.const_value() == D)) { ok = false; break; }
+          uses.push_back({gi, 2});
+        } else { ok = false; break; }
+      }
+      if (!ok || uses.empty()) continue;
+      c.groups[pi].emit_stats = 1;
+      c.stats_width[raw] = static_cast<int>(D);
+      for (auto& u : uses) {
+        Group& G = c.groups[u.first];
+        (u.second == 1 ? G.ln_a : G.ln_res) = raw;
+        G.ln_gamma = L.gamma; G.ln_beta = L.beta; G.ln_eps = L.eps;
+        for (int t : {L.gamma, L.beta}) if (std::find(G.ext_in.begin(), G.ext_in.end(), t) == G.ext_in.end()) G.ext_in.push_back(t);
+      }
+      c.storage[ln] = Storage{Storage::ALIAS, L.nodes[0], raw, -1, 0};
+      // the LayerNorm operator now runs inside its consumers; it is reported with the first of them, and the
+      // dependency walk passes through it to the producer of the raw rows
+      c.groups[uses[0].first].nodes.push_back(L.nodes[0]);
+      assigned[L.nodes[0]] = -1;
+      g.nodes[L.nodes[0]].group = uses[0].first;
+      drop[li] = 1;
+    }
+    // remove the folded groups
+    std::vector<int> remap(c.groups.size(), -1);
+    std::vector<Group> kept;
+    for (size_t gi = 0; gi < c.groups.size(); ++gi) if (!drop[gi]) { remap[gi] = static_cast<int>(kept.size()); kept.push_back(c.groups[gi]); }
+    if (kept.size() == c.groups.size()) return;
+    c.groups.swap(kept);
+    for (auto& a : assigned) if (a >= 0) a = remap[a];
+    for (auto& n : g.nodes) if (n.group >= 0) n.group = remap[n.group];
+  }
+
   Status run() {
     // 1. nodes evaluated by RDP itself: every output has a fully known value map (shape arithmetic)
     c.node_folded.assign(g.nodes.size(), 0);
@@ -508,6 +583,7 @@ struct Fuser {
         }
       }
     }
+    fold_layernorms();
     // 4. partition at execution-determined operators (Section 4.3): a node's sub-graph index is
     // one more than that of any execution-determined producer it (transitively) depends on.
     std::vector<int> tsub(g.tensors.size(), 0);
@@ -567,13 +643,25 @@ struct Fuser {
     // 6. weights that the tcgen05 GEMM wants K-major
     for (auto& G2 : c.groups)
       if (G2.kind == GKind::GEMM && g.tensors[G2.w].dtype == DType::BF16) {
-        if (std::find(c.packed_consts.begin(), c.packed_consts.end(), G2.w) == c.packed_consts.end()) {
-          c.packed_consts.push_back(G2.w);
-          c.packed_off.push_back(c.packed_bytes);
-          const ShapeVal& s = g.tensors[G2.w].S;
-          size_t bytes = static_cast<size_t>(s.dims[0].e.const_value() * s.dims[1].e.const_value() * 2);
-          c.packed_bytes += (bytes + 255) & ~size_t(255);
+        const ShapeVal& s = g.tensors[G2.w].S;
+        const size_t wbytes = static_cast<size_t>(s.dims[0].e.const_value() * s.dims[1].e.const_value() * 2);
+        bool found = false;
+        for (size_t i = 0; i < c.packed_consts.size(); ++i)
+          if (c.packed_consts[i] == G2.w) {
+            const Compiled::PackedLn& e = c.packed_ln[i];
+            if (G2.ln_a >= 0 ? (e.gamma == G2.ln_gamma && e.beta == G2.ln_beta && e.bias == G2.bias) : e.gamma < 0) found = true;
+          }
+        if (found) continue;
+        c.packed_consts.push_back(G2.w);
+        c.packed_off.push_back(c.packed_bytes);
+        Compiled::PackedLn e;
+        size_t bytes = (wbytes + 255) & ~size_t(255);
+        if (G2.ln_a >= 0) {   // gamma-scaled copy followed by the two fp32 epilogue vectors
+          e.gamma = G2.ln_gamma; e.beta = G2.ln_beta; e.bias = G2.bias;
+          bytes += (static_cast<size_t>(s.dims[1].e.const_value()) * 8 + 255) & ~size_t(255);
         }
+        c.packed_ln.push_back(e);
+        c.packed_bytes += bytes;
       }
     // ... and convolution weights as [Cout, (dy, dx, ci)] for the implicit GEMM
     for (auto& G2 : c.groups)
@@ -581,6 +669,7 @@ struct Fuser {
         if (std::find(c.packed_consts.begin(), c.packed_consts.end(), G2.w) == c.packed_consts.end()) {
           c.packed_consts.push_back(G2.w);
           c.packed_off.push_back(c.packed_bytes);
+          c.packed_ln.push_back(Compiled::PackedLn());
           const auto& wd = g.tensors[G2.w].S.dims;
           size_t kk = static_cast<size_t>(wd[1].e.const_value() * wd[2].e.const_value() * wd[3].e.const_value());
           kk = (kk + 63) / 64 * 64;   // thin-channel convolutions pad K to a whole k-chunk

@@ -37,7 +37,37 @@ struct GemmEpilogue {
   int* status;                // device word; set non-zero if a bounded wait ran out
   int splits;                 // split-K kernels: number of K ranges per tile (work item = tile x range), else unused
   int stages_per_split;       // split-K kernels: pipeline stages per K range
+  // ---- LayerNorm folded into the GEMM (template parameters LN / EMIT).  Row statistics are (mean, M2) pairs,
+  // M2 = sum of squared deviations from that mean, one pair per row and slot of `ln_cols` consecutive columns;
+  // slot s of row i is at [s * pitch + i], i counted from this launch's first row.
+  const float2* ln_stats;     // LN != 0: statistics of the rows being normalised (A rows for LN = 1, residual rows for LN = 2)
+  long long ln_pitch;
+  int ln_slots, ln_cols;      // slots per row and columns per slot (slots * cols = normalised width)
+  float ln_eps;
+  const float* ln_c1;         // LN = 1: [N] column sums of the gamma-scaled weights
+  const float* ln_c2;         // LN = 1: [N] beta . W + bias (replaces `bias`)
+  const __nv_bfloat16* ln_gamma;  // LN = 2: [N]
+  const __nv_bfloat16* ln_beta;   // LN = 2: [N]
+  float2* emit_stats;         // EMIT: receives the statistics of the stored output rows: slot = 2 * n-tile + column half
+  long long emit_pitch;
 };
+
+// One row's LayerNorm statistics from its partial (mean, M2) pairs, merged in slot order (pairwise update of
+// mean and sum of squared deviations): the same result whichever kernel reads them.
+__device__ __forceinline__ void ln_merge_stats(const float2* st, long long pitch, int slots, int cols, float eps, float* mean_out, float* rstd_out) {
+  float n = 0.f, mean = 0.f, m2 = 0.f;
+  const float c = static_cast<float>(cols);
+  for (int s = 0; s < slots; ++s) {
+    const float2 q = st[s * pitch];
+    const float nn = n + c;
+    const float d = q.x - mean;
+    mean = fmaf(d, c / nn, mean);
+    m2 += q.y + d * d * (n * c / nn);
+    n = nn;
+  }
+  *mean_out = mean;
+  *rstd_out = 1.0f / sqrtf(m2 / n + eps);
+}
 
 constexpr int GEMM_BM = 128;
 constexpr int GEMM_THREADS = 384;
@@ -102,7 +132,14 @@ __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 256;"
 // `range` of an fp32 [ranges, M, N] workspace (tmOut is then a 3-D fp32 map with boxes of 32 columns)
 // and a finishing kernel adds the slabs in a fixed order and applies bias, residual and LayerNorm.
 // This spreads a GEMM with few output tiles and a long K over all SMs, deterministically.
-template <int BN, int KCH, int STAGES, int ACT, bool SPLITK = false, bool RES = false>
+// LN = 1: A is the raw input of a folded LayerNorm and the weights carry its gamma: the epilogue computes
+//   rstd_i * (acc - mean_i * c1[n]) + c2[n]   (= LayerNorm(A) * W + bias) before the activation.
+// LN = 2 (with RES): the staged residual tile holds raw rows; the epilogue adds (r - mean_i) * rstd_i * gamma[n] + beta[n].
+// EMIT: the epilogue also writes the statistics of the rows it stores (of the bf16 values as stored), one
+// (mean, M2) pair per row, n-tile and 32-column-per-pass half; needs N % BN == 0.
+// With LN != 0 the per-column vectors (bias / c2, c1 / gamma, beta) live single-buffered in the 2 KB vector area,
+// guarded by a second barrier of the epilogue warps per tile; LN = 2 needs BN <= 128 to fit three of them.
+template <int BN, int KCH, int STAGES, int ACT, bool SPLITK = false, bool RES = false, int LN = 0, bool EMIT = false>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmRes,
@@ -330,18 +367,52 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         }
       }
     } else {
+    static_assert(LN == 0 || !SPLITK, "folded LayerNorm and split-K do not combine");
+    static_assert(LN != 2 || (RES && BN <= 128), "a normalised residual needs the residual path and three vectors of BN floats");
+    static_assert(LN != 1 || !RES, "a normalised A operand is not combined with a residual");
+    constexpr int NVEC = LN == 1 ? 2 : LN == 2 ? 3 : 1;
     int j = 0, u = 0;
-    auto load_bias = [&](int t) -> float {
+    // column vectors of tile t: v0 = bias (LN = 1: c2), v1 = c1 (LN = 1) or gamma (LN = 2), v2 = beta (LN = 2)
+    auto load_vec = [&](int t, int which) -> float {
       const int idx = (t / tiles_m) * BN + et;
-      return (ep.bias && et < BN && t < num_tiles && idx < N) ? __bfloat162float(ep.bias[idx]) : 0.0f;
+      if (!(et < BN && t < num_tiles && idx < N)) return 0.0f;
+      if (which == 0) {
+        if constexpr (LN == 1) return ep.ln_c2[idx];
+        else return ep.bias ? __bfloat162float(ep.bias[idx]) : 0.0f;
+      }
+      if (which == 1) {
+        if constexpr (LN == 1) return ep.ln_c1[idx];
+        else return __bfloat162float(ep.ln_gamma[idx]);
+      }
+      return __bfloat162float(ep.ln_beta[idx]);
     };
-    float bias_next = load_bias(blockIdx.x);
+    float vec_next[NVEC];
+#pragma unroll
+    for (int w = 0; w < NVEC; ++w) vec_next[w] = load_vec(blockIdx.x, w);
     const float relu2_floor = ep.act2 == ACT_RELU ? 0.0f : -INFINITY;  // post-residual activation, branch-free
     for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++j) {
       const int acc = j & 1;
-      float* bias_t = bias_s + (j & 1) * 256;      // this tile's bias, prefetched during the last tile
-      bias_t[et] = bias_next;
-      bias_next = load_bias(t + gridDim.x);
+      float* bias_t;
+      if constexpr (LN == 0) {
+        bias_t = bias_s + (j & 1) * 256;           // this tile's bias, prefetched during the last tile
+        bias_t[et] = vec_next[0];
+      } else {
+        bias_t = bias_s;                           // single-buffered vectors: every warp has left the previous tile
+        epi_bar_sync();
+        if (et < BN) {
+#pragma unroll
+          for (int w = 0; w < NVEC; ++w) bias_t[w * BN + et] = vec_next[w];
+        }
+      }
+#pragma unroll
+      for (int w = 0; w < NVEC; ++w) vec_next[w] = load_vec(t + gridDim.x, w);
+      // statistics of this thread's row (hidden behind the main loop of the tile)
+      const int grow = (t % tiles_m) * GEMM_BM + row;
+      float ln_mean = 0.f, ln_rstd = 0.f;
+      if constexpr (LN != 0) {
+        if (grow < M) ln_merge_stats(ep.ln_stats + grow, ep.ln_pitch, ep.ln_slots, ep.ln_cols, ep.ln_eps, &ln_mean, &ln_rstd);
+      }
+      float em_n = 0.f, em_mean = 0.f, em_m2 = 0.f;    // EMIT: running statistics of this thread's columns of the row
       // one warp polls for the accumulator, the others park at the hardware barrier: seven more polling
       // lanes cost the main loop 3-4 % of its issue slots
       if (warp == 3) ptx::mbar_wait_warp(&tmem_full[acc], (j >> 1) & 1, dead);
@@ -369,8 +440,14 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         // values that the agent never stores
         const float* bp = bias_t + ps * GEMM_PASS_COLS + half * 32;
         float v[32];
+        if constexpr (LN == 1) {
+          const float nmr = -ln_mean * ln_rstd;    // rstd * (acc - mean * c1) + c2
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = apply_act<ACT>(__uint_as_float(r[ps & 1][i]) + bp[i]);
+          for (int i = 0; i < 32; ++i) v[i] = apply_act<ACT>(fmaf(ln_rstd, __uint_as_float(r[ps & 1][i]), fmaf(nmr, bp[BN + i], bp[i])));
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = apply_act<ACT>(__uint_as_float(r[ps & 1][i]) + bp[i]);
+        }
         uint4 pk[4];
         if constexpr (!RES) {
 #pragma unroll
@@ -393,7 +470,12 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&pk[g]);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              const float2 f = __bfloat1622float2(h[i]);
+              float2 f = __bfloat1622float2(h[i]);
+              if constexpr (LN == 2) {
+                const int cidx = g * 8 + 2 * i;
+                f.x = fmaf(f.x - ln_mean, ln_rstd * bp[BN + cidx], bp[2 * BN + cidx]);
+                f.y = fmaf(f.y - ln_mean, ln_rstd * bp[BN + cidx + 1], bp[2 * BN + cidx + 1]);
+              }
               oh[i] = __floats2bfloat162_rn(fmaxf(v[g * 8 + 2 * i] + f.x, relu2_floor), fmaxf(v[g * 8 + 2 * i + 1] + f.y, relu2_floor));
             }
           }
@@ -403,6 +485,35 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         ptx::fence_proxy_async();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&buf_filled[bsel]);
+        if constexpr (EMIT) {
+          // statistics of the 32 values just stored (as rounded to bf16), merged into the row's running pair
+          float xs[32];
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            const __nv_bfloat162* oh = reinterpret_cast<const __nv_bfloat162*>(&pk[g]);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float2 f = __bfloat1622float2(oh[i]);
+              xs[g * 8 + 2 * i] = f.x;
+              xs[g * 8 + 2 * i + 1] = f.y;
+            }
+          }
+          float sum = 0.f;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) sum += xs[i];
+          const float mb = sum * (1.0f / 32.0f);
+          float qb = 0.f;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) { const float d = xs[i] - mb; qb = fmaf(d, d, qb); }
+          const float nn = em_n + 32.0f;
+          const float d = mb - em_mean;
+          em_mean = fmaf(d, 32.0f / nn, em_mean);
+          em_m2 += qb + d * d * (em_n * 32.0f / nn);
+          em_n = nn;
+        }
+      }
+      if constexpr (EMIT) {
+        if (grow < M) ep.emit_stats[(static_cast<long long>(t / tiles_m) * 2 + half) * ep.emit_pitch + grow] = make_float2(em_mean, em_m2);
       }
     }
     }

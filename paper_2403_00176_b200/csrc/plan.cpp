@@ -163,6 +163,16 @@ struct Planner {
       if (per_request) off += (bytes + 15) & ~int64_t(15);
       else off = bytes;
     }
+    if (t < static_cast<int>(c.stats_width.size()) && c.stats_width[t] > 0) {
+      // LayerNorm row statistics written by the producing GEMM live behind the tensor's instances: one
+      // (mean, M2) float pair per packed row and slot of 32 columns (the most any tile version writes)
+      const int64_t row_bytes = static_cast<int64_t>(c.stats_width[t]) * esz;
+      if (!per_request || off % row_bytes) return fail(E_INTERNAL, "row statistics need densely packed rows: " + T.name);
+      R.stats_rows = off / row_bytes;
+      R.stats_slots = c.stats_width[t] / 32;
+      R.stats_off = off;
+      off += R.stats_rows * R.stats_slots * 8;
+    }
     R.bytes = off;
     if (T.kind == TKind::INPUT) { R.where = RootBuf::INPUT; R.io_index = T.io_index; }
     else if (T.kind == TKind::CONST) { R.where = RootBuf::CONST; }
@@ -279,18 +289,30 @@ struct Planner {
     for (int t : g.outputs) { Status s = resolve(t); if (s != OK) return s; }
     static const bool prof = getenv("SOD2_HOST_PROFILE") != nullptr;
     auto t1 = std::chrono::steady_clock::now();
+    // GEMM groups that will run as one persistent kernel: their members overlap in time
+    {
+      Status cs = detect_chains(&p);
+      if (cs != OK) return cs;
+    }
     // liveness of arena roots over the group sequence
     int steps = static_cast<int>(c.groups.size());
     for (int s = 0; s < steps; ++s) {
       const Group& G = c.groups[s];
+      // a member of a chain reads and writes at any time between the chain's first and last step
+      int lo = s, hi = s;
+      if (s < static_cast<int>(p.chain_of.size()) && p.chain_of[s] >= 0) {
+        const Plan::Chain& ch = p.chains[p.chain_of[s]];
+        lo = ch.groups.front();
+        hi = ch.groups.back();
+      }
       auto touch = [&](int t, bool def) {
         if (c.storage[t].kind == Storage::FOLDED || !resolved[t]) return;
         int root = p.views[t][0].root;
         if (root < 0) return;
         RootBuf& R = p.roots[root];
-        if (def && R.def_step < 0) R.def_step = s;
-        R.last_step = std::max(R.last_step, s);
-        if (R.def_step < 0) R.def_step = s;
+        if (R.def_step < 0 || lo < R.def_step) R.def_step = lo;
+        R.last_step = std::max(R.last_step, hi);
+        (void)def;
       };
       for (int t : G.ext_out) touch(t, true);
       for (int t : G.ext_in) touch(t, false);
@@ -311,7 +333,10 @@ struct Planner {
   // device status word.
   Status plan_arena(int steps) {
     // header: status word (256 B) + one 8-byte count slot per (runtime symbol, request)
-    const size_t HEADER = (256 + 8 * g.cx.atoms.size() * static_cast<size_t>(p.n_req) + 255) & ~size_t(255);
+    // ... + the row-block counters of the GEMM chains
+    p.chain_counter_off = (256 + 8 * g.cx.atoms.size() * static_cast<size_t>(p.n_req) + 15) & ~size_t(15);
+    const size_t HEADER = (p.chain_counter_off + 4 * p.chain_counter_words + 255) & ~size_t(255);
+    p.header_clear_bytes = p.chain_counter_words ? HEADER : 256;
     std::vector<int> ids;
     for (size_t t = 0; t < p.roots.size(); ++t)
       if (p.roots[t].where == RootBuf::ARENA && p.roots[t].def_step >= 0) ids.push_back(static_cast<int>(t));

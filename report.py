@@ -79,14 +79,14 @@ def _units(cfg, reqs):
     return reqs[0].inputs["x"].shape[0], "images"
 
 
-def measure(cfg: int, reps: int, device: str = "cuda:0"):
+def measure(cfg: int, reps: int, device: str = "cuda:0", opt_flags: int = 0):
     import torch
     from paper_2403_00176_b200 import workloads as WL
     from paper_2403_00176_b200.session import Session
 
     hbm, tf, src = _peaks()
     wl = {1: WL.cfg1, 2: WL.cfg2, 3: WL.cfg3, 4: WL.cfg4, 5: WL.cfg5}[cfg]()
-    sess = Session(wl, device=device)
+    sess = Session(wl, device=device, opt_flags=opt_flags)
     n_batches = 3 if cfg in (4, 5) else 5
     preps = [sess.prepare(wl.batch(j)) for j in range(n_batches)]
     dev = sess.dev
@@ -215,10 +215,11 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="1,2,3,4,5")
     ap.add_argument("--reps", type=int, default=30)
+    ap.add_argument("--opt-flags", type=int, default=0, help="SOD2_OPT_* bits for sod2_graph_create (A/B measurements)")
     a = ap.parse_args()
     rows = []
     for c in [int(x) for x in a.configs.split(",")]:
-        r = measure(c, a.reps)
+        r = measure(c, a.reps, opt_flags=a.opt_flags)
         print(json.dumps(r), flush=True)
         rows.append(r)
     print("\n| cfg | ms per inference (median, min) | as one CUDA graph (median, min) | ms per request | sum t_roof / t_step | worst group: fraction, bound | bind+plan us (cache hit) | arena / peak-live MB |")

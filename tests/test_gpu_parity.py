@@ -114,6 +114,89 @@ def test_cfg2_small_encoder_edge_lengths_lockstep():
         assert not bad, (req.syms, bad)
 
 
+def test_cfg2_small_encoder_layernorm_fold_against_unfolded():
+    # Opt-in: a LayerNorm between two GEMMs is folded into them (the producer writes row statistics, the
+    # consumers normalise in their epilogues, the normalised tensor is never stored).  Without the flag the
+    # LayerNorm kernel runs: both forms meet the oracle group by group, and each other end to end.
+    wl, reqs = _encoder_edge()
+    s0, p0, o0 = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE)
+    s1, p1, o1 = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE | B.OPT_LN_FOLD)
+    k0 = [s0.graph.group_info(i)["kind"] for i in range(s0.graph.num_groups())]
+    k1 = [s1.graph.group_info(i)["kind"] for i in range(s1.graph.num_groups())]
+    assert k0.count("layernorm") == 4 and k1.count("layernorm") == 1
+    for r, req in enumerate(reqs):
+        errs = lockstep(wl, s1, p1, o1, r, BF16_TOL)
+        bad = {k: v for k, v in errs.items() if not (isinstance(v, float) and v <= BF16_TOL)}
+        assert errs and not bad, (req.syms, bad)
+        assert O.rel_err(o1[r]["y"], o0[r]["y"]) <= BF16_TOL, req.syms
+    # deterministic: the folded form gives the same bits when run again
+    _, _, o2 = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE | B.OPT_LN_FOLD)
+    for a, b in zip(o1, o2):
+        assert np.array_equal(a["y"], b["y"])
+
+
+def test_layernorm_fold_with_affine_parameters_and_offset_rows():
+    # gamma, beta away from (1, 0) and rows whose mean is several standard deviations from zero: the folded
+    # form subtracts mean * column-sum from the product of the raw rows, so this is where it would lose bits
+    wl = WL.cfg2(layers=2, D=128, H=2, F=256, n_requests=1, lmin=1, lmax=512)
+    rng = np.random.default_rng(23)
+    consts = dict(wl.consts)
+    n_affine = 0
+    for name in list(consts):
+        base = name.split(".")[-1]
+        if base.startswith("g_"):
+            consts[name] = bf16_round(rng.uniform(0.5, 1.5, consts[name].shape).astype(np.float32))
+            n_affine += 1
+        if base.startswith("be_"):
+            consts[name] = bf16_round(rng.normal(0, 0.3, consts[name].shape).astype(np.float32))
+    assert n_affine == 4
+    wl2 = WL.Workload(wl.name, wl.dtype, wl.ir, consts, wl.sym_names, wl.outputs, wl.meta)
+    reqs = [Request({"L": L}, {"x": bf16_round((rng.standard_normal((1, L, 128)) + 3.0).astype(np.float32))}) for L in (1, 77, 130, 300)]
+    s, p, outs = run_batch(wl2, reqs, opt_flags=B.OPT_NO_REUSE | B.OPT_LN_FOLD)
+    assert [s.graph.group_info(i)["kind"] for i in range(s.graph.num_groups())].count("layernorm") == 1
+    for r, req in enumerate(reqs):
+        # end to end the bound is the storage noise of the two layers (as in the full-size test below); the
+        # per-group bound, in lock-step, is the strict one
+        ref = O.run(wl2.ir, wl2.consts, req.inputs)["y"]
+        noisy = O.run(wl2.ir, wl2.consts, req.inputs, storage_round=lambda a: bf16_round(a.astype(np.float32)).astype(np.float64))["y"]
+        assert O.rel_err(outs[r]["y"], ref) <= max(BF16_TOL, 2 * O.rel_err(noisy, ref))
+        errs = lockstep(wl2, s, p, outs, r, BF16_TOL)
+        bad = {k: v for k, v in errs.items() if not (isinstance(v, float) and v <= BF16_TOL)}
+        assert errs and not bad, (req.syms, bad)
+
+
+def test_gemm_chain_kernel_against_one_launch_per_gemm():
+    # Opt-in: consecutive dependent GEMM groups (projection -> FFN1 -> FFN2 -> next layer's QKV, LayerNorm folded)
+    # run as one persistent kernel with row-block dependency counters.  Against one launch per GEMM: fewer
+    # launches, the same results within the tolerance, each form in lock-step with the oracle; run twice for
+    # determinism (the counters are cleared by every run).
+    wl, reqs = _encoder_edge(layers=3)
+    s0, p0, o0 = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE)
+    s1, p1, o1 = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE | B.OPT_LN_FOLD | B.OPT_GEMM_CHAIN)
+    assert p1.run().gpu_launches < p0.run().gpu_launches
+    p1.check_device_status()
+    o1b = p1.outputs()
+    for r, req in enumerate(reqs):
+        assert np.array_equal(o1[r]["y"], o1b[r]["y"])
+        assert O.rel_err(o1[r]["y"], o0[r]["y"]) <= BF16_TOL, req.syms
+        for s_, p_, o_ in ((s0, p0, o0), (s1, p1, o1)):
+            errs = lockstep(wl, s_, p_, o_, r, BF16_TOL)
+            bad = {k: v for k, v in errs.items() if not (isinstance(v, float) and v <= BF16_TOL)}
+            assert errs and not bad, (req.syms, bad)
+    # a batch of several requests (several row blocks, ragged last block), with arena reuse on
+    wl2 = WL.cfg2(layers=2, D=128, H=2, F=256, n_requests=6, lmin=1, lmax=300)
+    reqs2 = wl2.batch(3)
+    _, _, a = run_batch(wl2, reqs2)
+    _, _, b = run_batch(wl2, reqs2, opt_flags=B.OPT_LN_FOLD | B.OPT_GEMM_CHAIN)
+    # without the fold only FFN1 -> FFN2 chain (a LayerNorm kernel sits between the others)
+    _, pc, cc = run_batch(wl2, reqs2, opt_flags=B.OPT_GEMM_CHAIN)
+    for r in range(len(reqs2)):
+        assert O.rel_err(cc[r]["y"], a[r]["y"]) <= BF16_TOL
+    for r, req in enumerate(reqs2):
+        ref = _oracle_out(wl2, req, "y")
+        assert O.rel_err(b[r]["y"], ref) <= BF16_TOL and O.rel_err(a[r]["y"], ref) <= BF16_TOL
+
+
 def test_cfg2_small_encoder_splitk_layernorm_groups_lockstep():
     # opt-in form of the residual GEMM + LayerNorm pair: split-K GEMM into fp32 slabs + finishing kernel
     # (F = 1024 gives the second GEMM 16 pipeline stages, i.e. several K ranges per tile)

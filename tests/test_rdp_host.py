@@ -84,6 +84,11 @@ def test_expected_smaps_per_config():
     assert "[1,L,2304]" in shapes.values() and "[1,L,3072]" in shapes.values() and shapes["y"] == "[1,L,768]"
     kinds = [g.group_info(i)["kind"] for i in range(g.num_groups())]
     assert kinds == ["gemm", "attention", "gemm", "layernorm", "gemm", "gemm", "layernorm"]
+    # opt-in: the LayerNorm between the attention projection and the FFN is folded into the GEMMs around it (the
+    # last one produces the graph output and stays); every operator still belongs to some group
+    gf = B.Graph(wl.ir, B.OPT_LN_FOLD)
+    assert [gf.group_info(i)["kind"] for i in range(gf.num_groups())] == ["gemm", "attention", "gemm", "gemm", "gemm", "layernorm"]
+    assert sum(gf.group_info(i)["n_ops"] for i in range(6)) == sum(g.group_info(i)["n_ops"] for i in range(7))
     # opt-in: the two residual GEMMs of a post-LN layer absorb their LayerNorm (split-K GEMM + finishing kernel)
     g2 = B.Graph(wl.ir, B.OPT_SPLITK_LN)
     kinds2 = [g2.group_info(i)["kind"] for i in range(g2.num_groups())]
