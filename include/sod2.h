@@ -130,6 +130,14 @@ sod2_status sod2_run_graph(sod2_plan_t* p, const void* const* inputs, void* cons
 sod2_status sod2_run_timed(sod2_plan_t* p, const void* const* inputs, void* const* outputs, void* arena,
                            size_t arena_bytes, void* cuda_stream, float* group_ms, int n_groups);
 
+/* The same with every launch issued `reps` times back to back between its two events, the time divided by
+ * reps: a kernel's duration as it is inside a busy stream, without the idle gap that follows an event when
+ * a lone launch has to travel from the host.  The repeated launches recompute the same values (results of
+ * groups that update a tensor in place, the gated convolutions, are not meaningful afterwards): a measuring
+ * aid for the encoder workloads. */
+sod2_status sod2_run_timed_repeat(sod2_plan_t* p, const void* const* inputs, void* const* outputs, void* arena,
+                                  size_t arena_bytes, void* cuda_stream, int reps, float* group_ms, int n_groups);
+
 /* Reads the device status word written by the last run (synchronises the stream).
  * SOD2_OK, or SOD2_E_TIMEOUT if a kernel gave up on a bounded wait. */
 sod2_status sod2_plan_device_status(sod2_plan_t* p, const void* arena, void* cuda_stream);
@@ -218,6 +226,14 @@ sod2_status sod2_nonzero_static(const void* dev_x, int dtype, int rank, const in
  * so their time is reported as a multiple of it rather than as a fraction of a roofline.
  * Asynchronous.  Errors: SOD2_E_CUDA; message through sod2_last_error(NULL). */
 sod2_status sod2_launch_empty(void* cuda_stream);
+
+/* Self-test of the bounded waits (Section 4: deterministic sequence of operations; a wait that cannot complete
+ * must end, not hang the device).  Launches one small kernel on cuda_stream that waits, with the library's
+ * bounded wait and a limit of 4096 polls, on a barrier nothing arrives on; the wait runs out, the kernel writes 1
+ * to the device word dev_status_word (the first word of an arena: what sod2_plan_device_status reads) and returns by
+ * itself.  Nothing traps and nothing waits without a limit.  Asynchronous.  Errors: SOD2_E_INVALID_ARG,
+ * SOD2_E_CUDA; message through sod2_last_error(NULL). */
+sod2_status sod2_selftest_bounded_wait(void* dev_status_word, void* cuda_stream);
 
 /* handle may be a graph, binding or plan; returns "" if there was no error. */
 const char* sod2_last_error(const void* any_handle);

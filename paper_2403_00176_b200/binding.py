@@ -58,6 +58,7 @@ def _load() -> C.CDLL:
         "sod2_run": [vp, P(vp), P(vp), vp, sz, vp, P(RunInfo)],
         "sod2_run_graph": [vp, P(vp), P(vp), vp, sz, vp, P(RunInfo)],
         "sod2_run_timed": [vp, P(vp), P(vp), vp, sz, vp, P(C.c_float), i32],
+        "sod2_run_timed_repeat": [vp, P(vp), P(vp), vp, sz, vp, i32, P(C.c_float), i32],
         "sod2_plan_device_status": [vp, vp, vp],
         "sod2_graph_tensor_info": [vp, cp, P(i32), P(i32), cp, sz],
         "sod2_graph_tensor_value": [vp, cp, cp, sz],
@@ -76,6 +77,7 @@ def _load() -> C.CDLL:
         "sod2_run_output_shape": [vp, vp, vp, i32, i32, P(i64), P(i32)],
         "sod2_nonzero_static": [vp, i32, i32, P(i64), vp, vp, vp],
         "sod2_launch_empty": [vp],
+        "sod2_selftest_bounded_wait": [vp, vp],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -95,11 +97,11 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = ["sod2_graph_create", "sod2_graph_destroy", "sod2_graph_set_const", "sod2_graph_prepack_bytes",
            "sod2_graph_prepack", "sod2_bind_dims", "sod2_binding_destroy", "sod2_plan", "sod2_plan_destroy", "sod2_graph_set_plan_cache", "sod2_plan_cached",
-           "sod2_run", "sod2_run_graph", "sod2_run_timed", "sod2_plan_device_status", "sod2_graph_tensor_info", "sod2_graph_tensor_value", "sod2_graph_tensor_dtype",
+           "sod2_run", "sod2_run_graph", "sod2_run_timed", "sod2_run_timed_repeat", "sod2_plan_device_status", "sod2_graph_tensor_info", "sod2_graph_tensor_value", "sod2_graph_tensor_dtype",
            "sod2_graph_num_ops", "sod2_graph_op_info", "sod2_graph_num_groups", "sod2_graph_group_info",
            "sod2_graph_num_subgraphs", "sod2_graph_rdp_sweeps", "sod2_classify", "sod2_graph_reanalyse", "sod2_graph_order_info",
            "sod2_binding_shape", "sod2_plan_slot", "sod2_plan_instance_offset", "sod2_plan_memory", "sod2_plan_group_cost", "sod2_plan_tensor_strides",
-           "sod2_run_output_shape", "sod2_nonzero_static", "sod2_launch_empty", "sod2_last_error"]
+           "sod2_run_output_shape", "sod2_nonzero_static", "sod2_launch_empty", "sod2_selftest_bounded_wait", "sod2_last_error"]
 
 
 def _check(status: int, handle=None):
@@ -120,6 +122,11 @@ NONZERO_STATIC_MAX_ELEMS = 16777216
 def sod2_launch_empty(stream: int) -> None:
     """One kernel that does nothing, on `stream`: the yardstick for launch-bound groups."""
     _check(lib.sod2_launch_empty(C.c_void_p(stream)))
+
+
+def sod2_selftest_bounded_wait(dev_status_word: int, stream: int) -> None:
+    """Launches the kernel whose bounded wait runs out: it sets the device status word and returns by itself."""
+    _check(lib.sod2_selftest_bounded_wait(C.c_void_p(dev_status_word), C.c_void_p(stream)))
 
 
 def sod2_nonzero_static(dev_x: int, dtype: int, dims: Sequence[int], dev_out: int, dev_count: int, stream: int) -> None:
@@ -298,12 +305,16 @@ class Plan:
         _check(lib.sod2_run_graph(self.h, ins, outs, C.c_void_p(arena), arena_bytes, C.c_void_p(stream), C.byref(info)), self.h)
         return info
 
-    def run_timed(self, inputs: Sequence[int], outputs: Sequence[int], arena: int, arena_bytes: int, stream: int) -> List[float]:
+    def run_timed(self, inputs: Sequence[int], outputs: Sequence[int], arena: int, arena_bytes: int, stream: int, reps: int = 1) -> List[float]:
+        """Device time per fused group (ms).  reps > 1: every launch repeated back to back, time divided by reps."""
         ins = (C.c_void_p * max(len(inputs), 1))(*inputs)
         outs = (C.c_void_p * max(len(outputs), 1))(*outputs)
         n = self.graph.num_groups()
         ms = (C.c_float * max(n, 1))()
-        _check(lib.sod2_run_timed(self.h, ins, outs, C.c_void_p(arena), arena_bytes, C.c_void_p(stream), ms, n), self.h)
+        if reps > 1:
+            _check(lib.sod2_run_timed_repeat(self.h, ins, outs, C.c_void_p(arena), arena_bytes, C.c_void_p(stream), reps, ms, n), self.h)
+        else:
+            _check(lib.sod2_run_timed(self.h, ins, outs, C.c_void_p(arena), arena_bytes, C.c_void_p(stream), ms, n), self.h)
         return list(ms[:n])
 
     def device_status(self, arena: int, stream: int):

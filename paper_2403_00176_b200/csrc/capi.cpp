@@ -248,6 +248,14 @@ sod2_status sod2_run_timed(sod2_plan_t* p, const void* const* inputs, void* cons
   return st(s);
 }
 
+sod2_status sod2_run_timed_repeat(sod2_plan_t* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes,
+                                  void* stream, int reps, float* group_ms, int n_groups) {
+  if (!p || !inputs || !outputs || !arena) return SOD2_E_INVALID_ARG;
+  Status s = run_plan_timed(&p->p, inputs, outputs, arena, arena_bytes, stream, group_ms, n_groups, reps);
+  if (s != OK) p->h.err = p->p.err;
+  return st(s);
+}
+
 sod2_status sod2_plan_device_status(sod2_plan_t* p, const void* arena, void* stream) {
   if (!p || !arena) return SOD2_E_INVALID_ARG;
   int word = 0;

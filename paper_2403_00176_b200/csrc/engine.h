@@ -300,7 +300,10 @@ Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* 
 
 // Same as run_plan, with CUDA events around every launch; synchronises the stream and returns the
 // device time per group (ms).
+// reps > 1: every launch is issued `reps` times back to back between its two events and the time divided by reps
+// (the kernel's duration without the idle gap between an event and a lone launch); only meaningful where a
+// launch may be repeated without changing its inputs.
 Status run_plan_timed(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream,
-                      float* group_ms, int n_groups);
+                      float* group_ms, int n_groups, int reps = 1);
 
 }  // namespace sod2

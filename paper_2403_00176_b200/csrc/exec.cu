@@ -1932,7 +1932,8 @@ Status prepack_weights(Compiled* c, void* workspace, size_t bytes, void* stream)
 }
 
 Status run_plan_timed(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream,
-                      float* group_ms, int n_groups) {
+                      float* group_ms, int n_groups, int reps) {
+  if (reps < 1) { p->err = "reps must be at least 1"; return E_INVALID_ARG; }
   if (!group_ms || n_groups != static_cast<int>(p->c->groups.size())) { p->err = "group_ms must hold one float per group"; return E_INVALID_ARG; }
   if (arena_bytes < p->arena_bytes) { p->err = "arena too small"; return E_ARENA_TOO_SMALL; }
   if (reinterpret_cast<uintptr_t>(arena) & 255) { p->err = "arena must be 256-byte aligned"; return E_MISALIGNED; }
@@ -1944,7 +1945,8 @@ Status run_plan_timed(Plan* p, const void* const* inputs, void* const* outputs, 
   Status st = OK;
   for (size_t i = 0; i < n && st == OK; ++i) {
     cudaEventRecord(ev[2 * i], x.stream);
-    if (p->launches[i]->fn(x) != cudaSuccess) { p->err = "launch failed"; st = E_CUDA; }
+    for (int r = 0; r < reps && st == OK; ++r)
+      if (p->launches[i]->fn(x) != cudaSuccess) { p->err = "launch failed"; st = E_CUDA; }
     cudaEventRecord(ev[2 * i + 1], x.stream);
   }
   if (cudaStreamSynchronize(x.stream) != cudaSuccess) { p->err = "stream synchronize failed"; st = E_CUDA; }
@@ -1953,6 +1955,7 @@ Status run_plan_timed(Plan* p, const void* const* inputs, void* const* outputs, 
     for (size_t i = 0; i < n; ++i) {
       float ms = 0.f;
       cudaEventElapsedTime(&ms, ev[2 * i], ev[2 * i + 1]);
+      ms /= static_cast<float>(reps);
       if (p->launches[i]->share.empty()) group_ms[p->launches[i]->group] += ms;
       else for (auto& sh : p->launches[i]->share) group_ms[sh.first] += ms * static_cast<float>(sh.second);   // a chain: by algorithmic flops
     }

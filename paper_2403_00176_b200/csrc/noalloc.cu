@@ -17,6 +17,7 @@
 //    make that first call outside of any stream capture.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include "ptx.cuh"
 
 #include <cstdint>
 #include <string>
@@ -177,7 +178,32 @@ extern "C" sod2_status sod2_nonzero_static(const void* dev_x, int dtype, int ran
 
 namespace {
 __global__ void empty_kernel() {}
+
+// One warp waits, with the library's bounded wait and a limit of a few thousand polls, on a barrier that
+// nothing ever arrives on; the wait runs out, raises the CTA's flag and the kernel records it in the status
+// word exactly as the tensor-core kernels do, then returns.
+__global__ void bounded_wait_selftest(int* status) {
+  __shared__ uint64_t bar;
+  __shared__ int dead;
+  if (threadIdx.x == 0) {
+    dead = 0;
+    sod2::ptx::mbar_init(&bar, 1);
+    sod2::ptx::fence_barrier_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) sod2::ptx::mbar_wait_limited(&bar, 0, &dead, 4096u);
+  __syncthreads();
+  if (threadIdx.x == 0 && dead && status) atomicExch(status, 1);
+}
 }  // namespace
+
+extern "C" sod2_status sod2_selftest_bounded_wait(void* dev_status_word, void* cuda_stream) {
+  if (!dev_status_word) return nzs_fail(SOD2_E_INVALID_ARG, "sod2_selftest_bounded_wait: null status word");
+  bounded_wait_selftest<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(static_cast<int*>(dev_status_word));
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return nzs_fail(SOD2_E_CUDA, std::string("sod2_selftest_bounded_wait: launch failed: ") + cudaGetErrorString(e));
+  return SOD2_OK;
+}
 
 extern "C" sod2_status sod2_launch_empty(void* cuda_stream) {
   empty_kernel<<<1, 1, 0, static_cast<cudaStream_t>(cuda_stream)>>>();

@@ -70,13 +70,16 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait. `dead` is a CTA-shared flag: once set, every wait returns at once.  Polls with
 // test_wait: measured on B200, a try_wait on a barrier whose phase has already completed takes about
 // 200 cycles, a test_wait about 65, and these waits sit on the critical path of the MMA issue loops.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* dead) {
-  for (uint32_t i = 0; i < SOD2_SPIN_LIMIT; ++i) {
+__device__ __forceinline__ bool mbar_wait_limited(uint64_t* bar, uint32_t parity, volatile int* dead, uint32_t limit) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_test_wait(bar, parity)) return true;
     if ((i & 1023u) == 1023u && *dead) return false;
   }
   *dead = 1;
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* dead) {
+  return mbar_wait_limited(bar, parity, dead, SOD2_SPIN_LIMIT);
 }
 
 // The same wait for a whole warp: lane 0 polls, the others join at the warp barrier (32 lanes polling

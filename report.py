@@ -21,18 +21,19 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
-def group_times(prep, reps: int = 5) -> List[float]:
-    """Median device time (ms) of every fused group over `reps` timed inferences."""
+def group_times(prep, reps: int = 5, repeat: int = 1) -> List[float]:
+    """Median device time (ms) of every fused group over `reps` timed inferences.  repeat > 1: every launch issued
+    `repeat` times back to back between its events (duration inside a busy stream, see sod2_run_timed_repeat)."""
     ins = [t.data_ptr() for t in prep.in_dev]
     outs = [t.data_ptr() for t in prep.out_dev]
-    runs = [prep.plan.run_timed(ins, outs, prep.arena.data_ptr(), prep.arena.numel(), prep.s.stream) for _ in range(reps)]
+    runs = [prep.plan.run_timed(ins, outs, prep.arena.data_ptr(), prep.arena.numel(), prep.s.stream, repeat) for _ in range(reps)]
     return [float(np.median([r[g] for r in runs])) for g in range(len(runs[0]))]
 
 
-def group_report(prep, hbm_gbs: float, tensor_tflops: float, reps: int = 5) -> List[Dict]:
+def group_report(prep, hbm_gbs: float, tensor_tflops: float, reps: int = 5, repeat: int = 1) -> List[Dict]:
     """Per group: kind, ms, algorithmic flops / bytes, roofline time and fraction."""
     g = prep.s.graph
-    ms = group_times(prep, reps)
+    ms = group_times(prep, reps, repeat)
     out = []
     for gi in range(g.num_groups()):
         info = g.group_info(gi)
