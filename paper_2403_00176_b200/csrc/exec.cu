@@ -834,68 +834,148 @@ struct Builder {
   }
 
   // ------------------------------------------------------------------------------ generic chain
-  void fill_operand(k::ChainOperand* o, int t, int r, const std::vector<int64_t>& odims) {
-    const Tensor& T = g.tensors[t];
-    std::memset(o, 0, sizeof(*o));
-    if (T.kind == TKind::FCONST) { o->ptr = nullptr; o->scalar = static_cast<float>(T.fdata); return; }
-    const View& v = p.views[t][T.kind == TKind::CONST ? 0 : r];
-    o->is_bf16 = T.dtype == DType::BF16;
-    const int rk = static_cast<int>(v.dims.size());
-    for (int i = 0; i < 4; ++i) {
-      int src = i - (4 - rk);
-      o->stride[i] = (src >= 0 && v.dims[src] != 1) ? v.strides[src] : 0;  // broadcast dims read in place
-    }
-    (void)odims;
-  }
+  // The requests of a batch go through one launch (a request table of up to CHAIN_MAX_REQ entries; a new launch
+  // starts when the table is full or a request's operand lies in another buffer than the table's).
   Status build_chain(int gi, const Group& G, bool ln_only = false) {
     const Tensor& O = g.tensors[G.out];
     if (O.S.rank > 4) return fail(E_UNSUPPORTED_OP, "chain kernel supports rank <= 4");
-    for (int r = 0; r < p.n_req; ++r) {
-      const View& ov = p.views[G.out][r];
-      if (!ov.contiguous()) return fail(E_UNSUPPORTED_OP, "chain output must be contiguous");
-      k::ChainParams cp{};
-      std::vector<int64_t> od(4, 1);
-      for (size_t i = 0; i < ov.dims.size(); ++i) od[4 - ov.dims.size() + i] = ov.dims[i];
-      for (int i = 0; i < 4; ++i) cp.dim[i] = od[i];
-      if (numel(ov.dims) == 0) continue;
-      fill_operand(&cp.in0, G.a, r, od);
-      cp.n_ops = ln_only ? 0 : static_cast<int>(G.chain_ops.size());
-      std::vector<Ptr> optr(k::CHAIN_MAX_OPS);
-      std::vector<char> has(k::CHAIN_MAX_OPS, 0);
-      for (int i = 0; i < cp.n_ops; ++i) {
-        cp.op[i] = G.chain_ops[i];
-        int t = G.chain_operands[i];
-        if (t >= 0) {
-          fill_operand(&cp.operand[i], t, r, od);
-          if (g.tensors[t].kind != TKind::FCONST) { optr[i] = ptr_of(t, g.tensors[t].kind == TKind::CONST ? 0 : r); has[i] = 1; }
-        }
+    const int n_ops = ln_only ? 0 : static_cast<int>(G.chain_ops.size());
+    const int red = ln_only ? 2 : G.red;
+    // operand k: 0 = in0, 1 + i = operand of operator i (absent for unary operators)
+    std::vector<int> opnd(1 + k::CHAIN_MAX_OPS, -1);
+    opnd[0] = G.a;
+    for (int i = 0; i < n_ops; ++i) opnd[1 + i] = G.chain_operands[i];
+    k::ChainBatch proto{};
+    proto.n_ops = n_ops;
+    for (int i = 0; i < n_ops; ++i) proto.op[i] = G.chain_ops[i];
+    proto.out_bf16 = O.dtype == DType::BF16;
+    proto.red = red;
+    proto.eps = G.eps;
+    proto.gb_bf16 = red == 2 ? g.tensors[G.gamma].dtype == DType::BF16 : 0;
+    for (int kx = 0; kx <= k::CHAIN_MAX_OPS; ++kx)
+      if (opnd[kx] >= 0) {
+        const Tensor& T = g.tensors[opnd[kx]];
+        proto.is_bf16[kx] = T.dtype == DType::BF16;
+        if (T.kind == TKind::FCONST) proto.scalar[kx] = static_cast<float>(T.fdata);
       }
-      cp.out_bf16 = O.dtype == DType::BF16;
-      cp.red = ln_only ? 2 : G.red;
-      cp.eps = G.eps;
-      Ptr pin = ptr_of(G.a, r), pout = ptr_of(G.out, r);
-      Ptr pg = cp.red == 2 ? ptr_of(G.gamma, 0) : Ptr(), pb = cp.red == 2 ? ptr_of(G.beta, 0) : Ptr();
-      cp.gb_bf16 = cp.red == 2 ? g.tensors[G.gamma].dtype == DType::BF16 : 0;
-      const int red = cp.red;
-      if (red && cp.dim[3] * 4 > 200 * 1024) return fail(E_UNSUPPORTED_OP, "row too long for the row-reduction kernel");
+    Ptr pg = red == 2 ? ptr_of(G.gamma, 0) : Ptr(), pb = red == 2 ? ptr_of(G.beta, 0) : Ptr();
+    // operands read through a pointer (the launch closures outlive this builder: they capture plain values only)
+    std::vector<char> has_ptr(1 + k::CHAIN_MAX_OPS, 0);
+    for (int kx = 0; kx <= k::CHAIN_MAX_OPS; ++kx) has_ptr[kx] = opnd[kx] >= 0 && g.tensors[opnd[kx]].kind != TKind::FCONST;
+    struct Pending {
+      k::ChainBatch cb;
+      std::vector<Ptr> base;      // per operand: pointer of the table's first request
+      Ptr out;
+      bool vec = true;            // every request qualifies for the 8-wide kernel
+      bool vec16 = true;          // ... and has a last extent that is a multiple of 16
+      int max_cols = 0;
+    };
+    auto fresh = [&]() { Pending q; q.cb = proto; q.base.assign(1 + k::CHAIN_MAX_OPS, Ptr()); return q; };
+    Pending cur = fresh();
+    auto flush = [&]() {
+      if (!cur.cb.n_req) return;
+      Pending q = cur;
+      cur = fresh();
       add(gi, 1, [=](const RunCtx& x) mutable {
-        cp.in0.ptr = x.resolve(pin);
-        for (int i = 0; i < cp.n_ops; ++i) if (has[i]) cp.operand[i].ptr = x.resolve(optr[i]);
-        cp.out = x.resolve(pout);
-        if (red == 2) { cp.gamma = x.resolve(pg); cp.beta = x.resolve(pb); }
+        k::ChainBatch& cb = q.cb;
+        for (int kx = 0; kx <= k::CHAIN_MAX_OPS; ++kx)
+          cb.base[kx] = has_ptr[kx] ? x.resolve(q.base[kx]) : nullptr;
+        cb.out = x.resolve(q.out);
+        if (red == 2) { cb.gamma = x.resolve(pg); cb.beta = x.resolve(pb); }
         if (!red) {
-          const long long total = cp.dim[0] * cp.dim[1] * cp.dim[2] * cp.dim[3];
-          const unsigned grid = static_cast<unsigned>(std::min<long long>((total + 255) / 256, 148 * 16));
-          k::chain_elementwise<<<grid, 256, 0, x.stream>>>(cp);
+          const unsigned grid = static_cast<unsigned>(std::max<long long>(1, std::min<long long>((cb.total + 255) / 256, 148 * 32)));
+          if (q.vec && q.vec16) {
+            // two vectors per item: the table was filled in units of 8 elements
+            for (int i = 0; i < cb.n_req; ++i) cb.r[i].first /= 2;
+            cb.total /= 2;
+            const unsigned g16 = static_cast<unsigned>(std::max<long long>(1, std::min<long long>((cb.total + 255) / 256, 148 * 32)));
+            k::chain_elementwise_vec<2><<<g16, 256, 0, x.stream>>>(cb);
+            for (int i = 0; i < cb.n_req; ++i) cb.r[i].first *= 2;
+            cb.total *= 2;
+          } else if (q.vec) k::chain_elementwise_vec<1><<<grid, 256, 0, x.stream>>>(cb);
+          else k::chain_elementwise<<<grid, 256, 0, x.stream>>>(cb);
+        } else if (q.max_cols <= k::ROWRED_WARP_COLS) {
+          const size_t smem = static_cast<size_t>(q.max_cols) * 4 * 8;
+          if (smem > 48 * 1024) { static bool once = (cudaFuncSetAttribute(k::chain_rowreduce_warp, cudaFuncAttributeMaxDynamicSharedMemorySize, k::ROWRED_WARP_COLS * 32), true); (void)once; }
+          const unsigned grid = static_cast<unsigned>(std::max<long long>(1, std::min<long long>((cb.total + 7) / 8, 148 * 8)));
+          k::chain_rowreduce_warp<<<grid, 256, smem, x.stream>>>(cb, q.max_cols);
         } else {
-          const long long rows = cp.dim[0] * cp.dim[1] * cp.dim[2];
-          const size_t smem = static_cast<size_t>(cp.dim[3]) * 4;
-          if (smem > 48 * 1024) cudaFuncSetAttribute(k::chain_rowreduce, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-          k::chain_rowreduce<<<static_cast<unsigned>(std::min<long long>(rows, 148 * 8)), 256, smem, x.stream>>>(cp);
+          const size_t smem = static_cast<size_t>(q.max_cols) * 4;
+          if (smem > 48 * 1024) { static bool once = (cudaFuncSetAttribute(k::chain_rowreduce, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024), true); (void)once; }
+          k::chain_rowreduce<<<static_cast<unsigned>(std::max<long long>(1, std::min<long long>(cb.total, 148 * 8))), 256, smem, x.stream>>>(cb);
         }
         return cudaGetLastError();
       });
+    };
+    for (int r = 0; r < p.n_req; ++r) {
+      const View& ov = p.views[G.out][r];
+      if (!ov.contiguous()) return fail(E_UNSUPPORTED_OP, "chain output must be contiguous");
+      if (numel(ov.dims) == 0) continue;
+      int64_t od[4] = {1, 1, 1, 1};
+      for (size_t i = 0; i < ov.dims.size(); ++i) od[4 - ov.dims.size() + i] = ov.dims[i];
+      for (int i = 0; i < 4; ++i) if (od[i] >= (int64_t(1) << 31)) return fail(E_UNSUPPORTED_OP, "chain extent above 2^31");
+      if (red && od[3] * 4 > 200 * 1024) return fail(E_UNSUPPORTED_OP, "row too long for the row-reduction kernel");
+      // this request's operands: pointer, strides (0 on broadcast dims: read in place)
+      std::vector<Ptr> ptrs(1 + k::CHAIN_MAX_OPS);
+      int strides[1 + k::CHAIN_MAX_OPS][4] = {};
+      for (int kx = 0; kx <= k::CHAIN_MAX_OPS; ++kx) {
+        const int t = opnd[kx];
+        if (t < 0 || g.tensors[t].kind == TKind::FCONST) continue;
+        const int rr = g.tensors[t].kind == TKind::CONST ? 0 : r;
+        const View& v = p.views[t][rr];
+        const int rk = static_cast<int>(v.dims.size());
+        for (int i = 0; i < 4; ++i) {
+          const int src = i - (4 - rk);
+          const int64_t st = (src >= 0 && v.dims[src] != 1) ? v.strides[src] : 0;
+          if (st >= (int64_t(1) << 31) || st < 0) return fail(E_UNSUPPORTED_OP, "chain operand stride out of range");
+          strides[kx][i] = static_cast<int>(st);
+        }
+        ptrs[kx] = ptr_of(t, rr);
+      }
+      Ptr pout = ptr_of(G.out, r);
+      // does it fit the open table?
+      bool fits = cur.cb.n_req < k::CHAIN_MAX_REQ;
+      if (fits && cur.cb.n_req) {
+        if (!same_base(pout, cur.out)) fits = false;
+        for (int kx = 0; kx <= k::CHAIN_MAX_OPS && fits; ++kx)
+          if (opnd[kx] >= 0 && g.tensors[opnd[kx]].kind != TKind::FCONST && !same_base(ptrs[kx], cur.base[kx])) fits = false;
+      }
+      if (!fits) flush();
+      if (!cur.cb.n_req) { cur.out = pout; for (int kx = 0; kx <= k::CHAIN_MAX_OPS; ++kx) cur.base[kx] = ptrs[kx]; }
+      k::ChainReq& R = cur.cb.r[cur.cb.n_req++];
+      const int oesz = dtype_size(O.dtype);
+      for (int i = 0; i < 4; ++i) R.dim[i] = static_cast<int>(od[i]);
+      R.out_off = (pout.off - cur.out.off) / oesz;
+      bool vec = !red && od[3] % 8 == 0 && R.out_off % 8 == 0 && cur.out.off % 16 == 0;
+      for (int kx = 0; kx <= k::CHAIN_MAX_OPS; ++kx) {
+        const int t = opnd[kx];
+        if (t < 0 || g.tensors[t].kind == TKind::FCONST) continue;
+        const int esz = dtype_size(g.tensors[t].dtype);
+        R.off[kx] = (ptrs[kx].off - cur.base[kx].off) / esz;
+        for (int i = 0; i < 4; ++i) R.stride[kx][i] = strides[kx][i];
+        if (strides[kx][3] == 1 || od[3] == 1) {
+          // read as 8-element vectors: every address a multiple of 16 bytes (32 for fp32 pairs of float4)
+          if (od[3] != 1 && (R.off[kx] % 8 || strides[kx][0] % 8 || strides[kx][1] % 8 || strides[kx][2] % 8 || cur.base[kx].off % 16)) vec = false;
+        } else if (strides[kx][3] != 0) vec = false;
+      }
+      const long long items = red ? od[0] * od[1] * od[2] : (vec && cur.vec ? numel(ov.dims) / 8 : numel(ov.dims));
+      if ((red ? items : numel(ov.dims)) >= (int64_t(1) << 31)) return fail(E_UNSUPPORTED_OP, "chain request above 2^31 elements");
+      if (!red && cur.vec && !vec) {
+        // the table falls back to one element per item: recount the earlier requests
+        long long first = 0;
+        for (int q = 0; q + 1 < cur.cb.n_req; ++q) {
+          cur.cb.r[q].first = first;
+          first += static_cast<long long>(cur.cb.r[q].dim[0]) * cur.cb.r[q].dim[1] * cur.cb.r[q].dim[2] * cur.cb.r[q].dim[3];
+        }
+        cur.cb.total = first;
+        cur.vec = false;
+      }
+      R.first = cur.cb.total;
+      cur.cb.total += (!red && !cur.vec) ? numel(ov.dims) : items;
+      cur.max_cols = std::max(cur.max_cols, static_cast<int>(od[3]));
+      if (od[3] % 16) cur.vec16 = false;
     }
+    flush();
     return OK;
   }
 

@@ -280,88 +280,261 @@ __global__ void __launch_bounds__(256) splitk_ln_finish(const float* __restrict_
 }
 
 // ---------------------------------------------------------------------------------------------
-// Generic fused chain: v = load(in0); v = op_i(v [, operand_i]) ...; optional softmax / LayerNorm
-// over the last dim; store. Index space = the group's output [d0..d3] (rank <= 4 after
-// right-alignment); every operand is read through its own strides, 0 on broadcast dims.
+// Generic fused chain (the paper's Fig. 4 form): v = load(in0); v = op_i(v [, operand_i]) ...; optional softmax /
+// LayerNorm over the last dim; store.  Index space = the group's output [d0..d3] (rank <= 4 after
+// right-alignment); every operand is read through its own strides, 0 on the dims RDP resolved to "broadcast".
+// All requests of a batch run in ONE launch through a request table (up to CHAIN_MAX_REQ entries): the operands of
+// the requests live in the same packed buffers, so an entry is extents, element offsets and strides.
+//   chain_elementwise_vec   work item = 8 or 16 consecutive outputs along the last dim: 128-bit loads / stores, operands
+//                           broadcast along the last dim fetched once per item; (row, column) decomposition in 32-bit
+//                           arithmetic, one division chain per item instead of per element
+//   chain_elementwise       work item = one output (any strides, any extents): the fallback
+//   chain_rowreduce_warp    a warp per row (rows up to ROWRED_WARP_COLS), the row staged in the warp's slice of shared
+//                           memory, statistics by shuffles: no CTA barrier, eight rows in flight per CTA
+//   chain_rowreduce         a CTA per row for longer rows
 constexpr int CHAIN_MAX_OPS = 8;
+constexpr int CHAIN_MAX_REQ = 8;
+constexpr int ROWRED_WARP_COLS = 2048;
 enum ChainOp : int { C_ADD = 0, C_SUB, C_RSUB, C_MUL, C_DIV, C_RDIV, C_RELU, C_GELU, C_SIGMOID };
 enum ChainRed : int { RED_NONE = 0, RED_SOFTMAX = 1, RED_LAYERNORM = 2 };
 
-struct ChainOperand {
-  const void* ptr;      // nullptr: use `scalar`
-  long long stride[4];  // elements
-  float scalar;
-  int is_bf16;
+struct ChainReq {
+  int dim[4];                               // output extents
+  long long first;                          // first work item of this request in the launch
+  long long out_off;                        // elements from `out`
+  long long off[1 + CHAIN_MAX_OPS];         // elements from base[k]; k = 0 is in0, k = 1 + i operand i
+  int stride[1 + CHAIN_MAX_OPS][4];         // elements
 };
-struct ChainParams {
-  ChainOperand in0;
-  ChainOperand operand[CHAIN_MAX_OPS];
+struct ChainBatch {
+  const void* base[1 + CHAIN_MAX_OPS];      // nullptr: use scalar[k]
+  float scalar[1 + CHAIN_MAX_OPS];
+  int is_bf16[1 + CHAIN_MAX_OPS];
   int op[CHAIN_MAX_OPS];
   int n_ops;
-  long long dim[4];
-  void* out;            // contiguous
+  void* out;                                // every request's output instance is contiguous
   int out_bf16;
   int red;
   const void* gamma; const void* beta; int gb_bf16; float eps;
+  int n_req;
+  long long total;                          // work items of all requests
+  ChainReq r[CHAIN_MAX_REQ];
 };
 
-__device__ __forceinline__ float chain_load(const ChainOperand& o, long long i0, long long i1, long long i2, long long i3) {
-  if (!o.ptr) return o.scalar;
-  const long long off = i0 * o.stride[0] + i1 * o.stride[1] + i2 * o.stride[2] + i3 * o.stride[3];
-  return o.is_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(o.ptr)[off]) : reinterpret_cast<const float*>(o.ptr)[off];
+__device__ __forceinline__ int chain_find_req(const ChainBatch& p, long long item) {
+  int ri = 0;
+  while (ri + 1 < p.n_req && item >= p.r[ri + 1].first) ++ri;
+  return ri;
 }
-__device__ __forceinline__ float chain_eval(const ChainParams& p, long long i0, long long i1, long long i2, long long i3) {
-  float v = chain_load(p.in0, i0, i1, i2, i3);
+__device__ __forceinline__ float chain_apply(int op, float v, float w) {
+  switch (op) {
+    case C_ADD: return v + w;
+    case C_SUB: return v - w;
+    case C_RSUB: return w - v;
+    case C_MUL: return v * w;
+    case C_DIV: return v / w;
+    case C_RDIV: return w / v;
+    case C_RELU: return fmaxf(v, 0.f);
+    case C_GELU: return act_apply(1, v);
+    default: return act_apply(3, v);
+  }
+}
+__device__ __forceinline__ float chain_load1(const ChainBatch& p, const ChainReq& R, int k, int i0, int i1, int i2, int i3) {
+  if (!p.base[k]) return p.scalar[k];
+  const long long off = R.off[k] + static_cast<long long>(i0) * R.stride[k][0] + static_cast<long long>(i1) * R.stride[k][1] +
+                        static_cast<long long>(i2) * R.stride[k][2] + static_cast<long long>(i3) * R.stride[k][3];
+  return p.is_bf16[k] ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.base[k])[off]) : reinterpret_cast<const float*>(p.base[k])[off];
+}
+__device__ __forceinline__ float chain_eval(const ChainBatch& p, const ChainReq& R, int i0, int i1, int i2, int i3) {
+  float v = chain_load1(p, R, 0, i0, i1, i2, i3);
   for (int k = 0; k < p.n_ops; ++k) {
     const int op = p.op[k];
-    if (op >= C_RELU) { v = act_apply(op == C_RELU ? 2 : op == C_GELU ? 1 : 3, v); continue; }
-    const float w = chain_load(p.operand[k], i0, i1, i2, i3);
-    switch (op) {
-      case C_ADD: v = v + w; break;
-      case C_SUB: v = v - w; break;
-      case C_RSUB: v = w - v; break;
-      case C_MUL: v = v * w; break;
-      case C_DIV: v = v / w; break;
-      default: v = w / v; break;
-    }
+    v = chain_apply(op, v, op >= C_RELU ? 0.f : chain_load1(p, R, 1 + k, i0, i1, i2, i3));
   }
   return v;
 }
-__device__ __forceinline__ void chain_store(const ChainParams& p, long long lin, float v) {
+__device__ __forceinline__ void chain_store1(const ChainBatch& p, long long lin, float v) {
   if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[lin] = __float2bfloat16_rn(v);
   else reinterpret_cast<float*>(p.out)[lin] = v;
 }
 
-// no reduction: one thread per output element, grid-stride
-__global__ void __launch_bounds__(256) chain_elementwise(ChainParams p) {
-  const long long total = p.dim[0] * p.dim[1] * p.dim[2] * p.dim[3];
-  for (long long lin = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; lin < total;
-       lin += static_cast<long long>(gridDim.x) * blockDim.x) {
-    long long r = lin;
-    const long long i3 = r % p.dim[3]; r /= p.dim[3];
-    const long long i2 = r % p.dim[2]; r /= p.dim[2];
-    const long long i1 = r % p.dim[1];
-    const long long i0 = r / p.dim[1];
-    chain_store(p, lin, chain_eval(p, i0, i1, i2, i3));
+// eight consecutive elements of operand k along the last dim (stride 1, 16-byte aligned), or one broadcast value
+__device__ __forceinline__ void chain_load8(const ChainBatch& p, const ChainReq& R, int k, int i0, int i1, int i2, int i3, float* w) {
+  if (!p.base[k]) {
+#pragma unroll
+    for (int t = 0; t < 8; ++t) w[t] = p.scalar[k];
+    return;
+  }
+  const long long off = R.off[k] + static_cast<long long>(i0) * R.stride[k][0] + static_cast<long long>(i1) * R.stride[k][1] +
+                        static_cast<long long>(i2) * R.stride[k][2] + static_cast<long long>(i3) * R.stride[k][3];
+  if (R.stride[k][3] == 0) {
+    const float x = p.is_bf16[k] ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.base[k])[off]) : reinterpret_cast<const float*>(p.base[k])[off];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) w[t] = x;
+  } else if (p.is_bf16[k]) {
+    const uint4 u = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.base[k]) + off);
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+    for (int t = 0; t < 4; ++t) { const float2 f = __bfloat1622float2(h[t]); w[2 * t] = f.x; w[2 * t + 1] = f.y; }
+  } else {
+    const float4 a = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p.base[k]) + off);
+    const float4 c = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p.base[k]) + off + 4);
+    w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w; w[4] = c.x; w[5] = c.y; w[6] = c.z; w[7] = c.w;
   }
 }
 
-// trailing row reduction: one CTA per row of the last dim, the row is staged in shared memory
-__global__ void __launch_bounds__(256) chain_rowreduce(ChainParams p) {
+// The host selects this kernel only if, for every request, dim[3] % (8 * NV) == 0, every operand's last-dim stride is
+// 0 or 1, and all offsets and leading strides of stride-1 operands (and the output offset) are multiples of 8
+// elements.  NV = 8-element vectors per work item (1 or 2): the index arithmetic is paid once per item.
+template <int NV>
+__global__ void __launch_bounds__(256) chain_elementwise_vec(const __grid_constant__ ChainBatch p) {
+  for (long long item = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; item < p.total;
+       item += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const ChainReq& R = p.r[chain_find_req(p, item)];
+    const unsigned li = static_cast<unsigned>(item - R.first);      // the host keeps a request below 2^31 items
+    const unsigned cv = static_cast<unsigned>(R.dim[3]) / (8 * NV);
+    unsigned row = li / cv;
+    const int i3 = static_cast<int>(li - row * cv) * (8 * NV);
+    const unsigned d2 = R.dim[2], d1 = R.dim[1];
+    const unsigned t2 = row / d2;
+    const int i2 = static_cast<int>(row - t2 * d2);
+    const unsigned t1 = t2 / d1;
+    const int i1 = static_cast<int>(t2 - t1 * d1), i0 = static_cast<int>(t1);
+    // While every operand so far is broadcast along the last dim the values of an item are one value: that prefix
+    // of the chain (Fig. 4: Sigmoid of the [I,1,1] operand) is evaluated once per item, not once per element.
+    float v[NV][8], w[NV][8];
+    int k0 = 0;
+    if (!p.base[0] || R.stride[0][3] == 0) {
+      float u = chain_load1(p, R, 0, i0, i1, i2, i3);
+      for (; k0 < p.n_ops; ++k0) {
+        const int op = p.op[k0];
+        if (op < C_RELU && p.base[1 + k0] && R.stride[1 + k0][3] != 0) break;
+        u = chain_apply(op, u, op >= C_RELU ? 0.f : chain_load1(p, R, 1 + k0, i0, i1, i2, i3));
+      }
+#pragma unroll
+      for (int n = 0; n < NV; ++n)
+#pragma unroll
+        for (int t = 0; t < 8; ++t) v[n][t] = u;
+    } else {
+#pragma unroll
+      for (int n = 0; n < NV; ++n) chain_load8(p, R, 0, i0, i1, i2, i3 + 8 * n, v[n]);
+    }
+    for (int k = k0; k < p.n_ops; ++k) {
+      const int op = p.op[k];
+      if (op < C_RELU) {
+#pragma unroll
+        for (int n = 0; n < NV; ++n) chain_load8(p, R, 1 + k, i0, i1, i2, i3 + 8 * n, w[n]);
+      }
+      // the operator is chosen once per item; the elements run through straight-line code
+      switch (op) {
+#define SOD2_CHAIN_CASE(OP_)                                                                                   \
+        case OP_:                                                                                              \
+          _Pragma("unroll") for (int n = 0; n < NV; ++n)                                                       \
+            _Pragma("unroll") for (int t = 0; t < 8; ++t) v[n][t] = chain_apply(OP_, v[n][t], w[n][t]);        \
+          break;
+        SOD2_CHAIN_CASE(C_ADD)
+        SOD2_CHAIN_CASE(C_SUB)
+        SOD2_CHAIN_CASE(C_RSUB)
+        SOD2_CHAIN_CASE(C_MUL)
+        SOD2_CHAIN_CASE(C_DIV)
+        SOD2_CHAIN_CASE(C_RDIV)
+        SOD2_CHAIN_CASE(C_RELU)
+        SOD2_CHAIN_CASE(C_GELU)
+        default:
+        SOD2_CHAIN_CASE(C_SIGMOID)
+#undef SOD2_CHAIN_CASE
+      }
+    }
+    const long long lin = R.out_off + static_cast<long long>(li) * (8 * NV);
+#pragma unroll
+    for (int n = 0; n < NV; ++n) {
+      if (p.out_bf16) {
+        uint4 o;
+        __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+        for (int t = 0; t < 4; ++t) oh[t] = __floats2bfloat162_rn(v[n][2 * t], v[n][2 * t + 1]);
+        *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + lin + 8 * n) = o;
+      } else {
+        float* o = reinterpret_cast<float*>(p.out) + lin + 8 * n;
+        *reinterpret_cast<float4*>(o) = make_float4(v[n][0], v[n][1], v[n][2], v[n][3]);
+        *reinterpret_cast<float4*>(o + 4) = make_float4(v[n][4], v[n][5], v[n][6], v[n][7]);
+      }
+    }
+  }
+}
+
+// fallback: one thread per output element, grid-stride
+__global__ void __launch_bounds__(256) chain_elementwise(const __grid_constant__ ChainBatch p) {
+  for (long long item = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; item < p.total;
+       item += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const ChainReq& R = p.r[chain_find_req(p, item)];
+    long long r = item - R.first;
+    const int i3 = static_cast<int>(r % R.dim[3]); r /= R.dim[3];
+    const int i2 = static_cast<int>(r % R.dim[2]); r /= R.dim[2];
+    const int i1 = static_cast<int>(r % R.dim[1]);
+    const int i0 = static_cast<int>(r / R.dim[1]);
+    chain_store1(p, R.out_off + (item - R.first), chain_eval(p, R, i0, i1, i2, i3));
+  }
+}
+
+__device__ __forceinline__ void chain_row_index(const ChainReq& R, long long row, int* i0, int* i1, int* i2) {
+  *i2 = static_cast<int>(row % R.dim[2]); row /= R.dim[2];
+  *i1 = static_cast<int>(row % R.dim[1]);
+  *i0 = static_cast<int>(row / R.dim[1]);
+}
+__device__ __forceinline__ float chain_gb(const ChainBatch& p, const void* v, int c) {
+  return p.gb_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(v)[c]) : reinterpret_cast<const float*>(v)[c];
+}
+
+// trailing row reduction, a warp per row: work item = row; dynamic shared memory = 8 rows of `max_cols` floats
+__global__ void __launch_bounds__(256) chain_rowreduce_warp(const __grid_constant__ ChainBatch p, int max_cols) {
+  extern __shared__ float rowbuf_all[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float* rowbuf = rowbuf_all + static_cast<size_t>(warp) * max_cols;
+  for (long long item = static_cast<long long>(blockIdx.x) * 8 + warp; item < p.total; item += static_cast<long long>(gridDim.x) * 8) {
+    const ChainReq& R = p.r[chain_find_req(p, item)];
+    const long long row = item - R.first;
+    const int cols = R.dim[3];
+    int i0, i1, i2;
+    chain_row_index(R, row, &i0, &i1, &i2);
+    float m = -INFINITY, s = 0.f;
+    for (int c = lane; c < cols; c += 32) {
+      const float v = chain_eval(p, R, i0, i1, i2, c);
+      rowbuf[c] = v;
+      m = fmaxf(m, v);
+      s += v;
+    }
+    const float st0 = p.red == RED_SOFTMAX ? warp_max(m) : warp_sum(s) / cols;
+    float q = 0.f;
+    for (int c = lane; c < cols; c += 32) {
+      if (p.red == RED_SOFTMAX) { const float e = __expf(rowbuf[c] - st0); rowbuf[c] = e; q += e; }
+      else { const float d = rowbuf[c] - st0; q += d * d; }
+    }
+    q = warp_sum(q);
+    const float st1 = p.red == RED_SOFTMAX ? 1.0f / q : rsqrtf(q / cols + p.eps);
+    const long long obase = R.out_off + row * cols;
+    for (int c = lane; c < cols; c += 32) {
+      const float v = p.red == RED_SOFTMAX ? rowbuf[c] * st1 : (rowbuf[c] - st0) * st1 * chain_gb(p, p.gamma, c) + chain_gb(p, p.beta, c);
+      chain_store1(p, obase + c, v);
+    }
+    __syncwarp();
+  }
+}
+
+// trailing row reduction, a CTA per row (long rows): dynamic shared memory = one row
+__global__ void __launch_bounds__(256) chain_rowreduce(const __grid_constant__ ChainBatch p) {
   extern __shared__ float rowbuf[];
   __shared__ float red[8];
   __shared__ float bc[2];
-  const long long cols = p.dim[3];
-  const long long rows = p.dim[0] * p.dim[1] * p.dim[2];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (long long row = blockIdx.x; row < rows; row += gridDim.x) {
-    long long r = row;
-    const long long i2 = r % p.dim[2]; r /= p.dim[2];
-    const long long i1 = r % p.dim[1];
-    const long long i0 = r / p.dim[1];
+  for (long long item = blockIdx.x; item < p.total; item += gridDim.x) {
+    const ChainReq& R = p.r[chain_find_req(p, item)];
+    const long long row = item - R.first;
+    const int cols = R.dim[3];
+    int i0, i1, i2;
+    chain_row_index(R, row, &i0, &i1, &i2);
     float m = -INFINITY, s = 0.f;
-    for (long long c = threadIdx.x; c < cols; c += blockDim.x) {
-      const float v = chain_eval(p, i0, i1, i2, c);
+    for (int c = threadIdx.x; c < cols; c += blockDim.x) {
+      const float v = chain_eval(p, R, i0, i1, i2, c);
       rowbuf[c] = v;
       m = fmaxf(m, v);
       s += v;
@@ -378,7 +551,7 @@ __global__ void __launch_bounds__(256) chain_rowreduce(ChainParams p) {
     __syncthreads();
     const float st0 = bc[0];
     float q = 0.f;
-    for (long long c = threadIdx.x; c < cols; c += blockDim.x) {
+    for (int c = threadIdx.x; c < cols; c += blockDim.x) {
       if (p.red == RED_SOFTMAX) { const float e = __expf(rowbuf[c] - st0); rowbuf[c] = e; q += e; }
       else { const float d = rowbuf[c] - st0; q += d * d; }
     }
@@ -393,15 +566,10 @@ __global__ void __launch_bounds__(256) chain_rowreduce(ChainParams p) {
     }
     __syncthreads();
     const float st1 = bc[1];
-    for (long long c = threadIdx.x; c < cols; c += blockDim.x) {
-      float v;
-      if (p.red == RED_SOFTMAX) v = rowbuf[c] * st1;
-      else {
-        const float g = p.gb_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.gamma)[c]) : reinterpret_cast<const float*>(p.gamma)[c];
-        const float b = p.gb_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.beta)[c]) : reinterpret_cast<const float*>(p.beta)[c];
-        v = (rowbuf[c] - st0) * st1 * g + b;
-      }
-      chain_store(p, row * cols + c, v);
+    const long long obase = R.out_off + row * cols;
+    for (int c = threadIdx.x; c < cols; c += blockDim.x) {
+      const float v = p.red == RED_SOFTMAX ? rowbuf[c] * st1 : (rowbuf[c] - st0) * st1 * chain_gb(p, p.gamma, c) + chain_gb(p, p.beta, c);
+      chain_store1(p, obase + c, v);
     }
     __syncthreads();
   }
