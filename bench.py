@@ -395,7 +395,7 @@ def run_ours(args):
                     "worst_group": r["worst_group"], "kinds": r["kinds"], "plan_us": r["plan_us_median"],
                     "plan_us_cache_hit": r["plan_us_cache_hit"], "arena_bytes": r["arena_bytes"], "peak_live_bytes": r["peak_live_bytes"],
                     "gpu_launches": r["gpu_launches"], "units": r["units_batch0"], "unit": r["unit"],
-                    **{k: r[k] for k in ("ms_one_request_per_inference", "ms_empty_kernel", "ratio_to_empty_kernel") if k in r}}
+                    **{k: r[k] for k in ("ms_one_request_per_inference", "ms_empty_kernel", "ratio_to_empty_kernel", "exact_edo") if k in r}}
             line["configs_note"] = ("ms / ms_graph: device time per inference (median, L2 flushed), stream-launched / replayed as one CUDA graph; "
                                     "e2e_ms: pinned H2D + bind + plan + run + D2H; group figures: CUDA events around every launch")
         print(json.dumps(line))

@@ -123,6 +123,21 @@ sod2_status sod2_run(sod2_plan_t* p, const void* const* inputs, void* const* out
 sod2_status sod2_run_graph(sod2_plan_t* p, const void* const* inputs, void* const* outputs, void* arena,
                            size_t arena_bytes, void* cuda_stream, sod2_run_info* info);
 
+/* The same inference with EXACT handling of execution-determined extents, the staging the paper describes
+ * (Section 3: the output shape of such an operator is known only once it has run; Section 4.3: the graph is
+ * partitioned at these operators; Section 4.4.1: memory is planned when the sizes are known).  p is the ordinary
+ * (bounded) plan of the binding: sod2_run keeps every count on the device and plans such tensors at their static
+ * upper bound, one uninterrupted launch sequence.  Here the sub-graphs of the partition run one after another; after
+ * each sub-graph that holds a Switch or NonZero the counts are copied to the host (the call SYNCHRONISES cuda_stream
+ * there), the run-time symbols are bound to them and the remaining sub-graphs are planned again at their true sizes:
+ * tensors that already exist keep their arena offsets, the others are laid out around them; group scratch and the
+ * Switch index lists sit at fixed offsets behind the arena header.  Same kernels, same results.  arena as for
+ * sod2_run (>= the bounded plan's arena_bytes).  info->reserved[2] = stages planned, reserved[3] = largest arena
+ * extent (bytes) any stage laid out (a stage places only the tensors of its own sub-graphs); reserved[4] = host nanoseconds spent binding and planning the stages.
+ * Errors as sod2_run, plus SOD2_E_ARENA_TOO_SMALL if a stage planned around the tensors in place does not fit. */
+sod2_status sod2_run_exact(sod2_plan_t* p, const void* const* inputs, void* const* outputs, void* arena,
+                           size_t arena_bytes, void* cuda_stream, sod2_run_info* info);
+
 /* Measurement aid: the same inference with CUDA events recorded on cuda_stream around every launch.
  * Synchronises the stream and returns the device time of each fused group in group_ms[n_groups]
  * (host array, milliseconds; n_groups must equal sod2_graph_num_groups).  A launch that runs several

@@ -57,6 +57,7 @@ def _load() -> C.CDLL:
         "sod2_plan_cached": [vp, i32, i32, P(cp), P(i64), P(vp), P(vp), P(sz), P(i32)],
         "sod2_run": [vp, P(vp), P(vp), vp, sz, vp, P(RunInfo)],
         "sod2_run_graph": [vp, P(vp), P(vp), vp, sz, vp, P(RunInfo)],
+        "sod2_run_exact": [vp, P(vp), P(vp), vp, sz, vp, P(RunInfo)],
         "sod2_run_timed": [vp, P(vp), P(vp), vp, sz, vp, P(C.c_float), i32],
         "sod2_run_timed_repeat": [vp, P(vp), P(vp), vp, sz, vp, i32, P(C.c_float), i32],
         "sod2_plan_device_status": [vp, vp, vp],
@@ -97,7 +98,7 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = ["sod2_graph_create", "sod2_graph_destroy", "sod2_graph_set_const", "sod2_graph_prepack_bytes",
            "sod2_graph_prepack", "sod2_bind_dims", "sod2_binding_destroy", "sod2_plan", "sod2_plan_destroy", "sod2_graph_set_plan_cache", "sod2_plan_cached",
-           "sod2_run", "sod2_run_graph", "sod2_run_timed", "sod2_run_timed_repeat", "sod2_plan_device_status", "sod2_graph_tensor_info", "sod2_graph_tensor_value", "sod2_graph_tensor_dtype",
+           "sod2_run", "sod2_run_graph", "sod2_run_exact", "sod2_run_timed", "sod2_run_timed_repeat", "sod2_plan_device_status", "sod2_graph_tensor_info", "sod2_graph_tensor_value", "sod2_graph_tensor_dtype",
            "sod2_graph_num_ops", "sod2_graph_op_info", "sod2_graph_num_groups", "sod2_graph_group_info",
            "sod2_graph_num_subgraphs", "sod2_graph_rdp_sweeps", "sod2_classify", "sod2_graph_reanalyse", "sod2_graph_order_info",
            "sod2_binding_shape", "sod2_plan_slot", "sod2_plan_instance_offset", "sod2_plan_memory", "sod2_plan_group_cost", "sod2_plan_tensor_strides",
@@ -303,6 +304,15 @@ class Plan:
         outs = (C.c_void_p * max(len(outputs), 1))(*outputs)
         info = RunInfo()
         _check(lib.sod2_run_graph(self.h, ins, outs, C.c_void_p(arena), arena_bytes, C.c_void_p(stream), C.byref(info)), self.h)
+        return info
+
+    def run_exact(self, inputs: Sequence[int], outputs: Sequence[int], arena: int, arena_bytes: int, stream: int) -> RunInfo:
+        """The inference with exact handling of execution-determined extents: counts read back after every Switch /
+        NonZero, the remaining sub-graphs planned again at their true sizes (synchronises the stream at each)."""
+        ins = (C.c_void_p * max(len(inputs), 1))(*inputs)
+        outs = (C.c_void_p * max(len(outputs), 1))(*outputs)
+        info = RunInfo()
+        _check(lib.sod2_run_exact(self.h, ins, outs, C.c_void_p(arena), arena_bytes, C.c_void_p(stream), C.byref(info)), self.h)
         return info
 
     def run_timed(self, inputs: Sequence[int], outputs: Sequence[int], arena: int, arena_bytes: int, stream: int, reps: int = 1) -> List[float]:

@@ -240,6 +240,28 @@ sod2_status sod2_run_graph(sod2_plan_t* p, const void* const* inputs, void* cons
   return st(s);
 }
 
+sod2_status sod2_run_exact(sod2_plan_t* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes,
+                           void* stream, sod2_run_info* info) {
+  if (!p || !inputs || !outputs || !arena) return SOD2_E_INVALID_ARG;
+  if (arena_bytes < p->p.arena_bytes) { p->h.err = "arena too small"; return SOD2_E_ARENA_TOO_SMALL; }
+  if (reinterpret_cast<uintptr_t>(arena) & 255) { p->h.err = "arena must be 256-byte aligned"; return SOD2_E_MISALIGNED; }
+  if (p->g->c.packed_bytes && !p->g->c.packed_ws) { p->h.err = "weights are not prepacked"; return SOD2_E_INVALID_ARG; }
+  if (!p->p.sm_count_known) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) p->p.sm_count = n;
+    p->p.sm_count_known = true;
+  }
+  int64_t inf[8] = {0};
+  std::string err;
+  Status s = run_exact(&p->g->c, p->p.b, &p->p, inputs, outputs, arena, arena_bytes, stream, inf, &err);
+  if (s != OK) p->h.err = err;
+  if (info) {
+    info->host_enqueue_ns = inf[0]; info->gpu_launches = inf[1];
+    info->reserved[2] = inf[2]; info->reserved[3] = inf[3]; info->reserved[4] = inf[4];
+  }
+  return st(s);
+}
+
 sod2_status sod2_run_timed(sod2_plan_t* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes,
                            void* stream, float* group_ms, int n_groups) {
   if (!p || !inputs || !outputs || !arena) return SOD2_E_INVALID_ARG;

@@ -207,6 +207,8 @@ struct Binding {
   std::string err;
 };
 Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* names, const int64_t* values, Binding* out);
+Status evaluate_dims(Binding* out);
+Status rebind_runtime(const Binding& base, const std::vector<std::vector<std::pair<int, int64_t>>>& rt_vals, Binding* out);
 
 // ---- plan
 struct View {                 // one tensor of one request, resolved to storage
@@ -270,6 +272,17 @@ struct Plan {
   size_t chain_counter_off = 0;           // byte offset in the arena header of the chains' row-block counters
   size_t chain_counter_words = 0;
   size_t header_clear_bytes = 256;        // what a run zeroes at the start of the arena (status word, tickets, chain counters)
+  // Staged planning (exact handling of execution-determined extents): `pinned` roots keep the arena offsets an
+  // earlier stage gave them; `front_reserve` > 0 puts the group scratch (front_scratch bytes) and the Switch index
+  // lists behind the header instead of behind the tensors, so that neither moves between stages.
+  std::vector<std::pair<int, size_t>> pinned;
+  size_t front_reserve = 0, front_scratch = 0, header_end = 0;
+  // a staged plan lays out only the tensors of its own steps: those defined at or before place_until_step and still
+  // live at place_from_step (earlier ones are dead, later ones are planned by a later stage, at their true sizes)
+  int place_from_step = 0, place_until_step = 1 << 30;
+  // [group] run-time symbols (atom ids) whose counts are in the arena header once the group has run: a gate whose
+  // kernel also partitions the sample ids, a Switch that partitions them itself, a NonZero
+  std::vector<std::vector<int>> rt_syms_after;
   std::string err;
   // device status word lives at arena offset 0 (first 256 bytes reserved)
   // CUDA graph of the whole launch sequence for one set of buffers (run_plan_graph)
@@ -295,8 +308,15 @@ Status run_plan_graph(Plan* p, const void* const* inputs, void* const* outputs, 
                       int64_t* info);
 Status build_launches(Plan* p);   // exec.cu
 Status detect_chains(Plan* p);    // exec.cu: fills Plan::chains / chain_of from the resolved views
+// step_lo..step_hi: only these groups (positions in execution order) are enqueued (all by default); the arena header
+// is cleared only by a run that starts at group 0.
 Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream,
-                int64_t* info);
+                int64_t* info, int step_lo = 0, int step_hi = 1 << 30);
+
+// Exact handling of execution-determined extents: see exec.cu.  `bounded` is the ordinary plan of b0 (its scratch
+// sizes fix the layout in front of the tensors); the arena must hold at least bounded->arena_bytes.
+Status run_exact(const Compiled* c, const Binding* b0, const Plan* bounded, const void* const* inputs, void* const* outputs, void* arena,
+                 size_t arena_bytes, void* stream, int64_t* info, std::string* err);
 
 // Same as run_plan, with CUDA events around every launch; synchronises the stream and returns the
 // device time per group (ms).

@@ -1045,6 +1045,7 @@ struct Builder {
     // the runtime symbol that names the count
     const Expr& ce = g.tensors[G.out].S.dims[1].e;
     const int sym = ce.terms.begin()->first[0].first;
+    count_known_after(gi, G.out);
     for (int r = 0; r < p.n_req; ++r) {
       const View& v = p.views[G.a][r];
       if (!v.contiguous()) return fail(E_UNSUPPORTED_OP, "NonZero needs a contiguous input");
@@ -1486,6 +1487,20 @@ struct Builder {
   // ------------------------------------------------------------------------------ run-time sample counts
   // A tensor whose leading extent is execution determined (gated sub-batch): extent = a + b * count,
   // where count is the run-time symbol's slot in the arena header, written by the Switch group.
+  int rt_symbol_of(int t) const {
+    const ShapeVal& sv = g.tensors[t].S;
+    for (const Dim& d : sv.dims)
+      if (d.known())
+        for (auto& term : d.e.terms)
+          for (auto& pw : term.first)
+            if (g.cx.atoms[pw.first].kind == AtomKind::SYM && g.cx.atoms[pw.first].runtime) return pw.first;
+    return -1;
+  }
+  void count_known_after(int gi, int tensor) {
+    if (p.rt_syms_after.size() != c.groups.size()) p.rt_syms_after.assign(c.groups.size(), {});
+    const int sym = rt_symbol_of(tensor);
+    if (sym >= 0) p.rt_syms_after[gi].push_back(sym);
+  }
   struct RtCount { bool rt = false; size_t slot_off = 0; int a = 0, b = 0; };
   RtCount runtime_count(int t, int r) const {
     RtCount rc;
@@ -1555,6 +1570,7 @@ struct Builder {
           aux_need += (static_cast<size_t>(2 * N) * 4 + 16 + 255) & ~size_t(255);
           part_slot = rc.slot_off;
           partition_fused.insert(S.gate);
+          count_known_after(gi, S.out);
           fuse_part = true;
           ++n_tickets;
           break;
@@ -1651,6 +1667,7 @@ struct Builder {
     if (!fused) {
       switch_aux[G.gate] = aux;
       aux_need += (static_cast<size_t>(2 * N) * 4 + 16 + 255) & ~size_t(255);
+      count_known_after(gi, G.out);
     }
     const bool indirect = c.storage[G.out].kind == Storage::INDIRECT_IN;
     if (fused && indirect) return OK;
@@ -1844,6 +1861,7 @@ struct Builder {
     p.group_flops.clear();
     p.group_bytes.clear();
     p.gpu_launches = 0;
+    p.rt_syms_after.assign(c.groups.size(), {});
     // the fp32 row kernel and the elementwise chains have no bounded waits, tickets or device-side counts
     // a pooling group right after a layout change of the SAME tensor: neither reads what the other writes, and the
     // shared input stays live over both steps, so the arena plan (liveness by step) cannot hand the pooled output a
@@ -1884,6 +1902,14 @@ struct Builder {
       }
       if (s != OK) return s;
       cost(G);
+    }
+    if (p.front_reserve) {
+      // staged plan: scratch and index lists at the fixed places behind the header that the first stage chose
+      const size_t sc = (scratch_need + 255) & ~size_t(255), ax = (aux_need + 255) & ~size_t(255);
+      if (sc > p.front_scratch || p.front_scratch + ax > p.front_reserve) return fail(E_INTERNAL, "stage needs more scratch than the bounded plan reserved");
+      p.scratch_off.assign(2, p.header_end);
+      p.scratch_off[1] = p.header_end + p.front_scratch;
+      return OK;
     }
     // one scratch region shared by all groups (they run in stream order), after the tensors
     p.scratch_off.assign(2, p.arena_bytes);
@@ -2112,7 +2138,8 @@ Status run_plan_graph(Plan* p, const void* const* inputs, void* const* outputs, 
   return OK;
 }
 
-Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream, int64_t* info) {
+Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes, void* stream, int64_t* info,
+                int step_lo, int step_hi) {
   if (!arena && p->arena_bytes) { p->err = "arena is null"; return E_INVALID_ARG; }
   if (arena_bytes < p->arena_bytes) { p->err = "arena too small"; return E_ARENA_TOO_SMALL; }
   if (reinterpret_cast<uintptr_t>(arena) & 255) { p->err = "arena must be 256-byte aligned"; return E_MISALIGNED; }
@@ -2124,14 +2151,17 @@ Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* 
     p->sm_count_known = true;
   }
   RunCtx x{inputs, outputs, static_cast<char*>(arena), static_cast<char*>(p->c->packed_ws), static_cast<cudaStream_t>(stream), p};
-  if (p->uses_header && cudaMemsetAsync(arena, 0, p->header_clear_bytes, x.stream) != cudaSuccess) { p->err = "cannot clear the status word"; return E_CUDA; }
+  if (p->uses_header && step_lo <= 0 && cudaMemsetAsync(arena, 0, p->header_clear_bytes, x.stream) != cudaSuccess) { p->err = "cannot clear the status word"; return E_CUDA; }
   if (!ensure_side_stream(p)) { p->err = "cannot create the second stream"; return E_CUDA; }
   const int n_groups = static_cast<int>(p->side_group.size());
   cudaStream_t side = static_cast<cudaStream_t>(p->side_stream);
   bool open_fork = false;
+  int64_t enqueued = 0;
   for (size_t i = 0; i < p->launches.size(); ++i) {
     auto& L = p->launches[i];
     const int g = L->group;
+    if (g < step_lo || g > step_hi) continue;
+    enqueued += L->n_kernels;
     const bool first_of_group = i == 0 || p->launches[i - 1]->group != g;
     const bool last_of_group = i + 1 == p->launches.size() || p->launches[i + 1]->group != g;
     const bool on_side = side && g >= 0 && g < n_groups && p->side_group[g] && open_fork;
@@ -2164,7 +2194,99 @@ Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* 
   }
   if (info) {
     info[0] = std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t0).count();
-    info[1] = p->gpu_launches;
+    info[1] = (step_lo <= 0 && step_hi >= (1 << 30)) ? p->gpu_launches : enqueued;
+  }
+  return OK;
+}
+
+// Exact handling of execution-determined extents (Section 3: the output shape of such an operator is known only
+// after it ran; Section 4.3: the graph is partitioned there; Section 4.4.1: memory is planned once the sizes are
+// known).  The groups run stage by stage; after a group that leaves a count on the device (the gate kernel that
+// partitions the sample ids, a Switch that partitions them itself, a NonZero) the counts are
+// read back (one copy + one stream synchronisation), the run-time symbols are bound to them, and the rest of the
+// graph is planned again at the true sizes: tensors that already exist keep their places, the others are laid
+// out around them.  info: [0] host ns, [1] kernels enqueued, [2] stages, [3] largest arena extent any stage laid out,
+// [4] host ns spent binding and planning the stages.
+Status run_exact(const Compiled* c, const Binding* b0, const Plan* bounded, const void* const* inputs, void* const* outputs, void* arena,
+                 size_t arena_bytes, void* stream, int64_t* info, std::string* err) {
+  auto t0 = std::chrono::steady_clock::now();
+  const Graph& g = c->g;
+  const int n_req = b0->n_req;
+  const int n_groups = static_cast<int>(c->groups.size());
+  // run-time symbols whose counts are on the device once a group has run (recorded by the bounded plan's builders)
+  std::vector<std::vector<int>> syms_of(n_groups);
+  for (int gi = 0; gi < n_groups && gi < static_cast<int>(bounded->rt_syms_after.size()); ++gi) syms_of[gi] = bounded->rt_syms_after[gi];
+  // the places of scratch and index lists: sized by the bounded plan, fixed for every stage
+  const size_t front_scratch = bounded->scratch_off[1] - bounded->scratch_off[0];
+  const size_t front_total = front_scratch + (bounded->arena_bytes - bounded->scratch_off[1]);
+  std::unique_ptr<Binding> bind(new Binding());
+  std::unique_ptr<Plan> plan(new Plan());
+  std::vector<std::vector<std::pair<int, int64_t>>> rt(n_req);
+  int64_t plan_ns = 0, launches = 0, stages = 0;
+  size_t peak_extent = 0;
+  auto make_stage = [&](const Plan* prev, int first_step, int last_step) -> Status {
+    auto tp = std::chrono::steady_clock::now();
+    std::unique_ptr<Binding> nb(new Binding());
+    Status s = rebind_runtime(*b0, rt, nb.get());
+    if (s != OK) { *err = nb->err; return s; }
+    std::unique_ptr<Plan> np(new Plan());
+    np->front_reserve = front_total;
+    np->front_scratch = front_scratch;
+    np->place_from_step = first_step;
+    np->place_until_step = last_step;
+    if (prev)
+      for (size_t t = 0; t < prev->roots.size(); ++t) {
+        const RootBuf& R = prev->roots[t];
+        if (R.where == RootBuf::ARENA && R.def_step >= 0 && R.def_step < first_step && R.last_step >= first_step) np->pinned.push_back({static_cast<int>(t), R.arena_off});
+      }
+    s = make_plan(c, nb.get(), np.get());
+    if (s != OK) { *err = np->err; return s; }
+    if (np->arena_bytes > arena_bytes) { *err = "arena too small for a stage planned around the tensors in place"; return E_ARENA_TOO_SMALL; }
+    peak_extent = std::max(peak_extent, np->arena_bytes);
+    np->sm_count = bounded->sm_count;
+    np->sm_count_known = bounded->sm_count_known;
+    bind = std::move(nb);
+    plan = std::move(np);
+    plan_ns += std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - tp).count();
+    ++stages;
+    return OK;
+  };
+  // stages: runs of groups up to and including one after which a count is known (a cut may fall inside a sub-graph
+  // of the partition: the gate kernel already knows the count that sizes the Switch outputs)
+  struct Stage { int first_step, last_step; std::vector<int> newly; };
+  std::vector<Stage> plan_stages;
+  {
+    int lo = 0;
+    for (int gi = 0; gi < n_groups; ++gi) {
+      if (syms_of[gi].empty() && gi + 1 < n_groups) continue;
+      plan_stages.push_back(Stage{lo, gi, syms_of[gi]});
+      lo = gi + 1;
+    }
+  }
+  const size_t n_atoms = g.cx.atoms.size();
+  std::vector<long long> counts(n_atoms * static_cast<size_t>(n_req));
+  for (size_t k = 0; k < plan_stages.size(); ++k) {
+    const Stage& st = plan_stages[k];
+    if (st.last_step < 0) continue;                       // no group in these sub-graphs
+    Status s = make_stage(k ? plan.get() : nullptr, st.first_step, st.last_step);
+    if (s != OK) return s;
+    int64_t inf[8] = {0};
+    s = run_plan(plan.get(), inputs, outputs, arena, arena_bytes, stream, inf, st.first_step, st.last_step);
+    if (s != OK) { *err = plan->err; return s; }
+    launches += inf[1];
+    if (k + 1 >= plan_stages.size() || st.newly.empty()) continue;
+    // read the counts and bind the symbols: the next stage is planned at the true sizes
+    if (cudaMemcpyAsync(counts.data(), static_cast<const char*>(arena) + 256, counts.size() * 8, cudaMemcpyDeviceToHost, static_cast<cudaStream_t>(stream)) != cudaSuccess ||
+        cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) { *err = "cannot read the run-time counts"; return E_CUDA; }
+    for (int r = 0; r < n_req; ++r)
+      for (int a : st.newly) rt[r].push_back({a, counts[static_cast<size_t>(a) * n_req + r]});
+  }
+  if (info) {
+    info[0] = std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t0).count();
+    info[1] = launches;
+    info[2] = stages;
+    info[3] = static_cast<int64_t>(peak_extent);
+    info[4] = plan_ns;
   }
   return OK;
 }

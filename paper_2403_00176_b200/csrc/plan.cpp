@@ -43,9 +43,26 @@ Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* na
         return E_SHAPE_CONFLICT;
       }
     }
-  // all non-linear atoms once per request (children first), then every distinct extent expression once
-  // per request as a flat polynomial; tensors pick their extents from that table
   auto t1 = std::chrono::steady_clock::now();
+  Status es = evaluate_dims(out);
+  if (es != OK) return es;
+  if (prof) {
+    auto t3 = std::chrono::steady_clock::now();
+    auto us = [](auto a, auto b) { return std::chrono::duration<double, std::micro>(b - a).count(); };
+    fprintf(stderr, "[sod2] bind: %zu assertions %.1f us, %zu extent expressions and %zu tensors %.1f us\n", g.asserts.size(), us(t0, t1),
+            c->dim_exprs.size(), g.tensors.size(), us(t1, t3));
+  }
+  return OK;
+}
+
+// Extents of every tensor for every request from the bound symbol values (out->vals): all non-linear atoms once per
+// request (children first), then every distinct extent expression once per request as a flat polynomial; tensors
+// pick their extents from that table.  An extent that depends on an unbound run-time symbol takes its static
+// upper bound.
+Status evaluate_dims(Binding* out) {
+  const Compiled* c = out->c;
+  const Graph& g = c->g;
+  const int n_req = out->n_req;
   const size_t U = c->dim_exprs.size();
   std::vector<int64_t> uval(static_cast<size_t>(n_req) * U);
   std::vector<char> uok(static_cast<size_t>(n_req) * U);
@@ -61,7 +78,6 @@ Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* na
       uok[r * U + u] = ok;
     }
   }
-  auto t2 = std::chrono::steady_clock::now();
   out->dims.reset(g.tensors.size(), n_req);
   for (size_t t = 0; t < g.tensors.size(); ++t) {
     const ShapeVal& s = g.tensors[t].S;
@@ -83,13 +99,21 @@ Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* na
       }
     }
   }
-  if (prof) {
-    auto t3 = std::chrono::steady_clock::now();
-    auto us = [](auto a, auto b) { return std::chrono::duration<double, std::micro>(b - a).count(); };
-    fprintf(stderr, "[sod2] bind: %zu assertions %.1f us, %zu extent expressions %.1f us, %zu tensors %.1f us\n", g.asserts.size(), us(t0, t1), U,
-            us(t1, t2), g.tensors.size(), us(t2, t3));
-  }
   return OK;
+}
+
+// A binding with some run-time symbols bound to the counts their operators produced (exact handling of
+// execution-determined extents): the same user symbols, `rt_vals[r]` = (atom, value) pairs for request r.
+Status rebind_runtime(const Binding& base, const std::vector<std::vector<std::pair<int, int64_t>>>& rt_vals, Binding* out) {
+  out->c = base.c;
+  out->n_req = base.n_req;
+  out->vals = base.vals;
+  for (int r = 0; r < base.n_req && r < static_cast<int>(rt_vals.size()); ++r)
+    for (auto& av : rt_vals[r]) {
+      if (av.first < 0 || av.first >= static_cast<int>(out->vals[r].size()) || av.second < 0) { out->err = "bad run-time symbol value"; return E_BAD_DIM; }
+      out->vals[r][av.first] = av.second;
+    }
+  return evaluate_dims(out);
 }
 
 namespace {
@@ -335,11 +359,17 @@ struct Planner {
     // header: status word (256 B) + one 8-byte count slot per (runtime symbol, request)
     // ... + the row-block counters of the GEMM chains
     p.chain_counter_off = (256 + 8 * g.cx.atoms.size() * static_cast<size_t>(p.n_req) + 15) & ~size_t(15);
-    const size_t HEADER = (p.chain_counter_off + 4 * p.chain_counter_words + 255) & ~size_t(255);
-    p.header_clear_bytes = p.chain_counter_words ? HEADER : 256;
+    const size_t HEADER0 = (p.chain_counter_off + 4 * p.chain_counter_words + 255) & ~size_t(255);
+    p.header_clear_bytes = p.chain_counter_words ? HEADER0 : 256;
+    // staged (exact) plans keep the group scratch and the Switch index lists at fixed places right behind the
+    // header, so that they do not move when a later stage plans the tensors again
+    p.header_end = HEADER0;
+    const size_t HEADER = HEADER0 + p.front_reserve;
     std::vector<int> ids;
     for (size_t t = 0; t < p.roots.size(); ++t)
-      if (p.roots[t].where == RootBuf::ARENA && p.roots[t].def_step >= 0) ids.push_back(static_cast<int>(t));
+      if (p.roots[t].where == RootBuf::ARENA && p.roots[t].def_step >= 0 && p.roots[t].def_step <= p.place_until_step &&
+          p.roots[t].last_step >= p.place_from_step)
+        ids.push_back(static_cast<int>(t));
     auto sz = [&](int t) { return (static_cast<size_t>(p.roots[t].bytes) + 255) & ~size_t(255); };
     // scratch of groups is planned like a tensor living for exactly that step
     std::vector<size_t> live(steps + 1, 0);
@@ -379,9 +409,20 @@ struct Planner {
       placed.push_back({best_off, need, R.def_step, R.last_step});
     };
     std::vector<char> done(p.roots.size(), 0);
+    // 0. tensors an earlier stage has already placed (and filled) stay where they are
+    for (auto& pin : p.pinned) {
+      const int t = pin.first;
+      if (t < 0 || t >= static_cast<int>(p.roots.size()) || p.roots[t].where != RootBuf::ARENA || p.roots[t].def_step < 0) continue;
+      if (std::find(ids.begin(), ids.end(), t) == ids.end()) continue;
+      if (pin.second < HEADER) return fail(E_INTERNAL, "pinned tensor inside the arena header");
+      p.roots[t].arena_off = pin.second;
+      placed.push_back({pin.second, sz(t), p.roots[t].def_step, p.roots[t].last_step});
+      top = std::max(top, pin.second + sz(t));
+      done[t] = 1;
+    }
     // 1. live set at the peak, in (def step, id) order
     std::vector<int> at_peak;
-    for (int t : ids) if (p.roots[t].def_step <= peak && p.roots[t].last_step >= peak) at_peak.push_back(t);
+    for (int t : ids) if (!done[t] && p.roots[t].def_step <= peak && p.roots[t].last_step >= peak) at_peak.push_back(t);
     std::sort(at_peak.begin(), at_peak.end(), [&](int x, int y) { return std::make_pair(p.roots[x].def_step, x) < std::make_pair(p.roots[y].def_step, y); });
     for (int t : at_peak) { place(t, true); done[t] = 1; }
     // 2. forward from the peak
@@ -398,7 +439,7 @@ struct Planner {
     // results outlive their large intermediates), the walk above fragments.  If it ended more than 2 %
     // above the live peak, a second placement is tried, largest tensor first at the lowest offset
     // that is free over its lifetime, and the smaller arena is kept.
-    if (!(c.flags & OPT_NO_REUSE) && top - HEADER > p.peak_live_bytes + p.peak_live_bytes / 50) {
+    if (p.pinned.empty() && !(c.flags & OPT_NO_REUSE) && top - HEADER > p.peak_live_bytes + p.peak_live_bytes / 50) {
       std::vector<size_t> first_off(ids.size());
       for (size_t i = 0; i < ids.size(); ++i) first_off[i] = p.roots[ids[i]].arena_off;
       const size_t first_top = top;

@@ -100,6 +100,11 @@ class Prepared:
         return self.plan.run_graph([t.data_ptr() for t in self.in_dev], [t.data_ptr() for t in self.out_dev],
                                    self.arena.data_ptr(), self.arena.numel(), self.s.stream)
 
+    def run_exact(self) -> B.RunInfo:
+        """The inference with counts read back and the remaining sub-graphs planned again at their true sizes."""
+        return self.plan.run_exact([t.data_ptr() for t in self.in_dev], [t.data_ptr() for t in self.out_dev],
+                                   self.arena.data_ptr(), self.arena.numel(), self.s.stream)
+
     def check_device_status(self):
         self.plan.device_status(self.arena.data_ptr(), self.s.stream)
 

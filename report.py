@@ -146,6 +146,24 @@ def measure(cfg: int, reps: int, device: str = "cuda:0", opt_flags: int = 0):
         single_ms = float(np.median([timed(p1.run, 10) for p1 in singles]))
         empty_ms = timed(lambda: B.sod2_launch_empty(sess.stream), 50)
         extra = {"ms_one_request_per_inference": single_ms, "ms_empty_kernel": empty_ms, "ratio_to_empty_kernel": single_ms / empty_ms}
+    if cfg == 5:
+        # execution-determined extents handled exactly (counts read back, the rest planned again at the true sizes)
+        # beside the default bounded form: wall time of the call (it synchronises the stream at every stage)
+        for p in preps:
+            p.run_exact()
+        torch.cuda.synchronize(dev)
+        ex = []
+        for i in range(max(5, reps // 2)):
+            flush.fill_(i & 0xFF)
+            torch.cuda.synchronize(dev)
+            p = preps[i % len(preps)]
+            t0 = time.perf_counter()
+            info = p.run_exact()
+            torch.cuda.synchronize(dev)
+            ex.append(((time.perf_counter() - t0) * 1e3, info.reserved[2], info.reserved[3], info.reserved[4] / 1e6))
+        extra = {"exact_edo": {"ms_wall": float(np.median([e[0] for e in ex])), "stages": int(ex[0][1]),
+                               "arena_bytes": int(np.median([e[2] for e in ex])), "bind_plan_ms": float(np.median([e[3] for e in ex])),
+                               "bounded_arena_bytes": int(preps[0].plan.arena_bytes)}}
     # per-group roofline on the first batch
     rep = group_report(preps[0], hbm, tf, reps=5)
     kinds = kind_summary(rep)

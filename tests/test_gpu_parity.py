@@ -768,6 +768,44 @@ def test_cfg5_all_skip_and_all_execute():
         assert np.all(gates == (1 if bias_val > 0 else 0))
 
 
+def test_cfg5_exact_staging_matches_the_bounded_run():
+    # Execution-determined extents handled exactly (counts read back after every Switch, the remaining sub-graphs
+    # planned again at their true sizes around the tensors in place) against the default bounded form (counts stay on
+    # the device, memory planned at the upper bound): same kernels, same bits, one stage per Switch, no larger arena
+    cases = [(WL.cfg5(B=6, side=32, widths=(64, 128), per_stage=2), 4, 0), (WL.cfg5(B=6, side=32, widths=(64, 128), per_stage=3), 6, B.OPT_COPY_REGROUP),
+             (WL.cfg5(B=45, side=32, widths=(64,), per_stage=2, calibrated=False), 2, 0)]
+    for bias_val in (-50.0, 50.0):                       # nothing executes (empty sub-batches) / everything executes
+        wl = WL.cfg5(B=4, side=32, widths=(64, 128), per_stage=2)
+        for k in list(wl.consts):
+            if k.endswith(".gb"):
+                wl.consts[k] = np.full_like(wl.consts[k], bias_val)
+        cases.append((wl, 4, 0))
+    for wl, n_blocks, flags in cases:
+        reqs = wl.batch(0)
+        s, p, ref = run_batch(wl, reqs, opt_flags=flags)
+        info = p.run_exact()
+        p.check_device_status()
+        got = p.outputs()
+        assert info.reserved[2] == n_blocks + 1, info.reserved[2]          # the first stage + one per Switch
+        assert 0 < info.reserved[3] <= p.plan.arena_bytes
+        for name in ref[0]:
+            assert np.array_equal(ref[0][name], got[0][name]), (wl.name, name)
+        # and again (the stages leave nothing behind), then the bounded form on the same buffers
+        p.run_exact()
+        again = p.outputs()
+        p.run()
+        bounded = p.outputs()
+        for name in ref[0]:
+            assert np.array_equal(ref[0][name], again[0][name]) and np.array_equal(ref[0][name], bounded[0][name])
+    # a graph without execution-determined operators is one stage
+    wl2, reqs2 = _encoder_edge(layers=1)
+    s2, p2, o2 = run_batch(wl2, reqs2[:4])
+    i2 = p2.run_exact()
+    assert i2.reserved[2] == 1
+    for a, b_ in zip(o2, p2.outputs()):
+        assert np.array_equal(a["y"], b_["y"])
+
+
 def test_cfg5_full_depth_reduced_batch_lockstep():
     # all 16 blocks and widths 64..512 at 224x224, 4 images (the oracle needs ~100 GFLOP in fp64)
     wl = WL.cfg5(B=4)
