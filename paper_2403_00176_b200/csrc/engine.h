@@ -36,6 +36,11 @@ enum class GKind {
   SWITCH,
   COMBINE,
   LAYOUT,      // NCHW <-> channels-last storage change at the ABI boundary of convolution graphs (act: 0 to, 1 from)
+  // stand-alone forms of operators that otherwise run inside fused groups (unfused mode, or outside their pattern)
+  BMM,         // MatMul of two activations (batched, strided operands)
+  SUMSQ,       // ReduceSumSquare over the last axis
+  TOPK,        // TopK over the last axis: values + int64 indices
+  GATHER,      // Gather along one axis by an int64 index tensor computed on the device
   UNSUPPORTED
 };
 const char* gkind_name(GKind k);

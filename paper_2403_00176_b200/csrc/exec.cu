@@ -18,6 +18,7 @@
 #include "gemm_chain_tcgen05.cuh"
 #include "kernels_compact.cuh"
 #include "kernels_rows.cuh"
+#include "kernels_unfused.cuh"
 #include "tmap.h"
 
 namespace sod2 {
@@ -979,6 +980,118 @@ struct Builder {
     return OK;
   }
 
+  // ------------------------------------------------------------------------------ stand-alone operators (unfused mode)
+  Status build_bmm(int gi, const Group& G) {
+    const Tensor& A = g.tensors[G.a];
+    if (A.dtype != g.tensors[G.w].dtype || A.dtype != g.tensors[G.out].dtype || (A.dtype != DType::BF16 && A.dtype != DType::F32))
+      return fail(E_UNSUPPORTED_OP, "MatMul of two activations: operands and result must share one float type");
+    for (int r = 0; r < p.n_req; ++r) {
+      const View &va = p.views[G.a][r], &vb = p.views[G.w][r], &vc = p.views[G.out][r];
+      const int rc = static_cast<int>(vc.dims.size());
+      if (rc < 2 || rc > 4 || va.dims.size() < 2 || vb.dims.size() < 2) return fail(E_UNSUPPORTED_OP, "MatMul of two activations supports ranks 2..4");
+      if (numel(vc.dims) == 0) continue;
+      k::BmmParams bp{};
+      bp.is_bf16 = A.dtype == DType::BF16;
+      bp.M = static_cast<int>(vc.dims[rc - 2]); bp.N = static_cast<int>(vc.dims[rc - 1]); bp.K = static_cast<int>(va.dims.back());
+      bp.B0 = rc >= 4 ? static_cast<int>(vc.dims[0]) : 1;
+      bp.B1 = rc >= 3 ? static_cast<int>(vc.dims[rc - 3]) : 1;
+      // strides of (b0, b1, row, col) per operand; batch dims right-aligned, extent-1 dims broadcast
+      auto fill = [&](const View& v, long long* st) {
+        const int rk = static_cast<int>(v.dims.size());
+        st[2] = v.strides[rk - 2]; st[3] = v.strides[rk - 1];
+        st[1] = (rk >= 3 && v.dims[rk - 3] != 1) ? v.strides[rk - 3] : 0;
+        st[0] = (rk >= 4 && v.dims[rk - 4] != 1) ? v.strides[rk - 4] : 0;
+      };
+      fill(va, bp.as); fill(vb, bp.bs); fill(vc, bp.cs);
+      if (vb.dims[vb.dims.size() - 2] != bp.K) return fail(E_SHAPE_CONFLICT, "MatMul inner dims differ");
+      Ptr pa = ptr_of(G.a, r), pb = ptr_of(G.w, r), pc = ptr_of(G.out, r);
+      add(gi, 1, [=](const RunCtx& x) mutable {
+        bp.a = x.resolve(pa); bp.b = x.resolve(pb); bp.c = x.resolve(pc);
+        k::bmm_strided<<<dim3((bp.N + 15) / 16, (bp.M + 15) / 16, bp.B0 * bp.B1), 256, 0, x.stream>>>(bp);
+        return cudaGetLastError();
+      });
+    }
+    return OK;
+  }
+  Status build_sumsq(int gi, const Group& G) {
+    const Tensor &X = g.tensors[G.a], &O = g.tensors[G.out];
+    for (int r = 0; r < p.n_req; ++r) {
+      const View &vx = p.views[G.a][r], &vo = p.views[G.out][r];
+      if (!vx.contiguous() || !vo.contiguous()) return fail(E_UNSUPPORTED_OP, "ReduceSumSquare needs contiguous operands");
+      if (numel(vx.dims) == 0) continue;
+      k::SumSqParams sp{};
+      sp.D = static_cast<int>(vx.dims.back());
+      sp.rows = numel(vx.dims) / sp.D;
+      sp.in_bf16 = X.dtype == DType::BF16; sp.out_bf16 = O.dtype == DType::BF16;
+      Ptr px = ptr_of(G.a, r), po = ptr_of(G.out, r);
+      add(gi, 1, [=](const RunCtx& x) mutable {
+        sp.x = x.resolve(px); sp.out = x.resolve(po);
+        k::reduce_sumsq_rows<<<static_cast<unsigned>((sp.rows + 7) / 8), 256, 0, x.stream>>>(sp);
+        return cudaGetLastError();
+      });
+    }
+    return OK;
+  }
+  Status build_topk_rows(int gi, const Group& G) {
+    const Tensor& X = g.tensors[G.a];
+    if (X.dtype != DType::BF16 && X.dtype != DType::F32) return fail(E_UNSUPPORTED_OP, "TopK ranks float scores");
+    for (int r = 0; r < p.n_req; ++r) {
+      // either output may be unused by the rest of the graph (then it has no storage)
+      const bool has_v = !p.views[G.out].empty(), has_i = !p.views[G.out2].empty();
+      if (!has_v && !has_i) continue;
+      const View& vx = p.views[G.a][r];
+      const View& vk = has_i ? p.views[G.out2][r] : p.views[G.out][r];
+      if (!vx.contiguous() || (has_v && !p.views[G.out][r].contiguous()) || (has_i && !p.views[G.out2][r].contiguous()))
+        return fail(E_UNSUPPORTED_OP, "TopK needs contiguous operands");
+      if (numel(vx.dims) == 0 || numel(vk.dims) == 0) continue;
+      k::TopkRowsParams tp{};
+      tp.n = static_cast<int>(vx.dims.back());
+      tp.k = static_cast<int>(vk.dims.back());
+      tp.rows = numel(vx.dims) / tp.n;
+      tp.largest = G.act2; tp.by_value = G.act; tp.is_bf16 = X.dtype == DType::BF16;
+      if (tp.k > tp.n) return fail(E_BAD_DIM, "TopK: k exceeds the axis length");
+      const size_t smem = static_cast<size_t>(tp.n) * 8;
+      if (smem > 200 * 1024) return fail(E_UNSUPPORTED_OP, "TopK: axis too long for the shared-memory score table");
+      Ptr px = ptr_of(G.a, r), pv = has_v ? ptr_of(G.out, r) : Ptr(), pi = has_i ? ptr_of(G.out2, r) : Ptr();
+      add(gi, 1, [=](const RunCtx& x) mutable {
+        tp.s = x.resolve(px);
+        tp.vals = has_v ? x.resolve(pv) : nullptr;
+        tp.idx = has_i ? reinterpret_cast<long long*>(x.resolve(pi)) : nullptr;
+        if (smem > 48 * 1024) { static bool once = (cudaFuncSetAttribute(k::topk_rows, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024), true); (void)once; }
+        k::topk_rows<<<static_cast<unsigned>(std::min<long long>(tp.rows, 148 * 4)), 256, smem, x.stream>>>(tp);
+        return cudaGetLastError();
+      });
+    }
+    return OK;
+  }
+  Status build_gather(int gi, const Group& G) {
+    const Tensor& X = g.tensors[G.a];
+    for (int r = 0; r < p.n_req; ++r) {
+      const View &vx = p.views[G.a][r], &vi = p.views[G.k][r], &vo = p.views[G.out][r];
+      if (!vx.contiguous() || !vi.contiguous() || !vo.contiguous()) return fail(E_UNSUPPORTED_OP, "Gather needs contiguous operands");
+      if (numel(vo.dims) == 0) continue;
+      const int rk = static_cast<int>(vx.dims.size());
+      const int ax = G.stride < 0 ? G.stride + rk : G.stride;
+      if (ax < 0 || ax >= rk) return fail(E_BAD_DIM, "Gather axis out of range");
+      k::GatherParams gp{};
+      gp.outer = 1; gp.inner = 1;
+      for (int i = 0; i < ax; ++i) gp.outer *= vx.dims[i];
+      for (int i = ax + 1; i < rk; ++i) gp.inner *= vx.dims[i];
+      gp.n_in = vx.dims[ax];
+      gp.n_idx = numel(vi.dims);
+      gp.esz = dtype_size(X.dtype);
+      if (gp.esz != 2 && gp.esz != 4 && gp.esz != 8) return fail(E_UNSUPPORTED_OP, "Gather element size");
+      Ptr px = ptr_of(G.a, r), pi = ptr_of(G.k, r), po = ptr_of(G.out, r);
+      const long long total = gp.outer * gp.n_idx * gp.inner;
+      add(gi, 1, [=](const RunCtx& x) mutable {
+        gp.x = x.resolve(px); gp.idx = reinterpret_cast<const long long*>(x.resolve(pi)); gp.out = x.resolve(po);
+        k::gather_axis<<<static_cast<unsigned>(std::max<long long>(1, std::min<long long>((total + 255) / 256, 148 * 16))), 256, 0, x.stream>>>(gp);
+        return cudaGetLastError();
+      });
+    }
+    return OK;
+  }
+
   // ------------------------------------------------------------------------------ top-k keep
   Status build_topk(int gi, const Group& G) {
     if (g.tensors[G.a].dtype != DType::BF16) return fail(E_UNSUPPORTED_OP, "top-k keep is bf16 only");
@@ -1874,7 +1987,8 @@ struct Builder {
     }
     p.uses_header = false;
     for (const Group& G : c.groups)
-      if (!((G.kind == GKind::GEMM && g.tensors[G.a].dtype == DType::F32) || G.kind == GKind::CHAIN)) p.uses_header = true;
+      if (!((G.kind == GKind::GEMM && g.tensors[G.a].dtype == DType::F32) || G.kind == GKind::CHAIN || G.kind == GKind::BMM ||
+            G.kind == GKind::SUMSQ || G.kind == GKind::TOPK || G.kind == GKind::GATHER)) p.uses_header = true;
     for (size_t gi = 0; gi < c.groups.size(); ++gi) {
       const Group& G = c.groups[gi];
       Status s = OK;
@@ -1898,6 +2012,10 @@ struct Builder {
         case GKind::GATE: s = build_gate(static_cast<int>(gi), G); break;
         case GKind::SWITCH: s = build_switch(static_cast<int>(gi), G); break;
         case GKind::COMBINE: s = build_combine(static_cast<int>(gi), G); break;
+        case GKind::BMM: s = build_bmm(static_cast<int>(gi), G); break;
+        case GKind::SUMSQ: s = build_sumsq(static_cast<int>(gi), G); break;
+        case GKind::TOPK: s = build_topk_rows(static_cast<int>(gi), G); break;
+        case GKind::GATHER: s = build_gather(static_cast<int>(gi), G); break;
         default: return fail(E_UNSUPPORTED_OP, std::string("no executor yet for group kind ") + gkind_name(G.kind));
       }
       if (s != OK) return s;

@@ -26,6 +26,10 @@ const char* gkind_name(GKind k) {
     case GKind::SWITCH: return "switch";
     case GKind::COMBINE: return "combine";
     case GKind::LAYOUT: return "layout";
+    case GKind::BMM: return "bmm";
+    case GKind::SUMSQ: return "sumsq";
+    case GKind::TOPK: return "topk";
+    case GKind::GATHER: return "gather";
     default: return "unsupported";
   }
 }
@@ -477,7 +481,8 @@ struct Fuser {
           absorb_epilogue(G, n.outs[0], false);
           finish(G);
         } else if (!try_attention(nid)) {
-          Group G; G.nodes = {nid}; G.why = "MatMul of two activations outside the attention pattern"; G.out = n.outs[0];
+          // MatMul of two activations outside the attention pattern (or in the unfused mode): stand-alone kernel
+          Group G; G.kind = GKind::BMM; G.nodes = {nid}; G.a = n.ins[0]; G.w = n.ins[1]; G.out = n.outs[0];
           finish(G);
         }
       } else if (op == "Conv") {
@@ -499,7 +504,13 @@ struct Fuser {
           finish(G);
         } else chain_group(nid);
       } else if (op == "ReduceSumSquare") {
-        if (!try_topk_keep(nid)) { Group G; G.nodes = {nid}; G.why = "standalone ReduceSumSquare"; G.out = n.outs[0]; finish(G); }
+        if (!try_topk_keep(nid)) {
+          Group G; G.nodes = {nid}; G.out = n.outs[0]; G.a = n.ins[0];
+          const int rk = g.tensors[n.ins[0]].S.rank;
+          if (n.attr_i("axis", -1) == -1 || n.attr_i("axis", -1) == rk - 1) G.kind = GKind::SUMSQ;
+          else G.why = "ReduceSumSquare over an axis other than the last";
+          finish(G);
+        }
       } else if (op == "NonZero") {
         Group G; G.kind = GKind::NONZERO; G.nodes = {nid}; G.a = n.ins[0]; G.out = n.outs[0]; finish(G);
       } else if (op == "GlobalAveragePool") {
@@ -512,6 +523,19 @@ struct Fuser {
         finish(G);
       } else if (op == "Combine") {
         Group G; G.kind = GKind::COMBINE; G.nodes = {nid}; G.a = n.ins[0]; G.res = n.ins[1]; G.gate = n.ins[2]; G.out = n.outs[0];
+        finish(G);
+      } else if (op == "TopK" && n.outs.size() == 2) {
+        Group G; G.nodes = {nid}; G.a = n.ins[0]; G.out = n.outs[0]; G.out2 = n.outs[1];
+        const int rk = g.tensors[n.ins[0]].S.rank;
+        if (n.attr_i("axis", -1) == -1 || n.attr_i("axis", -1) == rk - 1) {
+          G.kind = GKind::TOPK;
+          G.act = n.attr_s("order", "value") == "value";     // 1: by rank, 0: kept positions ascending
+          G.act2 = static_cast<int>(n.attr_i("largest", 1));
+        } else G.why = "TopK over an axis other than the last";
+        finish(G);
+      } else if (op == "Gather" && g.tensors[n.ins[1]].dtype == DType::I64) {
+        Group G; G.kind = GKind::GATHER; G.nodes = {nid}; G.a = n.ins[0]; G.k = n.ins[1]; G.out = n.outs[0];
+        G.stride = static_cast<int>(n.attr_i("axis", 0));
         finish(G);
       } else {
         Group G; G.nodes = {nid}; G.why = "no kernel for " + op; G.out = n.outs.empty() ? -1 : n.outs[0];

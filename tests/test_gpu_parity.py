@@ -101,6 +101,42 @@ def test_cfg1_unfused_execution_equals_fused_and_oracle():
         assert O.rel_err(o1[r]["Y"], o0[r]["Y"]) <= F32_TOL
 
 
+def test_unfused_execution_of_the_encoder_and_the_pruning_stack():
+    # SOD2_OPT_NO_FUSION: one kernel per operator, every intermediate materialised in the graph's storage type
+    # (attention as MatMul, Mul, Softmax, MatMul; pruning as ReduceSumSquare, TopK, Gather).  Every operator output
+    # in lock-step with the oracle; the encoder's final output against the fused run.
+    wl, reqs = _encoder_edge()
+    reqs = [reqs[i] for i in (0, 3, 7, 10)]
+    s0, p0, o0 = run_batch(wl, reqs)
+    s1, p1, o1 = run_batch(wl, reqs, opt_flags=B.OPT_NO_FUSION | B.OPT_NO_REUSE)
+    kinds = [s1.graph.group_info(i)["kind"] for i in range(s1.graph.num_groups())]
+    assert "attention" not in kinds and kinds.count("bmm") == 4 and s1.graph.num_groups() > 2 * s0.graph.num_groups()
+    for r, req in enumerate(reqs):
+        errs = lockstep(wl, s1, p1, o1, r, BF16_TOL)
+        assert len(errs) >= 30
+        bad = {k: v for k, v in errs.items() if not (isinstance(v, float) and v <= BF16_TOL)}
+        assert not bad, (req.syms, bad)
+        # about twice as many storage roundings as the fused run: compare with the noise of unfused bf16 storage
+        ref = _oracle_out(wl, req, "y")
+        noisy = O.run(wl.ir, wl.consts, req.inputs, storage_round=lambda a: bf16_round(a.astype(np.float32)).astype(np.float64))["y"]
+        assert O.rel_err(o1[r]["y"], ref) <= max(BF16_TOL, 2 * O.rel_err(noisy, ref)), req.syms
+    wl3 = WL.cfg3(layers=2, D=128, H=2, F=256, n_requests=1, nmin=4, nmax=800)
+    rng = np.random.default_rng(17)
+    reqs3 = [Request({"N0": n}, {"x": bf16_round(rng.standard_normal((1, n, 128)).astype(np.float32))}) for n in (4, 65, 300)]
+    s3, p3, o3 = run_batch(wl3, reqs3, opt_flags=B.OPT_NO_FUSION | B.OPT_NO_REUSE)
+    kinds3 = [s3.graph.group_info(i)["kind"] for i in range(s3.graph.num_groups())]
+    assert kinds3.count("sumsq") == 2 and kinds3.count("topk") == 2 and kinds3.count("gather") == 2 and "topk_keep" not in kinds3
+    for r, req in enumerate(reqs3):
+        # the kept indices are decided on the stored (bf16) scores: bit-exact against the oracle's TopK of those scores
+        errs = lockstep(wl3, s3, p3, o3, r, BF16_TOL)
+        bad = {k: v for k, v in errs.items() if not (isinstance(v, float) and v <= BF16_TOL)}
+        assert errs and not bad, (req.syms, bad)
+        n = req.syms["N0"]
+        for l in range(2):
+            n = (7 * n + 9) // 10
+            assert o3[r][f"idx{l}"].shape == (1, n) and np.all(np.diff(o3[r][f"idx{l}"][0]) > 0)
+
+
 def test_bounded_wait_runs_out_and_is_reported():
     # Every device-side wait gives up after a bounded number of polls, raises the status word and returns.  The
     # self-test kernel waits on a barrier that nothing ever arrives on, with a limit of a few thousand polls: it must
