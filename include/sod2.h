@@ -47,6 +47,7 @@ typedef enum {
 #define SOD2_OPT_MULTI_VERSION 64u /* fuse elementwise chains across broadcasts RDP cannot resolve: 2^d fused versions (Section 4.2), the version (a stride table) chosen at bind time */
 #define SOD2_OPT_NO_SEP 32u /* groups run in their default topological order: no static execution planning (Section 4.3) */
 #define SOD2_OPT_LN_FOLD 128u /* a LayerNorm between bf16 GEMMs is folded into its neighbours (Section 4.2: fusion removes the materialised intermediate): the producing GEMM writes per-row statistics, the consuming GEMMs read the raw rows and normalise in their epilogues, the normalised tensor is never stored.  Opt-in: measured slower on the encoder workloads, where the LayerNorm kernel runs beside the next GEMM's pipeline fill */
+#define SOD2_OPT_GUARD_BANDS 512u /* debugging aid: every arena tensor gets a slot of its own (a band another tensor may cover at another time proves nothing) with 256 bytes behind it, also behind the scratch regions (sod2_plan_poison_arena / sod2_plan_check_guards) */
 #define SOD2_OPT_GEMM_CHAIN 256u /* consecutive GEMM groups that depend on each other row block by row block run as one persistent kernel with per-row-block dependency counters in the arena header (their operands stay live over the whole chain).  Opt-in: measured slower than one launch per GEMM at a few thousand rows */
 #define SOD2_OPT_SPLITK_LN 4u /* bf16 GEMM (+bias, +residual) -> LayerNorm as one group: split-K GEMM into fp32 slabs + finishing kernel */
 
@@ -137,6 +138,18 @@ sod2_status sod2_run_graph(sod2_plan_t* p, const void* const* inputs, void* cons
  * Errors as sod2_run, plus SOD2_E_ARENA_TOO_SMALL if a stage planned around the tensors in place does not fit. */
 sod2_status sod2_run_exact(sod2_plan_t* p, const void* const* inputs, void* const* outputs, void* arena,
                            size_t arena_bytes, void* cuda_stream, sod2_run_info* info);
+
+/* Debugging aids for graphs created with SOD2_OPT_GUARD_BANDS (they stand in for a memory checker: every kernel of
+ * the library takes its bounds from the plan, Section 4.4.1, so a store past the end of a planned tensor is a
+ * planning or kernel defect).  sod2_plan_poison_arena fills the arena behind its header with 0xFF bytes (NaN in bf16
+ * and fp32: a read of memory that nothing wrote shows up in the results); call it before sod2_run.
+ * sod2_plan_check_guards, after the run, counts the 256-byte bands behind tensors and scratch regions that no longer
+ * hold those bytes (*n_damaged) and names the tensor behind which the lowest damaged band lies (first_name, host
+ * buffer, may be NULL).  It overwrites header bytes 16..127 and synchronises cuda_stream.  Errors:
+ * SOD2_E_INVALID_ARG (graph without the option), SOD2_E_ARENA_TOO_SMALL, SOD2_E_CUDA. */
+sod2_status sod2_plan_poison_arena(sod2_plan_t* p, void* arena, size_t arena_bytes, void* cuda_stream);
+sod2_status sod2_plan_check_guards(sod2_plan_t* p, void* arena, void* cuda_stream, int* n_damaged, char* first_name,
+                                   size_t first_name_len);
 
 /* Measurement aid: the same inference with CUDA events recorded on cuda_stream around every launch.
  * Synchronises the stream and returns the device time of each fused group in group_ms[n_groups]

@@ -25,6 +25,7 @@ OPT_NO_SEP = 32
 OPT_MULTI_VERSION = 64
 OPT_LN_FOLD = 128
 OPT_GEMM_CHAIN = 256
+OPT_GUARD_BANDS = 512
 DYN_CLASS = ["ISDO", "ISDOS", "ISVDOS", "EDO"]
 
 
@@ -61,6 +62,8 @@ def _load() -> C.CDLL:
         "sod2_run_timed": [vp, P(vp), P(vp), vp, sz, vp, P(C.c_float), i32],
         "sod2_run_timed_repeat": [vp, P(vp), P(vp), vp, sz, vp, i32, P(C.c_float), i32],
         "sod2_plan_device_status": [vp, vp, vp],
+        "sod2_plan_poison_arena": [vp, vp, sz, vp],
+        "sod2_plan_check_guards": [vp, vp, vp, P(i32), cp, sz],
         "sod2_graph_tensor_info": [vp, cp, P(i32), P(i32), cp, sz],
         "sod2_graph_tensor_value": [vp, cp, cp, sz],
         "sod2_graph_tensor_dtype": [vp, cp, P(i32)],
@@ -98,7 +101,7 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = ["sod2_graph_create", "sod2_graph_destroy", "sod2_graph_set_const", "sod2_graph_prepack_bytes",
            "sod2_graph_prepack", "sod2_bind_dims", "sod2_binding_destroy", "sod2_plan", "sod2_plan_destroy", "sod2_graph_set_plan_cache", "sod2_plan_cached",
-           "sod2_run", "sod2_run_graph", "sod2_run_exact", "sod2_run_timed", "sod2_run_timed_repeat", "sod2_plan_device_status", "sod2_graph_tensor_info", "sod2_graph_tensor_value", "sod2_graph_tensor_dtype",
+           "sod2_run", "sod2_run_graph", "sod2_run_exact", "sod2_run_timed", "sod2_run_timed_repeat", "sod2_plan_device_status", "sod2_plan_poison_arena", "sod2_plan_check_guards", "sod2_graph_tensor_info", "sod2_graph_tensor_value", "sod2_graph_tensor_dtype",
            "sod2_graph_num_ops", "sod2_graph_op_info", "sod2_graph_num_groups", "sod2_graph_group_info",
            "sod2_graph_num_subgraphs", "sod2_graph_rdp_sweeps", "sod2_classify", "sod2_graph_reanalyse", "sod2_graph_order_info",
            "sod2_binding_shape", "sod2_plan_slot", "sod2_plan_instance_offset", "sod2_plan_memory", "sod2_plan_group_cost", "sod2_plan_tensor_strides",
@@ -326,6 +329,17 @@ class Plan:
         else:
             _check(lib.sod2_run_timed(self.h, ins, outs, C.c_void_p(arena), arena_bytes, C.c_void_p(stream), ms, n), self.h)
         return list(ms[:n])
+
+    def poison_arena(self, arena: int, arena_bytes: int, stream: int):
+        """Fill the arena behind its header with 0xFF bytes (graphs created with OPT_GUARD_BANDS)."""
+        _check(lib.sod2_plan_poison_arena(self.h, C.c_void_p(arena), arena_bytes, C.c_void_p(stream)), self.h)
+
+    def check_guards(self, arena: int, stream: int):
+        """(damaged bands, name of the tensor behind which the lowest damaged band lies)."""
+        n = C.c_int()
+        buf = C.create_string_buffer(256)
+        _check(lib.sod2_plan_check_guards(self.h, C.c_void_p(arena), C.c_void_p(stream), C.byref(n), buf, 256), self.h)
+        return n.value, buf.value.decode()
 
     def device_status(self, arena: int, stream: int):
         _check(lib.sod2_plan_device_status(self.h, C.c_void_p(arena), C.c_void_p(stream)), self.h)

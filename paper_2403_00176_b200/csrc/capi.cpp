@@ -262,6 +262,24 @@ sod2_status sod2_run_exact(sod2_plan_t* p, const void* const* inputs, void* cons
   return st(s);
 }
 
+sod2_status sod2_plan_poison_arena(sod2_plan_t* p, void* arena, size_t arena_bytes, void* stream) {
+  if (!p || !arena) return SOD2_E_INVALID_ARG;
+  Status s = poison_arena(&p->p, arena, arena_bytes, stream);
+  if (s != OK) p->h.err = s == E_ARENA_TOO_SMALL ? "arena too small" : "cannot fill the arena";
+  return st(s);
+}
+
+sod2_status sod2_plan_check_guards(sod2_plan_t* p, void* arena, void* stream, int* n_damaged, char* first_name, size_t first_name_len) {
+  if (!p || !arena || !n_damaged) return SOD2_E_INVALID_ARG;
+  if (!(p->g->c.flags & OPT_GUARD_BANDS)) { p->h.err = "the graph was not created with SOD2_OPT_GUARD_BANDS"; return SOD2_E_INVALID_ARG; }
+  int bad = 0, first = -3;
+  Status s = check_guards(&p->p, arena, stream, &bad, &first);
+  if (s != OK) { p->h.err = "cannot check the guard bands"; return st(s); }
+  *n_damaged = bad;
+  copy_str(first >= 0 ? p->g->c.g.tensors[first].name : first == -1 ? "<group scratch>" : first == -2 ? "<index lists>" : "", first_name, first_name_len);
+  return SOD2_OK;
+}
+
 sod2_status sod2_run_timed(sod2_plan_t* p, const void* const* inputs, void* const* outputs, void* arena, size_t arena_bytes,
                            void* stream, float* group_ms, int n_groups) {
   if (!p || !inputs || !outputs || !arena) return SOD2_E_INVALID_ARG;

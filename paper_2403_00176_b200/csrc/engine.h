@@ -20,6 +20,7 @@ enum OptFlags : uint32_t {
   OPT_NO_SEP = 32u,     // groups run in their default topological order (no static execution planning)
   OPT_SPLITK_LN = 4u,   // a bf16 GEMM (+bias, +residual) followed by LayerNorm becomes one group: split-K GEMM + finishing kernel
   OPT_LN_FOLD = 128u,     // a LayerNorm between bf16 GEMMs is folded into their epilogues (the normalised tensor is never stored)
+  OPT_GUARD_BANDS = 512u, // 256 poison bytes behind every arena tensor and scratch region, checked after a run (sod2_plan_check_guards)
   OPT_GEMM_CHAIN = 256u,  // consecutive dependent GEMM groups run as one persistent kernel with row-block dependency counters
 };
 
@@ -288,6 +289,8 @@ struct Plan {
   // [group] run-time symbols (atom ids) whose counts are in the arena header once the group has run: a gate whose
   // kernel also partitions the sample ids, a Switch that partitions them itself, a NonZero
   std::vector<std::vector<int>> rt_syms_after;
+  // OPT_GUARD_BANDS: (arena offset of a 256-byte band, tensor it follows or -1 = scratch, -2 = index lists)
+  std::vector<std::pair<size_t, int>> guard_bands;
   std::string err;
   // device status word lives at arena offset 0 (first 256 bytes reserved)
   // CUDA graph of the whole launch sequence for one set of buffers (run_plan_graph)
@@ -322,6 +325,10 @@ Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* 
 // sizes fix the layout in front of the tensors); the arena must hold at least bounded->arena_bytes.
 Status run_exact(const Compiled* c, const Binding* b0, const Plan* bounded, const void* const* inputs, void* const* outputs, void* arena,
                  size_t arena_bytes, void* stream, int64_t* info, std::string* err);
+
+// Guard bands (OPT_GUARD_BANDS): fill the arena behind the header with 0xFF bytes; count the bands a run damaged.
+Status poison_arena(const Plan* p, void* arena, size_t arena_bytes, void* stream);
+Status check_guards(const Plan* p, void* arena, void* stream, int* n_bad, int* first_tensor);
 
 // Same as run_plan, with CUDA events around every launch; synchronises the stream and returns the
 // device time per group (ms).

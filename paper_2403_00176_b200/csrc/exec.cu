@@ -2030,10 +2030,13 @@ struct Builder {
       return OK;
     }
     // one scratch region shared by all groups (they run in stream order), after the tensors
+    const size_t band = (c.flags & OPT_GUARD_BANDS) ? 256 : 0;
     p.scratch_off.assign(2, p.arena_bytes);
     p.arena_bytes += (scratch_need + 255) & ~size_t(255);
+    if (band) { p.guard_bands.push_back({p.arena_bytes, -1}); p.arena_bytes += band; }
     p.scratch_off[1] = p.arena_bytes;     // index lists of Switch groups: live until their Combine
     p.arena_bytes += (aux_need + 255) & ~size_t(255);
+    if (band) { p.guard_bands.push_back({p.arena_bytes, -2}); p.arena_bytes += band; }
     return OK;
   }
 };
@@ -2314,6 +2317,63 @@ Status run_plan(Plan* p, const void* const* inputs, void* const* outputs, void* 
     info[0] = std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t0).count();
     info[1] = (step_lo <= 0 && step_hi >= (1 << 30)) ? p->gpu_launches : enqueued;
   }
+  return OK;
+}
+
+// ---- guard bands (OPT_GUARD_BANDS): the arena behind the header is filled with 0xFF bytes (NaN in bf16 and fp32, so
+// a read of memory nothing wrote shows in the results), and after a run every 256-byte band behind a tensor or scratch
+// region must still hold them: a kernel that stored past the end of its tensor has damaged the band behind it.
+namespace {
+struct GuardList { const size_t* off; int n; };
+__global__ void check_guard_bands(const char* arena, GuardList gl, unsigned long long* result) {
+  // one warp per band: 64 words of 4 bytes; result[0] = damaged bands, result[1] = lowest damaged band index
+  const int band = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (band >= gl.n) return;
+  const unsigned* w = reinterpret_cast<const unsigned*>(arena + gl.off[band]);
+  const bool bad = w[lane] != 0xFFFFFFFFu || w[lane + 32] != 0xFFFFFFFFu;
+  if (__any_sync(0xffffffffu, bad) && lane == 0) {
+    atomicAdd(result, 1ull);
+    atomicMin(result + 1, static_cast<unsigned long long>(band));
+  }
+}
+}  // namespace
+
+Status poison_arena(const Plan* p, void* arena, size_t arena_bytes, void* stream) {
+  if (arena_bytes < p->arena_bytes) return E_ARENA_TOO_SMALL;
+  const size_t from = p->header_end ? p->header_end : 256;
+  if (p->arena_bytes > from && cudaMemsetAsync(static_cast<char*>(arena) + from, 0xFF, p->arena_bytes - from, static_cast<cudaStream_t>(stream)) != cudaSuccess) return E_CUDA;
+  return OK;
+}
+
+// n_bad: damaged bands; first_tensor: tensor id behind which the lowest damaged band lies (-1 scratch, -2 index lists,
+// -3 none).  The library allocates no device memory: the band offsets reach the kernel through the arena header's
+// unused bytes 32..127, twelve at a time, and the result comes back through bytes 16..31.  Synchronises the stream.
+Status check_guards(const Plan* p, void* arena, void* stream, int* n_bad, int* first_tensor) {
+  *n_bad = 0;
+  *first_tensor = -3;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (p->guard_bands.empty()) return OK;
+  // header bytes 16..31 take the result, bytes 32..127 twelve band offsets at a time
+  char* hdr = static_cast<char*>(arena);
+  unsigned long long init[2] = {0ull, ~0ull};
+  if (cudaMemcpyAsync(hdr + 16, init, 16, cudaMemcpyHostToDevice, st) != cudaSuccess) return E_CUDA;
+  const int per = 12;
+  unsigned long long res[2] = {0, ~0ull};
+  unsigned long long total_bad = 0;
+  long long first_band = -1;
+  for (size_t b0 = 0; b0 < p->guard_bands.size(); b0 += per) {
+    size_t offs[per];
+    const int n = static_cast<int>(std::min<size_t>(per, p->guard_bands.size() - b0));
+    for (int i = 0; i < n; ++i) offs[i] = p->guard_bands[b0 + i].first;
+    if (cudaMemcpyAsync(hdr + 16, init, 16, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(hdr + 32, offs, sizeof(size_t) * n, cudaMemcpyHostToDevice, st) != cudaSuccess) return E_CUDA;
+    check_guard_bands<<<(n + 7) / 8, 256, 0, st>>>(hdr, GuardList{reinterpret_cast<const size_t*>(hdr + 32), n}, reinterpret_cast<unsigned long long*>(hdr + 16));
+    if (cudaMemcpyAsync(res, hdr + 16, 16, cudaMemcpyDeviceToHost, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) return E_CUDA;
+    total_bad += res[0];
+    if (res[0] && first_band < 0) first_band = static_cast<long long>(b0) + static_cast<long long>(res[1]);
+  }
+  *n_bad = static_cast<int>(total_bad);
+  if (first_band >= 0) *first_tensor = p->guard_bands[static_cast<size_t>(first_band)].second;
   return OK;
 }
 

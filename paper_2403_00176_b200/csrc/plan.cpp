@@ -370,7 +370,8 @@ struct Planner {
       if (p.roots[t].where == RootBuf::ARENA && p.roots[t].def_step >= 0 && p.roots[t].def_step <= p.place_until_step &&
           p.roots[t].last_step >= p.place_from_step)
         ids.push_back(static_cast<int>(t));
-    auto sz = [&](int t) { return (static_cast<size_t>(p.roots[t].bytes) + 255) & ~size_t(255); };
+    const size_t band = (c.flags & OPT_GUARD_BANDS) ? 256 : 0;
+    auto sz = [&](int t) { return ((static_cast<size_t>(p.roots[t].bytes) + 255) & ~size_t(255)) + band; };
     // scratch of groups is planned like a tensor living for exactly that step
     std::vector<size_t> live(steps + 1, 0);
     p.sum_bytes = 0;
@@ -389,7 +390,8 @@ struct Planner {
     auto place = [&](int t, bool smallest_gap) {
       RootBuf& R = p.roots[t];
       size_t need = sz(t);
-      if (c.flags & OPT_NO_REUSE) { R.arena_off = top; top += need; placed.push_back({R.arena_off, need, R.def_step, R.last_step}); return; }
+      // guard bands only mean something where no other tensor ever covers them: every tensor its own slot
+      if (c.flags & (OPT_NO_REUSE | OPT_GUARD_BANDS)) { R.arena_off = top; top += need; placed.push_back({R.arena_off, need, R.def_step, R.last_step}); return; }
       // free gaps among tensors whose lifetime overlaps this one
       std::vector<std::pair<size_t, size_t>> busy;
       for (auto& q : placed) if (!(q.last < R.def_step || q.def > R.last_step)) busy.push_back({q.off, q.off + q.size});
@@ -439,7 +441,7 @@ struct Planner {
     // results outlive their large intermediates), the walk above fragments.  If it ended more than 2 %
     // above the live peak, a second placement is tried, largest tensor first at the lowest offset
     // that is free over its lifetime, and the smaller arena is kept.
-    if (p.pinned.empty() && !(c.flags & OPT_NO_REUSE) && top - HEADER > p.peak_live_bytes + p.peak_live_bytes / 50) {
+    if (p.pinned.empty() && !(c.flags & (OPT_NO_REUSE | OPT_GUARD_BANDS)) && top - HEADER > p.peak_live_bytes + p.peak_live_bytes / 50) {
       std::vector<size_t> first_off(ids.size());
       for (size_t i = 0; i < ids.size(); ++i) first_off[i] = p.roots[ids[i]].arena_off;
       const size_t first_top = top;
@@ -456,6 +458,9 @@ struct Planner {
       }
     }
     p.arena_bytes = top;
+    p.guard_bands.clear();
+    if (band)
+      for (int t : ids) p.guard_bands.push_back({p.roots[t].arena_off + sz(t) - band, t});
     return OK;
   }
 };

@@ -137,6 +137,39 @@ def test_unfused_execution_of_the_encoder_and_the_pruning_stack():
             assert o3[r][f"idx{l}"].shape == (1, n) and np.all(np.diff(o3[r][f"idx{l}"][0]) > 0)
 
 
+def test_guard_bands_and_poisoned_arena():
+    # SOD2_OPT_GUARD_BANDS: 256 bytes behind every arena tensor and scratch region.  With the arena filled with NaN
+    # bytes before the run, results must not change (nothing reads memory that nothing wrote) and every band must
+    # survive (no kernel stores past the end of its tensor), on every kind of workload; a band damaged from the host
+    # is found and named.
+    cases = [(_encoder_edge()[0], _encoder_edge()[1][:6]), (WL.cfg3(layers=2, D=128, H=2, F=256), None), (WL.cfg4(blocks=2), None),
+             (WL.cfg5(B=6, side=32, widths=(64, 128), per_stage=2), None)]
+    for wl, reqs in cases:
+        reqs = reqs if reqs is not None else wl.batch(0)
+        if wl.meta.get("cfg") == 4:
+            reqs = _conv_requests(wl, [(17, 33), (8, 200), (40, 96)])
+        _, _, ref = run_batch(wl, reqs)
+        s = Session(wl, opt_flags=B.OPT_GUARD_BANDS)
+        p = s.prepare(reqs)
+        assert p.plan.arena_bytes > 0
+        p.plan.poison_arena(p.arena.data_ptr(), p.arena.numel(), s.stream)
+        p.run()
+        p.check_device_status()
+        n_bad, name = p.plan.check_guards(p.arena.data_ptr(), s.stream)
+        assert n_bad == 0, (wl.name, n_bad, name)
+        got = p.outputs()
+        for r in range(len(reqs)):
+            for nm in ref[r]:
+                assert np.array_equal(ref[r][nm], got[r][nm]), (wl.name, nm)
+    # damage the band behind one tensor from the host: reported with the tensor's name
+    name = "stem"
+    slot = p.plan.slot(name)
+    band = slot["offset"] + (slot["bytes"] + 255) // 256 * 256
+    p.arena[band + 100: band + 104] = 0
+    n_bad, first = p.plan.check_guards(p.arena.data_ptr(), s.stream)
+    assert n_bad == 1 and first == name, (n_bad, first)
+
+
 def test_bounded_wait_runs_out_and_is_reported():
     # Every device-side wait gives up after a bounded number of polls, raises the status word and returns.  The
     # self-test kernel waits on a barrier that nothing ever arrives on, with a limit of a few thousand polls: it must
