@@ -20,7 +20,7 @@ stable argsort; NonZero against numpy.nonzero; Switch/Combine against masked
 execute-all; the Fig. 4 chain against explicit loops; GlobalAveragePool, the gate chain
 (pool -> linear -> Greater, with a logit of exactly zero), LayerNorm and Softmax values against
 loops; Greater, Range, ConstantOfShape, Cast, Div, Sub, Reshape's 0 / -1 rules, ReduceSumSquare,
-Relu, Shape, Transpose, Concat, Gather and Slice against literal arrays.  Nothing here is
+Relu, Shape, Transpose, Concat, Gather, Slice and Expand against literal arrays.  Nothing here is
 "parity unpinned" except the reading of tolerances and decision bands, which is a convention,
 not a value.
 """
@@ -298,6 +298,9 @@ def run(text: str, consts: Dict[str, np.ndarray], inputs: Dict[str, np.ndarray],
             out = np.arange(int(x[0]), int(x[1]), int(x[2]), dtype=np.int64)
         elif op == "ConstantOfShape":
             out = np.full([int(v) for v in x[0]], float(a.get("value", 0.0)))
+        elif op == "Expand":
+            # broadcast x against the VALUE of the shape operand (multidirectional: either side may be 1)
+            out = np.array(x[0] * np.ones([int(v) for v in x[1]], dtype=x[0].dtype))
         elif op == "Greater":
             out = (x[0] > x[1])
         elif op == "Switch":

@@ -42,6 +42,7 @@ enum class GKind {
   SUMSQ,       // ReduceSumSquare over the last axis
   TOPK,        // TopK over the last axis: values + int64 indices
   GATHER,      // Gather along one axis by an int64 index tensor computed on the device
+  FILL,        // Range / ConstantOfShape whose extent is only known at bind time: out[i] = start + i * step
   UNSUPPORTED
 };
 const char* gkind_name(GKind k);

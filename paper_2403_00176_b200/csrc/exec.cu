@@ -1092,6 +1092,39 @@ struct Builder {
     return OK;
   }
 
+  Status build_fill(int gi, const Group& G) {
+    const Tensor& O = g.tensors[G.out];
+    const Node& n = g.nodes[G.nodes[0]];
+    const int dt = O.dtype == DType::I64 ? 2 : O.dtype == DType::BF16 ? 1 : O.dtype == DType::F32 ? 0 : -1;
+    if (dt < 0) return fail(E_UNSUPPORTED_OP, "fill: output type");
+    for (int r = 0; r < p.n_req; ++r) {
+      const View& vo = p.views[G.out][r];
+      if (!vo.contiguous()) return fail(E_UNSUPPORTED_OP, "fill: contiguous output");
+      if (numel(vo.dims) == 0) continue;
+      k::FillParams fp{};
+      fp.n = numel(vo.dims);
+      fp.dtype = dt;
+      if (G.act) {     // Range(start, limit, delta): the value maps hold the operands as expressions of the symbols
+        const ValueVal &a = g.tensors[n.ins[0]].V, &d = g.tensors[n.ins[2]].V;
+        if (!a.all_known() || !d.all_known() || a.elems.size() != 1 || d.elems.size() != 1) return fail(E_UNSUPPORTED_OP, "Range: start and delta must be known from shapes");
+        bool ok1, ok2;
+        fp.start = static_cast<double>(e_eval(g.cx, a.elems[0].e, p.b->vals[r], &ok1));
+        fp.step = static_cast<double>(e_eval(g.cx, d.elems[0].e, p.b->vals[r], &ok2));
+        if (!ok1 || !ok2) return fail(E_UNBOUND_SYMBOL, "Range: operands not bound");
+      } else {
+        fp.start = G.scale;
+        fp.step = 0.0;
+      }
+      Ptr po = ptr_of(G.out, r);
+      add(gi, 1, [=](const RunCtx& x) mutable {
+        fp.out = x.resolve(po);
+        k::fill_linear<<<static_cast<unsigned>(std::max<long long>(1, std::min<long long>((fp.n + 255) / 256, 148 * 8))), 256, 0, x.stream>>>(fp);
+        return cudaGetLastError();
+      });
+    }
+    return OK;
+  }
+
   // ------------------------------------------------------------------------------ top-k keep
   Status build_topk(int gi, const Group& G) {
     if (g.tensors[G.a].dtype != DType::BF16) return fail(E_UNSUPPORTED_OP, "top-k keep is bf16 only");
@@ -1988,7 +2021,7 @@ struct Builder {
     p.uses_header = false;
     for (const Group& G : c.groups)
       if (!((G.kind == GKind::GEMM && g.tensors[G.a].dtype == DType::F32) || G.kind == GKind::CHAIN || G.kind == GKind::BMM ||
-            G.kind == GKind::SUMSQ || G.kind == GKind::TOPK || G.kind == GKind::GATHER)) p.uses_header = true;
+            G.kind == GKind::SUMSQ || G.kind == GKind::TOPK || G.kind == GKind::GATHER || G.kind == GKind::FILL)) p.uses_header = true;
     for (size_t gi = 0; gi < c.groups.size(); ++gi) {
       const Group& G = c.groups[gi];
       Status s = OK;
@@ -2016,6 +2049,7 @@ struct Builder {
         case GKind::SUMSQ: s = build_sumsq(static_cast<int>(gi), G); break;
         case GKind::TOPK: s = build_topk_rows(static_cast<int>(gi), G); break;
         case GKind::GATHER: s = build_gather(static_cast<int>(gi), G); break;
+        case GKind::FILL: s = build_fill(static_cast<int>(gi), G); break;
         default: return fail(E_UNSUPPORTED_OP, std::string("no executor yet for group kind ") + gkind_name(G.kind));
       }
       if (s != OK) return s;

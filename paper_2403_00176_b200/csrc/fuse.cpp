@@ -30,6 +30,7 @@ const char* gkind_name(GKind k) {
     case GKind::SUMSQ: return "sumsq";
     case GKind::TOPK: return "topk";
     case GKind::GATHER: return "gather";
+    case GKind::FILL: return "fill";
     default: return "unsupported";
   }
 }
@@ -523,6 +524,14 @@ struct Fuser {
         finish(G);
       } else if (op == "Combine") {
         Group G; G.kind = GKind::COMBINE; G.nodes = {nid}; G.a = n.ins[0]; G.res = n.ins[1]; G.gate = n.ins[2]; G.out = n.outs[0];
+        finish(G);
+      } else if (op == "Expand") {
+        // a copy through the chain kernel: the operand is read with stride 0 along the dims it broadcasts over
+        Group G; G.kind = GKind::CHAIN; G.nodes = {nid}; G.a = n.ins[0]; G.out = n.outs[0];
+        finish(G);
+      } else if (op == "Range" || op == "ConstantOfShape") {
+        Group G; G.kind = GKind::FILL; G.nodes = {nid}; G.out = n.outs[0]; G.act = op == "Range";
+        G.scale = static_cast<float>(n.attr_f("value", 0.0));
         finish(G);
       } else if (op == "TopK" && n.outs.size() == 2) {
         Group G; G.nodes = {nid}; G.a = n.ins[0]; G.out = n.outs[0]; G.out2 = n.outs[1];

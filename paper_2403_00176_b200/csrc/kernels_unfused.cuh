@@ -126,5 +126,16 @@ __global__ void __launch_bounds__(256) gather_axis(GatherParams p) {
   }
 }
 
+// out[i] = start + i * step for i < n: Range (int64) and ConstantOfShape (step 0; fp32, bf16 or int64).
+struct FillParams { void* out; long long n; double start, step; int dtype; /* 0 f32, 1 bf16, 2 i64 */ };
+__global__ void __launch_bounds__(256) fill_linear(FillParams p) {
+  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < p.n; i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const double v = p.start + static_cast<double>(i) * p.step;
+    if (p.dtype == 2) reinterpret_cast<long long*>(p.out)[i] = static_cast<long long>(v);
+    else if (p.dtype == 1) reinterpret_cast<__nv_bfloat16*>(p.out)[i] = __float2bfloat16_rn(static_cast<float>(v));
+    else reinterpret_cast<float*>(p.out)[i] = static_cast<float>(v);
+  }
+}
+
 }  // namespace k
 }  // namespace sod2

@@ -902,8 +902,10 @@ struct Rdp {
 
   // ---------------------------------------------------------------- backward Update functions
   // Only refinements that are unambiguous are applied: same-shape operators, the contracted dim of
-  // MatMul, Transpose, Conv channels. Broadcasting operators give only a set {1, d} per dim
-  // (Section 3), which the lattice cannot hold, so they propagate the rank when it is certain.
+  // MatMul, Transpose, Conv channels, the input of Shape from the value of its output, the one unknown
+  // extent of a Reshape input from the element count, the one unknown Concat operand.  Broadcasting operators
+  // give a set {1, d} per dim in general (Section 3), which the lattice cannot hold: they propagate the rank
+  // when it is certain, and an extent where the partner's is the constant 1.
   bool backward(int nid, int pred_tensor) {
     const Tensor& P = g.tensors[pred_tensor];
     if (!P.S.any_undef()) return false;
@@ -943,12 +945,78 @@ struct Rdp {
         if (o.rank == 4) s.dims[0] = o.dims[0];
         ch |= refine_shape(pred_tensor, s);
       }
-    } else if ((op == "Add" || op == "Sub" || op == "Mul" || op == "Div") && P.S.rank == RANK_UNDEF) {
-      // rank certain only if the partner has lower rank than the output
+    } else if (op == "Add" || op == "Sub" || op == "Mul" || op == "Div") {
       const ShapeVal& o = S(n.outs[0]);
       int other = pred_tensor == n.ins[0] ? n.ins[1] : n.ins[0];
-      if (o.rank >= 0 && S(other).rank >= 0 && S(other).rank < o.rank) {
+      const ShapeVal& q = S(other);
+      if (P.S.rank == RANK_UNDEF) {
+        // rank certain only if the partner has lower rank than the output
+        if (o.rank >= 0 && q.rank >= 0 && q.rank < o.rank) {
+          ShapeVal s; s.rank = o.rank; s.dims.assign(o.rank, Dim());
+          ch |= refine_shape(pred_tensor, s);
+        }
+      } else if (o.rank >= 0 && q.rank >= 0 && P.S.rank == o.rank) {
+        // broadcasting leaves {1, d} for an extent in general; where the PARTNER's extent is the constant 1 (or the
+        // partner has no such dim) and the output's is another value, this operand must carry the output's extent
+        ShapeVal s = P.S;
+        for (int i = 0; i < o.rank; ++i) {
+          const int qi = i - (o.rank - q.rank);
+          const bool partner_one = qi < 0 || (q.dims[qi].known() && q.dims[qi].e.is_const() && q.dims[qi].e.const_value() == 1);
+          const bool out_not_one = o.dims[i].known() && !(o.dims[i].e.is_const() && o.dims[i].e.const_value() == 1);
+          if (s.dims[i].kind == Dim::UNDEF && partner_one && out_not_one) s.dims[i] = o.dims[i];
+        }
+        ch |= refine_shape(pred_tensor, s);
+      }
+    } else if (op == "Shape" && pred_tensor == n.ins[0]) {
+      // F^bs of the shape-determined-output class: the VALUE of Shape's output is its input's shape
+      const ValueVal& v = V(n.outs[0]);
+      if (v.kind == ValueVal::KNOWN) {
+        ShapeVal s; s.rank = static_cast<int>(v.elems.size()); s.dims = v.elems;
+        ch |= refine_shape(pred_tensor, s);
+      } else if (S(n.outs[0]).rank == 1 && S(n.outs[0]).dims[0].known() && S(n.outs[0]).dims[0].e.is_const() && P.S.rank == RANK_UNDEF) {
+        ShapeVal s; s.rank = static_cast<int>(S(n.outs[0]).dims[0].e.const_value()); s.dims.assign(s.rank, Dim());
+        ch |= refine_shape(pred_tensor, s);
+      }
+    } else if (op == "Reshape" && pred_tensor == n.ins[0]) {
+      // one unknown input extent follows from the element count of a fully known output
+      const ShapeVal& o = S(n.outs[0]);
+      if (o.fully_known() && P.S.rank >= 1) {
+        int unknown = -1, n_unknown = 0;
+        Expr known_prod(1), total(1);
+        for (int i = 0; i < P.S.rank; ++i) {
+          if (P.S.dims[i].kind == Dim::UNDEF) { unknown = i; ++n_unknown; }
+          else if (P.S.dims[i].known()) known_prod = known_prod * P.S.dims[i].e;
+          else n_unknown = 99;
+        }
+        for (auto& d : o.dims) total = total * d.e;
+        bool okq = false;
+        const Expr quot = n_unknown == 1 ? e_exact_div(total, known_prod, &okq) : Expr();
+        if (n_unknown == 1 && okq) {
+          ShapeVal s = P.S;
+          s.dims[unknown] = Dim::val(quot);
+          ch |= refine_shape(pred_tensor, s);
+        }
+      }
+    } else if (op == "Concat") {
+      // the extents off the axis equal the output's; on the axis the one unknown operand takes what is left
+      const ShapeVal& o = S(n.outs[0]);
+      if (o.rank >= 1 && (P.S.rank == o.rank || P.S.rank == RANK_UNDEF)) {
+        const int ax = norm_axis(n.attr_i("axis", 0), o.rank);
         ShapeVal s; s.rank = o.rank; s.dims.assign(o.rank, Dim());
+        if (P.S.rank == o.rank) s = P.S;
+        for (int i = 0; i < o.rank; ++i) if (i != ax && s.dims[i].kind == Dim::UNDEF) s.dims[i] = o.dims[i];
+        if (s.dims[ax].kind == Dim::UNDEF && o.dims[ax].known()) {
+          Expr rest = o.dims[ax].e;
+          bool ok = true;
+          int mine = 0;
+          for (int in_t : n.ins) {
+            if (in_t == pred_tensor) { ++mine; continue; }
+            const ShapeVal& x = S(in_t);
+            if (x.rank != o.rank || !x.dims[ax].known()) { ok = false; break; }
+            rest = rest - x.dims[ax].e;
+          }
+          if (ok && mine == 1) s.dims[ax] = Dim::val(rest);
+        }
         ch |= refine_shape(pred_tensor, s);
       }
     }

@@ -170,6 +170,29 @@ def test_guard_bands_and_poisoned_arena():
     assert n_bad == 1 and first == name, (n_bad, first)
 
 
+def test_expand_range_constant_of_shape_executors():
+    # shape-and-value determined operators whose extents are expressions of the bound symbols: Expand against
+    # Shape(y) (a copy with broadcast strides), Range(0, N, 1) and ConstantOfShape([2, N]) filled on the device
+    ir = ("sym N 1 4096\ninput x bf16 [1,N,1]\ninput y bf16 [2,N,8]\niconst i0 i64 [] = 0\niconst i1 i64 [] = 1\niconst ix1 i64 [1] = 1\n"
+          "iconst two i64 [1] = 2\nnode Shape y -> sy\nnode Expand x sy -> e\nnode Add e y -> z\nnode Gather sy ix1 -> nvec {axis=0}\n"
+          "iconst shp0 i64 [0] =\nnode Reshape nvec shp0 -> n\nnode Range i0 n i1 -> r\nnode Concat two nvec -> cs {axis=0}\n"
+          "node ConstantOfShape cs -> c {value=1.5}\noutput z\noutput e\noutput r\noutput c\n")
+    rng = np.random.default_rng(4)
+    reqs = [Request({"N": n}, {"x": bf16_round(rng.standard_normal((1, n, 1)).astype(np.float32)), "y": bf16_round(rng.standard_normal((2, n, 8)).astype(np.float32))})
+            for n in (1, 7, 300)]
+    wl = WL.Workload("expand_range", "bf16", ir, {}, ["N"], ["z", "e", "r", "c"], {"batch_fn": lambda j: reqs})
+    s, p, outs = run_batch(wl, reqs)
+    kinds = [s.graph.group_info(i)["kind"] for i in range(s.graph.num_groups())]
+    assert kinds.count("fill") == 2 and kinds.count("chain") == 2, kinds
+    for r, req in enumerate(reqs):
+        env = O.run(ir, {}, req.inputs)
+        n = req.syms["N"]
+        assert np.array_equal(outs[r]["r"], np.arange(n)) and np.array_equal(outs[r]["r"], env["r"])
+        assert outs[r]["c"].shape == (2, n) and np.all(outs[r]["c"] == 1.5)
+        assert outs[r]["e"].shape == (2, n, 8) and np.array_equal(outs[r]["e"].astype(np.float64), env["e"])
+        assert O.rel_err(outs[r]["z"], env["z"]) <= BF16_TOL
+
+
 def test_bounded_wait_runs_out_and_is_reported():
     # Every device-side wait gives up after a bounded number of polls, raises the status word and returns.  The
     # self-test kernel waits on a barrier that nothing ever arrives on, with a limit of a few thousand polls: it must

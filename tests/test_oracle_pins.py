@@ -380,3 +380,10 @@ def test_layernorm_values_vs_loops():
         var = sum((v - mu) ** 2 for v in x[i]) / 5
         for j in range(5):
             assert abs(y[i, j] - ((x[i, j] - mu) / math.sqrt(var + 1e-3) * g[j] + b[j])) < 1e-13
+
+
+def test_expand_literals():
+    x = np.array([[1.0], [2.0], [3.0]])                       # [3,1]
+    env = _run("input x f32 [3,1]\niconst s1 i64 [2] = 3 4\niconst s2 i64 [3] = 2 1 4\nnode Expand x s1 -> a\nnode Expand x s2 -> b\n", {"x": x})
+    assert env["a"].tolist() == [[1.0] * 4, [2.0] * 4, [3.0] * 4]
+    assert env["b"].shape == (2, 3, 4) and env["b"][1].tolist() == [[1.0] * 4, [2.0] * 4, [3.0] * 4]   # the 1 in the target keeps x's 3

@@ -234,6 +234,63 @@ output s
     assert g.tensor_value("s").count("d") == 3
 
 
+def test_backward_transfer_more_operator_classes():
+    # broadcast operands: where the partner's extent is the constant 1 and the output's is not, the operand must carry
+    # the output's extent (an extent the partner shares stays undetermined: {1, d})
+    g = B.Graph("""
+input a f32 [?,?,?]
+input b f32 [1,6,1]
+input c f32 [?,?,?]
+input d f32 [4,6,8]
+const W f32 [8,16]
+node Add a b -> t
+node Relu t -> u
+node MatMul u W -> z
+node Add c d -> q
+node Relu q -> v
+node MatMul v W -> z2
+output z
+output z2
+""")
+    # MatMul fixes u's last extent (8), Relu hands it to t, and since b's last extent is 1 it must come from a
+    assert g.tensor_info("t")[2].endswith(",8]") and g.tensor_info("a")[2].endswith(",8]")
+    # c + d: d's extents are 4, 6, 8 (none is 1), so c's stay undetermined by this operator ({1, d} each): they are
+    # named by fresh symbols, not copied from d
+    assert g.tensor_info("q")[2].endswith(",8]") and g.tensor_info("c")[2] != "[4,6,8]"
+    # Shape: the VALUE of its output is the shape of its input (backward, shape-determined-output class)
+    g = B.Graph("""
+sym N 1 64
+input x f32 [?,?]
+input y f32 [N,32]
+node Shape y -> sy
+node Reshape x sy -> r
+node Shape r -> sr
+output sr
+""")
+    assert g.tensor_value("sr") == "[N,32]"
+    # Reshape: one unknown input extent from the element count of the known output
+    g = B.Graph("""
+sym N 1 64
+input x f32 [?,16]
+input y f32 [N,4,4]
+node Shape y -> sy
+node Reshape x sy -> r
+output r
+""")
+    assert g.tensor_info("r")[2] == "[N,4,4]" and g.tensor_info("x")[2] == "[N,16]"
+    # Concat: the operand left unknown on the axis takes what the others leave; off the axis it copies the output
+    g = B.Graph("""
+sym N 1 64
+input a f32 [N,5]
+input b f32 [?,?]
+const W f32 [12,3]
+node Concat a b -> t {axis=1}
+node MatMul t W -> z
+output z
+""")
+    assert g.tensor_info("t")[2] == "[N,12]" and g.tensor_info("b")[2] == "[N,7]"
+
+
 def test_nac_partition_and_runtime_symbol():
     g = B.Graph(WL.nonzero_graph().ir)
     rank, kinds, txt = g.tensor_info("nz")
