@@ -95,7 +95,9 @@ __global__ void __launch_bounds__(256) topk_flags(const __grid_constant__ TopkPa
   ptx::pdl_launch();
   const int tid = threadIdx.x;
   const double* sc = p.score + (R.row0 - p.first_row);
-  for (int i = tid; i < R.n; i += 256) s_score[i] = sc[i];
+  // a NaN score (an overflow upstream) compares false with everything and would be kept by every chunk: it ranks
+  // last instead, ties among NaNs by index, so that exactly k tokens are kept whatever the data
+  for (int i = tid; i < R.n; i += 256) { const double v = sc[i]; s_score[i] = v == v ? v : -INFINITY; }
   __syncthreads();
   const int i = chunk * TOPK_CHUNK + (tid >> 2), part = tid & 3;
   int rank = 0;

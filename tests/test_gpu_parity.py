@@ -193,6 +193,32 @@ def test_expand_range_constant_of_shape_executors():
         assert O.rel_err(outs[r]["z"], env["z"]) <= BF16_TOL
 
 
+def test_topk_keep_with_nan_rows_keeps_exactly_k():
+    # a row of NaN (an overflow upstream) has a NaN score, which compares false with everything: it must rank last, not
+    # be kept by every chunk, so that exactly k rows are kept (in ascending order) and nothing is written past them
+    ir = ("sym N 1 4096\ninput y bf16 [1,N,64]\niconst k i64 [1] = 5\niconst i_m1 i64 [1] = -1\n"
+          "node ReduceSumSquare y -> sc {axis=-1 keepdims=0}\nnode TopK sc k -> tv idx {axis=-1 largest=1 order=index}\n"
+          "node Reshape idx i_m1 -> ix\nnode Gather y ix -> keep {axis=1}\noutput keep\noutput idx\n")
+    rng = np.random.default_rng(8)
+    reqs = []
+    for n, bad in ((12, [0, 3, 4, 5, 6, 7, 9]), (200, list(range(60, 140)))):
+        y = bf16_round(rng.standard_normal((1, n, 64)).astype(np.float32))
+        y[0, bad, 3] = np.nan
+        reqs.append(Request({"N": n}, {"y": y}))
+    wl = WL.Workload("topk_nan", "bf16", ir, {}, ["N"], ["keep", "idx"], {"batch_fn": lambda j: reqs})
+    s, p, outs = run_batch(wl, reqs)
+    assert [s.graph.group_info(i)["kind"] for i in range(s.graph.num_groups())] == ["topk_keep"]
+    for r, req in enumerate(reqs):
+        y = req.inputs["y"][0].astype(np.float64)
+        idx = outs[r]["idx"][0]
+        assert idx.shape == (5,) and np.all(np.diff(idx) > 0)
+        sc = (y * y).sum(-1)
+        finite = np.flatnonzero(np.isfinite(sc))
+        want = np.sort(finite[np.argsort(-sc[finite], kind="stable")[:5]])
+        assert np.array_equal(idx, want), (idx, want)          # the NaN rows rank behind every finite one
+        assert np.array_equal(outs[r]["keep"][0], req.inputs["y"][0][idx])
+
+
 def test_bounded_wait_runs_out_and_is_reported():
     # Every device-side wait gives up after a bounded number of polls, raises the status word and returns.  The
     # self-test kernel waits on a barrier that nothing ever arrives on, with a limit of a few thousand polls: it must
