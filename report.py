@@ -230,12 +230,53 @@ def measure(cfg: int, reps: int, device: str = "cuda:0", opt_flags: int = 0):
     }
 
 
+def chain_case(spec: str, reps: int = 20, device: str = "cuda:0"):
+    """The paper's fusion example (Fig. 4: Sigmoid(A[I,1,1]) + B[I,J,K], one fused group) at a given size:
+    spec = "I,J,K,dtype,n_requests".  Device time of the whole inference (one launch) against the HBM roofline of its
+    algorithmic bytes (B in, C out; A is I values)."""
+    import torch
+    from paper_2403_00176_b200 import workloads as WL
+    from paper_2403_00176_b200.session import Session
+    from paper_2403_00176_b200.workloads import Request, bf16_round
+    i, j, k, dt, n = spec.split(",")
+    i, j, k, n = int(i), int(j), int(k), int(n)
+    hbm, _, src = _peaks()
+    wl = WL.fig4_chain(dt)
+    rng = np.random.default_rng(0)
+    rnd = (lambda a: bf16_round(a.astype(np.float32))) if dt == "bf16" else (lambda a: a.astype(np.float32))
+    reqs = [Request({"I": i, "J": j, "K": k}, {"A": rnd(rng.standard_normal((i, 1, 1))), "B": rnd(rng.standard_normal((i, j, k)))}) for _ in range(n)]
+    sess = Session(wl, device=device)
+    p = sess.prepare(reqs)
+    p.run()
+    torch.cuda.synchronize(sess.dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=sess.dev)
+    stream = torch.cuda.current_stream(sess.dev)
+    lone = []
+    for it in range(reps):
+        flush.fill_(it & 0xFF)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        p.run()
+        e1.record(stream)
+        torch.cuda.synchronize(sess.dev)
+        lone.append(e0.elapsed_time(e1))
+    b2b = group_times(p, reps=5, repeat=20)[0]
+    _, nbytes = p.plan.group_cost(0)
+    ms = float(np.median(lone))
+    return {"case": spec, "launches": int(p.run().gpu_launches), "bytes": nbytes, "ms_lone_launch": ms, "gbs_lone_launch": nbytes / ms / 1e6,
+            "ms_back_to_back": b2b, "gbs_back_to_back": nbytes / b2b / 1e6, "frac_of_hbm_back_to_back": nbytes / b2b / 1e6 / hbm, "peaks": src}
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--chain-case", default=None, help="I,J,K,dtype,n_requests: time the Fig. 4 fused chain at this size instead of the configs")
     ap.add_argument("--configs", default="1,2,3,4,5")
     ap.add_argument("--reps", type=int, default=30)
     ap.add_argument("--opt-flags", type=int, default=0, help="SOD2_OPT_* bits for sod2_graph_create (A/B measurements)")
     a = ap.parse_args()
+    if a.chain_case:
+        print(json.dumps(chain_case(a.chain_case)))
+        return
     rows = []
     for c in [int(x) for x in a.configs.split(",")]:
         r = measure(c, a.reps, opt_flags=a.opt_flags)
