@@ -26,6 +26,7 @@ OPT_MULTI_VERSION = 64
 OPT_LN_FOLD = 128
 OPT_GEMM_CHAIN = 256
 OPT_GUARD_BANDS = 512
+OPT_GEMM_PAIR = 1024
 DYN_CLASS = ["ISDO", "ISDOS", "ISVDOS", "EDO"]
 
 

@@ -21,6 +21,7 @@ enum OptFlags : uint32_t {
   OPT_SPLITK_LN = 4u,   // a bf16 GEMM (+bias, +residual) followed by LayerNorm becomes one group: split-K GEMM + finishing kernel
   OPT_LN_FOLD = 128u,     // a LayerNorm between bf16 GEMMs is folded into their epilogues (the normalised tensor is never stored)
   OPT_GUARD_BANDS = 512u, // 256 poison bytes behind every arena tensor and scratch region, checked after a run (sod2_plan_check_guards)
+  OPT_GEMM_PAIR = 1024u,  // bf16 GEMMs on CTA pairs (tcgen05.mma.cta_group::2) where the makespan estimate favours them
   OPT_GEMM_CHAIN = 256u,  // consecutive dependent GEMM groups run as one persistent kernel with row-block dependency counters
 };
 

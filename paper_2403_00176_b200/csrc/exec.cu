@@ -16,6 +16,7 @@
 #include "engine.h"
 #include "gemm_tcgen05.cuh"
 #include "gemm_chain_tcgen05.cuh"
+#include "gemm_pair_tcgen05.cuh"
 #include "kernels_compact.cuh"
 #include "kernels_rows.cuh"
 #include "kernels_unfused.cuh"
@@ -66,6 +67,26 @@ cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t sme
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
+// The same with a thread-block cluster of two CTAs along x (the CTA-pair GEMM).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl_pair(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = 2;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
 
@@ -130,6 +151,27 @@ cudaError_t gemm_dispatch(int act, bool res, int ln, bool emit, dim3 grid, cudaS
   }
 #undef SOD2_GV
   return cudaErrorInvalidValue;
+}
+
+template <int BN, int KCH, int ST, int ACT, bool RES>
+cudaError_t launch_gemm_pair_variant(dim3 grid, cudaStream_t st, const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to,
+                                     const CUtensorMap& tr, int M, int N, int K, const k::GemmEpilogue& ep) {
+  constexpr int smem = k::GemmPairSmem<BN, KCH, ST>::TOTAL;
+  static bool once = (cudaFuncSetAttribute(k::gemm_pair_bf16_tcgen05<BN, KCH, ST, ACT, RES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), true);
+  (void)once;
+  return launch_pdl_pair(k::gemm_pair_bf16_tcgen05<BN, KCH, ST, ACT, RES>, grid, dim3(k::GEMM_THREADS), smem, st, ta, tb, to, tr, M, N, K, ep);
+}
+template <int BN, int KCH, int ST>
+cudaError_t gemm_pair_dispatch(int act, bool res, dim3 grid, cudaStream_t st, const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to,
+                               const CUtensorMap& tr, int M, int N, int K, const k::GemmEpilogue& ep) {
+  switch (act * 2 + (res ? 1 : 0)) {
+    case 0: return launch_gemm_pair_variant<BN, KCH, ST, 0, false>(grid, st, ta, tb, to, tr, M, N, K, ep);
+    case 1: return launch_gemm_pair_variant<BN, KCH, ST, 0, true>(grid, st, ta, tb, to, tr, M, N, K, ep);
+    case 2: return launch_gemm_pair_variant<BN, KCH, ST, 1, false>(grid, st, ta, tb, to, tr, M, N, K, ep);
+    case 3: return launch_gemm_pair_variant<BN, KCH, ST, 1, true>(grid, st, ta, tb, to, tr, M, N, K, ep);
+    case 4: return launch_gemm_pair_variant<BN, KCH, ST, 2, false>(grid, st, ta, tb, to, tr, M, N, K, ep);
+    default: return launch_gemm_pair_variant<BN, KCH, ST, 2, true>(grid, st, ta, tb, to, tr, M, N, K, ep);
+  }
 }
 
 struct Builder {
@@ -384,6 +426,21 @@ struct Builder {
         bn_group = bn;
         p.stats_layout[G.out] = {static_cast<int>(N / bn) * 2, bn / 2};
       }
+      // CTA pairs (tcgen05.mma.cta_group::2, 256 x BN tiles): each CTA loads its own A rows and half of the weight tile,
+      // a third to a half fewer operand bytes per flop.  Same makespan estimate, per 64-wide k-chunk and pair of SMs.
+      int pair_bn = 0;
+      if ((c.flags & OPT_GEMM_PAIR) && !lna && !lnr && !emit && G.act2 == 0 && tiles_m >= 2 && N >= 128) {
+        auto pair_span = [&](int bn_) {
+          const double pairs = std::ceil(tiles_m / 2.0) * ((N + bn_ - 1) / bn_);
+          const double waves = std::ceil(pairs / (sms / 2));
+          const double mma = 4 * (bn_ / 2.0), tma = (128 + bn_ / 2) * 128.0 / 70.0;
+          return waves * std::ceil(K / 64.0) * std::max(mma, tma);
+        };
+        const double single = bn == 256 ? makespan(256, 1) : makespan(128, 2);
+        const int pb = (N >= 256 && pair_span(256) <= pair_span(128)) ? 256 : 128;
+        static const bool force_pair = getenv("SOD2_GEMM_PAIR_FORCE") != nullptr;   // tests: the pair kernel wherever it is eligible
+        if (pair_span(pb) < single || force_pair) pair_bn = pb;
+      }
       const bool hb = G.bias >= 0, hr = G.res >= 0;
       const int act = G.act;
       const int act2 = G.act2;
@@ -409,8 +466,9 @@ struct Builder {
         void* O = x.resolve(po);
         const void* R = hr ? x.resolve(pr) : O;
         if (cache->a != A || cache->w != Wt || cache->o != O || cache->r != R) {
-          const int kch = bn == 256 ? 1 : 2;
-          if (!encode_bf16_kchunks(&cache->ta, A, M, K, lda, 128, kch) || !encode_bf16_kchunks(&cache->tb, Wt, N, K, K, bn, kch) ||
+          const int kch = pair_bn ? (pair_bn == 256 ? 1 : 2) : (bn == 256 ? 1 : 2);
+          const int brows = pair_bn ? pair_bn / 2 : bn;      // a CTA of a pair loads half of the weight tile
+          if (!encode_bf16_kchunks(&cache->ta, A, M, K, lda, 128, kch) || !encode_bf16_kchunks(&cache->tb, Wt, N, K, K, brows, kch) ||
               !encode_bf16_2d(&cache->to, O, M, N, ldo, 128) || !encode_bf16_2d(&cache->tr, R, M, N, hr ? ldr : ldo, 128))
             return cudaErrorInvalidValue;
           cache->a = A; cache->w = Wt; cache->o = O; cache->r = R;
@@ -438,10 +496,17 @@ struct Builder {
           ep.emit_stats = reinterpret_cast<float2*>(x.resolve(ps_out));
           ep.emit_pitch = pitch_out;
         }
+        const int Ni = static_cast<int>(N), Ki = static_cast<int>(K);
+        if (pair_bn) {
+          const int pairs = ((tiles_m + 1) / 2) * static_cast<int>((N + pair_bn - 1) / pair_bn);
+          const dim3 gp(2 * std::max(1, std::min(pairs, x.plan->sm_count / 2)));
+          const cudaError_t ep2 = pair_bn == 256 ? gemm_pair_dispatch<256, 1, 6>(act, hr, gp, x.stream, cache->ta, cache->tb, cache->to, cache->tr, M, Ni, Ki, ep)
+                                                 : gemm_pair_dispatch<128, 2, 4>(act, hr, gp, x.stream, cache->ta, cache->tb, cache->to, cache->tr, M, Ni, Ki, ep);
+          return ep2 != cudaSuccess ? ep2 : cudaGetLastError();
+        }
         const int tiles = tiles_m * static_cast<int>((N + bn - 1) / bn);
         const int grid = std::min(tiles, x.plan->sm_count);
         const dim3 gd(grid);
-        const int Ni = static_cast<int>(N), Ki = static_cast<int>(K);
         cudaError_t e;
         if (bn == 256) e = gemm_dispatch<256, 1, 4>(act, hr, ln, emit, gd, x.stream, cache->ta, cache->tb, cache->to, cache->tr, M, Ni, Ki, ep);
         else if (bn == 128) e = gemm_dispatch<128, 2, 3>(act, hr, ln, emit, gd, x.stream, cache->ta, cache->tb, cache->to, cache->tr, M, Ni, Ki, ep);

@@ -751,6 +751,51 @@ def test_gemm_epilogue_forms_ragged_shapes():
             assert O.rel_err(outs[r]["y"], ref) <= BF16_TOL, (K, N, act, residual, req.syms)
 
 
+def test_gemm_on_cta_pairs_matches_the_single_cta_kernel_and_the_oracle():
+    # SOD2_OPT_GEMM_PAIR: two CTAs of a cluster share a 256-row tile (tcgen05.mma.cta_group::2), each loading its own
+    # rows and half of the weight tile.  Row counts around the 256-row pair tile (an odd number of 128-row tiles leaves
+    # the second CTA of the last pair without rows), both tile widths, every epilogue form; against the oracle and
+    # against the single-CTA kernel.  SOD2_GEMM_PAIR_FORCE makes the planner take the pair kernel wherever it can.
+    import os
+    os.environ["SOD2_GEMM_PAIR_FORCE"] = "1"
+    try:
+        rng = np.random.default_rng(19)
+        # (the last two shapes are wide enough for the planner to take the 256-wide pair tile at 1929 rows)
+        cases = [(64, 256, None, False), (128, 136, "Relu", False), (192, 768, "Gelu", False), (768, 768, None, True), (320, 520, "Gelu", False),
+                 (128, 2304, None, False), (64, 2048, "Gelu", True)]
+        for K, N, act, residual in cases:
+            ir = _gemm_graph(K, N, act, residual)
+            consts = {"W": bf16_round((rng.standard_normal((K, N)) / np.sqrt(K)).astype(np.float32)),
+                      "b": bf16_round(rng.standard_normal(N).astype(np.float32))}
+            reqs = []
+            for M in (129, 256, 257, 385, 902):
+                ins = {"x": bf16_round(rng.standard_normal((1, M, K)).astype(np.float32))}
+                if residual:
+                    ins["r"] = bf16_round(rng.standard_normal((1, M, N)).astype(np.float32))
+                reqs.append(Request({"M": M}, ins))
+            wl = WL.Workload("gemm_pair_case", "bf16", ir, consts, ["M"], ["y"], {"batch_fn": lambda j: reqs})
+            # one request per plan (each its own row count), then all of them packed into one launch (1929 rows)
+            for group in ([[r] for r in reqs] + [reqs]):
+                s1, p1, o1 = run_batch(wl, group, opt_flags=B.OPT_GEMM_PAIR)
+                s0, p0, o0 = run_batch(wl, group)
+                for r, req in enumerate(group):
+                    ref = O.run(ir, consts, req.inputs)["y"]
+                    assert O.rel_err(o1[r]["y"], ref) <= BF16_TOL, (K, N, act, residual, req.syms)
+                    assert O.rel_err(o1[r]["y"], o0[r]["y"]) <= 1e-2, (K, N, act, residual, req.syms)
+                p1.run()
+                for a, b_ in zip(o1, p1.outputs()):
+                    assert np.array_equal(a["y"], b_["y"])
+        # the encoder with every eligible GEMM on pairs
+        wl, reqs = _encoder_edge()
+        s, p, outs = run_batch(wl, reqs, opt_flags=B.OPT_NO_REUSE | B.OPT_GEMM_PAIR)
+        for r, req in enumerate(reqs):
+            errs = lockstep(wl, s, p, outs, r, BF16_TOL)
+            bad = {k: v for k, v in errs.items() if not (isinstance(v, float) and v <= BF16_TOL)}
+            assert errs and not bad, (req.syms, bad)
+    finally:
+        del os.environ["SOD2_GEMM_PAIR_FORCE"]
+
+
 def test_branched_graph_planned_order_matches_default_order_and_oracle():
     # static execution planning reorders the groups of a branched graph (smaller live peak); the result
     # is bit-identical to the default order's and agrees with the oracle
