@@ -402,8 +402,8 @@ sod2_status sod2_binding_shape(const sod2_binding* b, int r, const char* name, i
 sod2_status sod2_plan_slot(const sod2_plan_t* p, const char* name, size_t* off, size_t* bytes, int* def, int* last) {
   if (!p || !name) return SOD2_E_INVALID_ARG;
   int t = p->g->c.g.tensor(name);
-  if (t < 0 || p->p.views[t].empty() || p->p.views[t][0].root < 0) return SOD2_E_INVALID_ARG;
-  if (p->p.views[t][0].root != t) return SOD2_E_INVALID_ARG;  // a view: it owns no slot
+  if (t < 0 || p->p.views[t].empty() || p->p.root_of[t] < 0) return SOD2_E_INVALID_ARG;
+  if (p->p.root_of[t] != t) return SOD2_E_INVALID_ARG;  // a view: it owns no slot
   const RootBuf& R = p->p.roots[t];
   if (R.where != RootBuf::ARENA) return SOD2_E_INVALID_ARG;
   if (off) *off = R.arena_off;
@@ -416,16 +416,16 @@ sod2_status sod2_plan_slot(const sod2_plan_t* p, const char* name, size_t* off, 
 sod2_status sod2_plan_instance_offset(const sod2_plan_t* p, const char* name, int r, size_t* off) {
   if (!p || !name || !off || r < 0 || r >= p->p.n_req) return SOD2_E_INVALID_ARG;
   int t = p->g->c.g.tensor(name);
-  if (t < 0 || p->p.views[t].empty() || p->p.views[t][0].root < 0) return SOD2_E_INVALID_ARG;
+  if (t < 0 || p->p.views[t].empty() || p->p.root_of[t] < 0) return SOD2_E_INVALID_ARG;
   const View& v = p->p.views[t][r];
-  *off = static_cast<size_t>(p->p.inst_off[v.root][r] + v.offset * dtype_size(p->g->c.g.tensors[t].dtype));
+  *off = static_cast<size_t>(p->p.inst_off[p->p.root_of[t]][r] + v.offset * dtype_size(p->g->c.g.tensors[t].dtype));
   return SOD2_OK;
 }
 
 sod2_status sod2_plan_tensor_strides(const sod2_plan_t* p, const char* name, int r, int64_t* strides, int* rank) {
   if (!p || !name || r < 0 || r >= p->p.n_req) return SOD2_E_INVALID_ARG;
   int t = p->g->c.g.tensor(name);
-  if (t < 0 || p->p.views[t].empty() || p->p.views[t][0].root < 0) return SOD2_E_INVALID_ARG;
+  if (t < 0 || p->p.views[t].empty() || p->p.root_of[t] < 0) return SOD2_E_INVALID_ARG;
   const View& v = p->p.views[t][r];
   if (rank) *rank = static_cast<int>(v.strides.size());
   if (strides) for (size_t i = 0; i < v.strides.size(); ++i) strides[i] = v.strides[i];

@@ -110,6 +110,12 @@ struct Compiled {
   // every distinct extent expression once: binding evaluates each per request, tensors index the table
   std::vector<Expr> dim_exprs;
   std::vector<std::vector<int>> dim_expr_id;   // [tensor][axis] -> dim_exprs index, -1 if the extent is unknown
+  // Shape classes: tensors of one dim_class have the same extent expressions axis by axis; tensors of one view_class
+  // resolve to the same offsets, extents and strides for every binding (same storage kind, same class of the tensor
+  // they are derived from, same view parameters, same element size and layout rule).  Binding and planning fill
+  // one table row per class and let the other members read it.
+  std::vector<int> dim_class, view_class;
+  int n_dim_classes = 0, n_view_classes = 0;
   // per tensor stored as a view: the operator's parameters read out of its attributes once (Transpose:
   // a = perm; Slice: a = start, b = step per axis of the input), so that planning touches no strings
   struct ViewParam { int op = -1; std::vector<int64_t> a, b; };   // op: 0 Transpose, 1 Reshape, 2 Slice
@@ -164,24 +170,33 @@ struct DimVec {
   bool operator!=(const DimVec& o) const { return !(*this == o); }
 };
 
+// Blocks of host memory for the per-batch tables, recycled between plans: a table of a batch is one to two
+// megabytes, and a fresh allocation of that size is mapped page by page on first touch, which cost more than filling
+// it.  block_acquire returns at least `need` bytes (the capacity in *cap); block_release hands the block back.
+unsigned char* block_acquire(size_t need, size_t* cap);
+void block_release(unsigned char* p, size_t cap);
+
 // [tensor][request] table in one block of memory: binding and planning fill a few thousand small entries per
 // batch, and one vector per tensor made the allocator the largest cost of both.  A row exists once make(t) was
-// called; the others read as empty.  T must be trivially destructible (nothing is destroyed).
+// called; the others read as empty.  A row made with make_shared holds ONE entry that every request index reads
+// (constants, and anything whose extents are equal for all requests of the batch); alias(t, rep) makes a tensor read
+// another tensor's row (tensors of one shape class: most of a model's tensors repeat a handful of shapes).  T must
+// be trivially destructible (nothing is destroyed).
 template <class T>
 class ReqTable {
  public:
   template <class U>
   class RowT {
    public:
-    RowT(U* p, int n) : p_(p), n_(n) {}
+    RowT(U* p, int n, int stride) : p_(p), n_(n), stride_(stride) {}
     bool empty() const { return n_ == 0; }
     size_t size() const { return static_cast<size_t>(n_); }
-    U& operator[](size_t r) const { return p_[r]; }
-    U* begin() const { return p_; }
-    U* end() const { return p_ + n_; }
+    U& operator[](size_t r) const { return p_[r * stride_]; }
+    bool shared() const { return stride_ == 0; }
    private:
     U* p_;
     int n_;
+    int stride_;   // 0: one entry stands for every request
   };
   using Row = RowT<T>;
   using ConstRow = RowT<const T>;
@@ -189,21 +204,37 @@ class ReqTable {
     static_assert(std::is_trivially_destructible<T>::value, "rows are never destroyed");
     n_req_ = n_req;
     has_.assign(n_tensors, 0);
+    at_.resize(n_tensors);
     const size_t need = n_tensors * static_cast<size_t>(n_req) * sizeof(T);
-    if (need > cap_) { raw_.reset(new unsigned char[need]); cap_ = need; }
+    if (need > cap_) { release(); raw_ = block_acquire(need, &cap_); }
   }
+  ReqTable() {}
+  ReqTable(const ReqTable&) = delete;
+  ReqTable& operator=(const ReqTable&) = delete;
+  ~ReqTable() { release(); }
+  // a row with one entry per request
   Row make(size_t t) {
-    T* p = reinterpret_cast<T*>(raw_.get()) + t * n_req_;
-    if (!has_[t]) { for (int r = 0; r < n_req_; ++r) new (p + r) T(); has_[t] = 1; }
-    return Row(p, n_req_);
+    if (!has_[t]) { at_[t] = static_cast<int>(t); T* p = slot(t); for (int r = 0; r < n_req_; ++r) new (p + r) T(); has_[t] = 1; }
+    return (*this)[t];
   }
-  Row operator[](size_t t) { return has_[t] ? Row(reinterpret_cast<T*>(raw_.get()) + t * n_req_, n_req_) : Row(nullptr, 0); }
-  ConstRow operator[](size_t t) const { return has_[t] ? ConstRow(reinterpret_cast<const T*>(raw_.get()) + t * n_req_, n_req_) : ConstRow(nullptr, 0); }
+  // a row whose single entry is what every request reads (the value does not depend on the request in this batch)
+  Row make_shared(size_t t) {
+    if (!has_[t]) { at_[t] = static_cast<int>(t); new (slot(t)) T(); has_[t] = 2; }
+    return (*this)[t];
+  }
+  // tensor t reads the row of tensor `rep` (same content by construction): nothing is copied
+  void alias(size_t t, size_t rep) { at_[t] = at_[rep]; has_[t] = has_[rep]; }
+  bool shared(size_t t) const { return has_[t] == 2; }
+  Row operator[](size_t t) { return has_[t] ? Row(slot(t), n_req_, has_[t] == 2 ? 0 : 1) : Row(nullptr, 0, 1); }
+  ConstRow operator[](size_t t) const { return has_[t] ? ConstRow(slot(t), n_req_, has_[t] == 2 ? 0 : 1) : ConstRow(nullptr, 0, 1); }
   size_t size() const { return has_.size(); }
  private:
-  std::unique_ptr<unsigned char[]> raw_;
+  T* slot(size_t t) const { return reinterpret_cast<T*>(raw_) + static_cast<size_t>(at_[t]) * n_req_; }
+  void release() { if (raw_) block_release(raw_, cap_); raw_ = nullptr; cap_ = 0; }
+  unsigned char* raw_ = nullptr;
   size_t cap_ = 0;
   std::vector<char> has_;
+  std::vector<int> at_;     // which tensor's slot holds the row (its own unless aliased)
   int n_req_ = 0;
 };
 
@@ -219,8 +250,7 @@ Status evaluate_dims(Binding* out);
 Status rebind_runtime(const Binding& base, const std::vector<std::vector<std::pair<int, int64_t>>>& rt_vals, Binding* out);
 
 // ---- plan
-struct View {                 // one tensor of one request, resolved to storage
-  int root = -1;              // tensor id owning the bytes
+struct View {                 // one tensor of one request, resolved to storage (which tensor owns the bytes: Plan::root_of)
   int64_t offset = 0;         // elements from the start of the root's instance for this request
   DimVec dims, strides;       // elements
   int ind_gate = -1;          // >= 0: sample n of this tensor is sample ids[n] of the root (ids = list `ind_list` of that gate's partition)
@@ -257,6 +287,7 @@ struct Plan {
   const Binding* b = nullptr;
   int n_req = 0;
   ReqTable<View> views;                   // [tensor][req]
+  std::vector<int> root_of;               // [tensor] id of the tensor that owns the bytes (-1: not resolved)
   ReqTable<int64_t> inst_off;             // [root tensor][req] byte offset of the request's instance in the root's packed storage
   std::vector<RootBuf> roots;             // [tensor]
   size_t arena_bytes = 0, peak_live_bytes = 0, sum_bytes = 0;

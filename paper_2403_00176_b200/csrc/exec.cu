@@ -185,11 +185,12 @@ struct Builder {
 
   Ptr ptr_of(int t, int r, int64_t extra_elems = 0) const {
     const View& v = p.views[t][r];
-    const RootBuf& R = p.roots[v.root];
+    const int root = p.root_of[t];
+    const RootBuf& R = p.roots[root];
     Ptr q;
     q.where = R.where;
-    q.index = (R.where == RootBuf::CONST) ? v.root : R.io_index;
-    q.off = p.inst_off[v.root][r] + (v.offset + extra_elems) * dtype_size(g.tensors[t].dtype);
+    q.index = (R.where == RootBuf::CONST) ? root : R.io_index;
+    q.off = p.inst_off[root][r] + (v.offset + extra_elems) * dtype_size(g.tensors[t].dtype);
     if (R.where == RootBuf::ARENA) q.off += static_cast<int64_t>(R.arena_off);
     return q;
   }
@@ -214,32 +215,32 @@ struct Builder {
 
   // rows of consecutive requests that form one contiguous matrix are merged into one launch
   struct Seg { int r0, r1; int64_t rows; };
+  std::vector<int64_t> row_count_;
   Status row_segments(const std::vector<int>& tensors, int64_t* cols_out, std::vector<int64_t>* lds, std::vector<Seg>* segs) {
     int nt = static_cast<int>(tensors.size());
     lds->assign(nt, 0);
-    std::vector<std::vector<int64_t>> rows(nt, std::vector<int64_t>(p.n_req));
-    for (int i = 0; i < nt; ++i)
+    row_count_.resize(p.n_req);   // rows of the first tensor, per request (the others must agree)
+    for (int i = 0; i < nt; ++i) {
+      auto views = p.views[tensors[i]];
       for (int r = 0; r < p.n_req; ++r) {
         int64_t rw, cl, ld;
-        if (!as_matrix(p.views[tensors[i]][r], &rw, &cl, &ld)) return fail(E_UNSUPPORTED_OP, "operand " + g.tensors[tensors[i]].name + " is not a row-major matrix view");
+        if (!as_matrix(views[r], &rw, &cl, &ld)) return fail(E_UNSUPPORTED_OP, "operand " + g.tensors[tensors[i]].name + " is not a row-major matrix view");
         if (r == 0) (*lds)[i] = ld;
         else if (ld != (*lds)[i] && rw > 1) return fail(E_UNSUPPORTED_OP, "row pitch differs between requests");
-        rows[i][r] = rw;
-        if (i == 0) cols_out[0] = cl;
-        if (rw != rows[0][r]) return fail(E_SHAPE_CONFLICT, "row counts differ inside a group");
+        if (i == 0) { row_count_[r] = rw; cols_out[0] = cl; }
+        if (rw != row_count_[r]) return fail(E_SHAPE_CONFLICT, "row counts differ inside a group");
       }
+    }
     segs->clear();
     for (int r = 0; r < p.n_req; ++r) {
       bool merge = !segs->empty();
-      if (merge) {
-        for (int i = 0; i < nt; ++i) {
-          Ptr a = ptr_of(tensors[i], segs->back().r0), b = ptr_of(tensors[i], r);
-          int esz = dtype_size(g.tensors[tensors[i]].dtype);
-          if (!same_base(a, b) || b.off != a.off + segs->back().rows * (*lds)[i] * esz) merge = false;
-        }
+      for (int i = 0; i < nt && merge; ++i) {
+        Ptr a = ptr_of(tensors[i], segs->back().r0), b = ptr_of(tensors[i], r);
+        int esz = dtype_size(g.tensors[tensors[i]].dtype);
+        if (!same_base(a, b) || b.off != a.off + segs->back().rows * (*lds)[i] * esz) merge = false;
       }
-      if (merge) { segs->back().r1 = r + 1; segs->back().rows += rows[0][r]; }
-      else segs->push_back({r, r + 1, rows[0][r]});
+      if (merge) { segs->back().r1 = r + 1; segs->back().rows += row_count_[r]; }
+      else segs->push_back({r, r + 1, row_count_[r]});
     }
     return OK;
   }
@@ -380,7 +381,7 @@ struct Builder {
     if (emit && lds[1] != N) return fail(E_UNSUPPORTED_OP, "row statistics need densely packed output rows");
     if (p.stats_layout.size() != g.tensors.size()) p.stats_layout.assign(g.tensors.size(), Plan::StatsLayout());
     auto stats_ptr = [&](int t, int r0, int64_t width, Ptr* out, int64_t* pitch) -> bool {
-      const int root = p.views[t][r0].root;
+      const int root = p.root_of[t];
       const RootBuf& RR = p.roots[root];
       if (RR.where != RootBuf::ARENA || RR.stats_off < 0 || p.views[t][r0].offset != 0) return false;
       const int64_t row0 = p.inst_off[root][r0] / (width * 2);
@@ -560,7 +561,7 @@ struct Builder {
   // the same bytes in the same order: root, offset, extents and strides of request 0 (the members are one segment)
   bool same_view(int t1, int t2) const {
     const View &a = p.views[t1][0], &b = p.views[t2][0];
-    return a.root == b.root && a.offset == b.offset && a.dims == b.dims && a.strides == b.strides;
+    return p.root_of[t1] == p.root_of[t2] && a.offset == b.offset && a.dims == b.dims && a.strides == b.strides;
   }
   // Maximal runs of consecutive chainable GEMM groups with equal row counts.  A member may read rows written by an
   // earlier member only as its A operand or its residual and only as the very view the earlier member wrote
@@ -586,15 +587,15 @@ struct Builder {
           if (g.tensors[t].kind == TKind::CONST || c.storage[t].kind == Storage::FOLDED || p.views[t].empty()) continue;
           for (int m : run) {
             const int o = c.groups[m].out;
-            if (p.views[t][0].root != p.views[o][0].root) continue;
+            if (p.root_of[t] != p.root_of[o]) continue;
             if (!((t == G.a || t == G.res) && same_view(t, o))) ok = false;
           }
         }
         // nothing a member writes may be storage an earlier member reads or writes
         for (int m : run) {
           const Group& E = c.groups[m];
-          for (int t : E.ext_in) if (!p.views[t].empty() && p.views[t][0].root == p.views[G.out][0].root) ok = false;
-          if (p.views[E.out][0].root == p.views[G.out][0].root) ok = false;
+          for (int t : E.ext_in) if (!p.views[t].empty() && p.root_of[t] == p.root_of[G.out]) ok = false;
+          if (p.root_of[E.out] == p.root_of[G.out]) ok = false;
         }
         if (!ok) break;
         run.push_back(static_cast<int>(gj));
@@ -632,7 +633,7 @@ struct Builder {
     };
     std::vector<Mem> ms(n);
     auto stats_ptr = [&](int t, int64_t width, Ptr* out, int64_t* pitch) -> bool {
-      const int root = p.views[t][0].root;
+      const int root = p.root_of[t];
       const RootBuf& RR = p.roots[root];
       if (RR.where != RootBuf::ARENA || RR.stats_off < 0 || p.views[t][0].offset != 0) return false;
       const int64_t row0 = p.inst_off[root][0] / (width * 2);
@@ -678,8 +679,8 @@ struct Builder {
       }
       for (int j = 0; j < i; ++j) {
         const int o = c.groups[ch.groups[j]].out;
-        if (p.views[G.a][0].root == p.views[o][0].root) m.dep_a = j;
-        if (m.hr && p.views[G.res][0].root == p.views[o][0].root) m.dep_r = j;
+        if (p.root_of[G.a] == p.root_of[o]) m.dep_a = j;
+        if (m.hr && p.root_of[G.res] == p.root_of[o]) m.dep_r = j;
       }
       fl[i] = 2.0 * static_cast<double>(m.cm.M) * N * K;
       flops_total += fl[i];
@@ -1599,15 +1600,16 @@ struct Builder {
       // index-indirect operands: offsets of their id lists in the Switch groups' index area
       long long ids_in = -1, ids_res = -1, ids_out = -1;
       {
-        auto ids_of = [&](const View& v, long long* off) -> bool {
+        auto ids_of = [&](int t, long long* off) -> bool {
+          const View& v = p.views[t][r];
           if (v.ind_gate < 0) return true;
           auto it = switch_aux.find(v.ind_gate);
           if (it == switch_aux.end()) return false;
-          const int Nall = static_cast<int>(p.views[v.root][r].dims[0]);
+          const int Nall = static_cast<int>(p.views[p.root_of[t]][r].dims[0]);
           *off = static_cast<long long>(it->second) + (v.ind_list ? static_cast<long long>(Nall) * 4 : 0);
           return true;
         };
-        if (!ids_of(vx, &ids_in) || !ids_of(vo, &ids_out) || (G.res >= 0 && !ids_of(p.views[G.res][r], &ids_res)))
+        if (!ids_of(G.a, &ids_in) || !ids_of(G.out, &ids_out) || (G.res >= 0 && !ids_of(G.res, &ids_res)))
           return fail(E_INTERNAL, "index-indirect convolution operand without a Switch");
       }
       // pixel patch of a tile: the 128-pixel shape that wastes the fewest padded pixels
@@ -1630,9 +1632,9 @@ struct Builder {
       const int K = ks * ks * Cin;
       const long long tiles = static_cast<long long>((cp.Wo + cp.TW - 1) / cp.TW) * ((cp.Ho + cp.TH - 1) / cp.TH) * cp.n_img * ((Cout + bn - 1) / bn);
       // images covered by each operand's tensor map: all images of the root for an index-indirect operand
-      const int n_in_map = static_cast<int>(vx.ind_gate >= 0 ? p.views[vx.root][r].dims[0] : vx.dims[0]);
-      const int n_out_map = static_cast<int>(vo.ind_gate >= 0 ? p.views[vo.root][r].dims[0] : vo.dims[0]);
-      const int n_res_map = G.res >= 0 ? static_cast<int>(p.views[G.res][r].ind_gate >= 0 ? p.views[p.views[G.res][r].root][r].dims[0] : p.views[G.res][r].dims[0]) : 0;
+      const int n_in_map = static_cast<int>(vx.ind_gate >= 0 ? p.views[p.root_of[G.a]][r].dims[0] : vx.dims[0]);
+      const int n_out_map = static_cast<int>(vo.ind_gate >= 0 ? p.views[p.root_of[G.out]][r].dims[0] : vo.dims[0]);
+      const int n_res_map = G.res >= 0 ? static_cast<int>(p.views[G.res][r].ind_gate >= 0 ? p.views[p.root_of[G.res]][r].dims[0] : p.views[G.res][r].dims[0]) : 0;
       if (rows) {
         RowsReq q{px, po, pr, H, Wd, cp.Ho, cp.Wo, cp.n_img, n_in_map, n_out_map, n_res_map, cp, rt, rt_slot, ids_in, ids_res, ids_out};
         // a run-time image count or id lists belong to one request: such a request is launched alone
@@ -1790,7 +1792,7 @@ struct Builder {
       // Per-sample channel sums: reuse the table if it describes this tensor's storage, else pool (two
       // launches) into a new table.  If the block is an in-place, index-indirect one, its last convolution
       // accumulates the executed samples' sums into the table and the next gate finds it up to date.
-      const int xroot = vx.root;
+      const int xroot = p.root_of[G.a];
       const bool whole = vx.offset == 0 && vx.ind_gate < 0;
       const bool have_sums = fuse_part && whole && gapsum_root >= 0 && gapsum_root == xroot;
       size_t table = gapsum_aux;
@@ -1803,7 +1805,7 @@ struct Builder {
         for (size_t ci = 0; ci < c.groups.size() && writer < 0; ++ci) {
           const Group& Cb = c.groups[ci];
           if (Cb.kind != GKind::COMBINE || Cb.gate != G.out || c.storage[Cb.out].kind != Storage::ALIAS) continue;
-          if (p.views[Cb.out].empty() || p.views[Cb.out][0].root != xroot) continue;
+          if (p.views[Cb.out].empty() || p.root_of[Cb.out] != xroot) continue;
           in_place = true;
           for (size_t wi = 0; wi < c.groups.size(); ++wi) {
             const Group& Wg = c.groups[wi];
@@ -2087,9 +2089,26 @@ struct Builder {
     for (const Group& G : c.groups)
       if (!((G.kind == GKind::GEMM && g.tensors[G.a].dtype == DType::F32) || G.kind == GKind::CHAIN || G.kind == GKind::BMM ||
             G.kind == GKind::SUMSQ || G.kind == GKind::TOPK || G.kind == GKind::GATHER || G.kind == GKind::FILL)) p.uses_header = true;
+    // SOD2_HOST_PROFILE: host time of building the launches, per group kind
+    static const bool prof = getenv("SOD2_HOST_PROFILE") != nullptr;
+    struct KindTimes {
+      double us[32] = {0};
+      int n[32] = {0};
+      bool on;
+      explicit KindTimes(bool o) : on(o) {}
+      ~KindTimes() {
+        if (!on) return;
+        for (int k = 0; k < 32; ++k) if (n[k]) fprintf(stderr, "[sod2] launches: %-10s %3d groups %.1f us\n", gkind_name(static_cast<GKind>(k)), n[k], us[k]);
+      }
+    } kt(prof);
     for (size_t gi = 0; gi < c.groups.size(); ++gi) {
       const Group& G = c.groups[gi];
       Status s = OK;
+      struct Tick {
+        KindTimes& kt; int k; std::chrono::steady_clock::time_point q0;
+        Tick(KindTimes& t, int kind) : kt(t), k(kind & 31) { if (kt.on) q0 = std::chrono::steady_clock::now(); }
+        ~Tick() { if (kt.on) { kt.us[k] += std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - q0).count(); ++kt.n[k]; } }
+      } tick(kt, static_cast<int>(G.kind));
       if (gi < p.chain_of.size() && p.chain_of[gi] >= 0) {
         // the first member builds the launch for the whole chain
         if (p.chains[p.chain_of[gi]].groups.front() == static_cast<int>(gi)) s = build_gemm_chain(p.chain_of[gi]);

@@ -757,10 +757,60 @@ static void index_view_params(Compiled* c) {
   }
 }
 
+// Shape classes of the tensors (engine.h): keys are built from what binding and planning read.
+static void index_shape_classes(Compiled* c) {
+  const Graph& g = c->g;
+  const size_t T = g.tensors.size();
+  c->dim_class.assign(T, -1);
+  c->view_class.assign(T, -1);
+  std::map<std::vector<int>, int> dseen;
+  for (size_t t = 0; t < T; ++t) {
+    if (g.tensors[t].S.rank < 0) continue;
+    auto it = dseen.emplace(c->dim_expr_id[t], static_cast<int>(dseen.size())).first;
+    c->dim_class[t] = it->second;
+  }
+  c->n_dim_classes = static_cast<int>(dseen.size());
+  std::map<std::vector<int64_t>, int> vseen;
+  std::vector<char> state(T, 0);   // 1: being visited (a cycle cannot happen; guards against one all the same)
+  std::function<int(int)> cls = [&](int t) -> int {
+    if (c->view_class[t] >= 0 || state[t]) return c->view_class[t];
+    if (t >= static_cast<int>(c->storage.size()) || c->dim_class[t] < 0) return -1;
+    state[t] = 1;
+    const Storage& st = c->storage[t];
+    const Tensor& X = g.tensors[t];
+    std::vector<int64_t> key{static_cast<int64_t>(st.kind), c->dim_class[t]};
+    if (st.kind == Storage::FOLDED) { state[t] = 0; return -1; }
+    if (st.kind == Storage::ROOT) {
+      const bool channels_last = g.has_conv && X.S.rank == 4 && X.kind == TKind::VALUE && !X.is_output && (X.dtype == DType::BF16 || X.dtype == DType::F32);
+      key.push_back(dtype_size(X.dtype));
+      key.push_back(X.kind == TKind::CONST);
+      key.push_back(channels_last);
+      key.push_back(t < c->stats_width.size() ? c->stats_width[t] : 0);
+    } else {
+      const int oc = st.other >= 0 ? cls(st.other) : -1;
+      if (oc < 0) { state[t] = 0; return -1; }
+      key.push_back(oc);
+      key.push_back(st.gate);
+      key.push_back(st.list);
+      const Compiled::ViewParam& vp = c->view_param[t];
+      key.push_back(vp.op);
+      key.push_back(static_cast<int64_t>(vp.a.size()));
+      key.insert(key.end(), vp.a.begin(), vp.a.end());
+      key.insert(key.end(), vp.b.begin(), vp.b.end());
+    }
+    auto it = vseen.emplace(key, static_cast<int>(vseen.size())).first;
+    c->view_class[t] = it->second;
+    state[t] = 0;
+    return it->second;
+  };
+  for (size_t t = 0; t < T; ++t) cls(static_cast<int>(t));
+  c->n_view_classes = static_cast<int>(vseen.size());
+}
+
 Status form_groups(Compiled* c) {
   Fuser f(*c);
   Status s = f.run();
-  if (s == OK) { index_dim_exprs(c); index_view_params(c); }
+  if (s == OK) { index_dim_exprs(c); index_view_params(c); index_shape_classes(c); }
   return s;
 }
 

@@ -7,11 +7,51 @@
 #include <cstdlib>
 #include <cstring>
 #include <map>
+#include <mutex>
 #include <tuple>
 
 #include "engine.h"
 
 namespace sod2 {
+
+// ---- recycled host blocks for the per-batch tables (engine.h)
+namespace {
+struct BlockPool {
+  std::mutex mu;
+  std::vector<std::pair<unsigned char*, size_t>> free_blocks;   // at most POOL_MAX, each at most BLOCK_MAX bytes
+  ~BlockPool() { for (auto& b : free_blocks) delete[] b.first; }
+};
+constexpr size_t POOL_MAX = 16, BLOCK_MAX = size_t(64) << 20;
+BlockPool& block_pool() { static BlockPool p; return p; }
+}  // namespace
+
+unsigned char* block_acquire(size_t need, size_t* cap) {
+  BlockPool& P = block_pool();
+  {
+    std::lock_guard<std::mutex> lk(P.mu);
+    // the smallest recycled block that fits
+    int best = -1;
+    for (size_t i = 0; i < P.free_blocks.size(); ++i)
+      if (P.free_blocks[i].second >= need && (best < 0 || P.free_blocks[i].second < P.free_blocks[best].second)) best = static_cast<int>(i);
+    if (best >= 0) {
+      auto b = P.free_blocks[best];
+      P.free_blocks.erase(P.free_blocks.begin() + best);
+      *cap = b.second;
+      return b.first;
+    }
+  }
+  *cap = need;
+  return new unsigned char[need];
+}
+
+void block_release(unsigned char* p, size_t cap) {
+  BlockPool& P = block_pool();
+  if (cap <= BLOCK_MAX) {
+    std::lock_guard<std::mutex> lk(P.mu);
+    if (P.free_blocks.size() < POOL_MAX) { P.free_blocks.push_back({p, cap}); return; }
+  }
+  delete[] p;
+}
 
 Status bind_dims(const Compiled* c, int n_req, int n_syms, const char* const* names, const int64_t* values, Binding* out) {
   const Graph& g = c->g;
@@ -78,10 +118,19 @@ Status evaluate_dims(Binding* out) {
       uok[r * U + u] = ok;
     }
   }
+  // extents equal for every request of this batch: their tensors get one shared table entry
+  std::vector<char> usame(U, 1);
+  for (size_t u = 0; u < U; ++u)
+    for (int r = 1; r < n_req; ++r)
+      if (uval[r * U + u] != uval[u] || uok[r * U + u] != uok[u]) { usame[u] = 0; break; }
   out->dims.reset(g.tensors.size(), n_req);
+  std::vector<int> class_rep(c->n_dim_classes, -1);   // the tensor whose row the class's other members read
   for (size_t t = 0; t < g.tensors.size(); ++t) {
     const ShapeVal& s = g.tensors[t].S;
     if (s.rank < 0) continue;
+    const int dc = t < c->dim_class.size() ? c->dim_class[t] : -1;
+    if (dc >= 0 && class_rep[dc] >= 0) { out->dims.alias(t, class_rep[dc]); continue; }
+    if (dc >= 0) class_rep[dc] = static_cast<int>(t);
     if (s.rank > MAX_RANK) { out->err = "rank above " + std::to_string(MAX_RANK) + " for " + g.tensors[t].name; return E_UNSUPPORTED_OP; }
     const std::vector<int>& ids = c->dim_expr_id[t];
     bool evaluable = true;
@@ -89,8 +138,10 @@ Status evaluate_dims(Binding* out) {
     for (int r = 0; r < n_req && evaluable; ++r)
       for (int i = 0; i < s.rank; ++i) if (!uok[r * U + ids[i]]) { evaluable = false; break; }
     if (!evaluable) continue;
-    auto per = out->dims.make(t);
-    for (int r = 0; r < n_req; ++r) {
+    bool same = true;
+    for (int i = 0; i < s.rank; ++i) if (!usame[ids[i]]) same = false;
+    auto per = same ? out->dims.make_shared(t) : out->dims.make(t);
+    for (int r = 0; r < (same ? 1 : n_req); ++r) {
       per[r].n = s.rank;
       for (int i = 0; i < s.rank; ++i) {
         const int64_t v = uval[r * U + ids[i]];
@@ -158,7 +209,9 @@ struct Planner {
   const Binding& b;
   Plan& p;
   std::vector<char> resolved;
-  Planner(const Compiled& cc, const Binding& bb, Plan& pp) : c(cc), g(cc.g), b(bb), p(pp), resolved(cc.g.tensors.size(), 0) {}
+  std::vector<int> class_rep;    // per view class: the first tensor resolved in this plan, whose rows the others read
+  Planner(const Compiled& cc, const Binding& bb, Plan& pp)
+      : c(cc), g(cc.g), b(bb), p(pp), resolved(cc.g.tensors.size(), 0), class_rep(cc.n_view_classes, -1) {}
 
   Status fail(Status s, const std::string& m) { p.err = m; return s; }
 
@@ -166,15 +219,34 @@ struct Planner {
     if (b.dims[t].empty()) return fail(E_INTERNAL, "no concrete shape for " + g.tensors[t].name);
     const Tensor& T = g.tensors[t];
     RootBuf& R = p.roots[t];
+    p.root_of[t] = t;
+    const int vc = c.view_class[t];
+    if (vc >= 0 && class_rep[vc] >= 0) {
+      // same extents, element size and layout rule as a root already made: read its rows
+      const int rep = class_rep[vc];
+      p.views.alias(t, rep);
+      p.inst_off.alias(t, rep);
+      const RootBuf& Q = p.roots[rep];
+      R.bytes = Q.bytes;
+      R.stats_off = Q.stats_off;
+      R.stats_rows = Q.stats_rows;
+      R.stats_slots = Q.stats_slots;
+      set_where(T, &R);
+      resolved[t] = 1;
+      return OK;
+    }
+    if (vc >= 0) class_rep[vc] = t;
     auto inst_off = p.inst_off.make(t);
     int64_t off = 0;
     int esz = dtype_size(T.dtype);
     bool per_request = T.kind != TKind::CONST;
-    for (int r = 0; r < p.n_req; ++r) {
-      View& v = p.views[t][r];
-      v.root = t;
+    const int nv = open_views(t, -1);
+    auto views = p.views[t];
+    auto dims = b.dims[t];
+    for (int r = 0; r < nv; ++r) {
+      View& v = views[r];
       v.offset = 0;
-      v.dims = b.dims[t][r];
+      v.dims = dims[r];
       v.strides = contiguous_strides(v.dims);
       // convolution graphs keep rank-4 float intermediates channels-last: [N,C,H,W] with C innermost
       if (g.has_conv && v.dims.size() == 4 && T.kind == TKind::VALUE && !T.is_output &&
@@ -182,8 +254,10 @@ struct Planner {
         const int64_t C = v.dims[1], H = v.dims[2], W = v.dims[3];
         v.strides = {H * W * C, 1, W * C, C};
       }
+    }
+    for (int r = 0; r < p.n_req; ++r) {
       inst_off[r] = per_request ? off : 0;
-      int64_t bytes = numel(v.dims) * esz;
+      int64_t bytes = numel(dims[r]) * esz;
       if (per_request) off += (bytes + 15) & ~int64_t(15);
       else off = bytes;
     }
@@ -198,28 +272,58 @@ struct Planner {
       off += R.stats_rows * R.stats_slots * 8;
     }
     R.bytes = off;
-    if (T.kind == TKind::INPUT) { R.where = RootBuf::INPUT; R.io_index = T.io_index; }
-    else if (T.kind == TKind::CONST) { R.where = RootBuf::CONST; }
-    else if (T.is_output) { R.where = RootBuf::OUTPUT; R.io_index = T.io_index; }
-    else R.where = RootBuf::ARENA;
+    set_where(T, &R);
     resolved[t] = 1;
     return OK;
+  }
+  static void set_where(const Tensor& T, RootBuf* R) {
+    if (T.kind == TKind::INPUT) { R->where = RootBuf::INPUT; R->io_index = T.io_index; }
+    else if (T.kind == TKind::CONST) { R->where = RootBuf::CONST; }
+    else if (T.is_output) { R->where = RootBuf::OUTPUT; R->io_index = T.io_index; }
+    else R->where = RootBuf::ARENA;
+  }
+
+  // Views of `t`: one entry per request, or one shared entry when neither its extents nor the views it derives from
+  // (`other`, if any) depend on the request.  Returns the number of entries to fill.
+  int open_views(int t, int other) {
+    const bool same = b.dims.shared(t) && (other < 0 || p.views.shared(other));
+    if (same) p.views.make_shared(t); else p.views.make(t);
+    return same ? 1 : p.n_req;
   }
 
   Status resolve(int t) {
     if (resolved[t]) return OK;
     const Storage& st = c.storage[t];
     if (st.kind == Storage::FOLDED) { resolved[t] = 1; return OK; }
-    p.views.make(t);
     if (st.kind == Storage::ROOT) return make_root(t);
     if (b.dims[t].empty()) return fail(E_INTERNAL, "no concrete shape for " + g.tensors[t].name);
+    {
+      // a view of the same class as one already resolved: same rows, the bytes belong to this one's own source
+      const int vc = c.view_class[t];
+      if (vc >= 0 && st.other >= 0) {
+        Status s = resolve(st.other);
+        if (s != OK) return s;
+        if (class_rep[vc] >= 0) {
+          p.views.alias(t, class_rep[vc]);
+          p.root_of[t] = p.root_of[st.other];
+          resolved[t] = 1;
+          return OK;
+        }
+        class_rep[vc] = t;
+      }
+      if (st.other >= 0) {
+        Status s = resolve(st.other);
+        if (s != OK) return s;
+        p.root_of[t] = p.root_of[st.other];
+      }
+    }
     if (st.kind == Storage::ALIAS) {
       Status s = resolve(st.other);
       if (s != OK) return s;
-      for (int r = 0; r < p.n_req; ++r) {
+      const int nv = open_views(t, st.other);
+      for (int r = 0; r < nv; ++r) {
         const View& vo = p.views[st.other][r];
         View& v = p.views[t][r];
-        v.root = vo.root;
         v.offset = vo.offset;
         v.dims = b.dims[t][r];
         v.strides = vo.strides;
@@ -232,10 +336,10 @@ struct Planner {
       // the samples of `other` selected by an id list: same storage, same strides, own (upper-bound) extents
       Status s = resolve(st.other);
       if (s != OK) return s;
-      for (int r = 0; r < p.n_req; ++r) {
+      const int nv = open_views(t, st.other);
+      for (int r = 0; r < nv; ++r) {
         const View& vo = p.views[st.other][r];
         View& v = p.views[t][r];
-        v.root = vo.root;
         v.offset = vo.offset;
         v.dims = b.dims[t][r];
         v.strides = vo.strides;
@@ -251,10 +355,10 @@ struct Planner {
       Status s = resolve(o);
       if (s != OK) return s;
       const std::vector<int64_t>& perm = c.view_param[t].a;
-      for (int r = 0; r < p.n_req; ++r) {
+      const int nv = open_views(t, o);
+      for (int r = 0; r < nv; ++r) {
         const View& vo = p.views[o][r];
         View& v = p.views[t][r];
-        v.root = vo.root;
         v.offset = vo.offset;
         v.dims = b.dims[t][r];
         v.strides.assign(v.dims.size(), 0);
@@ -273,10 +377,10 @@ struct Planner {
     const std::vector<int64_t>& sl_start = vp.a;
     const std::vector<int64_t>& sl_step = vp.b;
     if (kind == 2 && sl_start.size() != p.views[in][0].dims.size()) return fail(E_INTERNAL, "slice parameters of " + g.tensors[t].name);
-    for (int r = 0; r < p.n_req; ++r) {
+    const int nv = open_views(t, in);
+    for (int r = 0; r < nv; ++r) {
       const View& vi = p.views[in][r];
       View& v = p.views[t][r];
-      v.root = vi.root;
       v.offset = vi.offset;
       v.dims = b.dims[t][r];
       if (kind == 0) {
@@ -303,6 +407,7 @@ struct Planner {
     size_t T = g.tensors.size();
     p.inst_off.reset(T, p.n_req);
     p.views.reset(T, p.n_req);   // rows are made per tensor when it is resolved
+    p.root_of.assign(T, -1);
     p.roots.assign(T, RootBuf());
     // resolve every tensor a group touches
     for (auto& G : c.groups) {
@@ -331,7 +436,7 @@ struct Planner {
       }
       auto touch = [&](int t, bool def) {
         if (c.storage[t].kind == Storage::FOLDED || !resolved[t]) return;
-        int root = p.views[t][0].root;
+        int root = p.root_of[t];
         if (root < 0) return;
         RootBuf& R = p.roots[root];
         if (R.def_step < 0 || lo < R.def_step) R.def_step = lo;
@@ -346,7 +451,10 @@ struct Planner {
     if (prof) {
       auto t3 = std::chrono::steady_clock::now();
       auto us = [](auto a, auto b) { return std::chrono::duration<double, std::micro>(b - a).count(); };
-      fprintf(stderr, "[sod2] plan: views %.1f us, liveness %.1f us, arena %.1f us\n", us(t0, t1), us(t1, t2), us(t2, t3));
+      int n_res = 0, n_rep = 0;
+      for (size_t t = 0; t < T; ++t) n_res += resolved[t] && c.storage[t].kind != Storage::FOLDED;
+      for (int r : class_rep) n_rep += r >= 0;
+      fprintf(stderr, "[sod2] plan: views %.1f us (%d tensors, %d table rows filled), liveness %.1f us, arena %.1f us\n", us(t0, t1), n_res, n_rep, us(t1, t2), us(t2, t3));
     }
     return s;
   }
