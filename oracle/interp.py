@@ -20,7 +20,9 @@ stable argsort; NonZero against numpy.nonzero; Switch/Combine against masked
 execute-all; the Fig. 4 chain against explicit loops; GlobalAveragePool, the gate chain
 (pool -> linear -> Greater, with a logit of exactly zero), LayerNorm and Softmax values against
 loops; Greater, Range, ConstantOfShape, Cast, Div, Sub, Reshape's 0 / -1 rules, ReduceSumSquare,
-Relu, Shape, Transpose, Concat, Gather, Slice and Expand against literal arrays.  Nothing here is
+Relu, Shape, Transpose, Concat, Gather, Slice and Expand against literal arrays; Resize / Upsample (nearest)
+against numpy.repeat for integer scales, a literal array for a fractional ratio and
+torch.nn.functional.interpolate.  Nothing here is
 "parity unpinned" except the reading of tolerances and decision bands, which is a convention,
 not a value.
 """
@@ -301,6 +303,19 @@ def run(text: str, consts: Dict[str, np.ndarray], inputs: Dict[str, np.ndarray],
         elif op == "Expand":
             # broadcast x against the VALUE of the shape operand (multidirectional: either side may be 1)
             out = np.array(x[0] * np.ones([int(v) for v in x[1]], dtype=x[0].dtype))
+        elif op in ("Resize", "Upsample"):
+            # nearest neighbour (Table 2 lists Resize / Upsample as input shape & value determined): the output extents
+            # are the VALUE of the sizes operand, or extent * integer scale; output index o along an axis reads source
+            # index floor(o * in / out)
+            src = x[0]
+            if len(x) > 1:
+                sizes = [int(v) for v in np.asarray(x[1]).reshape(-1)]
+            else:
+                sizes = [d * int(v) for d, v in zip(src.shape, a["scales"].split(","))]
+            out = src
+            for ax, (n_in, n_out) in enumerate(zip(src.shape, sizes)):
+                pick = [min(n_in - 1, (o * n_in) // n_out) for o in range(n_out)]
+                out = np.take(out, pick, axis=ax)
         elif op == "Greater":
             out = (x[0] > x[1])
         elif op == "Switch":

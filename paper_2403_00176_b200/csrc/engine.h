@@ -44,6 +44,7 @@ enum class GKind {
   TOPK,        // TopK over the last axis: values + int64 indices
   GATHER,      // Gather along one axis by an int64 index tensor computed on the device
   FILL,        // Range / ConstantOfShape whose extent is only known at bind time: out[i] = start + i * step
+  RESIZE,      // Resize / Upsample, nearest neighbour: out[.., o, ..] = x[.., floor(o * in / out), ..]
   UNSUPPORTED
 };
 const char* gkind_name(GKind k);

@@ -1191,6 +1191,41 @@ struct Builder {
     return OK;
   }
 
+  // ------------------------------------------------------------------------------ Resize / Upsample (nearest)
+  Status build_resize(int gi, const Group& G) {
+    const Tensor& X = g.tensors[G.a];
+    if (g.tensors[G.out].dtype != X.dtype) return fail(E_UNSUPPORTED_OP, "Resize: output type differs from the input type");
+    const int esz = dtype_size(X.dtype);
+    if (esz != 2 && esz != 4 && esz != 8) return fail(E_UNSUPPORTED_OP, "Resize: element size");
+    for (int r = 0; r < p.n_req; ++r) {
+      const View &vx = p.views[G.a][r], &vo = p.views[G.out][r];
+      const int rank = static_cast<int>(vo.dims.size());
+      if (rank != static_cast<int>(vx.dims.size()) || rank > 6) return fail(E_UNSUPPORTED_OP, "Resize: rank (at most 6, equal to the input's)");
+      k::ResizeParams rp{};
+      rp.rank = rank;
+      rp.esz = esz;
+      rp.total = numel(vo.dims);
+      if (rp.total == 0) continue;
+      if (numel(vx.dims) == 0) return fail(E_BAD_DIM, "Resize: empty input, non-empty output");
+      for (int d = 0; d < rank; ++d) {
+        rp.in_dim[d] = vx.dims[d]; rp.out_dim[d] = vo.dims[d];
+        rp.in_stride[d] = vx.strides[d]; rp.out_stride[d] = vo.strides[d];
+        rp.order[d] = rank - 1 - d;
+      }
+      // walk the output in its storage order: axes by ascending stride
+      std::stable_sort(rp.order, rp.order + rank, [&](int a, int b) { return vo.strides[a] < vo.strides[b]; });
+      Ptr px = ptr_of(G.a, r), po = ptr_of(G.out, r);
+      add(gi, 1, [=](const RunCtx& x) mutable {
+        rp.x = x.resolve(px);
+        rp.out = x.resolve(po);
+        const unsigned grid = static_cast<unsigned>(std::max<long long>(1, std::min<long long>((rp.total + 255) / 256, 148 * 16)));
+        k::resize_nearest<<<grid, 256, 0, x.stream>>>(rp);
+        return cudaGetLastError();
+      });
+    }
+    return OK;
+  }
+
   // ------------------------------------------------------------------------------ top-k keep
   Status build_topk(int gi, const Group& G) {
     if (g.tensors[G.a].dtype != DType::BF16) return fail(E_UNSUPPORTED_OP, "top-k keep is bf16 only");
@@ -2088,7 +2123,7 @@ struct Builder {
     p.uses_header = false;
     for (const Group& G : c.groups)
       if (!((G.kind == GKind::GEMM && g.tensors[G.a].dtype == DType::F32) || G.kind == GKind::CHAIN || G.kind == GKind::BMM ||
-            G.kind == GKind::SUMSQ || G.kind == GKind::TOPK || G.kind == GKind::GATHER || G.kind == GKind::FILL)) p.uses_header = true;
+            G.kind == GKind::SUMSQ || G.kind == GKind::TOPK || G.kind == GKind::GATHER || G.kind == GKind::FILL || G.kind == GKind::RESIZE)) p.uses_header = true;
     // SOD2_HOST_PROFILE: host time of building the launches, per group kind
     static const bool prof = getenv("SOD2_HOST_PROFILE") != nullptr;
     struct KindTimes {
@@ -2134,6 +2169,7 @@ struct Builder {
         case GKind::TOPK: s = build_topk_rows(static_cast<int>(gi), G); break;
         case GKind::GATHER: s = build_gather(static_cast<int>(gi), G); break;
         case GKind::FILL: s = build_fill(static_cast<int>(gi), G); break;
+        case GKind::RESIZE: s = build_resize(static_cast<int>(gi), G); break;
         default: return fail(E_UNSUPPORTED_OP, std::string("no executor yet for group kind ") + gkind_name(G.kind));
       }
       if (s != OK) return s;

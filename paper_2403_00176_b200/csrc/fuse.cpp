@@ -31,6 +31,7 @@ const char* gkind_name(GKind k) {
     case GKind::TOPK: return "topk";
     case GKind::GATHER: return "gather";
     case GKind::FILL: return "fill";
+    case GKind::RESIZE: return "resize";
     default: return "unsupported";
   }
 }
@@ -528,6 +529,10 @@ struct Fuser {
       } else if (op == "Expand") {
         // a copy through the chain kernel: the operand is read with stride 0 along the dims it broadcasts over
         Group G; G.kind = GKind::CHAIN; G.nodes = {nid}; G.a = n.ins[0]; G.out = n.outs[0];
+        finish(G);
+      } else if (op == "Resize" || op == "Upsample") {
+        Group G; G.kind = GKind::RESIZE; G.nodes = {nid}; G.a = n.ins[0]; G.out = n.outs[0];
+        if (n.attr_s("mode", "nearest") != "nearest") { G.kind = GKind::UNSUPPORTED; G.why = "Resize: only nearest-neighbour interpolation has an executor"; }
         finish(G);
       } else if (op == "Range" || op == "ConstantOfShape") {
         Group G; G.kind = GKind::FILL; G.nodes = {nid}; G.out = n.outs[0]; G.act = op == "Range";

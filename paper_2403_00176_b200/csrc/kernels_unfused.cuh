@@ -126,6 +126,36 @@ __global__ void __launch_bounds__(256) gather_axis(GatherParams p) {
   }
 }
 
+// Resize / Upsample, nearest neighbour (Table 2: input shape & value determined output shape): along every axis the
+// source index of output index o is floor(o * in / out), the "asymmetric" coordinate rule with the index rounded down;
+// for integer scales this repeats every element `scale` times.  Operands are addressed through their strides (element
+// units), so packed and channels-last storage both work; one thread per output element in the output's storage
+// order (`order[k]` = k-th fastest axis of the output), so stores coalesce.
+struct ResizeParams {
+  const void* x; void* out;
+  long long in_dim[6], out_dim[6], in_stride[6], out_stride[6];
+  int order[6];
+  int rank, esz;
+  long long total;
+};
+__global__ void __launch_bounds__(256) resize_nearest(ResizeParams p) {
+  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < p.total; i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    long long rem = i, so = 0, si = 0;
+    for (int k = 0; k < p.rank; ++k) {
+      const int ax = p.order[k];
+      const long long o = rem % p.out_dim[ax];
+      rem /= p.out_dim[ax];
+      long long src = o * p.in_dim[ax] / p.out_dim[ax];
+      if (src > p.in_dim[ax] - 1) src = p.in_dim[ax] - 1;
+      so += o * p.out_stride[ax];
+      si += src * p.in_stride[ax];
+    }
+    if (p.esz == 2) reinterpret_cast<uint16_t*>(p.out)[so] = reinterpret_cast<const uint16_t*>(p.x)[si];
+    else if (p.esz == 4) reinterpret_cast<uint32_t*>(p.out)[so] = reinterpret_cast<const uint32_t*>(p.x)[si];
+    else reinterpret_cast<uint64_t*>(p.out)[so] = reinterpret_cast<const uint64_t*>(p.x)[si];
+  }
+}
+
 // out[i] = start + i * step for i < n: Range (int64) and ConstantOfShape (step 0; fp32, bf16 or int64).
 struct FillParams { void* out; long long n; double start, step; int dtype; /* 0 f32, 1 bf16, 2 i64 */ };
 __global__ void __launch_bounds__(256) fill_linear(FillParams p) {

@@ -416,6 +416,8 @@ struct Planner {
       for (int t : G.ext_out) { Status s = resolve(t); if (s != OK) return s; }
     }
     for (int t : g.outputs) { Status s = resolve(t); if (s != OK) return s; }
+    // an input of which only the shape is read still has an instance per request in the caller's buffer
+    for (int t : g.inputs) if (!b.dims[t].empty()) { Status s = resolve(t); if (s != OK) return s; }
     static const bool prof = getenv("SOD2_HOST_PROFILE") != nullptr;
     auto t1 = std::chrono::steady_clock::now();
     // GEMM groups that will run as one persistent kernel: their members overlap in time

@@ -332,7 +332,7 @@ void insert_layout_nodes(Graph* g) {
     Tensor& T = g->tensors[t];
     if (T.producer < 0 || T.kind != TKind::VALUE) continue;
     const std::string& pop = g->nodes[T.producer].op;
-    if (pop != "Conv" && pop != "Add" && pop != "Relu" && pop != "Combine") continue;   // rank known only after RDP: restrict to conv-chain producers
+    if (pop != "Conv" && pop != "Add" && pop != "Relu" && pop != "Combine" && pop != "Resize" && pop != "Upsample") continue;   // rank known only after RDP: restrict to conv-chain producers
     int cl = new_tensor(g, g->tensors[t].name + "@cl");
     Tensor& O = g->tensors[t];
     Tensor& C = g->tensors[cl];

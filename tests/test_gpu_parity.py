@@ -193,6 +193,42 @@ def test_expand_range_constant_of_shape_executors():
         assert O.rel_err(outs[r]["z"], env["z"]) <= BF16_TOL
 
 
+def test_resize_upsample_nearest_executor():
+    # Resize / Upsample (nearest): integer scales, and a sizes operand computed from the Shape of another runtime-sized
+    # tensor (the output extents are expressions of the bound symbols); fp32 packed, bf16 behind a convolution
+    # (channels-last storage), fractional ratios both up and down.  A copy: the values must be bit-exact.
+    ir = ("sym H 1 512\nsym W 1 512\nsym P 1 512\nsym Q 1 512\ninput x f32 [2,3,H,W]\ninput t f32 [2,3,P,Q]\n"
+          "node Resize x -> a {scales=1,1,2,3}\nnode Shape t -> st\nnode Resize x st -> b\nnode Upsample a -> c {scales=1,2,1,1}\n"
+          "output a\noutput b\noutput c\n")
+    rng = np.random.default_rng(12)
+    reqs = [Request({"H": h, "W": w, "P": pp, "Q": q}, {"x": rng.standard_normal((2, 3, h, w)).astype(np.float32), "t": np.zeros((2, 3, pp, q), np.float32)})
+            for h, w, pp, q in ((1, 1, 5, 4), (4, 5, 6, 3), (37, 29, 100, 11), (64, 96, 33, 200))]
+    wl = WL.Workload("resize_f32", "f32", ir, {}, ["H", "W", "P", "Q"], ["a", "b", "c"], {"batch_fn": lambda j: reqs})
+    s, p, outs = run_batch(wl, reqs)
+    kinds = [s.graph.group_info(i)["kind"] for i in range(s.graph.num_groups())]
+    assert kinds.count("resize") == 3, kinds
+    for r, req in enumerate(reqs):
+        env = O.run(ir, {}, req.inputs)
+        for name in ("a", "b", "c"):
+            assert outs[r][name].shape == env[name].shape, (name, outs[r][name].shape, env[name].shape)
+            assert np.array_equal(outs[r][name].astype(np.float64), env[name]), (r, name)
+    # bf16, channels-last: 1x1 convolution -> Upsample x2 -> 1x1 convolution (the feature-pyramid pattern)
+    C = 64
+    ir2 = (f"sym H 1 512\nsym W 1 512\ninput x bf16 [1,{C},H,W]\nconst w1 bf16 [{C},{C},1,1]\nconst w2 bf16 [{C},{C},1,1]\n"
+           "node Conv x w1 -> y {stride=1 pad=0}\nnode Resize y -> u {scales=1,1,2,2}\nnode Conv u w2 -> z {stride=1 pad=0}\noutput z\noutput u\n")
+    consts = {"w1": bf16_round((rng.standard_normal((C, C, 1, 1)) / 8).astype(np.float32)), "w2": bf16_round((rng.standard_normal((C, C, 1, 1)) / 8).astype(np.float32))}
+    reqs2 = [Request({"H": h, "W": w}, {"x": bf16_round(rng.standard_normal((1, C, h, w)).astype(np.float32))}) for h, w in ((8, 8), (13, 21))]
+    wl2 = WL.Workload("resize_bf16", "bf16", ir2, consts, ["H", "W"], ["z", "u"], {"batch_fn": lambda j: reqs2})
+    for req in reqs2:
+        s2, p2, outs2 = run_batch(wl2, [req])
+        env = O.run(ir2, consts, req.inputs)
+        u = outs2[0]["u"].astype(np.float64)
+        assert u.shape == env["u"].shape
+        # the upsampled map repeats the convolution output exactly
+        assert np.array_equal(u[:, :, ::2, ::2], u[:, :, 1::2, 1::2]) and np.array_equal(u[:, :, ::2, ::2], u[:, :, ::2, 1::2])
+        assert O.rel_err(u, env["u"]) <= BF16_TOL and O.rel_err(outs2[0]["z"], env["z"]) <= BF16_TOL
+
+
 def test_topk_keep_with_nan_rows_keeps_exactly_k():
     # a row of NaN (an overflow upstream) has a NaN score, which compares false with everything: it must rank last, not
     # be kept by every chunk, so that exactly k rows are kept (in ascending order) and nothing is written past them

@@ -387,3 +387,26 @@ def test_expand_literals():
     env = _run("input x f32 [3,1]\niconst s1 i64 [2] = 3 4\niconst s2 i64 [3] = 2 1 4\nnode Expand x s1 -> a\nnode Expand x s2 -> b\n", {"x": x})
     assert env["a"].tolist() == [[1.0] * 4, [2.0] * 4, [3.0] * 4]
     assert env["b"].shape == (2, 3, 4) and env["b"][1].tolist() == [[1.0] * 4, [2.0] * 4, [3.0] * 4]   # the 1 in the target keeps x's 3
+
+
+def test_resize_nearest_vs_repeat_literal_and_torch():
+    import torch
+    import torch.nn.functional as F
+    x = rng.standard_normal((2, 3, 4, 5))
+    env = _run("input x f32 [2,3,4,5]\niconst sz i64 [4] = 2 3 6 3\nnode Resize x -> a {scales=1,1,2,3}\nnode Upsample x -> b {scales=1,2,1,1}\n"
+               "node Resize x sz -> c\n", {"x": x})
+    # integer scales repeat every element: numpy.repeat along each axis is the definition
+    assert np.array_equal(env["a"], np.repeat(np.repeat(x, 2, axis=2), 3, axis=3))
+    assert np.array_equal(env["b"], np.repeat(x, 2, axis=1))
+    # fractional ratio 4 -> 6 rows and 5 -> 3 columns: source indices floor(o * in / out) written out by hand
+    rows, cols = [0, 0, 1, 2, 2, 3], [0, 1, 3]
+    for i, r_ in enumerate(rows):
+        for j, c_ in enumerate(cols):
+            assert np.array_equal(env["c"][:, :, i, j], x[:, :, r_, c_])
+    # the library's nearest mode uses the same rule (source = floor(o * in / out))
+    t = torch.from_numpy(x)
+    assert np.array_equal(env["a"], F.interpolate(t, scale_factor=(2, 3), mode="nearest").numpy())
+    assert np.array_equal(env["c"], F.interpolate(t, size=(6, 3), mode="nearest").numpy())
+    # a 1-D literal
+    e2 = _run("input v f32 [3]\nnode Resize v -> w {scales=2}\n", {"v": np.array([1.0, 2.0, 3.0])})
+    assert e2["w"].tolist() == [1.0, 1.0, 2.0, 2.0, 3.0, 3.0]
