@@ -223,6 +223,11 @@ sod2_status sod2_plan_memory(const sod2_plan_t* p, size_t* arena_bytes, size_t* 
  * HBM-bound groups) and bytes = every external input and output once, constants once, nothing for
  * tensors that stay inside the group. */
 sod2_status sod2_plan_group_cost(const sod2_plan_t* p, int group, double* flops, double* bytes);
+/* *on_side = 1 if the group's kernels run on the plan's second stream beside the previous group (Section 4.3 orders
+ * the groups; two consecutive groups overlap only where neither reads what the other writes AND both read the same
+ * tensor, so that the memory plan, which knows liveness by step, cannot hand one of them a slot the other still
+ * reads), else 0. */
+sod2_status sod2_plan_group_on_side_stream(const sod2_plan_t* p, int group, int* on_side);
 /* True shape of an output after a run (execution-determined extents are read back from the device;
  * synchronises cuda_stream). */
 sod2_status sod2_run_output_shape(sod2_plan_t* p, const void* arena, void* cuda_stream, int request, int output,

@@ -78,6 +78,7 @@ def _load() -> C.CDLL:
         "sod2_plan_instance_offset": [vp, cp, i32, P(sz)],
         "sod2_plan_memory": [vp, P(sz), P(sz), P(sz)],
         "sod2_plan_group_cost": [vp, i32, P(C.c_double), P(C.c_double)],
+        "sod2_plan_group_on_side_stream": [vp, i32, P(C.c_int)],
         "sod2_plan_tensor_strides": [vp, cp, i32, P(i64), P(i32)],
         "sod2_run_output_shape": [vp, vp, vp, i32, i32, P(i64), P(i32)],
         "sod2_nonzero_static": [vp, i32, i32, P(i64), vp, vp, vp],
@@ -105,7 +106,7 @@ EXPORTS = ["sod2_graph_create", "sod2_graph_destroy", "sod2_graph_set_const", "s
            "sod2_run", "sod2_run_graph", "sod2_run_exact", "sod2_run_timed", "sod2_run_timed_repeat", "sod2_plan_device_status", "sod2_plan_poison_arena", "sod2_plan_check_guards", "sod2_graph_tensor_info", "sod2_graph_tensor_value", "sod2_graph_tensor_dtype",
            "sod2_graph_num_ops", "sod2_graph_op_info", "sod2_graph_num_groups", "sod2_graph_group_info",
            "sod2_graph_num_subgraphs", "sod2_graph_rdp_sweeps", "sod2_classify", "sod2_graph_reanalyse", "sod2_graph_order_info",
-           "sod2_binding_shape", "sod2_plan_slot", "sod2_plan_instance_offset", "sod2_plan_memory", "sod2_plan_group_cost", "sod2_plan_tensor_strides",
+           "sod2_binding_shape", "sod2_plan_slot", "sod2_plan_instance_offset", "sod2_plan_memory", "sod2_plan_group_cost", "sod2_plan_group_on_side_stream", "sod2_plan_tensor_strides",
            "sod2_run_output_shape", "sod2_nonzero_static", "sod2_launch_empty", "sod2_selftest_bounded_wait", "sod2_last_error"]
 
 
@@ -371,6 +372,11 @@ class Plan:
         f, b = C.c_double(), C.c_double()
         _check(lib.sod2_plan_group_cost(self.h, group, C.byref(f), C.byref(b)), self.h)
         return f.value, b.value
+
+    def group_on_side_stream(self, group: int) -> bool:
+        v = C.c_int()
+        _check(lib.sod2_plan_group_on_side_stream(self.h, group, C.byref(v)), self.h)
+        return bool(v.value)
 
     def output_shape(self, arena: int, stream: int, request: int, output: int) -> List[int]:
         dims = (C.c_int64 * 16)()

@@ -439,6 +439,12 @@ sod2_status sod2_plan_group_cost(const sod2_plan_t* p, int group, double* flops,
   return SOD2_OK;
 }
 
+sod2_status sod2_plan_group_on_side_stream(const sod2_plan_t* p, int group, int* on_side) {
+  if (!p || !on_side || group < 0 || group >= static_cast<int>(p->p.side_group.size())) return SOD2_E_INVALID_ARG;
+  *on_side = p->p.side_group[group] ? 1 : 0;
+  return SOD2_OK;
+}
+
 sod2_status sod2_plan_memory(const sod2_plan_t* p, size_t* arena, size_t* peak, size_t* sum) {
   if (!p) return SOD2_E_INVALID_ARG;
   if (arena) *arena = p->p.arena_bytes;

@@ -352,3 +352,30 @@ def test_run_rejects_bad_arena_before_touching_the_device():
     with pytest.raises(B.Sod2Error) as e:
         p.run([0], [fake], fake, p.arena_bytes, 0)
     assert e.value.status_name == "SOD2_E_INVALID_ARG"
+
+
+def test_side_stream_only_for_a_pooling_group_that_reads_the_layout_groups_own_input():
+    # A pooling group runs beside the preceding layout change only when both read the SAME tensor: the memory plan
+    # knows liveness by step, so with different inputs the pooled output could be given the slot of a tensor the
+    # layout kernel still reads.  Case 1: the output's layout change and the pooling both read the last block (the
+    # documented case).  Case 2: the layout change reads X, the pooling reads Y and writes an arena tensor.
+    C = 64
+    ir1 = (f"sym H 8 64\nsym W 8 64\ninput x bf16 [1,{C},H,W]\nconst w bf16 [{C},{C},1,1]\n"
+           "node Conv x w -> y {stride=1 pad=0}\nnode GlobalAveragePool y -> gp\noutput gp\noutput y\n")
+    g1 = B.Graph(ir1, 0)
+    p1 = g1.bind_dims(["H", "W"], [[16, 24]]).plan()
+    kinds1 = [g1.group_info(i)["kind"] for i in range(g1.num_groups())]
+    gi = kinds1.index("gap")
+    assert kinds1[gi - 1] == "layout" and p1.group_on_side_stream(gi)
+    ir2 = (f"sym H 8 64\nsym W 8 64\ninput x bf16 [1,{C},H,W]\ninput z bf16 [1,{C},H,W]\nconst w bf16 [{C},{C},1,1]\nconst v bf16 [{C},{C},1,1]\n"
+           "node Conv x w -> y {stride=1 pad=0}\nnode GlobalAveragePool z -> gp\nnode Conv z v -> u {stride=1 pad=0}\nnode Sigmoid gp -> sg\n"
+           "output sg\noutput y\noutput u\n")
+    g2 = B.Graph(ir2, 0)
+    p2 = g2.bind_dims(["H", "W"], [[16, 24]]).plan()
+    kinds2 = [g2.group_info(i)["kind"] for i in range(g2.num_groups())]
+    gi2 = kinds2.index("gap")
+    # the group before the pooling is the layout change of the convolution output u; the pooling reads z and writes an
+    # arena tensor (the Sigmoid's input): different tensors, so it stays on the main stream
+    assert kinds2[gi2 - 1] == "layout" and kinds2[gi2 - 2] == "conv", kinds2
+    assert not any(p2.group_on_side_stream(i) for i in range(len(kinds2))), kinds2
+    assert p2.slot("gp")["bytes"] > 0
