@@ -19,10 +19,10 @@ namespace {
 struct BlockPool {
   std::mutex mu;
   std::vector<std::pair<unsigned char*, size_t>> free_blocks;   // at most POOL_MAX, each at most BLOCK_MAX bytes
-  ~BlockPool() { for (auto& b : free_blocks) delete[] b.first; }
 };
-constexpr size_t POOL_MAX = 16, BLOCK_MAX = size_t(64) << 20;
-BlockPool& block_pool() { static BlockPool p; return p; }
+constexpr size_t POOL_MAX = 8, BLOCK_MAX = size_t(16) << 20;   // at most 128 MB parked
+// never destroyed: handles may be released after the static destructors of this library have run
+BlockPool& block_pool() { static BlockPool* p = new BlockPool; return *p; }
 }  // namespace
 
 unsigned char* block_acquire(size_t need, size_t* cap) {
