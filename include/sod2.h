@@ -48,7 +48,7 @@ typedef enum {
 #define SOD2_OPT_NO_SEP 32u /* groups run in their default topological order: no static execution planning (Section 4.3) */
 #define SOD2_OPT_LN_FOLD 128u /* a LayerNorm between bf16 GEMMs is folded into its neighbours (Section 4.2: fusion removes the materialised intermediate): the producing GEMM writes per-row statistics, the consuming GEMMs read the raw rows and normalise in their epilogues, the normalised tensor is never stored.  Opt-in: measured slower on the encoder workloads, where the LayerNorm kernel runs beside the next GEMM's pipeline fill */
 #define SOD2_OPT_GUARD_BANDS 512u /* debugging aid: every arena tensor gets a slot of its own (a band another tensor may cover at another time proves nothing) with 256 bytes behind it, also behind the scratch regions (sod2_plan_poison_arena / sod2_plan_check_guards) */
-#define SOD2_OPT_GEMM_PAIR 1024u /* bf16 GEMMs on CTA pairs: two CTAs of a cluster share a 256 x N tile, each loading its own rows and half of the weight tile (tcgen05.mma.cta_group::2), chosen per bound shape where the estimated makespan is shorter (Section 4.4.2: one more code version).  Opt-in: results equal the single-CTA kernel's, measured slower at a few thousand rows (the pair's MMA instructions retire at about half the single-CTA rate in this kernel) */
+#define SOD2_OPT_GEMM_PAIR 1024u /* bf16 GEMMs on CTA pairs: two CTAs of a cluster share a 256 x N tile, each loading its own rows and half of the weight tile (tcgen05.mma.cta_group::2), chosen per bound shape where the estimated makespan is shorter (Section 4.4.2: one more code version).  Opt-in: results equal the single-CTA kernel's; measured 0.5 - 1.5 us slower per kernel at a few thousand rows, where the main loop does not wait for operands and the cluster launch costs more than the saved loads */
 #define SOD2_OPT_GEMM_CHAIN 256u /* consecutive GEMM groups that depend on each other row block by row block run as one persistent kernel with per-row-block dependency counters in the arena header (their operands stay live over the whole chain).  Opt-in: measured slower than one launch per GEMM at a few thousand rows */
 #define SOD2_OPT_SPLITK_LN 4u /* bf16 GEMM (+bias, +residual) -> LayerNorm as one group: split-K GEMM into fp32 slabs + finishing kernel */
 

