@@ -269,6 +269,19 @@ sod2_status sod2_launch_empty(void* cuda_stream);
  * SOD2_E_CUDA; message through sod2_last_error(NULL). */
 sod2_status sod2_selftest_bounded_wait(void* dev_status_word, void* cuda_stream);
 
+/* Measurement of the tensor pipe's issue rate (no counterpart in the paper: it records the machine facts behind the
+ * multi-version kernels of Section 4.4.2 and lets a test pin them).  On `clusters` pairs of SMs (1..74), one thread
+ * per CTA (pair = 0: tcgen05.mma.cta_group::1, 128 x n_cols x 16, both CTAs of every cluster at once) or one per CTA
+ * pair (pair = 1: cta_group::2, 256 x n_cols x 16) issues `iters` bf16 MMAs on fixed shared-memory operands, in
+ * stages of `per_stage` instructions.  handshake: 0 = MMAs only, 1 = a tcgen05.commit after every stage, 2 = the
+ * full / empty barrier handshake of the GEMM main loops after every stage (all waits satisfied at once).
+ * *cycles_per_mma (host) = SM cycles of the first issuing thread / iters.  n_cols in {64, 128, 256}; per_stage in
+ * 1..64 and dividing iters; iters <= 65536.  Allocates and frees one small device buffer; synchronises cuda_stream.
+ * Every wait in the kernel is bounded.  Errors: SOD2_E_INVALID_ARG, SOD2_E_CUDA, SOD2_E_TIMEOUT (a wait ran out);
+ * message through sod2_last_error(NULL). */
+sod2_status sod2_selftest_mma_rate(int pair, int n_cols, int per_stage, int handshake, int iters, int clusters,
+                                   void* cuda_stream, double* cycles_per_mma);
+
 /* handle may be a graph, binding or plan; returns "" if there was no error. */
 const char* sod2_last_error(const void* any_handle);
 

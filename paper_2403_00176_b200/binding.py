@@ -84,6 +84,7 @@ def _load() -> C.CDLL:
         "sod2_nonzero_static": [vp, i32, i32, P(i64), vp, vp, vp],
         "sod2_launch_empty": [vp],
         "sod2_selftest_bounded_wait": [vp, vp],
+        "sod2_selftest_mma_rate": [i32, i32, i32, i32, i32, i32, vp, P(C.c_double)],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -107,7 +108,7 @@ EXPORTS = ["sod2_graph_create", "sod2_graph_destroy", "sod2_graph_set_const", "s
            "sod2_graph_num_ops", "sod2_graph_op_info", "sod2_graph_num_groups", "sod2_graph_group_info",
            "sod2_graph_num_subgraphs", "sod2_graph_rdp_sweeps", "sod2_classify", "sod2_graph_reanalyse", "sod2_graph_order_info",
            "sod2_binding_shape", "sod2_plan_slot", "sod2_plan_instance_offset", "sod2_plan_memory", "sod2_plan_group_cost", "sod2_plan_group_on_side_stream", "sod2_plan_tensor_strides",
-           "sod2_run_output_shape", "sod2_nonzero_static", "sod2_launch_empty", "sod2_selftest_bounded_wait", "sod2_last_error"]
+           "sod2_run_output_shape", "sod2_nonzero_static", "sod2_launch_empty", "sod2_selftest_bounded_wait", "sod2_selftest_mma_rate", "sod2_last_error"]
 
 
 def _check(status: int, handle=None):
@@ -133,6 +134,14 @@ def sod2_launch_empty(stream: int) -> None:
 def sod2_selftest_bounded_wait(dev_status_word: int, stream: int) -> None:
     """Launches the kernel whose bounded wait runs out: it sets the device status word and returns by itself."""
     _check(lib.sod2_selftest_bounded_wait(C.c_void_p(dev_status_word), C.c_void_p(stream)))
+
+
+def sod2_selftest_mma_rate(pair: bool, n_cols: int, per_stage: int, handshake: int, stream: int, iters: int = 4096, clusters: int = 74) -> float:
+    """SM cycles per tcgen05.mma (128 x n_cols x 16 on one CTA, 256 x n_cols x 16 on a CTA pair) issued in stages of
+    `per_stage`; handshake 0 = MMAs only, 1 = commit per stage, 2 = full / empty barrier handshake per stage."""
+    out = C.c_double()
+    _check(lib.sod2_selftest_mma_rate(int(bool(pair)), n_cols, per_stage, handshake, iters, clusters, C.c_void_p(stream), C.byref(out)))
+    return out.value
 
 
 def sod2_nonzero_static(dev_x: int, dtype: int, dims: Sequence[int], dev_out: int, dev_count: int, stream: int) -> None:

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsod2.so")
-SOURCES = ["expr.cpp", "rdp.cpp", "fuse.cpp", "sep.cpp", "plan.cpp", "capi.cpp", "exec.cu", "noalloc.cu"]
+SOURCES = ["expr.cpp", "rdp.cpp", "fuse.cpp", "sep.cpp", "plan.cpp", "capi.cpp", "exec.cu", "noalloc.cu", "selftest_mma.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-Wall,-Wno-unused-function", "--expt-relaxed-constexpr"]
 

@@ -267,8 +267,42 @@ def chain_case(spec: str, reps: int = 20, device: str = "cuda:0"):
             "ms_back_to_back": b2b, "gbs_back_to_back": nbytes / b2b / 1e6, "frac_of_hbm_back_to_back": nbytes / b2b / 1e6 / hbm, "peaks": src}
 
 
+def gemm_sweep(spec: str, device: str = "cuda:0"):
+    """Kernel time of one bias GEMM against K: spec = "M,N,K1:K2:...".  For the single-CTA kernel and for the CTA-pair
+    kernel (SOD2_OPT_GEMM_PAIR, forced wherever it is eligible): device time of one launch with 20 launches back to back
+    between the events.  The slope over K is the main loop's time per 64-wide k-stage; what is left at K -> 0 is the
+    fixed part of the kernel (fill, epilogue, launch)."""
+    import torch
+    from paper_2403_00176_b200 import binding as B
+    from paper_2403_00176_b200 import workloads as WL
+    from paper_2403_00176_b200.session import Session
+    from paper_2403_00176_b200.workloads import Request, bf16_round
+    os.environ["SOD2_GEMM_PAIR_FORCE"] = "1"      # read once by the library, only under the flag
+    m, n, ks = spec.split(",")
+    m, n, ks = int(m), int(n), [int(x) for x in ks.split(":")]
+    rng = np.random.default_rng(0)
+    rows = []
+    for name, flags in (("one CTA per tile", 0), ("CTA pair per tile", B.OPT_GEMM_PAIR)):
+        us = []
+        for k in ks:
+            ir = (f"sym M 1 16384\ninput x bf16 [1,M,{k}]\nconst w bf16 [{k},{n}]\nconst b bf16 [{n}]\n"
+                  "node MatMul x w -> y0\nnode Add y0 b -> y\noutput y\n")
+            consts = {"w": bf16_round((rng.standard_normal((k, n)) * 0.02).astype(np.float32)), "b": bf16_round((rng.standard_normal(n) * 0.02).astype(np.float32))}
+            req = Request({"M": m}, {"x": bf16_round(rng.standard_normal((1, m, k)).astype(np.float32))})
+            wl = WL.Workload(f"gemm_{m}x{n}x{k}", "bf16", ir, consts, ["M"], ["y"], {"batch_fn": lambda j: [req]})
+            sess = Session(wl, device=device, opt_flags=flags)
+            p = sess.prepare([req])
+            p.run()
+            torch.cuda.synchronize(sess.dev)
+            us.append(group_times(p, reps=7, repeat=20)[0] * 1e3)
+        slope = (us[-1] - us[-2]) / ((ks[-1] - ks[-2]) / 64) if len(ks) > 1 else None
+        rows.append({"kernel": name, "M": m, "N": n, "K": ks, "us": us, "us_per_k_stage_at_the_large_end": slope})
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--gemm-sweep", default=None, help="M,N,K1:K2:...: kernel time of one bias GEMM against K, single-CTA and CTA-pair kernel")
     ap.add_argument("--chain-case", default=None, help="I,J,K,dtype,n_requests: time the Fig. 4 fused chain at this size instead of the configs")
     ap.add_argument("--configs", default="1,2,3,4,5")
     ap.add_argument("--reps", type=int, default=30)
@@ -276,6 +310,10 @@ def main():
     a = ap.parse_args()
     if a.chain_case:
         print(json.dumps(chain_case(a.chain_case)))
+        return
+    if a.gemm_sweep:
+        for r in gemm_sweep(a.gemm_sweep):
+            print(json.dumps(r))
         return
     rows = []
     for c in [int(x) for x in a.configs.split(",")]:

@@ -229,6 +229,33 @@ def test_resize_upsample_nearest_executor():
         assert O.rel_err(u, env["u"]) <= BF16_TOL and O.rel_err(outs2[0]["z"], env["z"]) <= BF16_TOL
 
 
+def test_mma_issue_rate_one_cta_and_cta_pair():
+    # The machine facts the GEMM versions are built on, pinned: a tcgen05.mma of 128 x 256 x 16 occupies the pipe for
+    # 128 cycles and the 256 x 256 x 16 form of a CTA pair for the same 128 (both SMs at full rate); narrower
+    # instructions do not get cheaper than ~74 cycles; the issuing thread's own work between stages (wait, fence,
+    # commit) is not overlapped by the pipe, for either form.  Printed with -s.
+    st = torch.cuda.current_stream().cuda_stream
+    rows = []
+    for pair in (False, True):
+        for n, per_stage in ((256, 4), (128, 8), (64, 8)):
+            r = [B.sod2_selftest_mma_rate(pair, n, per_stage, hs, st) for hs in (0, 1, 2)]
+            rows.append((pair, n, per_stage, r))
+            print(f"{'pair 256' if pair else 'one CTA 128'}x{n}x16, {per_stage} per stage: MMAs only {r[0]:.1f}, + commit {r[1]:.1f}, "
+                  f"+ full/empty handshake {r[2]:.1f} cycles per MMA")
+    rate = {(pair, n): r for pair, n, _, r in rows}
+    for pair in (False, True):
+        assert 126.0 <= rate[(pair, 256)][0] <= 132.0          # 8192 flop / clk / SM
+        assert 126.0 <= rate[(pair, 256)][1] <= 134.0          # a commit per stage is free
+        assert 70.0 <= rate[(pair, 128)][0] <= 80.0 and 70.0 <= rate[(pair, 64)][0] <= 80.0
+        assert rate[(pair, 256)][2] >= rate[(pair, 256)][0] + 15.0    # the handshake is exposed
+    # the pair is neither slower nor faster per instruction than one CTA
+    for n in (256, 128, 64):
+        for hs in range(3):
+            assert abs(rate[(True, n)][hs] - rate[(False, n)][hs]) <= 0.05 * rate[(False, n)][hs] + 2.0
+    with pytest.raises(B.Sod2Error):
+        B.sod2_selftest_mma_rate(False, 96, 4, 0, st)
+
+
 def test_topk_keep_with_nan_rows_keeps_exactly_k():
     # a row of NaN (an overflow upstream) has a NaN score, which compares false with everything: it must rank last, not
     # be kept by every chunk, so that exactly k rows are kept (in ascending order) and nothing is written past them
