@@ -186,6 +186,9 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     for (int b = 0; b < NSB; ++b) { ptx::mbar_init(&buf_ready[b], 1); ptx::mbar_init(&buf_filled[b], SPLITK ? 4 : 8); }
     *dead = 0;
     ptx::fence_barrier_init();
+    // without a residual the staging buffers start out free: their first phase is completed here, before the
+    // block-wide barrier below, so the epilogue need not wait for its first NSB units at all
+    if (!SPLITK && !RES) { for (int b = 0; b < NSB; ++b) ptx::mbar_arrive(&buf_ready[b]); }
     ptx::fence_proxy_async();
     ptx::prefetch_tmap(&tmA);
     ptx::prefetch_tmap(&tmB);
@@ -298,7 +301,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           ptx::mbar_arrive(&buf_ready[bsel]);
         }
       };
-      for (int u = 0; u < NSB && u < U; ++u) prepare(u);
+      if (SPLITK || RES) { for (int u = 0; u < NSB && u < U; ++u) prepare(u); }   // else: done at barrier initialisation
       for (int u = 0; u < U; ++u) {
         const int bsel = u % NSB;
         ptx::mbar_wait(&buf_filled[bsel], (u / NSB) & 1, dead);
@@ -445,8 +448,16 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] = apply_act<ACT>(fmaf(ln_rstd, __uint_as_float(r[ps & 1][i]), fmaf(nmr, bp[BN + i], bp[i])));
         } else {
+          // the 32 bias values as eight 16-byte broadcast loads (the offset is a multiple of 128 bytes)
+          const float4* bp4 = reinterpret_cast<const float4*>(bp);
 #pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = apply_act<ACT>(__uint_as_float(r[ps & 1][i]) + bp[i]);
+          for (int i4 = 0; i4 < 8; ++i4) {
+            const float4 b4 = bp4[i4];
+            v[4 * i4] = apply_act<ACT>(__uint_as_float(r[ps & 1][4 * i4]) + b4.x);
+            v[4 * i4 + 1] = apply_act<ACT>(__uint_as_float(r[ps & 1][4 * i4 + 1]) + b4.y);
+            v[4 * i4 + 2] = apply_act<ACT>(__uint_as_float(r[ps & 1][4 * i4 + 2]) + b4.z);
+            v[4 * i4 + 3] = apply_act<ACT>(__uint_as_float(r[ps & 1][4 * i4 + 3]) + b4.w);
+          }
         }
         uint4 pk[4];
         if constexpr (!RES) {
@@ -457,7 +468,9 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             for (int i = 0; i < 4; ++i) oh[i] = __floats2bfloat162_rn(v[g * 8 + 2 * i], v[g * 8 + 2 * i + 1]);
           }
         }
-        ptx::mbar_wait_warp(&buf_ready[bsel], (u / NSB) & 1, dead);
+        // without a residual the first NSB units find their buffers free (first phase completed at barrier
+        // initialisation): even a satisfied wait costs a barrier round trip on the epilogue's critical path
+        if (RES || u >= NSB) ptx::mbar_wait_warp(&buf_ready[bsel], (u / NSB) & 1, dead);
         if constexpr (RES) {
           // the four residual loads first, then the arithmetic, then the four stores: loads and stores go
           // to the same buffer, so interleaved the compiler keeps each load behind the previous store
