@@ -6,16 +6,19 @@
 //   P_j = exp2(S_j*c - m)  softmax threads: two threads per query row, each owns 64 of the block's 128
 //                          score columns and reads them from TMEM in two 32-column halves, twice: once for
 //                          the row maximum, once for the exponentials (a TMEM read is cheaper than holding
-//                          64 scores in registers at two CTAs per SM); P_j goes as bf16 into two swizzled
-//                          [128 x 64] tiles
-//   O  += P_j V_j          tcgen05.mma, M=128, N=64, K=128; V_j is the natural [key, d] tile, used
-//                          as an MN-major B operand
+//                          64 scores in registers at two CTAs per SM); P_j goes as packed bf16 pairs into 64
+//                          columns of TMEM (tcgen05.st: each thread its own row)
+//   O  += P_j V_j          tcgen05.mma with the A operand in TMEM, M=128, N=64, K=128; V_j is the natural
+//                          [key, d] tile, used as an MN-major B operand
 //   (O *= corr)            only when a block's maximum moves the exponent reference by more than 2^8
 // A block of 128 keys halves the number of hand-overs per key (barrier round trips, the row-maximum
-// exchange, the P hand-over cost about as much as the exponentials of 64 keys).  S (128 columns) and O
-// (64 columns) live in TMEM; S is single buffered: the softmax threads release it after their last read,
+// exchange, the P hand-over cost about as much as the exponentials of 64 keys).  S (128 columns), O (64) and P (64)
+// live in TMEM -- handing P over through shared memory (32 KB of stores per block, a proxy fence) took 680-750 cycles
+// of a 3300-cycle block, through TMEM 180 --; S is single buffered: the softmax threads release it after their last read,
 // about half way through the block, and the next S = Q K^T runs under the second half of the
-// exponentials.  K and P are single buffered, V double buffered; two CTAs share an SM.
+// exponentials (tried: half of them as a cubic on the FMA pipe -- slower, the block is bound by issue slots and
+// latencies at 80 registers, not by the special-function pipe).  K and P are single buffered, V double buffered; two
+// CTAs share an SM.
 // Q, K, V are 2-D tensor maps over the packed [tokens, row stride] buffers; a tile that runs past a
 // request's rows reads the next request's rows (finite data) or zeros past the end of the buffer, and
 // those keys are masked to -inf before the softmax; query rows past the request are never written.
@@ -53,8 +56,9 @@ struct AtcParams {
 constexpr int ATC_KB = 128;               // keys per block
 constexpr int ATC_Q_BYTES = 128 * 128;    // 128 rows x 64 bf16
 constexpr int ATC_KV_BYTES = ATC_KB * 128;   // 128 keys x 64 bf16
-constexpr int ATC_P_BYTES = 2 * 128 * 128;   // 128 rows x 128 keys bf16: two [128 x 64] chunks
-constexpr int ATC_SMEM = ATC_Q_BYTES + 3 * ATC_KV_BYTES + ATC_P_BYTES + 2048 /*row maxima*/ + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int ATC_O_BYTES = 128 * 128;       // output staging: 128 rows x 64 bf16
+constexpr int ATC_SMEM = ATC_Q_BYTES + 3 * ATC_KV_BYTES + ATC_O_BYTES + 2048 /*row maxima*/ + 1024 /*align*/ + 256 /*barriers*/;
+constexpr uint32_t ATC_TMEM_S = 0, ATC_TMEM_O = 128, ATC_TMEM_P = 192;   // columns: scores, output, probabilities (packed bf16 pairs)
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
@@ -70,8 +74,8 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   uint8_t* sQ = base;
   uint8_t* sK = sQ + ATC_Q_BYTES;
   uint8_t* sV = sK + ATC_KV_BYTES;          // [2]
-  uint8_t* sP = sV + 2 * ATC_KV_BYTES;
-  float* xmax = reinterpret_cast<float*>(sP + ATC_P_BYTES);   // [block parity][column half][row]
+  uint8_t* sO = sV + 2 * ATC_KV_BYTES;
+  float* xmax = reinterpret_cast<float*>(sO + ATC_O_BYTES);   // [block parity][column half][row]
   uint64_t* bars = reinterpret_cast<uint64_t*>(xmax + 512);
   uint64_t* q_full = bars;            // 1
   uint64_t* k_full = bars + 1;        // K_j landed (one phase per block)
@@ -152,7 +156,6 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       // the V stage and the P buffer.  The softmax warps rescale O (rarely) before they hand over P_j,
       // so the accumulator needs no barrier of its own.
       constexpr uint32_t idesc_pv = ptx::idesc_bf16(128, 64) | (1u << 16);   // B (= V tile) is MN-major
-      const uint32_t aP = ptx::smem_u32(sP);
       for (int i = 0; i < nkv; ++i) {
         const int b = i & 1;
         ptx::mbar_wait(&v_full[b], (i >> 1) & 1, dead);
@@ -160,8 +163,8 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         ptx::tc_fence_after();
         const uint32_t aV = ptx::smem_u32(sV + b * ATC_KV_BYTES);
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk)   // 16 keys per step: 32 B along P's rows (chunk kk / 4), 16 rows (2048 B) down V
-          ptx::mma_bf16(tmem + 128, ptx::smem_desc_sw128(aP + (kk >> 2) * (128 * 128)) + 2 * (kk & 3), ptx::smem_desc_sw128(aV + kk * 2048), idesc_pv, (i | kk) != 0);
+        for (int kk = 0; kk < 8; ++kk)   // 16 keys per step: 8 packed columns of P in tensor memory, 16 rows (2048 B) down V
+          ptx::mma_bf16_a_tmem(tmem + ATC_TMEM_O, tmem + ATC_TMEM_P + kk * 8, ptx::smem_desc_sw128(aV + kk * 2048), idesc_pv, (i | kk) != 0);
         ptx::mma_commit(&o_full[b]);
         SOD2_TRACE(1, 20 + i)
       }
@@ -184,8 +187,9 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     // back from TMEM.  l and O always refer to the same m, so O / l at the end is the softmax average.
     float m = -INFINITY, l = 0.f;
     const float c = p.scale_log2e;
-    const uint32_t o_addr = tmem + lane_base + 128 + hh * 32;
-    const uint32_t s_addr = tmem + lane_base + hh * 64;      // this thread's 64 score columns of the block
+    const uint32_t o_addr = tmem + lane_base + ATC_TMEM_O + hh * 32;
+    const uint32_t s_addr = tmem + lane_base + ATC_TMEM_S + hh * 64;      // this thread's 64 score columns of the block
+    const uint32_t p_addr = tmem + lane_base + ATC_TMEM_P + hh * 32;      // ... and its 32 packed probability columns
     for (int j = 0; j < nkv; ++j) {
       const int b = j & 1;
       ptx::mbar_wait_warp(s_full, j & 1, dead);
@@ -275,24 +279,21 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       }
       l += sum0 + sum1;
       if (tracer) { SOD2_TRACE(2, 40 + j) }
-      // P_j into the two swizzled chunks once the MMA that read the buffer for the last block has finished
-      if (j >= 1) ptx::mbar_wait_warp(&o_full[(j - 1) & 1], ((j - 1) >> 1) & 1, dead);    // O_{j-1} done: the P buffer is free
-      {
-        uint8_t* prow = sP + hh * (128 * 128) + row * 128;     // chunk hh holds this thread's 64 keys
-#pragma unroll
-        for (int g = 0; g < 8; ++g)
-          *reinterpret_cast<uint4*>(prow + ((g ^ (row & 7)) << 4)) =
-              make_uint4(pk[g >> 2][4 * (g & 3)], pk[g >> 2][4 * (g & 3) + 1], pk[g >> 2][4 * (g & 3) + 2], pk[g >> 2][4 * (g & 3) + 3]);
-      }
-      ptx::fence_proxy_async();
+      // P_j into tensor memory (32 columns of packed bf16 pairs per thread: its 64 keys) once the MMA that read the
+      // P columns for the last block has finished; the product reads it from there as its A operand
+      if (j >= 1) ptx::mbar_wait_warp(&o_full[(j - 1) & 1], ((j - 1) >> 1) & 1, dead);    // O_{j-1} done: the P columns are free
+      ptx::tc_fence_after();
+      ptx::tmem_st32(p_addr, &pk[0][0]);
+      ptx::tmem_st_wait();
+      ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(p_full);
       if (tracer) { SOD2_TRACE(2, 50 + j) }
     }
     // ---- output: O / l.  The row sums of the two halves are added through shared memory, the scaled rows
-    // are staged (swizzled) in P buffer 0 and written four full 128-byte rows per instruction.
+    // are staged (swizzled) in shared memory and written four full 128-byte rows per instruction.
     {
-      ptx::mbar_wait_warp(&o_full[(nkv - 1) & 1], ((nkv - 1) >> 1) & 1, dead);   // every product has landed; the P buffers are free
+      ptx::mbar_wait_warp(&o_full[(nkv - 1) & 1], ((nkv - 1) >> 1) & 1, dead);   // every product has landed
       ptx::tc_fence_after();
       uint32_t r[32];
       ptx::tmem_ld32(o_addr, r);
@@ -303,7 +304,7 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       asm volatile("bar.sync 1, 256;" ::: "memory");
       const float lt = l + xmax[(hh ^ 1) * 128 + row];
       const float inv = warp_live ? 1.0f / lt : 0.f;
-      uint8_t* prow = sP + row * 128;
+      uint8_t* prow = sO + row * 128;
 #pragma unroll
       for (int g = 0; g < 4; ++g) {
         uint4 v;
@@ -317,7 +318,7 @@ attention_tcgen05_bf16(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int rr = q * 32 + hh * 16 + i * 4 + (lane >> 3), ch = lane & 7;
-        const uint4 v = *reinterpret_cast<const uint4*>(sP + rr * 128 + ((ch ^ (rr & 7)) << 4));
+        const uint4 v = *reinterpret_cast<const uint4*>(sO + rr * 128 + ((ch ^ (rr & 7)) << 4));
         if (q0 + rr < L) *reinterpret_cast<uint4*>(og + static_cast<long long>(q0 + rr) * p.o_ts + ch * 8) = v;
       }
     }
